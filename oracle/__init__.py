@@ -1,0 +1,185 @@
+"""ctypes front end of the TileLens ORACLE (test infrastructure only).
+
+The arithmetic lives in ``tlo.c``; this file only compiles it with gcc, loads
+it and marshals numpy arrays.  Nothing here imports, or is imported by, the
+CUDA package.  Callers: the tests, the smoke check and the CPU-baseline leg of
+the benchmark.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tlo.c")
+_HDR = os.path.join(_HERE, "tlo.h")
+_LIB = os.path.join(_HERE, "libtlo.so")
+
+ROW_MAJOR, COL_MAJOR, TILE_MAJOR = 0, 1, 2
+TO_TILE_MAJOR, TO_ROW_MAJOR = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile tlo.c into libtlo.so (plain -O2, OpenMP, no SIMD flags)."""
+    stale = (not os.path.exists(_LIB)
+             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)))
+    if force or stale:
+        tmp = f"{_LIB}.{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC",
+                               "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i64, u64p, vp = ctypes.c_int64, ctypes.POINTER(ctypes.c_uint64), ctypes.c_void_p
+        for name in ("tlo_off_row", "tlo_off_col"):
+            getattr(L, name).restype = i64
+            getattr(L, name).argtypes = [i64] * 5
+        L.tlo_off_tile.restype = i64
+        L.tlo_off_tile.argtypes = [i64] * 7
+        L.tlo_off.restype = i64
+        L.tlo_off.argtypes = [ctypes.c_int] + [i64] * 7
+        L.tlo_eq1.restype = None
+        L.tlo_eq1.argtypes = [i64] * 4 + [ctypes.POINTER(i64)]
+        for name in ("tlo_eq2", "tlo_eq3"):
+            getattr(L, name).restype = i64
+            getattr(L, name).argtypes = [i64] * 7
+        L.tlo_relayout.restype = ctypes.c_int
+        L.tlo_relayout.argtypes = [vp, vp, i64, i64, i64, i64, i64, ctypes.c_int]
+        L.tlo_bf16_to_double.restype = ctypes.c_double
+        L.tlo_bf16_to_double.argtypes = [ctypes.c_uint16]
+        L.tlo_matmul_at.restype = ctypes.c_int
+        L.tlo_matmul_at.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, i64, i64, vp, vp, vp, vp]
+        L.tlo_matmul.restype = ctypes.c_int
+        L.tlo_matmul.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, i64, vp, vp]
+        L.tlo_read_amp.restype = ctypes.c_int
+        L.tlo_read_amp.argtypes = [i64] * 6 + [ctypes.c_int] + [i64] * 4 + [u64p, u64p, u64p, vp, vp]
+        L.tlo_read_amp_grouped.restype = ctypes.c_int
+        L.tlo_read_amp_grouped.argtypes = ([vp, ctypes.c_int] + [i64] * 5 + [ctypes.c_int] + [i64] * 4
+                                           + [u64p, u64p, u64p])
+        L.tlo_num_threads.restype = ctypes.c_int
+        L.tlo_num_threads.argtypes = []
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().tlo_num_threads())
+
+
+def _ptr(a: np.ndarray) -> ctypes.c_void_p:
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def off_row(r, c, rows, cols, s):
+    return int(lib().tlo_off_row(r, c, rows, cols, s))
+
+
+def off_col(r, c, rows, cols, s):
+    return int(lib().tlo_off_col(r, c, rows, cols, s))
+
+
+def off_tile(r, c, rows, cols, br, bc, s):
+    return int(lib().tlo_off_tile(r, c, rows, cols, br, bc, s))
+
+
+def off(layout, r, c, rows, cols, br, bc, s):
+    return int(lib().tlo_off(layout, r, c, rows, cols, br, bc, s))
+
+
+def eq1(i, j, a, b):
+    out = (ctypes.c_int64 * 4)()
+    lib().tlo_eq1(i, j, a, b, out)
+    return tuple(int(x) for x in out)
+
+
+def eq2(i, j, K, N, a, b, s):
+    return int(lib().tlo_eq2(i, j, K, N, a, b, s))
+
+
+def eq3(i, j, K, N, a, b, s):
+    return int(lib().tlo_eq3(i, j, K, N, a, b, s))
+
+
+def relayout(src: np.ndarray, rows: int, cols: int, s: int, br: int, bc: int, direction: int) -> np.ndarray:
+    """src: contiguous uint8 array of rows*cols*s bytes.  Returns the permuted bytes."""
+    src = np.ascontiguousarray(src).view(np.uint8).reshape(-1)
+    assert src.size == rows * cols * s
+    dst = np.empty_like(src)
+    rc = lib().tlo_relayout(_ptr(src), _ptr(dst), rows, cols, s, br, bc, direction)
+    if rc != 0:
+        raise ValueError(f"tlo_relayout rejected its arguments (rc={rc})")
+    return dst
+
+
+def bf16_to_double(h: int) -> float:
+    return float(lib().tlo_bf16_to_double(h))
+
+
+def matmul(A_bits: np.ndarray, B_bits: np.ndarray, layout: int, br: int, bc: int, M: int, N: int, K: int):
+    """A_bits: uint16 [M,K] row-major; B_bits: uint16 buffer of K*N in `layout`.  Returns (C, S) fp64 [M,N]."""
+    A_bits = np.ascontiguousarray(A_bits, dtype=np.uint16)
+    B_bits = np.ascontiguousarray(B_bits, dtype=np.uint16)
+    assert A_bits.size == M * K and B_bits.size == K * N
+    C = np.empty((M, N), dtype=np.float64)
+    S = np.empty((M, N), dtype=np.float64)
+    rc = lib().tlo_matmul(_ptr(A_bits), _ptr(B_bits), layout, br, bc, M, N, K, _ptr(C), _ptr(S))
+    if rc != 0:
+        raise ValueError(f"tlo_matmul rejected its arguments (rc={rc})")
+    return C, S
+
+
+def matmul_at(A_bits, B_bits, layout, br, bc, M, N, K, idx_i, idx_j):
+    """The product at the listed (i, j) only.  Returns (C, S) fp64 vectors."""
+    A_bits = np.ascontiguousarray(A_bits, dtype=np.uint16)
+    B_bits = np.ascontiguousarray(B_bits, dtype=np.uint16)
+    assert A_bits.size == M * K and B_bits.size == K * N
+    ii = np.ascontiguousarray(idx_i, dtype=np.int64)
+    jj = np.ascontiguousarray(idx_j, dtype=np.int64)
+    assert ii.shape == jj.shape and ii.ndim == 1
+    C = np.empty(ii.size, dtype=np.float64)
+    S = np.empty(ii.size, dtype=np.float64)
+    rc = lib().tlo_matmul_at(_ptr(A_bits), _ptr(B_bits), layout, br, bc, M, N, K, ii.size,
+                             _ptr(ii), _ptr(jj), _ptr(C), _ptr(S))
+    if rc != 0:
+        raise ValueError(f"tlo_matmul_at rejected its arguments (rc={rc})")
+    return C, S
+
+
+def read_amp(M, N, K, BM, BN, BK, layout, G, br, bc, s, per_tile=False):
+    """Returns (fetched, used, requests) or, with per_tile, also the two per-CTA-tile arrays."""
+    f, u, q = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    pf = pu = None
+    a = b = ctypes.c_void_p(None)
+    if per_tile:
+        mt, nt = -(-M // BM), -(-N // BN)
+        pf = np.zeros(mt * nt, dtype=np.uint64)
+        pu = np.zeros(mt * nt, dtype=np.uint64)
+        a, b = _ptr(pf), _ptr(pu)
+    rc = lib().tlo_read_amp(M, N, K, BM, BN, BK, layout, G, br, bc, s,
+                            ctypes.byref(f), ctypes.byref(u), ctypes.byref(q), a, b)
+    if rc != 0:
+        raise ValueError(f"tlo_read_amp rejected its arguments (rc={rc})")
+    if per_tile:
+        return int(f.value), int(u.value), int(q.value), pf, pu
+    return int(f.value), int(u.value), int(q.value)
+
+
+def read_amp_grouped(offsets, N, K, BM, BN, BK, layout, G, br, bc, s):
+    offs = np.ascontiguousarray(offsets, dtype=np.int32)
+    f, u, q = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    rc = lib().tlo_read_amp_grouped(_ptr(offs), offs.size - 1, N, K, BM, BN, BK, layout, G, br, bc, s,
+                                    ctypes.byref(f), ctypes.byref(u), ctypes.byref(q))
+    if rc != 0:
+        raise ValueError(f"tlo_read_amp_grouped rejected its arguments (rc={rc})")
+    return int(f.value), int(u.value), int(q.value)

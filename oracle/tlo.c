@@ -1,0 +1,284 @@
+/*
+ * tlo -- TileLens ORACLE (test infrastructure only; see tlo.h).
+ * Plain C, fp64 arithmetic, integer division and modulo written out,
+ * OpenMP "parallel for" over independent outputs and nothing else.
+ */
+#include "tlo.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int tlo_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---------------------------------------------------------------- layouts */
+
+/* Section 2.4: a row is contiguous. */
+int64_t tlo_off_row(int64_t r, int64_t c, int64_t rows, int64_t cols, int64_t s) {
+    (void)rows;
+    return (r * cols + c) * s;
+}
+
+/* Section 2.4 / Section 3.2: a column is contiguous, offset (j*K + i)*s. */
+int64_t tlo_off_col(int64_t r, int64_t c, int64_t rows, int64_t cols, int64_t s) {
+    (void)cols;
+    return (c * rows + r) * s;
+}
+
+/* Eq. 1 + Eq. 2 in the row flavour: the contiguous direction is the column
+ * index c, so (i, a, K) of the printed form become (c, bc, cols) and
+ * (j, b, N) become (r, br, rows). */
+int64_t tlo_off_tile(int64_t r, int64_t c, int64_t rows, int64_t cols,
+                     int64_t br, int64_t bc, int64_t s) {
+    (void)rows;
+    int64_t Tr = r / br, rp = r % br;          /* Eq. 1 */
+    int64_t Tc = c / bc, cp = c % bc;
+    int64_t tiles_per_tile_row = cols / bc;
+    int64_t linear_tile = Tr * tiles_per_tile_row + Tc;   /* tiles ordered along the contiguous direction first */
+    int64_t intra = rp * bc + cp;                          /* same order inside the tile */
+    return linear_tile * (br * bc * s) + intra * s;        /* Eq. 2 */
+}
+
+int64_t tlo_off(int layout, int64_t r, int64_t c, int64_t rows, int64_t cols,
+                int64_t br, int64_t bc, int64_t s) {
+    if (layout == TLO_ROW_MAJOR) return tlo_off_row(r, c, rows, cols, s);
+    if (layout == TLO_COL_MAJOR) return tlo_off_col(r, c, rows, cols, s);
+    return tlo_off_tile(r, c, rows, cols, br, bc, s);
+}
+
+/* Eq. 1 exactly as printed. */
+void tlo_eq1(int64_t i, int64_t j, int64_t a, int64_t b, int64_t out[4]) {
+    out[0] = i % a;   /* i'  */
+    out[1] = j % b;   /* j'  */
+    out[2] = i / a;   /* T_i */
+    out[3] = j / b;   /* T_j */
+}
+
+/* Eq. 2 exactly as printed: K x N matrix, K contiguous, memory tile a x b. */
+int64_t tlo_eq2(int64_t i, int64_t j, int64_t K, int64_t N, int64_t a, int64_t b, int64_t s) {
+    (void)N;
+    int64_t q[4];
+    tlo_eq1(i, j, a, b, q);
+    int64_t ip = q[0], jp = q[1], Ti = q[2], Tj = q[3];
+    return (Tj * (K / a) + Ti) * (a * b * s) + (jp * a + ip) * s;
+}
+
+/* Eq. 3: shape (a, b, K/a, N/b), stride (1, a, ab, Kb) in elements. */
+int64_t tlo_eq3(int64_t i, int64_t j, int64_t K, int64_t N, int64_t a, int64_t b, int64_t s) {
+    (void)N;
+    int64_t q[4];
+    tlo_eq1(i, j, a, b, q);
+    int64_t stride[4] = {1, a, a * b, K * b};
+    int64_t e = 0;
+    for (int d = 0; d < 4; ++d) e += q[d] * stride[d];
+    return e * s;
+}
+
+/* --------------------------------------------------------------- relayout */
+
+int tlo_relayout(const void* src, void* dst, int64_t rows, int64_t cols, int64_t s,
+                 int64_t br, int64_t bc, int direction) {
+    if (rows < 0 || cols < 0 || s <= 0 || br <= 0 || bc <= 0) return -1;
+    if (rows % br != 0 || cols % bc != 0) return -1;       /* Section 3.3 */
+    const unsigned char* in = (const unsigned char*)src;
+    unsigned char* out = (unsigned char*)dst;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t c = 0; c < cols; ++c) {
+            int64_t o_row = tlo_off_row(r, c, rows, cols, s);
+            int64_t o_tile = tlo_off_tile(r, c, rows, cols, br, bc, s);
+            if (direction == TLO_TO_TILE_MAJOR)
+                memcpy(out + o_tile, in + o_row, (size_t)s);
+            else
+                memcpy(out + o_row, in + o_tile, (size_t)s);
+        }
+    }
+    return 0;
+}
+
+/* ----------------------------------------------------------------- matmul */
+
+double tlo_bf16_to_double(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Section 2.3: one output element, the sum over k written out. */
+static void dot_at(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
+                   int64_t N, int64_t K, int64_t i, int64_t j, double* c_out, double* s_out) {
+    double acc = 0.0, abs_acc = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+        double a = tlo_bf16_to_double(A[i * K + k]);
+        int64_t off = tlo_off(layout, k, j, K, N, br, bc, 2);
+        double b = tlo_bf16_to_double(B[off / 2]);
+        double p = a * b;
+        acc += p;
+        abs_acc += fabs(p);
+    }
+    *c_out = acc;
+    *s_out = abs_acc;
+}
+
+int tlo_matmul_at(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
+                  int64_t M, int64_t N, int64_t K, int64_t n,
+                  const int64_t* idx_i, const int64_t* idx_j, double* C, double* S) {
+    if (layout == TLO_TILE_MAJOR && (br <= 0 || bc <= 0 || K % br != 0 || N % bc != 0)) return -1;
+    for (int64_t t = 0; t < n; ++t)
+        if (idx_i[t] < 0 || idx_i[t] >= M || idx_j[t] < 0 || idx_j[t] >= N) return -1;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t t = 0; t < n; ++t)
+        dot_at(A, B, layout, br, bc, N, K, idx_i[t], idx_j[t], &C[t], &S[t]);
+    return 0;
+}
+
+int tlo_matmul(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
+               int64_t M, int64_t N, int64_t K, double* C, double* S) {
+    if (layout == TLO_TILE_MAJOR && (br <= 0 || bc <= 0 || K % br != 0 || N % bc != 0)) return -1;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t t = 0; t < M * N; ++t)
+        dot_at(A, B, layout, br, bc, N, K, t / N, t % N, &C[t], &S[t]);
+    return 0;
+}
+
+/* ----------------------------------------------------- read amplification */
+
+/* One weight-tile load: rows k in [k0,k1), columns n in [n0,n1) of the K x N
+ * operand.  Visits every element, marks the block of its first and of its
+ * last byte, counts marks that were new, then clears them again. */
+static uint64_t blocks_touched(unsigned char* mark, int layout, int64_t K, int64_t N,
+                               int64_t br, int64_t bc, int64_t s, int64_t G,
+                               int64_t k0, int64_t k1, int64_t n0, int64_t n1) {
+    uint64_t count = 0;
+    for (int64_t k = k0; k < k1; ++k)
+        for (int64_t n = n0; n < n1; ++n) {
+            int64_t off = tlo_off(layout, k, n, K, N, br, bc, s);
+            int64_t first = off / G, last = (off + s - 1) / G;
+            if (!mark[first]) { mark[first] = 1; ++count; }
+            if (!mark[last])  { mark[last] = 1;  ++count; }
+        }
+    for (int64_t k = k0; k < k1; ++k)
+        for (int64_t n = n0; n < n1; ++n) {
+            int64_t off = tlo_off(layout, k, n, K, N, br, bc, s);
+            mark[off / G] = 0;
+            mark[(off + s - 1) / G] = 0;
+        }
+    return count;
+}
+
+static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+/* All weight-tile loads issued by ONE row of CTA tiles (one m-tile): every
+ * n-tile, every K iteration.  per_ntile_* (length n-tiles) may be NULL. */
+static int weight_loads_one_mtile(int64_t N, int64_t K, int64_t BN, int64_t BK,
+                                  int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                                  uint64_t* fetched, uint64_t* used, uint64_t* requests,
+                                  uint64_t* per_ntile_fetched, uint64_t* per_ntile_used) {
+    int64_t nt = ceil_div(N, BN), kt = ceil_div(K, BK);
+    int64_t total_blocks = ceil_div(K * N * s, G) + 1;
+    uint64_t f_sum = 0, u_sum = 0, q_sum = 0;
+    int failed = 0;
+#pragma omp parallel reduction(+ : f_sum, u_sum, q_sum)
+    {
+        unsigned char* mark = (unsigned char*)calloc((size_t)total_blocks, 1);
+        if (!mark) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t tn = 0; tn < nt; ++tn) {
+            if (!mark) continue;
+            int64_t n0 = tn * BN, n1 = n0 + BN < N ? n0 + BN : N;
+            uint64_t f_tile = 0, u_tile = 0;
+            for (int64_t tk = 0; tk < kt; ++tk) {
+                int64_t k0 = tk * BK, k1 = k0 + BK < K ? k0 + BK : K;
+                uint64_t blocks = blocks_touched(mark, layout, K, N, br, bc, s, G, k0, k1, n0, n1);
+                f_tile += blocks * (uint64_t)G;
+                u_tile += (uint64_t)((k1 - k0) * (n1 - n0) * s);
+                q_sum += blocks;
+            }
+            f_sum += f_tile;
+            u_sum += u_tile;
+            if (per_ntile_fetched) per_ntile_fetched[tn] = f_tile;
+            if (per_ntile_used) per_ntile_used[tn] = u_tile;
+        }
+        free(mark);
+    }
+    if (failed) return -2;
+    *fetched = f_sum;
+    *used = u_sum;
+    *requests = q_sum;
+    return 0;
+}
+
+static int read_amp_args_ok(int64_t N, int64_t K, int64_t BM, int64_t BN, int64_t BK,
+                            int layout, int64_t G, int64_t br, int64_t bc, int64_t s) {
+    if (N <= 0 || K <= 0 || BM <= 0 || BN <= 0 || BK <= 0 || G <= 0 || s <= 0) return 0;
+    if (layout == TLO_TILE_MAJOR) {
+        if (br <= 0 || bc <= 0 || br * bc * s != G) return 0;     /* Section 3.1: h*w*s = G */
+        if (K % br != 0 || N % bc != 0) return 0;                 /* Section 3.3 */
+    } else if (layout != TLO_ROW_MAJOR && layout != TLO_COL_MAJOR) {
+        return 0;
+    }
+    return 1;
+}
+
+int tlo_read_amp(int64_t M, int64_t N, int64_t K, int64_t BM, int64_t BN, int64_t BK,
+                 int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                 uint64_t* fetched, uint64_t* used, uint64_t* requests,
+                 uint64_t* per_tile_fetched, uint64_t* per_tile_used) {
+    if (M < 0 || !read_amp_args_ok(N, K, BM, BN, BK, layout, G, br, bc, s)) return -1;
+    int64_t mt = ceil_div(M, BM), nt = ceil_div(N, BN);
+    uint64_t f = 0, u = 0, q = 0;
+    uint64_t* pf = NULL;
+    uint64_t* pu = NULL;
+    if (per_tile_fetched && per_tile_used && mt > 0) { pf = per_tile_fetched; pu = per_tile_used; }
+    int rc = weight_loads_one_mtile(N, K, BN, BK, layout, G, br, bc, s, &f, &u, &q, pf, pu);
+    if (rc) return rc;
+    /* every m-tile's CTAs issue the same weight loads */
+    for (int64_t tm = 1; tm < mt && pf; ++tm)
+        for (int64_t tn = 0; tn < nt; ++tn) {
+            pf[tm * nt + tn] = pf[tn];
+            pu[tm * nt + tn] = pu[tn];
+        }
+    *fetched = f * (uint64_t)mt;
+    *used = u * (uint64_t)mt;
+    if (requests) *requests = q * (uint64_t)mt;
+    return 0;
+}
+
+int tlo_read_amp_grouped(const int32_t* offsets, int E, int64_t N, int64_t K,
+                         int64_t BM, int64_t BN, int64_t BK,
+                         int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                         uint64_t* fetched, uint64_t* used, uint64_t* requests) {
+    if (E < 0 || !read_amp_args_ok(N, K, BM, BN, BK, layout, G, br, bc, s)) return -1;
+    uint64_t f1 = 0, u1 = 0, q1 = 0;
+    /* every expert's weight has the same shape and starts on a G boundary,
+     * so one expert's one-m-tile count serves all of them */
+    int rc = weight_loads_one_mtile(N, K, BN, BK, layout, G, br, bc, s, &f1, &u1, &q1, NULL, NULL);
+    if (rc) return rc;
+    uint64_t f = 0, u = 0, q = 0;
+    for (int e = 0; e < E; ++e) {
+        int64_t Me = (int64_t)offsets[e + 1] - (int64_t)offsets[e];
+        if (Me < 0) return -1;
+        if (Me == 0) continue;                    /* an expert with no token launches no CTA */
+        uint64_t mt = (uint64_t)ceil_div(Me, BM);
+        f += f1 * mt;
+        u += u1 * mt;
+        q += q1 * mt;
+    }
+    *fetched = f;
+    *used = u;
+    if (requests) *requests = q;
+    return 0;
+}

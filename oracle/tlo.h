@@ -1,0 +1,106 @@
+/*
+ * tlo -- TileLens ORACLE.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, obviously-correct CPU statement of what the tile-major hot
+ * path computes: the layout index functions, the relayout permutation, the
+ * fp64 matrix product and the brute-force count of G-byte blocks touched by
+ * every weight-tile load.  Nothing here is blocked, fused or reordered beyond
+ * what the paper's definitions state, and nothing here is shared with the
+ * CUDA library (no common header, helper, table or constant).  Only tests,
+ * the smoke check and the CPU-baseline leg of the benchmark may call it; the
+ * product path never does.
+ *
+ * Orientation (one reading used everywhere): the weight operand B is logically
+ * K x N and is stored with N contiguous ("row-major" as in Section 2.4 and the
+ * 128x256 example of Section 6.5, where each tile row is one contiguous strip).
+ * The paper writes its equations for the K-contiguous (column-major) flavour
+ * and states that the other flavour follows by exchanging rows and columns
+ * (Section 3.2); tlo_off_tile is that exchanged form, tlo_eq2 is the literal
+ * printed form, and the tests check one against the other.
+ *
+ * Pins (see tests/test_oracle_*.py): every function below is pinned to values
+ * the paper prints, to closed forms, to invariants or to brute force on tiny
+ * inputs.  No function here is "parity unpinned".
+ */
+#ifndef TLO_H
+#define TLO_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { TLO_ROW_MAJOR = 0, TLO_COL_MAJOR = 1, TLO_TILE_MAJOR = 2 };
+enum { TLO_TO_TILE_MAJOR = 0, TLO_TO_ROW_MAJOR = 1 };
+
+/* Section 2.4: byte offset of element (r,c) of a rows x cols matrix of s-byte
+ * elements when a row / a column is contiguous. */
+int64_t tlo_off_row(int64_t r, int64_t c, int64_t rows, int64_t cols, int64_t s);
+int64_t tlo_off_col(int64_t r, int64_t c, int64_t rows, int64_t cols, int64_t s);
+
+/* Eq. 1 + Eq. 2 with rows and columns exchanged (Section 3.2, first sentence):
+ * memory tile = br rows x bc contiguous columns; tiles ordered row-major over
+ * the tile grid, elements row-major inside a tile. */
+int64_t tlo_off_tile(int64_t r, int64_t c, int64_t rows, int64_t cols,
+                     int64_t br, int64_t bc, int64_t s);
+
+/* One switch over the three layouts (layout = TLO_*_MAJOR). */
+int64_t tlo_off(int layout, int64_t r, int64_t c, int64_t rows, int64_t cols,
+                int64_t br, int64_t bc, int64_t s);
+
+/* Eq. 1 as printed: out = {i', j', T_i, T_j} for memory tile a x b. */
+void tlo_eq1(int64_t i, int64_t j, int64_t a, int64_t b, int64_t out[4]);
+/* Eq. 2 as printed (K x N matrix, K contiguous, memory tile a x b). */
+int64_t tlo_eq2(int64_t i, int64_t j, int64_t K, int64_t N, int64_t a, int64_t b, int64_t s);
+/* Eq. 3: the 4-D coordinate of Eq. 1 dotted with stride (1, a, ab, Kb), in bytes. */
+int64_t tlo_eq3(int64_t i, int64_t j, int64_t K, int64_t N, int64_t a, int64_t b, int64_t s);
+
+/* Section 4.3 "Default tile-major for LGMS allocations" / Section 5.1: the
+ * weights are rewritten once into tile-major order; same bytes, new places.
+ * Copies every element through the index functions.  Returns 0, or -1 when
+ * br/bc do not divide rows/cols (Section 3.3 requires divisibility). */
+int tlo_relayout(const void* src, void* dst, int64_t rows, int64_t cols, int64_t s,
+                 int64_t br, int64_t bc, int direction);
+
+/* bf16 bit pattern -> double (exact: bf16 is a prefix of binary32). */
+double tlo_bf16_to_double(uint16_t h);
+
+/* Section 2.3: C = A x B with A M x K (bf16, row-major) and B K x N (bf16,
+ * stored in `layout` with memory tile br x bc), evaluated only at the n listed
+ * (idx_i[t], idx_j[t]) positions, as the plain sum over k in fp64.
+ * C[t] = sum_k A[i][k]*B[k][j];  S[t] = sum_k |A[i][k]*B[k][j]|. */
+int tlo_matmul_at(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
+                  int64_t M, int64_t N, int64_t K, int64_t n,
+                  const int64_t* idx_i, const int64_t* idx_j, double* C, double* S);
+/* The same at every (i,j): C and S are M x N row-major. */
+int tlo_matmul(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
+               int64_t M, int64_t N, int64_t K, double* C, double* S);
+
+/* Sections 1, 2.5, 6.5: read amplification of the weight operand under access
+ * granularity G.  The tiled product has ceil(M/BM) x ceil(N/BN) CTA tiles and
+ * ceil(K/BK) iterations; each (CTA tile, iteration) loads the clipped BK x BN
+ * rectangle of B.  For every such load, the set of distinct G-byte blocks that
+ * hold any byte of the rectangle is built element by element; fetched += |set|*G,
+ * used += elements*s, requests += |set|.  No sharing is credited between loads.
+ * If per_tile_fetched/used are non-NULL they receive one entry per
+ * (m-tile, n-tile), m-tile major. */
+int tlo_read_amp(int64_t M, int64_t N, int64_t K, int64_t BM, int64_t BN, int64_t BK,
+                 int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                 uint64_t* fetched, uint64_t* used, uint64_t* requests,
+                 uint64_t* per_tile_fetched, uint64_t* per_tile_used);
+
+/* Section 2.3 (MoE: every expert performs the same product): the same count
+ * summed over experts e with offsets[e+1]-offsets[e] > 0 rows, each expert's
+ * K x N weight its own G-aligned allocation. */
+int tlo_read_amp_grouped(const int32_t* offsets, int E, int64_t N, int64_t K,
+                         int64_t BM, int64_t BN, int64_t BK,
+                         int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                         uint64_t* fetched, uint64_t* used, uint64_t* requests);
+
+/* Threads the parallel loops above will use. */
+int tlo_num_threads(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif
