@@ -1,0 +1,186 @@
+/*
+ * tilelens.h -- C ABI of the B200 (sm_100a) tile-major GEMM hot path.
+ *
+ * The operations are the ones the TileLens paper states: a weight matrix is
+ * rewritten once into tile-major order (Section 3), a tiled matmul reads it
+ * through tensor-map (TMA) views (Sections 2.3, 4.1, 4.2), and the read
+ * amplification a G-byte-granular memory would see is counted per CTA tile
+ * load (Sections 1, 2.5, 6.5).
+ *
+ * Conventions that hold for every call
+ *   - Orientation.  The weight operand B is logically K x N.  "Row-major"
+ *     keeps N contiguous; a memory tile ("block") is block_rows K-rows by
+ *     block_cols contiguous N-columns, block_rows*block_cols*elem_bytes == G.
+ *     Blocks are packed row-major over the block grid and are row-major
+ *     inside (Eq. 1 and Eq. 2 with rows and columns exchanged, as Section 3.2
+ *     allows).  The paper's (a, b) is (block_cols, block_rows).
+ *   - Pointers named d_* or documented "device" are CUDA device pointers of
+ *     the current device; h_* are host pointers.  The caller owns every
+ *     buffer it passes.  Nothing the library allocates has to be freed by
+ *     the caller.
+ *   - Streams are `cudaStream_t` passed as void*; NULL is the default stream.
+ *     Calls that take a stream enqueue work and return without waiting.
+ *   - Every function returns a tl_status (0 = TL_OK).  Argument errors are
+ *     found on the host before anything is enqueued.  A device-side wait that
+ *     ran out (every wait in the kernels is bounded) raises a flag that
+ *     tl_device_status() reports after synchronising.
+ *   - Divisibility (Section 3.3): rows % block_rows == 0 and
+ *     cols % block_cols == 0, otherwise TL_ERR_INVALID_ARG; the caller pads.
+ *     block_rows and block_cols must be powers of two (Section 3.2), otherwise
+ *     TL_ERR_UNSUPPORTED.
+ */
+#ifndef TILELENS_H
+#define TILELENS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TL_OK = 0,
+    TL_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, G != rows*cols*s of the block, divisibility */
+    TL_ERR_UNSUPPORTED = 2,   /* valid request outside what the kernels instantiate */
+    TL_ERR_ALIGNMENT = 3,     /* pointer or pitch not aligned as the call requires */
+    TL_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed: see tl_last_cuda_error() */
+    TL_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired */
+    TL_ERR_WORKSPACE = 6      /* caller-supplied workspace too small */
+} tl_status;
+
+typedef enum { TL_TO_TILE_MAJOR = 0, TL_TO_ROW_MAJOR = 1 } tl_direction;
+typedef enum { TL_LAYOUT_ROW_MAJOR = 0, TL_LAYOUT_COL_MAJOR = 1, TL_LAYOUT_TILE_MAJOR = 2 } tl_layout;
+
+/* ------------------------------------------------------------------ misc */
+
+const char* tl_status_string(int status);
+/* Last cudaError_t / CUresult seen by a call that returned TL_ERR_CUDA (0 if none). */
+int tl_last_cuda_error(void);
+/* Stream used by the calls that take none (tl_relayout, tl_read_amp*).  Default: NULL stream. */
+int tl_set_stream(void* cuda_stream);
+/* Synchronises the device, then returns TL_ERR_TIMEOUT if any kernel since the
+ * last call gave up on a bounded wait (and clears the flag), else TL_OK.
+ * *detail (may be NULL) receives a code saying which wait expired. */
+int tl_device_status(uint32_t* detail);
+
+/* -------------------------------------------------------------- relayout */
+
+/*
+ * Row-major <-> tile-major rewrite of a rows x cols matrix of elem_bytes-wide
+ * elements (Section 3: same bytes, every contiguous G-byte block becomes a
+ * block_rows x block_cols rectangle; Section 5.1: done once at weight load).
+ *   d_src, d_dst  device, rows*cols*elem_bytes bytes each, must not overlap.
+ *   elem_bytes    1, 2 or 4.          G == block_rows*block_cols*elem_bytes.
+ *   direction     tl_direction.
+ * Enqueues one kernel on the tl_set_stream() stream.  A 16-byte-vectorised
+ * kernel staged through shared memory is used when cols*elem_bytes is a
+ * multiple of 16 and both pointers are 16-byte aligned; otherwise an
+ * element-wise kernel (same result, slower).  rows == 0 or cols == 0 is a no-op.
+ */
+int tl_relayout(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes,
+                int64_t G, int block_rows, int block_cols, int direction);
+/* The same on an explicit stream. */
+int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes,
+                   int64_t G, int block_rows, int block_cols, int direction, void* cuda_stream);
+
+/* ------------------------------------------------------------------ GEMM */
+
+/*
+ * C[M x N] (fp32, row-major) = A[M x K] (bf16, row-major) x B[K x N] (bf16),
+ * Section 2.3.  B is tile-major with G-byte blocks of block_rows x block_cols
+ * (Section 3; read through the multi-dimensional tensor-map view of Section
+ * 4.2, one TMA box per memory tile or per part of it inside the CTA tile), or
+ * plain row-major when block_rows == 0 (then G and block_cols are ignored).
+ * Products are accumulated in fp32 in tensor memory.
+ *   d_A, d_B     device, 16-byte aligned (d_B 128-byte aligned when tile-major).
+ *   d_C          device, M*N floats, fully overwritten.
+ *   cta_m/n/k    the CTA tile: cta_m token rows x cta_n weight columns per CTA,
+ *                cta_k weight rows per pipeline stage.  0,0,0 lets the library
+ *                choose.  Instantiated: cta_n in {128, 256}, cta_k in {64, 128},
+ *                cta_m a multiple of 16 in [16, 256] (cta_n == 256: at most 128).
+ *                Tiles may overhang M, N and K.
+ *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,
+ *   N % block_cols == 0, block_rows >= 8, block_cols*2 >= 16 bytes;
+ *   row-major: N % 64 == 0.  Other block shapes: TL_ERR_UNSUPPORTED.
+ * When M <= 64 (decode) the K loop of every output tile is cut stream-K
+ * fashion over all SMs; partial tiles go through a workspace and are summed
+ * in a fixed order, so results are reproducible run to run.  The workspace is
+ * the caller's (tl_set_workspace) or one the library grows on demand.
+ * M == 0 is a no-op.
+ */
+int tl_gemm(const void* d_A_rowmajor, const void* d_B_tilemajor, float* d_C,
+            int64_t M, int64_t N, int64_t K,
+            int64_t G, int block_rows, int block_cols,
+            int cta_m, int cta_n, int cta_k, void* cuda_stream);
+
+/*
+ * Grouped (mixture-of-experts) form, Section 2.3: rows of A are sorted by
+ * expert; expert e owns rows [offsets[e], offsets[e+1]) and multiplies them
+ * with its own K x N weight.  The E weights are separate tile-major (or
+ * row-major) buffers of K*N*2 bytes laid end to end in d_B_experts.
+ *   d_offsets    device, E+1 int32, non-decreasing, offsets[0] == 0,
+ *                offsets[E] == total_rows.  Experts with no row cost nothing.
+ *   d_C          total_rows x N floats; every row is written.
+ * cta_m is an upper bound: each tile uses the smallest instantiated token
+ * count that covers its rows.
+ */
+int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
+                    const int32_t* d_offsets, int E, int64_t total_rows,
+                    int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                    int cta_m, int cta_n, int cta_k, void* cuda_stream);
+
+/* Bytes of workspace tl_gemm / tl_gemm_grouped may need for these sizes on the current device. */
+size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k);
+/* Hands the library a caller-owned device workspace (256-byte aligned); (NULL, 0) returns to the
+ * internal one.  The buffer must stay valid until the last call using it has finished. */
+int tl_set_workspace(void* d_ptr, size_t bytes);
+
+/*
+ * End-to-end form with host buffers: copies A and the ROW-MAJOR weight to the
+ * device, rewrites the weight into tile-major blocks (block_rows == 0: keeps
+ * it row-major), multiplies, copies C back and waits for it.
+ *   h_A, h_B_rowmajor, h_C   host (pinned memory makes the copies asynchronous).
+ *   d_scratch                device, at least tl_gemm_host_scratch_bytes() bytes, 256-byte aligned.
+ */
+int tl_gemm_host(const void* h_A, const void* h_B_rowmajor, float* h_C,
+                 int64_t M, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                 int cta_m, int cta_n, int cta_k,
+                 void* d_scratch, size_t scratch_bytes, void* cuda_stream);
+size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
+
+/* --------------------------------------------------- read amplification */
+
+/*
+ * Read amplification of the weight operand under access granularity G
+ * (Sections 1, 2.5; "requests per compute tile" of Section 6.5).  The schedule
+ * is the GEMM's: ceil(M/cta_m) x ceil(N/cta_n) CTA tiles, ceil(K/cta_k)
+ * iterations, each loading the clipped cta_k x cta_n rectangle of B.  Per
+ * load, the distinct G-byte blocks holding any byte of the rectangle are
+ * counted (B starts on a G boundary); nothing is shared between loads.
+ *   bytes_fetched = sum of blocks * G,  bytes_used = sum of rectangle bytes,
+ *   requests (may be NULL) = sum of blocks.  All host out-parameters; exact.
+ * layout is a tl_layout; block_rows/block_cols only matter for tile-major.
+ * Any positive tile sizes are accepted (not only the GEMM's).  Runs one small
+ * kernel (one warp per CTA tile) on the tl_set_stream() stream and waits.
+ */
+int tl_read_amp(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
+                int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
+                uint64_t* bytes_fetched, uint64_t* bytes_used, uint64_t* requests);
+
+/* Grouped form: sum over experts with rows; h_offsets is a HOST array of E+1 int32. */
+int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K,
+                        int cta_m, int cta_n, int cta_k,
+                        int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
+                        uint64_t* bytes_fetched, uint64_t* bytes_used, uint64_t* requests);
+
+/* Per-CTA-tile form: d_fetched / d_used are DEVICE arrays of
+ * ceil(M/cta_m)*ceil(N/cta_n) uint64, m-tile major.  Asynchronous on cuda_stream. */
+int tl_read_amp_per_cta(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
+                        int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
+                        uint64_t* d_fetched, uint64_t* d_used, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TILELENS_H */

@@ -1,0 +1,181 @@
+"""Thin Python binding of the tilelens C ABI (``include/tilelens.h``): argument marshalling only.
+
+Every step of the path runs inside ``libtilelens.so``.  torch is used for device
+memory and streams, nothing else.  There is no fallback: if the library has not
+been built, or a call returns a non-zero status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtilelens.so")
+
+TL_OK = 0
+TO_TILE_MAJOR, TO_ROW_MAJOR = 0, 1
+LAYOUT_ROW_MAJOR, LAYOUT_COL_MAJOR, LAYOUT_TILE_MAJOR = 0, 1, 2
+
+# Every symbol include/tilelens.h declares: (name, restype, argtypes)
+_i64, _int, _vp, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
+_u64p = ctypes.POINTER(ctypes.c_uint64)
+_SIGNATURES = {
+    "tl_status_string": (ctypes.c_char_p, [_int]),
+    "tl_last_cuda_error": (_int, []),
+    "tl_set_stream": (_int, [_vp]),
+    "tl_device_status": (_int, [ctypes.POINTER(ctypes.c_uint32)]),
+    "tl_relayout": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int]),
+    "tl_relayout_on": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int, _vp]),
+    "tl_gemm": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_grouped": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int, _int, _int]),
+    "tl_set_workspace": (_int, [_vp, _sz]),
+    "tl_gemm_host": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp, _sz, _vp]),
+    "tl_gemm_host_scratch_bytes": (_sz, [_i64, _i64, _i64]),
+    "tl_read_amp": (_int, [_i64, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int, _u64p, _u64p, _u64p]),
+    "tl_read_amp_grouped": (_int, [_vp, _int, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int,
+                                   _u64p, _u64p, _u64p]),
+    "tl_read_amp_per_cta": (_int, [_i64, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int, _vp, _vp, _vp]),
+}
+
+_lib = None
+
+
+class TileLensError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().tl_status_string(status).decode()
+        extra = f" (cuda error {lib().tl_last_cuda_error()})" if status == 4 else ""
+        super().__init__(f"{where}: {msg}{extra}")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libtilelens.so; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2607_04031_b200.build` "
+                "(nvcc, sm_100a). The CUDA library is the only implementation of this path.")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(L, name)          # AttributeError if the library lacks a declared symbol
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def declared_symbols():
+    return list(_SIGNATURES)
+
+
+def _check(status: int, where: str):
+    if status != TL_OK:
+        raise TileLensError(status, where)
+
+
+def _dev_ptr(t: torch.Tensor) -> int:
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def status_string(status: int) -> str:
+    return lib().tl_status_string(status).decode()
+
+
+def set_stream(stream=None):
+    _check(lib().tl_set_stream(_stream_ptr(stream)), "tl_set_stream")
+
+
+def device_status():
+    """Synchronises; raises TileLensError(TL_ERR_TIMEOUT) if a kernel abandoned a bounded wait."""
+    detail = ctypes.c_uint32(0)
+    st = lib().tl_device_status(ctypes.byref(detail))
+    if st != TL_OK:
+        raise TileLensError(st, f"tl_device_status detail=0x{detail.value:x}")
+
+
+def relayout(src: torch.Tensor, dst: torch.Tensor, rows: int, cols: int, elem_bytes: int, G: int,
+             block_rows: int, block_cols: int, direction: int, stream=None):
+    _check(lib().tl_relayout_on(_dev_ptr(src), _dev_ptr(dst), rows, cols, elem_bytes, G, block_rows, block_cols,
+                                direction, _stream_ptr(stream)), "tl_relayout")
+
+
+def gemm(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, M: int, N: int, K: int, G: int = 4096,
+         block_rows: int = 16, block_cols: int = 128, cta=(0, 0, 0), stream=None):
+    """C (fp32 [M,N]) = A (bf16 [M,K]) x B (bf16, tile-major blocks; block_rows == 0: row-major [K,N])."""
+    _check(lib().tl_gemm(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), M, N, K, G, block_rows, block_cols,
+                         cta[0], cta[1], cta[2], _stream_ptr(stream)), "tl_gemm")
+
+
+def gemm_grouped(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, offsets: torch.Tensor, E: int,
+                 total_rows: int, N: int, K: int, G: int = 4096, block_rows: int = 16, block_cols: int = 128,
+                 cta=(0, 0, 0), stream=None):
+    _check(lib().tl_gemm_grouped(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), _dev_ptr(offsets), E, total_rows, N, K, G,
+                                 block_rows, block_cols, cta[0], cta[1], cta[2], _stream_ptr(stream)),
+           "tl_gemm_grouped")
+
+
+def gemm_workspace_bytes(M: int, N: int, K: int, cta=(0, 0, 0)) -> int:
+    return int(lib().tl_gemm_workspace_bytes(M, N, K, cta[0], cta[1], cta[2]))
+
+
+def set_workspace(buf: torch.Tensor | None):
+    if buf is None:
+        _check(lib().tl_set_workspace(None, 0), "tl_set_workspace")
+    else:
+        _check(lib().tl_set_workspace(_dev_ptr(buf), buf.numel() * buf.element_size()), "tl_set_workspace")
+
+
+def gemm_host_scratch_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().tl_gemm_host_scratch_bytes(M, N, K))
+
+
+def gemm_host(A_host: torch.Tensor, B_rowmajor_host: torch.Tensor, C_host: torch.Tensor, M: int, N: int, K: int,
+              scratch: torch.Tensor, G: int = 4096, block_rows: int = 16, block_cols: int = 128, cta=(0, 0, 0),
+              stream=None):
+    """Host buffers in, host buffer out: H2D copies, relayout, GEMM and D2H copy all inside the call."""
+    for t in (A_host, B_rowmajor_host, C_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("gemm_host takes contiguous host tensors")
+    _check(lib().tl_gemm_host(A_host.data_ptr(), B_rowmajor_host.data_ptr(), C_host.data_ptr(), M, N, K, G,
+                              block_rows, block_cols, cta[0], cta[1], cta[2], _dev_ptr(scratch),
+                              scratch.numel() * scratch.element_size(), _stream_ptr(stream)), "tl_gemm_host")
+
+
+def read_amp(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int = 0, block_cols: int = 0,
+             elem_bytes: int = 2):
+    """Returns (bytes_fetched, bytes_used, requests), exact integers."""
+    f, u, q = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    _check(lib().tl_read_amp(M, N, K, cta[0], cta[1], cta[2], layout, G, block_rows, block_cols, elem_bytes,
+                             ctypes.byref(f), ctypes.byref(u), ctypes.byref(q)), "tl_read_amp")
+    return int(f.value), int(u.value), int(q.value)
+
+
+def read_amp_grouped(offsets_host, N: int, K: int, cta, layout: int, G: int, block_rows: int = 0,
+                     block_cols: int = 0, elem_bytes: int = 2):
+    import numpy as np
+    offs = np.ascontiguousarray(offsets_host, dtype=np.int32)
+    f, u, q = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    _check(lib().tl_read_amp_grouped(offs.ctypes.data, offs.size - 1, N, K, cta[0], cta[1], cta[2], layout, G,
+                                     block_rows, block_cols, elem_bytes, ctypes.byref(f), ctypes.byref(u),
+                                     ctypes.byref(q)), "tl_read_amp_grouped")
+    return int(f.value), int(u.value), int(q.value)
+
+
+def read_amp_per_cta(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int, block_cols: int,
+                     elem_bytes: int, fetched: torch.Tensor, used: torch.Tensor, stream=None):
+    _check(lib().tl_read_amp_per_cta(M, N, K, cta[0], cta[1], cta[2], layout, G, block_rows, block_cols, elem_bytes,
+                                     _dev_ptr(fetched), _dev_ptr(used), _stream_ptr(stream)), "tl_read_amp_per_cta")

@@ -1,0 +1,708 @@
+// Tiled bf16 GEMM reading a tile-major (or row-major) weight operand, for sm_100a.
+//
+//   C[M x N] (fp32) = A[M x K] (bf16, K contiguous) x B[K x N] (bf16)          (Section 2.3)
+//
+// B is read through a 5-D tensor-map view of the tile-major buffer (the 4-D view of Eq. 3 in the
+// N-contiguous flavour, with the contiguous extent of a memory tile split into 128-byte atoms):
+// one TMA box per memory tile, or per part of a memory tile that lies inside the CTA tile.
+// The boxes land in shared memory in exactly the canonical "MN-major, 128-byte swizzle" form
+// that tcgen05.mma reads, so the weights are the M-side operand of the MMA (128 weight columns
+// per instruction) and the token rows are its N-side operand (16..256 tokens, K-major).  The
+// accumulator therefore holds C transposed: TMEM lane = weight column, TMEM column = token.
+//
+// One persistent CTA per SM, six warps:
+//   warp 0      TMA producer   (one lane)   ring of shared-memory stages, mbarrier expect-tx
+//   warp 1      MMA issuer     (one lane)   tcgen05.mma into one of two TMEM accumulators
+//   warps 2..5  epilogue                    tcgen05.ld -> fp32 -> C (128-byte coalesced rows)
+// Work is a list of (output tile, K range).  Data-parallel mode hands whole tiles round-robin;
+// stream-K mode cuts the flattened (tile, K iteration) space into one contiguous range per CTA
+// (decode: all SMs stream weights even when there are fewer tiles than SMs).  Partial tiles go to
+// a workspace; the CTA that arrives last at a tile's counter adds the partials in K order, so the
+// result does not depend on arrival order.  Nothing ever spins on another CTA.
+// Every mbarrier wait is bounded (see mbar_wait_bounded).
+#include "tl_common.cuh"
+
+#include <cstring>
+
+namespace tl {
+
+constexpr int kGemmThreads = 192;
+constexpr int kMaxStages = 16;
+constexpr int kMaxExperts = 1024;
+constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 256 rows
+constexpr int kAtomBytes = 128;            // one swizzle row: 64 bf16
+constexpr uint32_t kCounterBytes = 65536;  // head of the workspace: per-tile arrival counters
+constexpr int kMaxCounterTiles = kCounterBytes / 4;
+
+struct alignas(64) GemmParams {
+    CUtensorMap tmap_a[kNumBoxChoices];
+    CUtensorMap tmap_b;
+    float* C;
+    float* partials;            // stream-K partial tiles: slot = BM x BN floats
+    uint32_t* counters;         // per output tile, zero outside a launch
+    const int32_t* offsets;     // grouped: device E+1 row offsets; dense: nullptr
+    uint32_t* status;
+    int64_t ldc;                // N
+    int M;                      // dense rows (grouped: total rows)
+    int N, K, E;
+    int BM;                     // token rows per CTA tile: 16, 32, 64, 128 or 256
+    int BN;                     // weight columns per CTA tile: 128 or 256
+    int n_tiles, k_iters;
+    int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
+    int num_stages;
+    // weight-operand geometry
+    int row_major;              // 1: B is [K][N] row-major (viewed as one big memory tile)
+    int br_log2, bc_log2;       // memory tile (tile-major only)
+    int k_coord_per_expert;     // added to the K coordinate per expert (K/br blocks, or K rows)
+    int box_rows, box_atoms;    // rows and 128-byte atoms of one box
+    int kbx, nbx;               // boxes per stage along K and along N
+    uint32_t box_bytes;
+    uint32_t lbo, sbo;          // descriptor strides of the MN-major operand, bytes
+    uint32_t kstep_off[8];      // byte offset of each 16-row K step inside a stage
+};
+
+struct TileInfo {
+    int n0;          // first weight column
+    int row0;        // first row of A / C
+    int rows;        // valid rows (<= BM)
+    int expert;
+};
+
+// ------------------------------------------------------------------ scheduler
+struct Work {
+    int tile, kbeg, kend;
+};
+
+struct Sched {
+    int stream_k, k_iters, tiles_total, grid_eff, cta;
+    int next_tile;
+    long long it, it_end, it_begin;
+
+    __device__ long long range_begin(int c) const {
+        return (static_cast<long long>(tiles_total) * k_iters * c) / grid_eff;
+    }
+    __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid, int cta_) {
+        stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_;
+        long long total = static_cast<long long>(tiles_total) * k_iters;
+        grid_eff = total < grid ? static_cast<int>(total) : grid;
+        next_tile = cta;
+        if (grid_eff == 0 || cta >= grid_eff) { it = it_end = it_begin = 0; next_tile = tiles_total; return; }
+        it_begin = it = range_begin(cta);
+        it_end = range_begin(cta + 1);
+    }
+    __device__ bool next(Work& w) {
+        if (!stream_k) {
+            if (next_tile >= tiles_total) return false;
+            w.tile = next_tile; w.kbeg = 0; w.kend = k_iters;
+            next_tile += gridDim.x;
+            return true;
+        }
+        if (it >= it_end) return false;
+        int t = static_cast<int>(it / k_iters);
+        int kb = static_cast<int>(it - static_cast<long long>(t) * k_iters);
+        long long left = it_end - it;
+        int ke = (k_iters - kb) < left ? k_iters : kb + static_cast<int>(left);
+        w.tile = t; w.kbeg = kb; w.kend = ke;
+        it += ke - kb;
+        return true;
+    }
+    // CTA whose range holds flattened iteration x.
+    __device__ int owner(long long x) const {
+        long long total = static_cast<long long>(tiles_total) * k_iters;
+        int c = static_cast<int>(((x + 1) * grid_eff + total - 1) / total) - 1;
+        if (c < 0) c = 0;
+        if (c >= grid_eff) c = grid_eff - 1;
+        while (c > 0 && range_begin(c) > x) --c;
+        while (c + 1 < grid_eff && range_begin(c + 1) <= x) ++c;
+        return c;
+    }
+    // Partial-tile slot of CTA c for tile t: 2c when the tile is the first thing c works on, else 2c+1.
+    __device__ int slot(int c, int t) const {
+        return 2 * c + (range_begin(c) < static_cast<long long>(t) * k_iters ? 1 : 0);
+    }
+};
+
+__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* prefix, int tile) {
+    // prefix[e] = tiles of experts before e; tiles of one expert: n-tile major, m-tile minor.
+    int lo = 0, hi = p.E;                  // find e with prefix[e] <= tile < prefix[e+1]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (prefix[mid] <= tile) lo = mid; else hi = mid;
+    }
+    const int e = lo;
+    const int local = tile - prefix[e];
+    const int mt = (prefix[e + 1] - prefix[e]) / p.n_tiles;
+    const int row_begin = p.offsets ? p.offsets[e] : 0;
+    const int row_end = p.offsets ? p.offsets[e + 1] : p.M;
+    TileInfo t;
+    t.expert = e;
+    t.n0 = (local / mt) * p.BN;
+    t.row0 = row_begin + (local % mt) * p.BM;
+    t.rows = row_end - t.row0 < p.BM ? row_end - t.row0 : p.BM;
+    return t;
+}
+
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    // start address, leading and stride byte offsets in 16-byte units; descriptor version 1 (bit 46);
+    // 128-byte swizzle (value 2 in bits 61..63)
+    return uint64_t((addr & 0x3FFFFu) >> 4) | (uint64_t(lbo >> 4) << 16) | (uint64_t(sbo >> 4) << 32) |
+           (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+
+__device__ __forceinline__ void epilogue_bar_sync() {
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+// kBK: weight rows per stage (64 or 128).  kNumN: 128-column groups per CTA tile (1 or 2).
+template <int kBK, int kNumN>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+    constexpr int kBN = 128 * kNumN;
+    constexpr int kKSteps = kBK / 16;
+    constexpr int kSubK = kBK / 64;                        // token boxes per stage
+    constexpr uint32_t kWBytes = kBK * kBN * 2;            // weight bytes per stage
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t acc_full_bar[2];
+    __shared__ __align__(8) uint64_t acc_empty_bar[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t abort_flag;
+    __shared__ uint32_t arrival_bcast;
+    __shared__ int prefix[kMaxExperts + 1];
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.BM * kAtomBytes;
+    uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    const int acc_cols = p.BM;                               // TMEM columns per 128-column group
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < uint32_t(2 * kNumN * acc_cols)) tmem_cols <<= 1;
+
+    // ---------------------------------------------------------------- set-up
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 4); }
+        abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&p.tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_slot, tmem_cols);
+        tmem_relinquish();
+    }
+    // tiles before each expert (dense: one "expert" holding all M rows)
+    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) prefix[e] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int e = 0; e < p.E; ++e) {
+            prefix[e] = acc;
+            const int rows = p.offsets ? p.offsets[e + 1] - p.offsets[e] : p.M;
+            acc += ((rows + p.BM - 1) / p.BM) * p.n_tiles;
+        }
+        prefix[p.E] = acc;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    const int tiles_total = prefix[p.E];
+
+    Sched sched;
+    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x);
+    volatile uint32_t* abort_ptr = &abort_flag;
+
+    if (warp == 0) {
+        // ============================================================ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            Work w;
+            bool ok = true;
+            while (ok && sched.next(w)) {
+                const TileInfo t = decode_tile(p, prefix, w.tile);
+                int bi = 0;
+                while ((16 << bi) < t.rows) ++bi;
+                const uint32_t a_bytes = uint32_t(16 << bi) * kAtomBytes;
+                const uint32_t tx = uint32_t(kSubK) * a_bytes + uint32_t(p.kbx * p.nbx) * p.box_bytes;
+                const int kc_expert = t.expert * p.k_coord_per_expert;
+                for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                    if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* sw = stages + size_t(stage) * stage_bytes;
+                    uint8_t* sa = sw + kWBytes;
+                    mbar_arrive_expect_tx(&full_bar[stage], tx);
+                    const int k0 = kit * kBK;
+#pragma unroll
+                    for (int sub = 0; sub < kSubK; ++sub)
+                        tma_load_2d(sa + size_t(sub) * p.BM * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
+                                    k0 + sub * 64, t.row0);
+                    for (int kb = 0; kb < p.kbx; ++kb) {
+                        const int k = k0 + kb * p.box_rows;
+                        for (int nb = 0; nb < p.nbx; ++nb) {
+                            const int n = t.n0 + nb * p.box_atoms * 64;
+                            uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
+                            if (p.row_major)
+                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k + kc_expert, n >> 6, 0, 0);
+                            else
+                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k & ((1 << p.br_log2) - 1),
+                                            (n & ((1 << p.bc_log2) - 1)) >> 6, n >> p.bc_log2,
+                                            (k >> p.br_log2) + kc_expert);
+                        }
+                    }
+                    ++issued;
+                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (!ok || *abort_ptr) {
+                // Giving up: let the copies already issued land before the CTA's shared memory goes away.
+                uint32_t s = stage, ph = phase;
+                const uint32_t back = issued < uint32_t(p.num_stages) ? issued : uint32_t(p.num_stages);
+                for (uint32_t i = 0; i < back; ++i) {
+                    if (s == 0) { s = p.num_stages; ph ^= 1; }
+                    --s;
+                    const uint64_t t0 = global_timer_ns();
+                    while (!mbar_try_wait(&full_bar[s], ph) && global_timer_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ============================================================= MMA issuer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            Work w;
+            bool ok = true;
+            while (ok && sched.next(w)) {
+                const TileInfo t = decode_tile(p, prefix, w.tile);
+                const uint32_t n_mma = uint32_t((t.rows + 15) & ~15);
+                // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = 128, N = n_mma
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((n_mma >> 3) << 17) |
+                                       ((128u >> 4) << 24);
+                if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * uint32_t(kNumN * acc_cols);
+                for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                    if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
+                    const uint32_t sa = sw + kWBytes;
+#pragma unroll
+                    for (int j = 0; j < kKSteps; ++j) {
+                        const uint64_t tok_desc = make_smem_desc(
+                            sa + uint32_t(j >> 2) * uint32_t(p.BM) * kAtomBytes + uint32_t(j & 3) * 32u, 16u, 1024u);
+#pragma unroll
+                        for (int u = 0; u < kNumN; ++u) {
+                            const uint64_t w_desc =
+                                make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * 2u * p.lbo, p.lbo, p.sbo);
+                            umma_bf16(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc,
+                                      (kit > w.kbeg || j > 0) ? 1u : 0u);
+                        }
+                    }
+                    umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
+                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full_bar[acc]);         // accumulator complete
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1;
+            }
+        }
+    } else {
+        // =============================================================== epilogue
+        const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31
+        const int et = (warp - 2) * 32 + lane;           // 0..127 among epilogue threads
+        uint32_t acc = 0, acc_phase = 0;
+        Work w;
+        while (sched.next(w)) {
+            const TileInfo t = decode_tile(p, prefix, w.tile);
+            const bool full = (w.kbeg == 0 && w.kend == p.k_iters);
+            const int n_mma = (t.rows + 15) & ~15;
+            bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
+            tc_fence_after_sync();
+            float* out;
+            int64_t ld;
+            if (full) {
+                out = p.C + int64_t(t.row0) * p.ldc + t.n0;
+                ld = p.ldc;
+            } else {
+                out = p.partials + size_t(sched.slot(sched.cta, w.tile)) * p.BM * kBN;
+                ld = kBN;
+            }
+            if (ok) {
+#pragma unroll
+                for (int u = 0; u < kNumN; ++u) {
+                    const int n_local = u * 128 + quarter * 32 + lane;
+                    const bool n_ok = full ? (t.n0 + n_local < p.N) : true;
+                    const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) +
+                                           acc * uint32_t(kNumN * acc_cols) + uint32_t(u * acc_cols);
+                    for (int c0 = 0; c0 < n_mma; c0 += 32) {
+                        if (n_mma - c0 >= 32) {
+                            uint32_t v[32];
+                            tmem_ld_32x32b_x32(taddr + c0, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                        } else {
+                            uint32_t v[16];
+                            tmem_ld_32x32b_x16(taddr + c0, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                        }
+                    }
+                }
+            }
+            // accumulator drained: hand it back to the MMA warp
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty_bar[acc]);
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1;
+
+            if (!full) {
+                // ---- stream-K fix-up: count arrivals; the last one adds the partials in K order.
+                __threadfence();
+                epilogue_bar_sync();
+                const long long tile_begin = static_cast<long long>(w.tile) * p.k_iters;
+                const int c_lo = sched.owner(tile_begin);
+                const int c_hi = sched.owner(tile_begin + p.k_iters - 1);
+                if (et == 0) {
+                    uint32_t old = (ok && !*abort_ptr) ? atomicAdd(&p.counters[w.tile], 1u) : 0xFFFFFFFFu;
+                    arrival_bcast = old;
+                }
+                epilogue_bar_sync();
+                const uint32_t old = arrival_bcast;
+                if (old == uint32_t(c_hi - c_lo)) {
+                    __threadfence();
+                    float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
+                    for (int u = 0; u < kNumN; ++u) {
+                        const int n_local = u * 128 + et;
+                        if (t.n0 + n_local >= p.N) continue;
+                        for (int r = 0; r < t.rows; ++r) {
+                            float sum = 0.f;
+                            for (int c = c_lo; c <= c_hi; ++c)
+                                sum += __ldcg(p.partials + size_t(sched.slot(c, w.tile)) * p.BM * kBN +
+                                              size_t(r) * kBN + n_local);
+                            dst[int64_t(r) * p.ldc + n_local] = sum;
+                        }
+                    }
+                    if (et == 0) p.counters[w.tile] = 0;     // ready for the next launch
+                }
+                epilogue_bar_sync();                          // arrival_bcast may be rewritten after this
+            }
+            if (*abort_ptr) break;
+        }
+    }
+
+    // --------------------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// ======================================================================== host
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                  const uint32_t* box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) {
+        state().last_cuda_error = int(cudaErrorSymbolNotFound);
+        return TL_ERR_CUDA;
+    }
+    cuuint64_t gdim[5], gstr[4];
+    cuuint32_t bdim[5], estr[5];
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bdim[i] = box[i]; estr[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i + 1];
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr, bdim,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        state().last_cuda_error = int(r);
+        return TL_ERR_CUDA;
+    }
+    return TL_OK;
+}
+
+static int ilog2(int64_t x) {
+    int l = 0;
+    while ((int64_t(1) << l) < x) ++l;
+    return l;
+}
+
+struct GemmPlan {
+    int BM, BN, BK;
+    int stream_k;
+    int grid;
+    int num_stages;
+    size_t smem_bytes;
+    size_t ws_bytes;
+};
+
+static int pick_bm(int64_t rows) {
+    int bm = 16;
+    while (bm < 256 && bm < rows) bm <<= 1;
+    return bm;
+}
+
+// Chooses / validates the CTA tile and the schedule.  rows_max: most rows any one problem has.
+static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
+                     bool grouped, GemmPlan* plan) {
+    if (int rc = ensure_device_info()) return rc;
+    const int sms = state().sm_count;
+    int BM = cta_m, BN = cta_n, BK = cta_k;
+    if (BM == 0 && BN == 0 && BK == 0) {
+        BM = pick_bm(rows_max);
+        BN = 128;
+        BK = 64;
+    }
+    if (BM != 16 && BM != 32 && BM != 64 && BM != 128 && BM != 256) return TL_ERR_UNSUPPORTED;
+    if (BN != 128 && BN != 256) return TL_ERR_UNSUPPORTED;
+    if (BK != 64 && BK != 128) return TL_ERR_UNSUPPORTED;
+    if (BN == 256 && BM > 128) return TL_ERR_UNSUPPORTED;   // 2 accumulators x 2 groups x BM columns <= 512
+    plan->BM = BM; plan->BN = BN; plan->BK = BK;
+    const size_t stage = size_t(BK) * BN * 2 + size_t(BK / 64) * BM * kAtomBytes;
+    const size_t budget = 227 * 1024 - 8 * 1024 - 1024;     // static barriers + prefix table + alignment slack
+    int stages = int(budget / stage);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return TL_ERR_UNSUPPORTED;
+    plan->num_stages = stages;
+    plan->smem_bytes = size_t(stages) * stage + 1024;
+    if (plan->smem_bytes < 120 * 1024) plan->smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
+    const int64_t k_iters = ceil_div(K, BK);
+    const int64_t total_iters = tile_bound * k_iters;
+    // Whole tiles when they fill the machine evenly enough, contiguous K ranges otherwise.
+    const int64_t waves = ceil_div(tile_bound, sms);
+    const bool even = tile_bound >= sms && double(tile_bound) / double(waves * sms) >= 0.92;
+    plan->stream_k = (grouped || !even) ? 1 : 0;
+    if (tile_bound > kMaxCounterTiles) plan->stream_k = 0;
+    int64_t grid = plan->stream_k ? (total_iters < sms ? total_iters : sms) : (tile_bound < sms ? tile_bound : sms);
+    if (grid < 1) grid = 1;
+    plan->grid = int(grid);
+    plan->ws_bytes = plan->stream_k ? kCounterBytes + size_t(2) * size_t(grid) * BM * BN * sizeof(float) : 0;
+    return TL_OK;
+}
+
+static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
+                       int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
+                       int cta_m, int cta_n, int cta_k, cudaStream_t stream) {
+    if (rows_total < 0 || N <= 0 || K <= 0 || E < 1) return TL_ERR_INVALID_ARG;
+    if (rows_total == 0) return TL_OK;
+    if (!d_A || !d_B || !d_C) return TL_ERR_INVALID_ARG;
+    if (rows_total >= (int64_t(1) << 31) || N >= (int64_t(1) << 31) || K * int64_t(E) >= (int64_t(1) << 31))
+        return TL_ERR_UNSUPPORTED;
+    if (E > kMaxExperts) return TL_ERR_UNSUPPORTED;
+    const bool row_major = br == 0;
+    if (!row_major) {
+        if (br < 0 || bc <= 0 || int64_t(br) * bc * 2 != G) return TL_ERR_INVALID_ARG;
+        if (!is_pow2(br) || !is_pow2(bc)) return TL_ERR_UNSUPPORTED;
+        if (K % br != 0 || N % bc != 0) return TL_ERR_INVALID_ARG;
+        if (br < 8 || bc < 64) return TL_ERR_UNSUPPORTED;       // TMA path: whole 8-row x 128-byte swizzle atoms
+    } else {
+        if (N % 64 != 0) return TL_ERR_UNSUPPORTED;
+    }
+    if (K % 8 != 0) return TL_ERR_UNSUPPORTED;                  // 16-byte row pitch of A
+    if (reinterpret_cast<uintptr_t>(d_A) % 16 != 0) return TL_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(d_B) % (row_major ? 16 : 128) != 0) return TL_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(d_C) % 4 != 0) return TL_ERR_ALIGNMENT;
+
+    GemmPlan plan;
+    {
+        // upper bound of tiles: every expert may add one ragged m-tile
+        const int bm_guess = (cta_m == 0 && cta_n == 0 && cta_k == 0) ? pick_bm(rows_max) : cta_m;
+        if (bm_guess <= 0) return TL_ERR_UNSUPPORTED;
+        const int bn_guess = (cta_n == 0) ? 128 : cta_n;
+        const int64_t mt_bound = d_offsets ? rows_total / bm_guess + E : ceil_div(rows_total, bm_guess);
+        if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K, cta_m, cta_n, cta_k,
+                               d_offsets != nullptr, &plan))
+            return rc;
+    }
+    if (d_offsets && K % plan.BK != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
+    if (int rc = ensure_control()) return rc;
+    void* ws = nullptr;
+    if (int rc = get_workspace(plan.ws_bytes, &ws)) return rc;
+
+    GemmParams p;
+    memset(&p, 0, sizeof p);
+    // ---- token operand A: [rows_total][K], boxes of 64 K-elements x {16..256} rows
+    for (int i = 0; i < kNumBoxChoices; ++i) {
+        const uint64_t dims[2] = {uint64_t(K), uint64_t(rows_total)};
+        const uint64_t str[2] = {2, uint64_t(K) * 2};
+        const uint32_t box[2] = {64, uint32_t(16 << i)};
+        if (int rc = encode(&p.tmap_a[i], d_A, 2, dims, str, box)) return rc;
+    }
+    // ---- weight operand B
+    const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
+    int RB, AB;
+    if (row_major) {
+        // [E*K][N] seen as (64, E*K, N/64): one box covers the whole stage.
+        RB = plan.BK;
+        AB = NA;
+        const uint64_t dims[5] = {64, uint64_t(K) * E, uint64_t(N / 64), 1, 1};
+        const uint64_t str[5] = {2, uint64_t(N) * 2, 128, uint64_t(N) * 2 * uint64_t(K) * E, uint64_t(N) * 2 * uint64_t(K) * E};
+        const uint32_t box[5] = {64, uint32_t(RB), uint32_t(AB), 1, 1};
+        if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+        p.k_coord_per_expert = int(K);
+    } else {
+        // Eq. 3 in the N-contiguous flavour, contiguous extent split into 64-element atoms:
+        // (64, br, bc/64, N/bc, E*K/br) with strides (1, bc, 64, br*bc, br*N) elements.
+        RB = br < plan.BK ? br : plan.BK;
+        AB = (bc < plan.BN ? bc : plan.BN) / 64;
+        const uint64_t dims[5] = {64, uint64_t(br), uint64_t(bc / 64), uint64_t(N / bc), uint64_t(K / br) * E};
+        const uint64_t str[5] = {2, uint64_t(bc) * 2, 128, uint64_t(G), uint64_t(br) * uint64_t(N) * 2};
+        const uint32_t box[5] = {64, uint32_t(RB), uint32_t(AB), 1, 1};
+        if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+        p.k_coord_per_expert = int(K / br);
+        p.br_log2 = ilog2(br);
+        p.bc_log2 = ilog2(bc);
+    }
+    p.row_major = row_major;
+    p.box_rows = RB;
+    p.box_atoms = AB;
+    p.kbx = plan.BK / RB;
+    p.nbx = NA / AB;
+    p.box_bytes = uint32_t(RB) * AB * kAtomBytes;
+    // Shared-memory image of a stage: [K box][N box][atom][row][64 elements].  Atom stride is RB*128
+    // everywhere; 8-row groups are 1024 bytes apart inside a box and one box row apart across boxes.
+    const uint32_t krow_bytes = uint32_t(NA) * RB * kAtomBytes;   // all boxes sharing one K range
+    p.lbo = uint32_t(RB) * kAtomBytes;
+    p.sbo = RB >= 16 ? 1024u : krow_bytes;
+    for (int j = 0; j < plan.BK / 16; ++j) {
+        const int row = j * 16;
+        p.kstep_off[j] = uint32_t(row / RB) * krow_bytes + uint32_t(row % RB) * kAtomBytes;
+    }
+    p.C = d_C;
+    p.counters = static_cast<uint32_t*>(ws);
+    p.partials = ws ? reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + kCounterBytes) : nullptr;
+    p.offsets = d_offsets;
+    p.status = state().ctl.d_status;
+    p.ldc = N;
+    p.M = int(rows_total);
+    p.N = int(N);
+    p.K = int(K);
+    p.E = E;
+    p.BM = plan.BM;
+    p.BN = plan.BN;
+    p.n_tiles = int(ceil_div(N, plan.BN));
+    p.k_iters = int(ceil_div(K, plan.BK));
+    p.stream_k = plan.stream_k;
+    p.num_stages = plan.num_stages;
+
+    cudaError_t err = cudaSuccess;
+#define TL_LAUNCH_GEMM(BK_, NN_)                                                                                   \
+    err = cudaFuncSetAttribute(gemm_kernel<BK_, NN_>, cudaFuncAttributeMaxDynamicSharedMemorySize,                 \
+                               int(plan.smem_bytes));                                                              \
+    if (err == cudaSuccess) gemm_kernel<BK_, NN_><<<plan.grid, kGemmThreads, plan.smem_bytes, stream>>>(p);
+    if (plan.BK == 64 && plan.BN == 128) { TL_LAUNCH_GEMM(64, 1) }
+    else if (plan.BK == 128 && plan.BN == 128) { TL_LAUNCH_GEMM(128, 1) }
+    else if (plan.BK == 64 && plan.BN == 256) { TL_LAUNCH_GEMM(64, 2) }
+    else { TL_LAUNCH_GEMM(128, 2) }
+#undef TL_LAUNCH_GEMM
+    if (err != cudaSuccess) return check_cuda(err);
+    return check_cuda(cudaGetLastError());
+}
+
+}  // namespace tl
+
+extern "C" {
+
+int tl_gemm(const void* d_A, const void* d_B, float* d_C, int64_t M, int64_t N, int64_t K, int64_t G, int block_rows,
+            int block_cols, int cta_m, int cta_n, int cta_k, void* cuda_stream) {
+    return tl::gemm_launch(d_A, d_B, d_C, nullptr, 1, M, M, N, K, G, block_rows, block_cols, cta_m, cta_n, cta_k,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
+int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C, const int32_t* d_offsets, int E,
+                    int64_t total_rows, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols, int cta_m,
+                    int cta_n, int cta_k, void* cuda_stream) {
+    if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
+    // Without a host copy of the offsets the largest expert is unknown: size tiles for the total.
+    return tl::gemm_launch(d_A_sorted, d_B_experts, d_C, d_offsets, E, total_rows, total_rows, N, K, G, block_rows,
+                           block_cols, cta_m, cta_n, cta_k, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {
+    tl::GemmPlan plan;
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    const int bm = (cta_m == 0 && cta_n == 0 && cta_k == 0) ? tl::pick_bm(M) : cta_m;
+    const int bn = cta_n == 0 ? 128 : cta_n;
+    if (bm <= 0) return 0;
+    // sized for the grouped schedule too (always stream-K, one CTA per SM)
+    if (tl::make_plan(M, (M / bm + 1) * tl::ceil_div(N, bn), N, K, cta_m, cta_n, cta_k, true, &plan)) return 0;
+    return plan.ws_bytes;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------ host-buffer form
+namespace tl {
+static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+}
+
+extern "C" {
+
+size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N <= 0 || K <= 0) return 0;
+    return tl::align256(size_t(M) * K * 2) + 2 * tl::align256(size_t(K) * N * 2) + tl::align256(size_t(M) * N * 4);
+}
+
+int tl_gemm_host(const void* h_A, const void* h_B_rowmajor, float* h_C, int64_t M, int64_t N, int64_t K, int64_t G,
+                 int block_rows, int block_cols, int cta_m, int cta_n, int cta_k, void* d_scratch,
+                 size_t scratch_bytes, void* cuda_stream) {
+    if (M < 0 || N <= 0 || K <= 0) return TL_ERR_INVALID_ARG;
+    if (M == 0) return TL_OK;
+    if (!h_A || !h_B_rowmajor || !h_C || !d_scratch) return TL_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_scratch) % 256 != 0) return TL_ERR_ALIGNMENT;
+    if (scratch_bytes < tl_gemm_host_scratch_bytes(M, N, K)) return TL_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(d_scratch);
+    const size_t a_bytes = size_t(M) * K * 2, b_bytes = size_t(K) * N * 2, c_bytes = size_t(M) * N * 4;
+    uint8_t* dA = base;
+    uint8_t* dB_row = dA + tl::align256(a_bytes);
+    uint8_t* dB_tile = dB_row + tl::align256(b_bytes);
+    float* dC = reinterpret_cast<float*>(dB_tile + tl::align256(b_bytes));
+    if (int rc = tl::check_cuda(cudaMemcpyAsync(dA, h_A, a_bytes, cudaMemcpyHostToDevice, stream))) return rc;
+    if (int rc = tl::check_cuda(cudaMemcpyAsync(dB_row, h_B_rowmajor, b_bytes, cudaMemcpyHostToDevice, stream)))
+        return rc;
+    const void* dB = dB_row;
+    if (block_rows != 0) {
+        if (int rc = tl_relayout_on(dB_row, dB_tile, K, N, 2, G, block_rows, block_cols, TL_TO_TILE_MAJOR, stream))
+            return rc;
+        dB = dB_tile;
+    }
+    if (int rc = tl_gemm(dA, dB, dC, M, N, K, G, block_rows, block_cols, cta_m, cta_n, cta_k, stream)) return rc;
+    if (int rc = tl::check_cuda(cudaMemcpyAsync(h_C, dC, c_bytes, cudaMemcpyDeviceToHost, stream))) return rc;
+    return tl::check_cuda(cudaStreamSynchronize(stream));
+}
+
+}  // extern "C"

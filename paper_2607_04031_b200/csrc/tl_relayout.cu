@@ -1,0 +1,281 @@
+// Row-major <-> tile-major relayout (Section 3; Eq. 1 and Eq. 2 in the N-contiguous flavour).
+//
+// Bandwidth-bound: every byte is read once and written once.  The fast kernel
+// moves 32 KB tiles through shared memory with 16-byte loads and stores on
+// both sides: the row-major side is walked in row order, the tile-major side
+// in block order, and shared memory absorbs the permutation.  When a block
+// row is shorter than 16 bytes the 16-byte vectors of the tile-major side are
+// assembled from several shared-memory rows.
+#include "tl_common.cuh"
+
+namespace tl {
+
+constexpr int kRelayoutThreads = 256;
+constexpr int kTileBytes = 32768;                       // shared-memory tile (payload)
+constexpr int kChunksPerThread = kTileBytes / 16 / kRelayoutThreads;   // 8
+constexpr int kRowPad = 16;                             // bytes of padding per shared-memory row
+
+struct RelayoutParams {
+    const uint8_t* src;
+    uint8_t* dst;
+    int64_t rows;
+    int64_t pitch;          // cols * elem_bytes
+    int64_t blocks_per_row; // cols / block_cols
+    int run_log2;           // log2(block_cols * elem_bytes): bytes of one block row
+    int br_log2;            // log2(block_rows)
+    int tile_cols_log2;     // log2(bytes of a matrix row covered by one tile)
+    int tile_rows_log2;     // log2(rows covered by one tile)
+    int64_t tiles_x;        // tiles along a row
+    int64_t tiles_total;
+    int to_tile_major;
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint8_t* p) {
+    return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ void st_stream(uint8_t* p, uint4 v) {
+    __stcs(reinterpret_cast<uint4*>(p), v);
+}
+
+// Byte offset in the tile-major buffer of byte column `cb` of matrix row `r` (Eq. 1 + Eq. 2,
+// written on bytes: a block row is `run` contiguous bytes; shifts and masks only).
+__device__ __forceinline__ int64_t tile_major_byte(const RelayoutParams& p, int64_t r, int64_t cb) {
+    int64_t Tr = r >> p.br_log2, rp = r & ((int64_t(1) << p.br_log2) - 1);
+    int64_t Tc = cb >> p.run_log2, cp = cb & ((int64_t(1) << p.run_log2) - 1);
+    return ((((Tr * p.blocks_per_row + Tc) << p.br_log2) + rp) << p.run_log2) + cp;
+}
+
+// kPiece = min(16, bytes of one block row): granularity at which the tile-major side is contiguous.
+template <int kPiece>
+__global__ void __launch_bounds__(kRelayoutThreads) relayout_kernel(const RelayoutParams p) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    const int tile_cols = 1 << p.tile_cols_log2;        // bytes
+    const int tile_rows = 1 << p.tile_rows_log2;
+    const int srow = tile_cols + kRowPad;               // shared-memory row pitch
+    const int chunks_per_row_log2 = p.tile_cols_log2 - 4;
+
+    // Block-order walk of the tile: index -> (block row, block col, row in block, byte in block row).
+    // rin = rows of one block inside the tile, cin = bytes of one block row inside the tile.
+    const int rin_log2 = min(p.tile_rows_log2, p.br_log2);
+    const int cin_log2 = min(p.tile_cols_log2, p.run_log2);
+    const int nbc_log2 = p.tile_cols_log2 - cin_log2;   // block columns in the tile
+
+    for (int64_t tile = blockIdx.x; tile < p.tiles_total; tile += gridDim.x) {
+        const int64_t row0 = (tile / p.tiles_x) << p.tile_rows_log2;
+        const int64_t cb0 = (tile % p.tiles_x) << p.tile_cols_log2;
+
+        uint4 v[kChunksPerThread];
+        // ---- phase 1: global -> registers (all loads in flight before any use)
+#pragma unroll
+        for (int i = 0; i < kChunksPerThread; ++i) {
+            const int idx = i * kRelayoutThreads + threadIdx.x;
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (p.to_tile_major) {
+                const int r = idx >> chunks_per_row_log2;
+                const int cb = (idx & ((1 << chunks_per_row_log2) - 1)) << 4;
+                if (row0 + r < p.rows && cb0 + cb < p.pitch)
+                    v[i] = ld_stream(p.src + (row0 + r) * p.pitch + cb0 + cb);
+            } else if (kPiece == 16) {
+                // 16-byte chunk of one block row
+                const int c16 = idx & ((1 << (cin_log2 - 4)) - 1);
+                const int rp = (idx >> (cin_log2 - 4)) & ((1 << rin_log2) - 1);
+                const int bcol = (idx >> (cin_log2 - 4 + rin_log2)) & ((1 << nbc_log2) - 1);
+                const int brow = idx >> (cin_log2 - 4 + rin_log2 + nbc_log2);
+                const int r = (brow << rin_log2) + rp;
+                const int cb = (bcol << cin_log2) + (c16 << 4);
+                if (row0 + r < p.rows && cb0 + cb < p.pitch)
+                    v[i] = ld_stream(p.src + tile_major_byte(p, row0 + r, cb0 + cb));
+            } else {
+                // a 16-byte vector of the tile-major side holds 16/kPiece consecutive block rows
+                constexpr int kRowsPerVec = 16 / kPiece;
+                const int vr = idx & ((1 << rin_log2) / kRowsPerVec - 1);
+                const int bcol = (idx / ((1 << rin_log2) / kRowsPerVec)) & ((1 << nbc_log2) - 1);
+                const int brow = idx / ((1 << rin_log2) / kRowsPerVec) >> nbc_log2;
+                const int r = (brow << rin_log2) + vr * kRowsPerVec;
+                const int cb = bcol << cin_log2;
+                if (row0 + r < p.rows && cb0 + cb < p.pitch)
+                    v[i] = ld_stream(p.src + tile_major_byte(p, row0 + r, cb0 + cb));
+            }
+        }
+        // ---- registers -> shared memory, always as the row-major image of the tile
+#pragma unroll
+        for (int i = 0; i < kChunksPerThread; ++i) {
+            const int idx = i * kRelayoutThreads + threadIdx.x;
+            if (p.to_tile_major) {
+                const int r = idx >> chunks_per_row_log2;
+                const int cb = (idx & ((1 << chunks_per_row_log2) - 1)) << 4;
+                *reinterpret_cast<uint4*>(smem + r * srow + cb) = v[i];
+            } else if (kPiece == 16) {
+                const int c16 = idx & ((1 << (cin_log2 - 4)) - 1);
+                const int rp = (idx >> (cin_log2 - 4)) & ((1 << rin_log2) - 1);
+                const int bcol = (idx >> (cin_log2 - 4 + rin_log2)) & ((1 << nbc_log2) - 1);
+                const int brow = idx >> (cin_log2 - 4 + rin_log2 + nbc_log2);
+                const int r = (brow << rin_log2) + rp;
+                const int cb = (bcol << cin_log2) + (c16 << 4);
+                *reinterpret_cast<uint4*>(smem + r * srow + cb) = v[i];
+            } else {
+                constexpr int kRowsPerVec = 16 / kPiece;
+                const int vr = idx & ((1 << rin_log2) / kRowsPerVec - 1);
+                const int bcol = (idx / ((1 << rin_log2) / kRowsPerVec)) & ((1 << nbc_log2) - 1);
+                const int brow = idx / ((1 << rin_log2) / kRowsPerVec) >> nbc_log2;
+                const int r = (brow << rin_log2) + vr * kRowsPerVec;
+                const int cb = bcol << cin_log2;
+                const uint8_t* bytes = reinterpret_cast<const uint8_t*>(&v[i]);
+#pragma unroll
+                for (int q = 0; q < kRowsPerVec; ++q)
+#pragma unroll
+                    for (int b = 0; b < kPiece; ++b) smem[(r + q) * srow + cb + b] = bytes[q * kPiece + b];
+            }
+        }
+        __syncthreads();
+        // ---- phase 2: shared memory -> global in the order of the destination
+#pragma unroll
+        for (int i = 0; i < kChunksPerThread; ++i) {
+            const int idx = i * kRelayoutThreads + threadIdx.x;
+            if (!p.to_tile_major) {
+                const int r = idx >> chunks_per_row_log2;
+                const int cb = (idx & ((1 << chunks_per_row_log2) - 1)) << 4;
+                if (row0 + r < p.rows && cb0 + cb < p.pitch)
+                    st_stream(p.dst + (row0 + r) * p.pitch + cb0 + cb,
+                              *reinterpret_cast<const uint4*>(smem + r * srow + cb));
+            } else if (kPiece == 16) {
+                const int c16 = idx & ((1 << (cin_log2 - 4)) - 1);
+                const int rp = (idx >> (cin_log2 - 4)) & ((1 << rin_log2) - 1);
+                const int bcol = (idx >> (cin_log2 - 4 + rin_log2)) & ((1 << nbc_log2) - 1);
+                const int brow = idx >> (cin_log2 - 4 + rin_log2 + nbc_log2);
+                const int r = (brow << rin_log2) + rp;
+                const int cb = (bcol << cin_log2) + (c16 << 4);
+                if (row0 + r < p.rows && cb0 + cb < p.pitch)
+                    st_stream(p.dst + tile_major_byte(p, row0 + r, cb0 + cb),
+                              *reinterpret_cast<const uint4*>(smem + r * srow + cb));
+            } else {
+                constexpr int kRowsPerVec = 16 / kPiece;
+                const int vr = idx & ((1 << rin_log2) / kRowsPerVec - 1);
+                const int bcol = (idx / ((1 << rin_log2) / kRowsPerVec)) & ((1 << nbc_log2) - 1);
+                const int brow = idx / ((1 << rin_log2) / kRowsPerVec) >> nbc_log2;
+                const int r = (brow << rin_log2) + vr * kRowsPerVec;
+                const int cb = bcol << cin_log2;
+                if (row0 + r < p.rows && cb0 + cb < p.pitch) {
+                    uint4 out;
+                    uint8_t* bytes = reinterpret_cast<uint8_t*>(&out);
+#pragma unroll
+                    for (int q = 0; q < kRowsPerVec; ++q)
+#pragma unroll
+                        for (int b = 0; b < kPiece; ++b) bytes[q * kPiece + b] = smem[(r + q) * srow + cb + b];
+                    st_stream(p.dst + tile_major_byte(p, row0 + r, cb0 + cb), out);
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Element-wise fallback for pitches or pointers that are not 16-byte aligned, and for G < 16.
+__global__ void relayout_elementwise_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
+                                            int64_t rows, int64_t cols, int s, int br, int bc, int to_tile_major) {
+    const int64_t total = rows * cols;
+    const int64_t blocks_per_row = cols / bc;
+    for (int64_t e = blockIdx.x * int64_t(blockDim.x) + threadIdx.x; e < total;
+         e += int64_t(gridDim.x) * blockDim.x) {
+        // e walks the tile-major buffer in element order
+        const int64_t blk = e / (int64_t(br) * bc), in = e % (int64_t(br) * bc);
+        const int64_t r = (blk / blocks_per_row) * br + in / bc;
+        const int64_t c = (blk % blocks_per_row) * bc + in % bc;
+        const int64_t row_off = (r * cols + c) * s, tile_off = e * s;
+        for (int b = 0; b < s; ++b) {
+            if (to_tile_major) dst[tile_off + b] = src[row_off + b];
+            else dst[row_off + b] = src[tile_off + b];
+        }
+    }
+}
+
+static int ilog2(int64_t x) {
+    int l = 0;
+    while ((int64_t(1) << l) < x) ++l;
+    return l;
+}
+
+int relayout_launch(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int s, int64_t G, int br, int bc,
+                    int direction, cudaStream_t stream) {
+    if (rows < 0 || cols < 0) return TL_ERR_INVALID_ARG;
+    if (s != 1 && s != 2 && s != 4) return TL_ERR_INVALID_ARG;
+    if (br <= 0 || bc <= 0 || int64_t(br) * bc * s != G) return TL_ERR_INVALID_ARG;
+    if (direction != TL_TO_TILE_MAJOR && direction != TL_TO_ROW_MAJOR) return TL_ERR_INVALID_ARG;
+    if (!is_pow2(br) || !is_pow2(bc)) return TL_ERR_UNSUPPORTED;
+    if (rows % br != 0 || cols % bc != 0) return TL_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return TL_OK;
+    if (!d_src || !d_dst) return TL_ERR_INVALID_ARG;
+    const int64_t bytes = rows * cols * s;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(d_src), b = reinterpret_cast<uintptr_t>(d_dst);
+    if (a < b + bytes && b < a + bytes) return TL_ERR_INVALID_ARG;      // overlap
+    if (int rc = ensure_device_info()) return rc;
+    const int sms = state().sm_count;
+
+    const int64_t pitch = cols * s;
+    const int64_t run = int64_t(bc) * s;
+    const bool fast = (pitch % 16 == 0) && (a % 16 == 0) && (b % 16 == 0) && G >= 16 && rows < (int64_t(1) << 40);
+    if (!fast) {
+        const int64_t total = rows * cols;
+        const int grid = int(total / 256 + 1 < int64_t(sms) * 16 ? total / 256 + 1 : int64_t(sms) * 16);
+        relayout_elementwise_kernel<<<grid, 256, 0, stream>>>(static_cast<const uint8_t*>(d_src),
+                                                              static_cast<uint8_t*>(d_dst), rows, cols, s, br, bc,
+                                                              direction == TL_TO_TILE_MAJOR);
+        return check_cuda(cudaGetLastError());
+    }
+
+    RelayoutParams p;
+    p.src = static_cast<const uint8_t*>(d_src);
+    p.dst = static_cast<uint8_t*>(d_dst);
+    p.rows = rows;
+    p.pitch = pitch;
+    p.blocks_per_row = cols / bc;
+    p.run_log2 = ilog2(run);
+    p.br_log2 = ilog2(br);
+    // Tile: as wide as one block row, but between 1 KB and 2 KB of a matrix row so that the
+    // row-major side moves long contiguous strips; rows fill the rest of the 32 KB.
+    int64_t tile_cols = run < 1024 ? 1024 : (run > 2048 ? 2048 : run);
+    int64_t tile_rows = kTileBytes / tile_cols;
+    // A 16-byte vector of the tile-major side needs 16/run block rows of the same block in the tile.
+    const int piece = run >= 16 ? 16 : int(run);
+    p.tile_cols_log2 = ilog2(tile_cols);
+    p.tile_rows_log2 = ilog2(tile_rows);
+    p.tiles_x = ceil_div(pitch, tile_cols);
+    p.tiles_total = p.tiles_x * ceil_div(rows, tile_rows);
+    p.to_tile_major = direction == TL_TO_TILE_MAJOR;
+
+    const size_t smem = size_t(tile_rows) * (tile_cols + kRowPad);
+    const int64_t max_grid = int64_t(sms) * 4;
+    const int grid = int(p.tiles_total < max_grid ? p.tiles_total : max_grid);
+    cudaError_t err = cudaSuccess;
+#define TL_LAUNCH_RELAYOUT(PIECE)                                                                              \
+    err = cudaFuncSetAttribute(relayout_kernel<PIECE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)); \
+    if (err == cudaSuccess) relayout_kernel<PIECE><<<grid, kRelayoutThreads, smem, stream>>>(p);
+    switch (piece) {
+        case 16: TL_LAUNCH_RELAYOUT(16) break;
+        case 8: TL_LAUNCH_RELAYOUT(8) break;
+        case 4: TL_LAUNCH_RELAYOUT(4) break;
+        case 2: TL_LAUNCH_RELAYOUT(2) break;
+        default: TL_LAUNCH_RELAYOUT(1) break;
+    }
+#undef TL_LAUNCH_RELAYOUT
+    if (err != cudaSuccess) return check_cuda(err);
+    return check_cuda(cudaGetLastError());
+}
+
+}  // namespace tl
+
+extern "C" {
+
+int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes, int64_t G,
+                   int block_rows, int block_cols, int direction, void* cuda_stream) {
+    return tl::relayout_launch(d_src, d_dst, rows, cols, elem_bytes, G, block_rows, block_cols, direction,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
+int tl_relayout(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes, int64_t G,
+                int block_rows, int block_cols, int direction) {
+    return tl::relayout_launch(d_src, d_dst, rows, cols, elem_bytes, G, block_rows, block_cols, direction,
+                               tl::state().stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,259 @@
+"""tcgen05 GEMM (dense, decode/stream-K, grouped) vs the oracle (GPU).
+
+Tolerance (from the arithmetic): inputs are exact in fp64, the kernel accumulates in fp32, so
+|C - C_ref| <= 1e-3 * sum_k |A_ik B_kj| with a wide margin; integer-valued and one-hot inputs
+must come out bit-exact in every variant because every partial sum is an exact fp32 integer.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as tlo
+from paper_2607_04031_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+ROW, TILE = tlo.ROW_MAJOR, tlo.TILE_MAJOR
+
+
+def _oracle_full(A, B_dev_buf, layout, br, bc, M, N, K):
+    return tlo.matmul(inputs.bits(A), inputs.bits(B_dev_buf.reshape(-1)), layout, br, bc, M, N, K)
+
+
+def test_config1_tiny_tile_major_and_row_major():
+    from gpu_util import DEV, check_against_oracle, run_gemm, tile_major_on_device
+    M, N, K, br, bc = 16, 512, 512, 16, 128
+    A = inputs.bf16_normal((M, K), 1.0, seed=101)
+    B = inputs.bf16_uniform((K, N), -1.0, 1.0, seed=102)
+    Bt = tile_major_on_device(B, K, N, br, bc)
+    C = run_gemm(A, Bt, M, N, K, br, bc)
+    check_against_oracle(C, A, Bt, TILE, br, bc, M, N, K)
+    C_row = run_gemm(A, B.to(DEV), M, N, K, 0, 0)
+    check_against_oracle(C_row, A, B.to(DEV), ROW, 0, 0, M, N, K)
+    # same kernel, same K order: the two layouts give the same bits
+    assert torch.equal(C, C_row)
+
+
+@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0)])
+@pytest.mark.parametrize("cta", [(0, 0, 0), (64, 128, 64), (128, 256, 64), (32, 128, 128), (128, 256, 128)])
+def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
+    # No arithmetic at all: catches any error in the tensor-map view, the swizzle or the descriptors.
+    from gpu_util import DEV, run_gemm, tile_major_on_device
+    M, N, K = 40, 1024, 512
+    A, ks = inputs.one_hot_rows(M, K, seed=7)
+    B = inputs.bf16_normal((K, N), 0.02, seed=8)
+    Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
+    C = run_gemm(A, Bd, M, N, K, br, bc, cta)
+    assert torch.equal(C.cpu(), B.float()[ks])
+
+
+SHAPES = [  # M, N, K
+    (1, 512, 512), (8, 1024, 2048), (33, 640, 1024), (64, 256, 8192), (100, 384, 320),
+    (300, 1152, 576), (257, 128, 64), (16, 8192, 1024),
+]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (0, 0)])
+def test_integer_inputs_are_bit_exact(M, N, K, br, bc):
+    from gpu_util import DEV, run_gemm, tile_major_on_device
+    A = inputs.bf16_integers((M, K), -8, 8, seed=M + N)
+    B = inputs.bf16_integers((K, N), -8, 8, seed=K)
+    Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
+    layout = TILE if br else ROW
+    C = run_gemm(A, Bd, M, N, K, br, bc)
+    ref, _ = _oracle_full(A, Bd, layout, br, bc, M, N, K) if M * N * K <= 2 ** 28 else (None, None)
+    if ref is None:
+        ii, jj = np.divmod(np.arange(0, M * N, max(1, M * N // 20000)), N)
+        ref_s, _ = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), layout, br, bc, M, N, K, ii, jj)
+        assert np.array_equal(C.cpu().numpy()[ii, jj].astype(np.float64), ref_s)
+    else:
+        assert np.array_equal(C.cpu().numpy().astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("cta", [(16, 128, 64), (32, 128, 64), (64, 128, 128), (128, 128, 64), (256, 128, 64),
+                                 (128, 256, 64), (64, 256, 128), (256, 128, 128)])
+def test_every_cta_tile_random_data(cta):
+    from gpu_util import check_against_oracle, run_gemm, tile_major_on_device
+    M, N, K, br, bc = 200, 768, 1024, 16, 128
+    A = inputs.bf16_normal((M, K), 1.0, seed=11)
+    B = inputs.bf16_normal((K, N), 0.02, seed=12)
+    Bt = tile_major_on_device(B, K, N, br, bc)
+    C = run_gemm(A, Bt, M, N, K, br, bc, cta)
+    check_against_oracle(C, A, Bt, TILE, br, bc, M, N, K)
+
+
+def test_all_ones_B_gives_row_sums():
+    from gpu_util import DEV, run_gemm, tile_major_on_device
+    M, N, K = 8, 256, 4096
+    A = inputs.bf16_integers((M, K), -3, 3, seed=5)
+    B = torch.ones((K, N), dtype=torch.bfloat16)
+    C = run_gemm(A, tile_major_on_device(B, K, N, 16, 128), M, N, K, 16, 128)
+    want = A.float().sum(dim=1, keepdim=True).expand(M, N)
+    assert torch.equal(C.cpu(), want)
+
+
+def test_results_are_reproducible_run_to_run():
+    from gpu_util import run_gemm, tile_major_on_device
+    M, N, K = 32, 1024, 8192          # stream-K with partial tiles
+    A = inputs.bf16_normal((M, K), 1.0, seed=1)
+    Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=2), K, N, 16, 128)
+    C0 = run_gemm(A, Bt, M, N, K, 16, 128)
+    for _ in range(5):
+        assert torch.equal(run_gemm(A, Bt, M, N, K, 16, 128), C0)
+
+
+@pytest.mark.parametrize("name,K,N", inputs.LLAMA70B_PROJ)
+@pytest.mark.parametrize("M", inputs.LLAMA_DECODE_M)
+def test_llama_decode_full_size_sampled(name, K, N, M):
+    # Same sizes and launch configuration (library heuristic) as the benchmark; 600 sampled outputs.
+    from gpu_util import DEV, check_against_oracle, run_gemm, sample_indices
+    from gpu_util import tl
+    A = inputs.bf16_normal((M, K), 1.0, seed=31 + M)
+    B = inputs.bf16_normal((K, N), 0.02, seed=(K % 997) + (N % 991), device=DEV)
+    Bt = torch.empty_like(B)
+    tl.relayout(B, Bt, K, N, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    C = run_gemm(A, Bt, M, N, K, 16, 128)
+    check_against_oracle(C, A, Bt, TILE, 16, 128, M, N, K, idx=sample_indices(M, N, 600, seed=M))
+    # property that holds at any size: the row-major comparator gives the same bits
+    assert torch.equal(run_gemm(A, B, M, N, K, 0, 0), C)
+
+
+def test_llama_prefill_full_size_sampled():
+    from gpu_util import DEV, check_against_oracle, run_gemm, sample_indices, tl
+    M, K, N = inputs.LLAMA_PREFILL_M, 8192, 10240
+    A = inputs.bf16_normal((M, K), 1.0, seed=41, device=DEV)
+    B = inputs.bf16_normal((K, N), 0.02, seed=42, device=DEV)
+    Bt = torch.empty_like(B)
+    tl.relayout(B, Bt, K, N, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    C = run_gemm(A, Bt, M, N, K, 16, 128)
+    ii, jj = sample_indices(M, N, 3000, seed=4)
+    # plus one full row and one full column through every tile
+    ii = np.concatenate([ii, np.full(N, 1234), np.arange(M)])
+    jj = np.concatenate([jj, np.arange(N), np.full(M, 4321)])
+    check_against_oracle(C, A.cpu(), Bt, TILE, 16, 128, M, N, K, idx=(ii, jj))
+    assert torch.isfinite(C).all()
+
+
+def _grouped_case(E, tokens, topk, K, N, br, bc, seed, cta=(0, 0, 0), integer=False):
+    from gpu_util import DEV, tl
+    offsets, counts, _ = inputs.zipf_topk_routing(tokens, E, topk, 1.1, seed=seed)
+    rows = int(offsets[-1])
+    gen = (lambda shape, s: inputs.bf16_integers(shape, -8, 8, seed=s)) if integer else \
+        (lambda shape, s: inputs.bf16_normal(shape, 1.0 if len(shape) == 2 else 0.02, seed=s))
+    A = gen((rows, K), seed + 1)
+    B = gen((E, K, N), seed + 2)
+    Bd = B.to(DEV)
+    if br:
+        Bt = torch.empty_like(Bd)
+        # experts are separate matrices laid end to end: relayout each (equal to one stacked E*K x N relayout)
+        tl.relayout(Bd, Bt, E * K, N, 2, br * bc * 2, br, bc, tl.TO_TILE_MAJOR)
+        Bd = Bt
+    C = torch.full((rows, N), float("nan"), dtype=torch.float32, device=DEV)
+    tl.gemm_grouped(A.to(DEV), Bd, C, torch.from_numpy(offsets).to(DEV), E, rows, N, K,
+                    br * bc * 2, br, bc, cta)
+    tl.device_status()
+    return offsets, counts, A, Bd, C
+
+
+def _check_grouped(offsets, A, Bd, C, E, K, N, br, bc, samples_per_expert, exact):
+    layout = TILE if br else ROW
+    Ch = C.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(Ch))
+    rng = np.random.default_rng(0)
+    worst = 0.0
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 == r0:
+            continue
+        Me = r1 - r0
+        Be = inputs.bits(Bd[e].reshape(-1))
+        Ae = inputs.bits(A[r0:r1])
+        ii = rng.integers(0, Me, samples_per_expert)
+        jj = rng.integers(0, N, samples_per_expert)
+        ii[:2] = [0, Me - 1]
+        jj[:2] = [0, N - 1]
+        ref, S = tlo.matmul_at(Ae, Be, layout, br, bc, Me, N, K, ii, jj)
+        got = Ch[r0 + ii, jj]
+        if exact:
+            assert np.array_equal(got, ref), f"expert {e}"
+        else:
+            assert np.all(np.abs(got - ref) <= 1e-3 * S), f"expert {e}"
+            worst = max(worst, float(np.max(np.abs(got - ref) / np.maximum(S, 1e-300))))
+    assert worst <= 1e-4
+
+
+@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (0, 0)])
+def test_grouped_small_integer_exact(br, bc):
+    E, K, N = 8, 256, 384
+    offsets, counts, A, Bd, C = _grouped_case(E, 40, 3, K, N, br, bc, seed=3, integer=True)
+    _check_grouped(offsets, A, Bd, C, E, K, N, br, bc, samples_per_expert=400, exact=True)
+
+
+def test_grouped_with_empty_experts_and_small_tile_cap():
+    from gpu_util import DEV, tl
+    E, K, N = 6, 128, 256
+    offsets = np.array([0, 0, 70, 70, 71, 200, 200], dtype=np.int32)
+    A = inputs.bf16_integers((200, K), -8, 8, seed=1)
+    B = inputs.bf16_integers((E, K, N), -8, 8, seed=2)
+    Bt = torch.empty((E, K, N), dtype=torch.bfloat16, device=DEV)
+    tl.relayout(B.to(DEV), Bt, E * K, N, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    C = torch.full((200, N), float("nan"), dtype=torch.float32, device=DEV)
+    tl.gemm_grouped(A.to(DEV), Bt, C, torch.from_numpy(offsets).to(DEV), E, 200, N, K, 4096, 16, 128, (32, 128, 64))
+    tl.device_status()
+    _check_grouped(offsets, A, Bt, C, E, K, N, 16, 128, samples_per_expert=300, exact=True)
+
+
+@pytest.mark.parametrize("name,K,N", inputs.QWEN_MOE_PROJ)
+def test_qwen_moe_full_size_sampled(name, K, N):
+    q = inputs.QWEN_MOE
+    offsets, counts, A, Bd, C = _grouped_case(q["experts"], q["tokens"], q["topk"], K, N, 16, 128, seed=0)
+    assert int(offsets[-1]) == q["tokens"] * q["topk"]
+    _check_grouped(offsets, A, Bd, C, q["experts"], K, N, 16, 128, samples_per_expert=48, exact=False)
+
+
+@pytest.mark.parametrize("name,K,N", inputs.QWEN_ATTN_PROJ)
+def test_qwen_attention_projections(name, K, N):
+    from gpu_util import check_against_oracle, run_gemm, sample_indices, tile_major_on_device
+    M = 256
+    A = inputs.bf16_normal((M, K), 1.0, seed=51)
+    Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=52), K, N, 16, 128)
+    C = run_gemm(A, Bt, M, N, K, 16, 128)
+    check_against_oracle(C, A, Bt, TILE, 16, 128, M, N, K, idx=sample_indices(M, N, 4000, seed=5))
+
+
+def test_host_buffer_entry_point():
+    from gpu_util import DEV, tl
+    M, N, K = 8, 512, 1024
+    A = inputs.bf16_integers((M, K), -8, 8, seed=1).pin_memory()
+    B = inputs.bf16_integers((K, N), -8, 8, seed=2).pin_memory()
+    C = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    scratch = torch.empty(tl.gemm_host_scratch_bytes(M, N, K), dtype=torch.uint8, device=DEV)
+    tl.gemm_host(A, B, C, M, N, K, scratch)
+    ref, _ = tlo.matmul(inputs.bits(A), inputs.bits(B), ROW, 0, 0, M, N, K)
+    assert np.array_equal(C.numpy().astype(np.float64), ref)
+
+
+def test_caller_workspace_and_errors():
+    from gpu_util import DEV, run_gemm, tile_major_on_device, tl
+    M, N, K = 16, 512, 4096
+    A = inputs.bf16_integers((M, K), -8, 8, seed=1)
+    Bt = tile_major_on_device(inputs.bf16_integers((K, N), -8, 8, seed=2), K, N, 16, 128)
+    want = run_gemm(A, Bt, M, N, K, 16, 128)
+    need = tl.gemm_workspace_bytes(M, N, K)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    tl.set_workspace(ws)
+    try:
+        assert torch.equal(run_gemm(A, Bt, M, N, K, 16, 128), want)
+        small = torch.empty(1024, dtype=torch.uint8, device=DEV)
+        tl.set_workspace(small)
+        with pytest.raises(tl.TileLensError) as e:
+            run_gemm(A, Bt, M, N, K, 16, 128)
+        assert e.value.status == 6
+    finally:
+        tl.set_workspace(None)
+    with pytest.raises(tl.TileLensError) as e:
+        run_gemm(A, Bt, M, N, K, 16, 128, cta=(48, 128, 64))
+    assert e.value.status == 2
+    C = torch.zeros((0, N), dtype=torch.float32, device=DEV)
+    tl.gemm(A.to(DEV)[:0], Bt, C, 0, N, K, 4096, 16, 128)          # no rows: no-op

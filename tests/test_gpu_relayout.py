@@ -1,0 +1,88 @@
+"""Relayout kernel vs the oracle: bit-exact (GPU)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as tlo
+from paper_2607_04031_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+CASES = [  # rows, cols, s, br, bc
+    (512, 512, 2, 16, 128),        # config 1
+    (512, 512, 2, 32, 64),
+    (512, 512, 2, 8, 256),
+    (512, 512, 2, 1, 2048 // 4),   # one-row blocks: identity
+    (256, 1024, 1, 64, 64),        # FP8 64 x 64 (Figure 1c)
+    (256, 1024, 4, 8, 128),
+    (96, 640, 2, 16, 16),          # 32-byte runs
+    (64, 256, 2, 8, 2),            # 4-byte runs: vectors gathered from 4 block rows
+    (64, 256, 2, 16, 1),           # 2-byte runs
+    (64, 256, 1, 32, 1),           # 1-byte runs
+    (128, 64, 4, 32, 2),           # 8-byte runs
+    (48, 40, 1, 4, 8),             # 40-byte pitch: element-wise fallback
+    (24, 20, 2, 4, 2),             # G = 16, pitch 40 B
+    (16, 8, 2, 2, 2),              # G = 8 < 16: element-wise
+    (1056, 2176, 2, 32, 64),       # tiles overhang both edges (1056 = 33*32, 2176 = 17*128)
+    (32, 8192, 2, 1, 2048),        # block row of 4 KB, wider than a tile
+    (64, 16384, 2, 32, 8192 // 2 // 1),  # 16 KB rows: bc = 4096 -> G = 256 KB
+    (8192, 16, 1, 4096, 1),        # column-major-like: 4096 x 1 blocks
+]
+
+
+@pytest.mark.parametrize("rows,cols,s,br,bc", CASES)
+def test_both_directions_match_oracle(rows, cols, s, br, bc):
+    from gpu_util import DEV, dev_bytes, tl
+    G = br * bc * s
+    src = inputs.random_bytes(rows * cols * s, seed=rows + 7 * cols + s)
+    want = tlo.relayout(src, rows, cols, s, br, bc, tlo.TO_TILE_MAJOR)
+    d_src = dev_bytes(src)
+    d_dst = torch.zeros_like(d_src)
+    tl.relayout(d_src, d_dst, rows, cols, s, G, br, bc, tl.TO_TILE_MAJOR)
+    got = d_dst.cpu().numpy()
+    assert np.array_equal(got, want)
+    d_back = torch.zeros_like(d_src)
+    tl.relayout(d_dst, d_back, rows, cols, s, G, br, bc, tl.TO_ROW_MAJOR)
+    assert np.array_equal(d_back.cpu().numpy(), src)
+    # the inverse direction on its own, from the oracle's tile-major bytes
+    d_t = dev_bytes(want)
+    d_r = torch.zeros_like(d_t)
+    tl.relayout(d_t, d_r, rows, cols, s, G, br, bc, tl.TO_ROW_MAJOR)
+    assert np.array_equal(d_r.cpu().numpy(), tlo.relayout(want, rows, cols, s, br, bc, tlo.TO_ROW_MAJOR))
+
+
+def test_unaligned_pointers_take_the_elementwise_path():
+    from gpu_util import DEV, dev_bytes, tl
+    rows, cols, s, br, bc = 64, 128, 2, 16, 64
+    src = inputs.random_bytes(rows * cols * s, seed=5)
+    buf = torch.zeros(rows * cols * s + 64, dtype=torch.uint8, device=DEV)
+    d_src = buf[2:2 + rows * cols * s]
+    d_src.copy_(torch.from_numpy(src))
+    d_dst = torch.zeros(rows * cols * s, dtype=torch.uint8, device=DEV)
+    tl.relayout(d_src, d_dst, rows, cols, s, br * bc * s, br, bc, tl.TO_TILE_MAJOR)
+    assert np.array_equal(d_dst.cpu().numpy(), tlo.relayout(src, rows, cols, s, br, bc, tlo.TO_TILE_MAJOR))
+
+
+def test_full_size_llama_weight_matches_oracle():
+    from gpu_util import DEV, tl
+    K, N, br, bc = 8192, 8192, 16, 128
+    B = inputs.bf16_normal((K, N), 0.02, seed=21, device=DEV)
+    out = torch.empty_like(B)
+    tl.relayout(B, out, K, N, 2, 4096, br, bc, tl.TO_TILE_MAJOR)
+    want = tlo.relayout(inputs.bits(B).view(np.uint8), K, N, 2, br, bc, tlo.TO_TILE_MAJOR)
+    assert np.array_equal(out.cpu().view(torch.uint8).numpy().reshape(-1), want)
+    back = torch.empty_like(B)
+    tl.relayout(out, back, K, N, 2, 4096, br, bc, tl.TO_ROW_MAJOR)
+    assert torch.equal(back, B)
+
+
+def test_errors():
+    from gpu_util import DEV, tl
+    a = torch.zeros(64 * 64 * 2, dtype=torch.uint8, device=DEV)
+    b = torch.zeros_like(a)
+    with pytest.raises(tl.TileLensError) as e:
+        tl.relayout(a, b, 64, 64, 2, 4096, 16, 64, tl.TO_TILE_MAJOR)
+    assert e.value.status == 1
+    with pytest.raises(tl.TileLensError) as e:
+        tl.relayout(a, a, 64, 64, 2, 2048, 16, 64, tl.TO_TILE_MAJOR)     # in place
+    assert e.value.status == 1
