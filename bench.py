@@ -1,0 +1,471 @@
+#!/usr/bin/env python
+"""Benchmark of the tile-major GEMM hot path on B200.
+
+One step = one pass of the whole path over the Llama-3.1-70B-shaped decode workload:
+  relayout (row-major -> tile-major, 4 KB blocks of 16 x 128 bf16) of the four projection weights,
+  then for M in {1, 8, 32} tokens the tile-major GEMM of every projection (12 GEMMs),
+  then the read-amplification count of every (projection, M) schedule (12 counts, exact integers).
+The metric is algorithmic bytes moved per second (TB/s): relayout 2*K*N*2 bytes, GEMM
+2*K*N + 2*M*K + 4*M*N bytes.  Beside it: the same GEMMs on row-major weights, the prefill
+(M = 4096, TFLOP/s) and Qwen MoE grouped legs, the end-to-end number through tl_gemm_host with
+pinned host buffers, and the CPU oracle on a bounded sample.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+N > 1 (under torchrun) runs N independent replicas: the path has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2607_04031_b200 import inputs
+
+G, BR, BC = inputs.DEFAULT_G, *inputs.DEFAULT_BLOCK
+METRIC = "tile_major_gemm_path_throughput"
+UNIT = "TB/s"
+WORKLOAD = "llama3.1-70b decode linear layers (qkv, o, gate_up, down; M in {1,8,32}), bf16 tile-major 4KB blocks 16x128"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode GEMM kernel, from the ncu
+# capture summarised in profiles/ (None until a capture exists for this kernel version).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_NOTE = None
+
+
+def gemm_bytes(M, N, K):
+    return 2 * K * N + 2 * M * K + 4 * M * N
+
+
+def relayout_bytes(N, K):
+    return 2 * K * N * 2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------ CPU oracle leg
+
+def oracle_sample(step_budget_s: float):
+    """Times the oracle, as it stands, on a bounded slab of the same workload.  Returns a dict."""
+    import oracle as tlo
+    K, N_full = 8192, 10240                      # the qkv projection
+    cores = tlo.num_threads()
+    A = {M: inputs.bf16_normal((M, K), 1.0, seed=900 + M) for M in inputs.LLAMA_DECODE_M}
+    # calibrate on 64 columns, then size the slab for the budget
+    n_cal = 128
+    Bc = inputs.bf16_normal((K, n_cal), 0.02, seed=901)
+    Bc_t = tlo.relayout(inputs.bits(Bc).view(np.uint8), K, n_cal, 2, BR, BC, tlo.TO_TILE_MAJOR).view(np.uint16)
+    t0 = time.perf_counter()
+    tlo.matmul(inputs.bits(A[8]), Bc_t, tlo.TILE_MAJOR, BR, BC, 8, n_cal, K)
+    rate = 8 * n_cal * K / (time.perf_counter() - t0)          # MAC/s
+    macs_per_col = sum(inputs.LLAMA_DECODE_M) * K
+    n_cols = int(step_budget_s * 0.8 * rate / macs_per_col) // BC * BC
+    n_cols = max(BC, min(N_full, n_cols))
+    B = inputs.bf16_normal((K, n_cols), 0.02, seed=902)
+    Bb = inputs.bits(B)
+    t0 = time.perf_counter()
+    Bt = tlo.relayout(Bb.view(np.uint8), K, n_cols, 2, BR, BC, tlo.TO_TILE_MAJOR).view(np.uint16)
+    for M in inputs.LLAMA_DECODE_M:
+        tlo.matmul(inputs.bits(A[M]), Bt, tlo.TILE_MAJOR, BR, BC, M, n_cols, K)
+    for M in inputs.LLAMA_DECODE_M:
+        tlo.read_amp(M, n_cols, K, 16 if M <= 16 else 32, 128, 64, tlo.TILE_MAJOR, G, BR, BC, 2)
+    dt = time.perf_counter() - t0
+    nbytes = relayout_bytes(n_cols, K) + sum(gemm_bytes(M, n_cols, K) for M in inputs.LLAMA_DECODE_M)
+    return {"value": nbytes / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
+            "sample": f"qkv projection K={K}, first {n_cols} of {N_full} columns: oracle relayout + fp64 matmul "
+                      f"for M in (1,8,32) + brute-force read-amp count"}
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, one bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle as tlo
+    tlo.build()
+    per_step = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(per_step)
+    vals = [oracle_sample(per_step) for _ in range(args.steps)]
+    secs = sum(v["seconds"] for v in vals)
+    value = statistics.mean(v["value"] for v in vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / max(1, args.steps) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": "n/a (host)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle",
+                         "sample": vals[-1]["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------ GPU legs
+
+class EventTimer:
+    """CUDA-event pairs on the current stream, grouped by label; read after a synchronize."""
+
+    def __init__(self):
+        self.pairs = {}
+
+    def time(self, label, fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        self.pairs.setdefault(label, []).append((a, b))
+
+    def totals_ms(self):
+        return {k: (sum(a.elapsed_time(b) for a, b in v), len(v)) for k, v in self.pairs.items()}
+
+
+def run_ours(args):
+    from paper_2607_04031_b200 import binding as tl
+    from paper_2607_04031_b200 import build as tl_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        tl_build.build()
+    if world > 1:
+        dist.barrier()
+    tl.lib()
+    peaks = measured_peaks()
+    stream = torch.cuda.current_stream()
+
+    # ---- resident inputs (seeded, synthetic)
+    W_row, W_tile, A_dec, C_dec = {}, {}, {}, {}
+    for i, (name, K, N) in enumerate(inputs.LLAMA70B_PROJ):
+        W_row[name] = inputs.bf16_normal((K, N), 0.02, seed=100 + i + 10 * rank, device=str(dev))
+        W_tile[name] = torch.empty_like(W_row[name])
+        for M in inputs.LLAMA_DECODE_M:
+            A_dec[name, M] = inputs.bf16_normal((M, K), 1.0, seed=200 + 10 * i + M, device=str(dev))
+            C_dec[name, M] = torch.empty((M, N), dtype=torch.float32, device=dev)
+    read_amp_out = {}
+
+    def one_step(timer: EventTimer | None):
+        def run(label, fn):
+            if timer:
+                timer.time(label, fn)
+            else:
+                fn()
+        for name, K, N in inputs.LLAMA70B_PROJ:
+            run("relayout", lambda: tl.relayout(W_row[name], W_tile[name], K, N, 2, G, BR, BC, tl.TO_TILE_MAJOR))
+        for M in inputs.LLAMA_DECODE_M:
+            for name, K, N in inputs.LLAMA70B_PROJ:
+                run("gemm_decode", lambda: tl.gemm(A_dec[name, M], W_tile[name], C_dec[name, M], M, N, K, G, BR, BC))
+        for M in inputs.LLAMA_DECODE_M:
+            for name, K, N in inputs.LLAMA70B_PROJ:
+                cta = (16 if M <= 16 else 32, 128, 64)
+                read_amp_out[name, M] = (
+                    tl.read_amp(M, N, K, cta, tl.LAYOUT_TILE_MAJOR, G, BR, BC, 2),
+                    tl.read_amp(M, N, K, cta, tl.LAYOUT_ROW_MAJOR, G, 0, 0, 2))
+
+    step_bytes = sum(relayout_bytes(N, K) for _, K, N in inputs.LLAMA70B_PROJ) + \
+        sum(gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
+    gemm_step_bytes = sum(gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
+    launches_per_step = 4 + 12 + 24
+
+    tl.set_stream(stream)
+    for _ in range(max(3, args.warmup)):
+        one_step(None)
+    tl.device_status()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    timer = EventTimer()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        one_step(timer)
+    ev1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    tl.device_status()
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    value = world * args.steps * step_bytes / (total_ms * 1e-3) / 1e12
+    kernel_ms = timer.totals_ms()
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (decode GEMM), live CUDA-event durations inside the timed region
+    g_ms, g_n = kernel_ms["gemm_decode"]
+    r_ms, r_n = kernel_ms["relayout"]
+    gemm_gbs = args.steps * gemm_step_bytes / (g_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "gemm_kernel<64,1> (stream-K decode)", "achieved": gemm_gbs,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
+                "peak_source": f"of {peaks['source']}", "frac_of_nominal_8TBs": gemm_gbs / 8000.0,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "traffic_note": NCU_TRAFFIC_NOTE,
+                "algorithmic_bytes_per_launch_avg": gemm_step_bytes / 12,
+                "avg_launch_us": g_ms / g_n * 1e3}
+    relayout_gbs = args.steps * sum(relayout_bytes(N, K) for _, K, N in inputs.LLAMA70B_PROJ) / (r_ms * 1e-3) / 1e9
+
+    extra = {}
+    # ---- per-shape decode table, tile-major next to row-major through the same kernel (cold L2: weights rotate)
+    def time_calls(calls, reps):
+        for c in calls:
+            c()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            for c in calls:
+                c()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    per_shape = []
+    for M in inputs.LLAMA_DECODE_M:
+        for layout in ("tile", "row"):
+            # one pass over all four weights per repetition: 1.7 GB between two uses of the same weight
+            evs = []
+            for rep in range(6):
+                for name, K, N in inputs.LLAMA70B_PROJ:
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    if layout == "tile":
+                        tl.gemm(A_dec[name, M], W_tile[name], C_dec[name, M], M, N, K, G, BR, BC)
+                    else:
+                        tl.gemm(A_dec[name, M], W_row[name], C_dec[name, M], M, N, K, 0, 0, 0)
+                    b.record()
+                    if rep > 0:
+                        evs.append((name, K, N, a, b))
+            torch.cuda.synchronize()
+            for name, K, N in inputs.LLAMA70B_PROJ:
+                ts = [a.elapsed_time(b) for (n_, _, _, a, b) in evs if n_ == name]
+                med = statistics.median(ts)
+                per_shape.append({"proj": name, "M": M, "layout": layout, "us": med * 1e3,
+                                  "GBps": gemm_bytes(M, N, K) / (med * 1e-3) / 1e9})
+    extra["decode_per_shape"] = per_shape
+    tile_t = sum(x["us"] for x in per_shape if x["layout"] == "tile")
+    row_t = sum(x["us"] for x in per_shape if x["layout"] == "row")
+    extra["tile_vs_row_time_ratio_decode"] = tile_t / row_t
+
+    # ---- prefill leg (M = 4096): tensor-core bound
+    Mp = inputs.LLAMA_PREFILL_M
+    prefill = []
+    for layout in ("tile", "row"):
+        for name, K, N in inputs.LLAMA70B_PROJ:
+            Ap = inputs.bf16_normal((Mp, K), 1.0, seed=300, device=str(dev))
+            Cp = torch.empty((Mp, N), dtype=torch.float32, device=dev)
+            if layout == "tile":
+                call = lambda: tl.gemm(Ap, W_tile[name], Cp, Mp, N, K, G, BR, BC)
+            else:
+                call = lambda: tl.gemm(Ap, W_row[name], Cp, Mp, N, K, 0, 0, 0)
+            ms = time_calls([call], 5)
+            prefill.append({"proj": name, "layout": layout, "ms": ms, "TFLOPs": 2.0 * Mp * N * K / (ms * 1e-3) / 1e12})
+            del Ap, Cp
+    pt = [x for x in prefill if x["layout"] == "tile"]
+    flops = sum(2.0 * Mp * N * K for _, K, N in inputs.LLAMA70B_PROJ)
+    tf = flops / (sum(x["ms"] for x in pt) * 1e-3) / 1e12
+    extra["prefill"] = {"per_shape": prefill, "TFLOPs_tile_major": tf,
+                        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                     "frac": tf / peaks["bf16_tflops"], "peak_source": f"of {peaks['source']} (burst)",
+                                     "frac_of_nominal_2250": tf / 2250.0},
+                        "tile_vs_row_time_ratio": sum(x["ms"] for x in pt) /
+                        sum(x["ms"] for x in prefill if x["layout"] == "row")}
+    tl.device_status()
+
+    # ---- Qwen-3-30B-A3B MoE grouped leg
+    q = inputs.QWEN_MOE
+    offsets, counts, _ = inputs.zipf_topk_routing(q["tokens"], q["experts"], q["topk"], q["zipf_alpha"], seed=0)
+    rows = int(offsets[-1])
+    d_off = torch.from_numpy(offsets).to(dev)
+    active = int((counts > 0).sum())
+    moe = []
+    for name, K, N in inputs.QWEN_MOE_PROJ:
+        # two copies of the expert weights so that consecutive launches do not hit L2 (403-805 MB each anyway)
+        Bm = inputs.bf16_normal((q["experts"], K, N), 0.02, seed=400, device=str(dev))
+        Bt = torch.empty_like(Bm)
+        tl.relayout(Bm, Bt, q["experts"] * K, N, 2, G, BR, BC, tl.TO_TILE_MAJOR)
+        Am = inputs.bf16_normal((rows, K), 1.0, seed=401, device=str(dev))
+        Cm = torch.empty((rows, N), dtype=torch.float32, device=dev)
+        for layout, buf, blk in (("tile", Bt, (BR, BC)), ("row", Bm, (0, 0))):
+            ms = time_calls([lambda: tl.gemm_grouped(Am, buf, Cm, d_off, q["experts"], rows, N, K, G, blk[0], blk[1])], 10)
+            nbytes = active * 2 * K * N + 2 * rows * K + 4 * rows * N
+            moe.append({"proj": name, "layout": layout, "us": ms * 1e3, "GBps": nbytes / (ms * 1e-3) / 1e9,
+                        "active_experts": active})
+        ra_t = tl.read_amp_grouped(offsets, N, K, (256, 256, 128), tl.LAYOUT_TILE_MAJOR, G, 32, 64, 2)
+        ra_r = tl.read_amp_grouped(offsets, N, K, (256, 256, 128), tl.LAYOUT_ROW_MAJOR, G, 0, 0, 2)
+        moe.append({"proj": name, "read_amp_128x256_weight_tile": {"tile_major_32x64": ra_t[0] / ra_t[1],
+                                                                  "row_major": ra_r[0] / ra_r[1]}})
+        del Bm, Bt, Am, Cm
+    extra["qwen_moe"] = moe
+    tl.device_status()
+
+    # ---- modelled read amplification at 4 KB (exact integers from the counter)
+    ra = {}
+    for (name, M), (t_, r_) in read_amp_out.items():
+        ra[f"{name}_M{M}"] = {"tile_major": t_[0] / t_[1], "row_major": r_[0] / r_[1],
+                              "fetched_tile": t_[0], "used": t_[1], "fetched_row": r_[0]}
+    extra["read_amp_4KB"] = ra
+
+    clocks = sampler.stop()
+
+    # ---- end to end: host buffers through tl_gemm_host (H2D of A and the row-major weight, relayout, GEMM, D2H of C)
+    e2e = None
+    try:
+        scratch = torch.empty(max(tl.gemm_host_scratch_bytes(32, N, K) for _, K, N in inputs.LLAMA70B_PROJ),
+                              dtype=torch.uint8, device=dev)
+        hW = {name: W_row[name].cpu().pin_memory() for name, _, _ in inputs.LLAMA70B_PROJ}
+        hA = {k: v.cpu().pin_memory() for k, v in A_dec.items()}
+        hC = {k: torch.empty(v.shape, dtype=torch.float32).pin_memory() for k, v in C_dec.items()}
+
+        def e2e_step():
+            for M in inputs.LLAMA_DECODE_M:
+                for name, K, N in inputs.LLAMA70B_PROJ:
+                    tl.gemm_host(hA[name, M], hW[name], hC[name, M], M, N, K, scratch, G, BR, BC)
+                    tl.read_amp(M, N, K, (16 if M <= 16 else 32, 128, 64), tl.LAYOUT_TILE_MAJOR, G, BR, BC, 2)
+        e2e_step()
+        n_e2e = max(1, min(args.steps, 3))
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record()
+        torch.cuda.synchronize()
+        e_ms = a.elapsed_time(b) / n_e2e
+        h2d = sum(2 * K * N + 2 * M * K for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
+        d2h = sum(4 * M * N for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M) + 12 * 24
+        # same byte accounting as the device-resident step: each call relayouts and multiplies once
+        e_bytes = sum(relayout_bytes(N, K) + gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ
+                      for M in inputs.LLAMA_DECODE_M)
+        e2e = {"value": world * e_bytes / (e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": n_e2e,
+               "note": "12 tl_gemm_host calls per step; every call copies A and the row-major weight from pinned host "
+                       "memory, relayouts, multiplies and copies C back"}
+        del scratch, hW
+    except Exception as exc:  # report, never hide
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+               "error": f"{type(exc).__name__}: {exc}"}
+
+    # ---- CPU oracle on a bounded sample
+    try:
+        import oracle as tlo
+        tlo.build()
+        cpu = oracle_sample(15.0)
+        cpu.pop("seconds", None)
+    except Exception as exc:
+        cpu = {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": f"failed: {exc}"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "G": G, "block": [BR, BC], "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2: 1.7 GB of weights stream between two uses of the same weight"},
+        "breakdown": {"gemm_decode_GBps": gemm_gbs, "relayout_GBps": relayout_gbs,
+                      "gemm_ms_per_step": g_ms / args.steps, "relayout_ms_per_step": r_ms / args.steps},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": launches_per_step * args.steps, "extra": extra,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

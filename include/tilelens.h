@@ -94,11 +94,11 @@ int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, i
  * plain row-major when block_rows == 0 (then G and block_cols are ignored).
  * Products are accumulated in fp32 in tensor memory.
  *   d_A, d_B     device, 16-byte aligned (d_B 128-byte aligned when tile-major).
- *   d_C          device, M*N floats, fully overwritten.
+ *   d_C          device, 16-byte aligned, M*N floats, fully overwritten.
  *   cta_m/n/k    the CTA tile: cta_m token rows x cta_n weight columns per CTA,
  *                cta_k weight rows per pipeline stage.  0,0,0 lets the library
  *                choose.  Instantiated: cta_n in {128, 256}, cta_k in {64, 128},
- *                cta_m a multiple of 16 in [16, 256] (cta_n == 256: at most 128).
+ *                cta_m in {16, 32, 64, 128, 256} (cta_n == 256: at most 128).
  *                Tiles may overhang M, N and K.
  *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,
  *   N % block_cols == 0, block_rows >= 8, block_cols*2 >= 16 bytes;

@@ -22,6 +22,7 @@
 // Every mbarrier wait is bounded (see mbar_wait_bounded).
 #include "tl_common.cuh"
 
+#include <cstdlib>
 #include <cstring>
 
 namespace tl {
@@ -386,16 +387,38 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 const uint32_t old = arrival_bcast;
                 if (old == uint32_t(c_hi - c_lo)) {
                     __threadfence();
+                    // Partials are [row][kBN] floats; 128 threads walk them as float4, four vectors each per pass,
+                    // adding the contributors in K order (c_lo first) whatever order they arrived in.
                     float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
-                    for (int u = 0; u < kNumN; ++u) {
-                        const int n_local = u * 128 + et;
-                        if (t.n0 + n_local >= p.N) continue;
-                        for (int r = 0; r < t.rows; ++r) {
-                            float sum = 0.f;
-                            for (int c = c_lo; c <= c_hi; ++c)
-                                sum += __ldcg(p.partials + size_t(sched.slot(c, w.tile)) * p.BM * kBN +
-                                              size_t(r) * kBN + n_local);
-                            dst[int64_t(r) * p.ldc + n_local] = sum;
+                    constexpr int kVecPerRow = kBN / 4;
+                    const int total_vec = t.rows * kVecPerRow;
+                    const size_t slot_floats = size_t(p.BM) * kBN;
+                    for (int v0 = 0; v0 < total_vec; v0 += 4 * 128) {
+                        float4 sum[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) sum[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int c = c_lo; c <= c_hi; ++c) {
+                            const float4* src = reinterpret_cast<const float4*>(
+                                p.partials + size_t(sched.slot(c, w.tile)) * slot_floats);
+                            float4 x[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int v = v0 + q * 128 + et;
+                                x[q] = v < total_vec ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                sum[q].x += x[q].x; sum[q].y += x[q].y; sum[q].z += x[q].z; sum[q].w += x[q].w;
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int v = v0 + q * 128 + et;
+                            if (v < total_vec) {
+                                const int r = v / kVecPerRow, c4 = (v % kVecPerRow) * 4;
+                                if (t.n0 + c4 < p.N)
+                                    *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
+                            }
                         }
                     }
                     if (et == 0) p.counters[w.tile] = 0;     // ready for the next launch
@@ -433,8 +456,35 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// Encoded maps are kept: encoding costs microseconds of host time per map and the same
+// (pointer, shape, box) recurs on every call of a serving loop.
+struct MapKey {
+    const void* base;
+    int rank;
+    uint64_t dims[5], strides[5];
+    uint32_t box[5];
+    bool operator==(const MapKey& o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
+};
+struct MapEntry {
+    MapKey key;
+    CUtensorMap map;
+};
+static constexpr int kMapCacheSize = 256;
+
 static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                   const uint32_t* box) {
+    static MapEntry* cache = new MapEntry[kMapCacheSize];
+    static int cache_n = 0, cache_next = 0;
+    MapKey key;
+    memset(&key, 0, sizeof key);
+    key.base = base;
+    key.rank = rank;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.strides[i] = strides_bytes[i]; key.box[i] = box[i]; }
+    for (int i = 0; i < cache_n; ++i)
+        if (cache[i].key == key) {
+            *out = cache[i].map;
+            return TL_OK;
+        }
     EncodeTiledFn fn = encode_fn();
     if (!fn) {
         state().last_cuda_error = int(cudaErrorSymbolNotFound);
@@ -451,6 +501,9 @@ static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* 
         state().last_cuda_error = int(r);
         return TL_ERR_CUDA;
     }
+    const int slot = cache_n < kMapCacheSize ? cache_n++ : (cache_next++ % kMapCacheSize);
+    cache[slot].key = key;
+    cache[slot].map = *out;
     return TL_OK;
 }
 
@@ -534,7 +587,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (K % 8 != 0) return TL_ERR_UNSUPPORTED;                  // 16-byte row pitch of A
     if (reinterpret_cast<uintptr_t>(d_A) % 16 != 0) return TL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(d_B) % (row_major ? 16 : 128) != 0) return TL_ERR_ALIGNMENT;
-    if (reinterpret_cast<uintptr_t>(d_C) % 4 != 0) return TL_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(d_C) % 16 != 0) return TL_ERR_ALIGNMENT;
 
     GemmPlan plan;
     {
@@ -563,7 +616,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     // ---- weight operand B
     const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
-    int RB, AB;
+    int RB, AB, nb_box = 1, kb_box = 1;         // box: rows, atoms, memory tiles along N and K
     if (row_major) {
         // [E*K][N] seen as (64, E*K, N/64): one box covers the whole stage.
         RB = plan.BK;
@@ -578,20 +631,26 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         // (64, br, bc/64, N/bc, E*K/br) with strides (1, bc, 64, br*bc, br*N) elements.
         RB = br < plan.BK ? br : plan.BK;
         AB = (bc < plan.BN ? bc : plan.BN) / 64;
+        // One TMA instruction per stage whose box is a whole number of memory tiles (box extents 3 and 4
+        // count tiles along N and K).  TL_BOX_PER_BLOCK=1 issues one instruction per memory tile instead
+        // (same bytes, same shared-memory image; measurably slower because instruction issue then limits).
+        static const bool per_block = getenv("TL_BOX_PER_BLOCK") && atoi(getenv("TL_BOX_PER_BLOCK")) != 0;
+        nb_box = per_block ? 1 : NA / AB;
+        kb_box = per_block ? 1 : plan.BK / RB;
         const uint64_t dims[5] = {64, uint64_t(br), uint64_t(bc / 64), uint64_t(N / bc), uint64_t(K / br) * E};
         const uint64_t str[5] = {2, uint64_t(bc) * 2, 128, uint64_t(G), uint64_t(br) * uint64_t(N) * 2};
-        const uint32_t box[5] = {64, uint32_t(RB), uint32_t(AB), 1, 1};
+        const uint32_t box[5] = {64, uint32_t(RB), uint32_t(AB), uint32_t(nb_box), uint32_t(kb_box)};
         if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
         p.k_coord_per_expert = int(K / br);
         p.br_log2 = ilog2(br);
         p.bc_log2 = ilog2(bc);
     }
     p.row_major = row_major;
-    p.box_rows = RB;
-    p.box_atoms = AB;
-    p.kbx = plan.BK / RB;
-    p.nbx = NA / AB;
-    p.box_bytes = uint32_t(RB) * AB * kAtomBytes;
+    p.kbx = plan.BK / (RB * kb_box);
+    p.nbx = NA / (AB * nb_box);
+    p.box_rows = RB * kb_box;                                     // K rows and atoms one instruction covers
+    p.box_atoms = AB * nb_box;
+    p.box_bytes = uint32_t(RB) * AB * kAtomBytes * nb_box * kb_box;
     // Shared-memory image of a stage: [K box][N box][atom][row][64 elements].  Atom stride is RB*128
     // everywhere; 8-row groups are 1024 bytes apart inside a box and one box row apart across boxes.
     const uint32_t krow_bytes = uint32_t(NA) * RB * kAtomBytes;   // all boxes sharing one K range
@@ -620,9 +679,15 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
 
     cudaError_t err = cudaSuccess;
 #define TL_LAUNCH_GEMM(BK_, NN_)                                                                                   \
-    err = cudaFuncSetAttribute(gemm_kernel<BK_, NN_>, cudaFuncAttributeMaxDynamicSharedMemorySize,                 \
-                               int(plan.smem_bytes));                                                              \
-    if (err == cudaSuccess) gemm_kernel<BK_, NN_><<<plan.grid, kGemmThreads, plan.smem_bytes, stream>>>(p);
+    {                                                                                                              \
+        static bool attr_set = false;                                                                              \
+        if (!attr_set) {                                                                                           \
+            err = cudaFuncSetAttribute(gemm_kernel<BK_, NN_>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
+                                       227 * 1024 - 5 * 1024);                                                     \
+            attr_set = err == cudaSuccess;                                                                         \
+        }                                                                                                          \
+        if (err == cudaSuccess) gemm_kernel<BK_, NN_><<<plan.grid, kGemmThreads, plan.smem_bytes, stream>>>(p);    \
+    }
     if (plan.BK == 64 && plan.BN == 128) { TL_LAUNCH_GEMM(64, 1) }
     else if (plan.BK == 128 && plan.BN == 128) { TL_LAUNCH_GEMM(128, 1) }
     else if (plan.BK == 64 && plan.BN == 256) { TL_LAUNCH_GEMM(64, 2) }
