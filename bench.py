@@ -454,14 +454,66 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+PROFILE_CASES = {
+    # name: (kind, M, K, N) -- small single-kernel cases for ncu captures (a few hundred MB on the device)
+    "decode_qkv_m8": ("gemm", 8, 8192, 10240),
+    "decode_o_m32": ("gemm", 32, 8192, 8192),
+    "decode_down_m1": ("gemm", 1, 28672, 8192),
+    "prefill_o": ("gemm", 4096, 8192, 8192),
+    "prefill_qkv": ("gemm", 4096, 8192, 10240),
+    "relayout_o": ("relayout", 0, 8192, 8192),
+    "moe_gate_up": ("moe", 0, 2048, 1536),
+}
+
+
+def run_case(args):
+    """Runs one named kernel `--steps` times on cuda:0 (tile-major, default tile); prints nothing timed."""
+    from paper_2607_04031_b200 import binding as tl
+    kind, M, K, N = PROFILE_CASES[args.case]
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    if kind == "moe":
+        q = inputs.QWEN_MOE
+        offsets, _, _ = inputs.zipf_topk_routing(q["tokens"], q["experts"], q["topk"], q["zipf_alpha"], seed=0)
+        rows = int(offsets[-1])
+        Bm = inputs.bf16_normal((q["experts"], K, N), 0.02, seed=400, device=dev)
+        Bt = torch.empty_like(Bm)
+        tl.relayout(Bm, Bt, q["experts"] * K, N, 2, G, BR, BC, tl.TO_TILE_MAJOR)
+        Am = inputs.bf16_normal((rows, K), 1.0, seed=401, device=dev)
+        Cm = torch.empty((rows, N), dtype=torch.float32, device=dev)
+        d_off = torch.from_numpy(offsets).to(dev)
+        for _ in range(args.steps):
+            tl.gemm_grouped(Am, Bt, Cm, d_off, q["experts"], rows, N, K, G, BR, BC)
+    else:
+        W = inputs.bf16_normal((K, N), 0.02, seed=100, device=dev)
+        Wt = torch.empty_like(W)
+        for _ in range(args.steps if kind == "relayout" else 1):
+            tl.relayout(W, Wt, K, N, 2, G, BR, BC, tl.TO_TILE_MAJOR)
+        if kind == "gemm":
+            A = inputs.bf16_normal((M, K), 1.0, seed=200, device=dev)
+            C = torch.empty((M, N), dtype=torch.float32, device=dev)
+            for _ in range(args.steps):
+                if args.layout == "row":
+                    tl.gemm(A, W, C, M, N, K, 0, 0, 0)
+                else:
+                    tl.gemm(A, Wt, C, M, N, K, G, BR, BC)
+    tl.device_status()
+    print(json.dumps({"case": args.case, "layout": args.layout, "launches": args.steps, "status": "ok"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, choices=sorted(PROFILE_CASES),
+                    help="run one small kernel case --steps times (for ncu); no benchmark line")
+    ap.add_argument("--layout", default="tile", choices=["tile", "row"])
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
