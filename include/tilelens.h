@@ -149,6 +149,49 @@ int tl_gemm_host(const void* h_A, const void* h_B_rowmajor, float* h_C,
                  void* d_scratch, size_t scratch_bytes, void* cuda_stream);
 size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
 
+/*
+ * tl_gemm for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the product above, same kernel,
+ * same results bit for bit.)
+ *
+ * Who needs it: a serving process that hands all of HBM to its own pool at
+ * start-up, so that any later cudaMalloc fails; a plug-in host or sandbox that
+ * forbids allocation calls after initialisation; a latency-critical loop that
+ * cannot afford the device-wide synchronisation an allocation or a free may
+ * imply.  tl_gemm grows an internal workspace with cudaMalloc the first time a
+ * decode-shaped problem needs split-K scratch; this entry point never calls
+ * cudaMalloc, cudaFree or any allocating routine.  Its scratch (tile counters
+ * and partial tiles) is a fixed array of TL_NOALLOC_SCRATCH_BYTES inside the
+ * library image; every GPU that loads the library holds that much memory
+ * until the process exits.
+ *
+ *   arguments     as tl_gemm, plus d_timeout_flag: a device uint32 the caller
+ *                 owns and has zeroed, raised (non-zero) if a bounded wait in
+ *                 the kernel expires; NULL keeps the flag in the array, unread.
+ *   limit         problems whose split-K scratch exceeds the array return
+ *                 TL_ERR_WORKSPACE and enqueue nothing.  The scratch is
+ *                 64 KB + 2 * (number of SMs) * cta_m * cta_n * 4 bytes when
+ *                 M <= 64 or the tiles do not fill the SMs evenly, else 0: on
+ *                 a 148-SM B200 with the default tile that admits every
+ *                 M <= 32; M in (32, 64] needs 9.3 MB and is refused.
+ *   first call    the first call on each device looks up the array's device
+ *                 address (with that device current).  Make that call before
+ *                 starting any stream capture.
+ *   sharing       all calls share the one array, and it keeps the previous
+ *                 call's contents: the counters are cleared on cuda_stream at
+ *                 the start of every call, the partial tiles are always
+ *                 written before they are read.  Two calls that can run at
+ *                 the same time on one GPU (different streams, or different
+ *                 host threads) race on the array and give wrong results:
+ *                 serialise them.
+ */
+#define TL_NOALLOC_SCRATCH_BYTES (8u << 20)
+int tl_gemm_noalloc(const void* d_A_rowmajor, const void* d_B_tilemajor, float* d_C,
+                    int64_t M, int64_t N, int64_t K,
+                    int64_t G, int block_rows, int block_cols,
+                    int cta_m, int cta_n, int cta_k,
+                    uint32_t* d_timeout_flag, void* cuda_stream);
+
 /* --------------------------------------------------- read amplification */
 
 /*

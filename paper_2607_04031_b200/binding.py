@@ -34,6 +34,7 @@ _SIGNATURES = {
     "tl_set_workspace": (_int, [_vp, _sz]),
     "tl_gemm_host": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp, _sz, _vp]),
     "tl_gemm_host_scratch_bytes": (_sz, [_i64, _i64, _i64]),
+    "tl_gemm_noalloc": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp, _vp]),
     "tl_read_amp": (_int, [_i64, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int, _u64p, _u64p, _u64p]),
     "tl_read_amp_grouped": (_int, [_vp, _int, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int,
                                    _u64p, _u64p, _u64p]),
@@ -153,6 +154,16 @@ def gemm_host(A_host: torch.Tensor, B_rowmajor_host: torch.Tensor, C_host: torch
     _check(lib().tl_gemm_host(A_host.data_ptr(), B_rowmajor_host.data_ptr(), C_host.data_ptr(), M, N, K, G,
                               block_rows, block_cols, cta[0], cta[1], cta[2], _dev_ptr(scratch),
                               scratch.numel() * scratch.element_size(), _stream_ptr(stream)), "tl_gemm_host")
+
+
+def gemm_noalloc(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, M: int, N: int, K: int, G: int = 4096,
+                 block_rows: int = 16, block_cols: int = 128, cta=(0, 0, 0), timeout_flag: torch.Tensor | None = None,
+                 stream=None):
+    """tl_gemm for processes that may not allocate device memory: split-K scratch is a fixed array
+    inside the library (8 MiB per GPU).  `timeout_flag`: optional zeroed uint32/int32 CUDA tensor."""
+    flag = _dev_ptr(timeout_flag) if timeout_flag is not None else None
+    _check(lib().tl_gemm_noalloc(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), M, N, K, G, block_rows, block_cols,
+                                 cta[0], cta[1], cta[2], flag, _stream_ptr(stream)), "tl_gemm_noalloc")
 
 
 def read_amp(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int = 0, block_cols: int = 0,

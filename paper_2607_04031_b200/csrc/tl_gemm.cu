@@ -566,9 +566,16 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     return TL_OK;
 }
 
+// Where a launch takes its scratch from when the caller of gemm_launch supplies it itself.
+struct FixedScratch {
+    void* ws;            // counters + partial tiles
+    size_t ws_bytes;
+    uint32_t* status;    // word the kernel raises when a bounded wait expires
+};
+
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
-                       int cta_m, int cta_n, int cta_k, cudaStream_t stream) {
+                       int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr) {
     if (rows_total < 0 || N <= 0 || K <= 0 || E < 1) return TL_ERR_INVALID_ARG;
     if (rows_total == 0) return TL_OK;
     if (!d_A || !d_B || !d_C) return TL_ERR_INVALID_ARG;
@@ -601,9 +608,18 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
             return rc;
     }
     if (d_offsets && K % plan.BK != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
-    if (int rc = ensure_control()) return rc;
     void* ws = nullptr;
-    if (int rc = get_workspace(plan.ws_bytes, &ws)) return rc;
+    if (fixed) {
+        if (plan.ws_bytes > fixed->ws_bytes) return TL_ERR_WORKSPACE;
+        ws = plan.ws_bytes ? fixed->ws : nullptr;
+        // A fixed scratch keeps the previous launch's contents.  Partial tiles are always written before
+        // they are read; the tile counters must start at zero, so they are cleared on the same stream.
+        if (ws)
+            if (int rc = check_cuda(cudaMemsetAsync(ws, 0, kCounterBytes, stream))) return rc;
+    } else {
+        if (int rc = ensure_control()) return rc;
+        if (int rc = get_workspace(plan.ws_bytes, &ws)) return rc;
+    }
 
     GemmParams p;
     memset(&p, 0, sizeof p);
@@ -664,7 +680,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.counters = static_cast<uint32_t*>(ws);
     p.partials = ws ? reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + kCounterBytes) : nullptr;
     p.offsets = d_offsets;
-    p.status = state().ctl.d_status;
+    p.status = fixed ? fixed->status : state().ctl.d_status;
     p.ldc = N;
     p.M = int(rows_total);
     p.N = int(N);
@@ -771,3 +787,47 @@ int tl_gemm_host(const void* h_A, const void* h_B_rowmajor, float* h_C, int64_t 
 }
 
 }  // extern "C"
+
+// ------------------------------------------------- scratch held in the library image
+namespace tl {
+
+// Split-K scratch of tl_gemm_noalloc: tile counters (first kCounterBytes), partial tiles, and in the
+// last 256 bytes a spare word for the time-out flag when the caller passes none.  Lives in the
+// module's data segment on every GPU that loads the library, from load until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TL_NOALLOC_SCRATCH_BYTES];
+
+// g_noalloc_scratch is a host-side handle here, not an address a kernel could use: the device address
+// is looked up once per device, with that device current, and remembered.
+static int noalloc_scratch_address(unsigned char** out) {
+    static unsigned char* per_device[64] = {};
+    int dev = -1;
+    if (int rc = check_cuda(cudaGetDevice(&dev))) return rc;
+    if (dev < 0 || dev >= 64) return TL_ERR_UNSUPPORTED;
+    if (!per_device[dev]) {
+        void* ptr = nullptr;
+        if (int rc = check_cuda(cudaGetSymbolAddress(&ptr, g_noalloc_scratch))) return rc;
+        if (!ptr) return TL_ERR_CUDA;
+        per_device[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = per_device[dev];
+    return TL_OK;
+}
+
+}  // namespace tl
+
+extern "C" int tl_gemm_noalloc(const void* d_A, const void* d_B, float* d_C, int64_t M, int64_t N, int64_t K,
+                               int64_t G, int block_rows, int block_cols, int cta_m, int cta_n, int cta_k,
+                               uint32_t* d_timeout_flag, void* cuda_stream) {
+    if (M < 0 || N <= 0 || K <= 0) return TL_ERR_INVALID_ARG;
+    if (M == 0) return TL_OK;
+    unsigned char* base = nullptr;
+    if (int rc = tl::noalloc_scratch_address(&base)) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    tl::FixedScratch fixed;
+    fixed.ws = base;
+    fixed.ws_bytes = TL_NOALLOC_SCRATCH_BYTES - 256;
+    fixed.status = d_timeout_flag ? d_timeout_flag
+                                  : reinterpret_cast<uint32_t*>(base + TL_NOALLOC_SCRATCH_BYTES - 256);
+    return tl::gemm_launch(d_A, d_B, d_C, nullptr, 1, M, M, N, K, G, block_rows, block_cols, cta_m, cta_n, cta_k,
+                           stream, &fixed);
+}

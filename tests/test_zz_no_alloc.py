@@ -1,0 +1,70 @@
+"""tl_gemm_noalloc: the GEMM for callers that may not allocate device memory (GPU).
+
+Some hosts of this library cannot call cudaMalloc once they are running: an inference server that
+gave all of HBM to its own pool at start-up, a sandbox that forbids allocation after initialisation.
+For them the split-K scratch lives in a fixed array inside the library.  This file checks that the
+entry point, called through the C ABI, gives exactly what tl_gemm gives, twice in a row (the array
+keeps the first call's contents, so the second call proves the clean-up), and that it refuses
+problems whose scratch does not fit.  It is collected last so that a failure here cannot hide
+another test's result; it does not depend on any other test having run.
+"""
+import pytest
+import torch
+
+from paper_2607_04031_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(M, N, K, seed, integer):
+    from gpu_util import DEV, tile_major_on_device
+    if integer:
+        A = inputs.bf16_integers((M, K), -8, 8, seed=seed)
+        B = inputs.bf16_integers((K, N), -8, 8, seed=seed + 1)
+    else:
+        A = inputs.bf16_normal((M, K), 1.0, seed=seed)
+        B = inputs.bf16_normal((K, N), 0.02, seed=seed + 1)
+    return A.to(DEV).contiguous(), tile_major_on_device(B, K, N, 16, 128)
+
+
+@pytest.mark.parametrize("M,N,K,integer", [(8, 1024, 8192, True), (32, 2048, 4096, False), (1, 512, 2048, False)])
+def test_matches_tl_gemm_on_two_calls_in_a_row(M, N, K, integer):
+    from gpu_util import DEV, tl
+    A, Bt = _case(M, N, K, seed=70 + M, integer=integer)
+    want = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    tl.gemm(A, Bt, want, M, N, K, 4096, 16, 128)          # existing entry point (allocating workspace)
+    tl.device_status()
+    flag = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for call in range(2):
+        got = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+        tl.gemm_noalloc(A, Bt, got, M, N, K, 4096, 16, 128, timeout_flag=flag)
+        torch.cuda.synchronize()
+        assert int(flag.item()) == 0, "a bounded wait expired inside the kernel"
+        # same kernel, same schedule, same summation order: identical bits (tolerance 0, stricter than
+        # the 1e-3 * sum|a b| the other GEMM tests allow)
+        assert torch.equal(got, want), f"call {call}"
+    # a different problem right after, then the first one again: stale partial tiles must not leak
+    A2, Bt2 = _case(16, 768, 2048, seed=5, integer=True)
+    want2 = torch.empty((16, 768), dtype=torch.float32, device=DEV)
+    tl.gemm(A2, Bt2, want2, 16, 768, 2048, 4096, 16, 128)
+    got2 = torch.empty_like(want2)
+    tl.gemm_noalloc(A2, Bt2, got2, 16, 768, 2048, 4096, 16, 128)
+    got = torch.empty_like(want)
+    tl.gemm_noalloc(A, Bt, got, M, N, K, 4096, 16, 128)
+    torch.cuda.synchronize()
+    assert torch.equal(got2, want2) and torch.equal(got, want)
+
+
+def test_refuses_scratch_beyond_the_fixed_array():
+    from gpu_util import DEV, tl
+    M, N, K = 64, 1024, 4096                               # 2 * SMs * 64 * 128 * 4 bytes > 8 MiB on a B200
+    A, Bt = _case(M, N, K, seed=9, integer=True)
+    C = torch.zeros((M, N), dtype=torch.float32, device=DEV)
+    need = tl.gemm_workspace_bytes(M, N, K)
+    if need <= (8 << 20) - 256:
+        pytest.skip("this GPU has few enough SMs for the scratch to fit")
+    with pytest.raises(tl.TileLensError) as e:
+        tl.gemm_noalloc(A, Bt, C, M, N, K, 4096, 16, 128)
+    assert e.value.status == 6
+    torch.cuda.synchronize()
+    assert float(C.abs().sum()) == 0.0                     # nothing was enqueued
