@@ -27,7 +27,8 @@
 
 namespace tl {
 
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 192;          // TMA path: producer, MMA issuer, four epilogue warps
+constexpr int kGenericThreads = 320;       // generic-address path: four more warps that load the weights by hand
 constexpr int kMaxStages = 16;
 constexpr int kMaxExperts = 1024;
 constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 256 rows
@@ -60,6 +61,11 @@ struct alignas(64) GemmParams {
     uint32_t box_bytes;
     uint32_t lbo, sbo;          // descriptor strides of the MN-major operand, bytes
     uint32_t kstep_off[8];      // byte offset of each 16-row K step inside a stage
+    // generic-address path (Section 4.4: memory tiles that TMA cannot box)
+    int generic_b;              // 1: warps 6..9 load the weights with Eq. 1-2 address arithmetic
+    const uint8_t* B;           // raw weight pointer (generic path only)
+    int64_t expert_bytes;       // K*N*2
+    int blocks_per_row;         // N / bc
 };
 
 struct TileInfo {
@@ -150,13 +156,71 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, 
            (uint64_t(1) << 46) | (uint64_t(2) << 61);
 }
 
+// Optional per-CTA timestamps (nanoseconds of %globaltimer), compiled in only with -DTL_TIMELINE:
+// slot 0 kernel entry, 1 set-up done, 2 first stage landed, 3 last MMA committed, 4 first epilogue
+// started, 5 last epilogue (and fix-up) done, 6 producer done.
+#ifdef TL_TIMELINE
+__device__ uint64_t* g_timeline = nullptr;
+#define TL_TIMELINE_INIT() uint64_t* const tl_tl = g_timeline ? g_timeline + blockIdx.x * 8 : nullptr; bool tl_once = true; (void)tl_once
+#define TL_STAMP(slot) do { if (tl_tl) tl_tl[(slot)] = global_timer_ns(); } while (0)
+#define TL_STAMP_ONCE(slot) do { if (tl_once) { tl_once = false; if (tl_tl) tl_tl[(slot)] = global_timer_ns(); } } while (0)
+#else
+#define TL_TIMELINE_INIT() do { } while (0)
+#define TL_STAMP(slot) do { } while (0)
+#define TL_STAMP_ONCE(slot) do { } while (0)
+#endif
+
 __device__ __forceinline__ void epilogue_bar_sync() {
     asm volatile("bar.sync 1, 128;" ::: "memory");
 }
 
+// One warp fills one stage of weights on the generic-address path.  The stage is kBK/br runs of
+// kBN/bc whole memory tiles; run r starts at src0 + r*krow_stride and is kBN*br*2 contiguous bytes.
+// Chunks of 16 bytes are read in memory order, 16 loads in flight per lane; kPieces = rows held by one
+// chunk (1 when a block row is at least 16 bytes).  Rows >= k_rows_left and columns >= n_cols_left
+// (tile overhang) are filled with zeros.
+template <int kBK, int kBN, int kPieces>
+__device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* src0, int64_t krow_stride, int br_log2,
+                                                   int bc_log2, int k_rows_left, int n_cols_left, int lane) {
+    constexpr int kChunks = kBK * kBN * 2 / 16;
+    const int run_log2 = bc_log2 + 1;                       // log2(bytes of one block row)
+    const int g_log2 = br_log2 + run_log2;                  // log2(G)
+    const int seg_log2 = br_log2 + 1 + (kBN == 128 ? 7 : 8);   // log2(kBN * br * 2): bytes of one run of tiles
+#pragma unroll 1
+    for (int base = 0; base < kChunks; base += 32 * 16) {
+        uint4 v[16];
+        int kl[16], nl[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int byte = (base + i * 32 + lane) << 4;   // byte offset inside the stage's memory image
+            const int seg = byte >> seg_log2, o = byte & ((1 << seg_log2) - 1);
+            const int ib = o & ((1 << g_log2) - 1);         // byte inside the memory tile
+            kl[i] = (seg << br_log2) + (ib >> run_log2);    // Eq. 1 inverted: row and column inside the stage
+            nl[i] = ((o >> g_log2) << bc_log2) + ((ib & ((1 << run_log2) - 1)) >> 1);
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (kl[i] < k_rows_left && nl[i] < n_cols_left)
+                v[i] = __ldg(reinterpret_cast<const uint4*>(src0 + int64_t(seg) * krow_stride + o));
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t word[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+            for (int pc = 0; pc < kPieces; ++pc) {
+                const int k = kl[i] + pc, n = nl[i];
+                uint8_t* dst = sw + (n >> 6) * (kBK * kAtomBytes) + k * kAtomBytes + ((((n & 63) >> 3) ^ (k & 7)) << 4) +
+                               (n & 7) * 2;
+                if (kPieces == 1) *reinterpret_cast<uint4*>(dst) = v[i];
+                else if (kPieces == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(word[2 * pc], word[2 * pc + 1]);
+                else if (kPieces == 4) *reinterpret_cast<uint32_t*>(dst) = word[pc];
+                else *reinterpret_cast<uint16_t*>(dst) = uint16_t(word[pc >> 1] >> ((pc & 1) * 16));
+            }
+        }
+    }
+}
+
 // kBK: weight rows per stage (64 or 128).  kNumN: 128-column groups per CTA tile (1 or 2).
 template <int kBK, int kNumN>
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+__global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
     constexpr int kBN = 128 * kNumN;
     constexpr int kKSteps = kBK / 16;
     constexpr int kSubK = kBK / 64;                        // token boxes per stage
@@ -174,6 +238,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    TL_TIMELINE_INIT();
+    if (threadIdx.x == 0) TL_STAMP(0);
     const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.BM * kAtomBytes;
     uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -183,11 +249,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
 
     // ---------------------------------------------------------------- set-up
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], p.generic_b ? 2 : 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 4); }
         abort_flag = 0;
         fence_mbar_init();
-        tma_prefetch_desc(&p.tmap_b);
+        if (!p.generic_b) tma_prefetch_desc(&p.tmap_b);
     }
     if (warp == 1) {
         tmem_alloc(&tmem_slot, tmem_cols);
@@ -210,6 +276,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     const int tiles_total = prefix[p.E];
+    if (threadIdx.x == 0) TL_STAMP(1);
 
     Sched sched;
     sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x);
@@ -259,6 +326,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
                 }
             }
+            TL_STAMP(6);
             if (!ok || *abort_ptr) {
                 // Giving up: let the copies already issued land before the CTA's shared memory goes away.
                 uint32_t s = stage, ph = phase;
@@ -295,6 +363,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                         break;
                     }
                     tc_fence_after_sync();
+                    TL_STAMP_ONCE(2);
                     const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
                     const uint32_t sa = sw + kWBytes;
 #pragma unroll
@@ -314,8 +383,52 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 }
                 if (!ok) break;
                 umma_commit(&acc_full_bar[acc]);         // accumulator complete
+                TL_STAMP(3);
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1;
+            }
+        }
+    } else if (warp >= 6) {
+        // ================================ generic-address weight loader (Section 4.4 of the paper)
+        // Memory tiles whose rows are shorter than a TMA box allows are fetched with plain loads.  A stage's
+        // weights are kBK/br runs of whole memory tiles, each run contiguous in the tile-major buffer, so
+        // the 16-byte chunks are read in memory order (fully coalesced for any tile shape); Eq. 1 inverted
+        // gives every chunk's (row, column), and the chunk (or its 16/(2 bc) row pieces) is stored where the
+        // 128-byte-swizzled MN-major operand layout wants it.  Warp w fills every fourth stage.
+        const int pw = warp - 6;
+        const int br = 1 << p.br_log2, bc = 1 << p.bc_log2;
+        const int run_bytes = bc * 2;                              // one block row
+        const int G = br * run_bytes;
+        const int pieces = run_bytes >= 16 ? 1 : 16 / run_bytes;  // rows held by one 16-byte chunk
+        uint32_t it_global = 0;
+        Work w;
+        bool ok = true;
+        while (ok && sched.next(w)) {
+            const TileInfo t = decode_tile(p, prefix, w.tile);
+            const uint8_t* Bexp = p.B + int64_t(t.expert) * p.expert_bytes;
+            const int nblk0 = t.n0 >> p.bc_log2;
+            for (int kit = w.kbeg; kit < w.kend; ++kit, ++it_global) {
+                if ((it_global & 3u) != uint32_t(pw)) continue;
+                const uint32_t stage = it_global % uint32_t(p.num_stages);
+                const uint32_t phase = (it_global / uint32_t(p.num_stages)) & 1u;
+                if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
+                    ok = false;
+                    break;
+                }
+                uint8_t* sw = stages + size_t(stage) * stage_bytes;
+                const int kblk0 = (kit * kBK) >> p.br_log2;
+                const uint8_t* src0 = Bexp + (int64_t(kblk0) * p.blocks_per_row + nblk0) * G;
+                const int k_rows_left = p.K - kit * kBK, n_cols_left = p.N - t.n0;
+                const int64_t krow_stride = int64_t(p.blocks_per_row) * G;      // bytes between runs of tiles
+                switch (pieces) {
+                    case 1: generic_fill_stage<kBK, kBN, 1>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                    case 2: generic_fill_stage<kBK, kBN, 2>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                    case 4: generic_fill_stage<kBK, kBN, 4>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                    default: generic_fill_stage<kBK, kBN, 8>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                }
+                fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor-core (async) proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[stage]);
             }
         }
     } else {
@@ -330,6 +443,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
             const int n_mma = (t.rows + 15) & ~15;
             bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
             tc_fence_after_sync();
+            if (et == 0) TL_STAMP_ONCE(4);
             float* out;
             int64_t ld;
             if (full) {
@@ -425,6 +539,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
                 }
                 epilogue_bar_sync();                          // arrival_bcast may be rewritten after this
             }
+            if (et == 0) TL_STAMP(5);
             if (*abort_ptr) break;
         }
     }
@@ -582,18 +697,20 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (rows_total >= (int64_t(1) << 31) || N >= (int64_t(1) << 31) || K * int64_t(E) >= (int64_t(1) << 31))
         return TL_ERR_UNSUPPORTED;
     if (E > kMaxExperts) return TL_ERR_UNSUPPORTED;
-    const bool row_major = br == 0;
-    if (!row_major) {
+    if (br != 0) {
         if (br < 0 || bc <= 0 || int64_t(br) * bc * 2 != G) return TL_ERR_INVALID_ARG;
         if (!is_pow2(br) || !is_pow2(bc)) return TL_ERR_UNSUPPORTED;
         if (K % br != 0 || N % bc != 0) return TL_ERR_INVALID_ARG;
-        if (br < 8 || bc < 64) return TL_ERR_UNSUPPORTED;       // TMA path: whole 8-row x 128-byte swizzle atoms
-    } else {
-        if (N % 64 != 0) return TL_ERR_UNSUPPORTED;
     }
+    // One-row memory tiles are row-major (Section 3.1: the (1, G/s) extreme).
+    const bool row_major = br == 0 || (br == 1 && N % 64 == 0);
+    // TMA boxes need whole 8-row x 128-byte swizzle atoms; anything smaller takes the generic-address path.
+    const bool generic = !row_major && (br < 8 || bc < 64);
+    if (row_major && N % 64 != 0) return TL_ERR_UNSUPPORTED;
+    if (generic && (G < 16 || br > 128 || bc > 256)) return TL_ERR_UNSUPPORTED;   // tile must fit the CTA tile
     if (K % 8 != 0) return TL_ERR_UNSUPPORTED;                  // 16-byte row pitch of A
     if (reinterpret_cast<uintptr_t>(d_A) % 16 != 0) return TL_ERR_ALIGNMENT;
-    if (reinterpret_cast<uintptr_t>(d_B) % (row_major ? 16 : 128) != 0) return TL_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(d_B) % (row_major || generic ? 16 : 128) != 0) return TL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(d_C) % 16 != 0) return TL_ERR_ALIGNMENT;
 
     GemmPlan plan;
@@ -633,7 +750,19 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     // ---- weight operand B
     const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
     int RB, AB, nb_box = 1, kb_box = 1;         // box: rows, atoms, memory tiles along N and K
-    if (row_major) {
+    if (generic) {
+        // No tensor map: warps 6..9 of the kernel compute Eq. 1-2 addresses themselves and build the
+        // canonical [atom][cta_k rows][64] image in shared memory.
+        if (plan.BK % br != 0 || plan.BN % bc != 0) return TL_ERR_UNSUPPORTED;
+        RB = plan.BK;
+        AB = NA;
+        p.generic_b = 1;
+        p.B = static_cast<const uint8_t*>(d_B);
+        p.expert_bytes = K * N * 2;
+        p.blocks_per_row = int(N / bc);
+        p.br_log2 = ilog2(br);
+        p.bc_log2 = ilog2(bc);
+    } else if (row_major) {
         // [E*K][N] seen as (64, E*K, N/64): one box covers the whole stage.
         RB = plan.BK;
         AB = NA;
@@ -662,8 +791,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.bc_log2 = ilog2(bc);
     }
     p.row_major = row_major;
-    p.kbx = plan.BK / (RB * kb_box);
-    p.nbx = NA / (AB * nb_box);
+    p.kbx = generic ? 0 : plan.BK / (RB * kb_box);
+    p.nbx = generic ? 0 : NA / (AB * nb_box);
     p.box_rows = RB * kb_box;                                     // K rows and atoms one instruction covers
     p.box_atoms = AB * nb_box;
     p.box_bytes = uint32_t(RB) * AB * kAtomBytes * nb_box * kb_box;
@@ -702,7 +831,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                                        227 * 1024 - 5 * 1024);                                                     \
             attr_set = err == cudaSuccess;                                                                         \
         }                                                                                                          \
-        if (err == cudaSuccess) gemm_kernel<BK_, NN_><<<plan.grid, kGemmThreads, plan.smem_bytes, stream>>>(p);    \
+        if (err == cudaSuccess)                                                                                    \
+            gemm_kernel<BK_, NN_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes, stream>>>(p);     \
     }
     if (plan.BK == 64 && plan.BN == 128) { TL_LAUNCH_GEMM(64, 1) }
     else if (plan.BK == 128 && plan.BN == 128) { TL_LAUNCH_GEMM(128, 1) }
@@ -831,3 +961,10 @@ extern "C" int tl_gemm_noalloc(const void* d_A, const void* d_B, float* d_C, int
     return tl::gemm_launch(d_A, d_B, d_C, nullptr, 1, M, M, N, K, G, block_rows, block_cols, cta_m, cta_n, cta_k,
                            stream, &fixed);
 }
+
+#ifdef TL_TIMELINE
+// Measurement builds only: d_buf holds 8 uint64 per CTA (zeroed by the caller); nullptr switches it off.
+extern "C" int tl_debug_set_timeline(void* d_buf) {
+    return tl::check_cuda(cudaMemcpyToSymbol(tl::g_timeline, &d_buf, sizeof d_buf));
+}
+#endif

@@ -33,7 +33,12 @@ def test_config1_tiny_tile_major_and_row_major():
     assert torch.equal(C, C_row)
 
 
-@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0)])
+# TMA-boxable tiles, row-major, one-row tiles (= row-major), and tiles only the generic-address path can read
+BLOCKS = [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0), (1, 1024), (1, 128),
+          (8, 2), (16, 1), (8, 16), (16, 8), (32, 4), (16, 32), (32, 16), (2, 64), (4, 128), (64, 8)]
+
+
+@pytest.mark.parametrize("br,bc", BLOCKS)
 @pytest.mark.parametrize("cta", [(0, 0, 0), (64, 128, 64), (128, 256, 64), (32, 128, 128), (128, 256, 128)])
 def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     # No arithmetic at all: catches any error in the tensor-map view, the swizzle or the descriptors.
@@ -46,6 +51,18 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     assert torch.equal(C.cpu(), B.float()[ks])
 
 
+def test_hand_addressed_tile_wider_than_the_cta_tile():
+    from gpu_util import run_gemm, tile_major_on_device, tl
+    M, N, K = 24, 512, 256
+    A, ks = inputs.one_hot_rows(M, K, seed=3)
+    B = inputs.bf16_normal((K, N), 0.02, seed=4)
+    Bd = tile_major_on_device(B, K, N, 4, 256)
+    assert torch.equal(run_gemm(A, Bd, M, N, K, 4, 256, (32, 256, 64)).cpu(), B.float()[ks])
+    with pytest.raises(tl.TileLensError) as e:
+        run_gemm(A, Bd, M, N, K, 4, 256, (32, 128, 64))        # a 256-wide tile does not fit 128 columns
+    assert e.value.status == 2
+
+
 SHAPES = [  # M, N, K
     (1, 512, 512), (8, 1024, 2048), (33, 640, 1024), (64, 256, 8192), (100, 384, 320),
     (300, 1152, 576), (257, 128, 64), (16, 8192, 1024),
@@ -53,7 +70,7 @@ SHAPES = [  # M, N, K
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
-@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (0, 0)])
+@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (0, 0), (8, 2), (16, 32), (1, 64)])
 def test_integer_inputs_are_bit_exact(M, N, K, br, bc):
     from gpu_util import DEV, run_gemm, tile_major_on_device
     A = inputs.bf16_integers((M, K), -8, 8, seed=M + N)
@@ -182,7 +199,7 @@ def _check_grouped(offsets, A, Bd, C, E, K, N, br, bc, samples_per_expert, exact
     assert worst <= 1e-4
 
 
-@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (0, 0)])
+@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (0, 0), (8, 16), (16, 1)])
 def test_grouped_small_integer_exact(br, bc):
     E, K, N = 8, 256, 384
     offsets, counts, A, Bd, C = _grouped_case(E, 40, 3, K, N, br, bc, seed=3, integer=True)
