@@ -97,12 +97,16 @@ int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, i
  *   d_C          device, 16-byte aligned, M*N floats, fully overwritten.
  *   cta_m/n/k    the CTA tile: cta_m token rows x cta_n weight columns per CTA,
  *                cta_k weight rows per pipeline stage.  0,0,0 lets the library
- *                choose.  Instantiated: cta_n in {128, 256}, cta_k in {64, 128},
+ *                choose.  Instantiated: cta_n in {64, 128, 256}, cta_k in {64, 128},
  *                cta_m in {16, 32, 64, 128, 256} (cta_n == 256: at most 128).
  *                Tiles may overhang M, N and K.
  *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,
- *   N % block_cols == 0, block_rows >= 8, block_cols*2 >= 16 bytes;
- *   row-major: N % 64 == 0.  Other block shapes: TL_ERR_UNSUPPORTED.
+ *   N % block_cols == 0; row-major: N % 64 == 0.
+ *   Memory tiles of at least 8 rows x 64 columns are read by TMA.  Smaller
+ *   ones (block rows down to 2 bytes) are read by the generic-address path of
+ *   Section 4.4 (plain loads with Eq. 1-2 arithmetic); there the memory tile
+ *   must fit inside the CTA tile (block_rows | cta_k, block_cols | cta_n) and
+ *   G >= 16, else TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
  * When M <= 64 (decode) the K loop of every output tile is cut stream-K
  * fashion over all SMs; partial tiles go through a workspace and are summed
  * in a fixed order, so results are reproducible run to run.  The workspace is

@@ -185,7 +185,7 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
     constexpr int kChunks = kBK * kBN * 2 / 16;
     const int run_log2 = bc_log2 + 1;                       // log2(bytes of one block row)
     const int g_log2 = br_log2 + run_log2;                  // log2(G)
-    const int seg_log2 = br_log2 + 1 + (kBN == 128 ? 7 : 8);   // log2(kBN * br * 2): bytes of one run of tiles
+    const int seg_log2 = br_log2 + 1 + (kBN == 64 ? 6 : kBN == 128 ? 7 : 8);   // log2(kBN * br * 2): bytes of one run of tiles
 #pragma unroll 1
     for (int base = 0; base < kChunks; base += 32 * 16) {
         uint4 v[16];
@@ -218,10 +218,12 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
     }
 }
 
-// kBK: weight rows per stage (64 or 128).  kNumN: 128-column groups per CTA tile (1 or 2).
-template <int kBK, int kNumN>
+// kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256): one MMA of
+// M = 64, one of M = 128, or two of M = 128 sharing the token operand.
+template <int kBK, int kBN>
 __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-    constexpr int kBN = 128 * kNumN;
+    constexpr int kNumN = kBN >= 128 ? kBN / 128 : 1;     // MMAs per K step
+    constexpr int kUmmaM = kBN >= 128 ? 128 : 64;         // weight columns per MMA
     constexpr int kKSteps = kBK / 16;
     constexpr int kSubK = kBK / 64;                        // token boxes per stage
     constexpr uint32_t kWBytes = kBK * kBN * 2;            // weight bytes per stage
@@ -348,9 +350,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             while (ok && sched.next(w)) {
                 const TileInfo t = decode_tile(p, prefix, w.tile);
                 const uint32_t n_mma = uint32_t((t.rows + 15) & ~15);
-                // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = 128, N = n_mma
+                // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = kUmmaM, N = n_mma
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((n_mma >> 3) << 17) |
-                                       ((128u >> 4) << 24);
+                                       ((uint32_t(kUmmaM) >> 4) << 24);
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
                     ok = false;
                     break;
@@ -456,8 +458,11 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             if (ok) {
 #pragma unroll
                 for (int u = 0; u < kNumN; ++u) {
-                    const int n_local = u * 128 + quarter * 32 + lane;
-                    const bool n_ok = full ? (t.n0 + n_local < p.N) : true;
+                    // M = 128: accumulator row r sits in TMEM lane r.  M = 64: rows 16q..16q+15 sit in the
+                    // lower half of lane quarter q, the upper 16 lanes of each quarter hold nothing.
+                    const int n_local = kUmmaM == 128 ? u * 128 + quarter * 32 + lane : quarter * 16 + lane;
+                    const bool lane_ok = kUmmaM == 128 || lane < 16;
+                    const bool n_ok = lane_ok && (full ? (t.n0 + n_local < p.N) : true);
                     const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) +
                                            acc * uint32_t(kNumN * acc_cols) + uint32_t(u * acc_cols);
                     for (int c0 = 0; c0 < n_mma; c0 += 32) {
@@ -655,7 +660,7 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
         BK = 64;
     }
     if (BM != 16 && BM != 32 && BM != 64 && BM != 128 && BM != 256) return TL_ERR_UNSUPPORTED;
-    if (BN != 128 && BN != 256) return TL_ERR_UNSUPPORTED;
+    if (BN != 64 && BN != 128 && BN != 256) return TL_ERR_UNSUPPORTED;
     if (BK != 64 && BK != 128) return TL_ERR_UNSUPPORTED;
     if (BN == 256 && BM > 128) return TL_ERR_UNSUPPORTED;   // 2 accumulators x 2 groups x BM columns <= 512
     plan->BM = BM; plan->BN = BN; plan->BK = BK;
@@ -834,10 +839,12 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (err == cudaSuccess)                                                                                    \
             gemm_kernel<BK_, NN_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes, stream>>>(p);     \
     }
-    if (plan.BK == 64 && plan.BN == 128) { TL_LAUNCH_GEMM(64, 1) }
-    else if (plan.BK == 128 && plan.BN == 128) { TL_LAUNCH_GEMM(128, 1) }
-    else if (plan.BK == 64 && plan.BN == 256) { TL_LAUNCH_GEMM(64, 2) }
-    else { TL_LAUNCH_GEMM(128, 2) }
+    if (plan.BK == 64 && plan.BN == 128) { TL_LAUNCH_GEMM(64, 128) }
+    else if (plan.BK == 128 && plan.BN == 128) { TL_LAUNCH_GEMM(128, 128) }
+    else if (plan.BK == 64 && plan.BN == 256) { TL_LAUNCH_GEMM(64, 256) }
+    else if (plan.BK == 128 && plan.BN == 256) { TL_LAUNCH_GEMM(128, 256) }
+    else if (plan.BK == 64 && plan.BN == 64) { TL_LAUNCH_GEMM(64, 64) }
+    else { TL_LAUNCH_GEMM(128, 64) }
 #undef TL_LAUNCH_GEMM
     if (err != cudaSuccess) return check_cuda(err);
     return check_cuda(cudaGetLastError());

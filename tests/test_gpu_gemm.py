@@ -39,7 +39,8 @@ BLOCKS = [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0), (1, 1024),
 
 
 @pytest.mark.parametrize("br,bc", BLOCKS)
-@pytest.mark.parametrize("cta", [(0, 0, 0), (64, 128, 64), (128, 256, 64), (32, 128, 128), (128, 256, 128)])
+@pytest.mark.parametrize("cta", [(0, 0, 0), (64, 128, 64), (128, 256, 64), (32, 128, 128), (128, 256, 128),
+                                 (64, 64, 64), (16, 64, 128)])
 def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     # No arithmetic at all: catches any error in the tensor-map view, the swizzle or the descriptors.
     from gpu_util import DEV, run_gemm, tile_major_on_device
@@ -47,6 +48,15 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     A, ks = inputs.one_hot_rows(M, K, seed=7)
     B = inputs.bf16_normal((K, N), 0.02, seed=8)
     Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
+    hand_addressed = br > 1 and (br < 8 or bc < 64)
+    cta_n, cta_k = (cta[1] or 128), (cta[2] or 64)
+    if hand_addressed and (bc > cta_n or br > cta_k):
+        # documented limit of the generic-address path: the memory tile must fit inside the CTA tile
+        from gpu_util import tl
+        with pytest.raises(tl.TileLensError) as e:
+            run_gemm(A, Bd, M, N, K, br, bc, cta)
+        assert e.value.status == 2
+        return
     C = run_gemm(A, Bd, M, N, K, br, bc, cta)
     assert torch.equal(C.cpu(), B.float()[ks])
 
@@ -88,7 +98,8 @@ def test_integer_inputs_are_bit_exact(M, N, K, br, bc):
 
 
 @pytest.mark.parametrize("cta", [(16, 128, 64), (32, 128, 64), (64, 128, 128), (128, 128, 64), (256, 128, 64),
-                                 (128, 256, 64), (64, 256, 128), (256, 128, 128)])
+                                 (128, 256, 64), (64, 256, 128), (256, 128, 128), (64, 64, 64), (256, 64, 64),
+                                 (128, 64, 128)])
 def test_every_cta_tile_random_data(cta):
     from gpu_util import check_against_oracle, run_gemm, tile_major_on_device
     M, N, K, br, bc = 200, 768, 1024, 16, 128
@@ -97,6 +108,36 @@ def test_every_cta_tile_random_data(cta):
     Bt = tile_major_on_device(B, K, N, br, bc)
     C = run_gemm(A, Bt, M, N, K, br, bc, cta)
     check_against_oracle(C, A, Bt, TILE, br, bc, M, N, K)
+
+
+def _sweep_layouts():
+    """Config 5: G x aspect (block rows 1, 8, 16, 32; block columns G / (2 rows)); invalid combinations skipped."""
+    out = []
+    for G in (32, 256, 1024, 4096, 16384):
+        for br in (1, 8, 16, 32):
+            bc = G // (2 * br)
+            if bc >= 1:
+                out.append((G, br, bc))
+    return out
+
+
+@pytest.mark.parametrize("G,br,bc", _sweep_layouts())
+def test_granularity_sweep_layouts_every_cta_tile(G, br, bc):
+    # Same layouts and CTA tiles as the sweep of the benchmark, on a 1024 x 8192 slice of its 8192 x 8192
+    # weight (bc goes up to 8192); integer data, so every sampled output must match the oracle exactly.
+    from gpu_util import DEV, run_gemm, tile_major_on_device, tl
+    K, N = 1024, 8192
+    B = inputs.bf16_integers((K, N), -8, 8, seed=G + br)
+    Bd = tile_major_on_device(B, K, N, br, bc)
+    for M in (1, 16, 128):
+        A = inputs.bf16_integers((M, K), -8, 8, seed=M)
+        rng = np.random.default_rng(M)
+        ii, jj = rng.integers(0, M, 400), rng.integers(0, N, 400)
+        ref, _ = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), TILE, br, bc, M, N, K, ii, jj)
+        for cta in ((64, 64, 64), (128, 128, 64), (256, 128, 64)):
+            C = run_gemm(A, Bd, M, N, K, br, bc, cta)
+            assert np.array_equal(C.cpu().numpy()[ii, jj].astype(np.float64), ref), (M, cta)
+            assert torch.isfinite(C).all()
 
 
 def test_all_ones_B_gives_row_sums():
