@@ -40,8 +40,9 @@ WORKLOAD = "llama3.1-70b decode linear layers (qkv, o, gate_up, down; M in {1,8,
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode GEMM kernel, from the ncu
 # capture summarised in profiles/ (None until a capture exists for this kernel version).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
-NCU_TRAFFIC_NOTE = None
+NCU_TRAFFIC_RATIO = 172.40 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
+NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 168.06 MB read + 4.34 MB written for 168.23 MB algorithmic; "
+                    "scaled to the step's average launch by bytes processed (traffic is proportional to the weight bytes)")
 
 
 def gemm_bytes(M, N, K):
@@ -282,7 +283,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "gemm_kernel<64,1> (stream-K decode)", "achieved": gemm_gbs,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
                 "peak_source": f"of {peaks['source']}", "frac_of_nominal_8TBs": gemm_gbs / 8000.0,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "traffic_note": NCU_TRAFFIC_NOTE,
+                "traffic": NCU_TRAFFIC_RATIO * gemm_step_bytes / 12, "traffic_note": NCU_TRAFFIC_NOTE,
                 "algorithmic_bytes_per_launch_avg": gemm_step_bytes / 12,
                 "avg_launch_us": g_ms / g_n * 1e3}
     relayout_gbs = args.steps * sum(relayout_bytes(N, K) for _, K, N in inputs.LLAMA70B_PROJ) / (r_ms * 1e-3) / 1e9
@@ -501,8 +502,69 @@ def run_case(args):
     print(json.dumps({"case": args.case, "layout": args.layout, "launches": args.steps, "status": "ok"}), flush=True)
 
 
+def run_sweep(args):
+    """Config 5: N = K = 8192 bf16 weight, M in {1, 16, 128}; G x block aspect x CTA tile.
+    Prints one JSON line per (G, block, CTA tile): exact read amplification (row-major vs tile-major) and
+    GEMM time / throughput per M.  Weights rotate over three copies (403 MB) so every launch is L2-cold."""
+    from paper_2607_04031_b200 import binding as tl
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    K = N = 8192
+    copies = 3
+    W = [inputs.bf16_normal((K, N), 0.02, seed=700 + c, device=dev) for c in range(copies)]
+    Wt = [torch.empty_like(w) for w in W]
+    A = {M: inputs.bf16_normal((M, K), 1.0, seed=710 + M, device=dev) for M in (1, 16, 128)}
+    C = {M: torch.empty((M, N), dtype=torch.float32, device=dev) for M in (1, 16, 128)}
+
+    def timed(M, buf_list, g, br, bc, cta, reps=4):
+        evs = []
+        for rep in range(reps + 1):
+            for c in range(copies):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                tl.gemm(A[M], buf_list[c], C[M], M, N, K, g, br, bc, cta)
+                b.record()
+                if rep:
+                    evs.append((a, b))
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3      # us
+
+    ctas = ((64, 64, 64), (128, 128, 64), (256, 128, 64))
+    base = {}
+    for cta in ctas:
+        for M in (1, 16, 128):
+            base[cta, M] = timed(M, W, 0, 0, 0, cta)
+    for g in (32, 256, 1024, 4096, 16384):
+        for br in (1, 8, 16, 32):
+            bc = g // (2 * br)
+            if bc < 1:
+                print(json.dumps({"G": g, "block": [br, "G/(2*%d) < 1" % br], "skipped": "block row shorter than one element"}))
+                continue
+            for c in range(copies):
+                tl.relayout(W[c], Wt[c], K, N, 2, g, br, bc, tl.TO_TILE_MAJOR)
+            path = "row-major view" if br == 1 else ("tma" if br >= 8 and bc >= 64 else "generic-address")
+            for cta in ctas:
+                ra_t = tl.read_amp(128, N, K, cta, tl.LAYOUT_TILE_MAJOR, g, br, bc, 2)
+                ra_r = tl.read_amp(128, N, K, cta, tl.LAYOUT_ROW_MAJOR, g, 0, 0, 2)
+                row = {"G": g, "block": [br, bc], "cta": list(cta), "path": path,
+                       "read_amp_tile_major": ra_t[0] / ra_t[1], "read_amp_row_major": ra_r[0] / ra_r[1],
+                       "requests_per_load_tile_major": ra_t[2] // (ra_t[1] // (cta[2] * cta[1] * 2)),
+                       "requests_per_load_row_major": ra_r[2] // (ra_r[1] // (cta[2] * cta[1] * 2))}
+                try:
+                    for M in (1, 16, 128):
+                        us = timed(M, Wt, g, br, bc, cta)
+                        row[f"M{M}_us"] = round(us, 1)
+                        row[f"M{M}_GBps"] = round(gemm_bytes(M, N, K) / us / 1e3)
+                        row[f"M{M}_vs_row_major_time"] = round(us / base[cta, M], 3)
+                except tl.TileLensError as exc:
+                    row["gemm"] = f"unsupported: {exc}"
+                print(json.dumps(row), flush=True)
+    tl.device_status()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--sweep", action="store_true", help="layout/granularity sweep on an 8192 x 8192 weight")
     ap.add_argument("--case", default=None, choices=sorted(PROFILE_CASES),
                     help="run one small kernel case --steps times (for ncu); no benchmark line")
     ap.add_argument("--layout", default="tile", choices=["tile", "row"])
@@ -511,7 +573,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
-    if args.case:
+    if args.sweep:
+        run_sweep(args)
+    elif args.case:
         run_case(args)
     elif args.impl == "reference":
         run_reference(args)
