@@ -1,7 +1,6 @@
 // Host-side state of the tilelens library: stream, workspace, control block, error reporting.
 #include "tl_common.cuh"
 
-#include <mutex>
 
 namespace tl {
 
@@ -35,8 +34,14 @@ int ensure_control() {
     void* p = nullptr;
     if (int rc = check_cuda(cudaMalloc(&p, 256))) return rc;
     if (int rc = check_cuda(cudaMemset(p, 0, 256))) return rc;
+    void* h = nullptr;
+    if (int rc = check_cuda(cudaHostAlloc(&h, 64, cudaHostAllocMapped))) return rc;
+    void* h_dev = nullptr;
+    if (int rc = check_cuda(cudaHostGetDevicePointer(&h_dev, h, 0))) return rc;
     s.ctl.d_status = static_cast<uint32_t*>(p);
     s.ctl.d_acc = reinterpret_cast<unsigned long long*>(static_cast<char*>(p) + 64);
+    s.ctl.h_acc = static_cast<unsigned long long*>(h);
+    s.ctl.h_acc_dev = static_cast<unsigned long long*>(h_dev);
     return TL_OK;
 }
 

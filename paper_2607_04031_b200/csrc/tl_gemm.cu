@@ -161,6 +161,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, 
 // started, 5 last epilogue (and fix-up) done, 6 producer done.
 #ifdef TL_TIMELINE
 __device__ uint64_t* g_timeline = nullptr;
+__device__ int g_reverse = 0;
 #define TL_TIMELINE_INIT() uint64_t* const tl_tl = g_timeline ? g_timeline + blockIdx.x * 8 : nullptr; bool tl_once = true; (void)tl_once
 #define TL_STAMP(slot) do { if (tl_tl) tl_tl[(slot)] = global_timer_ns(); } while (0)
 #define TL_STAMP_ONCE(slot) do { if (tl_once) { tl_once = false; if (tl_tl) tl_tl[(slot)] = global_timer_ns(); } } while (0)
@@ -256,6 +257,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         abort_flag = 0;
         fence_mbar_init();
         if (!p.generic_b) tma_prefetch_desc(&p.tmap_b);
+        for (int i = 0; i < kNumBoxChoices; ++i) tma_prefetch_desc(&p.tmap_a[i]);
     }
     if (warp == 1) {
         tmem_alloc(&tmem_slot, tmem_cols);
@@ -281,7 +283,13 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     if (threadIdx.x == 0) TL_STAMP(1);
 
     Sched sched;
+#ifdef TL_TIMELINE
+    // measurement builds: optionally hand the ranges out in reverse CTA order; record the SM id
+    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, g_reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x);
+    if (threadIdx.x == 0 && tl_tl) { uint32_t smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); tl_tl[7] = smid; }
+#else
     sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x);
+#endif
     volatile uint32_t* abort_ptr = &abort_flag;
 
     if (warp == 0) {
@@ -493,19 +501,23 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 
             if (!full) {
                 // ---- stream-K fix-up: count arrivals; the last one adds the partials in K order.
-                __threadfence();
+                // The CTA barrier orders every epilogue thread's partial stores before thread 0's release
+                // (cumulative at GPU scope); the acquire half plus the second barrier orders the last
+                // arriver's loads after every other contributor's release.
                 epilogue_bar_sync();
                 const long long tile_begin = static_cast<long long>(w.tile) * p.k_iters;
                 const int c_lo = sched.owner(tile_begin);
                 const int c_hi = sched.owner(tile_begin + p.k_iters - 1);
                 if (et == 0) {
-                    uint32_t old = (ok && !*abort_ptr) ? atomicAdd(&p.counters[w.tile], 1u) : 0xFFFFFFFFu;
+                    uint32_t old = 0xFFFFFFFFu;
+                    if (ok && !*abort_ptr)
+                        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;"
+                                     : "=r"(old) : "l"(p.counters + w.tile) : "memory");
                     arrival_bcast = old;
                 }
                 epilogue_bar_sync();
                 const uint32_t old = arrival_bcast;
                 if (old == uint32_t(c_hi - c_lo)) {
-                    __threadfence();
                     // Partials are [row][kBN] floats; 128 threads walk them as float4, four vectors each per pass,
                     // adding the contributors in K order (c_lo first) whatever order they arrived in.
                     float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
@@ -516,18 +528,26 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                         float4 sum[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) sum[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int c = c_lo; c <= c_hi; ++c) {
-                            const float4* src = reinterpret_cast<const float4*>(
-                                p.partials + size_t(sched.slot(c, w.tile)) * slot_floats);
-                            float4 x[4];
+                        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {     // four contributors' loads in flight together
+                            float4 x[4][4];
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const int v = v0 + q * 128 + et;
-                                x[q] = v < total_vec ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            for (int j = 0; j < 4; ++j) {
+                                const bool c_ok = c0 + j <= c_hi;
+                                const float4* src = reinterpret_cast<const float4*>(
+                                    p.partials + size_t(sched.slot(c_ok ? c0 + j : c_lo, w.tile)) * slot_floats);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const int v = v0 + q * 128 + et;
+                                    x[j][q] = (c_ok && v < total_vec) ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
                             }
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                sum[q].x += x[q].x; sum[q].y += x[q].y; sum[q].z += x[q].z; sum[q].w += x[q].w;
+                            for (int j = 0; j < 4; ++j) {
+                                if (c0 + j > c_hi) break;                 // absent contributors add nothing (not even +0)
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    sum[q].x += x[j][q].x; sum[q].y += x[j][q].y; sum[q].z += x[j][q].z; sum[q].w += x[j][q].w;
+                                }
                             }
                         }
 #pragma unroll
@@ -973,5 +993,8 @@ extern "C" int tl_gemm_noalloc(const void* d_A, const void* d_B, float* d_C, int
 // Measurement builds only: d_buf holds 8 uint64 per CTA (zeroed by the caller); nullptr switches it off.
 extern "C" int tl_debug_set_timeline(void* d_buf) {
     return tl::check_cuda(cudaMemcpyToSymbol(tl::g_timeline, &d_buf, sizeof d_buf));
+}
+extern "C" int tl_debug_set_reverse(int on) {
+    return tl::check_cuda(cudaMemcpyToSymbol(tl::g_reverse, &on, sizeof on));
 }
 #endif

@@ -2,8 +2,9 @@
 //
 // For the GEMM's tile schedule it counts, per weight-tile load, the distinct
 // G-byte blocks that hold bytes of the cta_k x cta_n rectangle.  One warp owns
-// one column of CTA tiles (one n-tile): its lanes split the work of every load
-// and warp shuffles add the pieces up.  The count is exact for any sizes:
+// one column of CTA tiles (one n-tile) for a group of eight K iterations: its
+// lanes split the lines of every load, warp shuffles pass interval ends between
+// neighbouring lines and add the pieces up.  The count is exact for any sizes:
 //   tile-major  a rectangle of the matrix covers a rectangle of the block grid;
 //   row-major   row r of the rectangle covers the block interval [lo_r, hi_r];
 //               both ends never decrease with r, so the union grows by
@@ -21,7 +22,10 @@ struct ReadAmpParams {
     int layout;
     int64_t n_tiles, k_iters;
     int64_t m_tiles;                 // multiplier for totals / replication for per-tile output
-    unsigned long long* d_acc;       // [fetched, used, requests] totals (may be null)
+    unsigned long long* d_acc;       // [fetched, used, requests, ticket] totals (may be null); zero between launches
+    unsigned long long* h_out;       // mapped pinned host memory: the last warp publishes the totals here
+    unsigned long long total_ctas;
+    int64_t iters_per_warp;          // K iterations one warp covers
     unsigned long long* d_fetched;   // per CTA tile (may be null)
     unsigned long long* d_used;
 };
@@ -32,17 +36,24 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
     return v;
 }
 
+constexpr int kItersPerWarp = 8;     // row-/column-major: K iterations one warp covers (tile-major: all of them)
+
 __global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
     const int lane = threadIdx.x & 31;
     const int64_t warp = (blockIdx.x * int64_t(blockDim.x) + threadIdx.x) >> 5;
-    if (warp >= p.n_tiles) return;
-    const int64_t n0 = warp * p.BN;
+    __shared__ unsigned long long cta_blocks[4], cta_used[4];
+    const int64_t k_chunks = (p.k_iters + p.iters_per_warp - 1) / p.iters_per_warp;
+    const bool has_work = warp < p.n_tiles * k_chunks;
+    const int64_t tn = has_work ? warp / k_chunks : 0, kc = has_work ? warp % k_chunks : 0;
+    const int64_t n0 = tn * p.BN;
     const int64_t n1 = n0 + p.BN < p.N ? n0 + p.BN : p.N;
+    const int64_t it0 = kc * p.iters_per_warp;
+    const int64_t it1 = !has_work ? it0 : (it0 + p.iters_per_warp < p.k_iters ? it0 + p.iters_per_warp : p.k_iters);
 
-    unsigned long long blocks = 0;   // this lane's share of the distinct blocks, all K iterations
+    unsigned long long blocks = 0;   // this lane's share of the distinct blocks of these tile loads
     if (p.layout == TL_LAYOUT_TILE_MAJOR) {
         const unsigned long long across = (unsigned long long)((n1 - 1) / p.bc - n0 / p.bc + 1);
-        for (int64_t it = lane; it < p.k_iters; it += 32) {
+        for (int64_t it = it0 + lane; it < it1; it += 32) {
             const int64_t k0 = it * p.BK;
             const int64_t k1 = k0 + p.BK < p.K ? k0 + p.BK : p.K;
             blocks += (unsigned long long)((k1 - 1) / p.br - k0 / p.br + 1) * across;
@@ -51,37 +62,55 @@ __global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
         // Lines of the rectangle: its rows (row-major, pitch N*s) or its columns (col-major, pitch K*s).
         const bool rowm = p.layout == TL_LAYOUT_ROW_MAJOR;
         const int64_t pitch = (rowm ? p.N : p.K) * p.s;
-        for (int64_t it = 0; it < p.k_iters; ++it) {
+        for (int64_t it = it0; it < it1; ++it) {
             const int64_t k0 = it * p.BK;
             const int64_t k1 = k0 + p.BK < p.K ? k0 + p.BK : p.K;
             const int64_t line0 = rowm ? k0 : n0, line1 = rowm ? k1 : n1;   // lines of this load
             const int64_t seg0 = (rowm ? n0 : k0) * p.s;                     // first byte inside a line
             const int64_t seg1 = (rowm ? n1 : k1) * p.s - 1;                 // last byte inside a line
-            for (int64_t l = line0 + lane; l < line1; l += 32) {
-                const int64_t lo = (l * pitch + seg0) / p.G;
-                const int64_t hi = (l * pitch + seg1) / p.G;
+            for (int64_t base = line0; base < line1; base += 32) {
+                const int64_t l = base + lane;
+                const bool active = l < line1;
+                const int64_t lo = active ? (l * pitch + seg0) / p.G : 0;
+                const int64_t hi = active ? (l * pitch + seg1) / p.G : 0;
+                // last block of the previous line: from the lane below, or computed by lane 0
+                int64_t hi_prev = __shfl_up_sync(0xffffffffu, hi, 1);
+                if (lane == 0 && l > line0) hi_prev = ((l - 1) * pitch + seg1) / p.G;
                 int64_t first_new = lo;
-                if (l > line0) {
-                    const int64_t hi_prev = ((l - 1) * pitch + seg1) / p.G;
-                    if (hi_prev + 1 > first_new) first_new = hi_prev + 1;
-                }
-                if (hi >= first_new) blocks += (unsigned long long)(hi - first_new + 1);
+                if (l > line0 && hi_prev + 1 > first_new) first_new = hi_prev + 1;
+                if (active && hi >= first_new) blocks += (unsigned long long)(hi - first_new + 1);
             }
         }
     }
     blocks = warp_sum(blocks);
-    if (lane != 0) return;
     const unsigned long long fetched = blocks * (unsigned long long)p.G;
-    const unsigned long long used = (unsigned long long)(p.K * (n1 - n0) * p.s);
-    if (p.d_acc) {
-        atomicAdd(&p.d_acc[0], fetched * (unsigned long long)p.m_tiles);
-        atomicAdd(&p.d_acc[1], used * (unsigned long long)p.m_tiles);
-        atomicAdd(&p.d_acc[2], blocks * (unsigned long long)p.m_tiles);
+    const int64_t k_lo = it0 * p.BK, k_hi = it1 * p.BK < p.K ? it1 * p.BK : p.K;
+    const unsigned long long used = has_work ? (unsigned long long)((k_hi - k_lo) * (n1 - n0) * p.s) : 0ull;
+    if (lane == 0) {
+        cta_blocks[threadIdx.x >> 5] = blocks;
+        cta_used[threadIdx.x >> 5] = used;
+        if (has_work && p.d_fetched && p.d_used) {      // zeroed by the host before the launch
+            for (int64_t tm = 0; tm < p.m_tiles; ++tm) {
+                atomicAdd(&p.d_fetched[tm * p.n_tiles + tn], fetched);
+                atomicAdd(&p.d_used[tm * p.n_tiles + tn], used);
+            }
+        }
     }
-    if (p.d_fetched && p.d_used) {
-        for (int64_t tm = 0; tm < p.m_tiles; ++tm) {
-            p.d_fetched[tm * p.n_tiles + warp] = fetched;
-            p.d_used[tm * p.n_tiles + warp] = used;
+    __syncthreads();
+    if (threadIdx.x == 0 && p.d_acc) {
+        unsigned long long b = 0, u = 0;
+        for (int w = 0; w < 4; ++w) { b += cta_blocks[w]; u += cta_used[w]; }
+        atomicAdd(&p.d_acc[0], b * (unsigned long long)p.G * (unsigned long long)p.m_tiles);
+        atomicAdd(&p.d_acc[1], u * (unsigned long long)p.m_tiles);
+        atomicAdd(&p.d_acc[2], b * (unsigned long long)p.m_tiles);
+        // The CTA that takes the last ticket publishes the totals to the host and leaves the
+        // accumulators at zero for the next launch: no memset before and no copy after the kernel.
+        __threadfence();
+        if (atomicAdd(&p.d_acc[3], 1ull) == p.total_ctas - 1) {
+            __threadfence();
+            for (int i = 0; i < 3; ++i) p.h_out[i] = atomicExch(&p.d_acc[i], 0ull);
+            p.d_acc[3] = 0;
+            __threadfence_system();
         }
     }
 }
@@ -110,9 +139,17 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
     p.k_iters = ceil_div(K, cta_k);
     p.m_tiles = m_tiles;
     p.d_acc = d_acc; p.d_fetched = d_fetched; p.d_used = d_used;
+    p.h_out = d_acc ? state().ctl.h_acc_dev : nullptr;
+    p.iters_per_warp = layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
     if (m_tiles == 0) return TL_OK;
     const int warps_per_cta = 4;
-    const int64_t grid = ceil_div(p.n_tiles, warps_per_cta);
+    const int64_t grid = ceil_div(p.n_tiles * ceil_div(p.k_iters, p.iters_per_warp), warps_per_cta);
+    p.total_ctas = (unsigned long long)grid;
+    if (d_fetched && d_used) {
+        const size_t bytes = size_t(m_tiles) * p.n_tiles * sizeof(unsigned long long);
+        if (int rc = check_cuda(cudaMemsetAsync(d_fetched, 0, bytes, stream))) return rc;
+        if (int rc = check_cuda(cudaMemsetAsync(d_used, 0, bytes, stream))) return rc;
+    }
     read_amp_kernel<<<unsigned(grid), warps_per_cta * 32, 0, stream>>>(p);
     return check_cuda(cudaGetLastError());
 }
@@ -122,12 +159,16 @@ static int read_amp_totals(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
     if (!fetched || !used) return TL_ERR_INVALID_ARG;
     if (int rc = ensure_control()) return rc;
     State& st = state();
-    if (int rc = check_cuda(cudaMemsetAsync(st.ctl.d_acc, 0, 3 * sizeof(unsigned long long), st.stream))) return rc;
+    if (m_tiles == 0) {
+        *fetched = *used = 0;
+        if (requests) *requests = 0;
+        return TL_OK;
+    }
     if (int rc = read_amp_launch(m_tiles, N, K, cta_n, cta_k, layout, G, br, bc, s, st.ctl.d_acc, nullptr, nullptr,
                                  st.stream))
         return rc;
-    unsigned long long h[3] = {0, 0, 0};
-    if (int rc = check_cuda(cudaMemcpyAsync(h, st.ctl.d_acc, sizeof h, cudaMemcpyDeviceToHost, st.stream))) return rc;
+    // the kernel's last warp wrote the totals into mapped pinned memory; the only wait is this one
+    volatile unsigned long long* h = st.ctl.h_acc;
     if (int rc = check_cuda(cudaStreamSynchronize(st.stream))) return rc;
     *fetched = h[0];
     *used = h[1];

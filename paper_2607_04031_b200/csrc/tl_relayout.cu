@@ -47,10 +47,9 @@ __device__ __forceinline__ int64_t tile_major_byte(const RelayoutParams& p, int6
 
 // kPiece = min(16, bytes of one block row): granularity at which the tile-major side is contiguous.
 template <int kPiece>
-__global__ void __launch_bounds__(kRelayoutThreads) relayout_kernel(const RelayoutParams p) {
+__global__ void __launch_bounds__(kRelayoutThreads, 4) relayout_kernel(const RelayoutParams p) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int tile_cols = 1 << p.tile_cols_log2;        // bytes
-    const int tile_rows = 1 << p.tile_rows_log2;
     const int srow = tile_cols + kRowPad;               // shared-memory row pitch
     const int chunks_per_row_log2 = p.tile_cols_log2 - 4;
 
@@ -213,7 +212,7 @@ int relayout_launch(const void* d_src, void* d_dst, int64_t rows, int64_t cols, 
 
     const int64_t pitch = cols * s;
     const int64_t run = int64_t(bc) * s;
-    const bool fast = (pitch % 16 == 0) && (a % 16 == 0) && (b % 16 == 0) && G >= 16 && rows < (int64_t(1) << 40);
+    const bool fast = (pitch % 16 == 0) && (a % 16 == 0) && (b % 16 == 0) && G >= 16;
     if (!fast) {
         const int64_t total = rows * cols;
         const int grid = int(total / 256 + 1 < int64_t(sms) * 16 ? total / 256 + 1 : int64_t(sms) * 16);
