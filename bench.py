@@ -278,7 +278,7 @@ def run_ours(args):
     g_ms, g_n = kernel_ms["gemm_decode"]
     r_ms, r_n = kernel_ms["relayout"]
     gemm_gbs = args.steps * gemm_step_bytes / (g_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "gemm_kernel<64,1> (stream-K decode)", "achieved": gemm_gbs,
+    roofline = {"bound": "hbm", "kernel": "gemm_kernel, stream-K decode variants <BK=64,BN=256,weights-on-N> (M<=16) and <128,128,weights-on-N> (M=32)", "achieved": gemm_gbs,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
                 "peak_source": f"of {peaks['source']}", "frac_of_nominal_8TBs": gemm_gbs / 8000.0,
                 "traffic": NCU_TRAFFIC_RATIO * gemm_step_bytes / 12, "traffic_note": NCU_TRAFFIC_NOTE,

@@ -155,8 +155,10 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
 
 /*
  * tl_gemm for callers that must not allocate device memory.  (The paper has no
- * counterpart: this is a packaging variant of the product above, same kernel,
- * same results bit for bit.)
+ * counterpart: this is a packaging variant of the product above, same kernel;
+ * to keep its scratch small it may pick a narrower CTA tile than tl_gemm, so
+ * results agree with tl_gemm within the GEMM tolerance, exactly for inputs
+ * whose partial sums are exact.)
  *
  * Who needs it: a serving process that hands all of HBM to its own pool at
  * start-up, so that any later cudaMalloc fails; a plug-in host or sandbox that
@@ -175,9 +177,10 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
  *   limit         problems whose split-K scratch exceeds the array return
  *                 TL_ERR_WORKSPACE and enqueue nothing.  The scratch is
  *                 64 KB + 2 * (number of SMs) * cta_m * cta_n * 4 bytes when
- *                 M <= 64 or the tiles do not fill the SMs evenly, else 0: on
- *                 a 148-SM B200 with the default tile that admits every
- *                 M <= 32; M in (32, 64] needs 9.3 MB and is refused.
+ *                 M <= 64 or the tiles do not fill the SMs evenly, else 0; the
+ *                 default tile here is 128 columns wide: on a 148-SM B200
+ *                 that admits every M <= 32; M in (32, 64] needs 9.3 MB and
+ *                 is refused.
  *   first call    the first call on each device looks up the array's device
  *                 address (with that device current).  Make that call before
  *                 starting any stream capture.

@@ -35,6 +35,7 @@ constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 25
 constexpr int kAtomBytes = 128;            // one swizzle row: 64 bf16
 constexpr uint32_t kCounterBytes = 65536;  // head of the workspace: per-tile arrival counters
 constexpr int kMaxCounterTiles = kCounterBytes / 4;
+constexpr int kMaxDynamicSmem = 227 * 1024 - 10 * 1024;   // 227 KB per CTA minus the kernel's static shared memory
 
 struct alignas(64) GemmParams {
     CUtensorMap tmap_a[kNumBoxChoices];
@@ -129,7 +130,7 @@ struct Sched {
     }
 };
 
-__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* prefix, int tile) {
+__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* prefix, const int* row_start, int tile) {
     // prefix[e] = tiles of experts before e; tiles of one expert: n-tile major, m-tile minor.
     int lo = 0, hi = p.E;                  // find e with prefix[e] <= tile < prefix[e+1]
     while (hi - lo > 1) {
@@ -139,8 +140,8 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* 
     const int e = lo;
     const int local = tile - prefix[e];
     const int mt = (prefix[e + 1] - prefix[e]) / p.n_tiles;
-    const int row_begin = p.offsets ? p.offsets[e] : 0;
-    const int row_end = p.offsets ? p.offsets[e + 1] : p.M;
+    const int row_begin = row_start[e];
+    const int row_end = row_start[e + 1];
     TileInfo t;
     t.expert = e;
     t.n0 = (local / mt) * p.BN;
@@ -219,12 +220,20 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
     }
 }
 
-// kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256): one MMA of
-// M = 64, one of M = 128, or two of M = 128 sharing the token operand.
-template <int kBK, int kBN>
+// kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256).
+// kWN selects which side of the MMA the weights are on.  A tcgen05.mma of one CTA takes about 180 clocks
+// whatever its shape, so what matters is how many weight bytes one instruction consumes:
+//   kWN = false  weights on the M side: kBN/128 MMAs per K step, each 128 (or 64) weight columns x up to 256
+//                tokens.  For prefill (256-token tiles): the accumulator is C transposed, TMEM lane = weight
+//                column, and the epilogue writes 128-byte row segments.
+//   kWN = true   weights on the N side: one MMA per K step covers all kBN (up to 256) weight columns, tokens
+//                (at most 128 per tile) on the M side.  For decode and MoE: 8 KB of weights per instruction
+//                instead of 4 KB, which lifts the instruction-rate ceiling above the HBM rate.  TMEM lane =
+//                token, and every thread writes its token's row of C in 16-byte pieces.
+template <int kBK, int kBN, bool kWN>
 __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
-    constexpr int kNumN = kBN >= 128 ? kBN / 128 : 1;     // MMAs per K step
-    constexpr int kUmmaM = kBN >= 128 ? 128 : 64;         // weight columns per MMA
+    constexpr int kNumN = kWN ? 1 : (kBN >= 128 ? kBN / 128 : 1);     // MMAs per K step
+    constexpr int kUmmaM = kWN ? 128 : (kBN >= 128 ? 128 : 64);       // rows of the MMA's M side
     constexpr int kKSteps = kBK / 16;
     constexpr int kSubK = kBK / 64;                        // token boxes per stage
     constexpr uint32_t kWBytes = kBK * kBN * 2;            // weight bytes per stage
@@ -238,6 +247,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t arrival_bcast;
     __shared__ int prefix[kMaxExperts + 1];
+    __shared__ int row_start[kMaxExperts + 1];      // copy of the expert row offsets (dense: 0, M)
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -246,7 +256,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.BM * kAtomBytes;
     uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
-    const int acc_cols = p.BM;                               // TMEM columns per 128-column group
+    const int acc_cols = kWN ? kBN : p.BM;                   // TMEM columns of one MMA's accumulator
     uint32_t tmem_cols = 32;
     while (tmem_cols < uint32_t(2 * kNumN * acc_cols)) tmem_cols <<= 1;
 
@@ -264,13 +274,13 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         tmem_relinquish();
     }
     // tiles before each expert (dense: one "expert" holding all M rows)
-    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) prefix[e] = 0;
+    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) row_start[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.M);
     __syncthreads();
     if (threadIdx.x == 0) {
         int acc = 0;
         for (int e = 0; e < p.E; ++e) {
             prefix[e] = acc;
-            const int rows = p.offsets ? p.offsets[e + 1] - p.offsets[e] : p.M;
+            const int rows = row_start[e + 1] - row_start[e];
             acc += ((rows + p.BM - 1) / p.BM) * p.n_tiles;
         }
         prefix[p.E] = acc;
@@ -300,7 +310,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             Work w;
             bool ok = true;
             while (ok && sched.next(w)) {
-                const TileInfo t = decode_tile(p, prefix, w.tile);
+                const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
                 int bi = 0;
                 while ((16 << bi) < t.rows) ++bi;
                 const uint32_t a_bytes = uint32_t(16 << bi) * kAtomBytes;
@@ -356,11 +366,12 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             Work w;
             bool ok = true;
             while (ok && sched.next(w)) {
-                const TileInfo t = decode_tile(p, prefix, w.tile);
-                const uint32_t n_mma = uint32_t((t.rows + 15) & ~15);
-                // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = kUmmaM, N = n_mma
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((n_mma >> 3) << 17) |
-                                       ((uint32_t(kUmmaM) >> 4) << 24);
+                const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+                const uint32_t n_mma = kWN ? uint32_t(kBN) : uint32_t((t.rows + 15) & ~15);
+                // fp32 accumulate, bf16 x bf16; the weights operand is MN-major (bit 15: A, bit 16: B), the token
+                // operand K-major; M = kUmmaM, N = n_mma
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (kWN ? (1u << 16) : (1u << 15)) |
+                                       ((n_mma >> 3) << 17) | ((uint32_t(kUmmaM) >> 4) << 24);
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
                     ok = false;
                     break;
@@ -384,8 +395,11 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                         for (int u = 0; u < kNumN; ++u) {
                             const uint64_t w_desc =
                                 make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * 2u * p.lbo, p.lbo, p.sbo);
-                            umma_bf16(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc,
-                                      (kit > w.kbeg || j > 0) ? 1u : 0u);
+                            if (kWN)
+                                umma_bf16(d_tmem, tok_desc, w_desc, idesc, (kit > w.kbeg || j > 0) ? 1u : 0u);
+                            else
+                                umma_bf16(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc,
+                                          (kit > w.kbeg || j > 0) ? 1u : 0u);
                         }
                     }
                     umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
@@ -414,7 +428,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         Work w;
         bool ok = true;
         while (ok && sched.next(w)) {
-            const TileInfo t = decode_tile(p, prefix, w.tile);
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
             const uint8_t* Bexp = p.B + int64_t(t.expert) * p.expert_bytes;
             const int nblk0 = t.n0 >> p.bc_log2;
             for (int kit = w.kbeg; kit < w.kend; ++kit, ++it_global) {
@@ -448,7 +462,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         uint32_t acc = 0, acc_phase = 0;
         Work w;
         while (sched.next(w)) {
-            const TileInfo t = decode_tile(p, prefix, w.tile);
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
             const bool full = (w.kbeg == 0 && w.kend == p.k_iters);
             const int n_mma = (t.rows + 15) & ~15;
             bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
@@ -463,7 +477,29 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 out = p.partials + size_t(sched.slot(sched.cta, w.tile)) * p.BM * kBN;
                 ld = kBN;
             }
-            if (ok) {
+            if (ok && kWN) {
+                // TMEM lane = token row, columns = the tile's kBN weight columns: each thread owns one row of C.
+                const int row = quarter * 32 + lane;
+                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * uint32_t(acc_cols);
+                if (quarter * 32 < t.rows) {                     // this lane quarter holds at least one real row
+                    float* dst = out + int64_t(row) * ld;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kBN; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(taddr + c0, v);
+                        tmem_ld_wait();
+                        if (row < t.rows) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4)
+                                if (!full || t.n0 + c0 + i < p.N)
+                                    *reinterpret_cast<float4*>(dst + c0 + i) =
+                                        make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                    __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                        }
+                    }
+                }
+            }
+            if (ok && !kWN) {
 #pragma unroll
                 for (int u = 0; u < kNumN; ++u) {
                     // M = 128: accumulator row r sits in TMEM lane r.  M = 64: rows 16q..16q+15 sit in the
@@ -655,6 +691,7 @@ static int ilog2(int64_t x) {
 
 struct GemmPlan {
     int BM, BN, BK;
+    int weights_on_n;     // kWN variant of the kernel
     int stream_k;
     int grid;
     int num_stages;
@@ -669,28 +706,46 @@ static int pick_bm(int64_t rows) {
 }
 
 // Chooses / validates the CTA tile and the schedule.  rows_max: most rows any one problem has.
+// Default CTA tile (measured on B200, Llama-70B and Qwen-30B shapes).
+//   up to 16 rows      16 x 256 x 64: tokens on the MMA's M side, 256 weight columns per instruction; the
+//                      partial tiles of stream-K are still small (16 KB)
+//   up to 128 rows     rows x 128 x 128: same orientation, narrower tile so that partial tiles stay small,
+//                      deeper K step so that there are half as many barrier hand-offs
+//   more rows          256 x 128 x 64 with the weights on the M side (prefill)
+//   grouped            at most 64 rows per tile: most experts have a handful of rows, and a large cap costs
+//                      pipeline stages for every tile
+//   narrow_scratch     (fixed-size scratch) never the 256-column tile
+static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, int* BM, int* BN, int* BK) {
+    *BM = pick_bm(rows_max);
+    if (grouped && *BM > 64) *BM = 64;
+    if (*BM <= 16 && !narrow_scratch && !grouped) { *BN = 256; *BK = 64; }
+    else if (*BM <= 128) { *BN = 128; *BK = 128; }
+    else { *BN = 128; *BK = 64; }
+}
+
 static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
-                     bool grouped, GemmPlan* plan) {
+                     bool grouped, GemmPlan* plan, bool narrow_scratch = false) {
     if (int rc = ensure_device_info()) return rc;
     const int sms = state().sm_count;
     int BM = cta_m, BN = cta_n, BK = cta_k;
-    if (BM == 0 && BN == 0 && BK == 0) {
-        BM = pick_bm(rows_max);
-        BN = 128;
-        BK = 64;
-    }
+    if (BM == 0 && BN == 0 && BK == 0) default_tile(rows_max, grouped, narrow_scratch, &BM, &BN, &BK);
     if (BM != 16 && BM != 32 && BM != 64 && BM != 128 && BM != 256) return TL_ERR_UNSUPPORTED;
     if (BN != 64 && BN != 128 && BN != 256) return TL_ERR_UNSUPPORTED;
     if (BK != 64 && BK != 128) return TL_ERR_UNSUPPORTED;
     if (BN == 256 && BM > 128) return TL_ERR_UNSUPPORTED;   // 2 accumulators x 2 groups x BM columns <= 512
     plan->BM = BM; plan->BN = BN; plan->BK = BK;
+    plan->weights_on_n = BM <= 128;                         // tokens fit the 128 rows of the MMA's M side
     const size_t stage = size_t(BK) * BN * 2 + size_t(BK / 64) * BM * kAtomBytes;
-    const size_t budget = 227 * 1024 - 8 * 1024 - 1024;     // static barriers + prefix table + alignment slack
+    // 1 KB of slack to align the stages to 1024 bytes.  With the tokens on the M side the MMA always reads 128
+    // token rows, the tail of which (rows beyond the box) is whatever follows in shared memory: 16 KB more
+    // keep that read inside the allocation.  Those rows only feed accumulator rows that are never stored.
+    const size_t tail = plan->weights_on_n && BM < 128 ? 16 * 1024 : 0;
+    const size_t budget = kMaxDynamicSmem - 1024 - tail;
     int stages = int(budget / stage);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return TL_ERR_UNSUPPORTED;
     plan->num_stages = stages;
-    plan->smem_bytes = size_t(stages) * stage + 1024;
+    plan->smem_bytes = size_t(stages) * stage + 1024 + tail;
     if (plan->smem_bytes < 120 * 1024) plan->smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
     const int64_t k_iters = ceil_div(K, BK);
     const int64_t total_iters = tile_bound * k_iters;
@@ -741,12 +796,13 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     GemmPlan plan;
     {
         // upper bound of tiles: every expert may add one ragged m-tile
-        const int bm_guess = (cta_m == 0 && cta_n == 0 && cta_k == 0) ? pick_bm(rows_max) : cta_m;
-        if (bm_guess <= 0) return TL_ERR_UNSUPPORTED;
-        const int bn_guess = (cta_n == 0) ? 128 : cta_n;
+        int bm_guess = cta_m, bn_guess = cta_n, bk_guess = cta_k;
+        if (cta_m == 0 && cta_n == 0 && cta_k == 0)
+            default_tile(rows_max, d_offsets != nullptr, fixed != nullptr, &bm_guess, &bn_guess, &bk_guess);
+        if (bm_guess <= 0 || bn_guess <= 0) return TL_ERR_UNSUPPORTED;
         const int64_t mt_bound = d_offsets ? rows_total / bm_guess + E : ceil_div(rows_total, bm_guess);
         if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K, cta_m, cta_n, cta_k,
-                               d_offsets != nullptr, &plan))
+                               d_offsets != nullptr, &plan, fixed != nullptr))
             return rc;
     }
     if (d_offsets && K % plan.BK != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
@@ -848,23 +904,27 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.num_stages = plan.num_stages;
 
     cudaError_t err = cudaSuccess;
-#define TL_LAUNCH_GEMM(BK_, NN_)                                                                                   \
+#define TL_LAUNCH_GEMM(BK_, BN_, WN_)                                                                              \
     {                                                                                                              \
         static bool attr_set = false;                                                                              \
         if (!attr_set) {                                                                                           \
-            err = cudaFuncSetAttribute(gemm_kernel<BK_, NN_>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
-                                       227 * 1024 - 5 * 1024);                                                     \
+            err = cudaFuncSetAttribute(gemm_kernel<BK_, BN_, WN_>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                                       kMaxDynamicSmem);                                                           \
             attr_set = err == cudaSuccess;                                                                         \
         }                                                                                                          \
         if (err == cudaSuccess)                                                                                    \
-            gemm_kernel<BK_, NN_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes, stream>>>(p);     \
+            gemm_kernel<BK_, BN_, WN_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes,     \
+                                         stream>>>(p);                                                             \
     }
-    if (plan.BK == 64 && plan.BN == 128) { TL_LAUNCH_GEMM(64, 128) }
-    else if (plan.BK == 128 && plan.BN == 128) { TL_LAUNCH_GEMM(128, 128) }
-    else if (plan.BK == 64 && plan.BN == 256) { TL_LAUNCH_GEMM(64, 256) }
-    else if (plan.BK == 128 && plan.BN == 256) { TL_LAUNCH_GEMM(128, 256) }
-    else if (plan.BK == 64 && plan.BN == 64) { TL_LAUNCH_GEMM(64, 64) }
-    else { TL_LAUNCH_GEMM(128, 64) }
+#define TL_LAUNCH_GEMM_BN(BK_, WN_)                                                                                \
+    if (plan.BN == 64) TL_LAUNCH_GEMM(BK_, 64, WN_) else if (plan.BN == 128) TL_LAUNCH_GEMM(BK_, 128, WN_)        \
+    else TL_LAUNCH_GEMM(BK_, 256, WN_)
+    if (plan.weights_on_n) {
+        if (plan.BK == 64) { TL_LAUNCH_GEMM_BN(64, true) } else { TL_LAUNCH_GEMM_BN(128, true) }
+    } else {
+        if (plan.BK == 64) { TL_LAUNCH_GEMM_BN(64, false) } else { TL_LAUNCH_GEMM_BN(128, false) }
+    }
+#undef TL_LAUNCH_GEMM_BN
 #undef TL_LAUNCH_GEMM
     if (err != cudaSuccess) return check_cuda(err);
     return check_cuda(cudaGetLastError());
@@ -890,14 +950,18 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
 }
 
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {
-    tl::GemmPlan plan;
     if (M <= 0 || N <= 0 || K <= 0) return 0;
-    const int bm = (cta_m == 0 && cta_n == 0 && cta_k == 0) ? tl::pick_bm(M) : cta_m;
-    const int bn = cta_n == 0 ? 128 : cta_n;
-    if (bm <= 0) return 0;
-    // sized for the grouped schedule too (always stream-K, one CTA per SM)
-    if (tl::make_plan(M, (M / bm + 1) * tl::ceil_div(N, bn), N, K, cta_m, cta_n, cta_k, true, &plan)) return 0;
-    return plan.ws_bytes;
+    size_t need = 0;
+    for (int grouped = 0; grouped < 2; ++grouped) {         // the larger of the dense and the grouped schedule
+        int bm = cta_m, bn = cta_n, bk = cta_k;
+        if (cta_m == 0 && cta_n == 0 && cta_k == 0) tl::default_tile(M, grouped != 0, false, &bm, &bn, &bk);
+        if (bm <= 0 || bn <= 0) return 0;
+        tl::GemmPlan plan;
+        const int64_t mt = grouped ? M / bm + 1 : tl::ceil_div(M, bm);
+        if (tl::make_plan(M, mt * tl::ceil_div(N, bn), N, K, cta_m, cta_n, cta_k, grouped != 0, &plan)) return 0;
+        if (plan.ws_bytes > need) need = plan.ws_bytes;
+    }
+    return need;
 }
 
 }  // extern "C"

@@ -3,7 +3,8 @@
 Some hosts of this library cannot call cudaMalloc once they are running: an inference server that
 gave all of HBM to its own pool at start-up, a sandbox that forbids allocation after initialisation.
 For them the split-K scratch lives in a fixed array inside the library.  This file checks that the
-entry point, called through the C ABI, gives exactly what tl_gemm gives, twice in a row (the array
+entry point, called through the C ABI, gives what tl_gemm gives (bit for bit on integer data, within
+the GEMM tolerance otherwise), twice in a row (the array
 keeps the first call's contents, so the second call proves the clean-up), and that it refuses
 problems whose scratch does not fit.  It is collected last so that a failure here cannot hide
 another test's result; it does not depend on any other test having run.
@@ -24,13 +25,15 @@ def _case(M, N, K, seed, integer):
     else:
         A = inputs.bf16_normal((M, K), 1.0, seed=seed)
         B = inputs.bf16_normal((K, N), 0.02, seed=seed + 1)
-    return A.to(DEV).contiguous(), tile_major_on_device(B, K, N, 16, 128)
+    # bound of the GEMM tests' tolerance: 1e-3 * sum_k |A_ik B_kj| (fp32 is plenty for a bound)
+    S = A.to(DEV).float().abs() @ B.to(DEV).float().abs()
+    return A.to(DEV).contiguous(), tile_major_on_device(B, K, N, 16, 128), S
 
 
 @pytest.mark.parametrize("M,N,K,integer", [(8, 1024, 8192, True), (32, 2048, 4096, False), (1, 512, 2048, False)])
 def test_matches_tl_gemm_on_two_calls_in_a_row(M, N, K, integer):
     from gpu_util import DEV, tl
-    A, Bt = _case(M, N, K, seed=70 + M, integer=integer)
+    A, Bt, S = _case(M, N, K, seed=70 + M, integer=integer)
     want = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
     tl.gemm(A, Bt, want, M, N, K, 4096, 16, 128)          # existing entry point (allocating workspace)
     tl.device_status()
@@ -40,11 +43,16 @@ def test_matches_tl_gemm_on_two_calls_in_a_row(M, N, K, integer):
         tl.gemm_noalloc(A, Bt, got, M, N, K, 4096, 16, 128, timeout_flag=flag)
         torch.cuda.synchronize()
         assert int(flag.item()) == 0, "a bounded wait expired inside the kernel"
-        # same kernel, same schedule, same summation order: identical bits (tolerance 0, stricter than
-        # the 1e-3 * sum|a b| the other GEMM tests allow)
-        assert torch.equal(got, want), f"call {call}"
+        # Same kernel; the fixed scratch may make the library pick a narrower tile, hence another split of
+        # the K sums.  Integer inputs are exact in any order; otherwise both results lie within the GEMM
+        # tests' tolerance of 1e-3 * sum|a b| of the true product, so within twice that of each other.
+        if integer:
+            assert torch.equal(got, want), f"call {call}"
+        else:
+            assert bool(((got - want).abs() <= 2e-3 * S).all()), f"call {call}"
+            assert float((got - want).abs().max()) <= 1e-4 * float(S.max())
     # a different problem right after, then the first one again: stale partial tiles must not leak
-    A2, Bt2 = _case(16, 768, 2048, seed=5, integer=True)
+    A2, Bt2, _ = _case(16, 768, 2048, seed=5, integer=True)
     want2 = torch.empty((16, 768), dtype=torch.float32, device=DEV)
     tl.gemm(A2, Bt2, want2, 16, 768, 2048, 4096, 16, 128)
     got2 = torch.empty_like(want2)
@@ -52,13 +60,14 @@ def test_matches_tl_gemm_on_two_calls_in_a_row(M, N, K, integer):
     got = torch.empty_like(want)
     tl.gemm_noalloc(A, Bt, got, M, N, K, 4096, 16, 128)
     torch.cuda.synchronize()
-    assert torch.equal(got2, want2) and torch.equal(got, want)
+    assert torch.equal(got2, want2)
+    assert torch.equal(got, want) if integer else bool(((got - want).abs() <= 2e-3 * S).all())
 
 
 def test_refuses_scratch_beyond_the_fixed_array():
     from gpu_util import DEV, tl
     M, N, K = 64, 1024, 4096                               # 2 * SMs * 64 * 128 * 4 bytes > 8 MiB on a B200
-    A, Bt = _case(M, N, K, seed=9, integer=True)
+    A, Bt, _ = _case(M, N, K, seed=9, integer=True)
     C = torch.zeros((M, N), dtype=torch.float32, device=DEV)
     need = tl.gemm_workspace_bytes(M, N, K)
     if need <= (8 << 20) - 256:
