@@ -22,6 +22,7 @@
 // Every mbarrier wait is bounded (see mbar_wait_bounded).
 #include "tl_common.cuh"
 
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -614,6 +615,10 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     }
 }
 
+}  // namespace tl
+#include "tl_gemm_pair.cuh"
+namespace tl {
+
 // ======================================================================== host
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -904,6 +909,36 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.num_stages = plan.num_stages;
 
     cudaError_t err = cudaSuccess;
+    // Large dense problems on TMA-readable weights: CTA pairs (cta_group::2 MMAs), see tl_gemm_pair.cuh.
+    static const bool no_pair = getenv("TL_NO_PAIR") && atoi(getenv("TL_NO_PAIR")) != 0;     // measurement switch
+    // Worth it once every cluster of the machine has at least one 256 x 256 tile; smaller problems keep the
+    // single-CTA kernel and its stream-K split.
+    if (!no_pair && !d_offsets && !generic && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
+        p.kbx == 1 && p.nbx == 1 && ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= state().sm_count) {
+        static int max_clusters = -1;
+        const int stages = int((kMaxDynamicSmem - 1024) / (64 * 128 * 2 + 128 * kAtomBytes));
+        p.num_stages = stages < kPairStagesMax ? stages : kPairStagesMax;
+        const size_t smem = size_t(p.num_stages) * (64 * 128 * 2 + 128 * kAtomBytes) + 1024;
+        if (max_clusters < 0) {
+            err = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            if (err != cudaSuccess) return check_cuda(err);
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * state().sm_count);
+            cfg.blockDim = dim3(kGemmThreads);
+            cfg.dynamicSmemBytes = smem;
+            int n = 0;
+            err = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel, &cfg);
+            if (err != cudaSuccess) return check_cuda(err);
+            max_clusters = n > 0 ? n : 1;
+        }
+        const int64_t pair_tiles = ceil_div(rows_total, 256) * ceil_div(N, 256);
+        const int clusters = int(pair_tiles < max_clusters ? pair_tiles : max_clusters);
+        if (getenv("TL_LOG"))
+            fprintf(stderr, "[tilelens] pair kernel: %lld tiles of 256x256, %d clusters (max active %d), %d stages, %zu B smem\n",
+                    (long long)pair_tiles, clusters, max_clusters, p.num_stages, smem);
+        gemm_pair_kernel<<<2 * clusters, kGemmThreads, smem, stream>>>(p);
+        return check_cuda(cudaGetLastError());
+    }
 #define TL_LAUNCH_GEMM(BK_, BN_, WN_)                                                                              \
     {                                                                                                              \
         static bool attr_set = false;                                                                              \

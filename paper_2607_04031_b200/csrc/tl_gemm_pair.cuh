@@ -1,0 +1,300 @@
+// Prefill GEMM on CTA pairs (included by tl_gemm.cu after GemmParams and the helpers).
+//
+// A tcgen05.mma issued for one CTA (cta_group::1) takes about 180 clocks whatever its shape, which caps a
+// 128 x 256 x 16 instruction at ~70 % of the tensor peak.  The cta_group::2 form, one instruction spanning
+// the tensor cores of two SMs of a cluster (M = 256), measured 128 clocks for 256 x 256 x 16: the full rate.
+// So for large M two CTAs share one 256-token x 256-column output tile:
+//   - each CTA loads ITS 128 weight columns (the same one-box-per-stage tile-major view as the single-CTA
+//     kernel) and HALF of the 256 token rows; 32 KB per CTA per 64-row K step instead of 48 KB, six stages;
+//   - the even ("leader") CTA issues every MMA; the instruction reads the M-side operand (weights, 128 rows
+//     from each CTA) and the N-side operand (tokens, 128 rows from each CTA) out of both shared memories
+//     and writes 128 accumulator lanes x 256 columns into each CTA's tensor memory;
+//   - TMA completions of both CTAs count on the leader's "full" barrier, which the leader arms for the bytes
+//     of both (a cluster-scope arrive per stage from the peer measured ~600 clocks and starved the MMAs);
+//     tcgen05.commit is multicast so the
+//     "stage free" and "accumulator ready" barriers of both CTAs fire together; "accumulator drained"
+//     arrivals of both CTAs' epilogue warps go to the leader;
+//   - each CTA's epilogue stores its own 128 columns of C, exactly as in the single-CTA kernel.
+// No TMA multicast is used.  Every wait is on a barrier in the waiter's own shared memory and is bounded.
+#pragma once
+
+namespace tl {
+
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t num_clusters_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr),
+                 "r"(bytes)
+                 : "memory");
+}
+// TMA loads of a CTA pair: the bytes land in the issuing CTA's shared memory, the completion is counted on
+// the barrier at `bar_cluster_addr` (the leader's).
+__device__ __forceinline__ void tma_pair_load_2d(void* dst, const void* tmap, uint32_t bar_cluster_addr, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], "
+        "[%2];" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tma_pair_load_5d(void* dst, const void* tmap, uint32_t bar_cluster_addr, int c0, int c1,
+                                                 int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, "
+        "%5, %6, %7}], [%2];" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+__device__ __forceinline__ void umma_pair_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrives on the barrier at the same shared-memory offset in both CTAs once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_pair_commit_both(uint64_t* bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(smem_u32(bar)), "h"(uint16_t(3))
+        : "memory");
+}
+
+constexpr int kPairStagesMax = 8;
+constexpr int kPairBand = 8;      // m-tiles per band of the tile order
+
+// Tile order: bands of kPairBand m-tiles, inside a band the n-tile index moves slowest.  The clusters that run
+// together then cover about 8 x 9 tiles instead of 16 x 4.6: fewer operand bytes per wave (every cluster of a
+// wave re-reads the A rows of its m-tile and the B columns of its n-tile; what they share is fetched from HBM
+// once), and the band's A rows stay warm in L2 while the wave front moves along N.
+__device__ __forceinline__ void pair_tile_coords(int tile, int m_tiles, int n_tiles, int* m_tile, int* n_tile) {
+    const int band_tiles = kPairBand * n_tiles;
+    const int band = tile / band_tiles, r = tile - band * band_tiles;
+    const int band_rows = m_tiles - band * kPairBand < kPairBand ? m_tiles - band * kPairBand : kPairBand;
+    *m_tile = band * kPairBand + r % band_rows;
+    *n_tile = r / band_rows;
+}
+
+// One cluster = one 256-token x 256-column output tile at a time; CTA rank r owns columns n0 + 128 r .. + 127.
+// Dense problems only (no experts, no stream-K, TMA-readable weights); p.BM == 256, per-CTA tile 128 columns.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_pair_kernel(const __grid_constant__ GemmParams p) {
+    constexpr int kBK = 64, kKSteps = 4;
+    constexpr uint32_t kWBytes = kBK * 128 * 2;           // this CTA's weight slab per stage
+    constexpr uint32_t kTokBytes = 128 * kAtomBytes;      // this CTA's half of the token tile per stage
+    constexpr uint32_t kStageBytes = kWBytes + kTokBytes;
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kPairStagesMax];     // used in the leader only
+    __shared__ __align__(8) uint64_t empty_bar[kPairStagesMax];    // one copy per CTA
+    __shared__ __align__(8) uint64_t acc_full_bar[2];              // one copy per CTA
+    __shared__ __align__(8) uint64_t acc_empty_bar[2];             // used in the leader only
+    __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();
+    uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 8); }
+        abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&p.tmap_b);
+        tma_prefetch_desc(&p.tmap_a[3]);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(512)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync();                 // both CTAs' barriers are initialised before anyone touches the peer's
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    volatile uint32_t* abort_ptr = &abort_flag;
+
+    const int m_tiles = (p.M + 255) / 256;
+    const int n_pair_tiles = (p.N + 255) / 256;
+    const int tiles_total = m_tiles * n_pair_tiles;
+    const int first_tile = int(cluster_id_x()), tile_step = int(num_clusters_x());
+
+#ifdef TL_TIMELINE
+    uint64_t* const dbg = g_timeline ? g_timeline + blockIdx.x * 8 : nullptr;
+    long long w_wait = 0, w_issue = 0;
+#define TL_CLK() clock64()
+#else
+#define TL_CLK() 0ll
+#endif
+    if (warp == 0) {
+        // ============================================================ TMA producer (one per CTA)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, issued = 0;
+            bool ok = true;
+            const long long t_begin = TL_CLK();
+            (void)t_begin;
+            for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
+                int m_tile, n_tile;
+                pair_tile_coords(tile, m_tiles, n_pair_tiles, &m_tile, &n_tile);
+                const int n0 = n_tile * 256 + int(rank) * 128;      // this CTA's weight columns
+                const int row0 = m_tile * 256 + int(rank) * 128;    // this CTA's half of the tokens
+                for (int kit = 0; kit < p.k_iters; ++kit) {
+                    const long long c0 = TL_CLK();
+                    if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
+                        ok = false;
+                        break;
+                    }
+                    const long long c1 = TL_CLK();
+                    (void)c0; (void)c1;
+                    uint8_t* sw = stages + size_t(stage) * kStageBytes;
+                    // The leader's producer alone arms the barrier, for the bytes of BOTH CTAs; the peer only
+                    // issues its copies.  Their completions may be counted before the leader has armed the
+                    // phase (the byte count then goes negative for a moment); the phase cannot complete before
+                    // the arrival, and the peer cannot run a whole ring ahead because its "stage free" barrier
+                    // is only signalled after the leader's MMAs have consumed the stage.
+                    const uint32_t full_leader = map_to_cta(smem_u32(&full_bar[stage]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kStageBytes);
+                    const int k = kit * kBK;
+                    tma_pair_load_2d(sw + kWBytes, &p.tmap_a[3], full_leader, k, row0);
+                    if (p.row_major)
+                        tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k, n0 >> 6, 0, 0);
+                    else
+                        tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k & ((1 << p.br_log2) - 1),
+                                         (n0 & ((1 << p.bc_log2) - 1)) >> 6, n0 >> p.bc_log2, k >> p.br_log2);
+                    ++issued;
+#ifdef TL_TIMELINE
+                    w_wait += c1 - c0; w_issue += TL_CLK() - c1;
+#endif
+                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
+                }
+            }
+            (void)issued;
+#ifdef TL_TIMELINE
+            if (dbg) { dbg[0] = TL_CLK() - t_begin; dbg[1] = w_wait; dbg[2] = w_issue; dbg[7] = rank; }
+#endif
+        }
+    } else if (warp == 1) {
+        // ============================================================= MMA issuer (leader CTA only)
+        if (rank == 0 && lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = 256 over the pair, N = 256
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+            bool ok = true;
+            const long long t_begin = TL_CLK();
+            (void)t_begin;
+            for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
+                const long long a0 = TL_CLK();
+                if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) break;
+#ifdef TL_TIMELINE
+                w_issue += TL_CLK() - a0;      // (MMA thread: w_issue = cycles waiting for a free accumulator)
+#endif
+                (void)a0;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * 256u;
+                for (int kit = 0; kit < p.k_iters; ++kit) {
+                    const long long c0 = TL_CLK();
+                    if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull)) {
+                        ok = false;
+                        break;
+                    }
+#ifdef TL_TIMELINE
+                    w_wait += TL_CLK() - c0;
+#endif
+                    (void)c0;
+                    tc_fence_after_sync();
+                    const uint32_t sw = smem_u32(stages + size_t(stage) * kStageBytes);
+                    const uint32_t sa = sw + kWBytes;
+#pragma unroll
+                    for (int j = 0; j < kKSteps; ++j) {
+                        const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j], p.lbo, p.sbo);
+                        const uint64_t tok_desc = make_smem_desc(sa + uint32_t(j) * 32u, 16u, 1024u);
+                        umma_pair_bf16(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                    }
+                    umma_pair_commit_both(&empty_bar[stage]);       // frees the stage in both CTAs
+                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_pair_commit_both(&acc_full_bar[acc]);          // accumulator complete, both CTAs
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1;
+            }
+#ifdef TL_TIMELINE
+            if (dbg) { dbg[3] = TL_CLK() - t_begin; dbg[4] = w_wait; dbg[5] = w_issue; }
+#endif
+        }
+    } else {
+        // =============================================================== epilogue (both CTAs)
+        const int quarter = warp & 3;
+        uint32_t acc = 0, acc_phase = 0;
+        for (int tile = first_tile; tile < tiles_total; tile += tile_step) {
+            int m_tile, n_tile;
+            pair_tile_coords(tile, m_tiles, n_pair_tiles, &m_tile, &n_tile);
+            const int n0 = n_tile * 256 + int(rank) * 128;
+            const int row0 = m_tile * 256;
+            const int rows = p.M - row0 < 256 ? p.M - row0 : 256;
+            const bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
+            tc_fence_after_sync();
+            if (ok) {
+                const int n_local = quarter * 32 + lane;
+                const bool n_ok = n0 + n_local < p.N;
+                float* out = p.C + int64_t(row0) * p.ldc + n0;
+                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256u;
+                for (int c0 = 0; c0 < 256; c0 += 32) {
+                    if (c0 >= rows) break;
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(taddr + c0, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (n_ok && c0 + i < rows) out[int64_t(c0 + i) * p.ldc + n_local] = __uint_as_float(v[i]);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty_bar[acc]), 0));
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1;
+            if (*abort_ptr) break;
+        }
+    }
+
+    // Neither CTA may leave while its peer can still signal its barriers or read its shared memory.
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+}  // namespace tl

@@ -140,6 +140,26 @@ def test_granularity_sweep_layouts_every_cta_tile(G, br, bc):
             assert torch.isfinite(C).all()
 
 
+@pytest.mark.parametrize("br,bc", [(16, 128), (32, 64), (64, 64), (0, 0)])
+def test_cta_pair_kernel_ragged_shapes(br, bc):
+    # Large dense problems run on CTA pairs (256 x 256 tiles, cta_group::2 MMAs).  700 rows leave a 188-row
+    # tail tile; 9600 columns are 37.5 pair tiles, so the last pair has only its first CTA in range.
+    from gpu_util import DEV, run_gemm, tile_major_on_device
+    M, N, K = 700, 9600, 320
+    B = inputs.bf16_integers((K, N), -8, 8, seed=3)
+    Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
+    A = inputs.bf16_integers((M, K), -8, 8, seed=4)
+    C = run_gemm(A, Bd, M, N, K, br, bc)
+    assert torch.isfinite(C).all()
+    rng = np.random.default_rng(0)
+    ii = np.concatenate([rng.integers(0, M, 3000), np.full(64, M - 1), np.arange(M)])
+    jj = np.concatenate([rng.integers(0, N, 3000), np.arange(N - 64, N), np.full(M, N - 1)])
+    ref, _ = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), TILE if br else ROW, br, bc, M, N, K, ii, jj)
+    assert np.array_equal(C.cpu().numpy()[ii, jj].astype(np.float64), ref)
+    A1, ks = inputs.one_hot_rows(M, K, seed=5)
+    assert torch.equal(run_gemm(A1, Bd, M, N, K, br, bc).cpu(), B.float()[ks])
+
+
 def test_all_ones_B_gives_row_sums():
     from gpu_util import DEV, run_gemm, tile_major_on_device
     M, N, K = 8, 256, 4096
