@@ -107,10 +107,12 @@ int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, i
  *   Section 4.4 (plain loads with Eq. 1-2 arithmetic); there the memory tile
  *   must fit inside the CTA tile (block_rows | cta_k, block_cols | cta_n) and
  *   G >= 16, else TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
- * When M <= 64 (decode) the K loop of every output tile is cut stream-K
- * fashion over all SMs; partial tiles go through a workspace and are summed
- * in a fixed order, so results are reproducible run to run.  The workspace is
- * the caller's (tl_set_workspace) or one the library grows on demand.
+ * When the output tiles do not fill the SMs (decode, small or grouped
+ * problems) the K loops are cut stream-K fashion over all SMs; partial tiles
+ * go through a workspace and a second small kernel adds them in a fixed
+ * order, so results are reproducible run to run.  The workspace is the
+ * caller's (tl_set_workspace) or one the library grows on demand; calls that
+ * may run concurrently on one GPU must not share a workspace.
  * M == 0 is a no-op.
  */
 int tl_gemm(const void* d_A_rowmajor, const void* d_B_tilemajor, float* d_C,
@@ -166,8 +168,8 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
  * cannot afford the device-wide synchronisation an allocation or a free may
  * imply.  tl_gemm grows an internal workspace with cudaMalloc the first time a
  * decode-shaped problem needs split-K scratch; this entry point never calls
- * cudaMalloc, cudaFree or any allocating routine.  Its scratch (tile counters
- * and partial tiles) is a fixed array of TL_NOALLOC_SCRATCH_BYTES inside the
+ * cudaMalloc, cudaFree or any allocating routine.  Its scratch (the partial
+ * tiles of the split-K schedule) is a fixed array of TL_NOALLOC_SCRATCH_BYTES inside the
  * library image; every GPU that loads the library holds that much memory
  * until the process exits.
  *
@@ -176,7 +178,7 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
  *                 the kernel expires; NULL keeps the flag in the array, unread.
  *   limit         problems whose split-K scratch exceeds the array return
  *                 TL_ERR_WORKSPACE and enqueue nothing.  The scratch is
- *                 64 KB + 2 * (number of SMs) * cta_m * cta_n * 4 bytes when
+ *                 2 * (number of SMs) * cta_m * cta_n * 4 bytes when
  *                 M <= 64 or the tiles do not fill the SMs evenly, else 0; the
  *                 default tile here is 128 columns wide: on a 148-SM B200
  *                 that admits every M <= 32; M in (32, 64] needs 9.3 MB and
@@ -185,9 +187,9 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
  *                 address (with that device current).  Make that call before
  *                 starting any stream capture.
  *   sharing       all calls share the one array, and it keeps the previous
- *                 call's contents: the counters are cleared on cuda_stream at
- *                 the start of every call, the partial tiles are always
- *                 written before they are read.  Two calls that can run at
+ *                 call's contents; nothing in it has to start at zero, because
+ *                 every partial tile is written by the GEMM kernel before the
+ *                 reduction kernel of the same call reads it.  Two calls that can run at
  *                 the same time on one GPU (different streams, or different
  *                 host threads) race on the array and give wrong results:
  *                 serialise them.

@@ -67,8 +67,6 @@ int get_workspace(size_t bytes, void** out) {
         size_t want = bytes + (bytes >> 2);
         void* p = nullptr;
         if (int rc = check_cuda(cudaMalloc(&p, want))) return rc;
-        // Tile counters inside the workspace must start at zero; kernels leave them at zero.
-        if (int rc = check_cuda(cudaMemset(p, 0, want))) return rc;
         s.own_ws = p;
         s.own_ws_bytes = want;
     }
@@ -108,8 +106,6 @@ int tl_set_workspace(void* d_ptr, size_t bytes) {
         return TL_OK;
     }
     if (reinterpret_cast<uintptr_t>(d_ptr) % 256 != 0) return TL_ERR_ALIGNMENT;
-    // The split-K tile counters at the head of the workspace must start at zero.
-    if (int rc = tl::check_cuda(cudaMemset(d_ptr, 0, bytes < 65536 ? bytes : 65536))) return rc;
     s.user_ws = d_ptr;
     s.user_ws_bytes = bytes;
     return TL_OK;

@@ -34,8 +34,6 @@ constexpr int kMaxStages = 16;
 constexpr int kMaxExperts = 1024;
 constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 256 rows
 constexpr int kAtomBytes = 128;            // one swizzle row: 64 bf16
-constexpr uint32_t kCounterBytes = 65536;  // head of the workspace: per-tile arrival counters
-constexpr int kMaxCounterTiles = kCounterBytes / 4;
 constexpr int kMaxDynamicSmem = 227 * 1024 - 10 * 1024;   // 227 KB per CTA minus the kernel's static shared memory
 
 struct alignas(64) GemmParams {
@@ -43,7 +41,6 @@ struct alignas(64) GemmParams {
     CUtensorMap tmap_b;
     float* C;
     float* partials;            // stream-K partial tiles: slot = BM x BN floats
-    uint32_t* counters;         // per output tile, zero outside a launch
     const int32_t* offsets;     // grouped: device E+1 row offsets; dense: nullptr
     uint32_t* status;
     int64_t ldc;                // N
@@ -82,18 +79,23 @@ struct Work {
     int tile, kbeg, kend;
 };
 
+constexpr int kRangeTabMax = 256;      // CTAs whose range starts are tabulated in shared memory
+
 struct Sched {
     int stream_k, k_iters, tiles_total, grid_eff, cta;
     int next_tile;
     long long it, it_end, it_begin;
+    const int* tab;     // tab[c] = first flattened iteration of CTA c (grid_eff + 1 entries), or nullptr
 
+    // Even split of the flattened (tile, K iteration) space; a fixed function of the CTA index.
+    __device__ static long long split(long long total, int grid_eff, int c) { return (total * c) / grid_eff; }
     __device__ long long range_begin(int c) const {
-        return (static_cast<long long>(tiles_total) * k_iters * c) / grid_eff;
+        return tab ? tab[c] : split(static_cast<long long>(tiles_total) * k_iters, grid_eff, c);
     }
-    __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid, int cta_) {
-        stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_;
-        long long total = static_cast<long long>(tiles_total) * k_iters;
-        grid_eff = total < grid ? static_cast<int>(total) : grid;
+    __device__ static int effective_grid(long long total, int grid) { return total < grid ? static_cast<int>(total) : grid; }
+    __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid, int cta_, const int* tab_) {
+        stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_; tab = tab_;
+        grid_eff = effective_grid(static_cast<long long>(tiles_total) * k_iters, grid);
         next_tile = cta;
         if (grid_eff == 0 || cta >= grid_eff) { it = it_end = it_begin = 0; next_tile = tiles_total; return; }
         it_begin = it = range_begin(cta);
@@ -117,6 +119,14 @@ struct Sched {
     }
     // CTA whose range holds flattened iteration x.
     __device__ int owner(long long x) const {
+        if (tab) {                                   // largest c with tab[c] <= x
+            int lo = 0, hi = grid_eff;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (tab[mid] <= x) lo = mid; else hi = mid;
+            }
+            return lo;
+        }
         long long total = static_cast<long long>(tiles_total) * k_iters;
         int c = static_cast<int>(((x + 1) * grid_eff + total - 1) / total) - 1;
         if (c < 0) c = 0;
@@ -151,6 +161,31 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* 
     return t;
 }
 
+// Expert row offsets into shared memory (dense problems: one "expert" holding rows 0..M).
+__device__ __forceinline__ void load_row_starts(const GemmParams& p, int* row_start) {
+    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) row_start[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.M);
+}
+
+// prefix[e] = output tiles of the experts before e (n_tiles x m-tiles each); one warp, shuffle scan.
+__device__ __forceinline__ void tile_prefix(const GemmParams& p, const int* row_start, int* prefix) {
+    const int lane = threadIdx.x & 31;
+    int carry = 0;
+    for (int base = 0; base < p.E; base += 32) {
+        const int e = base + lane;
+        int v = 0;
+        if (e < p.E) v = ((row_start[e + 1] - row_start[e] + p.BM - 1) / p.BM) * p.n_tiles;
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (e < p.E) prefix[e] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) prefix[p.E] = carry;
+}
+
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
     // start address, leading and stride byte offsets in 16-byte units; descriptor version 1 (bit 46);
     // 128-byte swizzle (value 2 in bits 61..63)
@@ -167,7 +202,14 @@ __device__ int g_reverse = 0;
 #define TL_TIMELINE_INIT() uint64_t* const tl_tl = g_timeline ? g_timeline + blockIdx.x * 8 : nullptr; bool tl_once = true; (void)tl_once
 #define TL_STAMP(slot) do { if (tl_tl) tl_tl[(slot)] = global_timer_ns(); } while (0)
 #define TL_STAMP_ONCE(slot) do { if (tl_once) { tl_once = false; if (tl_tl) tl_tl[(slot)] = global_timer_ns(); } } while (0)
+// cycle counters per CTA (16 per CTA): 0 producer wait-empty, 1 producer issue, 2 stages issued, 3 MMA wait-full,
+// 4 MMA wait-accumulator, 5 MMA issue, 6 epilogue wait, 7 epilogue drain, 8 epilogue fix-up, 9 work items
+__device__ unsigned long long* g_counters = nullptr;
+#define TL_CLOCK() clock64()
+#define TL_COUNT(slot, v) do { if (g_counters) atomicAdd(&g_counters[blockIdx.x * 16 + (slot)], (unsigned long long)(v)); } while (0)
 #else
+#define TL_CLOCK() 0ll
+#define TL_COUNT(slot, v) do { } while (0)
 #define TL_TIMELINE_INIT() do { } while (0)
 #define TL_STAMP(slot) do { } while (0)
 #define TL_STAMP_ONCE(slot) do { } while (0)
@@ -246,14 +288,14 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     __shared__ __align__(8) uint64_t acc_empty_bar[2];
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
-    __shared__ uint32_t arrival_bcast;
     __shared__ int prefix[kMaxExperts + 1];
     __shared__ int row_start[kMaxExperts + 1];      // copy of the expert row offsets (dense: 0, M)
+    __shared__ int range_tab[kRangeTabMax + 1];     // stream-K: first flattened iteration of every CTA
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     TL_TIMELINE_INIT();
-    if (threadIdx.x == 0) TL_STAMP(0);
+    if (threadIdx.x == 0) { TL_STAMP(0); TL_COUNT(10, TL_CLOCK()); TL_COUNT(12, global_timer_ns()); }
     const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.BM * kAtomBytes;
     uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -275,31 +317,33 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         tmem_relinquish();
     }
     // tiles before each expert (dense: one "expert" holding all M rows)
-    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) row_start[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.M);
+    load_row_starts(p, row_start);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int e = 0; e < p.E; ++e) {
-            prefix[e] = acc;
-            const int rows = row_start[e + 1] - row_start[e];
-            acc += ((rows + p.BM - 1) / p.BM) * p.n_tiles;
-        }
-        prefix[p.E] = acc;
-    }
+    if (warp == 2) tile_prefix(p, row_start, prefix);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     const int tiles_total = prefix[p.E];
+    // Range starts of all CTAs, once, so that nothing on the critical path divides 64-bit numbers.
+    const long long total_iters = static_cast<long long>(tiles_total) * p.k_iters;
+    const int grid_eff0 = Sched::effective_grid(total_iters, gridDim.x);
+    const bool use_tab = p.stream_k && grid_eff0 > 0 && grid_eff0 <= kRangeTabMax && total_iters < (1ll << 31);
+    if (use_tab) {
+        for (int c = threadIdx.x; c <= grid_eff0; c += blockDim.x)
+            range_tab[c] = static_cast<int>(Sched::split(total_iters, grid_eff0, c));
+        __syncthreads();
+    }
     if (threadIdx.x == 0) TL_STAMP(1);
 
     Sched sched;
 #ifdef TL_TIMELINE
     // measurement builds: optionally hand the ranges out in reverse CTA order; record the SM id
-    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, g_reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x);
+    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, g_reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x,
+               use_tab ? range_tab : nullptr);
     if (threadIdx.x == 0 && tl_tl) { uint32_t smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); tl_tl[7] = smid; }
 #else
-    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x);
+    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
 #endif
     volatile uint32_t* abort_ptr = &abort_flag;
 
@@ -318,10 +362,13 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 const uint32_t tx = uint32_t(kSubK) * a_bytes + uint32_t(p.kbx * p.nbx) * p.box_bytes;
                 const int kc_expert = t.expert * p.k_coord_per_expert;
                 for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                    const long long cc0 = TL_CLOCK();
                     if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
                         ok = false;
                         break;
                     }
+                    const long long cc1 = TL_CLOCK();
+                    (void)cc0; (void)cc1;
                     uint8_t* sw = stages + size_t(stage) * stage_bytes;
                     uint8_t* sa = sw + kWBytes;
                     mbar_arrive_expect_tx(&full_bar[stage], tx);
@@ -344,6 +391,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                         }
                     }
                     ++issued;
+                    TL_COUNT(0, cc1 - cc0); TL_COUNT(1, TL_CLOCK() - cc1); TL_COUNT(2, 1);
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
                 }
             }
@@ -373,17 +421,23 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 // operand K-major; M = kUmmaM, N = n_mma
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (kWN ? (1u << 16) : (1u << 15)) |
                                        ((n_mma >> 3) << 17) | ((uint32_t(kUmmaM) >> 4) << 24);
+                const long long ca0 = TL_CLOCK();
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
                     ok = false;
                     break;
                 }
+                TL_COUNT(4, TL_CLOCK() - ca0);
+                (void)ca0;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * uint32_t(kNumN * acc_cols);
                 for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                    const long long cm0 = TL_CLOCK();
                     if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull)) {
                         ok = false;
                         break;
                     }
+                    const long long cm1 = TL_CLOCK();
+                    (void)cm0; (void)cm1;
                     tc_fence_after_sync();
                     TL_STAMP_ONCE(2);
                     const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
@@ -404,6 +458,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                         }
                     }
                     umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
+                    TL_COUNT(3, cm1 - cm0); TL_COUNT(5, TL_CLOCK() - cm1);
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
@@ -466,7 +521,10 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
             const bool full = (w.kbeg == 0 && w.kend == p.k_iters);
             const int n_mma = (t.rows + 15) & ~15;
+            const long long ce0 = TL_CLOCK();
             bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
+            const long long ce1 = TL_CLOCK();
+            (void)ce0; (void)ce1;
             tc_fence_after_sync();
             if (et == 0) TL_STAMP_ONCE(4);
             float* out;
@@ -533,75 +591,13 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty_bar[acc]);
+            const long long ce2 = TL_CLOCK();
+            (void)ce2;
+            if (et == 0) { TL_COUNT(6, ce1 - ce0); TL_COUNT(7, ce2 - ce1); TL_COUNT(9, 1); }
             acc ^= 1;
             if (acc == 0) acc_phase ^= 1;
 
-            if (!full) {
-                // ---- stream-K fix-up: count arrivals; the last one adds the partials in K order.
-                // The CTA barrier orders every epilogue thread's partial stores before thread 0's release
-                // (cumulative at GPU scope); the acquire half plus the second barrier orders the last
-                // arriver's loads after every other contributor's release.
-                epilogue_bar_sync();
-                const long long tile_begin = static_cast<long long>(w.tile) * p.k_iters;
-                const int c_lo = sched.owner(tile_begin);
-                const int c_hi = sched.owner(tile_begin + p.k_iters - 1);
-                if (et == 0) {
-                    uint32_t old = 0xFFFFFFFFu;
-                    if (ok && !*abort_ptr)
-                        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;"
-                                     : "=r"(old) : "l"(p.counters + w.tile) : "memory");
-                    arrival_bcast = old;
-                }
-                epilogue_bar_sync();
-                const uint32_t old = arrival_bcast;
-                if (old == uint32_t(c_hi - c_lo)) {
-                    // Partials are [row][kBN] floats; 128 threads walk them as float4, four vectors each per pass,
-                    // adding the contributors in K order (c_lo first) whatever order they arrived in.
-                    float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
-                    constexpr int kVecPerRow = kBN / 4;
-                    const int total_vec = t.rows * kVecPerRow;
-                    const size_t slot_floats = size_t(p.BM) * kBN;
-                    for (int v0 = 0; v0 < total_vec; v0 += 4 * 128) {
-                        float4 sum[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) sum[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {     // four contributors' loads in flight together
-                            float4 x[4][4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const bool c_ok = c0 + j <= c_hi;
-                                const float4* src = reinterpret_cast<const float4*>(
-                                    p.partials + size_t(sched.slot(c_ok ? c0 + j : c_lo, w.tile)) * slot_floats);
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const int v = v0 + q * 128 + et;
-                                    x[j][q] = (c_ok && v < total_vec) ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-                                }
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                if (c0 + j > c_hi) break;                 // absent contributors add nothing (not even +0)
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    sum[q].x += x[j][q].x; sum[q].y += x[j][q].y; sum[q].z += x[j][q].z; sum[q].w += x[j][q].w;
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int v = v0 + q * 128 + et;
-                            if (v < total_vec) {
-                                const int r = v / kVecPerRow, c4 = (v % kVecPerRow) * 4;
-                                if (t.n0 + c4 < p.N)
-                                    *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
-                            }
-                        }
-                    }
-                    if (et == 0) p.counters[w.tile] = 0;     // ready for the next launch
-                }
-                epilogue_bar_sync();                          // arrival_bcast may be rewritten after this
-            }
-            if (et == 0) TL_STAMP(5);
+            if (et == 0) { TL_STAMP(5); TL_COUNT(8, TL_CLOCK() - ce2); }
             if (*abort_ptr) break;
         }
     }
@@ -609,9 +605,78 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     // --------------------------------------------------------------- teardown
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) { TL_COUNT(11, TL_CLOCK()); TL_COUNT(13, global_timer_ns()); }
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// Stream-K reduction.  The GEMM kernel leaves the partial sum of every (CTA, split tile) in its workspace slot
+// and does no synchronisation of its own; this kernel, ordered after it by the stream, adds the partials of
+// each split tile in K order (lowest CTA first) and writes C.  One CTA per boundary between two ranges of
+// the GEMM grid: the boundary's tile is reduced by the first boundary that falls inside it.
+__global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_constant__ GemmParams p, int gemm_grid) {
+    __shared__ int prefix[kMaxExperts + 1];
+    __shared__ int row_start[kMaxExperts + 1];
+    // Launched with programmatic stream serialisation: this grid may be set up while the GEMM grid is still
+    // running; nothing the GEMM kernel wrote is read before this wait, which returns once that grid has
+    // completed and its writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    load_row_starts(p, row_start);
+    __syncthreads();
+    if (threadIdx.x < 32) tile_prefix(p, row_start, prefix);
+    __syncthreads();
+    Sched sched;
+    sched.init(1, p.k_iters, prefix[p.E], gemm_grid, 0, nullptr);
+    const int c = int(blockIdx.x) + 1;                     // boundary between CTA c-1 and CTA c
+    if (c >= sched.grid_eff) return;
+    const long long b = sched.range_begin(c);
+    const int tile = int(b / p.k_iters);
+    const long long tile_begin = static_cast<long long>(tile) * p.k_iters;
+    if (b == tile_begin) return;                           // the boundary coincides with a tile boundary
+    if (sched.range_begin(c - 1) > tile_begin) return;     // an earlier boundary lies in this tile: it reduces
+    const int c_lo = c - 1;
+    const int c_hi = sched.owner(tile_begin + p.k_iters - 1);
+    const TileInfo t = decode_tile(p, prefix, row_start, tile);
+    float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
+    const int vec_per_row = p.BN / 4;
+    const int total_vec = t.rows * vec_per_row;
+    const size_t slot_floats = size_t(p.BM) * p.BN;
+    for (int v0 = 0; v0 < total_vec; v0 += 4 * 128) {
+        float4 sum[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sum[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {         // four contributors' loads in flight together
+            float4 x[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool c_ok = c0 + j <= c_hi;
+                const float4* src =
+                    reinterpret_cast<const float4*>(p.partials + size_t(sched.slot(c_ok ? c0 + j : c_lo, tile)) * slot_floats);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int v = v0 + q * 128 + int(threadIdx.x);
+                    x[j][q] = (c_ok && v < total_vec) ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (c0 + j > c_hi) break;                  // absent contributors add nothing (not even +0)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    sum[q].x += x[j][q].x; sum[q].y += x[j][q].y; sum[q].z += x[j][q].z; sum[q].w += x[j][q].w;
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int v = v0 + q * 128 + int(threadIdx.x);
+            if (v < total_vec) {
+                const int r = v / vec_per_row, c4 = (v % vec_per_row) * 4;
+                if (t.n0 + c4 < p.N) *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
+            }
+        }
     }
 }
 
@@ -749,6 +814,10 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     int stages = int(budget / stage);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return TL_ERR_UNSUPPORTED;
+    if (const char* e = getenv("TL_MAX_STAGES")) {          // measurement hook
+        const int cap = atoi(e);
+        if (cap >= 2 && cap < stages) stages = cap;
+    }
     plan->num_stages = stages;
     plan->smem_bytes = size_t(stages) * stage + 1024 + tail;
     if (plan->smem_bytes < 120 * 1024) plan->smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
@@ -758,17 +827,16 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     const int64_t waves = ceil_div(tile_bound, sms);
     const bool even = tile_bound >= sms && double(tile_bound) / double(waves * sms) >= 0.92;
     plan->stream_k = (grouped || !even) ? 1 : 0;
-    if (tile_bound > kMaxCounterTiles) plan->stream_k = 0;
     int64_t grid = plan->stream_k ? (total_iters < sms ? total_iters : sms) : (tile_bound < sms ? tile_bound : sms);
     if (grid < 1) grid = 1;
     plan->grid = int(grid);
-    plan->ws_bytes = plan->stream_k ? kCounterBytes + size_t(2) * size_t(grid) * BM * BN * sizeof(float) : 0;
+    plan->ws_bytes = plan->stream_k ? size_t(2) * size_t(grid) * BM * BN * sizeof(float) : 0;   // two slots per CTA
     return TL_OK;
 }
 
 // Where a launch takes its scratch from when the caller of gemm_launch supplies it itself.
 struct FixedScratch {
-    void* ws;            // counters + partial tiles
+    void* ws;            // partial tiles
     size_t ws_bytes;
     uint32_t* status;    // word the kernel raises when a bounded wait expires
 };
@@ -815,10 +883,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (fixed) {
         if (plan.ws_bytes > fixed->ws_bytes) return TL_ERR_WORKSPACE;
         ws = plan.ws_bytes ? fixed->ws : nullptr;
-        // A fixed scratch keeps the previous launch's contents.  Partial tiles are always written before
-        // they are read; the tile counters must start at zero, so they are cleared on the same stream.
-        if (ws)
-            if (int rc = check_cuda(cudaMemsetAsync(ws, 0, kCounterBytes, stream))) return rc;
+        // A fixed scratch keeps the previous launch's contents; nothing in it has to start at zero: every
+        // partial tile is written by the GEMM kernel before the reduction kernel reads it.
     } else {
         if (int rc = ensure_control()) return rc;
         if (int rc = get_workspace(plan.ws_bytes, &ws)) return rc;
@@ -892,8 +958,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.kstep_off[j] = uint32_t(row / RB) * krow_bytes + uint32_t(row % RB) * kAtomBytes;
     }
     p.C = d_C;
-    p.counters = static_cast<uint32_t*>(ws);
-    p.partials = ws ? reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + kCounterBytes) : nullptr;
+    p.partials = static_cast<float*>(ws);
     p.offsets = d_offsets;
     p.status = fixed ? fixed->status : state().ctl.d_status;
     p.ldc = N;
@@ -960,6 +1025,19 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (plan.BK == 64) { TL_LAUNCH_GEMM_BN(64, false) } else { TL_LAUNCH_GEMM_BN(128, false) }
     }
 #undef TL_LAUNCH_GEMM_BN
+    // stream-K: add up the partial tiles, one CTA per boundary between two CTA ranges
+    if (err == cudaSuccess && plan.stream_k && plan.grid > 1) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(plan.grid - 1);
+        cfg.blockDim = dim3(128);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // overlap its launch with the GEMM grid
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, streamk_reduce_kernel, p, plan.grid);
+    }
 #undef TL_LAUNCH_GEMM
     if (err != cudaSuccess) return check_cuda(err);
     return check_cuda(cudaGetLastError());
@@ -1047,8 +1125,7 @@ int tl_gemm_host(const void* h_A, const void* h_B_rowmajor, float* h_C, int64_t 
 // ------------------------------------------------- scratch held in the library image
 namespace tl {
 
-// Split-K scratch of tl_gemm_noalloc: tile counters (first kCounterBytes), partial tiles, and in the
-// last 256 bytes a spare word for the time-out flag when the caller passes none.  Lives in the
+// Split-K scratch of tl_gemm_noalloc: partial tiles, and in the last 256 bytes a spare word for the time-out flag when the caller passes none.  Lives in the
 // module's data segment on every GPU that loads the library, from load until the process exits.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[TL_NOALLOC_SCRATCH_BYTES];
 
@@ -1092,6 +1169,9 @@ extern "C" int tl_gemm_noalloc(const void* d_A, const void* d_B, float* d_C, int
 // Measurement builds only: d_buf holds 8 uint64 per CTA (zeroed by the caller); nullptr switches it off.
 extern "C" int tl_debug_set_timeline(void* d_buf) {
     return tl::check_cuda(cudaMemcpyToSymbol(tl::g_timeline, &d_buf, sizeof d_buf));
+}
+extern "C" int tl_debug_set_counters(void* d_buf) {
+    return tl::check_cuda(cudaMemcpyToSymbol(tl::g_counters, &d_buf, sizeof d_buf));
 }
 extern "C" int tl_debug_set_reverse(int on) {
     return tl::check_cuda(cudaMemcpyToSymbol(tl::g_reverse, &on, sizeof on));
