@@ -334,6 +334,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             range_tab[c] = static_cast<int>(Sched::split(total_iters, grid_eff0, c));
         __syncthreads();
     }
+    // Stream-K: let the reduction kernel that follows in the stream be scheduled already; it does its own
+    // set-up and then blocks until this whole grid has finished.
+    if (p.stream_k && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) TL_STAMP(1);
 
     Sched sched;
@@ -619,10 +622,13 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_constant__ GemmParams p, int gemm_grid) {
     __shared__ int prefix[kMaxExperts + 1];
     __shared__ int row_start[kMaxExperts + 1];
-    // Launched with programmatic stream serialisation: this grid may be set up while the GEMM grid is still
-    // running; nothing the GEMM kernel wrote is read before this wait, which returns once that grid has
-    // completed and its writes are visible.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Launched with programmatic stream serialisation, and the GEMM kernel lets its dependents launch as soon
+    // as it has started: this grid is resident and has done all of its index arithmetic (which reads only
+    // the call's inputs) while the GEMM grid is still running.  Nothing the GEMM kernel wrote is read before
+    // griddepcontrol.wait, which returns once that grid has completed and its writes are visible.
+#ifdef TL_TIMELINE
+    if (threadIdx.x == 0 && g_timeline) g_timeline[(256 + blockIdx.x) * 8 + 0] = global_timer_ns();
+#endif
     load_row_starts(p, row_start);
     __syncthreads();
     if (threadIdx.x < 32) tile_prefix(p, row_start, prefix);
@@ -640,6 +646,14 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
     const int c_hi = sched.owner(tile_begin + p.k_iters - 1);
     const TileInfo t = decode_tile(p, prefix, row_start, tile);
     float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
+    // slots of the contributors, computed before the wait (the load loop below must not divide)
+    __shared__ int slot_of[kRangeTabMax];
+    for (int j = threadIdx.x; j <= c_hi - c_lo && j < kRangeTabMax; j += blockDim.x) slot_of[j] = sched.slot(c_lo + j, tile);
+    __syncthreads();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef TL_TIMELINE
+    if (threadIdx.x == 0 && g_timeline) g_timeline[(256 + blockIdx.x) * 8 + 1] = global_timer_ns();
+#endif
     const int vec_per_row = p.BN / 4;
     const int total_vec = t.rows * vec_per_row;
     const size_t slot_floats = size_t(p.BM) * p.BN;
@@ -652,8 +666,9 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const bool c_ok = c0 + j <= c_hi;
-                const float4* src =
-                    reinterpret_cast<const float4*>(p.partials + size_t(sched.slot(c_ok ? c0 + j : c_lo, tile)) * slot_floats);
+                const int jj = c_ok ? c0 + j - c_lo : 0;
+                const int slot = jj < kRangeTabMax ? slot_of[jj] : sched.slot(c_lo + jj, tile);
+                const float4* src = reinterpret_cast<const float4*>(p.partials + size_t(slot) * slot_floats);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int v = v0 + q * 128 + int(threadIdx.x);
@@ -678,6 +693,9 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
             }
         }
     }
+#ifdef TL_TIMELINE
+    if (threadIdx.x == 0 && g_timeline) g_timeline[(256 + blockIdx.x) * 8 + 2] = global_timer_ns();
+#endif
 }
 
 }  // namespace tl
@@ -810,7 +828,8 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     // token rows, the tail of which (rows beyond the box) is whatever follows in shared memory: 16 KB more
     // keep that read inside the allocation.  Those rows only feed accumulator rows that are never stored.
     const size_t tail = plan->weights_on_n && BM < 128 ? 16 * 1024 : 0;
-    const size_t budget = kMaxDynamicSmem - 1024 - tail;
+    // 12 KB stay free so that a CTA of the stream-K reduction kernel can be resident next to this one.
+    const size_t budget = kMaxDynamicSmem - 1024 - tail - 12 * 1024;
     int stages = int(budget / stage);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return TL_ERR_UNSUPPORTED;
