@@ -40,8 +40,8 @@ WORKLOAD = "llama3.1-70b decode linear layers (qkv, o, gate_up, down; M in {1,8,
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode GEMM kernel, from the ncu
 # capture summarised in profiles/ (None until a capture exists for this kernel version).
-NCU_TRAFFIC_RATIO = 172.40 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
-NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 168.06 MB read + 4.34 MB written for 168.23 MB algorithmic; "
+NCU_TRAFFIC_RATIO = 173.02 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
+NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 168.00 MB read + 5.02 MB written for 168.23 MB algorithmic; "
                     "scaled to the step's average launch by bytes processed (traffic is proportional to the weight bytes)")
 
 
@@ -237,7 +237,7 @@ def run_ours(args):
     step_bytes = sum(relayout_bytes(N, K) for _, K, N in inputs.LLAMA70B_PROJ) + \
         sum(gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
     gemm_step_bytes = sum(gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
-    launches_per_step = 4 + 12 + 12
+    launches_per_step = 4 + 12 * 2 + 12      # relayouts, GEMM + stream-K reduction per product, counters
 
     tl.set_stream(stream)
     for _ in range(max(3, args.warmup)):
