@@ -46,13 +46,18 @@ int ensure_device_info();
 // Workspace of at least `bytes` (user's if set, else internal, grown with cudaMalloc).
 int get_workspace(size_t bytes, void** out);
 
+// Encodes (and caches) a tiled tensor map; dtype / swizzle are CUtensorMapDataType / CUtensorMapSwizzle values,
+// strides_bytes[0] is the element size and is not passed to the driver.
+int encode_tensor_map(CUtensorMap* out, const void* base, int dtype, int swizzle, int rank, const uint64_t* dims,
+                      const uint64_t* strides_bytes, const uint32_t* box);
+
 inline bool is_pow2(int64_t x) { return x > 0 && (x & (x - 1)) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // Detail codes stored in the status word by kernels that give up.
 enum : uint32_t {
     kWaitProducerEmpty = 0x100, kWaitMmaFull = 0x200, kWaitMmaAccEmpty = 0x300,
-    kWaitEpilogueAccFull = 0x400, kWaitTeardown = 0x500
+    kWaitEpilogueAccFull = 0x400, kWaitTeardown = 0x500, kWaitRelayoutFull = 0x600
 };
 
 // ------------------------------------------------------------- device helpers
@@ -136,6 +141,37 @@ __device__ __forceinline__ void tma_load_5d(void* dst, const void* tmap, uint64_
         "%7}], [%2];" ::"r"(smem_u32(dst)),
         "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const void* tmap, uint64_t* bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const void* tmap, const void* src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+// Untiled bulk copies: both addresses 16-byte aligned, size a multiple of 16 bytes.
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store_1d(void* dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(reinterpret_cast<uint64_t>(dst)), "r"(smem_u32(src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Waits until at most kPending of this thread's committed bulk groups are still reading shared memory.
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_group_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
 }
 
 // ---- tcgen05 (5th-generation tensor cores, accumulators in tensor memory)

@@ -724,7 +724,7 @@ static EncodeTiledFn encode_fn() {
 // (pointer, shape, box) recurs on every call of a serving loop.
 struct MapKey {
     const void* base;
-    int rank;
+    int rank, dtype, swizzle;
     uint64_t dims[5], strides[5];
     uint32_t box[5];
     bool operator==(const MapKey& o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
@@ -735,14 +735,16 @@ struct MapEntry {
 };
 static constexpr int kMapCacheSize = 256;
 
-static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                  const uint32_t* box) {
+int encode_tensor_map(CUtensorMap* out, const void* base, int dtype, int swizzle, int rank, const uint64_t* dims,
+                      const uint64_t* strides_bytes, const uint32_t* box) {
     static MapEntry* cache = new MapEntry[kMapCacheSize];
     static int cache_n = 0, cache_next = 0;
     MapKey key;
     memset(&key, 0, sizeof key);
     key.base = base;
     key.rank = rank;
+    key.dtype = dtype;
+    key.swizzle = swizzle;
     for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.strides[i] = strides_bytes[i]; key.box[i] = box[i]; }
     for (int i = 0; i < cache_n; ++i)
         if (cache[i].key == key) {
@@ -758,8 +760,8 @@ static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* 
     cuuint32_t bdim[5], estr[5];
     for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bdim[i] = box[i]; estr[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i + 1];
-    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, cuuint32_t(rank), const_cast<void*>(base), gdim, gstr, bdim,
-                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    CUresult r = fn(out, CUtensorMapDataType(dtype), cuuint32_t(rank), const_cast<void*>(base), gdim, gstr, bdim, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CUtensorMapSwizzle(swizzle), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         state().last_cuda_error = int(r);
@@ -769,6 +771,13 @@ static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* 
     cache[slot].key = key;
     cache[slot].map = *out;
     return TL_OK;
+}
+
+// bf16 operands of the GEMM, 128-byte swizzle
+static int encode(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                  const uint32_t* box) {
+    return encode_tensor_map(out, base, int(CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), int(CU_TENSOR_MAP_SWIZZLE_128B), rank, dims,
+                             strides_bytes, box);
 }
 
 static int ilog2(int64_t x) {

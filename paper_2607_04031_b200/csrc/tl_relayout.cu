@@ -8,6 +8,9 @@
 // assembled from several shared-memory rows.
 #include "tl_common.cuh"
 
+#include <cstdlib>
+#include <cstring>
+
 namespace tl {
 
 constexpr int kRelayoutThreads = 256;
@@ -188,6 +191,140 @@ __global__ void relayout_elementwise_kernel(const uint8_t* __restrict__ src, uin
     }
 }
 
+
+// ------------------------------------------------------------------ TMA path
+// For block rows of 16 bytes to 1 KB and memory tiles of at most 32 KB the copy engine does the permutation by
+// itself.  The row-major matrix is described as a 3-D tensor of 32-bit words (words of a block row, matrix row,
+// block column): a box of (block row, br rows, nb block columns) is nb whole memory tiles, which TMA writes to
+// shared memory tile after tile: exactly their image in the tile-major buffer, where they are one contiguous
+// run of nb*G bytes.  So a step is one tensor copy on the row-major side and one untiled bulk copy on the
+// tile-major side (load then store, in the order the direction needs), one thread per CTA driving a ring of
+// 32 KB buffers.  No registers, no block-wide barriers.
+#ifndef TL_TMA_TILE
+#define TL_TMA_TILE 32768
+#endif
+#ifndef TL_TMA_STAGES
+#define TL_TMA_STAGES 3
+#endif
+#ifndef TL_TMA_CTAS
+#define TL_TMA_CTAS 2
+#endif
+constexpr int kTmaTileBytes = TL_TMA_TILE;
+constexpr int kTmaStages = TL_TMA_STAGES;        // ring of buffers per CTA
+constexpr int kTmaCtasPerSm = TL_TMA_CTAS;
+
+struct RelayoutTmaParams {
+    CUtensorMap row_map;     // row-major side
+    uint8_t* tile_base;      // tile-major side
+    uint32_t* status;
+    int64_t G;
+    int br, nb;              // rows of a memory tile, memory tiles per step
+    int blocks_per_row, block_rows;
+    int64_t steps_x, steps_total;
+    int to_tile_major;
+};
+
+__global__ void __launch_bounds__(32, kTmaCtasPerSm) relayout_tma_kernel(const __grid_constant__ RelayoutTmaParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_tma[];
+    __shared__ __align__(8) uint64_t full_bar[kTmaStages];
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x != 0) return;
+    uint8_t* bufs = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_tma) + 127) & ~uintptr_t(127));
+    for (int s = 0; s < kTmaStages; ++s) mbar_init(&full_bar[s], 1);
+    abort_flag = 0;
+    fence_mbar_init();
+    tma_prefetch_desc(&p.row_map);
+    volatile uint32_t* abort_ptr = &abort_flag;
+
+    const int64_t first = blockIdx.x, stride = gridDim.x;
+    const int64_t mine = first < p.steps_total ? (p.steps_total - first + stride - 1) / stride : 0;
+    auto issue_load = [&](int64_t i) {
+        const int64_t step = first + i * stride;
+        const int s = int(i % kTmaStages);
+        const int64_t brow = step / p.steps_x;
+        const int b0 = int(step % p.steps_x) * p.nb;
+        const int nbt = p.blocks_per_row - b0 < p.nb ? p.blocks_per_row - b0 : p.nb;
+        uint8_t* buf = bufs + size_t(s) * kTmaTileBytes;
+        if (p.to_tile_major) {
+            mbar_arrive_expect_tx(&full_bar[s], uint32_t(p.nb) * uint32_t(p.G));      // a box always counts in full
+            tma_load_3d(buf, &p.row_map, &full_bar[s], 0, int(brow) * p.br, b0);
+        } else {
+            mbar_arrive_expect_tx(&full_bar[s], uint32_t(nbt) * uint32_t(p.G));
+            bulk_load_1d(buf, p.tile_base + (brow * p.blocks_per_row + b0) * p.G, uint32_t(nbt) * uint32_t(p.G), &full_bar[s]);
+        }
+    };
+    const int64_t ahead = mine < kTmaStages - 1 ? mine : kTmaStages - 1;
+    for (int64_t i = 0; i < ahead; ++i) issue_load(i);
+    for (int64_t i = 0; i < mine; ++i) {
+        const int s = int(i % kTmaStages);
+        if (!mbar_wait_bounded(&full_bar[s], uint32_t(i / kTmaStages) & 1u, abort_ptr, p.status, kWaitRelayoutFull)) break;
+        const int64_t step = first + i * stride;
+        const int64_t brow = step / p.steps_x;
+        const int b0 = int(step % p.steps_x) * p.nb;
+        const int nbt = p.blocks_per_row - b0 < p.nb ? p.blocks_per_row - b0 : p.nb;
+        const uint8_t* buf = bufs + size_t(s) * kTmaTileBytes;
+        if (p.to_tile_major)
+            bulk_store_1d(p.tile_base + (brow * p.blocks_per_row + b0) * p.G, buf, uint32_t(nbt) * uint32_t(p.G));
+        else
+            tma_store_3d(&p.row_map, buf, 0, int(brow) * p.br, b0);       // the part of the box outside the matrix is not written
+        bulk_commit_group();
+        // The buffer the NEXT load goes to is the one whose store was committed one step ago.
+        if (i + kTmaStages - 1 < mine) {
+            bulk_wait_group_read<1>();
+            issue_load(i + kTmaStages - 1);
+        }
+    }
+    bulk_wait_group_read<0>();       // shared memory must outlive the last stores' reads
+}
+
+static int relayout_tma_launch(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int s, int64_t G, int br, int bc,
+                               int direction, cudaStream_t stream, bool* taken) {
+    *taken = false;
+    const int64_t run = int64_t(bc) * s, pitch = cols * s;
+    if (run < 16 || run > 1024 || G > kTmaTileBytes || br > 256) return TL_OK;
+    if (pitch % 16 != 0 || pitch >= (int64_t(1) << 40) || rows >= (int64_t(1) << 31)) return TL_OK;
+    const bool to_tile = direction == TL_TO_TILE_MAJOR;
+    const void* row_side = to_tile ? d_src : d_dst;
+    void* tile_side = to_tile ? d_dst : const_cast<void*>(d_src);
+    if (reinterpret_cast<uintptr_t>(row_side) % 16 != 0 || reinterpret_cast<uintptr_t>(tile_side) % 16 != 0) return TL_OK;
+    if (int rc = ensure_control()) return rc;
+    if (int rc = ensure_device_info()) return rc;
+    RelayoutTmaParams p;
+    memset(&p, 0, sizeof p);
+    int nb = int(kTmaTileBytes / G);
+    if (nb > 256) nb = 256;
+    const int64_t blocks_per_row = cols / bc;
+    if (nb > blocks_per_row) nb = int(blocks_per_row);
+    const uint64_t dims[3] = {uint64_t(run / 4), uint64_t(rows), uint64_t(blocks_per_row)};
+    const uint64_t strides[3] = {4, uint64_t(pitch), uint64_t(run)};
+    const uint32_t box[3] = {uint32_t(run / 4), uint32_t(br), uint32_t(nb)};
+    if (int rc = encode_tensor_map(&p.row_map, row_side, int(CU_TENSOR_MAP_DATA_TYPE_UINT32), int(CU_TENSOR_MAP_SWIZZLE_NONE), 3, dims,
+                                   strides, box))
+        return rc;
+    p.tile_base = static_cast<uint8_t*>(tile_side);
+    p.status = state().ctl.d_status;
+    p.G = G;
+    p.br = br;
+    p.nb = nb;
+    p.blocks_per_row = int(blocks_per_row);
+    p.block_rows = int(rows / br);
+    p.steps_x = ceil_div(blocks_per_row, nb);
+    p.steps_total = p.steps_x * (rows / br);
+    p.to_tile_major = to_tile;
+    const size_t smem = size_t(kTmaStages) * kTmaTileBytes + 128;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (int rc = check_cuda(cudaFuncSetAttribute(relayout_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))))
+            return rc;
+        attr_set = true;
+    }
+    const int64_t max_grid = int64_t(state().sm_count) * kTmaCtasPerSm;
+    const int grid = int(p.steps_total < max_grid ? p.steps_total : max_grid);
+    relayout_tma_kernel<<<grid, 32, smem, stream>>>(p);
+    *taken = true;
+    return check_cuda(cudaGetLastError());
+}
+
 static int ilog2(int64_t x) {
     int l = 0;
     while ((int64_t(1) << l) < x) ++l;
@@ -210,6 +347,15 @@ int relayout_launch(const void* d_src, void* d_dst, int64_t rows, int64_t cols, 
     if (int rc = ensure_device_info()) return rc;
     const int sms = state().sm_count;
 
+    {
+        // copy-engine path when the shape allows it (TL_RELAYOUT_NO_TMA=1 keeps the shared-memory kernel)
+        static const bool no_tma = getenv("TL_RELAYOUT_NO_TMA") && atoi(getenv("TL_RELAYOUT_NO_TMA")) != 0;
+        bool taken = false;
+        if (!no_tma) {
+            if (int rc = relayout_tma_launch(d_src, d_dst, rows, cols, s, G, br, bc, direction, stream, &taken)) return rc;
+            if (taken) return TL_OK;
+        }
+    }
     const int64_t pitch = cols * s;
     const int64_t run = int64_t(bc) * s;
     const bool fast = (pitch % 16 == 0) && (a % 16 == 0) && (b % 16 == 0) && G >= 16;
