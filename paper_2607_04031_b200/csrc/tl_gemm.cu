@@ -809,12 +809,12 @@ static int pick_bm(int64_t rows) {
 //   up to 128 rows     rows x 128 x 128: same orientation, narrower tile so that partial tiles stay small,
 //                      deeper K step so that there are half as many barrier hand-offs
 //   more rows          256 x 128 x 64 with the weights on the M side (prefill)
-//   grouped            at most 64 rows per tile: most experts have a handful of rows, and a large cap costs
-//                      pipeline stages for every tile
+//   grouped            at most 32 rows per tile: most experts have a handful of rows, and a large cap costs
+//                      pipeline stages and partial-tile bytes for every tile
 //   narrow_scratch     (fixed-size scratch) never the 256-column tile
 static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, int* BM, int* BN, int* BK) {
     *BM = pick_bm(rows_max);
-    if (grouped && *BM > 64) *BM = 64;
+    if (grouped && *BM > 32) *BM = 32;
     if (*BM <= 16 && !narrow_scratch && !grouped) { *BN = 256; *BK = 64; }
     else if (*BM <= 128) { *BN = 128; *BK = 128; }
     else { *BN = 128; *BK = 64; }

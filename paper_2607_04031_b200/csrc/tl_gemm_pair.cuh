@@ -275,7 +275,7 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (n_ok && c0 + i < rows) out[int64_t(c0 + i) * p.ldc + n_local] = __uint_as_float(v[i]);
+                        if (n_ok && c0 + i < rows) __stcs(out + int64_t(c0 + i) * p.ldc + n_local, __uint_as_float(v[i]));
                 }
             }
             tc_fence_before_sync();
