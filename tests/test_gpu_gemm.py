@@ -123,16 +123,17 @@ def _sweep_layouts():
 
 @pytest.mark.parametrize("G,br,bc", _sweep_layouts())
 def test_granularity_sweep_layouts_every_cta_tile(G, br, bc):
-    # Same layouts and CTA tiles as the sweep of the benchmark, on a 1024 x 8192 slice of its 8192 x 8192
-    # weight (bc goes up to 8192); integer data, so every sampled output must match the oracle exactly.
+    # Same layouts, CTA tiles, M and the full 8192 x 8192 weight of the benchmark's sweep; integer data, so
+    # every sampled output must match the oracle exactly.
     from gpu_util import DEV, run_gemm, tile_major_on_device, tl
-    K, N = 1024, 8192
-    B = inputs.bf16_integers((K, N), -8, 8, seed=G + br)
+    K, N = 8192, 8192
+    B = inputs.bf16_integers((K, N), -8, 8, seed=G + br, device=DEV)
     Bd = tile_major_on_device(B, K, N, br, bc)
     for M in (1, 16, 128):
         A = inputs.bf16_integers((M, K), -8, 8, seed=M)
         rng = np.random.default_rng(M)
-        ii, jj = rng.integers(0, M, 400), rng.integers(0, N, 400)
+        ii, jj = rng.integers(0, M, 150), rng.integers(0, N, 150)
+        ii[:2], jj[:2] = [0, M - 1], [0, N - 1]
         ref, _ = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), TILE, br, bc, M, N, K, ii, jj)
         for cta in ((64, 64, 64), (128, 128, 64), (256, 128, 64)):
             C = run_gemm(A, Bd, M, N, K, br, bc, cta)
@@ -196,20 +197,25 @@ def test_llama_decode_full_size_sampled(name, K, N, M):
     assert torch.equal(run_gemm(A, B, M, N, K, 0, 0), C)
 
 
-def test_llama_prefill_full_size_sampled():
+@pytest.mark.parametrize("name,K,N", inputs.LLAMA70B_PROJ)
+def test_llama_prefill_full_size_sampled(name, K, N):
     from gpu_util import DEV, check_against_oracle, run_gemm, sample_indices, tl
-    M, K, N = inputs.LLAMA_PREFILL_M, 8192, 10240
+    M = inputs.LLAMA_PREFILL_M
     A = inputs.bf16_normal((M, K), 1.0, seed=41, device=DEV)
     B = inputs.bf16_normal((K, N), 0.02, seed=42, device=DEV)
     Bt = torch.empty_like(B)
     tl.relayout(B, Bt, K, N, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
     C = run_gemm(A, Bt, M, N, K, 16, 128)
-    ii, jj = sample_indices(M, N, 3000, seed=4)
-    # plus one full row and one full column through every tile
-    ii = np.concatenate([ii, np.full(N, 1234), np.arange(M)])
-    jj = np.concatenate([jj, np.arange(N), np.full(M, 4321)])
-    check_against_oracle(C, A.cpu(), Bt, TILE, 16, 128, M, N, K, idx=(ii, jj))
+    ii, jj = sample_indices(M, N, 1500, seed=4)
+    # plus one full column and a strided row through every tile
+    cols = np.arange(0, N, 7)
+    ii = np.concatenate([ii, np.full(cols.size, 1234), np.arange(M)])
+    jj = np.concatenate([jj, cols, np.full(M, 4321)])
+    Cs = C[torch.from_numpy(ii).to(DEV), torch.from_numpy(jj).to(DEV)]
     assert torch.isfinite(C).all()
+    ref, S = tlo.matmul_at(inputs.bits(A.cpu()), inputs.bits(Bt.reshape(-1)), TILE, 16, 128, M, N, K, ii, jj)
+    err = np.abs(Cs.cpu().numpy().astype(np.float64) - ref)
+    assert np.all(err <= 1e-3 * S) and float(np.max(err / np.maximum(S, 1e-300))) <= 1e-4
 
 
 def _grouped_case(E, tokens, topk, K, N, br, bc, seed, cta=(0, 0, 0), integer=False):
