@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "tlo.c")
 _HDR = os.path.join(_HERE, "tlo.h")
 _LIB = os.path.join(_HERE, "libtlo.so")
 
-ROW_MAJOR, COL_MAJOR, TILE_MAJOR = 0, 1, 2
+ROW_MAJOR, COL_MAJOR, TILE_MAJOR, TILE_MAJOR_K = 0, 1, 2, 3
 TO_TILE_MAJOR, TO_ROW_MAJOR = 0, 1
 
 

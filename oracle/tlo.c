@@ -52,6 +52,8 @@ int64_t tlo_off(int layout, int64_t r, int64_t c, int64_t rows, int64_t cols,
                 int64_t br, int64_t bc, int64_t s) {
     if (layout == TLO_ROW_MAJOR) return tlo_off_row(r, c, rows, cols, s);
     if (layout == TLO_COL_MAJOR) return tlo_off_col(r, c, rows, cols, s);
+    /* Eq. 2 as printed: (r, c) = (i, j) of the K x N matrix, a = bc along K, b = br along N */
+    if (layout == TLO_TILE_MAJOR_K) return tlo_eq2(r, c, rows, cols, bc, br, s);
     return tlo_off_tile(r, c, rows, cols, br, bc, s);
 }
 
@@ -134,6 +136,7 @@ int tlo_matmul_at(const uint16_t* A, const uint16_t* B, int layout, int64_t br, 
                   int64_t M, int64_t N, int64_t K, int64_t n,
                   const int64_t* idx_i, const int64_t* idx_j, double* C, double* S) {
     if (layout == TLO_TILE_MAJOR && (br <= 0 || bc <= 0 || K % br != 0 || N % bc != 0)) return -1;
+    if (layout == TLO_TILE_MAJOR_K && (br <= 0 || bc <= 0 || K % bc != 0 || N % br != 0)) return -1;
     for (int64_t t = 0; t < n; ++t)
         if (idx_i[t] < 0 || idx_i[t] >= M || idx_j[t] < 0 || idx_j[t] >= N) return -1;
 #pragma omp parallel for schedule(dynamic, 16)
@@ -145,6 +148,7 @@ int tlo_matmul_at(const uint16_t* A, const uint16_t* B, int layout, int64_t br, 
 int tlo_matmul(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
                int64_t M, int64_t N, int64_t K, double* C, double* S) {
     if (layout == TLO_TILE_MAJOR && (br <= 0 || bc <= 0 || K % br != 0 || N % bc != 0)) return -1;
+    if (layout == TLO_TILE_MAJOR_K && (br <= 0 || bc <= 0 || K % bc != 0 || N % br != 0)) return -1;
 #pragma omp parallel for schedule(dynamic, 64)
     for (int64_t t = 0; t < M * N; ++t)
         dot_at(A, B, layout, br, bc, N, K, t / N, t % N, &C[t], &S[t]);
@@ -227,6 +231,9 @@ static int read_amp_args_ok(int64_t N, int64_t K, int64_t BM, int64_t BN, int64_
     if (layout == TLO_TILE_MAJOR) {
         if (br <= 0 || bc <= 0 || br * bc * s != G) return 0;     /* Section 3.1: h*w*s = G */
         if (K % br != 0 || N % bc != 0) return 0;                 /* Section 3.3 */
+    } else if (layout == TLO_TILE_MAJOR_K) {
+        if (br <= 0 || bc <= 0 || br * bc * s != G) return 0;
+        if (K % bc != 0 || N % br != 0) return 0;
     } else if (layout != TLO_ROW_MAJOR && layout != TLO_COL_MAJOR) {
         return 0;
     }

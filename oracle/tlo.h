@@ -30,7 +30,9 @@
 extern "C" {
 #endif
 
-enum { TLO_ROW_MAJOR = 0, TLO_COL_MAJOR = 1, TLO_TILE_MAJOR = 2 };
+/* TLO_TILE_MAJOR_K is the tile-major layout exactly as the paper prints it (Eq. 2): the K x N weight with K
+ * contiguous, memory tile a (along K) x b (along N); there br/bc of the calls below carry (b, a). */
+enum { TLO_ROW_MAJOR = 0, TLO_COL_MAJOR = 1, TLO_TILE_MAJOR = 2, TLO_TILE_MAJOR_K = 3 };
 enum { TLO_TO_TILE_MAJOR = 0, TLO_TO_ROW_MAJOR = 1 };
 
 /* Section 2.4: byte offset of element (r,c) of a rows x cols matrix of s-byte

@@ -167,3 +167,17 @@ def test_relayout_rejects_non_divisible_shapes():
     src = np.zeros(10 * 10, dtype=np.uint8)
     with pytest.raises(ValueError):
         tlo.relayout(src, 10, 10, 1, 4, 2, tlo.TO_TILE_MAJOR)
+
+
+def test_k_contiguous_flavour_is_eq2_and_the_transposed_relayout():
+    # Layout code TILE_MAJOR_K: the weight exactly as the paper prints it (K contiguous, a along K, b along N).
+    K, N, a, b, s = 64, 48, 16, 8, 2
+    for i in (0, 1, 15, 16, 63):
+        for j in (0, 7, 8, 47):
+            assert tlo.off(tlo.TILE_MAJOR_K, i, j, K, N, b, a, s) == tlo.eq2(i, j, K, N, a, b, s)
+    # relayout of the [N][K] array (K contiguous) with blocks of b rows x a columns produces that buffer
+    w = np.arange(K * N, dtype=np.uint16).reshape(N, K)            # w[j][i]: element (i, j)
+    buf = tlo.relayout(w.view(np.uint8), N, K, 2, b, a, tlo.TO_TILE_MAJOR).view(np.uint16)
+    for i in range(0, K, 5):
+        for j in range(0, N, 7):
+            assert buf[tlo.off(tlo.TILE_MAJOR_K, i, j, K, N, b, a, s) // 2] == w[j, i]

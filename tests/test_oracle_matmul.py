@@ -98,3 +98,14 @@ def test_sampled_product_equals_full_product():
     assert np.array_equal(Cs, C[ii, jj]) and np.array_equal(Ss, S[ii, jj])
     with pytest.raises(ValueError):
         tlo.matmul_at(inputs.bits(A), B_tile, tlo.TILE_MAJOR, br, bc, M, N, K, [M], [0])
+
+
+def test_k_contiguous_tile_major_gives_the_same_product():
+    M, N, K, a, b = 5, 96, 128, 64, 32                   # the paper's (64, 32) memory tile
+    A = inputs.bf16_normal((M, K), 1.0, seed=21)
+    B = inputs.bf16_normal((K, N), 0.02, seed=22)
+    want, _ = tlo.matmul(inputs.bits(A), inputs.bits(B), tlo.ROW_MAJOR, 0, 0, M, N, K)
+    w_nk = np.ascontiguousarray(inputs.bits(B).T)        # [N][K], K contiguous
+    buf = tlo.relayout(w_nk.view(np.uint8), N, K, 2, b, a, tlo.TO_TILE_MAJOR).view(np.uint16)
+    got, _ = tlo.matmul(inputs.bits(A), buf, tlo.TILE_MAJOR_K, b, a, M, N, K)
+    assert np.array_equal(got, want)

@@ -195,3 +195,19 @@ def test_bad_arguments_are_rejected():
         tlo.read_amp(1, 64, 64, 1, 64, 64, TILE, 4096, 16, 64, 2)      # 16*64*2 != 4096
     with pytest.raises(ValueError):
         tlo.read_amp(1, 60, 64, 1, 64, 64, TILE, 256, 8, 16, 2)        # N not a multiple of bc
+
+
+def test_k_contiguous_flavour_counts_like_the_transposed_problem():
+    # The paper's own example again (Section 6.5), now literally: K contiguous, memory tile (a, b) = (64, 32):
+    # a 128 (K) x 256 (N) compute tile of a K = 4096 weight needs 16 requests; column-major needs 256
+    # (one 4 KB block per column, pitch 8 KB).
+    K, N, s, G = 4096, 512, 2, 4096
+    f, u, q = tlo.read_amp(1, N, K, 1, 256, 128, tlo.TILE_MAJOR_K, G, 32, 64, s)
+    loads = (N // 256) * (K // 128)
+    assert q == 16 * loads and f == u
+    assert tlo.read_amp(1, N, K, 1, 256, 128, COL, G, 0, 0, s)[2] == 256 * loads
+    # transposition invariance ties the two flavours together
+    # (the K x N weight with K contiguous IS an N x K matrix with its columns contiguous: same blocks, tile loads
+    # with their two extents exchanged)
+    assert tlo.read_amp(3, N, K, 2, 96, 80, tlo.TILE_MAJOR_K, 512, 8, 32, s) == \
+        tlo.read_amp(3, K, N, 2, 80, 96, TILE, 512, 8, 32, s)
