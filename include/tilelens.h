@@ -50,7 +50,10 @@ typedef enum {
 } tl_status;
 
 typedef enum { TL_TO_TILE_MAJOR = 0, TL_TO_ROW_MAJOR = 1 } tl_direction;
-typedef enum { TL_LAYOUT_ROW_MAJOR = 0, TL_LAYOUT_COL_MAJOR = 1, TL_LAYOUT_TILE_MAJOR = 2 } tl_layout;
+/* TL_LAYOUT_TILE_MAJOR_K: the K-contiguous flavour, Eq. 2 exactly as printed; block_rows x block_cols is then
+ * the memory tile of the stored [N][K] array: b rows along N by a contiguous columns along K. */
+typedef enum { TL_LAYOUT_ROW_MAJOR = 0, TL_LAYOUT_COL_MAJOR = 1, TL_LAYOUT_TILE_MAJOR = 2,
+               TL_LAYOUT_TILE_MAJOR_K = 3 } tl_layout;
 
 /* ------------------------------------------------------------------ misc */
 
@@ -136,6 +139,24 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
                     int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
                     int cta_m, int cta_n, int cta_k, void* cuda_stream);
 
+/*
+ * The same products for weights stored the way deployments keep them (Section 2.4): [N][K] with K contiguous
+ * (the "column-major" K x N matrix), tile-major exactly as Eq. 2 prints it: memory tiles of tile_k contiguous
+ * K-elements (the paper's a) by tile_n rows along N (the paper's b), tile_n*tile_k*2 == G, tiles ordered along
+ * K first.  tile_n == 0: the plain [N][K] array.  tl_relayout(rows = N, cols = K, block_rows = tile_n,
+ * block_cols = tile_k) produces this buffer.  The weights are then the K-major operand of the MMA.
+ *   tile_k >= 64 (one 128-byte swizzle row), K % 64 == 0; N % tile_n == 0, K % tile_k == 0; otherwise as tl_gemm
+ *   and tl_gemm_grouped (experts laid end to end).  No generic-address path in this flavour.
+ */
+int tl_gemm_kmajor(const void* d_A_rowmajor, const void* d_B_nk_tilemajor, float* d_C,
+                   int64_t M, int64_t N, int64_t K,
+                   int64_t G, int tile_n, int tile_k,
+                   int cta_m, int cta_n, int cta_k, void* cuda_stream);
+int tl_gemm_grouped_kmajor(const void* d_A_sorted, const void* d_B_experts_nk, float* d_C,
+                           const int32_t* d_offsets, int E, int64_t total_rows,
+                           int64_t N, int64_t K, int64_t G, int tile_n, int tile_k,
+                           int cta_m, int cta_n, int cta_k, void* cuda_stream);
+
 /* Bytes of workspace tl_gemm / tl_gemm_grouped may need for these sizes on the current device. */
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k);
 /* Hands the library a caller-owned device workspace (256-byte aligned); (NULL, 0) returns to the
@@ -212,7 +233,7 @@ int tl_gemm_noalloc(const void* d_A_rowmajor, const void* d_B_tilemajor, float* 
  * counted (B starts on a G boundary); nothing is shared between loads.
  *   bytes_fetched = sum of blocks * G,  bytes_used = sum of rectangle bytes,
  *   requests (may be NULL) = sum of blocks.  All host out-parameters; exact.
- * layout is a tl_layout; block_rows/block_cols only matter for tile-major.
+ * layout is a tl_layout; block_rows/block_cols only matter for the two tile-major flavours.
  * Any positive tile sizes are accepted (not only the GEMM's).  Runs one small
  * kernel (one warp per CTA tile) on the tl_set_stream() stream and waits.
  */

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libtilelens.so")
 
 TL_OK = 0
 TO_TILE_MAJOR, TO_ROW_MAJOR = 0, 1
-LAYOUT_ROW_MAJOR, LAYOUT_COL_MAJOR, LAYOUT_TILE_MAJOR = 0, 1, 2
+LAYOUT_ROW_MAJOR, LAYOUT_COL_MAJOR, LAYOUT_TILE_MAJOR, LAYOUT_TILE_MAJOR_K = 0, 1, 2, 3
 
 # Every symbol include/tilelens.h declares: (name, restype, argtypes)
 _i64, _int, _vp, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
@@ -30,6 +30,9 @@ _SIGNATURES = {
     "tl_relayout_on": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int, _vp]),
     "tl_gemm": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_grouped_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int,
+                                      _vp]),
     "tl_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int, _int, _int]),
     "tl_set_workspace": (_int, [_vp, _sz]),
     "tl_gemm_host": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp, _sz, _vp]),
@@ -127,6 +130,21 @@ def gemm_grouped(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, offsets: tor
     _check(lib().tl_gemm_grouped(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), _dev_ptr(offsets), E, total_rows, N, K, G,
                                  block_rows, block_cols, cta[0], cta[1], cta[2], _stream_ptr(stream)),
            "tl_gemm_grouped")
+
+
+def gemm_kmajor(A: torch.Tensor, B_nk: torch.Tensor, C: torch.Tensor, M: int, N: int, K: int, G: int = 4096,
+                tile_n: int = 32, tile_k: int = 64, cta=(0, 0, 0), stream=None):
+    """Weights stored [N][K] (K contiguous), tile-major as Eq. 2 prints it; tile_n == 0: the plain [N][K] array."""
+    _check(lib().tl_gemm_kmajor(_dev_ptr(A), _dev_ptr(B_nk), _dev_ptr(C), M, N, K, G, tile_n, tile_k,
+                                cta[0], cta[1], cta[2], _stream_ptr(stream)), "tl_gemm_kmajor")
+
+
+def gemm_grouped_kmajor(A: torch.Tensor, B_nk: torch.Tensor, C: torch.Tensor, offsets: torch.Tensor, E: int,
+                        total_rows: int, N: int, K: int, G: int = 4096, tile_n: int = 32, tile_k: int = 64,
+                        cta=(0, 0, 0), stream=None):
+    _check(lib().tl_gemm_grouped_kmajor(_dev_ptr(A), _dev_ptr(B_nk), _dev_ptr(C), _dev_ptr(offsets), E, total_rows,
+                                        N, K, G, tile_n, tile_k, cta[0], cta[1], cta[2], _stream_ptr(stream)),
+           "tl_gemm_grouped_kmajor")
 
 
 def gemm_workspace_bytes(M: int, N: int, K: int, cta=(0, 0, 0)) -> int:

@@ -52,13 +52,15 @@ struct alignas(64) GemmParams {
     int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
     int num_stages;
     // weight-operand geometry
-    int row_major;              // 1: B is [K][N] row-major (viewed as one big memory tile)
-    int br_log2, bc_log2;       // memory tile (tile-major only)
-    int k_coord_per_expert;     // added to the K coordinate per expert (K/br blocks, or K rows)
+    int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
+    int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
+    int br_log2, bc_log2;       // memory tile: rows x contiguous columns of the stored matrix (tiled layouts only)
+    int k_coord_per_expert;     // added per expert to the coordinate of the stacked dimension (blocks or rows)
     int box_rows, box_atoms;    // rows and 128-byte atoms of one box
     int kbx, nbx;               // boxes per stage along K and along N
     uint32_t box_bytes;
-    uint32_t lbo, sbo;          // descriptor strides of the MN-major operand, bytes
+    uint32_t lbo, sbo;          // descriptor strides of the weight operand, bytes
+    uint32_t ugroup_off;        // bytes between the 128-column groups of a 256-column tile
     uint32_t kstep_off[8];      // byte offset of each 16-row K step inside a stage
     // generic-address path (Section 4.4: memory tiles that TMA cannot box)
     int generic_b;              // 1: warps 6..9 load the weights with Eq. 1-2 address arithmetic
@@ -385,7 +387,15 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                         for (int nb = 0; nb < p.nbx; ++nb) {
                             const int n = t.n0 + nb * p.box_atoms * 64;
                             uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
-                            if (p.row_major)
+                            if (p.w_kmajor) {
+                                // [N][K] storage: (64 K-elements, row in tile, tile along N, atom in tile, tile along K)
+                                if (p.row_major)
+                                    tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n + kc_expert, 0, k >> 6, 0);
+                                else
+                                    tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n & ((1 << p.br_log2) - 1),
+                                                (n >> p.br_log2) + kc_expert, (k & ((1 << p.bc_log2) - 1)) >> 6,
+                                                k >> p.bc_log2);
+                            } else if (p.row_major)
                                 tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k + kc_expert, n >> 6, 0, 0);
                             else
                                 tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k & ((1 << p.br_log2) - 1),
@@ -422,8 +432,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 const uint32_t n_mma = kWN ? uint32_t(kBN) : uint32_t((t.rows + 15) & ~15);
                 // fp32 accumulate, bf16 x bf16; the weights operand is MN-major (bit 15: A, bit 16: B), the token
                 // operand K-major; M = kUmmaM, N = n_mma
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (kWN ? (1u << 16) : (1u << 15)) |
-                                       ((n_mma >> 3) << 17) | ((uint32_t(kUmmaM) >> 4) << 24);
+                const uint32_t w_major = p.w_kmajor ? 0u : (kWN ? (1u << 16) : (1u << 15));
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | w_major | ((n_mma >> 3) << 17) |
+                                       ((uint32_t(kUmmaM) >> 4) << 24);
                 const long long ca0 = TL_CLOCK();
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
                     ok = false;
@@ -452,7 +463,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 #pragma unroll
                         for (int u = 0; u < kNumN; ++u) {
                             const uint64_t w_desc =
-                                make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * 2u * p.lbo, p.lbo, p.sbo);
+                                make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * p.ugroup_off, p.lbo, p.sbo);
                             if (kWN)
                                 umma_bf16(d_tmem, tok_desc, w_desc, idesc, (kit > w.kbeg || j > 0) ? 1u : 0u);
                             else
@@ -871,23 +882,29 @@ struct FixedScratch {
 
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
-                       int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr) {
+                       int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
+                       bool kmajor = false) {
     if (rows_total < 0 || N <= 0 || K <= 0 || E < 1) return TL_ERR_INVALID_ARG;
     if (rows_total == 0) return TL_OK;
     if (!d_A || !d_B || !d_C) return TL_ERR_INVALID_ARG;
     if (rows_total >= (int64_t(1) << 31) || N >= (int64_t(1) << 31) || K * int64_t(E) >= (int64_t(1) << 31))
         return TL_ERR_UNSUPPORTED;
     if (E > kMaxExperts) return TL_ERR_UNSUPPORTED;
+    // br x bc is the memory tile of the STORED matrix: K-rows x N-columns, or N-rows x K-columns when kmajor.
     if (br != 0) {
         if (br < 0 || bc <= 0 || int64_t(br) * bc * 2 != G) return TL_ERR_INVALID_ARG;
         if (!is_pow2(br) || !is_pow2(bc)) return TL_ERR_UNSUPPORTED;
-        if (K % br != 0 || N % bc != 0) return TL_ERR_INVALID_ARG;
+        if (kmajor ? (N % br != 0 || K % bc != 0) : (K % br != 0 || N % bc != 0)) return TL_ERR_INVALID_ARG;
+    }
+    if (kmajor) {
+        // K-major operand: 64 contiguous K-elements per swizzle row; shorter tile rows have no path here
+        if ((br != 0 && bc < 64) || K % 64 != 0) return TL_ERR_UNSUPPORTED;
     }
     // One-row memory tiles are row-major (Section 3.1: the (1, G/s) extreme).
-    const bool row_major = br == 0 || (br == 1 && N % 64 == 0);
+    const bool row_major = br == 0 || (!kmajor && br == 1 && N % 64 == 0);
     // TMA boxes need whole 8-row x 128-byte swizzle atoms; anything smaller takes the generic-address path.
-    const bool generic = !row_major && (br < 8 || bc < 64);
-    if (row_major && N % 64 != 0) return TL_ERR_UNSUPPORTED;
+    const bool generic = !kmajor && !row_major && (br < 8 || bc < 64);
+    if (!kmajor && row_major && N % 64 != 0) return TL_ERR_UNSUPPORTED;
     if (generic && (G < 16 || br > 128 || bc > 256)) return TL_ERR_UNSUPPORTED;   // tile must fit the CTA tile
     if (K % 8 != 0) return TL_ERR_UNSUPPORTED;                  // 16-byte row pitch of A
     if (reinterpret_cast<uintptr_t>(d_A) % 16 != 0) return TL_ERR_ALIGNMENT;
@@ -930,7 +947,33 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     // ---- weight operand B
     const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
     int RB, AB, nb_box = 1, kb_box = 1;         // box: rows, atoms, memory tiles along N and K
-    if (generic) {
+    if (kmajor) {
+        // Weights [N][K], K contiguous.  Tiled (Eq. 2 as printed, a = bc along K, b = br along N): the 5-D view
+        // (64, b, E*N/b, a/64, K/a) with strides (1, a, b*K, 64, a*b) elements; the box takes, for every
+        // 64-element K atom of the stage, all rows of the CTA tile, so the bytes land as [atom][cta_n rows][64]:
+        // the canonical K-major, 128-byte-swizzled operand.  Untiled: (64, E*N, 1, K/64, 1).
+        RB = plan.BK;
+        AB = NA;
+        if (row_major) {
+            const uint64_t dims[5] = {64, uint64_t(N) * E, 1, uint64_t(K / 64), 1};
+            const uint64_t str[5] = {2, uint64_t(K) * 2, uint64_t(K) * 2 * uint64_t(N) * E, 128, uint64_t(K) * 2 * uint64_t(N) * E};
+            const uint32_t box[5] = {64, uint32_t(plan.BN), 1, uint32_t(plan.BK / 64), 1};
+            if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+            p.k_coord_per_expert = int(N);
+        } else {
+            const int rows_box = br < plan.BN ? br : plan.BN;
+            const int k_box = bc < plan.BK ? bc : plan.BK;
+            const uint64_t dims[5] = {64, uint64_t(br), uint64_t(N / br) * E, uint64_t(bc / 64), uint64_t(K / bc)};
+            const uint64_t str[5] = {2, uint64_t(bc) * 2, uint64_t(br) * uint64_t(K) * 2, 128, uint64_t(G)};
+            const uint32_t box[5] = {64, uint32_t(rows_box), uint32_t(plan.BN / rows_box), uint32_t(k_box / 64),
+                                     uint32_t(plan.BK / k_box)};
+            if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+            p.k_coord_per_expert = int(N / br);
+            p.br_log2 = ilog2(br);
+            p.bc_log2 = ilog2(bc);
+        }
+        p.w_kmajor = 1;
+    } else if (generic) {
         // No tensor map: warps 6..9 of the kernel compute Eq. 1-2 addresses themselves and build the
         // canonical [atom][cta_k rows][64] image in shared memory.
         if (plan.BK % br != 0 || plan.BN % bc != 0) return TL_ERR_UNSUPPORTED;
@@ -981,9 +1024,23 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     const uint32_t krow_bytes = uint32_t(NA) * RB * kAtomBytes;   // all boxes sharing one K range
     p.lbo = uint32_t(RB) * kAtomBytes;
     p.sbo = RB >= 16 ? 1024u : krow_bytes;
+    p.ugroup_off = 2u * p.lbo;
     for (int j = 0; j < plan.BK / 16; ++j) {
         const int row = j * 16;
         p.kstep_off[j] = uint32_t(row / RB) * krow_bytes + uint32_t(row % RB) * kAtomBytes;
+    }
+    if (kmajor) {
+        // K-major image: [64-element atom][cta_n rows][128 bytes]; 8-row groups 1024 bytes apart, a K step of
+        // 16 elements is 32 bytes further inside the swizzle row, the next atom cta_n rows further.
+        p.lbo = 16;
+        p.sbo = 1024;
+        p.ugroup_off = 128u * kAtomBytes;
+        for (int j = 0; j < plan.BK / 16; ++j)
+            p.kstep_off[j] = uint32_t(j / 4) * uint32_t(plan.BN) * kAtomBytes + uint32_t(j % 4) * 32u;
+        p.box_rows = plan.BK;
+        p.box_atoms = NA;
+        p.kbx = p.nbx = 1;
+        p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
     }
     p.C = d_C;
     p.partials = static_cast<float*>(ws);
@@ -1088,6 +1145,20 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
     // Without a host copy of the offsets the largest expert is unknown: size tiles for the total.
     return tl::gemm_launch(d_A_sorted, d_B_experts, d_C, d_offsets, E, total_rows, total_rows, N, K, G, block_rows,
                            block_cols, cta_m, cta_n, cta_k, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int tl_gemm_kmajor(const void* d_A, const void* d_B_nk, float* d_C, int64_t M, int64_t N, int64_t K, int64_t G, int tile_n,
+                   int tile_k, int cta_m, int cta_n, int cta_k, void* cuda_stream) {
+    return tl::gemm_launch(d_A, d_B_nk, d_C, nullptr, 1, M, M, N, K, G, tile_n, tile_k, cta_m, cta_n, cta_k,
+                           static_cast<cudaStream_t>(cuda_stream), nullptr, true);
+}
+
+int tl_gemm_grouped_kmajor(const void* d_A_sorted, const void* d_B_experts_nk, float* d_C, const int32_t* d_offsets, int E,
+                           int64_t total_rows, int64_t N, int64_t K, int64_t G, int tile_n, int tile_k, int cta_m,
+                           int cta_n, int cta_k, void* cuda_stream) {
+    if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
+    return tl::gemm_launch(d_A_sorted, d_B_experts_nk, d_C, d_offsets, E, total_rows, total_rows, N, K, G, tile_n, tile_k,
+                           cta_m, cta_n, cta_k, static_cast<cudaStream_t>(cuda_stream), nullptr, true);
 }
 
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {

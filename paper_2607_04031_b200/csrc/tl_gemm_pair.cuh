@@ -185,7 +185,13 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kStageBytes);
                     const int k = kit * kBK;
                     tma_pair_load_2d(sw + kWBytes, &p.tmap_a[3], full_leader, k, row0);
-                    if (p.row_major)
+                    if (p.w_kmajor) {
+                        if (p.row_major)
+                            tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0, 0, k >> 6, 0);
+                        else
+                            tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0 & ((1 << p.br_log2) - 1), n0 >> p.br_log2,
+                                             (k & ((1 << p.bc_log2) - 1)) >> 6, k >> p.bc_log2);
+                    } else if (p.row_major)
                         tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k, n0 >> 6, 0, 0);
                     else
                         tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k & ((1 << p.br_log2) - 1),
@@ -207,7 +213,9 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
         if (rank == 0 && lane == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = 256 over the pair, N = 256
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+            // (weights K-major when they are stored [N][K])
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (p.w_kmajor ? 0u : (1u << 15)) | ((256u >> 3) << 17) |
+                                   ((256u >> 4) << 24);
             bool ok = true;
             const long long t_begin = TL_CLK();
             (void)t_begin;

@@ -122,6 +122,9 @@ static int read_amp_validate(int64_t N, int64_t K, int cta_m, int cta_n, int cta
     if (layout == TL_LAYOUT_TILE_MAJOR) {
         if (br <= 0 || bc <= 0 || int64_t(br) * bc * s != G) return TL_ERR_INVALID_ARG;
         if (K % br != 0 || N % bc != 0) return TL_ERR_INVALID_ARG;
+    } else if (layout == TL_LAYOUT_TILE_MAJOR_K) {
+        if (br <= 0 || bc <= 0 || int64_t(br) * bc * s != G) return TL_ERR_INVALID_ARG;
+        if (N % br != 0 || K % bc != 0) return TL_ERR_INVALID_ARG;
     } else if (layout != TL_LAYOUT_ROW_MAJOR && layout != TL_LAYOUT_COL_MAJOR) {
         return TL_ERR_INVALID_ARG;
     }
@@ -135,12 +138,19 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
     ReadAmpParams p;
     p.N = N; p.K = K; p.BN = cta_n; p.BK = cta_k; p.G = G; p.s = s;
     p.br = br > 0 ? br : 1; p.bc = bc > 0 ? bc : 1; p.layout = layout;
-    p.n_tiles = ceil_div(N, cta_n);
-    p.k_iters = ceil_div(K, cta_k);
+    if (layout == TL_LAYOUT_TILE_MAJOR_K) {
+        // The K x N weight stored with K contiguous IS an N x K matrix with contiguous columns: same blocks,
+        // same tile loads with their two extents exchanged, hence the same count.
+        if (d_fetched || d_used) return TL_ERR_UNSUPPORTED;       // per-tile arrays are indexed by n-tile
+        p.N = K; p.K = N; p.BN = cta_k; p.BK = cta_n;
+        p.layout = TL_LAYOUT_TILE_MAJOR;
+    }
+    p.n_tiles = ceil_div(p.N, p.BN);
+    p.k_iters = ceil_div(p.K, p.BK);
     p.m_tiles = m_tiles;
     p.d_acc = d_acc; p.d_fetched = d_fetched; p.d_used = d_used;
     p.h_out = d_acc ? state().ctl.h_acc_dev : nullptr;
-    p.iters_per_warp = layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
+    p.iters_per_warp = p.layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
     if (m_tiles == 0) return TL_OK;
     const int warps_per_cta = 4;
     const int64_t grid = ceil_div(p.n_tiles * ceil_div(p.k_iters, p.iters_per_warp), warps_per_cta);
