@@ -364,6 +364,35 @@ def run_ours(args):
                         sum(x["ms"] for x in prefill if x["layout"] == "row")}
     tl.device_status()
 
+    # ---- K-contiguous flavour (weights kept [N][K]; Eq. 2 as printed with the (64, 32) memory tile), M = 8
+    W_nk, W_nk_tile = {}, {}
+    for name, K, N in inputs.LLAMA70B_PROJ:
+        W_nk[name] = W_row[name].t().contiguous()
+        W_nk_tile[name] = torch.empty_like(W_nk[name])
+        tl.relayout(W_nk[name], W_nk_tile[name], N, K, 2, G, 32, 64, tl.TO_TILE_MAJOR)
+    kcont = []
+    for layout in ("tile_major_k_32x64", "plain_NK"):
+        evs = []
+        for rep in range(6):
+            for name, K, N in inputs.LLAMA70B_PROJ:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                if layout == "plain_NK":
+                    tl.gemm_kmajor(A_dec[name, 8], W_nk[name], C_dec[name, 8], 8, N, K, 0, 0, 0)
+                else:
+                    tl.gemm_kmajor(A_dec[name, 8], W_nk_tile[name], C_dec[name, 8], 8, N, K, G, 32, 64)
+                b.record()
+                if rep > 0:
+                    evs.append((name, a, b))
+        torch.cuda.synchronize()
+        for name, K, N in inputs.LLAMA70B_PROJ:
+            med = statistics.median(a.elapsed_time(b) for (n_, a, b) in evs if n_ == name)
+            kcont.append({"proj": name, "M": 8, "layout": layout, "us": med * 1e3,
+                          "GBps": gemm_bytes(8, N, K) / (med * 1e-3) / 1e9})
+    extra["k_contiguous_decode_m8"] = kcont
+    del W_nk, W_nk_tile
+    tl.device_status()
+
     # ---- Qwen-3-30B-A3B MoE grouped leg
     q = inputs.QWEN_MOE
     offsets, counts, _ = inputs.zipf_topk_routing(q["tokens"], q["experts"], q["topk"], q["zipf_alpha"], seed=0)
