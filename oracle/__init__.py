@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.tlo_bf16_to_double.argtypes = [ctypes.c_uint16]
         L.tlo_matmul_at.restype = ctypes.c_int
         L.tlo_matmul_at.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, i64, i64, vp, vp, vp, vp]
+        L.tlo_fp8_e4m3_to_double.restype = ctypes.c_double
+        L.tlo_fp8_e4m3_to_double.argtypes = [ctypes.c_uint8]
+        L.tlo_matmul_at_fp8.restype = ctypes.c_int
+        L.tlo_matmul_at_fp8.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, i64, i64, vp, vp, vp, vp]
         L.tlo_matmul.restype = ctypes.c_int
         L.tlo_matmul.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, i64, vp, vp]
         L.tlo_read_amp.restype = ctypes.c_int
@@ -153,6 +157,27 @@ def matmul_at(A_bits, B_bits, layout, br, bc, M, N, K, idx_i, idx_j):
                              _ptr(ii), _ptr(jj), _ptr(C), _ptr(S))
     if rc != 0:
         raise ValueError(f"tlo_matmul_at rejected its arguments (rc={rc})")
+    return C, S
+
+
+def fp8_e4m3_to_double(h: int) -> float:
+    return float(lib().tlo_fp8_e4m3_to_double(h))
+
+
+def matmul_at_fp8(A_bits, B_bits, layout, br, bc, M, N, K, idx_i, idx_j):
+    """FP8 (E4M3) operands as uint8 bit patterns; otherwise as matmul_at."""
+    A_bits = np.ascontiguousarray(A_bits, dtype=np.uint8)
+    B_bits = np.ascontiguousarray(B_bits, dtype=np.uint8)
+    assert A_bits.size == M * K and B_bits.size == K * N
+    ii = np.ascontiguousarray(idx_i, dtype=np.int64)
+    jj = np.ascontiguousarray(idx_j, dtype=np.int64)
+    assert ii.shape == jj.shape and ii.ndim == 1
+    C = np.empty(ii.size, dtype=np.float64)
+    S = np.empty(ii.size, dtype=np.float64)
+    rc = lib().tlo_matmul_at_fp8(_ptr(A_bits), _ptr(B_bits), layout, br, bc, M, N, K, ii.size,
+                                 _ptr(ii), _ptr(jj), _ptr(C), _ptr(S))
+    if rc != 0:
+        raise ValueError(f"tlo_matmul_at_fp8 rejected its arguments (rc={rc})")
     return C, S
 
 

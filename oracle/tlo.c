@@ -155,6 +155,45 @@ int tlo_matmul(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int
     return 0;
 }
 
+/* FP8 in the E4M3 encoding GPUs use for inference (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no
+ * infinities, S.1111.111 is NaN): the value written out from its fields. */
+double tlo_fp8_e4m3_to_double(uint8_t h) {
+    int sign = h >> 7, e = (h >> 3) & 15, m = h & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);           /* subnormal: 0.m x 2^(1-bias) */
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* Section 2.3 with s = 1 (Section 3.1 treats FP8 beside the 16-bit types): the same sum over k on FP8 operands. */
+static void dot_at_fp8(const uint8_t* A, const uint8_t* B, int layout, int64_t br, int64_t bc,
+                       int64_t N, int64_t K, int64_t i, int64_t j, double* c_out, double* s_out) {
+    double acc = 0.0, abs_acc = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+        double a = tlo_fp8_e4m3_to_double(A[i * K + k]);
+        double b = tlo_fp8_e4m3_to_double(B[tlo_off(layout, k, j, K, N, br, bc, 1)]);
+        double p = a * b;
+        acc += p;
+        abs_acc += fabs(p);
+    }
+    *c_out = acc;
+    *s_out = abs_acc;
+}
+
+int tlo_matmul_at_fp8(const uint8_t* A, const uint8_t* B, int layout, int64_t br, int64_t bc,
+                      int64_t M, int64_t N, int64_t K, int64_t n,
+                      const int64_t* idx_i, const int64_t* idx_j, double* C, double* S) {
+    if (layout == TLO_TILE_MAJOR && (br <= 0 || bc <= 0 || K % br != 0 || N % bc != 0)) return -1;
+    if (layout == TLO_TILE_MAJOR_K && (br <= 0 || bc <= 0 || K % bc != 0 || N % br != 0)) return -1;
+    for (int64_t t = 0; t < n; ++t)
+        if (idx_i[t] < 0 || idx_i[t] >= M || idx_j[t] < 0 || idx_j[t] >= N) return -1;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t t = 0; t < n; ++t)
+        dot_at_fp8(A, B, layout, br, bc, N, K, idx_i[t], idx_j[t], &C[t], &S[t]);
+    return 0;
+}
+
 /* ----------------------------------------------------- read amplification */
 
 /* One weight-tile load: rows k in [k0,k1), columns n in [n0,n1) of the K x N

@@ -78,6 +78,13 @@ int tlo_matmul_at(const uint16_t* A, const uint16_t* B, int layout, int64_t br, 
 int tlo_matmul(const uint16_t* A, const uint16_t* B, int layout, int64_t br, int64_t bc,
                int64_t M, int64_t N, int64_t K, double* C, double* S);
 
+/* FP8 (E4M3, the no-infinity encoding: bias 7, S.1111.111 = NaN) bit pattern -> double, exact. */
+double tlo_fp8_e4m3_to_double(uint8_t h);
+/* tlo_matmul_at on FP8 operands (s = 1; Section 3.1 and Figure 1(c) use FP8 with 64 x 64 memory tiles). */
+int tlo_matmul_at_fp8(const uint8_t* A, const uint8_t* B, int layout, int64_t br, int64_t bc,
+                      int64_t M, int64_t N, int64_t K, int64_t n,
+                      const int64_t* idx_i, const int64_t* idx_j, double* C, double* S);
+
 /* Sections 1, 2.5, 6.5: read amplification of the weight operand under access
  * granularity G.  The tiled product has ceil(M/BM) x ceil(N/BN) CTA tiles and
  * ceil(K/BK) iterations; each (CTA tile, iteration) loads the clipped BK x BN

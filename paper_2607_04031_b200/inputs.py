@@ -75,6 +75,28 @@ def bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view(np.uint16)
 
 
+FP8 = torch.float8_e4m3fn
+
+
+def fp8_normal(shape, std: float, seed: int, device: str = "cpu") -> torch.Tensor:
+    """N(0, std) in fp32, rounded once to FP8 (E4M3)."""
+    x = torch.randn(shape, generator=_gen(seed, device), device=device, dtype=torch.float32)
+    return (x * std).clamp_(-448.0, 448.0).to(FP8)
+
+
+def fp8_integers(shape, lo: int, hi: int, seed: int, device: str = "cpu") -> torch.Tensor:
+    """Integer-valued FP8 in [lo, hi] (|values| <= 16 are exact in E4M3)."""
+    assert -16 <= lo <= hi <= 16
+    x = torch.randint(lo, hi + 1, shape, generator=_gen(seed, device), device=device)
+    return x.to(torch.float32).to(FP8)
+
+
+def bits8(t: torch.Tensor) -> np.ndarray:
+    """FP8 tensor -> uint8 numpy array of the same shape (host copy of the bit patterns)."""
+    assert t.dtype == FP8
+    return t.detach().contiguous().cpu().view(torch.uint8).numpy()
+
+
 def zipf_topk_routing(tokens: int, experts: int, topk: int, alpha: float, seed: int):
     """Top-k routing with Zipf(alpha) expert popularity.
 

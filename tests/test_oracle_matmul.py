@@ -109,3 +109,40 @@ def test_k_contiguous_tile_major_gives_the_same_product():
     buf = tlo.relayout(w_nk.view(np.uint8), N, K, 2, b, a, tlo.TO_TILE_MAJOR).view(np.uint16)
     got, _ = tlo.matmul(inputs.bits(A), buf, tlo.TILE_MAJOR_K, b, a, M, N, K)
     assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------------------ FP8 (E4M3)
+def test_fp8_decoding_matches_torch_for_every_bit_pattern_and_known_values():
+    allbits = np.arange(256, dtype=np.uint8)
+    want = torch.from_numpy(allbits).view(inputs.FP8).to(torch.float64).numpy()
+    got = np.array([tlo.fp8_e4m3_to_double(int(h)) for h in allbits])
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok], want[ok]) and np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.isnan(got).sum() == 2 and not np.isinf(got).any()          # S.1111.111 only; no infinities
+    # the format's landmarks, written out: 1.0, -1.0, largest finite 448, smallest subnormal 2^-9, smallest normal 2^-6
+    assert tlo.fp8_e4m3_to_double(0x38) == 1.0 and tlo.fp8_e4m3_to_double(0xB8) == -1.0
+    assert tlo.fp8_e4m3_to_double(0x7E) == 448.0 and tlo.fp8_e4m3_to_double(0x01) == 2.0 ** -9
+    assert tlo.fp8_e4m3_to_double(0x08) == 2.0 ** -6 and tlo.fp8_e4m3_to_double(0x00) == 0.0
+    assert tlo.fp8_e4m3_to_double(0x55) == 13.0                          # 0 1010 101: 1.101b x 2^(10-7)
+
+
+def test_fp8_product_matches_numpy_and_exact_integers_in_every_layout():
+    M, N, K, b, a = 6, 128, 256, 64, 64                       # the 64 x 64 FP8 memory tile of Figure 1(c)
+    A = inputs.fp8_normal((M, K), 1.0, seed=31)
+    B = inputs.fp8_normal((K, N), 0.5, seed=32)
+    a64, b64 = A.to(torch.float64).numpy(), B.to(torch.float64).numpy()
+    want, want_S = a64 @ b64, np.abs(a64) @ np.abs(b64)
+    ii, jj = np.repeat(np.arange(M), N), np.tile(np.arange(N), M)
+    w_nk = np.ascontiguousarray(inputs.bits8(B).T)            # [N][K]
+    tiled = tlo.relayout(w_nk, N, K, 1, b, a, tlo.TO_TILE_MAJOR)
+    for layout, buf, br, bc in ((tlo.ROW_MAJOR, inputs.bits8(B), 0, 0), (tlo.COL_MAJOR, w_nk, 0, 0),
+                                (tlo.TILE_MAJOR_K, tiled, b, a)):
+        C, S = tlo.matmul_at_fp8(inputs.bits8(A), buf, layout, br, bc, M, N, K, ii, jj)
+        assert np.all(np.abs(C.reshape(M, N) - want) <= 1e-13 * want_S + 1e-300)
+        assert np.all(np.abs(S.reshape(M, N) - want_S) <= 1e-13 * want_S + 1e-300)
+    Ai = inputs.fp8_integers((M, K), -8, 8, seed=33)
+    Bi = inputs.fp8_integers((K, N), -8, 8, seed=34)
+    wi = Ai.to(torch.float32).to(torch.int64) @ Bi.to(torch.float32).to(torch.int64)
+    tiled_i = tlo.relayout(np.ascontiguousarray(inputs.bits8(Bi).T), N, K, 1, b, a, tlo.TO_TILE_MAJOR)
+    C, _ = tlo.matmul_at_fp8(inputs.bits8(Ai), tiled_i, tlo.TILE_MAJOR_K, b, a, M, N, K, ii, jj)
+    assert np.array_equal(C.reshape(M, N), wi.numpy().astype(np.float64))
