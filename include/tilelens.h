@@ -145,8 +145,9 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
  * K-elements (the paper's a) by tile_n rows along N (the paper's b), tile_n*tile_k*2 == G, tiles ordered along
  * K first.  tile_n == 0: the plain [N][K] array.  tl_relayout(rows = N, cols = K, block_rows = tile_n,
  * block_cols = tile_k) produces this buffer.  The weights are then the K-major operand of the MMA.
- *   tile_k >= 64 (one 128-byte swizzle row), K % 64 == 0; N % tile_n == 0, K % tile_k == 0; otherwise as tl_gemm
- *   and tl_gemm_grouped (experts laid end to end).  No generic-address path in this flavour.
+ *   tile_k >= 16 (a tile row is one swizzle row of 128, 64 or 32 bytes); N % tile_n == 0, K % tile_k == 0; the
+ *   plain array needs K % 64 == 0; otherwise as tl_gemm and tl_gemm_grouped (experts laid end to end).  Shorter
+ *   tile rows return TL_ERR_UNSUPPORTED: there is no generic-address path in this flavour.
  */
 int tl_gemm_kmajor(const void* d_A_rowmajor, const void* d_B_nk_tilemajor, float* d_C,
                    int64_t M, int64_t N, int64_t K,
@@ -156,6 +157,21 @@ int tl_gemm_grouped_kmajor(const void* d_A_sorted, const void* d_B_experts_nk, f
                            const int32_t* d_offsets, int E, int64_t total_rows,
                            int64_t N, int64_t K, int64_t G, int tile_n, int tile_k,
                            int cta_m, int cta_n, int cta_k, void* cuda_stream);
+
+/*
+ * FP8 form (Section 3.1 and Figure 1(c): a 4 KB block of 8-bit elements is a 64 x 64 memory tile): A is M x K and
+ * the weights are [N][K], both E4M3 bytes (bias 7, no infinities); C = A x B^T in fp32, products exact,
+ * accumulation in fp32.  tile_n * tile_k == G; tile_k >= 32; the plain array (tile_n == 0) needs K % 128 == 0.
+ * cta_k counts K elements and is 0, 128 or 256.  Everything else as tl_gemm_kmajor / tl_gemm_grouped_kmajor.
+ */
+int tl_gemm_fp8_kmajor(const void* d_A_rowmajor_fp8, const void* d_B_nk_tilemajor_fp8, float* d_C,
+                       int64_t M, int64_t N, int64_t K,
+                       int64_t G, int tile_n, int tile_k,
+                       int cta_m, int cta_n, int cta_k, void* cuda_stream);
+int tl_gemm_grouped_fp8_kmajor(const void* d_A_sorted_fp8, const void* d_B_experts_nk_fp8, float* d_C,
+                               const int32_t* d_offsets, int E, int64_t total_rows,
+                               int64_t N, int64_t K, int64_t G, int tile_n, int tile_k,
+                               int cta_m, int cta_n, int cta_k, void* cuda_stream);
 
 /* Bytes of workspace tl_gemm / tl_gemm_grouped may need for these sizes on the current device. */
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k);

@@ -33,6 +33,9 @@ _SIGNATURES = {
     "tl_gemm_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int,
                                       _vp]),
+    "tl_gemm_fp8_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_grouped_fp8_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int,
+                                          _int, _vp]),
     "tl_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int, _int, _int]),
     "tl_set_workspace": (_int, [_vp, _sz]),
     "tl_gemm_host": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp, _sz, _vp]),
@@ -145,6 +148,21 @@ def gemm_grouped_kmajor(A: torch.Tensor, B_nk: torch.Tensor, C: torch.Tensor, of
     _check(lib().tl_gemm_grouped_kmajor(_dev_ptr(A), _dev_ptr(B_nk), _dev_ptr(C), _dev_ptr(offsets), E, total_rows,
                                         N, K, G, tile_n, tile_k, cta[0], cta[1], cta[2], _stream_ptr(stream)),
            "tl_gemm_grouped_kmajor")
+
+
+def gemm_fp8_kmajor(A: torch.Tensor, B_nk: torch.Tensor, C: torch.Tensor, M: int, N: int, K: int, G: int = 4096,
+                    tile_n: int = 64, tile_k: int = 64, cta=(0, 0, 0), stream=None):
+    """FP8 (E4M3) A [M,K] and weights [N,K] (tile-major tile_n x tile_k bytes, or plain when tile_n == 0); C fp32."""
+    _check(lib().tl_gemm_fp8_kmajor(_dev_ptr(A), _dev_ptr(B_nk), _dev_ptr(C), M, N, K, G, tile_n, tile_k,
+                                    cta[0], cta[1], cta[2], _stream_ptr(stream)), "tl_gemm_fp8_kmajor")
+
+
+def gemm_grouped_fp8_kmajor(A: torch.Tensor, B_nk: torch.Tensor, C: torch.Tensor, offsets: torch.Tensor, E: int,
+                            total_rows: int, N: int, K: int, G: int = 4096, tile_n: int = 64, tile_k: int = 64,
+                            cta=(0, 0, 0), stream=None):
+    _check(lib().tl_gemm_grouped_fp8_kmajor(_dev_ptr(A), _dev_ptr(B_nk), _dev_ptr(C), _dev_ptr(offsets), E, total_rows,
+                                            N, K, G, tile_n, tile_k, cta[0], cta[1], cta[2], _stream_ptr(stream)),
+           "tl_gemm_grouped_fp8_kmajor")
 
 
 def gemm_workspace_bytes(M: int, N: int, K: int, cta=(0, 0, 0)) -> int:

@@ -54,6 +54,10 @@ struct alignas(64) GemmParams {
     // weight-operand geometry
     int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
     int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
+    int fp8;                    // 1: both operands are 8-bit floating point (E4M3); needs w_kmajor
+    int k_shift;                // log2(K elements per 2 bytes): a stage holds (BK << k_shift) K-elements
+    int w_atom_log2;            // K-major weights: log2(elements in one swizzle row of 128, 64 or 32 bytes)
+    uint32_t w_layout;          // swizzle mode field of the weight operand's shared-memory descriptor
     int br_log2, bc_log2;       // memory tile: rows x contiguous columns of the stored matrix (tiled layouts only)
     int k_coord_per_expert;     // added per expert to the coordinate of the stacked dimension (blocks or rows)
     int box_rows, box_atoms;    // rows and 128-byte atoms of one box
@@ -188,11 +192,11 @@ __device__ __forceinline__ void tile_prefix(const GemmParams& p, const int* row_
     if (lane == 0) prefix[p.E] = carry;
 }
 
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout = 2u) {
     // start address, leading and stride byte offsets in 16-byte units; descriptor version 1 (bit 46);
-    // 128-byte swizzle (value 2 in bits 61..63)
+    // swizzle mode in bits 61..63: 2 = 128-byte, 4 = 64-byte, 6 = 32-byte
     return uint64_t((addr & 0x3FFFFu) >> 4) | (uint64_t(lbo >> 4) << 16) | (uint64_t(sbo >> 4) << 32) |
-           (uint64_t(1) << 46) | (uint64_t(2) << 61);
+           (uint64_t(1) << 46) | (uint64_t(layout) << 61);
 }
 
 // Optional per-CTA timestamps (nanoseconds of %globaltimer), compiled in only with -DTL_TIMELINE:
@@ -377,24 +381,26 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     uint8_t* sw = stages + size_t(stage) * stage_bytes;
                     uint8_t* sa = sw + kWBytes;
                     mbar_arrive_expect_tx(&full_bar[stage], tx);
-                    const int k0 = kit * kBK;
+                    const int k0 = (kit * kBK) << p.k_shift;        // first K element of the stage
 #pragma unroll
                     for (int sub = 0; sub < kSubK; ++sub)
                         tma_load_2d(sa + size_t(sub) * p.BM * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
-                                    k0 + sub * 64, t.row0);
+                                    k0 + ((sub * 64) << p.k_shift), t.row0);
                     for (int kb = 0; kb < p.kbx; ++kb) {
                         const int k = k0 + kb * p.box_rows;
                         for (int nb = 0; nb < p.nbx; ++nb) {
                             const int n = t.n0 + nb * p.box_atoms * 64;
                             uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
                             if (p.w_kmajor) {
-                                // [N][K] storage: (64 K-elements, row in tile, tile along N, atom in tile, tile along K)
+                                // [N][K] storage: (swizzle row of K-elements, row in tile, tile along N, swizzle
+                                // row in tile, tile along K)
                                 if (p.row_major)
-                                    tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n + kc_expert, 0, k >> 6, 0);
+                                    tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n + kc_expert, 0,
+                                                k >> p.w_atom_log2, 0);
                                 else
                                     tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n & ((1 << p.br_log2) - 1),
-                                                (n >> p.br_log2) + kc_expert, (k & ((1 << p.bc_log2) - 1)) >> 6,
-                                                k >> p.bc_log2);
+                                                (n >> p.br_log2) + kc_expert,
+                                                (k & ((1 << p.bc_log2) - 1)) >> p.w_atom_log2, k >> p.bc_log2);
                             } else if (p.row_major)
                                 tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k + kc_expert, n >> 6, 0, 0);
                             else
@@ -433,8 +439,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 // fp32 accumulate, bf16 x bf16; the weights operand is MN-major (bit 15: A, bit 16: B), the token
                 // operand K-major; M = kUmmaM, N = n_mma
                 const uint32_t w_major = p.w_kmajor ? 0u : (kWN ? (1u << 16) : (1u << 15));
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | w_major | ((n_mma >> 3) << 17) |
-                                       ((uint32_t(kUmmaM) >> 4) << 24);
+                // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
+                const uint32_t idesc = (1u << 4) | (p.fp8 ? 0u : (1u << 7) | (1u << 10)) | w_major |
+                                       ((n_mma >> 3) << 17) | ((uint32_t(kUmmaM) >> 4) << 24);
                 const long long ca0 = TL_CLOCK();
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
                     ok = false;
@@ -462,13 +469,16 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                             sa + uint32_t(j >> 2) * uint32_t(p.BM) * kAtomBytes + uint32_t(j & 3) * 32u, 16u, 1024u);
 #pragma unroll
                         for (int u = 0; u < kNumN; ++u) {
-                            const uint64_t w_desc =
-                                make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * p.ugroup_off, p.lbo, p.sbo);
-                            if (kWN)
-                                umma_bf16(d_tmem, tok_desc, w_desc, idesc, (kit > w.kbeg || j > 0) ? 1u : 0u);
-                            else
-                                umma_bf16(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc,
-                                          (kit > w.kbeg || j > 0) ? 1u : 0u);
+                            const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * p.ugroup_off,
+                                                                   p.lbo, p.sbo, p.w_layout);
+                            const uint32_t accum = (kit > w.kbeg || j > 0) ? 1u : 0u;
+                            if (p.fp8) {
+                                if (kWN) umma_f8(d_tmem, tok_desc, w_desc, idesc, accum);
+                                else umma_f8(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc, accum);
+                            } else {
+                                if (kWN) umma_bf16(d_tmem, tok_desc, w_desc, idesc, accum);
+                                else umma_bf16(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc, accum);
+                            }
                         }
                     }
                     umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
@@ -883,7 +893,10 @@ struct FixedScratch {
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
                        int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
-                       bool kmajor = false) {
+                       bool kmajor = false, int elem_bytes = 2) {
+    const int es = elem_bytes;                       // 2: bf16, 1: FP8 (E4M3), K-contiguous weights only
+    const int k_shift = es == 1 ? 1 : 0;
+    if (es != 2 && !(es == 1 && kmajor)) return TL_ERR_UNSUPPORTED;
     if (rows_total < 0 || N <= 0 || K <= 0 || E < 1) return TL_ERR_INVALID_ARG;
     if (rows_total == 0) return TL_OK;
     if (!d_A || !d_B || !d_C) return TL_ERR_INVALID_ARG;
@@ -892,13 +905,14 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (E > kMaxExperts) return TL_ERR_UNSUPPORTED;
     // br x bc is the memory tile of the STORED matrix: K-rows x N-columns, or N-rows x K-columns when kmajor.
     if (br != 0) {
-        if (br < 0 || bc <= 0 || int64_t(br) * bc * 2 != G) return TL_ERR_INVALID_ARG;
+        if (br < 0 || bc <= 0 || int64_t(br) * bc * es != G) return TL_ERR_INVALID_ARG;
         if (!is_pow2(br) || !is_pow2(bc)) return TL_ERR_UNSUPPORTED;
         if (kmajor ? (N % br != 0 || K % bc != 0) : (K % br != 0 || N % bc != 0)) return TL_ERR_INVALID_ARG;
     }
     if (kmajor) {
-        // K-major operand: 64 contiguous K-elements per swizzle row; shorter tile rows have no path here
-        if ((br != 0 && bc < 64) || K % 64 != 0) return TL_ERR_UNSUPPORTED;
+        // K-major operand: a tile row is one swizzle row of 128, 64 or 32 bytes; shorter rows have no path here
+        if (br != 0 && bc * es < 32) return TL_ERR_UNSUPPORTED;
+        if (K % (br != 0 ? 32 / es : 128 / es) != 0) return TL_ERR_UNSUPPORTED;
     }
     // One-row memory tiles are row-major (Section 3.1: the (1, G/s) extreme).
     const bool row_major = br == 0 || (!kmajor && br == 1 && N % 64 == 0);
@@ -906,7 +920,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     const bool generic = !kmajor && !row_major && (br < 8 || bc < 64);
     if (!kmajor && row_major && N % 64 != 0) return TL_ERR_UNSUPPORTED;
     if (generic && (G < 16 || br > 128 || bc > 256)) return TL_ERR_UNSUPPORTED;   // tile must fit the CTA tile
-    if (K % 8 != 0) return TL_ERR_UNSUPPORTED;                  // 16-byte row pitch of A
+    if ((K * es) % 16 != 0) return TL_ERR_UNSUPPORTED;          // 16-byte row pitch of A
     if (reinterpret_cast<uintptr_t>(d_A) % 16 != 0) return TL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(d_B) % (row_major || generic ? 16 : 128) != 0) return TL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(d_C) % 16 != 0) return TL_ERR_ALIGNMENT;
@@ -919,11 +933,12 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
             default_tile(rows_max, d_offsets != nullptr, fixed != nullptr, &bm_guess, &bn_guess, &bk_guess);
         if (bm_guess <= 0 || bn_guess <= 0) return TL_ERR_UNSUPPORTED;
         const int64_t mt_bound = d_offsets ? rows_total / bm_guess + E : ceil_div(rows_total, bm_guess);
-        if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K, cta_m, cta_n, cta_k,
+        // (the plan counts K in 2-byte units: an 8-bit stage holds twice as many elements)
+        if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
                                d_offsets != nullptr, &plan, fixed != nullptr))
             return rc;
     }
-    if (d_offsets && K % plan.BK != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
+    if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
     void* ws = nullptr;
     if (fixed) {
         if (plan.ws_bytes > fixed->ws_bytes) return TL_ERR_WORKSPACE;
@@ -937,42 +952,58 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
 
     GemmParams p;
     memset(&p, 0, sizeof p);
-    // ---- token operand A: [rows_total][K], boxes of 64 K-elements x {16..256} rows
+    // ---- token operand A: [rows_total][K], boxes of 128 bytes of K x {16..256} rows
+    const int dtype = es == 1 ? int(CU_TENSOR_MAP_DATA_TYPE_UINT8) : int(CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     for (int i = 0; i < kNumBoxChoices; ++i) {
         const uint64_t dims[2] = {uint64_t(K), uint64_t(rows_total)};
-        const uint64_t str[2] = {2, uint64_t(K) * 2};
-        const uint32_t box[2] = {64, uint32_t(16 << i)};
-        if (int rc = encode(&p.tmap_a[i], d_A, 2, dims, str, box)) return rc;
+        const uint64_t str[2] = {uint64_t(es), uint64_t(K) * es};
+        const uint32_t box[2] = {uint32_t(128 / es), uint32_t(16 << i)};
+        if (int rc = encode_tensor_map(&p.tmap_a[i], d_A, dtype, int(CU_TENSOR_MAP_SWIZZLE_128B), 2, dims, str, box))
+            return rc;
     }
+    p.fp8 = es == 1;
+    p.k_shift = k_shift;
+    p.w_layout = 2;
     // ---- weight operand B
     const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
     int RB, AB, nb_box = 1, kb_box = 1;         // box: rows, atoms, memory tiles along N and K
+    int w_row_bytes = kAtomBytes;                // K-major weights: bytes of one swizzle row
     if (kmajor) {
-        // Weights [N][K], K contiguous.  Tiled (Eq. 2 as printed, a = bc along K, b = br along N): the 5-D view
-        // (64, b, E*N/b, a/64, K/a) with strides (1, a, b*K, 64, a*b) elements; the box takes, for every
-        // 64-element K atom of the stage, all rows of the CTA tile, so the bytes land as [atom][cta_n rows][64]:
-        // the canonical K-major, 128-byte-swizzled operand.  Untiled: (64, E*N, 1, K/64, 1).
+        // Weights [N][K], K contiguous.  Tiled (Eq. 2 as printed, a = bc along K, b = br along N), with the tile
+        // row cut into swizzle rows of r = min(128 bytes, tile row) holding e elements: the 5-D view
+        // (e, b, E*N/b, a/e, K/a) with strides (1, a, b*K, e, a*b) elements; the box takes, for every swizzle row
+        // of the stage's K range, all weight rows of the CTA tile, so the bytes land as [K row][cta_n rows][r]:
+        // the canonical K-major operand in 128-, 64- or 32-byte swizzle.  Untiled: (e, E*N, 1, K/e, 1), r = 128.
         RB = plan.BK;
         AB = NA;
+        const int bk_el = plan.BK << k_shift;                    // K elements per stage
+        w_row_bytes = row_major ? kAtomBytes : (bc * es < kAtomBytes ? bc * es : kAtomBytes);
+        const int e = w_row_bytes / es;
+        const int swz = w_row_bytes == 128 ? int(CU_TENSOR_MAP_SWIZZLE_128B)
+                                           : w_row_bytes == 64 ? int(CU_TENSOR_MAP_SWIZZLE_64B) : int(CU_TENSOR_MAP_SWIZZLE_32B);
         if (row_major) {
-            const uint64_t dims[5] = {64, uint64_t(N) * E, 1, uint64_t(K / 64), 1};
-            const uint64_t str[5] = {2, uint64_t(K) * 2, uint64_t(K) * 2 * uint64_t(N) * E, 128, uint64_t(K) * 2 * uint64_t(N) * E};
-            const uint32_t box[5] = {64, uint32_t(plan.BN), 1, uint32_t(plan.BK / 64), 1};
-            if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+            const uint64_t big = uint64_t(K) * es * uint64_t(N) * E;
+            const uint64_t dims[5] = {uint64_t(e), uint64_t(N) * E, 1, uint64_t(K / e), 1};
+            const uint64_t str[5] = {uint64_t(es), uint64_t(K) * es, big, uint64_t(w_row_bytes), big};
+            const uint32_t box[5] = {uint32_t(e), uint32_t(plan.BN), 1, uint32_t(bk_el / e), 1};
+            if (int rc = encode_tensor_map(&p.tmap_b, d_B, dtype, swz, 5, dims, str, box)) return rc;
             p.k_coord_per_expert = int(N);
         } else {
             const int rows_box = br < plan.BN ? br : plan.BN;
-            const int k_box = bc < plan.BK ? bc : plan.BK;
-            const uint64_t dims[5] = {64, uint64_t(br), uint64_t(N / br) * E, uint64_t(bc / 64), uint64_t(K / bc)};
-            const uint64_t str[5] = {2, uint64_t(bc) * 2, uint64_t(br) * uint64_t(K) * 2, 128, uint64_t(G)};
-            const uint32_t box[5] = {64, uint32_t(rows_box), uint32_t(plan.BN / rows_box), uint32_t(k_box / 64),
-                                     uint32_t(plan.BK / k_box)};
-            if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+            const int k_box = bc < bk_el ? bc : bk_el;
+            const uint64_t dims[5] = {uint64_t(e), uint64_t(br), uint64_t(N / br) * E, uint64_t(bc / e), uint64_t(K / bc)};
+            const uint64_t str[5] = {uint64_t(es), uint64_t(bc) * es, uint64_t(br) * uint64_t(K) * es, uint64_t(w_row_bytes),
+                                     uint64_t(G)};
+            const uint32_t box[5] = {uint32_t(e), uint32_t(rows_box), uint32_t(plan.BN / rows_box), uint32_t(k_box / e),
+                                     uint32_t(bk_el / k_box)};
+            if (int rc = encode_tensor_map(&p.tmap_b, d_B, dtype, swz, 5, dims, str, box)) return rc;
             p.k_coord_per_expert = int(N / br);
             p.br_log2 = ilog2(br);
             p.bc_log2 = ilog2(bc);
         }
         p.w_kmajor = 1;
+        p.w_atom_log2 = ilog2(e);
+        p.w_layout = w_row_bytes == 128 ? 2u : w_row_bytes == 64 ? 4u : 6u;
     } else if (generic) {
         // No tensor map: warps 6..9 of the kernel compute Eq. 1-2 addresses themselves and build the
         // canonical [atom][cta_k rows][64] image in shared memory.
@@ -1030,14 +1061,15 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.kstep_off[j] = uint32_t(row / RB) * krow_bytes + uint32_t(row % RB) * kAtomBytes;
     }
     if (kmajor) {
-        // K-major image: [64-element atom][cta_n rows][128 bytes]; 8-row groups 1024 bytes apart, a K step of
-        // 16 elements is 32 bytes further inside the swizzle row, the next atom cta_n rows further.
+        // K-major image: [swizzle row along K][cta_n rows][r bytes]; 8-row groups 8r bytes apart, a K step of one
+        // instruction (32 bytes) is 32 bytes further inside the swizzle row, the next swizzle row cta_n rows further.
+        const uint32_t r = uint32_t(w_row_bytes), steps_per_row = r / 32u;
         p.lbo = 16;
-        p.sbo = 1024;
-        p.ugroup_off = 128u * kAtomBytes;
+        p.sbo = 8u * r;
+        p.ugroup_off = 128u * r;
         for (int j = 0; j < plan.BK / 16; ++j)
-            p.kstep_off[j] = uint32_t(j / 4) * uint32_t(plan.BN) * kAtomBytes + uint32_t(j % 4) * 32u;
-        p.box_rows = plan.BK;
+            p.kstep_off[j] = (uint32_t(j) / steps_per_row) * uint32_t(plan.BN) * r + (uint32_t(j) % steps_per_row) * 32u;
+        p.box_rows = plan.BK << k_shift;
         p.box_atoms = NA;
         p.kbx = p.nbx = 1;
         p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
@@ -1054,7 +1086,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.BM = plan.BM;
     p.BN = plan.BN;
     p.n_tiles = int(ceil_div(N, plan.BN));
-    p.k_iters = int(ceil_div(K, plan.BK));
+    p.k_iters = int(ceil_div(K, int64_t(plan.BK) << k_shift));
     p.stream_k = plan.stream_k;
     p.num_stages = plan.num_stages;
 
@@ -1159,6 +1191,22 @@ int tl_gemm_grouped_kmajor(const void* d_A_sorted, const void* d_B_experts_nk, f
     if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
     return tl::gemm_launch(d_A_sorted, d_B_experts_nk, d_C, d_offsets, E, total_rows, total_rows, N, K, G, tile_n, tile_k,
                            cta_m, cta_n, cta_k, static_cast<cudaStream_t>(cuda_stream), nullptr, true);
+}
+
+int tl_gemm_fp8_kmajor(const void* d_A, const void* d_B_nk, float* d_C, int64_t M, int64_t N, int64_t K, int64_t G,
+                       int tile_n, int tile_k, int cta_m, int cta_n, int cta_k, void* cuda_stream) {
+    if (cta_k != 0 && cta_k != 128 && cta_k != 256) return TL_ERR_UNSUPPORTED;
+    return tl::gemm_launch(d_A, d_B_nk, d_C, nullptr, 1, M, M, N, K, G, tile_n, tile_k, cta_m, cta_n, cta_k / 2,
+                           static_cast<cudaStream_t>(cuda_stream), nullptr, true, 1);
+}
+
+int tl_gemm_grouped_fp8_kmajor(const void* d_A_sorted, const void* d_B_experts_nk, float* d_C, const int32_t* d_offsets,
+                               int E, int64_t total_rows, int64_t N, int64_t K, int64_t G, int tile_n, int tile_k,
+                               int cta_m, int cta_n, int cta_k, void* cuda_stream) {
+    if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
+    if (cta_k != 0 && cta_k != 128 && cta_k != 256) return TL_ERR_UNSUPPORTED;
+    return tl::gemm_launch(d_A_sorted, d_B_experts_nk, d_C, d_offsets, E, total_rows, total_rows, N, K, G, tile_n, tile_k,
+                           cta_m, cta_n, cta_k / 2, static_cast<cudaStream_t>(cuda_stream), nullptr, true, 1);
 }
 
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {

@@ -78,6 +78,15 @@ __device__ __forceinline__ void umma_pair_bf16(uint32_t d_tmem, uint64_t a_desc,
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+__device__ __forceinline__ void umma_pair_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // Arrives on the barrier at the same shared-memory offset in both CTAs once the MMAs issued so far are done.
 __device__ __forceinline__ void umma_pair_commit_both(uint64_t* bar) {
     asm volatile(
@@ -183,14 +192,14 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     // is only signalled after the leader's MMAs have consumed the stage.
                     const uint32_t full_leader = map_to_cta(smem_u32(&full_bar[stage]), 0);
                     if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kStageBytes);
-                    const int k = kit * kBK;
+                    const int k = (kit * kBK) << p.k_shift;         // K element (8-bit types: twice as many per stage)
                     tma_pair_load_2d(sw + kWBytes, &p.tmap_a[3], full_leader, k, row0);
                     if (p.w_kmajor) {
                         if (p.row_major)
-                            tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0, 0, k >> 6, 0);
+                            tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0, 0, k >> p.w_atom_log2, 0);
                         else
                             tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0 & ((1 << p.br_log2) - 1), n0 >> p.br_log2,
-                                             (k & ((1 << p.bc_log2) - 1)) >> 6, k >> p.bc_log2);
+                                             (k & ((1 << p.bc_log2) - 1)) >> p.w_atom_log2, k >> p.bc_log2);
                     } else if (p.row_major)
                         tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k, n0 >> 6, 0, 0);
                     else
@@ -214,8 +223,9 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = 256 over the pair, N = 256
             // (weights K-major when they are stored [N][K])
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (p.w_kmajor ? 0u : (1u << 15)) | ((256u >> 3) << 17) |
-                                   ((256u >> 4) << 24);
+            // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
+            const uint32_t idesc = (1u << 4) | (p.fp8 ? 0u : (1u << 7) | (1u << 10)) | (p.w_kmajor ? 0u : (1u << 15)) |
+                                   ((256u >> 3) << 17) | ((256u >> 4) << 24);
             bool ok = true;
             const long long t_begin = TL_CLK();
             (void)t_begin;
@@ -243,9 +253,10 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     const uint32_t sa = sw + kWBytes;
 #pragma unroll
                     for (int j = 0; j < kKSteps; ++j) {
-                        const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j], p.lbo, p.sbo);
+                        const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j], p.lbo, p.sbo, p.w_layout);
                         const uint64_t tok_desc = make_smem_desc(sa + uint32_t(j) * 32u, 16u, 1024u);
-                        umma_pair_bf16(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                        if (p.fp8) umma_pair_f8(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                        else umma_pair_bf16(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
                     }
                     umma_pair_commit_both(&empty_bar[stage]);       // frees the stage in both CTAs
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }

@@ -28,7 +28,7 @@ def _run(A, W, M, N, K, tile_n, tile_k, cta=(0, 0, 0)):
     return C
 
 
-TILES = [(32, 64), (16, 128), (8, 256), (64, 64), (1, 2048 // 2), (4, 512), (0, 0)]     # (tile_n, tile_k); (32, 64) = the paper's (a, b) = (64, 32)
+TILES = [(32, 64), (16, 128), (8, 256), (64, 64), (1, 2048 // 2), (4, 512), (0, 0), (64, 32), (128, 16)]     # (tile_n, tile_k); (32, 64) = the paper's (a, b) = (64, 32)
 
 
 @pytest.mark.parametrize("tile_n,tile_k", TILES)
@@ -125,7 +125,7 @@ def test_errors():
     W = torch.zeros((512, 512), dtype=torch.bfloat16, device=DEV)
     C = torch.zeros((8, 512), dtype=torch.float32, device=DEV)
     with pytest.raises(tl.TileLensError) as e:
-        tl.gemm_kmajor(A, W, C, 8, 512, 512, 4096, 64, 32)        # tile rows of 64 bytes: no path in this flavour
+        tl.gemm_kmajor(A, W, C, 8, 512, 512, 4096, 256, 8)        # tile rows of 16 bytes: no path in this flavour
     assert e.value.status == 2
     with pytest.raises(tl.TileLensError) as e:
         tl.gemm_kmajor(A, W, C, 8, 512, 512, 2048, 32, 64)        # G != tile_n * tile_k * 2
