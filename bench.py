@@ -390,6 +390,33 @@ def run_ours(args):
             kcont.append({"proj": name, "M": 8, "layout": layout, "us": med * 1e3,
                           "GBps": gemm_bytes(8, N, K) / (med * 1e-3) / 1e9})
     extra["k_contiguous_decode_m8"] = kcont
+    # FP8 (E4M3) on the same shapes: 4 KB memory tiles of 32 x 128 bytes (and the 64 x 64 tile of Figure 1(c))
+    fp8 = []
+    A8 = {name: inputs.fp8_normal((8, K), 1.0, seed=700 + i, device=str(dev)).view(torch.uint8)
+          for i, (name, K, N) in enumerate(inputs.LLAMA70B_PROJ)}
+    for tn, tk in ((32, 128), (64, 64)):
+        W8 = {}
+        for i, (name, K, N) in enumerate(inputs.LLAMA70B_PROJ):
+            w = inputs.fp8_normal((N, K), 0.05, seed=710 + i, device=str(dev)).view(torch.uint8)
+            W8[name] = torch.empty_like(w)
+            tl.relayout(w, W8[name], N, K, 1, G, tn, tk, tl.TO_TILE_MAJOR)
+            del w
+        evs = []
+        for rep in range(6):
+            for name, K, N in inputs.LLAMA70B_PROJ:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                tl.gemm_fp8_kmajor(A8[name], W8[name], C_dec[name, 8], 8, N, K, G, tn, tk)
+                b.record()
+                if rep > 0:
+                    evs.append((name, a, b))
+        torch.cuda.synchronize()
+        for name, K, N in inputs.LLAMA70B_PROJ:
+            med = statistics.median(a.elapsed_time(b) for (n_, a, b) in evs if n_ == name)
+            fp8.append({"proj": name, "M": 8, "tile": [tn, tk], "us": med * 1e3,
+                        "GBps": (K * N + 8 * K + 4 * 8 * N) / (med * 1e-3) / 1e9})
+        del W8
+    extra["fp8_decode_m8"] = fp8
     del W_nk, W_nk_tile
     tl.device_status()
 

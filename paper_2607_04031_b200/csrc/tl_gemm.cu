@@ -57,7 +57,7 @@ struct alignas(64) GemmParams {
     int fp8;                    // 1: both operands are 8-bit floating point (E4M3); needs w_kmajor
     int k_shift;                // log2(K elements per 2 bytes): a stage holds (BK << k_shift) K-elements
     int w_atom_log2;            // K-major weights: log2(elements in one swizzle row of 128, 64 or 32 bytes)
-    uint32_t w_layout;          // swizzle mode field of the weight operand's shared-memory descriptor
+    uint64_t w_desc_hi;         // weight operand's shared-memory descriptor without its start address
     int br_log2, bc_log2;       // memory tile: rows x contiguous columns of the stored matrix (tiled layouts only)
     int k_coord_per_expert;     // added per expert to the coordinate of the stacked dimension (blocks or rows)
     int box_rows, box_atoms;    // rows and 128-byte atoms of one box
@@ -192,11 +192,16 @@ __device__ __forceinline__ void tile_prefix(const GemmParams& p, const int* row_
     if (lane == 0) prefix[p.E] = carry;
 }
 
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout = 2u) {
-    // start address, leading and stride byte offsets in 16-byte units; descriptor version 1 (bit 46);
-    // swizzle mode in bits 61..63: 2 = 128-byte, 4 = 64-byte, 6 = 32-byte
-    return uint64_t((addr & 0x3FFFFu) >> 4) | (uint64_t(lbo >> 4) << 16) | (uint64_t(sbo >> 4) << 32) |
-           (uint64_t(1) << 46) | (uint64_t(layout) << 61);
+// Shared-memory matrix descriptor: start address, leading and stride byte offsets in 16-byte units; descriptor
+// version 1 (bit 46); swizzle mode in bits 61..63: 2 = 128-byte, 4 = 64-byte, 6 = 32-byte.
+__host__ __device__ __forceinline__ uint64_t smem_desc_hi(uint32_t lbo, uint32_t sbo, uint32_t layout) {
+    return (uint64_t(lbo >> 4) << 16) | (uint64_t(sbo >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(layout) << 61);
+}
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return uint64_t((addr & 0x3FFFFu) >> 4) | smem_desc_hi(lbo, sbo, 2u);
+}
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint64_t hi) {
+    return uint64_t((addr & 0x3FFFFu) >> 4) | hi;
 }
 
 // Optional per-CTA timestamps (nanoseconds of %globaltimer), compiled in only with -DTL_TIMELINE:
@@ -279,7 +284,7 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
 //                (at most 128 per tile) on the M side.  For decode and MoE: 8 KB of weights per instruction
 //                instead of 4 KB, which lifts the instruction-rate ceiling above the HBM rate.  TMEM lane =
 //                token, and every thread writes its token's row of C in 16-byte pieces.
-template <int kBK, int kBN, bool kWN>
+template <int kBK, int kBN, bool kWN, bool kFp8>
 __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
     constexpr int kNumN = kWN ? 1 : (kBN >= 128 ? kBN / 128 : 1);     // MMAs per K step
     constexpr int kUmmaM = kWN ? 128 : (kBN >= 128 ? 128 : 64);       // rows of the MMA's M side
@@ -440,7 +445,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 // operand K-major; M = kUmmaM, N = n_mma
                 const uint32_t w_major = p.w_kmajor ? 0u : (kWN ? (1u << 16) : (1u << 15));
                 // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
-                const uint32_t idesc = (1u << 4) | (p.fp8 ? 0u : (1u << 7) | (1u << 10)) | w_major |
+                const uint32_t idesc = (1u << 4) | (kFp8 ? 0u : (1u << 7) | (1u << 10)) | w_major |
                                        ((n_mma >> 3) << 17) | ((uint32_t(kUmmaM) >> 4) << 24);
                 const long long ca0 = TL_CLOCK();
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
@@ -469,10 +474,10 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                             sa + uint32_t(j >> 2) * uint32_t(p.BM) * kAtomBytes + uint32_t(j & 3) * 32u, 16u, 1024u);
 #pragma unroll
                         for (int u = 0; u < kNumN; ++u) {
-                            const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * p.ugroup_off,
-                                                                   p.lbo, p.sbo, p.w_layout);
+                            const uint64_t w_desc =
+                                make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * p.ugroup_off, p.w_desc_hi);
                             const uint32_t accum = (kit > w.kbeg || j > 0) ? 1u : 0u;
-                            if (p.fp8) {
+                            if (kFp8) {
                                 if (kWN) umma_f8(d_tmem, tok_desc, w_desc, idesc, accum);
                                 else umma_f8(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc, accum);
                             } else {
@@ -963,7 +968,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     p.fp8 = es == 1;
     p.k_shift = k_shift;
-    p.w_layout = 2;
+    uint32_t w_layout = 2;
     // ---- weight operand B
     const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
     int RB, AB, nb_box = 1, kb_box = 1;         // box: rows, atoms, memory tiles along N and K
@@ -1003,7 +1008,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         }
         p.w_kmajor = 1;
         p.w_atom_log2 = ilog2(e);
-        p.w_layout = w_row_bytes == 128 ? 2u : w_row_bytes == 64 ? 4u : 6u;
+        w_layout = w_row_bytes == 128 ? 2u : w_row_bytes == 64 ? 4u : 6u;
     } else if (generic) {
         // No tensor map: warps 6..9 of the kernel compute Eq. 1-2 addresses themselves and build the
         // canonical [atom][cta_k rows][64] image in shared memory.
@@ -1074,6 +1079,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.kbx = p.nbx = 1;
         p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
     }
+    p.w_desc_hi = smem_desc_hi(p.lbo, p.sbo, w_layout);
     p.C = d_C;
     p.partials = static_cast<float*>(ws);
     p.offsets = d_offsets;
@@ -1102,14 +1108,16 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.num_stages = stages < kPairStagesMax ? stages : kPairStagesMax;
         const size_t smem = size_t(p.num_stages) * (64 * 128 * 2 + 128 * kAtomBytes) + 1024;
         if (max_clusters < 0) {
-            err = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            err = cudaFuncSetAttribute(gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            if (err != cudaSuccess) return check_cuda(err);
+            err = cudaFuncSetAttribute(gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
             if (err != cudaSuccess) return check_cuda(err);
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(2 * state().sm_count);
             cfg.blockDim = dim3(kGemmThreads);
             cfg.dynamicSmemBytes = smem;
             int n = 0;
-            err = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel, &cfg);
+            err = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<false>, &cfg);
             if (err != cudaSuccess) return check_cuda(err);
             max_clusters = n > 0 ? n : 1;
         }
@@ -1118,21 +1126,24 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (getenv("TL_LOG"))
             fprintf(stderr, "[tilelens] pair kernel: %lld tiles of 256x256, %d clusters (max active %d), %d stages, %zu B smem\n",
                     (long long)pair_tiles, clusters, max_clusters, p.num_stages, smem);
-        gemm_pair_kernel<<<2 * clusters, kGemmThreads, smem, stream>>>(p);
+        if (es == 1) gemm_pair_kernel<true><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
+        else gemm_pair_kernel<false><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
         return check_cuda(cudaGetLastError());
     }
-#define TL_LAUNCH_GEMM(BK_, BN_, WN_)                                                                              \
+#define TL_LAUNCH_GEMM_T(BK_, BN_, WN_, F8_)                                                                        \
     {                                                                                                              \
         static bool attr_set = false;                                                                              \
         if (!attr_set) {                                                                                           \
-            err = cudaFuncSetAttribute(gemm_kernel<BK_, BN_, WN_>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+            err = cudaFuncSetAttribute(gemm_kernel<BK_, BN_, WN_, F8_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                        kMaxDynamicSmem);                                                           \
             attr_set = err == cudaSuccess;                                                                         \
         }                                                                                                          \
         if (err == cudaSuccess)                                                                                    \
-            gemm_kernel<BK_, BN_, WN_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes,     \
-                                         stream>>>(p);                                                             \
+            gemm_kernel<BK_, BN_, WN_, F8_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes, \
+                                              stream>>>(p);                                                        \
     }
+#define TL_LAUNCH_GEMM(BK_, BN_, WN_)                                                                              \
+    { if (es == 1) TL_LAUNCH_GEMM_T(BK_, BN_, WN_, true) else TL_LAUNCH_GEMM_T(BK_, BN_, WN_, false) }
 #define TL_LAUNCH_GEMM_BN(BK_, WN_)                                                                                \
     if (plan.BN == 64) TL_LAUNCH_GEMM(BK_, 64, WN_) else if (plan.BN == 128) TL_LAUNCH_GEMM(BK_, 128, WN_)        \
     else TL_LAUNCH_GEMM(BK_, 256, WN_)
@@ -1156,6 +1167,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         err = cudaLaunchKernelEx(&cfg, streamk_reduce_kernel, p, plan.grid);
     }
 #undef TL_LAUNCH_GEMM
+#undef TL_LAUNCH_GEMM_T
     if (err != cudaSuccess) return check_cuda(err);
     return check_cuda(cudaGetLastError());
 }

@@ -112,6 +112,7 @@ __device__ __forceinline__ void pair_tile_coords(int tile, int m_tiles, int n_ti
 
 // One cluster = one 256-token x 256-column output tile at a time; CTA rank r owns columns n0 + 128 r .. + 127.
 // Dense problems only (no experts, no stream-K, TMA-readable weights); p.BM == 256, per-CTA tile 128 columns.
+template <bool kFp8>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ GemmParams p) {
     constexpr int kBK = 64, kKSteps = 4;
@@ -224,7 +225,7 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             // fp32 accumulate, bf16 x bf16, A (weights) MN-major, B (tokens) K-major, M = 256 over the pair, N = 256
             // (weights K-major when they are stored [N][K])
             // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
-            const uint32_t idesc = (1u << 4) | (p.fp8 ? 0u : (1u << 7) | (1u << 10)) | (p.w_kmajor ? 0u : (1u << 15)) |
+            const uint32_t idesc = (1u << 4) | (kFp8 ? 0u : (1u << 7) | (1u << 10)) | (p.w_kmajor ? 0u : (1u << 15)) |
                                    ((256u >> 3) << 17) | ((256u >> 4) << 24);
             bool ok = true;
             const long long t_begin = TL_CLK();
@@ -253,9 +254,9 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     const uint32_t sa = sw + kWBytes;
 #pragma unroll
                     for (int j = 0; j < kKSteps; ++j) {
-                        const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j], p.lbo, p.sbo, p.w_layout);
+                        const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j], p.w_desc_hi);
                         const uint64_t tok_desc = make_smem_desc(sa + uint32_t(j) * 32u, 16u, 1024u);
-                        if (p.fp8) umma_pair_f8(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                        if (kFp8) umma_pair_f8(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
                         else umma_pair_bf16(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
                     }
                     umma_pair_commit_both(&empty_bar[stage]);       // frees the stage in both CTAs
