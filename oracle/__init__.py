@@ -34,6 +34,13 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+class HwDesc(ctypes.Structure):
+    """Mirror of tlo_hw_desc (Section 4.3: a tensor view plus the memory tile (a, b) and the leading stride K)."""
+    _fields_ = [("rank", ctypes.c_int32), ("s", ctypes.c_int32), ("dims", ctypes.c_int64 * 5),
+                ("strides", ctypes.c_int64 * 5), ("box", ctypes.c_int64 * 5), ("a", ctypes.c_int64),
+                ("b", ctypes.c_int64), ("K", ctypes.c_int64)]
+
+
 _lib = None
 
 
@@ -71,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.tlo_read_amp_grouped.restype = ctypes.c_int
         L.tlo_read_amp_grouped.argtypes = ([vp, ctypes.c_int] + [i64] * 5 + [ctypes.c_int] + [i64] * 4
                                            + [u64p, u64p, u64p])
+        L.tlo_hw_box_offsets.restype = ctypes.c_int
+        L.tlo_hw_box_offsets.argtypes = [ctypes.POINTER(HwDesc), vp, vp]
         L.tlo_num_threads.restype = ctypes.c_int
         L.tlo_num_threads.argtypes = []
         _lib = L
@@ -198,6 +207,28 @@ def read_amp(M, N, K, BM, BN, BK, layout, G, br, bc, s, per_tile=False):
     if per_tile:
         return int(f.value), int(u.value), int(q.value), pf, pu
     return int(f.value), int(u.value), int(q.value)
+
+
+def hw_desc(dims, strides, box, s, a, b, K) -> HwDesc:
+    d = HwDesc()
+    d.rank, d.s, d.a, d.b, d.K = len(dims), s, a, b, K
+    for k in range(len(dims)):
+        d.dims[k], d.strides[k], d.box[k] = dims[k], strides[k], box[k]
+    return d
+
+
+def hw_box_offsets(desc: HwDesc, coords) -> np.ndarray:
+    """Source byte offsets of one box load in counter order (Section 4.3)."""
+    c = np.ascontiguousarray(coords, dtype=np.int64)
+    assert c.size == desc.rank
+    n = 1
+    for k in range(desc.rank):
+        n *= int(desc.box[k])
+    out = np.empty(n, dtype=np.int64)
+    rc = lib().tlo_hw_box_offsets(ctypes.byref(desc), _ptr(c), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"tlo_hw_box_offsets rejected its arguments (rc={rc})")
+    return out
 
 
 def read_amp_grouped(offsets, N, K, BM, BN, BK, layout, G, br, bc, s):

@@ -12,6 +12,78 @@
 #include <omp.h>
 #endif
 
+/* ------------------------------------------------ Section 4.3: TileLens-HW */
+
+static int is_pow2_i64(int64_t x) { return x > 0 && (x & (x - 1)) == 0; }
+static int log2_i64(int64_t x) { int l = 0; while (((int64_t)1 << l) < x) ++l; return l; }
+
+int tlo_hw_box_offsets(const tlo_hw_desc* d, const int64_t* coords, int64_t* out) {
+    if (d->rank < 2 || d->rank > 5 || d->s <= 0 || d->strides[0] != 1) return -1;
+    if (!is_pow2_i64(d->a) || !is_pow2_i64(d->b) || d->K <= 0 || d->K % d->a != 0) return -1;
+    const int64_t u = d->box[0];
+    if (!is_pow2_i64(u) || u > d->a) return -1;           /* invariant 1; the section covers a == u and a > u */
+    /* Case 2 computes everything "as if the memory tile size is u x b" */
+    const int64_t a_eff = u;
+
+    /* Phase 1: split and sum.  Products with a stride below the leading stride add up to i, the rest to K*j. */
+    int64_t i = 0, Kj = 0;
+    for (int k = 0; k < d->rank; ++k) {
+        if (coords[k] < 0 || d->box[k] <= 0) return -1;
+        if (d->strides[k] < d->K) i += coords[k] * d->strides[k];
+        else Kj += coords[k] * d->strides[k];
+    }
+    if (i % a_eff != 0 || Kj % (d->K * d->b) != 0) return -1;     /* aligned to memory tiles (Eq. 4's premise) */
+    const int64_t tile_base = (Kj + i * d->b) * d->s;             /* Eq. 4 */
+
+    /* Phase 2: the counters.  Every dimension keeps its counter except the one whose stride is K, which becomes
+     * an inner counter of b steps of stride a and an outer one of v/b steps of stride b*K (Eq. 5).  A stride below
+     * K moves along a column of the matrix by a multiple of the tile width, i.e. over whole memory tiles, each
+     * a*b elements further (Eq. 4's i*b term); a stride above K moves over whole tile columns (its K*j term). */
+    int64_t ext[6], str[6];
+    int n = 0;
+    for (int k = 0; k < d->rank; ++k) {
+        const int64_t sg = d->strides[k], v = d->box[k];
+        if (k == 0) { ext[n] = u; str[n] = 1; ++n; }
+        else if (sg == d->K) {
+            if (v % d->b != 0) return -1;
+            ext[n] = d->b; str[n] = a_eff; ++n;
+            ext[n] = v / d->b; str[n] = d->b * d->K; ++n;
+        } else if (sg < d->K) {
+            if (sg % a_eff != 0) return -1;
+            ext[n] = v; str[n] = sg * d->b; ++n;
+        } else {
+            if (sg % (d->b * d->K) != 0) return -1;
+            ext[n] = v; str[n] = sg; ++n;
+        }
+    }
+    /* Case 2: bit permutation of the intra-tile element offset, (sub-tile | col | row) -> (col | sub-tile | row) */
+    const int row_bits = log2_i64(u), col_bits = log2_i64(d->b), sub_bits = log2_i64(d->a / u);
+
+    int64_t cnt[6] = {0, 0, 0, 0, 0, 0};
+    int64_t total = 1;
+    for (int k = 0; k < n; ++k) total *= ext[k];
+    for (int64_t t = 0; t < total; ++t) {
+        int64_t src = tile_base;
+        for (int k = 0; k < n; ++k) src += cnt[k] * str[k] * d->s;
+        if (sub_bits > 0) {
+            int64_t e = src / d->s;                                  /* element index */
+            const int64_t intra_mask = ((int64_t)1 << (row_bits + col_bits + sub_bits)) - 1;
+            const int64_t intra = e & intra_mask;
+            const int64_t row = intra & (((int64_t)1 << row_bits) - 1);
+            const int64_t col = (intra >> row_bits) & (((int64_t)1 << col_bits) - 1);
+            const int64_t sub = intra >> (row_bits + col_bits);
+            const int64_t fixed = (col << (sub_bits + row_bits)) | (sub << row_bits) | row;
+            src = ((e & ~intra_mask) | fixed) * d->s;
+        }
+        out[t] = src;
+        for (int k = 0; k < n; ++k) {                                /* increment the nested counters */
+            if (++cnt[k] < ext[k]) break;
+            cnt[k] = 0;
+        }
+    }
+    return 0;
+}
+
 int tlo_num_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

@@ -106,6 +106,28 @@ int tlo_read_amp_grouped(const int32_t* offsets, int E, int64_t N, int64_t K,
                          int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
                          uint64_t* fetched, uint64_t* used, uint64_t* requests);
 
+/* Section 4.3 (tile-major aware TMA): a tensor-map-like descriptor of a VIEW of the column-major K x N matrix
+ * (dims/strides/box in elements, strides[0] == 1, dimension 0 contiguous) extended by the two fields the paper
+ * adds: the memory tile (a, b), a contiguous, and the leading stride K. */
+typedef struct {
+    int32_t rank;            /* 2..5 */
+    int32_t s;               /* element bytes */
+    int64_t dims[5];
+    int64_t strides[5];
+    int64_t box[5];          /* the TMA tile; box[0] = u, and v = the extent in the dimension whose stride is K */
+    int64_t a, b;            /* field 1 */
+    int64_t K;               /* field 2 */
+} tlo_hw_desc;
+
+/* The source byte offset of every element of one box load at `coords`, in the order the engine's counters
+ * produce them (dimension 0 fastest), computed the way Section 4.3 describes the hardware: split-and-sum of
+ * coordinate x stride products into i and K*j, tileBase by Eq. 4, the stride-K counter replaced by two nested
+ * counters (Eq. 5), and for a > u (Case 2) everything as if the memory tile were u x b followed by the bit
+ * permutation of the intra-tile offset.  out holds prod(box) entries.  Returns 0, or -1 for a descriptor or
+ * coordinate the section does not cover (u > a, v not a multiple of b, unaligned coordinates, a stride that is
+ * neither below K and a multiple of u, equal to K, nor a multiple of b*K). */
+int tlo_hw_box_offsets(const tlo_hw_desc* d, const int64_t* coords, int64_t* out);
+
 /* Threads the parallel loops above will use. */
 int tlo_num_threads(void);
 
