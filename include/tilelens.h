@@ -45,7 +45,7 @@ typedef enum {
     TL_ERR_UNSUPPORTED = 2,   /* valid request outside what the kernels instantiate */
     TL_ERR_ALIGNMENT = 3,     /* pointer or pitch not aligned as the call requires */
     TL_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed: see tl_last_cuda_error() */
-    TL_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired */
+    TL_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired, or a kernel refused an input (detail code) */
     TL_ERR_WORKSPACE = 6      /* caller-supplied workspace too small */
 } tl_status;
 
@@ -237,6 +237,46 @@ int tl_gemm_noalloc(const void* d_A_rowmajor, const void* d_B_tilemajor, float* 
                     int64_t G, int block_rows, int block_cols,
                     int cta_m, int cta_n, int cta_k,
                     uint32_t* d_timeout_flag, void* cuda_stream);
+
+/* ------------------------------------- tile-major aware box loads (TileLens-HW) */
+
+/*
+ * Section 4.3 proposes to extend the TMA's source-address computation so that kernels keep their tensor views and
+ * only the descriptor changes.  These two calls emulate that engine in software on a tile-major buffer.
+ * The descriptor is a tensor-map-like VIEW of the column-major K x N matrix (K contiguous): extents, strides and
+ * box in ELEMENTS, strides[0] == 1, the other dimensions in any order, plus the two fields the section adds:
+ * the memory tile (tile_a contiguous K-elements x tile_b columns, Eq. 1-2) and the leading stride K.
+ * Covered, as in the section: box[0] = u a power of two with u == tile_a (case 1) or u dividing tile_a (case 2);
+ * the box extent in the dimension whose stride equals K a multiple of tile_b; every other stride either below K
+ * and a multiple of u, or a multiple of tile_b*K.  Anything else returns TL_ERR_UNSUPPORTED (TL_ERR_INVALID_ARG
+ * for malformed descriptors).  Coordinates must be tile-aligned (Eq. 4) and the box inside the tensor; a box that
+ * is not raises the status word (tl_device_status() -> TL_ERR_TIMEOUT with detail 0x900) and is skipped.
+ */
+typedef struct tl_hw_desc {
+    int32_t rank;              /* 2..5 */
+    int32_t elem_bytes;        /* s: 1, 2 or 4 */
+    int64_t dims[5];
+    int64_t strides[5];
+    int32_t box[5];
+    int32_t tile_a, tile_b;    /* field 1: memory tile, tile_a * tile_b * s = G */
+    int64_t leading_stride;    /* field 2: K */
+} tl_hw_desc;
+
+/*
+ * Source byte offsets (into the tile-major buffer) of every element of n_boxes box loads, in the order the
+ * engine's counters produce them (dimension 0 fastest): d_offsets[box * prod(box) + t].  Skipped boxes are
+ * filled with ~0.  desc: host.  d_coords: device, n_boxes x rank int32.  d_offsets: device.  Asynchronous.
+ */
+int tl_hw_box_offsets(const tl_hw_desc* desc, const int32_t* d_coords, int64_t n_boxes, uint64_t* d_offsets,
+                      void* cuda_stream);
+/*
+ * The loads themselves: box i lands densely at d_dst + i * prod(box) * s in coordinate order (the destination
+ * address "simply increments", Section 4.3), read from the tile-major buffer d_src_tilemajor of src_bytes bytes
+ * (the K x N matrix as tl_relayout(rows = N, cols = K, block_rows = tile_b, block_cols = tile_a) writes it).
+ * Nothing outside [0, src_bytes) is read.  Asynchronous on cuda_stream.
+ */
+int tl_hw_box_load(const tl_hw_desc* desc, const void* d_src_tilemajor, uint64_t src_bytes, const int32_t* d_coords,
+                   int64_t n_boxes, void* d_dst, void* cuda_stream);
 
 /* --------------------------------------------------- read amplification */
 

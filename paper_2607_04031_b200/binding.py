@@ -36,6 +36,8 @@ _SIGNATURES = {
     "tl_gemm_fp8_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped_fp8_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int,
                                           _int, _vp]),
+    "tl_hw_box_offsets": (_int, [_vp, _vp, _i64, _vp, _vp]),
+    "tl_hw_box_load": (_int, [_vp, _vp, ctypes.c_uint64, _vp, _i64, _vp, _vp]),
     "tl_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int, _int, _int]),
     "tl_set_workspace": (_int, [_vp, _sz]),
     "tl_gemm_host": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp, _sz, _vp]),
@@ -200,6 +202,34 @@ def gemm_noalloc(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, M: int, N: i
     flag = _dev_ptr(timeout_flag) if timeout_flag is not None else None
     _check(lib().tl_gemm_noalloc(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), M, N, K, G, block_rows, block_cols,
                                  cta[0], cta[1], cta[2], flag, _stream_ptr(stream)), "tl_gemm_noalloc")
+
+
+class HwDesc(ctypes.Structure):
+    """tl_hw_desc: a tensor view of the column-major K x N matrix plus the memory tile (a, b) and the leading stride."""
+    _fields_ = [("rank", ctypes.c_int32), ("elem_bytes", ctypes.c_int32), ("dims", ctypes.c_int64 * 5),
+                ("strides", ctypes.c_int64 * 5), ("box", ctypes.c_int32 * 5), ("tile_a", ctypes.c_int32),
+                ("tile_b", ctypes.c_int32), ("leading_stride", ctypes.c_int64)]
+
+
+def hw_desc(dims, strides, box, elem_bytes: int, tile_a: int, tile_b: int, leading_stride: int) -> HwDesc:
+    d = HwDesc()
+    d.rank, d.elem_bytes, d.tile_a, d.tile_b, d.leading_stride = len(dims), elem_bytes, tile_a, tile_b, leading_stride
+    for k in range(min(len(dims), 5)):
+        d.dims[k], d.strides[k], d.box[k] = dims[k], strides[k], box[k]
+    return d
+
+
+def hw_box_offsets(desc: HwDesc, coords: torch.Tensor, offsets: torch.Tensor, stream=None):
+    """coords: int32 CUDA tensor [n_boxes, rank]; offsets: uint64/int64 CUDA tensor [n_boxes * prod(box)]."""
+    _check(lib().tl_hw_box_offsets(ctypes.addressof(desc), _dev_ptr(coords), coords.shape[0], _dev_ptr(offsets),
+                                   _stream_ptr(stream)), "tl_hw_box_offsets")
+
+
+def hw_box_load(desc: HwDesc, src: torch.Tensor, coords: torch.Tensor, dst: torch.Tensor, stream=None):
+    """src: the tile-major buffer; dst: n_boxes dense boxes."""
+    _check(lib().tl_hw_box_load(ctypes.addressof(desc), _dev_ptr(src), src.numel() * src.element_size(),
+                                _dev_ptr(coords), coords.shape[0], _dev_ptr(dst), _stream_ptr(stream)),
+           "tl_hw_box_load")
 
 
 def read_amp(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int = 0, block_cols: int = 0,
