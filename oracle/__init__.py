@@ -78,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.tlo_read_amp_grouped.restype = ctypes.c_int
         L.tlo_read_amp_grouped.argtypes = ([vp, ctypes.c_int] + [i64] * 5 + [ctypes.c_int] + [i64] * 4
                                            + [u64p, u64p, u64p])
+        L.tlo_read_amp_shared.restype = ctypes.c_int
+        L.tlo_read_amp_shared.argtypes = [i64] * 7 + [ctypes.c_int] + [i64] * 4 + [u64p, u64p, u64p]
+        L.tlo_prefetch_degree.restype = i64
+        L.tlo_prefetch_degree.argtypes = [ctypes.c_double, ctypes.c_double, i64, i64, i64, i64, i64, i64, ctypes.c_double]
         L.tlo_hw_box_offsets.restype = ctypes.c_int
         L.tlo_hw_box_offsets.argtypes = [ctypes.POINTER(HwDesc), vp, vp]
         L.tlo_num_threads.restype = ctypes.c_int
@@ -207,6 +211,23 @@ def read_amp(M, N, K, BM, BN, BK, layout, G, br, bc, s, per_tile=False):
     if per_tile:
         return int(f.value), int(u.value), int(q.value), pf, pu
     return int(f.value), int(u.value), int(q.value)
+
+
+def read_amp_shared(M, N, K, BM, BN, BK, P, layout, G, br, bc, s):
+    """(fetched, needed, requests) when the P co-resident CTA tiles share the blocks they want at the same K step."""
+    f, u, q = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    rc = lib().tlo_read_amp_shared(M, N, K, BM, BN, BK, P, layout, G, br, bc, s,
+                                   ctypes.byref(f), ctypes.byref(u), ctypes.byref(q))
+    if rc != 0:
+        raise ValueError(f"tlo_read_amp_shared rejected its arguments (rc={rc})")
+    return int(f.value), int(u.value), int(q.value)
+
+
+def prefetch_degree(bandwidth, latency, G, n_sm, ctas_per_sm, p_tile, K, tile_k, collision_factor=1.0) -> int:
+    d = int(lib().tlo_prefetch_degree(bandwidth, latency, G, n_sm, ctas_per_sm, p_tile, K, tile_k, collision_factor))
+    if d < 0:
+        raise ValueError("tlo_prefetch_degree rejected its arguments")
+    return d
 
 
 def hw_desc(dims, strides, box, s, a, b, K) -> HwDesc:

@@ -400,3 +400,83 @@ int tlo_read_amp_grouped(const int32_t* offsets, int E, int64_t N, int64_t K,
     if (requests) *requests = q;
     return 0;
 }
+
+/* Sections 2.5 and 6.5 (requests shared between CTAs): the count when the CTAs that are resident together step
+ * through K together and a block wanted by several of them at the same step is fetched once.  CTA tiles are
+ * numbered n-tile major, m-tile minor; wave w holds tiles [w*P, (w+1)*P).  For every wave and every K iteration
+ * the blocks of all its tiles' weight rectangles are marked element by element in one set. */
+int tlo_read_amp_shared(int64_t M, int64_t N, int64_t K, int64_t BM, int64_t BN, int64_t BK, int64_t P,
+                        int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                        uint64_t* fetched, uint64_t* needed, uint64_t* requests) {
+    if (M < 0 || P <= 0 || !read_amp_args_ok(N, K, BM, BN, BK, layout, G, br, bc, s)) return -1;
+    const int64_t mt = ceil_div(M, BM), nt = ceil_div(N, BN), kt = ceil_div(K, BK);
+    const int64_t T = mt * nt, waves = ceil_div(T, P);
+    const int64_t total_blocks = ceil_div(K * N * s, G) + 1;
+    uint64_t f_sum = 0, u_sum = 0, q_sum = 0;
+    int failed = 0;
+#pragma omp parallel reduction(+ : f_sum, u_sum, q_sum)
+    {
+        unsigned char* mark = (unsigned char*)calloc((size_t)total_blocks, 1);
+        unsigned char* col_seen = (unsigned char*)calloc((size_t)N, 1);
+        if (!mark || !col_seen) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t w = 0; w < waves; ++w) {
+            if (!mark || !col_seen) continue;
+            const int64_t t0 = w * P, t1 = t0 + P < T ? t0 + P : T;
+            for (int64_t tk = 0; tk < kt; ++tk) {
+                const int64_t k0 = tk * BK, k1 = k0 + BK < K ? k0 + BK : K;
+                uint64_t blocks = 0, cols = 0;
+                for (int64_t t = t0; t < t1; ++t) {               /* every CTA tile of the wave */
+                    const int64_t tn = t / mt;
+                    const int64_t n0 = tn * BN, n1 = n0 + BN < N ? n0 + BN : N;
+                    for (int64_t k = k0; k < k1; ++k)
+                        for (int64_t n = n0; n < n1; ++n) {
+                            int64_t off = tlo_off(layout, k, n, K, N, br, bc, s);
+                            int64_t first = off / G, last = (off + s - 1) / G;
+                            if (!mark[first]) { mark[first] = 1; ++blocks; }
+                            if (!mark[last])  { mark[last] = 1;  ++blocks; }
+                        }
+                    for (int64_t n = n0; n < n1; ++n)
+                        if (!col_seen[n]) { col_seen[n] = 1; ++cols; }
+                }
+                for (int64_t t = t0; t < t1; ++t) {               /* clear the marks again */
+                    const int64_t tn = t / mt;
+                    const int64_t n0 = tn * BN, n1 = n0 + BN < N ? n0 + BN : N;
+                    for (int64_t k = k0; k < k1; ++k)
+                        for (int64_t n = n0; n < n1; ++n) {
+                            int64_t off = tlo_off(layout, k, n, K, N, br, bc, s);
+                            mark[off / G] = 0;
+                            mark[(off + s - 1) / G] = 0;
+                        }
+                    for (int64_t n = n0; n < n1; ++n) col_seen[n] = 0;
+                }
+                f_sum += blocks * (uint64_t)G;
+                q_sum += blocks;
+                u_sum += cols * (uint64_t)(k1 - k0) * (uint64_t)s;
+            }
+        }
+        free(mark);
+        free(col_seen);
+    }
+    if (failed) return -2;
+    *fetched = f_sum;
+    *needed = u_sum;
+    *requests = q_sum;
+    return 0;
+}
+
+/* Section 5.2, Eq. 6: prefetch degree.  BL = bandwidth * latency / G requests keep the bus busy; a wave issues
+ * p_wave = n_sm * ctas_per_sm * p_tile demand requests per K iteration; d = min(floor(c * BL / p_wave), K / TILE_K)
+ * with c = 1 as printed (the text then doubles the first term in practice: c = 2). */
+int64_t tlo_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64_t G, int64_t n_sm, int64_t ctas_per_sm,
+                            int64_t p_tile, int64_t K, int64_t tile_k, double collision_factor) {
+    if (G <= 0 || n_sm <= 0 || ctas_per_sm <= 0 || p_tile <= 0 || K <= 0 || tile_k <= 0) return -1;
+    const double BL = bandwidth_bytes_per_s * latency_s / (double)G;
+    const double p_wave = (double)n_sm * (double)ctas_per_sm * (double)p_tile;
+    int64_t d = (int64_t)floor(collision_factor * BL / p_wave);
+    const int64_t cap = K / tile_k;
+    return d < cap ? d : cap;
+}

@@ -106,6 +106,21 @@ int tlo_read_amp_grouped(const int32_t* offsets, int E, int64_t N, int64_t K,
                          int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
                          uint64_t* fetched, uint64_t* used, uint64_t* requests);
 
+/* Sections 2.5 / 6.5 (CTAs share requests): as tlo_read_amp, but the P CTA tiles resident together (tiles numbered
+ * n-tile major, m-tile minor; wave w = tiles [w*P, (w+1)*P)) step through K together and fetch a block once per
+ * step however many of them want it.  needed = distinct weight bytes the wave's tiles use per step, summed.
+ * P = 1 reproduces tlo_read_amp.  The paper's 10.1x / 3.9x come from its simulator's caches and are not this
+ * count: the function is pinned to closed forms and to tlo_read_amp, not to those figures. */
+int tlo_read_amp_shared(int64_t M, int64_t N, int64_t K, int64_t BM, int64_t BN, int64_t BK, int64_t P,
+                        int layout, int64_t G, int64_t br, int64_t bc, int64_t s,
+                        uint64_t* fetched, uint64_t* needed, uint64_t* requests);
+
+/* Eq. 6 (Section 5.2): stride-prefetch degree d = min(floor(c*B*L/p_wave), K/TILE_K), B*L in requests of G bytes,
+ * p_wave = n_sm * ctas_per_sm * p_tile; c = 1 as printed, 2 "in practice".  Pinned by the inequality the paper
+ * derives it from (p_wave*(d+1) >= B*L > p_wave*d when not capped) and its monotonicity, not by a printed value. */
+int64_t tlo_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64_t G, int64_t n_sm, int64_t ctas_per_sm,
+                            int64_t p_tile, int64_t K, int64_t tile_k, double collision_factor);
+
 /* Section 4.3 (tile-major aware TMA): a tensor-map-like descriptor of a VIEW of the column-major K x N matrix
  * (dims/strides/box in elements, strides[0] == 1, dimension 0 contiguous) extended by the two fields the paper
  * adds: the memory tile (a, b), a contiguous, and the leading stride K. */

@@ -211,3 +211,68 @@ def test_k_contiguous_flavour_counts_like_the_transposed_problem():
     # with their two extents exchanged)
     assert tlo.read_amp(3, N, K, 2, 96, 80, tlo.TILE_MAJOR_K, 512, 8, 32, s) == \
         tlo.read_amp(3, K, N, 2, 80, 96, TILE, 512, 8, 32, s)
+
+
+# ------------------------------------------------------------------ requests shared between co-resident CTAs
+def test_shared_count_with_one_cta_per_wave_is_the_plain_count():
+    for layout, br, bc in ((tlo.ROW_MAJOR, 0, 0), (tlo.COL_MAJOR, 0, 0), (tlo.TILE_MAJOR, 4, 16), (tlo.TILE_MAJOR_K, 8, 8)):
+        M, N, K, cta, G, s = 70, 96, 64, (32, 24, 16), 128, 2
+        f, u, q = tlo.read_amp(M, N, K, *cta, layout, G, br, bc, s)
+        assert tlo.read_amp_shared(M, N, K, *cta, 1, layout, G, br, bc, s) == (f, u, q)
+
+
+def test_shared_count_hand_worked_row_major():
+    # 4 x 16 matrix of bytes, G = 8: every row is two blocks.  CTA tiles 4 columns wide, 2 rows deep, one m-tile.
+    # Alone, each of the 4 n-tiles fetches 2 rows x 1 block per K step: 4 tiles x 2 steps x 2 = 16 blocks.
+    # Two tiles per wave: tiles 0,1 both live in columns 0-7 -> the same block per row: 2 waves x 2 steps x 2 = 8.
+    # All four together: each row's two blocks once: 2 steps x 2 rows x 2 blocks = 8 as well.
+    args = (1, 16, 4, 1, 4, 2)
+    assert tlo.read_amp_shared(*args, 1, tlo.ROW_MAJOR, 8, 0, 0, 1) == (16 * 8, 4 * 16, 16)
+    assert tlo.read_amp_shared(*args, 2, tlo.ROW_MAJOR, 8, 0, 0, 1) == (8 * 8, 4 * 16, 8)
+    assert tlo.read_amp_shared(*args, 4, tlo.ROW_MAJOR, 8, 0, 0, 1) == (8 * 8, 4 * 16, 8)
+    # three m-tiles over the same weights, wave of 3 = one n-tile's three CTAs: fetched once, not three times
+    assert tlo.read_amp_shared(3, 16, 4, 1, 4, 2, 3, tlo.ROW_MAJOR, 8, 0, 0, 1) == (16 * 8, 4 * 16, 16)
+    assert tlo.read_amp(3, 16, 4, 1, 4, 2, tlo.ROW_MAJOR, 8, 0, 0, 1)[0] == 3 * 16 * 8
+
+
+@pytest.mark.parametrize("P", [1, 3, 8, 1000])
+def test_shared_count_closed_forms(P):
+    M, N, K, s, G = 256, 1024, 256, 2, 4096
+    cta = (128, 256, 128)
+    # tile-major with tiles inside the CTA tile: every fetched byte is needed, however the waves fall
+    f, u, q = tlo.read_amp_shared(M, N, K, *cta, P, tlo.TILE_MAJOR, G, 16, 128, s)
+    assert f == u
+    f, u, q = tlo.read_amp_shared(M, N, K, *cta, P, tlo.TILE_MAJOR_K, G, 32, 64, s)
+    assert f == u
+    # row-major, pitch 2 KB: a 4 KB block is two whole rows.  A wave covering every n-tile needs whole rows: ratio 1.
+    f, u, q = tlo.read_amp_shared(M, N, K, *cta, P, tlo.ROW_MAJOR, G, 0, 0, s)
+    if P >= 8:
+        assert f == u == K * N * s
+    else:
+        assert u < f <= tlo.read_amp(M, N, K, *cta, tlo.ROW_MAJOR, G, 0, 0, s)[0]
+    # never more than without sharing, never less than what is needed
+    for layout, br, bc in ((tlo.ROW_MAJOR, 0, 0), (tlo.COL_MAJOR, 0, 0)):
+        fs, us, _ = tlo.read_amp_shared(M, N, K, *cta, P, layout, G, br, bc, s)
+        assert us <= fs <= tlo.read_amp(M, N, K, *cta, layout, G, br, bc, s)[0]
+
+
+def test_prefetch_degree_satisfies_the_inequality_it_is_derived_from():
+    # Eq. 6: the largest d with p_wave * d <= B*L (so that p_wave * (d + 1) >= B*L), capped at K / TILE_K
+    B, L, G = 4.9e12, 5e-6, 4096
+    BL = B * L / G
+    for n_sm, c_sm, p_tile, K, tk in [(132, 1, 16, 2048, 128), (132, 1, 128, 2048, 128), (148, 2, 16, 8192, 64),
+                                      (8, 1, 4, 65536, 64), (1, 1, 1, 1 << 20, 64)]:
+        p_wave = n_sm * c_sm * p_tile
+        d = tlo.prefetch_degree(B, L, G, n_sm, c_sm, p_tile, K, tk)
+        cap = K // tk
+        assert 0 <= d <= cap
+        if d < cap:
+            assert p_wave * d <= BL < p_wave * (d + 1)
+        else:
+            assert p_wave * cap <= BL
+        assert tlo.prefetch_degree(B, L, G, n_sm, c_sm, p_tile, K, tk, 2.0) >= d      # "in practice": first term doubled
+    # as thread blocks retire p_wave shrinks and d grows (Section 5.2)
+    ds = [tlo.prefetch_degree(B, L, G, n, 1, 16, 1 << 20, 64) for n in (132, 66, 33, 8, 1)]
+    assert ds == sorted(ds) and ds[0] < ds[-1]
+    # 8x more requests per tile (row-major, Section 6.5) leaves no room for prefetching on the same bus
+    assert tlo.prefetch_degree(B, L, G, 132, 1, 128, 2048, 128) == 0 < tlo.prefetch_degree(B, L, G, 132, 1, 16, 2048, 128)
