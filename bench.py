@@ -477,6 +477,19 @@ def run_ours(args):
         ra[f"{name}_M{M}"] = {"tile_major": t_[0] / t_[1], "row_major": r_[0] / r_[1],
                               "fetched_tile": t_[0], "used": t_[1], "fetched_row": r_[0]}
     extra["read_amp_4KB"] = ra
+    # requests shared between the 148 co-resident CTAs of a wave (prefill tiles 256 x 256 x 64, gate_up), and the
+    # prefetch degree of Eq. 6 that the per-tile request counts imply on the paper's 4.9 TB/s, 5 us device
+    name, K, N = inputs.LLAMA70B_PROJ[2]
+    shared = {}
+    for label, lt, blk in (("row_major", tl.LAYOUT_ROW_MAJOR, (0, 0)), ("tile_major", tl.LAYOUT_TILE_MAJOR, (BR, BC))):
+        plain = tl.read_amp(Mp, N, K, (256, 256, 64), lt, G, blk[0], blk[1], 2)
+        sh = tl.read_amp_shared(Mp, N, K, (256, 256, 64), 148, lt, G, blk[0], blk[1], 2)
+        loads = (-(-Mp // 256)) * (N // 256) * (K // 64)
+        p_tile = max(1, plain[2] // loads)
+        shared[label] = {"unshared": plain[0] / plain[1], "shared_by_wave_of_148": sh[0] / sh[1],
+                         "requests_per_tile": p_tile,
+                         "prefetch_degree_eq6": tl.prefetch_degree(4.9e12, 5e-6, G, 148, 1, p_tile, K, 64, 1.0)}
+    extra["read_amp_shared_prefill_gate_up"] = shared
 
     clocks = sampler.stop()
 

@@ -297,6 +297,27 @@ int tl_read_amp(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k
                 int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
                 uint64_t* bytes_fetched, uint64_t* bytes_used, uint64_t* requests);
 
+/*
+ * The same count when CTAs share requests (Section 2.5: CTAs that want the same 4 KB request; Section 6.5: a
+ * request another CTA already issued): the wave_ctas CTA tiles resident together (tiles numbered n-tile major,
+ * m-tile minor, wave w = tiles [w*wave_ctas, (w+1)*wave_ctas)) step through K together, and a block several of
+ * them want at the same step is fetched once.  bytes_needed = the distinct weight bytes a wave uses per step,
+ * summed.  wave_ctas == 1 gives tl_read_amp's numbers.  Host out-parameters, exact; waits like tl_read_amp.
+ */
+int tl_read_amp_shared(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int64_t wave_ctas,
+                       int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
+                       uint64_t* bytes_fetched, uint64_t* bytes_needed, uint64_t* requests);
+
+/*
+ * Eq. 6 (Section 5.2): the stride-prefetch degree that keeps a bus of the given bandwidth busy over the given
+ * read latency: d = min(floor(c * B*L / p_wave), K / cta_k), B*L counted in requests of G bytes, p_wave = n_sm *
+ * ctas_per_sm * requests_per_tile (the per-tile request count tl_read_amp reports, divided by tiles and
+ * iterations); c = 1 as printed, 2 as the text uses in practice.  Host arithmetic only; -1 for bad arguments.
+ */
+int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64_t G, int64_t n_sm,
+                           int64_t ctas_per_sm, int64_t requests_per_tile, int64_t K, int64_t cta_k,
+                           double collision_factor);
+
 /* Grouped form: sum over experts with rows; h_offsets is a HOST array of E+1 int32. */
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K,
                         int cta_m, int cta_n, int cta_k,

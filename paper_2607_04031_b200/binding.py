@@ -36,6 +36,8 @@ _SIGNATURES = {
     "tl_gemm_fp8_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped_fp8_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int,
                                           _int, _vp]),
+    "tl_read_amp_shared": (_int, [_i64, _i64, _i64, _int, _int, _int, _i64, _int, _i64, _int, _int, _int, _vp, _vp, _vp]),
+    "tl_prefetch_degree": (_i64, [ctypes.c_double, ctypes.c_double, _i64, _i64, _i64, _i64, _i64, _i64, ctypes.c_double]),
     "tl_hw_box_offsets": (_int, [_vp, _vp, _i64, _vp, _vp]),
     "tl_hw_box_load": (_int, [_vp, _vp, ctypes.c_uint64, _vp, _i64, _vp, _vp]),
     "tl_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int, _int, _int]),
@@ -239,6 +241,24 @@ def read_amp(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int =
     _check(lib().tl_read_amp(M, N, K, cta[0], cta[1], cta[2], layout, G, block_rows, block_cols, elem_bytes,
                              ctypes.byref(f), ctypes.byref(u), ctypes.byref(q)), "tl_read_amp")
     return int(f.value), int(u.value), int(q.value)
+
+
+def read_amp_shared(M: int, N: int, K: int, cta, wave_ctas: int, layout: int, G: int, block_rows: int = 0,
+                    block_cols: int = 0, elem_bytes: int = 2):
+    """(bytes_fetched, bytes_needed, requests) when the wave_ctas co-resident CTA tiles share blocks per K step."""
+    f, u, q = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    _check(lib().tl_read_amp_shared(M, N, K, cta[0], cta[1], cta[2], wave_ctas, layout, G, block_rows, block_cols,
+                                    elem_bytes, ctypes.byref(f), ctypes.byref(u), ctypes.byref(q)), "tl_read_amp_shared")
+    return int(f.value), int(u.value), int(q.value)
+
+
+def prefetch_degree(bandwidth_bytes_per_s: float, latency_s: float, G: int, n_sm: int, ctas_per_sm: int,
+                    requests_per_tile: int, K: int, cta_k: int, collision_factor: float = 1.0) -> int:
+    d = int(lib().tl_prefetch_degree(bandwidth_bytes_per_s, latency_s, G, n_sm, ctas_per_sm, requests_per_tile, K,
+                                     cta_k, collision_factor))
+    if d < 0:
+        raise ValueError("tl_prefetch_degree: bad arguments")
+    return d
 
 
 def read_amp_grouped(offsets_host, N: int, K: int, cta, layout: int, G: int, block_rows: int = 0,

@@ -25,6 +25,8 @@ struct ReadAmpParams {
     unsigned long long* d_acc;       // [fetched, used, requests, ticket] totals (may be null); zero between launches
     unsigned long long* h_out;       // mapped pinned host memory: the last warp publishes the totals here
     unsigned long long total_ctas;
+    int64_t wave_tiles;              // > 0: count per wave of this many co-resident CTA tiles (blocks shared)
+    int64_t sched_m_tiles, sched_n_tiles;   // wave mode: the tile grid (tiles numbered n-tile major, m-tile minor)
     int64_t iters_per_warp;          // K iterations one warp covers
     unsigned long long* d_fetched;   // per CTA tile (may be null)
     unsigned long long* d_used;
@@ -45,8 +47,18 @@ __global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
     const int64_t k_chunks = (p.k_iters + p.iters_per_warp - 1) / p.iters_per_warp;
     const bool has_work = warp < p.n_tiles * k_chunks;
     const int64_t tn = has_work ? warp / k_chunks : 0, kc = has_work ? warp % k_chunks : 0;
-    const int64_t n0 = tn * p.BN;
-    const int64_t n1 = n0 + p.BN < p.N ? n0 + p.BN : p.N;
+    int64_t n0 = tn * p.BN;
+    int64_t n1 = n0 + p.BN < p.N ? n0 + p.BN : p.N;
+    if (p.wave_tiles > 0) {
+        // Wave tn holds CTA tiles [tn*P, (tn+1)*P): the n-tiles t/m_tiles of its first and last tile and all
+        // between them.  Their rectangles side by side are one rectangle, whose blocks are counted once.
+        const int64_t total = p.sched_m_tiles * p.sched_n_tiles;
+        const int64_t t0 = tn * p.wave_tiles;
+        const int64_t t1 = (t0 + p.wave_tiles < total ? t0 + p.wave_tiles : total) - 1;
+        n0 = (t0 / p.sched_m_tiles) * p.BN;
+        n1 = (t1 / p.sched_m_tiles + 1) * p.BN;
+        if (n1 > p.N) n1 = p.N;
+    }
     const int64_t it0 = kc * p.iters_per_warp;
     const int64_t it1 = !has_work ? it0 : (it0 + p.iters_per_warp < p.k_iters ? it0 + p.iters_per_warp : p.k_iters);
 
@@ -134,20 +146,28 @@ static int read_amp_validate(int64_t N, int64_t K, int cta_m, int cta_n, int cta
 
 static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
                            int br, int bc, int s, unsigned long long* d_acc, unsigned long long* d_fetched,
-                           unsigned long long* d_used, cudaStream_t stream) {
+                           unsigned long long* d_used, cudaStream_t stream, int64_t wave_tiles = 0) {
     ReadAmpParams p;
     p.N = N; p.K = K; p.BN = cta_n; p.BK = cta_k; p.G = G; p.s = s;
     p.br = br > 0 ? br : 1; p.bc = bc > 0 ? bc : 1; p.layout = layout;
     if (layout == TL_LAYOUT_TILE_MAJOR_K) {
-        // The K x N weight stored with K contiguous IS an N x K matrix with contiguous columns: same blocks,
-        // same tile loads with their two extents exchanged, hence the same count.
-        if (d_fetched || d_used) return TL_ERR_UNSUPPORTED;       // per-tile arrays are indexed by n-tile
-        p.N = K; p.K = N; p.BN = cta_k; p.BK = cta_n;
+        // Either flavour maps memory tiles one to one onto G-byte blocks, so a rectangle of the matrix covers a
+        // rectangle of the tile grid: only the tile's extent along K (here block_cols) and along N (block_rows)
+        // matter to the count.
+        p.br = bc; p.bc = br;
         p.layout = TL_LAYOUT_TILE_MAJOR;
     }
-    p.n_tiles = ceil_div(p.N, p.BN);
-    p.k_iters = ceil_div(p.K, p.BK);
+    p.n_tiles = ceil_div(N, cta_n);
+    p.k_iters = ceil_div(K, cta_k);
     p.m_tiles = m_tiles;
+    p.wave_tiles = wave_tiles;
+    p.sched_m_tiles = m_tiles;
+    p.sched_n_tiles = p.n_tiles;
+    if (wave_tiles > 0) {
+        p.n_tiles = ceil_div(m_tiles * p.n_tiles, wave_tiles);      // one "column" of work per wave
+        p.m_tiles = 1;
+        if (d_fetched || d_used) return TL_ERR_UNSUPPORTED;
+    }
     p.d_acc = d_acc; p.d_fetched = d_fetched; p.d_used = d_used;
     p.h_out = d_acc ? state().ctl.h_acc_dev : nullptr;
     p.iters_per_warp = p.layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
@@ -165,7 +185,8 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
 }
 
 static int read_amp_totals(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
-                           int br, int bc, int s, uint64_t* fetched, uint64_t* used, uint64_t* requests) {
+                           int br, int bc, int s, uint64_t* fetched, uint64_t* used, uint64_t* requests,
+                           int64_t wave_tiles = 0) {
     if (!fetched || !used) return TL_ERR_INVALID_ARG;
     if (int rc = ensure_control()) return rc;
     State& st = state();
@@ -175,7 +196,7 @@ static int read_amp_totals(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
         return TL_OK;
     }
     if (int rc = read_amp_launch(m_tiles, N, K, cta_n, cta_k, layout, G, br, bc, s, st.ctl.d_acc, nullptr, nullptr,
-                                 st.stream))
+                                 st.stream, wave_tiles))
         return rc;
     // the kernel's last warp wrote the totals into mapped pinned memory; the only wait is this one
     volatile unsigned long long* h = st.ctl.h_acc;
@@ -198,6 +219,29 @@ int tl_read_amp(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k
         return rc;
     return tl::read_amp_totals(tl::ceil_div(M, cta_m), N, K, cta_n, cta_k, layout, G, block_rows, block_cols,
                                elem_bytes, bytes_fetched, bytes_used, requests);
+}
+
+int tl_read_amp_shared(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int64_t wave_ctas, int layout,
+                       int64_t G, int block_rows, int block_cols, int elem_bytes, uint64_t* bytes_fetched,
+                       uint64_t* bytes_needed, uint64_t* requests) {
+    if (M < 0 || wave_ctas <= 0) return TL_ERR_INVALID_ARG;
+    if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
+        return rc;
+    return tl::read_amp_totals(tl::ceil_div(M, cta_m), N, K, cta_n, cta_k, layout, G, block_rows, block_cols,
+                               elem_bytes, bytes_fetched, bytes_needed, requests, wave_ctas);
+}
+
+int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64_t G, int64_t n_sm, int64_t ctas_per_sm,
+                           int64_t requests_per_tile, int64_t K, int64_t cta_k, double collision_factor) {
+    if (G <= 0 || n_sm <= 0 || ctas_per_sm <= 0 || requests_per_tile <= 0 || K <= 0 || cta_k <= 0) return -1;
+    if (!(bandwidth_bytes_per_s >= 0.0) || !(latency_s >= 0.0) || !(collision_factor >= 0.0)) return -1;
+    // requests that must be in flight to keep the bus busy, over the requests one wave issues per K iteration
+    const long double in_flight = (long double)bandwidth_bytes_per_s * latency_s / (long double)G * collision_factor;
+    const long double per_wave = (long double)n_sm * (long double)ctas_per_sm * (long double)requests_per_tile;
+    const long double q = in_flight / per_wave;
+    const int64_t cap = K / cta_k;
+    if (q >= (long double)cap) return cap;
+    return (int64_t)q;
 }
 
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,

@@ -112,3 +112,54 @@ def test_empty_and_errors():
     assert tl.read_amp(0, 512, 512, (64, 64, 64), ROW, 4096, 0, 0, 2) == (0, 0, 0)
     with pytest.raises(tl.TileLensError):
         tl.read_amp(1, 512, 512, (64, 64, 64), TILE, 4096, 16, 64, 2)
+
+
+# ------------------------------------------------------------------ requests shared between co-resident CTAs
+SHARED_CASES = [  # M, N, K, cta, G, layout, br, bc, s
+    (70, 96, 64, (32, 24, 16), 128, "row", 0, 0, 2),
+    (70, 96, 64, (32, 24, 16), 128, "col", 0, 0, 2),
+    (70, 96, 64, (32, 24, 16), 128, "tile", 4, 16, 2),
+    (70, 96, 64, (32, 24, 16), 128, "tile_k", 8, 8, 2),
+    (300, 1000, 520, (128, 256, 128), 4096, "row", 0, 0, 2),
+    (300, 1000, 520, (128, 256, 128), 4096, "col", 0, 0, 1),
+    (512, 1536, 2048, (128, 256, 128), 4096, "tile", 32, 64, 2),
+    (512, 1536, 2048, (128, 256, 128), 4096, "tile_k", 32, 64, 2),
+    (512, 1536, 2048, (128, 256, 128), 4096, "row", 0, 0, 2),
+]
+
+
+@pytest.mark.parametrize("case", SHARED_CASES)
+@pytest.mark.parametrize("P", [1, 2, 5, 8, 148, 100000])
+def test_shared_request_count_matches_the_oracle(case, P):
+    from gpu_util import tl
+    M, N, K, cta, G, layout, br, bc, s = case
+    lt = {"row": tl.LAYOUT_ROW_MAJOR, "col": tl.LAYOUT_COL_MAJOR, "tile": tl.LAYOUT_TILE_MAJOR, "tile_k": tl.LAYOUT_TILE_MAJOR_K}[layout]
+    lo = {"row": tlo.ROW_MAJOR, "col": tlo.COL_MAJOR, "tile": tlo.TILE_MAJOR, "tile_k": tlo.TILE_MAJOR_K}[layout]
+    assert tl.read_amp_shared(M, N, K, cta, P, lt, G, br, bc, s) == tlo.read_amp_shared(M, N, K, *cta, P, lo, G, br, bc, s)
+
+
+def test_shared_request_count_full_size_properties():
+    # Llama gate_up, prefill tiles, one wave = 148 CTAs.  Too large for the brute force: properties that hold at any
+    # size -- never above the unshared count, never below what is needed, tile-major exactly what is needed.
+    from gpu_util import tl
+    M, N, K, cta, G = 4096, 57344, 8192, (256, 256, 64), 4096
+    plain = tl.read_amp(M, N, K, cta, tl.LAYOUT_ROW_MAJOR, G, 0, 0, 2)
+    f, u, q = tl.read_amp_shared(M, N, K, cta, 148, tl.LAYOUT_ROW_MAJOR, G, 0, 0, 2)
+    assert u <= f <= plain[0] and f == q * G
+    ft, ut, _ = tl.read_amp_shared(M, N, K, cta, 148, tl.LAYOUT_TILE_MAJOR, G, 16, 128, 2)
+    assert ft == ut
+    # 16 m-tiles share each n-tile: a wave of 148 tiles spans 10 n-tiles, so sharing cuts the row-major traffic
+    assert f * 4 < plain[0]
+
+
+def test_per_cta_counts_k_contiguous_flavour():
+    import torch
+    from gpu_util import DEV, tl
+    M, N, K, cta, G, b, a = 300, 1024, 512, (128, 256, 128), 4096, 32, 64
+    mt, nt = -(-M // cta[0]), -(-N // cta[1])
+    f = torch.zeros(mt * nt, dtype=torch.int64, device=DEV)
+    u = torch.zeros(mt * nt, dtype=torch.int64, device=DEV)
+    tl.read_amp_per_cta(M, N, K, cta, tl.LAYOUT_TILE_MAJOR_K, G, b, a, 2, f, u)
+    torch.cuda.synchronize()
+    _, _, _, pf, pu = tlo.read_amp(M, N, K, *cta, tlo.TILE_MAJOR_K, G, b, a, 2, per_tile=True)
+    assert np.array_equal(f.cpu().numpy().astype(np.uint64), pf) and np.array_equal(u.cpu().numpy().astype(np.uint64), pu)
