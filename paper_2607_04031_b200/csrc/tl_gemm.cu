@@ -51,6 +51,7 @@ struct alignas(64) GemmParams {
     int n_tiles, k_iters;
     int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
     int num_stages;
+    int prefetch_stages;        // stages of weights each CTA asks into L2 before it waits for its predecessor
     // weight-operand geometry
     int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
     int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
@@ -274,6 +275,29 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
     }
 }
 
+// Tensor-map coordinates of the weight box that starts at K element k and weight column n (kc_expert: the
+// expert's offset along the stacked dimension).
+__device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, int n, int kc_expert, int (&c)[5]) {
+    c[0] = 0;
+    if (p.w_kmajor) {
+        // [N][K] storage: (swizzle row of K-elements, row in tile, tile along N, swizzle row in tile, tile along K)
+        if (p.row_major) { c[1] = n + kc_expert; c[2] = 0; c[3] = k >> p.w_atom_log2; c[4] = 0; }
+        else {
+            c[1] = n & ((1 << p.br_log2) - 1);
+            c[2] = (n >> p.br_log2) + kc_expert;
+            c[3] = (k & ((1 << p.bc_log2) - 1)) >> p.w_atom_log2;
+            c[4] = k >> p.bc_log2;
+        }
+    } else if (p.row_major) { c[1] = k + kc_expert; c[2] = n >> 6; c[3] = 0; c[4] = 0; }
+    else {
+        // (64 N-elements, row in tile, atom in tile, tile along N, tile along K)
+        c[1] = k & ((1 << p.br_log2) - 1);
+        c[2] = (n & ((1 << p.bc_log2) - 1)) >> 6;
+        c[3] = n >> p.bc_log2;
+        c[4] = (k >> p.br_log2) + kc_expert;
+    }
+}
+
 // kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256).
 // kWN selects which side of the MMA the weights are on.  A tcgen05.mma of one CTA takes about 180 clocks
 // whatever its shape, so what matters is how many weight bytes one instruction consumes:
@@ -327,6 +351,35 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         tmem_alloc(&tmem_slot, tmem_cols);
         tmem_relinquish();
     }
+    // Dense stream-K problems: while the kernel before this one in the stream is still finishing, ask for the
+    // first stages of this CTA's weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is
+    // the point of coherence, so this is safe whatever that kernel is still writing; it takes the cold start
+    // (page walks, first DRAM accesses) off this kernel's critical path.
+    if (threadIdx.x == 0 && p.stream_k && !p.generic_b && p.offsets == nullptr && p.prefetch_stages > 0) {
+        const int mt = (p.M + p.BM - 1) / p.BM;
+        const long long total = static_cast<long long>(mt) * p.n_tiles * p.k_iters;
+        const int geff = Sched::effective_grid(total, gridDim.x);
+        if (int(blockIdx.x) < geff) {
+            long long it = Sched::split(total, geff, blockIdx.x);
+            const long long it_end = Sched::split(total, geff, blockIdx.x + 1);
+            for (int s = 0; s < p.prefetch_stages && it < it_end; ++s, ++it) {
+                const int tile = int(it / p.k_iters), kit = int(it - static_cast<long long>(tile) * p.k_iters);
+                const int n0 = (tile / mt) * p.BN;
+                const int k0 = (kit * kBK) << p.k_shift;
+                for (int kb = 0; kb < p.kbx; ++kb)
+                    for (int nb = 0; nb < p.nbx; ++nb) {
+                        int c[5];
+                        weight_box_coords(p, k0 + kb * p.box_rows, n0 + nb * p.box_atoms * 64, 0, c);
+                        tma_prefetch_5d(&p.tmap_b, c[0], c[1], c[2], c[3], c[4]);
+                    }
+            }
+        }
+    }
+    // Launched with programmatic stream serialisation: everything above (barriers, tensor memory, descriptor
+    // prefetch) may run while the kernel before this one in the stream is still finishing.  Nothing that kernel
+    // may have written (tokens, expert offsets, the partial-tile workspace, C) is touched before this wait, which
+    // returns once it has completed and its writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // tiles before each expert (dense: one "expert" holding all M rows)
     load_row_starts(p, row_start);
     __syncthreads();
@@ -396,22 +449,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                         for (int nb = 0; nb < p.nbx; ++nb) {
                             const int n = t.n0 + nb * p.box_atoms * 64;
                             uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
-                            if (p.w_kmajor) {
-                                // [N][K] storage: (swizzle row of K-elements, row in tile, tile along N, swizzle
-                                // row in tile, tile along K)
-                                if (p.row_major)
-                                    tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n + kc_expert, 0,
-                                                k >> p.w_atom_log2, 0);
-                                else
-                                    tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, n & ((1 << p.br_log2) - 1),
-                                                (n >> p.br_log2) + kc_expert,
-                                                (k & ((1 << p.bc_log2) - 1)) >> p.w_atom_log2, k >> p.bc_log2);
-                            } else if (p.row_major)
-                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k + kc_expert, n >> 6, 0, 0);
-                            else
-                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], 0, k & ((1 << p.br_log2) - 1),
-                                            (n & ((1 << p.bc_log2) - 1)) >> 6, n >> p.bc_log2,
-                                            (k >> p.br_log2) + kc_expert);
+                            int c[5];
+                            weight_box_coords(p, k, n, kc_expert, c);
+                            tma_load_5d(dst, &p.tmap_b, &full_bar[stage], c[0], c[1], c[2], c[3], c[4]);
                         }
                     }
                     ++issued;
@@ -655,6 +695,9 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
 #ifdef TL_TIMELINE
     if (threadIdx.x == 0 && g_timeline) g_timeline[(256 + blockIdx.x) * 8 + 0] = global_timer_ns();
 #endif
+    // The kernel after this one in the stream may start its own set-up now; it waits for this grid to complete
+    // before it reads or writes anything.
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     load_row_starts(p, row_start);
     __syncthreads();
     if (threadIdx.x < 32) tile_prefix(p, row_start, prefix);
@@ -955,6 +998,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (int rc = get_workspace(plan.ws_bytes, &ws)) return rc;
     }
 
+    static const bool pdl_ok = !(getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0);
     GemmParams p;
     memset(&p, 0, sizeof p);
     // ---- token operand A: [rows_total][K], boxes of 128 bytes of K x {16..256} rows
@@ -1095,6 +1139,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.k_iters = int(ceil_div(K, int64_t(plan.BK) << k_shift));
     p.stream_k = plan.stream_k;
     p.num_stages = plan.num_stages;
+    static const int prefetch_env = getenv("TL_PREFETCH_STAGES") ? atoi(getenv("TL_PREFETCH_STAGES")) : -1;   // measurement hook
+    p.prefetch_stages = !pdl_ok ? 0 : (prefetch_env >= 0 ? prefetch_env : plan.num_stages);
 
     cudaError_t err = cudaSuccess;
     // Large dense problems on TMA-readable weights: CTA pairs (cta_group::2 MMAs), see tl_gemm_pair.cuh.
@@ -1130,6 +1176,9 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         else gemm_pair_kernel<false><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
         return check_cuda(cudaGetLastError());
     }
+    // The GEMM kernel may be scheduled while its predecessor in the stream is finishing (it waits before touching
+    // memory).  TL_NO_PDL=1 restores plain stream order for measurement.
+    const bool pdl_gemm = pdl_ok;
 #define TL_LAUNCH_GEMM_T(BK_, BN_, WN_, F8_)                                                                        \
     {                                                                                                              \
         static bool attr_set = false;                                                                              \
@@ -1138,9 +1187,19 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                                        kMaxDynamicSmem);                                                           \
             attr_set = err == cudaSuccess;                                                                         \
         }                                                                                                          \
-        if (err == cudaSuccess)                                                                                    \
-            gemm_kernel<BK_, BN_, WN_, F8_><<<plan.grid, generic ? kGenericThreads : kGemmThreads, plan.smem_bytes, \
-                                              stream>>>(p);                                                        \
+        if (err == cudaSuccess) {                                                                                  \
+            cudaLaunchConfig_t cfg = {};                                                                           \
+            cfg.gridDim = dim3(plan.grid);                                                                         \
+            cfg.blockDim = dim3(generic ? kGenericThreads : kGemmThreads);                                         \
+            cfg.dynamicSmemBytes = plan.smem_bytes;                                                                \
+            cfg.stream = stream;                                                                                   \
+            cudaLaunchAttribute attr[1];                                                                           \
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                       \
+            attr[0].val.programmaticStreamSerializationAllowed = 1;                                                \
+            cfg.attrs = attr;                                                                                      \
+            cfg.numAttrs = pdl_gemm ? 1 : 0;                                                                       \
+            err = cudaLaunchKernelEx(&cfg, gemm_kernel<BK_, BN_, WN_, F8_>, p);                                    \
+        }                                                                                                          \
     }
 #define TL_LAUNCH_GEMM(BK_, BN_, WN_)                                                                              \
     { if (es == 1) TL_LAUNCH_GEMM_T(BK_, BN_, WN_, true) else TL_LAUNCH_GEMM_T(BK_, BN_, WN_, false) }
