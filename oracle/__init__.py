@@ -82,6 +82,12 @@ def lib() -> ctypes.CDLL:
         L.tlo_read_amp_shared.argtypes = [i64] * 7 + [ctypes.c_int] + [i64] * 4 + [u64p, u64p, u64p]
         L.tlo_prefetch_degree.restype = i64
         L.tlo_prefetch_degree.argtypes = [ctypes.c_double, ctypes.c_double, i64, i64, i64, i64, i64, i64, ctypes.c_double]
+        L.tlo_double_to_bf16.restype = ctypes.c_uint16
+        L.tlo_double_to_bf16.argtypes = [ctypes.c_double]
+        L.tlo_silu.restype = ctypes.c_double
+        L.tlo_silu.argtypes = [ctypes.c_double]
+        L.tlo_moe_ffn_rows.restype = ctypes.c_int
+        L.tlo_moe_ffn_rows.argtypes = [vp, vp, vp, vp, ctypes.c_int, i64, i64, ctypes.c_int, i64, i64, i64, vp, vp, vp, vp]
         L.tlo_hw_box_offsets.restype = ctypes.c_int
         L.tlo_hw_box_offsets.argtypes = [ctypes.POINTER(HwDesc), vp, vp]
         L.tlo_num_threads.restype = ctypes.c_int
@@ -228,6 +234,33 @@ def prefetch_degree(bandwidth, latency, G, n_sm, ctas_per_sm, p_tile, K, tile_k,
     if d < 0:
         raise ValueError("tlo_prefetch_degree rejected its arguments")
     return d
+
+
+def double_to_bf16(x: float) -> int:
+    return int(lib().tlo_double_to_bf16(x))
+
+
+def silu(x: float) -> float:
+    return float(lib().tlo_silu(x))
+
+
+def moe_ffn_rows(X_bits, Wgu_bits, Wd_bits, offsets, hidden, inter, layout, br, bc, rows):
+    """Returns (H bf16 bits [n, inter], Y fp64 [n, hidden], S fp64 [n, hidden]) for the listed rows."""
+    X_bits = np.ascontiguousarray(X_bits, dtype=np.uint16)
+    Wgu_bits = np.ascontiguousarray(Wgu_bits, dtype=np.uint16)
+    Wd_bits = np.ascontiguousarray(Wd_bits, dtype=np.uint16)
+    offs = np.ascontiguousarray(offsets, dtype=np.int32)
+    E = offs.size - 1
+    assert Wgu_bits.size == E * hidden * 2 * inter and Wd_bits.size == E * inter * hidden
+    rr = np.ascontiguousarray(rows, dtype=np.int64)
+    H = np.empty((rr.size, inter), dtype=np.uint16)
+    Y = np.empty((rr.size, hidden), dtype=np.float64)
+    S = np.empty((rr.size, hidden), dtype=np.float64)
+    rc = lib().tlo_moe_ffn_rows(_ptr(X_bits), _ptr(Wgu_bits), _ptr(Wd_bits), _ptr(offs), E, hidden, inter, layout, br, bc,
+                                rr.size, _ptr(rr), _ptr(H), _ptr(Y), _ptr(S))
+    if rc != 0:
+        raise ValueError(f"tlo_moe_ffn_rows rejected its arguments (rc={rc})")
+    return H, Y, S
 
 
 def hw_desc(dims, strides, box, s, a, b, K) -> HwDesc:

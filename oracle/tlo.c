@@ -480,3 +480,67 @@ int64_t tlo_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int6
     const int64_t cap = K / tile_k;
     return d < cap ? d : cap;
 }
+
+/* ------------------------------------------- MoE expert FFN (Section 2.3 names the workload; epilogues are ours)
+ *
+ * The paper's MoE kernel is the two grouped products of an expert FFN; it does not describe what happens between
+ * them.  What is computed here is the usual gated form: h = silu(x W_gate) * (x W_up), rounded once to bf16 (the
+ * intermediate dtype), y = h W_down, everything else in fp64. */
+
+/* double -> bf16 bit pattern, round to nearest, ties to even (through binary32, which holds every bf16 exactly:
+ * the double is first rounded to binary32 by the C conversion, then the low 16 bits are rounded away). */
+uint16_t tlo_double_to_bf16(double x) {
+    float f = (float)x;
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);     /* NaN stays NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+double tlo_silu(double x) { return x / (1.0 + exp(-x)); }
+
+/* h[j] for one row of one expert: gate/up columns interleaved (column 2j = gate_j, 2j+1 = up_j) in the K x 2I weight. */
+static uint16_t ffn_h_at(const uint16_t* x_row, const uint16_t* W_gu, int layout, int64_t br, int64_t bc,
+                         int64_t K, int64_t I, int64_t j) {
+    double g = 0.0, u = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+        double a = tlo_bf16_to_double(x_row[k]);
+        g += a * tlo_bf16_to_double(W_gu[tlo_off(layout, k, 2 * j, K, 2 * I, br, bc, 2) / 2]);
+        u += a * tlo_bf16_to_double(W_gu[tlo_off(layout, k, 2 * j + 1, K, 2 * I, br, bc, 2) / 2]);
+    }
+    return tlo_double_to_bf16(tlo_silu(g) * u);
+}
+
+/* Rows listed in `rows` (indices into the expert-sorted X): H_out[r][0..I) as bf16 bits, Y_out[r][0..hidden) and
+ * S_out[r][.] = sum_j |h_j * Wd[j][c]| in fp64.  offsets: E+1 row offsets of the experts.  Each expert's W_gate_up is
+ * K x 2I, its W_down I x hidden, both in `layout` with memory tile br x bc, experts laid end to end. */
+int tlo_moe_ffn_rows(const uint16_t* X, const uint16_t* W_gu, const uint16_t* W_down, const int32_t* offsets, int E,
+                     int64_t hidden, int64_t I, int layout, int64_t br, int64_t bc,
+                     int64_t n_rows, const int64_t* rows, uint16_t* H_out, double* Y_out, double* S_out) {
+    if (layout == TLO_TILE_MAJOR && (br <= 0 || bc <= 0 || hidden % br || (2 * I) % bc || I % br || hidden % bc)) return -1;
+    for (int64_t t = 0; t < n_rows; ++t)
+        if (rows[t] < 0 || rows[t] >= offsets[E]) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t t = 0; t < n_rows; ++t) {
+        int e = 0;
+        while (!(offsets[e] <= rows[t] && rows[t] < offsets[e + 1])) ++e;
+        const uint16_t* x_row = X + rows[t] * hidden;
+        const uint16_t* wgu = W_gu + (int64_t)e * hidden * 2 * I;
+        const uint16_t* wd = W_down + (int64_t)e * I * hidden;
+        uint16_t* h = H_out + t * I;
+        for (int64_t j = 0; j < I; ++j) h[j] = ffn_h_at(x_row, wgu, layout, br, bc, hidden, I, j);
+        for (int64_t c = 0; c < hidden; ++c) {
+            double acc = 0.0, sab = 0.0;
+            for (int64_t j = 0; j < I; ++j) {
+                double p = tlo_bf16_to_double(h[j]) * tlo_bf16_to_double(wd[tlo_off(layout, j, c, I, hidden, br, bc, 2) / 2]);
+                acc += p;
+                sab += fabs(p);
+            }
+            Y_out[t * hidden + c] = acc;
+            S_out[t * hidden + c] = sab;
+        }
+    }
+    return 0;
+}

@@ -143,6 +143,17 @@ typedef struct {
  * neither below K and a multiple of u, equal to K, nor a multiple of b*K). */
 int tlo_hw_box_offsets(const tlo_hw_desc* d, const int64_t* coords, int64_t* out);
 
+/* double -> bf16 bits (round to nearest even) and silu(x) = x / (1 + exp(-x)). */
+uint16_t tlo_double_to_bf16(double x);
+double tlo_silu(double x);
+/* Gated expert FFN around the two grouped products of the MoE workload (Section 2.3; the paper is silent on what
+ * lies between them): h = bf16(silu(x Wg) * (x Wu)), y = h Wd, gate/up columns interleaved (2j, 2j+1) in the
+ * hidden x 2I weight, for the listed rows of the expert-sorted X.  H_out: n_rows x I bf16 bits, Y_out and
+ * S_out (sum of |h * w| terms): n_rows x hidden doubles. */
+int tlo_moe_ffn_rows(const uint16_t* X, const uint16_t* W_gu, const uint16_t* W_down, const int32_t* offsets, int E,
+                     int64_t hidden, int64_t I, int layout, int64_t br, int64_t bc,
+                     int64_t n_rows, const int64_t* rows, uint16_t* H_out, double* Y_out, double* S_out);
+
 /* Threads the parallel loops above will use. */
 int tlo_num_threads(void);
 
