@@ -464,6 +464,22 @@ def run_ours(args):
         moe.append({"proj": name, "read_amp_128x256_weight_tile": {"tile_major_32x64": ra_t[0] / ra_t[1],
                                                                   "row_major": ra_r[0] / ra_r[1]}})
         del Bm, Bt, Am, Cm
+    # the whole expert FFN in one call: gate_up with the gated epilogue (bf16 h) -> down
+    hid, inter = q["hidden"], q["inter"]
+    Wgu = inputs.bf16_normal((q["experts"], hid, 2 * inter), 0.02, seed=410, device=str(dev))
+    Wdn = inputs.bf16_normal((q["experts"], inter, hid), 0.02, seed=411, device=str(dev))
+    Wgu_t, Wdn_t = torch.empty_like(Wgu), torch.empty_like(Wdn)
+    tl.relayout(Wgu, Wgu_t, q["experts"] * hid, 2 * inter, 2, G, BR, BC, tl.TO_TILE_MAJOR)
+    tl.relayout(Wdn, Wdn_t, q["experts"] * inter, hid, 2, G, BR, BC, tl.TO_TILE_MAJOR)
+    del Wgu, Wdn
+    Xm = inputs.bf16_normal((rows, hid), 1.0, seed=412, device=str(dev))
+    Hm = torch.empty((rows, inter), dtype=torch.bfloat16, device=dev)
+    Ym = torch.empty((rows, hid), dtype=torch.float32, device=dev)
+    ms = time_calls([lambda: tl.moe_ffn(Xm, Wgu_t, Wdn_t, Hm, Ym, d_off, q["experts"], rows, hid, inter, G, BR, BC)], 10)
+    ffn_bytes = active * 2 * (hid * 2 * inter + inter * hid) + 2 * rows * hid + 2 * 2 * rows * inter + 4 * rows * hid
+    moe.append({"proj": "expert_ffn_chain", "layout": "tile", "us": ms * 1e3, "GBps": ffn_bytes / (ms * 1e-3) / 1e9,
+                "active_experts": active, "note": "tl_moe_ffn: grouped gate_up + silu*mul epilogue -> bf16 h -> grouped down"})
+    del Wgu_t, Wdn_t, Xm, Hm, Ym
     extra["qwen_moe"] = moe
     tl.device_status()
 

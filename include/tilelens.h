@@ -140,6 +140,25 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
                     int cta_m, int cta_n, int cta_k, void* cuda_stream);
 
 /*
+ * The expert FFN around the two grouped products (the paper names the fused MoE kernel as its workload, Section
+ * 2.3 and 6.2, and is silent on what lies between the products; the gated form below is this library's choice).
+ * tl_gemm_grouped_swiglu: tl_gemm_grouped whose N = 2*I weight columns hold gate_j in column 2j and up_j in column
+ * 2j+1; instead of C it writes H[row][j] = bf16(silu(g) * u) (fp32 arithmetic, one rounding to nearest even),
+ * d_H_bf16: total_rows x I bf16, 16-byte aligned.  N % 64 == 0; tiles of at most 128 rows (cta_m <= 128), else
+ * TL_ERR_UNSUPPORTED.
+ * tl_moe_ffn: that call followed by tl_gemm_grouped on H and the experts' I x hidden down weights:
+ * Y (fp32, total_rows x hidden) = H x W_down.  Two kernels (plus their stream-K reductions) in stream order, no
+ * host synchronisation; d_H_bf16 is caller-owned scratch that holds H afterwards.
+ */
+int tl_gemm_grouped_swiglu(const void* d_A_sorted, const void* d_B_experts_gate_up, void* d_H_bf16,
+                           const int32_t* d_offsets, int E, int64_t total_rows,
+                           int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                           int cta_m, int cta_n, int cta_k, void* cuda_stream);
+int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_down, void* d_H_bf16, float* d_Y,
+               const int32_t* d_offsets, int E, int64_t total_rows, int64_t hidden, int64_t inter,
+               int64_t G, int block_rows, int block_cols, void* cuda_stream);
+
+/*
  * The same products for weights stored the way deployments keep them (Section 2.4): [N][K] with K contiguous
  * (the "column-major" K x N matrix), tile-major exactly as Eq. 2 prints it: memory tiles of tile_k contiguous
  * K-elements (the paper's a) by tile_n rows along N (the paper's b), tile_n*tile_k*2 == G, tiles ordered along

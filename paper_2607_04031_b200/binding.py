@@ -30,6 +30,9 @@ _SIGNATURES = {
     "tl_relayout_on": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int, _vp]),
     "tl_gemm": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_grouped_swiglu": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int,
+                                      _vp]),
+    "tl_moe_ffn": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _vp]),
     "tl_gemm_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int,
                                       _vp]),
@@ -137,6 +140,23 @@ def gemm_grouped(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, offsets: tor
     _check(lib().tl_gemm_grouped(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), _dev_ptr(offsets), E, total_rows, N, K, G,
                                  block_rows, block_cols, cta[0], cta[1], cta[2], _stream_ptr(stream)),
            "tl_gemm_grouped")
+
+
+def gemm_grouped_swiglu(A: torch.Tensor, B_gate_up: torch.Tensor, H: torch.Tensor, offsets: torch.Tensor, E: int,
+                        total_rows: int, N: int, K: int, G: int = 4096, block_rows: int = 16, block_cols: int = 128,
+                        cta=(0, 0, 0), stream=None):
+    """H (bf16 [rows, N/2]) = silu(gate) * up, gate/up = columns 2j / 2j+1 of A x B."""
+    _check(lib().tl_gemm_grouped_swiglu(_dev_ptr(A), _dev_ptr(B_gate_up), _dev_ptr(H), _dev_ptr(offsets), E, total_rows,
+                                        N, K, G, block_rows, block_cols, cta[0], cta[1], cta[2], _stream_ptr(stream)),
+           "tl_gemm_grouped_swiglu")
+
+
+def moe_ffn(X: torch.Tensor, W_gate_up: torch.Tensor, W_down: torch.Tensor, H: torch.Tensor, Y: torch.Tensor,
+            offsets: torch.Tensor, E: int, total_rows: int, hidden: int, inter: int, G: int = 4096,
+            block_rows: int = 16, block_cols: int = 128, stream=None):
+    _check(lib().tl_moe_ffn(_dev_ptr(X), _dev_ptr(W_gate_up), _dev_ptr(W_down), _dev_ptr(H), _dev_ptr(Y),
+                            _dev_ptr(offsets), E, total_rows, hidden, inter, G, block_rows, block_cols,
+                            _stream_ptr(stream)), "tl_moe_ffn")
 
 
 def gemm_kmajor(A: torch.Tensor, B_nk: torch.Tensor, C: torch.Tensor, M: int, N: int, K: int, G: int = 4096,

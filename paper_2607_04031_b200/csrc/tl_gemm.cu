@@ -22,6 +22,8 @@
 // Every mbarrier wait is bounded (see mbar_wait_bounded).
 #include "tl_common.cuh"
 
+#include <cuda_bf16.h>
+
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -52,6 +54,11 @@ struct alignas(64) GemmParams {
     int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
     int num_stages;
     int prefetch_stages;        // stages of weights each CTA asks into L2 before it waits for its predecessor
+    // Gated epilogue (expert FFN): weight columns 2j / 2j+1 hold gate_j / up_j; H[row][j] = bf16(silu(g) * u)
+    // replaces C.  Weights-on-N kernels only.
+    int epi_swiglu;
+    __nv_bfloat16* H;
+    int64_t ldh;
     // weight-operand geometry
     int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
     int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
@@ -273,6 +280,11 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
             }
         }
     }
+}
+
+// silu(g) * u in fp32, rounded once to bf16 (nearest even).
+__device__ __forceinline__ __nv_bfloat16 swiglu_bf16(float g, float u) {
+    return __float2bfloat16_rn(g / (1.0f + expf(-g)) * u);
 }
 
 // Tensor-map coordinates of the weight box that starts at K element k and weight column n (kc_expert: the
@@ -611,12 +623,28 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * uint32_t(acc_cols);
                 if (quarter * 32 < t.rows) {                     // this lane quarter holds at least one real row
                     float* dst = out + int64_t(row) * ld;
+                    const bool gated = full && p.epi_swiglu;
+                    __nv_bfloat16* hdst = p.H + int64_t(t.row0 + row) * p.ldh + (t.n0 >> 1);
 #pragma unroll 1
                     for (int c0 = 0; c0 < kBN; c0 += 32) {
                         uint32_t v[32];
                         tmem_ld_32x32b_x32(taddr + c0, v);
                         tmem_ld_wait();
-                        if (row < t.rows) {
+                        if (gated) {
+                            // 32 columns = 16 (gate, up) pairs -> 16 bf16 = two 16-byte stores
+                            if (row < t.rows && t.n0 + c0 < p.N) {
+                                uint32_t h2[8];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const __nv_bfloat16 lo = swiglu_bf16(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]));
+                                    const __nv_bfloat16 hi = swiglu_bf16(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                                    h2[i] = uint32_t(__bfloat16_as_ushort(lo)) | (uint32_t(__bfloat16_as_ushort(hi)) << 16);
+                                }
+                                uint4* q = reinterpret_cast<uint4*>(hdst + (c0 >> 1));
+                                q[0] = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+                                q[1] = make_uint4(h2[4], h2[5], h2[6], h2[7]);
+                            }
+                        } else if (row < t.rows) {
 #pragma unroll
                             for (int i = 0; i < 32; i += 4)
                                 if (!full || t.n0 + c0 + i < p.N)
@@ -758,7 +786,15 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
             const int v = v0 + q * 128 + int(threadIdx.x);
             if (v < total_vec) {
                 const int r = v / vec_per_row, c4 = (v % vec_per_row) * 4;
-                if (t.n0 + c4 < p.N) *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
+                if (t.n0 + c4 < p.N) {
+                    if (p.epi_swiglu) {
+                        const __nv_bfloat16 lo = swiglu_bf16(sum[q].x, sum[q].y), hi = swiglu_bf16(sum[q].z, sum[q].w);
+                        *reinterpret_cast<uint32_t*>(p.H + int64_t(t.row0 + r) * p.ldh + ((t.n0 + c4) >> 1)) =
+                            uint32_t(__bfloat16_as_ushort(lo)) | (uint32_t(__bfloat16_as_ushort(hi)) << 16);
+                    } else {
+                        *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
+                    }
+                }
             }
         }
     }
@@ -941,13 +977,14 @@ struct FixedScratch {
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
                        int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
-                       bool kmajor = false, int elem_bytes = 2) {
+                       bool kmajor = false, int elem_bytes = 2, void* d_H_swiglu = nullptr) {
     const int es = elem_bytes;                       // 2: bf16, 1: FP8 (E4M3), K-contiguous weights only
     const int k_shift = es == 1 ? 1 : 0;
     if (es != 2 && !(es == 1 && kmajor)) return TL_ERR_UNSUPPORTED;
     if (rows_total < 0 || N <= 0 || K <= 0 || E < 1) return TL_ERR_INVALID_ARG;
     if (rows_total == 0) return TL_OK;
-    if (!d_A || !d_B || !d_C) return TL_ERR_INVALID_ARG;
+    if (!d_A || !d_B || (!d_C && !d_H_swiglu)) return TL_ERR_INVALID_ARG;
+    if (d_H_swiglu && (N % 64 != 0 || reinterpret_cast<uintptr_t>(d_H_swiglu) % 16 != 0)) return TL_ERR_INVALID_ARG;
     if (rows_total >= (int64_t(1) << 31) || N >= (int64_t(1) << 31) || K * int64_t(E) >= (int64_t(1) << 31))
         return TL_ERR_UNSUPPORTED;
     if (E > kMaxExperts) return TL_ERR_UNSUPPORTED;
@@ -986,7 +1023,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                                d_offsets != nullptr, &plan, fixed != nullptr))
             return rc;
     }
-    if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
+    if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
+    if (d_H_swiglu && !plan.weights_on_n) return TL_ERR_UNSUPPORTED;        // the gated epilogue pairs columns of one token row   // a K tail would read the next expert's rows
     void* ws = nullptr;
     if (fixed) {
         if (plan.ws_bytes > fixed->ws_bytes) return TL_ERR_WORKSPACE;
@@ -1125,6 +1163,9 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     p.w_desc_hi = smem_desc_hi(p.lbo, p.sbo, w_layout);
     p.C = d_C;
+    p.epi_swiglu = d_H_swiglu != nullptr;
+    p.H = static_cast<__nv_bfloat16*>(d_H_swiglu);
+    p.ldh = N / 2;
     p.partials = static_cast<float*>(ws);
     p.offsets = d_offsets;
     p.status = fixed ? fixed->status : state().ctl.d_status;
@@ -1147,7 +1188,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     static const bool no_pair = getenv("TL_NO_PAIR") && atoi(getenv("TL_NO_PAIR")) != 0;     // measurement switch
     // Worth it once every cluster of the machine has at least one 256 x 256 tile; smaller problems keep the
     // single-CTA kernel and its stream-K split.
-    if (!no_pair && !d_offsets && !generic && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
+    if (!no_pair && !d_offsets && !generic && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
         p.kbx == 1 && p.nbx == 1 && ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= state().sm_count) {
         static int max_clusters = -1;
         const int stages = int((kMaxDynamicSmem - 1024) / (64 * 128 * 2 + 128 * kAtomBytes));
@@ -1278,6 +1319,27 @@ int tl_gemm_grouped_fp8_kmajor(const void* d_A_sorted, const void* d_B_experts_n
     if (cta_k != 0 && cta_k != 128 && cta_k != 256) return TL_ERR_UNSUPPORTED;
     return tl::gemm_launch(d_A_sorted, d_B_experts_nk, d_C, d_offsets, E, total_rows, total_rows, N, K, G, tile_n, tile_k,
                            cta_m, cta_n, cta_k / 2, static_cast<cudaStream_t>(cuda_stream), nullptr, true, 1);
+}
+
+int tl_gemm_grouped_swiglu(const void* d_A_sorted, const void* d_B_experts_gate_up, void* d_H_bf16, const int32_t* d_offsets,
+                           int E, int64_t total_rows, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                           int cta_m, int cta_n, int cta_k, void* cuda_stream) {
+    if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
+    if (!d_H_bf16) return TL_ERR_INVALID_ARG;
+    return tl::gemm_launch(d_A_sorted, d_B_experts_gate_up, nullptr, d_offsets, E, total_rows, total_rows, N, K, G,
+                           block_rows, block_cols, cta_m, cta_n, cta_k, static_cast<cudaStream_t>(cuda_stream), nullptr,
+                           false, 2, d_H_bf16);
+}
+
+int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_down, void* d_H_bf16, float* d_Y,
+               const int32_t* d_offsets, int E, int64_t total_rows, int64_t hidden, int64_t inter, int64_t G,
+               int block_rows, int block_cols, void* cuda_stream) {
+    if (hidden <= 0 || inter <= 0) return TL_ERR_INVALID_ARG;
+    if (int rc = tl_gemm_grouped_swiglu(d_X_sorted, d_W_gate_up, d_H_bf16, d_offsets, E, total_rows, 2 * inter, hidden, G,
+                                        block_rows, block_cols, 0, 0, 0, cuda_stream))
+        return rc;
+    return tl_gemm_grouped(d_H_bf16, d_W_down, d_Y, d_offsets, E, total_rows, hidden, inter, G, block_rows, block_cols, 0,
+                           0, 0, cuda_stream);
 }
 
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {
