@@ -54,6 +54,7 @@ struct alignas(64) GemmParams {
     int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
     int num_stages;
     int prefetch_stages;        // stages of weights each CTA asks into L2 before it waits for its predecessor
+    int pair_big_tiles;         // pair kernel with 512-token tiles: how many tiles are of that size (the rest 256)
     // Gated epilogue (expert FFN): weight columns 2j / 2j+1 hold gate_j / up_j; H[row][j] = bf16(silu(g) * u)
     // replaces C.  Weights-on-N kernels only.
     int epi_swiglu;
@@ -1191,30 +1192,48 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (!no_pair && !d_offsets && !generic && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
         p.kbx == 1 && p.nbx == 1 && ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= state().sm_count) {
         static int max_clusters = -1;
-        const int stages = int((kMaxDynamicSmem - 1024) / (64 * 128 * 2 + 128 * kAtomBytes));
-        p.num_stages = stages < kPairStagesMax ? stages : kPairStagesMax;
-        const size_t smem = size_t(p.num_stages) * (64 * 128 * 2 + 128 * kAtomBytes) + 1024;
         if (max_clusters < 0) {
-            err = cudaFuncSetAttribute(gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
-            if (err != cudaSuccess) return check_cuda(err);
-            err = cudaFuncSetAttribute(gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            err = cudaFuncSetAttribute(gemm_pair_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            if (err == cudaSuccess)
+                err = cudaFuncSetAttribute(gemm_pair_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            if (err == cudaSuccess)
+                err = cudaFuncSetAttribute(gemm_pair_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            if (err == cudaSuccess)
+                err = cudaFuncSetAttribute(gemm_pair_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
             if (err != cudaSuccess) return check_cuda(err);
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(2 * state().sm_count);
             cfg.blockDim = dim3(kGemmThreads);
-            cfg.dynamicSmemBytes = smem;
+            cfg.dynamicSmemBytes = kMaxDynamicSmem;
             int n = 0;
-            err = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<false>, &cfg);
+            err = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<false, 1>, &cfg);
             if (err != cudaSuccess) return check_cuda(err);
             max_clusters = n > 0 ? n : 1;
         }
-        const int64_t pair_tiles = ceil_div(rows_total, 256) * ceil_div(N, 256);
+        // 512-token tiles (one weight slab per stage for two token blocks) as long as they fill whole waves of
+        // clusters; what is left of the tile grid runs as 256-token tiles.  TL_PAIR_HALVES=1: 256-token tiles only.
+        static const bool halves_off = getenv("TL_PAIR_HALVES") && atoi(getenv("TL_PAIR_HALVES")) == 1;
+        const int64_t big_total = ceil_div(rows_total, 512) * ceil_div(N, 256);
+        const int64_t big_tiles = halves_off ? 0 : (big_total / max_clusters) * max_clusters;
+        const int halves = big_tiles > 0 ? 2 : 1;
+        const size_t stage_bytes = 64 * 128 * 2 + size_t(halves) * 128 * kAtomBytes;
+        const int stages = int((kMaxDynamicSmem - 1024) / stage_bytes);
+        p.num_stages = stages < kPairStagesMax ? stages : kPairStagesMax;
+        p.pair_big_tiles = int(big_tiles);
+        const size_t smem = size_t(p.num_stages) * stage_bytes + 1024;
+        const int64_t pair_tiles = halves == 2 ? big_tiles + 2 * (big_total - big_tiles)
+                                               : ceil_div(rows_total, 256) * ceil_div(N, 256);
         const int clusters = int(pair_tiles < max_clusters ? pair_tiles : max_clusters);
         if (getenv("TL_LOG"))
-            fprintf(stderr, "[tilelens] pair kernel: %lld tiles of 256x256, %d clusters (max active %d), %d stages, %zu B smem\n",
-                    (long long)pair_tiles, clusters, max_clusters, p.num_stages, smem);
-        if (es == 1) gemm_pair_kernel<true><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
-        else gemm_pair_kernel<false><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
+            fprintf(stderr, "[tilelens] pair kernel: %lld tiles (%lld of 512 tokens), %d clusters (max active %d), %d stages, %zu B smem\n",
+                    (long long)pair_tiles, (long long)big_tiles, clusters, max_clusters, p.num_stages, smem);
+        if (halves == 2) {
+            if (es == 1) gemm_pair_kernel<true, 2><<<2 * clusters, kGenericThreads, smem, stream>>>(p);
+            else gemm_pair_kernel<false, 2><<<2 * clusters, kGenericThreads, smem, stream>>>(p);
+        } else {
+            if (es == 1) gemm_pair_kernel<true, 1><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
+            else gemm_pair_kernel<false, 1><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
+        }
         return check_cuda(cudaGetLastError());
     }
     // The GEMM kernel may be scheduled while its predecessor in the stream is finishing (it waits before touching

@@ -110,15 +110,49 @@ __device__ __forceinline__ void pair_tile_coords(int tile, int m_tiles, int n_ti
     *n_tile = r / band_rows;
 }
 
-// One cluster = one 256-token x 256-column output tile at a time; CTA rank r owns columns n0 + 128 r .. + 127.
+// One output tile of the pair kernel: rows [row0, row0 + 256 * halves) x weight columns of pair tile n_tile.
+struct PairTile {
+    int row0, n_tile, halves;
+};
+
+// kHalves = 1: every tile is 256 tokens x 256 columns.  kHalves = 2: the first p.pair_big_tiles tiles are
+// 512 tokens x 256 columns (numbered like the 256-token tiles, over 512-row m-tiles); what is left of the grid
+// of big tiles follows as 256-token tiles, two per big tile, so that the last wave is not half empty.
+template <int kHalves>
+__device__ __forceinline__ PairTile pair_decode(const GemmParams& p, int tile, int m_tiles, int n_tiles) {
+    PairTile t;
+    int m_tile;
+    if (kHalves == 1) {
+        pair_tile_coords(tile, m_tiles, n_tiles, &m_tile, &t.n_tile);
+        t.row0 = m_tile * 256;
+        t.halves = 1;
+    } else if (tile < p.pair_big_tiles) {
+        pair_tile_coords(tile, m_tiles, n_tiles, &m_tile, &t.n_tile);
+        t.row0 = m_tile * 512;
+        t.halves = p.M - t.row0 > 256 ? 2 : 1;
+    } else {
+        const int s = tile - p.pair_big_tiles;
+        pair_tile_coords(p.pair_big_tiles + (s >> 1), m_tiles, n_tiles, &m_tile, &t.n_tile);
+        t.row0 = m_tile * 512 + (s & 1) * 256;
+        t.halves = t.row0 < p.M ? 1 : 0;                  // 0: nothing there (a ragged last m-tile)
+    }
+    return t;
+}
+
+// One cluster = one output tile at a time (256 or 512 tokens x 256 columns); CTA rank r owns columns
+// n0 + 128 r .. + 127 and loads half of every 256-token block.  With 512-token tiles a stage carries one weight
+// slab for two token blocks (48 KB per CTA instead of 2 x 32 KB for the same work: a quarter less traffic from
+// L2, which is what limits the 256-token form), both accumulators belong to one tile and the epilogue is no
+// longer hidden behind the next tile's MMAs.
 // Dense problems only (no experts, no stream-K, TMA-readable weights); p.BM == 256, per-CTA tile 128 columns.
-template <bool kFp8>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+// kHalves = 2 runs with four more epilogue warps (one set per token block): its epilogue is exposed.
+template <bool kFp8, int kHalves>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kHalves == 2 ? kGenericThreads : kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ GemmParams p) {
     constexpr int kBK = 64, kKSteps = 4;
     constexpr uint32_t kWBytes = kBK * 128 * 2;           // this CTA's weight slab per stage
-    constexpr uint32_t kTokBytes = 128 * kAtomBytes;      // this CTA's half of the token tile per stage
-    constexpr uint32_t kStageBytes = kWBytes + kTokBytes;
+    constexpr uint32_t kTokBytes = 128 * kAtomBytes;      // this CTA's half of one 256-token block per stage
+    constexpr uint32_t kStageBytes = kWBytes + kHalves * kTokBytes;
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kPairStagesMax];     // used in the leader only
@@ -134,7 +168,7 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 8 * kHalves); }
         abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&p.tmap_b);
@@ -153,9 +187,10 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
     const uint32_t tmem_base = tmem_slot;
     volatile uint32_t* abort_ptr = &abort_flag;
 
-    const int m_tiles = (p.M + 255) / 256;
+    const int m_tiles = (p.M + 256 * kHalves - 1) / (256 * kHalves);
     const int n_pair_tiles = (p.N + 255) / 256;
-    const int tiles_total = m_tiles * n_pair_tiles;
+    const int tiles_total = kHalves == 1 ? m_tiles * n_pair_tiles
+                                         : p.pair_big_tiles + 2 * (m_tiles * n_pair_tiles - p.pair_big_tiles);
     const int first_tile = int(cluster_id_x()), tile_step = int(num_clusters_x());
 
 #ifdef TL_TIMELINE
@@ -173,10 +208,10 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             const long long t_begin = TL_CLK();
             (void)t_begin;
             for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
-                int m_tile, n_tile;
-                pair_tile_coords(tile, m_tiles, n_pair_tiles, &m_tile, &n_tile);
-                const int n0 = n_tile * 256 + int(rank) * 128;      // this CTA's weight columns
-                const int row0 = m_tile * 256 + int(rank) * 128;    // this CTA's half of the tokens
+                const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
+                if (pt.halves == 0) continue;
+                const int n0 = pt.n_tile * 256 + int(rank) * 128;   // this CTA's weight columns
+                const int row0 = pt.row0 + int(rank) * 128;         // this CTA's half of the (first) token block
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const long long c0 = TL_CLK();
                     if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
@@ -192,9 +227,11 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     // the arrival, and the peer cannot run a whole ring ahead because its "stage free" barrier
                     // is only signalled after the leader's MMAs have consumed the stage.
                     const uint32_t full_leader = map_to_cta(smem_u32(&full_bar[stage]), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kStageBytes);
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * (kWBytes + uint32_t(pt.halves) * kTokBytes));
                     const int k = (kit * kBK) << p.k_shift;         // K element (8-bit types: twice as many per stage)
                     tma_pair_load_2d(sw + kWBytes, &p.tmap_a[3], full_leader, k, row0);
+                    if (kHalves == 2 && pt.halves == 2)
+                        tma_pair_load_2d(sw + kWBytes + kTokBytes, &p.tmap_a[3], full_leader, k, row0 + 256);
                     if (p.w_kmajor) {
                         if (p.row_major)
                             tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0, 0, k >> p.w_atom_log2, 0);
@@ -231,6 +268,8 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             const long long t_begin = TL_CLK();
             (void)t_begin;
             for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
+                const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
+                if (pt.halves == 0) continue;
                 const long long a0 = TL_CLK();
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) break;
 #ifdef TL_TIMELINE
@@ -258,13 +297,18 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                         const uint64_t tok_desc = make_smem_desc(sa + uint32_t(j) * 32u, 16u, 1024u);
                         if (kFp8) umma_pair_f8(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
                         else umma_pair_bf16(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                        if (kHalves == 2 && pt.halves == 2) {       // the same weights on the second token block
+                            const uint64_t tok2_desc = make_smem_desc(sa + kTokBytes + uint32_t(j) * 32u, 16u, 1024u);
+                            if (kFp8) umma_pair_f8(d_tmem + 256u, w_desc, tok2_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                            else umma_pair_bf16(d_tmem + 256u, w_desc, tok2_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
+                        }
                     }
                     umma_pair_commit_both(&empty_bar[stage]);       // frees the stage in both CTAs
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
                 umma_pair_commit_both(&acc_full_bar[acc]);          // accumulator complete, both CTAs
-                acc ^= 1;
+                if (kHalves == 1) acc ^= 1;                         // (512-token tiles own both accumulators)
                 if (acc == 0) acc_phase ^= 1;
             }
 #ifdef TL_TIMELINE
@@ -274,34 +318,37 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
     } else {
         // =============================================================== epilogue (both CTAs)
         const int quarter = warp & 3;
+        const int my_half = kHalves == 2 ? (warp - 2) >> 2 : 0;     // warps 2..5 drain token block 0, 6..9 block 1
         uint32_t acc = 0, acc_phase = 0;
         for (int tile = first_tile; tile < tiles_total; tile += tile_step) {
-            int m_tile, n_tile;
-            pair_tile_coords(tile, m_tiles, n_pair_tiles, &m_tile, &n_tile);
-            const int n0 = n_tile * 256 + int(rank) * 128;
-            const int row0 = m_tile * 256;
-            const int rows = p.M - row0 < 256 ? p.M - row0 : 256;
+            const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
+            if (pt.halves == 0) continue;
+            const int n0 = pt.n_tile * 256 + int(rank) * 128;
             const bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
             tc_fence_after_sync();
             if (ok) {
                 const int n_local = quarter * 32 + lane;
                 const bool n_ok = n0 + n_local < p.N;
-                float* out = p.C + int64_t(row0) * p.ldc + n0;
-                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256u;
-                for (int c0 = 0; c0 < 256; c0 += 32) {
-                    if (c0 >= rows) break;
-                    uint32_t v[32];
-                    tmem_ld_32x32b_x32(taddr + c0, v);
-                    tmem_ld_wait();
+                for (int h = my_half; h < pt.halves; h += kHalves) {
+                    const int row0 = pt.row0 + h * 256;
+                    const int rows = p.M - row0 < 256 ? p.M - row0 : 256;
+                    float* out = p.C + int64_t(row0) * p.ldc + n0;
+                    const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256u + uint32_t(h) * 256u;
+                    for (int c0 = 0; c0 < 256; c0 += 32) {
+                        if (c0 >= rows) break;
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(taddr + c0, v);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (n_ok && c0 + i < rows) __stcs(out + int64_t(c0 + i) * p.ldc + n_local, __uint_as_float(v[i]));
+                        for (int i = 0; i < 32; ++i)
+                            if (n_ok && c0 + i < rows) __stcs(out + int64_t(c0 + i) * p.ldc + n_local, __uint_as_float(v[i]));
+                    }
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty_bar[acc]), 0));
-            acc ^= 1;
+            if (kHalves == 1) acc ^= 1;
             if (acc == 0) acc_phase ^= 1;
             if (*abort_ptr) break;
         }

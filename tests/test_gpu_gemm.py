@@ -161,6 +161,24 @@ def test_cta_pair_kernel_ragged_shapes(br, bc):
     assert torch.equal(run_gemm(A1, Bd, M, N, K, br, bc).cpu(), B.float()[ks])
 
 
+@pytest.mark.parametrize("M,N", [(1800, 5120), (1224, 7680), (4096, 2560)])
+def test_cta_pair_kernel_512_token_tiles_and_their_remainder(M, N):
+    # Whole waves of clusters take 512-token tiles, what is left of the tile grid runs as 256-token tiles; the last
+    # 512-row m-tile is ragged (264 rows: eight in its second block; 200 rows: second block absent).
+    from gpu_util import run_gemm, tile_major_on_device
+    K, br, bc = 384, 16, 128
+    B = inputs.bf16_integers((K, N), -8, 8, seed=13)
+    Bd = tile_major_on_device(B, K, N, br, bc)
+    A = inputs.bf16_integers((M, K), -8, 8, seed=14)
+    C = run_gemm(A, Bd, M, N, K, br, bc)
+    want = (A.to(torch.float64) @ B.to(torch.float64)).to(torch.float32)          # exact integers
+    rng = np.random.default_rng(2)
+    ii, jj = rng.integers(0, M, 2000), rng.integers(0, N, 2000)
+    ref, _ = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), TILE, br, bc, M, N, K, ii, jj)
+    assert np.array_equal(C.cpu().numpy()[ii, jj].astype(np.float64), ref)
+    assert torch.equal(C.cpu(), want)                                             # every element, against the exact product
+
+
 def test_all_ones_B_gives_row_sums():
     from gpu_util import DEV, run_gemm, tile_major_on_device
     M, N, K = 8, 256, 4096
