@@ -368,7 +368,8 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     // first stages of this CTA's weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is
     // the point of coherence, so this is safe whatever that kernel is still writing; it takes the cold start
     // (page walks, first DRAM accesses) off this kernel's critical path.
-    if (threadIdx.x == 0 && p.stream_k && !p.generic_b && p.offsets == nullptr && p.prefetch_stages > 0) {
+    // (issued by an epilogue thread, which has nothing else to do yet, so that the producer is not held up)
+    if (threadIdx.x == 64 && p.stream_k && !p.generic_b && p.offsets == nullptr && p.prefetch_stages > 0) {
         const int mt = (p.M + p.BM - 1) / p.BM;
         const long long total = static_cast<long long>(mt) * p.n_tiles * p.k_iters;
         const int geff = Sched::effective_grid(total, gridDim.x);
