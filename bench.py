@@ -169,6 +169,23 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------ replicas (the path does not shard)
+
+def max_over_ranks(ms: float, device, world: int) -> float:
+    """The slowest rank's device time; every rank gets the same number."""
+    if world <= 1:
+        return float(ms)
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, steps: int, step_bytes: int, total_ms: float) -> float:
+    """TB/s over all replicas: every rank runs the same step on its own data (weak scaling)."""
+    return world * steps * step_bytes / (total_ms * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------ GPU legs
 
 class EventTimer:
@@ -269,11 +286,8 @@ def run_ours(args):
         dist.barrier()
     total_ms = ev0.elapsed_time(ev1)
     tl.device_status()
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
-    value = world * args.steps * step_bytes / (total_ms * 1e-3) / 1e12
+    total_ms = max_over_ranks(total_ms, dev, world)
+    value = whole_job_value(world, args.steps, step_bytes, total_ms)
     kernel_ms = timer.totals_ms()
 
     if rank != 0:
