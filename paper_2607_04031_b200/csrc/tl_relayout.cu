@@ -235,6 +235,11 @@ __global__ void __launch_bounds__(32, kTmaCtasPerSm) relayout_tma_kernel(const _
     fence_mbar_init();
     tma_prefetch_desc(&p.row_map);
     volatile uint32_t* abort_ptr = &abort_flag;
+    // Launched with programmatic stream serialisation: the set-up above may run while the kernel before this one
+    // in the stream finishes; nothing is read or written before it has completed.  The kernel after this one
+    // may start its own set-up at once (it waits for this grid in the same way).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int64_t first = blockIdx.x, stride = gridDim.x;
     const int64_t mine = first < p.steps_total ? (p.steps_total - first + stride - 1) / stride : 0;
@@ -320,9 +325,19 @@ static int relayout_tma_launch(const void* d_src, void* d_dst, int64_t rows, int
     }
     const int64_t max_grid = int64_t(state().sm_count) * kTmaCtasPerSm;
     const int grid = int(p.steps_total < max_grid ? p.steps_total : max_grid);
-    relayout_tma_kernel<<<grid, 32, smem, stream>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    static const bool no_pdl = getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0;     // measurement switch
+    cfg.numAttrs = no_pdl ? 0 : 1;
     *taken = true;
-    return check_cuda(cudaGetLastError());
+    return check_cuda(cudaLaunchKernelEx(&cfg, relayout_tma_kernel, p));
 }
 
 static int ilog2(int64_t x) {
