@@ -337,6 +337,15 @@ int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64
                            int64_t ctas_per_sm, int64_t requests_per_tile, int64_t K, int64_t cta_k,
                            double collision_factor);
 
+/*
+ * tl_read_amp without the wait: the three totals (bytes_fetched, bytes_used, requests) are written to d_totals,
+ * 3 uint64 in DEVICE memory (or mapped pinned host memory), by the kernel's last CTA.  Asynchronous on
+ * cuda_stream; successive counter calls must be ordered by one stream (they share their accumulators).
+ */
+int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
+                      int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
+                      uint64_t* d_totals, void* cuda_stream);
+
 /* Grouped form: sum over experts with rows; h_offsets is a HOST array of E+1 int32. */
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K,
                         int cta_m, int cta_n, int cta_k,

@@ -39,6 +39,7 @@ _SIGNATURES = {
     "tl_gemm_fp8_kmajor": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped_fp8_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int,
                                           _int, _vp]),
+    "tl_read_amp_async": (_int, [_i64, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int, _vp, _vp]),
     "tl_read_amp_shared": (_int, [_i64, _i64, _i64, _int, _int, _int, _i64, _int, _i64, _int, _int, _int, _vp, _vp, _vp]),
     "tl_prefetch_degree": (_i64, [ctypes.c_double, ctypes.c_double, _i64, _i64, _i64, _i64, _i64, _i64, ctypes.c_double]),
     "tl_hw_box_offsets": (_int, [_vp, _vp, _i64, _vp, _vp]),
@@ -261,6 +262,13 @@ def read_amp(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int =
     _check(lib().tl_read_amp(M, N, K, cta[0], cta[1], cta[2], layout, G, block_rows, block_cols, elem_bytes,
                              ctypes.byref(f), ctypes.byref(u), ctypes.byref(q)), "tl_read_amp")
     return int(f.value), int(u.value), int(q.value)
+
+
+def read_amp_async(M: int, N: int, K: int, cta, layout: int, G: int, block_rows: int, block_cols: int, elem_bytes: int,
+                   totals: torch.Tensor, stream=None):
+    """totals: CUDA tensor of 3 int64/uint64 that receives (bytes_fetched, bytes_used, requests); no wait."""
+    _check(lib().tl_read_amp_async(M, N, K, cta[0], cta[1], cta[2], layout, G, block_rows, block_cols, elem_bytes,
+                                   _dev_ptr(totals), _stream_ptr(stream)), "tl_read_amp_async")
 
 
 def read_amp_shared(M: int, N: int, K: int, cta, wave_ctas: int, layout: int, G: int, block_rows: int = 0,

@@ -12,6 +12,8 @@
 //   col-major   the same with the roles of rows and columns exchanged.
 #include "tl_common.cuh"
 
+#include <cstdlib>
+
 namespace tl {
 
 struct ReadAmpParams {
@@ -44,6 +46,7 @@ __global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
     const int lane = threadIdx.x & 31;
     const int64_t warp = (blockIdx.x * int64_t(blockDim.x) + threadIdx.x) >> 5;
     __shared__ unsigned long long cta_blocks[4], cta_used[4];
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t k_chunks = (p.k_iters + p.iters_per_warp - 1) / p.iters_per_warp;
     const bool has_work = warp < p.n_tiles * k_chunks;
     const int64_t tn = has_work ? warp / k_chunks : 0, kc = has_work ? warp % k_chunks : 0;
@@ -95,6 +98,10 @@ __global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
         }
     }
     blocks = warp_sum(blocks);
+    // Everything above is arithmetic on the launch parameters.  The kernel is launched with programmatic stream
+    // serialisation: only from here on does it touch memory (the accumulators shared with the previous counter
+    // launch, the per-tile arrays the host has just cleared), so only here does it wait for its predecessor.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const unsigned long long fetched = blocks * (unsigned long long)p.G;
     const int64_t k_lo = it0 * p.BK, k_hi = it1 * p.BK < p.K ? it1 * p.BK : p.K;
     const unsigned long long used = has_work ? (unsigned long long)((k_hi - k_lo) * (n1 - n0) * p.s) : 0ull;
@@ -146,7 +153,8 @@ static int read_amp_validate(int64_t N, int64_t K, int cta_m, int cta_n, int cta
 
 static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
                            int br, int bc, int s, unsigned long long* d_acc, unsigned long long* d_fetched,
-                           unsigned long long* d_used, cudaStream_t stream, int64_t wave_tiles = 0) {
+                           unsigned long long* d_used, cudaStream_t stream, int64_t wave_tiles = 0,
+                           unsigned long long* totals_out = nullptr) {
     ReadAmpParams p;
     p.N = N; p.K = K; p.BN = cta_n; p.BK = cta_k; p.G = G; p.s = s;
     p.br = br > 0 ? br : 1; p.bc = bc > 0 ? bc : 1; p.layout = layout;
@@ -169,7 +177,7 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
         if (d_fetched || d_used) return TL_ERR_UNSUPPORTED;
     }
     p.d_acc = d_acc; p.d_fetched = d_fetched; p.d_used = d_used;
-    p.h_out = d_acc ? state().ctl.h_acc_dev : nullptr;
+    p.h_out = d_acc ? (totals_out ? totals_out : state().ctl.h_acc_dev) : nullptr;
     p.iters_per_warp = p.layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
     if (m_tiles == 0) return TL_OK;
     const int warps_per_cta = 4;
@@ -180,8 +188,17 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
         if (int rc = check_cuda(cudaMemsetAsync(d_fetched, 0, bytes, stream))) return rc;
         if (int rc = check_cuda(cudaMemsetAsync(d_used, 0, bytes, stream))) return rc;
     }
-    read_amp_kernel<<<unsigned(grid), warps_per_cta * 32, 0, stream>>>(p);
-    return check_cuda(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(grid));
+    cfg.blockDim = dim3(warps_per_cta * 32);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    static const bool no_pdl = getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0;     // measurement switch
+    cfg.numAttrs = no_pdl ? 0 : 1;
+    return check_cuda(cudaLaunchKernelEx(&cfg, read_amp_kernel, p));
 }
 
 static int read_amp_totals(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
@@ -242,6 +259,21 @@ int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64
     const int64_t cap = K / cta_k;
     if (q >= (long double)cap) return cap;
     return (int64_t)q;
+}
+
+int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int layout, int64_t G,
+                      int block_rows, int block_cols, int elem_bytes, uint64_t* d_totals, void* cuda_stream) {
+    if (M < 0 || !d_totals) return TL_ERR_INVALID_ARG;
+    if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
+        return rc;
+    if (int rc = tl::ensure_control()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (M == 0) return tl::check_cuda(cudaMemsetAsync(d_totals, 0, 3 * sizeof(uint64_t), st));
+    // The accumulators are shared by all launches on the device: launches must be ordered by one stream (they
+    // are between tl_read_amp* calls, which all use the stream they are given or the tl_set_stream() stream).
+    return tl::read_amp_launch(tl::ceil_div(M, cta_m), N, K, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes,
+                               tl::state().ctl.d_acc, nullptr, nullptr, st, 0,
+                               reinterpret_cast<unsigned long long*>(d_totals));
 }
 
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,

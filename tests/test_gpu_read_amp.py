@@ -163,3 +163,17 @@ def test_per_cta_counts_k_contiguous_flavour():
     torch.cuda.synchronize()
     _, _, _, pf, pu = tlo.read_amp(M, N, K, *cta, tlo.TILE_MAJOR_K, G, b, a, 2, per_tile=True)
     assert np.array_equal(f.cpu().numpy().astype(np.uint64), pf) and np.array_equal(u.cpu().numpy().astype(np.uint64), pu)
+
+
+def test_async_totals_match_the_waiting_call_when_queued_back_to_back():
+    import torch
+    from gpu_util import DEV, tl
+    cases = [(8, 10240, 8192, (16, 128, 64), tl.LAYOUT_TILE_MAJOR, 16, 128), (32, 8192, 8192, (32, 128, 64), tl.LAYOUT_ROW_MAJOR, 0, 0),
+             (300, 1000, 520, (128, 256, 128), tl.LAYOUT_COL_MAJOR, 0, 0), (0, 512, 512, (16, 128, 64), tl.LAYOUT_ROW_MAJOR, 0, 0),
+             (1, 57344, 8192, (16, 256, 64), tl.LAYOUT_TILE_MAJOR_K, 32, 64)]
+    out = torch.full((len(cases), 3), -1, dtype=torch.int64, device=DEV)
+    for i, (M, N, K, cta, layout, br, bc) in enumerate(cases):          # all queued before any result is read
+        tl.read_amp_async(M, N, K, cta, layout, 4096, br, bc, 2, out[i])
+    got = out.cpu().numpy()
+    for i, (M, N, K, cta, layout, br, bc) in enumerate(cases):
+        assert tuple(int(x) for x in got[i]) == tl.read_amp(M, N, K, cta, layout, 4096, br, bc, 2)
