@@ -366,31 +366,6 @@ def run_ours(args):
     row_t = sum(x["us"] for x in per_shape if x["layout"] == "row")
     extra["tile_vs_row_time_ratio_decode"] = tile_t / row_t
 
-    # ---- prefill leg (M = 4096): tensor-core bound
-    Mp = inputs.LLAMA_PREFILL_M
-    prefill = []
-    for layout in ("tile", "row"):
-        for name, K, N in inputs.LLAMA70B_PROJ:
-            Ap = inputs.bf16_normal((Mp, K), 1.0, seed=300, device=str(dev))
-            Cp = torch.empty((Mp, N), dtype=torch.float32, device=dev)
-            if layout == "tile":
-                call = lambda: tl.gemm(Ap, W_tile[name], Cp, Mp, N, K, G, BR, BC)
-            else:
-                call = lambda: tl.gemm(Ap, W_row[name], Cp, Mp, N, K, 0, 0, 0)
-            ms = time_calls([call], 5)
-            prefill.append({"proj": name, "layout": layout, "ms": ms, "TFLOPs": 2.0 * Mp * N * K / (ms * 1e-3) / 1e12})
-            del Ap, Cp
-    pt = [x for x in prefill if x["layout"] == "tile"]
-    flops = sum(2.0 * Mp * N * K for _, K, N in inputs.LLAMA70B_PROJ)
-    tf = flops / (sum(x["ms"] for x in pt) * 1e-3) / 1e12
-    extra["prefill"] = {"per_shape": prefill, "TFLOPs_tile_major": tf,
-                        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                                     "frac": tf / peaks["bf16_tflops"], "peak_source": f"of {peaks['source']} (burst)",
-                                     "frac_of_nominal_2250": tf / 2250.0},
-                        "tile_vs_row_time_ratio": sum(x["ms"] for x in pt) /
-                        sum(x["ms"] for x in prefill if x["layout"] == "row")}
-    tl.device_status()
-
     # ---- K-contiguous flavour (weights kept [N][K]; Eq. 2 as printed with the (64, 32) memory tile), M = 8
     W_nk, W_nk_tile = {}, {}
     for name, K, N in inputs.LLAMA70B_PROJ:
@@ -445,6 +420,31 @@ def run_ours(args):
         del W8
     extra["fp8_decode_m8"] = fp8
     del W_nk, W_nk_tile
+    tl.device_status()
+
+    # ---- prefill leg (M = 4096): tensor-core bound
+    Mp = inputs.LLAMA_PREFILL_M
+    prefill = []
+    for layout in ("tile", "row"):
+        for name, K, N in inputs.LLAMA70B_PROJ:
+            Ap = inputs.bf16_normal((Mp, K), 1.0, seed=300, device=str(dev))
+            Cp = torch.empty((Mp, N), dtype=torch.float32, device=dev)
+            if layout == "tile":
+                call = lambda: tl.gemm(Ap, W_tile[name], Cp, Mp, N, K, G, BR, BC)
+            else:
+                call = lambda: tl.gemm(Ap, W_row[name], Cp, Mp, N, K, 0, 0, 0)
+            ms = time_calls([call], 5)
+            prefill.append({"proj": name, "layout": layout, "ms": ms, "TFLOPs": 2.0 * Mp * N * K / (ms * 1e-3) / 1e12})
+            del Ap, Cp
+    pt = [x for x in prefill if x["layout"] == "tile"]
+    flops = sum(2.0 * Mp * N * K for _, K, N in inputs.LLAMA70B_PROJ)
+    tf = flops / (sum(x["ms"] for x in pt) * 1e-3) / 1e12
+    extra["prefill"] = {"per_shape": prefill, "TFLOPs_tile_major": tf,
+                        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                     "frac": tf / peaks["bf16_tflops"], "peak_source": f"of {peaks['source']} (burst)",
+                                     "frac_of_nominal_2250": tf / 2250.0},
+                        "tile_vs_row_time_ratio": sum(x["ms"] for x in pt) /
+                        sum(x["ms"] for x in prefill if x["layout"] == "row")}
     tl.device_status()
 
     # ---- tile-major aware box loads (Section 4.3, emulated): every 64 x 256 weight-tile load of the gate_up weight
