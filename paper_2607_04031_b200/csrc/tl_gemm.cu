@@ -63,6 +63,7 @@ struct alignas(64) GemmParams {
     // weight-operand geometry
     int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
     int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
+    int k_inner;                // 1: tensor-map dimensions ordered (64, row in tile, tile along K, atom, tile along N)
     int fp8;                    // 1: both operands are 8-bit floating point (E4M3); needs w_kmajor
     int k_shift;                // log2(K elements per 2 bytes): a stage holds (BK << k_shift) K-elements
     int w_atom_log2;            // K-major weights: log2(elements in one swizzle row of 128, 64 or 32 bytes)
@@ -302,7 +303,13 @@ __device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, in
             c[4] = k >> p.bc_log2;
         }
     } else if (p.row_major) { c[1] = k + kc_expert; c[2] = n >> 6; c[3] = 0; c[4] = 0; }
-    else {
+    else if (p.k_inner) {
+        // (64 N-elements, row in tile, tile along K, atom in tile, tile along N)
+        c[1] = k & ((1 << p.br_log2) - 1);
+        c[2] = (k >> p.br_log2) + kc_expert;
+        c[3] = (n & ((1 << p.bc_log2) - 1)) >> 6;
+        c[4] = n >> p.bc_log2;
+    } else {
         // (64 N-elements, row in tile, atom in tile, tile along N, tile along K)
         c[1] = k & ((1 << p.br_log2) - 1);
         c[2] = (n & ((1 << p.bc_log2) - 1)) >> 6;
@@ -1003,8 +1010,10 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     // One-row memory tiles are row-major (Section 3.1: the (1, G/s) extreme).
     const bool row_major = br == 0 || (!kmajor && br == 1 && N % 64 == 0);
-    // TMA boxes need whole 8-row x 128-byte swizzle atoms; anything smaller takes the generic-address path.
-    const bool generic = !kmajor && !row_major && (br < 8 || bc < 64);
+    // TMA boxes need 128-byte rows (64 columns); narrower memory tiles take the generic-address path.
+    // 16- and 32-column memory tiles (32- and 64-byte rows) are TMA-boxable with the narrower swizzles.
+    const bool narrow = !kmajor && !row_major && (bc == 16 || bc == 32);
+    const bool generic = !kmajor && !row_major && bc < 64 && !narrow;
     if (!kmajor && row_major && N % 64 != 0) return TL_ERR_UNSUPPORTED;
     if (generic && (G < 16 || br > 128 || bc > 256)) return TL_ERR_UNSUPPORTED;   // tile must fit the CTA tile
     if ((K * es) % 16 != 0) return TL_ERR_UNSUPPORTED;          // 16-byte row pitch of A
@@ -1117,6 +1126,39 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     } else {
         // Eq. 3 in the N-contiguous flavour, contiguous extent split into 64-element atoms:
         // (64, br, bc/64, N/bc, E*K/br) with strides (1, bc, 64, br*bc, br*N) elements.
+        if (narrow) {
+            // Tile rows of 32 or 64 bytes: one tile row is one swizzle row (32- or 64-byte swizzle), dimensions in the
+            // K-inner order described below; the stage lands as [bc-column atom][cta_k rows][bc*2 bytes].
+            const int rows_box = br < plan.BK ? br : plan.BK;
+            RB = plan.BK;
+            AB = NA;
+            const uint64_t dims[5] = {uint64_t(bc), uint64_t(br), uint64_t(K / br) * E, 1, uint64_t(N / bc)};
+            const uint64_t str[5] = {2, uint64_t(bc) * 2, uint64_t(br) * uint64_t(N) * 2, uint64_t(bc) * 2, uint64_t(G)};
+            const uint32_t box[5] = {uint32_t(bc), uint32_t(rows_box), uint32_t(plan.BK / rows_box), 1, uint32_t(plan.BN / bc)};
+            if (int rc = encode_tensor_map(&p.tmap_b, d_B, dtype, bc == 32 ? int(CU_TENSOR_MAP_SWIZZLE_64B) : int(CU_TENSOR_MAP_SWIZZLE_32B),
+                                           5, dims, str, box))
+                return rc;
+            p.k_coord_per_expert = int(K / br);
+            p.br_log2 = ilog2(br);
+            p.bc_log2 = ilog2(bc);
+            p.k_inner = 1;
+        } else if (br < 8) {
+            // Memory tiles shorter than the 8 rows of a swizzle atom: the same view with its dimensions in another
+            // order, (64, br, E*K/br, bc/64, N/bc) with strides (1, bc, br*N, 64, br*bc).  The box takes all K
+            // tiles of the stage before it moves to the next 64-column atom, so under every atom the stage's K
+            // rows follow each other: [N tile][atom][K tile][row][64] = [atom][cta_k rows][64], canonical again.
+            RB = plan.BK;
+            AB = (bc < plan.BN ? bc : plan.BN) / 64;
+            nb_box = NA / AB;
+            const uint64_t dims[5] = {64, uint64_t(br), uint64_t(K / br) * E, uint64_t(bc / 64), uint64_t(N / bc)};
+            const uint64_t str[5] = {2, uint64_t(bc) * 2, uint64_t(br) * uint64_t(N) * 2, 128, uint64_t(G)};
+            const uint32_t box[5] = {64, uint32_t(br), uint32_t(plan.BK / br), uint32_t(AB), uint32_t(nb_box)};
+            if (int rc = encode(&p.tmap_b, d_B, 5, dims, str, box)) return rc;
+            p.k_coord_per_expert = int(K / br);
+            p.br_log2 = ilog2(br);
+            p.bc_log2 = ilog2(bc);
+            p.k_inner = 1;
+        } else {
         RB = br < plan.BK ? br : plan.BK;
         AB = (bc < plan.BN ? bc : plan.BN) / 64;
         // One TMA instruction per stage whose box is a whole number of memory tiles (box extents 3 and 4
@@ -1132,6 +1174,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.k_coord_per_expert = int(K / br);
         p.br_log2 = ilog2(br);
         p.bc_log2 = ilog2(bc);
+        }
     }
     p.row_major = row_major;
     p.kbx = generic ? 0 : plan.BK / (RB * kb_box);
@@ -1148,6 +1191,20 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     for (int j = 0; j < plan.BK / 16; ++j) {
         const int row = j * 16;
         p.kstep_off[j] = uint32_t(row / RB) * krow_bytes + uint32_t(row % RB) * kAtomBytes;
+    }
+    if (narrow) {
+        // MN-major image with narrow atoms: [bc-column atom][cta_k rows][r = bc*2 bytes]; 8-row groups 8r apart, the
+        // next atom cta_k rows further, a K step of 16 rows 16r further.
+        const uint32_t r = uint32_t(bc) * 2u;
+        p.lbo = uint32_t(plan.BK) * r;
+        p.sbo = 8u * r;
+        p.ugroup_off = (128u / uint32_t(bc)) * p.lbo;
+        for (int j = 0; j < plan.BK / 16; ++j) p.kstep_off[j] = uint32_t(j) * 16u * r;
+        p.box_rows = plan.BK;
+        p.box_atoms = NA;
+        p.kbx = p.nbx = 1;
+        p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
+        w_layout = bc == 32 ? 4u : 6u;
     }
     if (kmajor) {
         // K-major image: [swizzle row along K][cta_n rows][r bytes]; 8-row groups 8r bytes apart, a K step of one

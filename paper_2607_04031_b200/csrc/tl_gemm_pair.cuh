@@ -232,17 +232,9 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     tma_pair_load_2d(sw + kWBytes, &p.tmap_a[3], full_leader, k, row0);
                     if (kHalves == 2 && pt.halves == 2)
                         tma_pair_load_2d(sw + kWBytes + kTokBytes, &p.tmap_a[3], full_leader, k, row0 + 256);
-                    if (p.w_kmajor) {
-                        if (p.row_major)
-                            tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0, 0, k >> p.w_atom_log2, 0);
-                        else
-                            tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, n0 & ((1 << p.br_log2) - 1), n0 >> p.br_log2,
-                                             (k & ((1 << p.bc_log2) - 1)) >> p.w_atom_log2, k >> p.bc_log2);
-                    } else if (p.row_major)
-                        tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k, n0 >> 6, 0, 0);
-                    else
-                        tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, k & ((1 << p.br_log2) - 1),
-                                         (n0 & ((1 << p.bc_log2) - 1)) >> 6, n0 >> p.bc_log2, k >> p.br_log2);
+                    int wc[5];
+                    weight_box_coords(p, k, n0, 0, wc);
+                    tma_pair_load_5d(sw, &p.tmap_b, full_leader, wc[0], wc[1], wc[2], wc[3], wc[4]);
                     ++issued;
 #ifdef TL_TIMELINE
                     w_wait += c1 - c0; w_issue += TL_CLK() - c1;

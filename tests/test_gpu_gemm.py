@@ -35,7 +35,8 @@ def test_config1_tiny_tile_major_and_row_major():
 
 # TMA-boxable tiles, row-major, one-row tiles (= row-major), and tiles only the generic-address path can read
 BLOCKS = [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0), (1, 1024), (1, 128),
-          (8, 2), (16, 1), (8, 16), (16, 8), (32, 4), (16, 32), (32, 16), (2, 64), (4, 128), (64, 8)]
+          (8, 2), (16, 1), (8, 16), (16, 8), (32, 4), (16, 32), (32, 16), (2, 64), (4, 128), (64, 8),
+          (2, 1024), (4, 512), (2, 256), (64, 32), (128, 16), (4, 32), (256, 16)]
 
 
 @pytest.mark.parametrize("br,bc", BLOCKS)
@@ -48,7 +49,7 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     A, ks = inputs.one_hot_rows(M, K, seed=7)
     B = inputs.bf16_normal((K, N), 0.02, seed=8)
     Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
-    hand_addressed = br > 1 and (br < 8 or bc < 64)
+    hand_addressed = br > 1 and bc < 16          # rows shorter than 32 bytes; everything else is TMA-boxable
     cta_n, cta_k = (cta[1] or 128), (cta[2] or 64)
     if hand_addressed and (bc > cta_n or br > cta_k):
         # documented limit of the generic-address path: the memory tile must fit inside the CTA tile
@@ -61,15 +62,18 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     assert torch.equal(C.cpu(), B.float()[ks])
 
 
-def test_hand_addressed_tile_wider_than_the_cta_tile():
+def test_short_tiles_wider_than_the_cta_tile_and_hand_addressed_tiles_taller_than_it():
     from gpu_util import run_gemm, tile_major_on_device, tl
     M, N, K = 24, 512, 256
     A, ks = inputs.one_hot_rows(M, K, seed=3)
     B = inputs.bf16_normal((K, N), 0.02, seed=4)
-    Bd = tile_major_on_device(B, K, N, 4, 256)
+    Bd = tile_major_on_device(B, K, N, 4, 256)                 # 4-row tiles are TMA-boxable: part of a tile per CTA tile is fine
     assert torch.equal(run_gemm(A, Bd, M, N, K, 4, 256, (32, 256, 64)).cpu(), B.float()[ks])
+    assert torch.equal(run_gemm(A, Bd, M, N, K, 4, 256, (32, 128, 64)).cpu(), B.float()[ks])
+    Bd = tile_major_on_device(B, K, N, 128, 8)                 # 16-byte rows: hand-addressed, the tile must fit the CTA tile
+    assert torch.equal(run_gemm(A, Bd, M, N, K, 128, 8, (32, 128, 128)).cpu(), B.float()[ks])
     with pytest.raises(tl.TileLensError) as e:
-        run_gemm(A, Bd, M, N, K, 4, 256, (32, 128, 64))        # a 256-wide tile does not fit 128 columns
+        run_gemm(A, Bd, M, N, K, 128, 8, (32, 128, 64))        # 128 rows do not fit 64
     assert e.value.status == 2
 
 
