@@ -687,7 +687,10 @@ def run_sweep(args):
                 continue
             for c in range(copies):
                 tl.relayout(W[c], Wt[c], K, N, 2, g, br, bc, tl.TO_TILE_MAJOR)
-            path = "row-major view" if br == 1 else ("tma" if br >= 8 and bc >= 64 else "generic-address")
+            # the library's rule: 1-row tiles are row-major; tile rows of at least 32 bytes are TMA boxes (128-byte
+            # swizzle from 64 columns, 64-/32-byte swizzle for 32/16 columns); shorter rows are hand-addressed
+            path = ("row-major view" if br == 1 else "tma" if bc >= 64 else
+                    "tma, %d-byte swizzle" % (bc * 2) if bc in (16, 32) else "generic-address")
             for cta in ctas:
                 ra_t = tl.read_amp(128, N, K, cta, tl.LAYOUT_TILE_MAJOR, g, br, bc, 2)
                 ra_r = tl.read_amp(128, N, K, cta, tl.LAYOUT_ROW_MAJOR, g, 0, 0, 2)

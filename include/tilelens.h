@@ -105,11 +105,12 @@ int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, i
  *                Tiles may overhang M, N and K.
  *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,
  *   N % block_cols == 0; row-major: N % 64 == 0.
- *   Memory tiles of at least 8 rows x 64 columns are read by TMA.  Smaller
- *   ones (block rows down to 2 bytes) are read by the generic-address path of
- *   Section 4.4 (plain loads with Eq. 1-2 arithmetic); there the memory tile
- *   must fit inside the CTA tile (block_rows | cta_k, block_cols | cta_n) and
- *   G >= 16, else TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
+ *   Memory tiles whose rows are at least 32 bytes (16 columns) are read by
+ *   TMA, whatever their height.  Narrower ones (block rows down to 2 bytes)
+ *   are read by the generic-address path of Section 4.4 (plain loads with
+ *   Eq. 1-2 arithmetic); there the memory tile must fit inside the CTA tile
+ *   (block_rows | cta_k, block_cols | cta_n) and G >= 16, else
+ *   TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
  * When the output tiles do not fill the SMs (decode, small or grouped
  * problems) the K loops are cut stream-K fashion over all SMs; partial tiles
  * go through a workspace and a second small kernel adds them in a fixed

@@ -64,6 +64,10 @@ struct alignas(64) GemmParams {
     int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
     int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
     int k_inner;                // 1: tensor-map dimensions ordered (64, row in tile, tile along K, atom, tile along N)
+    // Tensor-map coordinates 1..4 of a weight box as shifts and masks of its first K element k and weight column n:
+    // c[i] = ((k >> ck_shift[i]) & ck_mask[i]) + ((n >> cn_shift[i]) & cn_mask[i]) + c_expert[i] * (expert offset).
+    // (Set by the host for the layout at hand: the producer's loop has no layout branches.)
+    int ck_shift[4], ck_mask[4], cn_shift[4], cn_mask[4], c_expert[4];
     int fp8;                    // 1: both operands are 8-bit floating point (E4M3); needs w_kmajor
     int k_shift;                // log2(K elements per 2 bytes): a stage holds (BK << k_shift) K-elements
     int w_atom_log2;            // K-major weights: log2(elements in one swizzle row of 128, 64 or 32 bytes)
@@ -293,29 +297,9 @@ __device__ __forceinline__ __nv_bfloat16 swiglu_bf16(float g, float u) {
 // expert's offset along the stacked dimension).
 __device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, int n, int kc_expert, int (&c)[5]) {
     c[0] = 0;
-    if (p.w_kmajor) {
-        // [N][K] storage: (swizzle row of K-elements, row in tile, tile along N, swizzle row in tile, tile along K)
-        if (p.row_major) { c[1] = n + kc_expert; c[2] = 0; c[3] = k >> p.w_atom_log2; c[4] = 0; }
-        else {
-            c[1] = n & ((1 << p.br_log2) - 1);
-            c[2] = (n >> p.br_log2) + kc_expert;
-            c[3] = (k & ((1 << p.bc_log2) - 1)) >> p.w_atom_log2;
-            c[4] = k >> p.bc_log2;
-        }
-    } else if (p.row_major) { c[1] = k + kc_expert; c[2] = n >> 6; c[3] = 0; c[4] = 0; }
-    else if (p.k_inner) {
-        // (64 N-elements, row in tile, tile along K, atom in tile, tile along N)
-        c[1] = k & ((1 << p.br_log2) - 1);
-        c[2] = (k >> p.br_log2) + kc_expert;
-        c[3] = (n & ((1 << p.bc_log2) - 1)) >> 6;
-        c[4] = n >> p.bc_log2;
-    } else {
-        // (64 N-elements, row in tile, atom in tile, tile along N, tile along K)
-        c[1] = k & ((1 << p.br_log2) - 1);
-        c[2] = (n & ((1 << p.bc_log2) - 1)) >> 6;
-        c[3] = n >> p.bc_log2;
-        c[4] = (k >> p.br_log2) + kc_expert;
-    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        c[i + 1] = ((k >> p.ck_shift[i]) & p.ck_mask[i]) + ((n >> p.cn_shift[i]) & p.cn_mask[i]) + p.c_expert[i] * kc_expert;
 }
 
 // kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256).
@@ -442,6 +426,11 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             uint32_t issued = 0;
             Work w;
             bool ok = true;
+            // the K part of the coordinate maps, in registers for the whole loop
+            const bool one_box = p.kbx == 1 && p.nbx == 1;
+            int ks[4], km[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { ks[i] = p.ck_shift[i]; km[i] = p.ck_mask[i]; }
             while (ok && sched.next(w)) {
                 const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
                 int bi = 0;
@@ -449,6 +438,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 const uint32_t a_bytes = uint32_t(16 << bi) * kAtomBytes;
                 const uint32_t tx = uint32_t(kSubK) * a_bytes + uint32_t(p.kbx * p.nbx) * p.box_bytes;
                 const int kc_expert = t.expert * p.k_coord_per_expert;
+                int cn[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) cn[i] = ((t.n0 >> p.cn_shift[i]) & p.cn_mask[i]) + p.c_expert[i] * kc_expert;
                 for (int kit = w.kbeg; kit < w.kend; ++kit) {
                     const long long cc0 = TL_CLOCK();
                     if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
@@ -465,14 +457,22 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     for (int sub = 0; sub < kSubK; ++sub)
                         tma_load_2d(sa + size_t(sub) * p.BM * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
                                     k0 + ((sub * 64) << p.k_shift), t.row0);
-                    for (int kb = 0; kb < p.kbx; ++kb) {
-                        const int k = k0 + kb * p.box_rows;
-                        for (int nb = 0; nb < p.nbx; ++nb) {
-                            const int n = t.n0 + nb * p.box_atoms * 64;
-                            uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
-                            int c[5];
-                            weight_box_coords(p, k, n, kc_expert, c);
-                            tma_load_5d(dst, &p.tmap_b, &full_bar[stage], c[0], c[1], c[2], c[3], c[4]);
+                    if (one_box) {
+                        // the usual case, one box per stage: the column part of the coordinates was worked out once
+                        // for the tile, only the K part changes from stage to stage
+                        tma_load_5d(sw, &p.tmap_b, &full_bar[stage], 0, ((k0 >> ks[0]) & km[0]) + cn[0],
+                                    ((k0 >> ks[1]) & km[1]) + cn[1], ((k0 >> ks[2]) & km[2]) + cn[2],
+                                    ((k0 >> ks[3]) & km[3]) + cn[3]);
+                    } else {
+                        for (int kb = 0; kb < p.kbx; ++kb) {
+                            const int k = k0 + kb * p.box_rows;
+                            for (int nb = 0; nb < p.nbx; ++nb) {
+                                const int n = t.n0 + nb * p.box_atoms * 64;
+                                uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
+                                int c[5];
+                                weight_box_coords(p, k, n, kc_expert, c);
+                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], c[0], c[1], c[2], c[3], c[4]);
+                            }
                         }
                     }
                     ++issued;
@@ -1176,6 +1176,37 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.bc_log2 = ilog2(bc);
         }
     }
+    {
+        // coordinate maps (see GemmParams): which bits of k and n each tensor-map dimension takes
+        auto set = [&](int i, int ks, int km, int ns, int nm, int ex) {
+            p.ck_shift[i] = ks; p.ck_mask[i] = km; p.cn_shift[i] = ns; p.cn_mask[i] = nm; p.c_expert[i] = ex;
+        };
+        const int all = -1;
+        for (int i = 0; i < 4; ++i) set(i, 0, 0, 0, 0, 0);
+        if (generic) {
+        } else if (kmajor && row_major) {           // (row of K-elements, N row, -, swizzle row along K, -)
+            set(0, 0, 0, 0, all, 1);
+            set(2, p.w_atom_log2, all, 0, 0, 0);
+        } else if (kmajor) {                        // (.., row in tile, tile along N, swizzle row in tile, tile along K)
+            set(0, 0, 0, 0, br - 1, 0);
+            set(1, 0, 0, p.br_log2, all, 1);
+            set(2, p.w_atom_log2, (bc >> p.w_atom_log2) - 1, 0, 0, 0);
+            set(3, p.bc_log2, all, 0, 0, 0);
+        } else if (row_major) {                     // (64 columns, K row, 64-column atom, -, -)
+            set(0, 0, all, 0, 0, 1);
+            set(1, 0, 0, 6, all, 0);
+        } else if (p.k_inner) {                     // (.., row in tile, tile along K, atom in tile, tile along N)
+            set(0, 0, br - 1, 0, 0, 0);
+            set(1, p.br_log2, all, 0, 0, 1);
+            set(2, 0, 0, 6, bc >= 64 ? (bc >> 6) - 1 : 0, 0);
+            set(3, 0, 0, p.bc_log2, all, 0);
+        } else {                                    // (.., row in tile, atom in tile, tile along N, tile along K)
+            set(0, 0, br - 1, 0, 0, 0);
+            set(1, 0, 0, 6, (bc >> 6) - 1, 0);
+            set(2, 0, 0, p.bc_log2, all, 0);
+            set(3, p.br_log2, all, 0, 0, 1);
+        }
+    }
     p.row_major = row_major;
     p.kbx = generic ? 0 : plan.BK / (RB * kb_box);
     p.nbx = generic ? 0 : NA / (AB * nb_box);
@@ -1240,7 +1271,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.stream_k = plan.stream_k;
     p.num_stages = plan.num_stages;
     static const int prefetch_env = getenv("TL_PREFETCH_STAGES") ? atoi(getenv("TL_PREFETCH_STAGES")) : -1;   // measurement hook
-    p.prefetch_stages = !pdl_ok ? 0 : (prefetch_env >= 0 ? prefetch_env : plan.num_stages);
+    // (at most four instructions: the thread that issues them holds up the CTA's first barrier for their duration)
+    p.prefetch_stages = !pdl_ok ? 0 : (prefetch_env >= 0 ? prefetch_env : (plan.num_stages < 4 ? plan.num_stages : 4));
 
     cudaError_t err = cudaSuccess;
     // Large dense problems on TMA-readable weights: CTA pairs (cta_group::2 MMAs), see tl_gemm_pair.cuh.
