@@ -85,7 +85,7 @@ def test_gemm_argument_checks_need_no_device(tl):
     assert call(G=2048) == 1                                 # G != br*bc*2
     assert call(K=520) == 1                                  # K % br
     assert call(br=12, bc=128, G=12 * 128 * 2) == 2          # not a power of two
-    assert call(br=4, bc=512) == 2                           # hand-addressed tiles must fit inside the CTA tile
+    assert call(br=256, bc=8) == 2                           # hand-addressed tiles (rows under 32 bytes) must fit inside the CTA tile
     assert call(B=ctypes.c_void_p(0x10010)) == 3             # tile-major operand must be 128-byte aligned
     assert L.tl_gemm_host_scratch_bytes(16, 512, 512) >= 16 * 512 * 2 + 2 * 512 * 512 * 2 + 16 * 512 * 4
 
