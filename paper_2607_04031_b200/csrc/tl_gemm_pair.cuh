@@ -207,11 +207,17 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             bool ok = true;
             const long long t_begin = TL_CLK();
             (void)t_begin;
+            int ks[4], km[4];                                       // K part of the coordinate maps, in registers
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { ks[i] = p.ck_shift[i]; km[i] = p.ck_mask[i]; }
             for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
                 const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
                 if (pt.halves == 0) continue;
                 const int n0 = pt.n_tile * 256 + int(rank) * 128;   // this CTA's weight columns
                 const int row0 = pt.row0 + int(rank) * 128;         // this CTA's half of the (first) token block
+                int cn[4];                                          // column part of the weight box's coordinates
+#pragma unroll
+                for (int i = 0; i < 4; ++i) cn[i] = (n0 >> p.cn_shift[i]) & p.cn_mask[i];
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const long long c0 = TL_CLK();
                     if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
@@ -232,9 +238,8 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     tma_pair_load_2d(sw + kWBytes, &p.tmap_a[3], full_leader, k, row0);
                     if (kHalves == 2 && pt.halves == 2)
                         tma_pair_load_2d(sw + kWBytes + kTokBytes, &p.tmap_a[3], full_leader, k, row0 + 256);
-                    int wc[5];
-                    weight_box_coords(p, k, n0, 0, wc);
-                    tma_pair_load_5d(sw, &p.tmap_b, full_leader, wc[0], wc[1], wc[2], wc[3], wc[4]);
+                    tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, ((k >> ks[0]) & km[0]) + cn[0], ((k >> ks[1]) & km[1]) + cn[1],
+                                     ((k >> ks[2]) & km[2]) + cn[2], ((k >> ks[3]) & km[3]) + cn[3]);
                     ++issued;
 #ifdef TL_TIMELINE
                     w_wait += c1 - c0; w_issue += TL_CLK() - c1;
