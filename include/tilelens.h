@@ -347,6 +347,18 @@ int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int
                       int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
                       uint64_t* d_totals, void* cuda_stream);
 
+/*
+ * Up to 16 tl_read_amp_async configurations in one kernel launch (the counters of all products of a step).
+ * h_cfgs: HOST array of n configurations; d_totals: DEVICE, n x 3 uint64 in the order of h_cfgs.  Asynchronous.
+ */
+typedef struct tl_read_amp_cfg {
+    int64_t M, N, K;
+    int32_t cta_m, cta_n, cta_k, layout;
+    int64_t G;
+    int32_t block_rows, block_cols, elem_bytes, reserved;
+} tl_read_amp_cfg;
+int tl_read_amp_batch(const tl_read_amp_cfg* h_cfgs, int n, uint64_t* d_totals, void* cuda_stream);
+
 /* Grouped form: sum over experts with rows; h_offsets is a HOST array of E+1 int32. */
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K,
                         int cta_m, int cta_n, int cta_k,

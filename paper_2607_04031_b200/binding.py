@@ -40,6 +40,7 @@ _SIGNATURES = {
     "tl_gemm_grouped_fp8_kmajor": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int,
                                           _int, _vp]),
     "tl_read_amp_async": (_int, [_i64, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int, _vp, _vp]),
+    "tl_read_amp_batch": (_int, [_vp, _int, _vp, _vp]),
     "tl_read_amp_shared": (_int, [_i64, _i64, _i64, _int, _int, _int, _i64, _int, _i64, _int, _int, _int, _vp, _vp, _vp]),
     "tl_prefetch_degree": (_i64, [ctypes.c_double, ctypes.c_double, _i64, _i64, _i64, _i64, _i64, _i64, ctypes.c_double]),
     "tl_hw_box_offsets": (_int, [_vp, _vp, _i64, _vp, _vp]),
@@ -269,6 +270,30 @@ def read_amp_async(M: int, N: int, K: int, cta, layout: int, G: int, block_rows:
     """totals: CUDA tensor of 3 int64/uint64 that receives (bytes_fetched, bytes_used, requests); no wait."""
     _check(lib().tl_read_amp_async(M, N, K, cta[0], cta[1], cta[2], layout, G, block_rows, block_cols, elem_bytes,
                                    _dev_ptr(totals), _stream_ptr(stream)), "tl_read_amp_async")
+
+
+class ReadAmpCfg(ctypes.Structure):
+    """tl_read_amp_cfg"""
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64), ("cta_m", ctypes.c_int32),
+                ("cta_n", ctypes.c_int32), ("cta_k", ctypes.c_int32), ("layout", ctypes.c_int32), ("G", ctypes.c_int64),
+                ("block_rows", ctypes.c_int32), ("block_cols", ctypes.c_int32), ("elem_bytes", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+def read_amp_cfgs(cfgs):
+    """cfgs: iterable of (M, N, K, cta, layout, G, block_rows, block_cols, elem_bytes) -> ctypes array for read_amp_batch."""
+    cfgs = list(cfgs)
+    arr = (ReadAmpCfg * len(cfgs))()
+    for a, (M, N, K, cta, layout, G, br, bc, s) in zip(arr, cfgs):
+        a.M, a.N, a.K, a.cta_m, a.cta_n, a.cta_k, a.layout, a.G = M, N, K, cta[0], cta[1], cta[2], layout, G
+        a.block_rows, a.block_cols, a.elem_bytes = br, bc, s
+    return arr
+
+
+def read_amp_batch(cfg_array, totals: torch.Tensor, stream=None):
+    """One launch for up to 16 configurations; totals: CUDA int64/uint64 tensor [n, 3]; no wait."""
+    _check(lib().tl_read_amp_batch(ctypes.addressof(cfg_array), len(cfg_array), _dev_ptr(totals), _stream_ptr(stream)),
+           "tl_read_amp_batch")
 
 
 def read_amp_shared(M: int, N: int, K: int, cta, wave_ctas: int, layout: int, G: int, block_rows: int = 0,

@@ -32,8 +32,8 @@ int ensure_control() {
     State& s = state();
     if (s.ctl.d_status) return TL_OK;
     void* p = nullptr;
-    if (int rc = check_cuda(cudaMalloc(&p, 256))) return rc;
-    if (int rc = check_cuda(cudaMemset(p, 0, 256))) return rc;
+    if (int rc = check_cuda(cudaMalloc(&p, 1024))) return rc;
+    if (int rc = check_cuda(cudaMemset(p, 0, 1024))) return rc;
     void* h = nullptr;
     if (int rc = check_cuda(cudaHostAlloc(&h, 64, cudaHostAllocMapped))) return rc;
     void* h_dev = nullptr;

@@ -18,10 +18,11 @@ namespace tl {
 
 // Device control block (lazily allocated, one per process):
 //   word 0      : timeout flag / detail code written by kernels whose bounded wait expired
-//   bytes 64..  : three uint64 accumulators and a ticket counter of the read-amplification kernel
+//   bytes 64..  : 17 sets of three uint64 accumulators and a ticket counter of the read-amplification kernel
 struct Control {
     uint32_t* d_status = nullptr;        // device
-    unsigned long long* d_acc = nullptr; // device, 4 entries (fetched, used, requests, ticket), zero between launches
+    unsigned long long* d_acc = nullptr; // device, 17 x 4 entries (fetched, used, requests, ticket): the single-shape
+                                         // calls use the first four, batch entry i the four after 4 (i + 1); zero between launches
     unsigned long long* h_acc = nullptr; // mapped pinned host memory the kernel publishes its totals to
     unsigned long long* h_acc_dev = nullptr;   // device-side address of h_acc
 };

@@ -13,6 +13,7 @@
 #include "tl_common.cuh"
 
 #include <cstdlib>
+#include <cstring>
 
 namespace tl {
 
@@ -42,11 +43,11 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
 
 constexpr int kItersPerWarp = 8;     // row-/column-major: K iterations one warp covers (tile-major: all of them)
 
-__global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
+// One CTA's share of one counter configuration; cta is the CTA's index within that configuration.
+__device__ __forceinline__ void read_amp_body(const ReadAmpParams& p, unsigned cta) {
     const int lane = threadIdx.x & 31;
-    const int64_t warp = (blockIdx.x * int64_t(blockDim.x) + threadIdx.x) >> 5;
+    const int64_t warp = (cta * int64_t(blockDim.x) + threadIdx.x) >> 5;
     __shared__ unsigned long long cta_blocks[4], cta_used[4];
-    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t k_chunks = (p.k_iters + p.iters_per_warp - 1) / p.iters_per_warp;
     const bool has_work = warp < p.n_tiles * k_chunks;
     const int64_t tn = has_work ? warp / k_chunks : 0, kc = has_work ? warp % k_chunks : 0;
@@ -134,6 +135,27 @@ __global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
     }
 }
 
+__global__ void __launch_bounds__(128) read_amp_kernel(const ReadAmpParams p) {
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    read_amp_body(p, blockIdx.x);
+}
+
+// Up to kBatchMax configurations in one launch: CTAs [cta_begin[i], cta_begin[i+1]) work on configuration i, each
+// configuration with its own accumulators and output slot.
+constexpr int kBatchMax = 16;
+struct ReadAmpBatch {
+    int n;
+    unsigned cta_begin[kBatchMax + 1];
+    ReadAmpParams p[kBatchMax];
+};
+
+__global__ void __launch_bounds__(128) read_amp_batch_kernel(const __grid_constant__ ReadAmpBatch b) {
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    int i = 0;
+    while (i + 1 < b.n && blockIdx.x >= b.cta_begin[i + 1]) ++i;
+    read_amp_body(b.p[i], blockIdx.x - b.cta_begin[i]);
+}
+
 static int read_amp_validate(int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int layout, int64_t G, int br,
                              int bc, int s) {
     if (N <= 0 || K <= 0 || cta_m <= 0 || cta_n <= 0 || cta_k <= 0 || G <= 0) return TL_ERR_INVALID_ARG;
@@ -151,11 +173,12 @@ static int read_amp_validate(int64_t N, int64_t K, int cta_m, int cta_n, int cta
     return TL_OK;
 }
 
-static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
-                           int br, int bc, int s, unsigned long long* d_acc, unsigned long long* d_fetched,
-                           unsigned long long* d_used, cudaStream_t stream, int64_t wave_tiles = 0,
-                           unsigned long long* totals_out = nullptr) {
-    ReadAmpParams p;
+// Fills the kernel parameters of one configuration; *grid = CTAs it needs (0: nothing to count).
+static int read_amp_fill(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
+                         int br, int bc, int s, unsigned long long* d_acc, unsigned long long* d_fetched,
+                         unsigned long long* d_used, int64_t wave_tiles, unsigned long long* totals_out,
+                         ReadAmpParams* out, int64_t* grid_out) {
+    ReadAmpParams& p = *out;
     p.N = N; p.K = K; p.BN = cta_n; p.BK = cta_k; p.G = G; p.s = s;
     p.br = br > 0 ? br : 1; p.bc = bc > 0 ? bc : 1; p.layout = layout;
     if (layout == TL_LAYOUT_TILE_MAJOR_K) {
@@ -179,10 +202,26 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
     p.d_acc = d_acc; p.d_fetched = d_fetched; p.d_used = d_used;
     p.h_out = d_acc ? (totals_out ? totals_out : state().ctl.h_acc_dev) : nullptr;
     p.iters_per_warp = p.layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
+    *grid_out = 0;
     if (m_tiles == 0) return TL_OK;
     const int warps_per_cta = 4;
     const int64_t grid = ceil_div(p.n_tiles * ceil_div(p.k_iters, p.iters_per_warp), warps_per_cta);
     p.total_ctas = (unsigned long long)grid;
+    *grid_out = grid;
+    return TL_OK;
+}
+
+static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int cta_k, int layout, int64_t G,
+                           int br, int bc, int s, unsigned long long* d_acc, unsigned long long* d_fetched,
+                           unsigned long long* d_used, cudaStream_t stream, int64_t wave_tiles = 0,
+                           unsigned long long* totals_out = nullptr) {
+    ReadAmpParams p;
+    int64_t grid = 0;
+    if (int rc = read_amp_fill(m_tiles, N, K, cta_n, cta_k, layout, G, br, bc, s, d_acc, d_fetched, d_used, wave_tiles,
+                               totals_out, &p, &grid))
+        return rc;
+    if (grid == 0) return TL_OK;
+    const int warps_per_cta = 4;
     if (d_fetched && d_used) {
         const size_t bytes = size_t(m_tiles) * p.n_tiles * sizeof(unsigned long long);
         if (int rc = check_cuda(cudaMemsetAsync(d_fetched, 0, bytes, stream))) return rc;
@@ -274,6 +313,49 @@ int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int
     return tl::read_amp_launch(tl::ceil_div(M, cta_m), N, K, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes,
                                tl::state().ctl.d_acc, nullptr, nullptr, st, 0,
                                reinterpret_cast<unsigned long long*>(d_totals));
+}
+
+int tl_read_amp_batch(const tl_read_amp_cfg* h_cfgs, int n, uint64_t* d_totals, void* cuda_stream) {
+    if (n < 0 || n > tl::kBatchMax || (n > 0 && (!h_cfgs || !d_totals))) return TL_ERR_INVALID_ARG;
+    if (n == 0) return TL_OK;
+    if (int rc = tl::ensure_control()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    tl::ReadAmpBatch b;
+    memset(&b, 0, sizeof b);
+    unsigned ctas = 0;
+    for (int i = 0; i < n; ++i) {
+        const tl_read_amp_cfg& c = h_cfgs[i];
+        if (c.M < 0) return TL_ERR_INVALID_ARG;
+        if (int rc = tl::read_amp_validate(c.N, c.K, c.cta_m, c.cta_n, c.cta_k, c.layout, c.G, c.block_rows, c.block_cols,
+                                           c.elem_bytes))
+            return rc;
+        int64_t grid = 0;
+        // configuration i accumulates in its own four words of the control block and publishes to its own slot
+        if (int rc = tl::read_amp_fill(tl::ceil_div(c.M, c.cta_m), c.N, c.K, c.cta_n, c.cta_k, c.layout, c.G, c.block_rows,
+                                       c.block_cols, c.elem_bytes, tl::state().ctl.d_acc + 4 * (i + 1), nullptr, nullptr, 0,
+                                       reinterpret_cast<unsigned long long*>(d_totals) + 3 * i, &b.p[b.n], &grid))
+            return rc;
+        if (grid == 0) {                                    // M == 0: nothing is launched for it, its totals are zero
+            if (int rc = tl::check_cuda(cudaMemsetAsync(d_totals + 3 * i, 0, 3 * sizeof(uint64_t), st))) return rc;
+            continue;
+        }
+        if (grid > (1u << 30) || ctas + grid > (1u << 30)) return TL_ERR_UNSUPPORTED;
+        b.cta_begin[b.n] = ctas;
+        ctas += unsigned(grid);
+        ++b.n;
+        b.cta_begin[b.n] = ctas;
+    }
+    if (b.n == 0) return TL_OK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(128);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return tl::check_cuda(cudaLaunchKernelEx(&cfg, tl::read_amp_batch_kernel, b));
 }
 
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,

@@ -177,3 +177,22 @@ def test_async_totals_match_the_waiting_call_when_queued_back_to_back():
     got = out.cpu().numpy()
     for i, (M, N, K, cta, layout, br, bc) in enumerate(cases):
         assert tuple(int(x) for x in got[i]) == tl.read_amp(M, N, K, cta, layout, 4096, br, bc, 2)
+
+
+def test_batched_counters_match_the_single_calls():
+    import torch
+    from gpu_util import DEV, tl
+    cases = [(8, 10240, 8192, (16, 128, 64), tl.LAYOUT_TILE_MAJOR, 4096, 16, 128, 2),
+             (32, 8192, 8192, (32, 128, 64), tl.LAYOUT_ROW_MAJOR, 4096, 0, 0, 2),
+             (300, 1000, 520, (128, 256, 128), tl.LAYOUT_COL_MAJOR, 4096, 0, 0, 1),
+             (0, 512, 512, (16, 128, 64), tl.LAYOUT_ROW_MAJOR, 4096, 0, 0, 2),
+             (1, 57344, 8192, (16, 256, 64), tl.LAYOUT_TILE_MAJOR_K, 4096, 32, 64, 2),
+             (70, 96, 64, (32, 24, 16), tl.LAYOUT_ROW_MAJOR, 128, 0, 0, 2)] * 2 + [(4096, 8192, 28672, (256, 128, 64), tl.LAYOUT_ROW_MAJOR, 4096, 0, 0, 2)]
+    out = torch.full((len(cases), 3), -1, dtype=torch.int64, device=DEV)
+    for rep in range(3):                                   # back to back: the accumulators must come back to zero
+        tl.read_amp_batch(tl.read_amp_cfgs(cases), out)
+    got = out.cpu().numpy()
+    for i, (M, N, K, cta, layout, G, br, bc, s) in enumerate(cases):
+        assert tuple(int(x) for x in got[i]) == tl.read_amp(M, N, K, cta, layout, G, br, bc, s), i
+    with pytest.raises(tl.TileLensError):
+        tl.read_amp_batch(tl.read_amp_cfgs(cases + cases), torch.zeros((26, 3), dtype=torch.int64, device=DEV))    # more than 16
