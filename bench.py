@@ -63,17 +63,37 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    """SM clock, power and throttle reasons read through NVML every few milliseconds by a thread (read-only
+    queries); falls back to `nvidia-smi -lms 200` when NVML cannot be loaded.  mark_timed() brackets the timed
+    region so that the samples taken inside it can be told from those taken during the other legs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+    REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
     def __init__(self, index: int):
-        self.rows = []
+        self.rows = []          # (time, sm MHz, max MHz, watts, set of reasons)
         self.proc = None
         self.index = index
+        self.nvml = None
+        self.stop_flag = False
+        self.t_begin = self.t_end = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = torch.cuda.get_device_properties(self.index).uuid
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.nvml = pynvml
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
@@ -83,31 +103,62 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+    def mark_timed(self, begin: bool):
+        if begin:
+            self.t_begin = time.perf_counter()
+        else:
+            self.t_end = time.perf_counter()
 
-    def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.25)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, pw, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+    def _poll(self):
+        n = self.nvml
+        mx = n.nvmlDeviceGetMaxClockInfo(self.handle, n.NVML_CLOCK_SM)
+        while not self.stop_flag:
             try:
-                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+                sm = n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)
+                watts = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                mask = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                why = {k for k, bit in self.REASONS.items() if mask & bit}
+                self.rows.append((time.perf_counter(), float(sm), float(mx), watts, why))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def _read(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.proc.stdout:
+            r = [x.strip() for x in line.split(",")]
+            try:
+                why = {nm for nm, v in zip(names, r[3:7]) if v.lower().startswith("active")}
+                self.rows.append((time.perf_counter(), float(r[0]), float(r[1]), float(r[2]), why))
             except (ValueError, IndexError):
                 continue
-            for name, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+    def stop(self):
+        if self.nvml is None and not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML and no nvidia-smi"]}
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+        else:
+            time.sleep(0.25)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        rows = list(self.rows)
+        inside = [r for r in rows if self.t_begin is not None and self.t_end is not None and self.t_begin <= r[0] <= self.t_end]
+        use = inside if inside else rows
+        reasons = set()
+        for r in rows:
+            reasons |= r[4]
+        return {"sm_mhz": statistics.median(r[1] for r in use) if use else None,
+                "sm_max_mhz": max(r[2] for r in rows) if rows else None,
+                "power_w_max": max(r[3] for r in rows) if rows else None,
+                "samples": len(rows), "samples_in_timed_region": len(inside),
+                "sm_mhz_min_in_timed_region": min(r[1] for r in inside) if inside else None,
+                "reasons_in_timed_region": sorted(set().union(*[r[4] for r in inside])) if inside else [],
+                "reasons": sorted(reasons), "source": "nvml" if self.nvml is not None else "nvidia-smi"}
 
 
 # ------------------------------------------------------------------ CPU oracle leg
@@ -150,7 +201,7 @@ def run_reference(args):
         return
     import oracle as tlo
     tlo.build()
-    per_step = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    per_step = max(0.6, min(20.0, 150.0 / max(1, args.steps + args.warmup)))      # the whole run: about 2.5 minutes
     for _ in range(args.warmup):
         oracle_sample(per_step)
     vals = [oracle_sample(per_step) for _ in range(args.steps)]
@@ -282,11 +333,13 @@ def run_ours(args):
     torch.cuda.synchronize()
     timer = EventTimer()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark_timed(True)
     ev0.record()
     for _ in range(args.steps):
         one_step(timer)
     ev1.record()
     torch.cuda.synchronize()
+    sampler.mark_timed(False)
     if world > 1:
         dist.barrier()
     total_ms = ev0.elapsed_time(ev1)
@@ -715,8 +768,8 @@ def main():
                     help="run one small kernel case --steps times (for ncu); no benchmark line")
     ap.add_argument("--layout", default="tile", choices=["tile", "row"])
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=200)      # ~0.3 s timed: long enough for clock samples inside it
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.sweep:
