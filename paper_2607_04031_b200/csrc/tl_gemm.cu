@@ -1,25 +1,30 @@
-// Tiled bf16 GEMM reading a tile-major (or row-major) weight operand, for sm_100a.
+// Tiled GEMM reading a tile-major (or row-major) weight operand, for sm_100a.
 //
-//   C[M x N] (fp32) = A[M x K] (bf16, K contiguous) x B[K x N] (bf16)          (Section 2.3)
+//   C[M x N] (fp32) = A[M x K] (bf16 or FP8, K contiguous) x B[K x N]                      (Section 2.3)
 //
-// B is read through a 5-D tensor-map view of the tile-major buffer (the 4-D view of Eq. 3 in the
-// N-contiguous flavour, with the contiguous extent of a memory tile split into 128-byte atoms):
-// one TMA box per memory tile, or per part of a memory tile that lies inside the CTA tile.
-// The boxes land in shared memory in exactly the canonical "MN-major, 128-byte swizzle" form
-// that tcgen05.mma reads, so the weights are the M-side operand of the MMA (128 weight columns
-// per instruction) and the token rows are its N-side operand (16..256 tokens, K-major).  The
-// accumulator therefore holds C transposed: TMEM lane = weight column, TMEM column = token.
+// B is read through a 5-D tensor-map view of the tile-major buffer (the 4-D view of Eq. 3 with the contiguous
+// extent of a memory tile split into swizzle rows of 128, 64 or 32 bytes).  One TMA instruction fills a pipeline
+// stage: its box is a whole number of memory tiles, or the part of a tile that lies inside the CTA tile, and it
+// lands in shared memory in exactly the canonical swizzled operand form that tcgen05.mma reads -- MN-major for
+// weights stored with N contiguous, K-major for weights stored [N][K] (Eq. 2 as printed).  The weights can sit on
+// either side of the instruction:
+//   weights on N (tiles of up to 128 token rows: decode, MoE)  tokens are the M-side operand, one MMA covers all
+//                cta_n weight columns; TMEM lane = token row;
+//   weights on M (256-token tiles)  TMEM lane = weight column, the accumulator holds C transposed.
+// Memory tiles whose rows are shorter than 32 bytes cannot be boxed: four more warps load them with Eq. 1-2
+// address arithmetic and build the operand image by hand (Section 4.4).
 //
-// One persistent CTA per SM, six warps:
+// One persistent CTA per SM:
 //   warp 0      TMA producer   (one lane)   ring of shared-memory stages, mbarrier expect-tx
 //   warp 1      MMA issuer     (one lane)   tcgen05.mma into one of two TMEM accumulators
-//   warps 2..5  epilogue                    tcgen05.ld -> fp32 -> C (128-byte coalesced rows)
-// Work is a list of (output tile, K range).  Data-parallel mode hands whole tiles round-robin;
-// stream-K mode cuts the flattened (tile, K iteration) space into one contiguous range per CTA
-// (decode: all SMs stream weights even when there are fewer tiles than SMs).  Partial tiles go to
-// a workspace; the CTA that arrives last at a tile's counter adds the partials in K order, so the
-// result does not depend on arrival order.  Nothing ever spins on another CTA.
-// Every mbarrier wait is bounded (see mbar_wait_bounded).
+//   warps 2..5  epilogue                    tcgen05.ld -> fp32 -> C, or silu(gate) * up -> bf16 (expert FFN)
+//   warps 6..9  hand-addressed weight loads (only when the memory tile cannot be boxed)
+// Work is a list of (output tile, K range).  Data-parallel mode hands whole tiles round-robin; stream-K mode cuts
+// the flattened (tile, K iteration) space into one contiguous range per CTA (decode: all SMs stream weights even
+// when there are fewer tiles than SMs).  Partial tiles go to a workspace and a second small kernel
+// (streamk_reduce_kernel, launched with programmatic stream serialisation so that it is resident before this one
+// ends) adds them in K order and writes C.  Nothing ever spins on another CTA; every mbarrier wait is bounded
+// (see mbar_wait_bounded).  Large dense problems run on CTA pairs instead (tl_gemm_pair.cuh).
 #include "tl_common.cuh"
 
 #include <cuda_bf16.h>

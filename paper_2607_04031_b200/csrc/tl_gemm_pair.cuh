@@ -15,6 +15,11 @@
 //     "stage free" and "accumulator ready" barriers of both CTAs fire together; "accumulator drained"
 //     arrivals of both CTAs' epilogue warps go to the leader;
 //   - each CTA's epilogue stores its own 128 columns of C, exactly as in the single-CTA kernel.
+// With 256 x 256 tiles the kernel is held back by operand traffic out of L2 (32 KB per CTA per 64-row K step).  A
+// tile may therefore cover two 256-token blocks (kHalves = 2): one weight slab per stage serves both (48 KB per CTA
+// for twice the work, four stages), two MMAs per K step into the two halves of tensor memory, and eight epilogue
+// warps because the epilogue is no longer hidden behind the next tile's MMAs.  Whole waves of clusters take such
+// tiles; what is left of the tile grid runs as 256-token tiles.
 // No TMA multicast is used.  Every wait is on a barrier in the waiter's own shared memory and is bounded.
 #pragma once
 
