@@ -1,11 +1,15 @@
-// Row-major <-> tile-major relayout (Section 3; Eq. 1 and Eq. 2 in the N-contiguous flavour).
+// Row-major <-> tile-major relayout (Section 3; Eq. 1 and Eq. 2 in the N-contiguous flavour; applied to the [N][K]
+// array it produces the K-contiguous flavour of Eq. 2 as printed).
 //
-// Bandwidth-bound: every byte is read once and written once.  The fast kernel
-// moves 32 KB tiles through shared memory with 16-byte loads and stores on
-// both sides: the row-major side is walked in row order, the tile-major side
-// in block order, and shared memory absorbs the permutation.  When a block
-// row is shorter than 16 bytes the 16-byte vectors of the tile-major side are
-// assembled from several shared-memory rows.
+// Bandwidth-bound: every byte is read once and written once.  Three kernels:
+//   relayout_tma_kernel   the copy engine does the permutation: a tensor-map box of the row-major side holds whole
+//                         memory tiles, which are contiguous runs of the tile-major side and move as untiled bulk
+//                         copies; one thread per CTA drives a ring of three 32 KB buffers (block rows 16 B .. 1 KB);
+//   relayout_kernel<P>    32 KB tiles through shared memory with 16-byte loads and stores on both sides: the
+//                         row-major side is walked in row order, the tile-major side in block order; when a block
+//                         row is shorter than 16 bytes the vectors of the tile-major side are assembled from
+//                         several shared-memory rows;
+//   element-wise          for unaligned pointers or pitches.
 #include "tl_common.cuh"
 
 #include <cstdlib>
