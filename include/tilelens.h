@@ -151,6 +151,15 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
  * Y (fp32, total_rows x hidden) = H x W_down.  Two kernels (plus their stream-K reductions) in stream order, no
  * host synchronisation; d_H_bf16 is caller-owned scratch that holds H afterwards.
  */
+/* tl_gemm / tl_gemm_grouped with C written as bf16 (fp32 accumulation, one rounding to nearest even): d_C_bf16
+ * M x N (total_rows x N) bf16, 16-byte aligned, N % 8 == 0.  The paper leaves the output type open. */
+int tl_gemm_bf16(const void* d_A_rowmajor, const void* d_B_tilemajor, void* d_C_bf16,
+                 int64_t M, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                 int cta_m, int cta_n, int cta_k, void* cuda_stream);
+int tl_gemm_grouped_bf16(const void* d_A_sorted, const void* d_B_experts, void* d_C_bf16,
+                         const int32_t* d_offsets, int E, int64_t total_rows,
+                         int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                         int cta_m, int cta_n, int cta_k, void* cuda_stream);
 int tl_gemm_grouped_swiglu(const void* d_A_sorted, const void* d_B_experts_gate_up, void* d_H_bf16,
                            const int32_t* d_offsets, int E, int64_t total_rows,
                            int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,

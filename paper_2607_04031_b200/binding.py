@@ -30,6 +30,8 @@ _SIGNATURES = {
     "tl_relayout_on": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int, _vp]),
     "tl_gemm": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_bf16": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_grouped_bf16": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped_swiglu": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int,
                                       _vp]),
     "tl_moe_ffn": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _vp]),
@@ -142,6 +144,21 @@ def gemm_grouped(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, offsets: tor
     _check(lib().tl_gemm_grouped(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C), _dev_ptr(offsets), E, total_rows, N, K, G,
                                  block_rows, block_cols, cta[0], cta[1], cta[2], _stream_ptr(stream)),
            "tl_gemm_grouped")
+
+
+def gemm_bf16(A: torch.Tensor, B: torch.Tensor, C_bf16: torch.Tensor, M: int, N: int, K: int, G: int = 4096,
+              block_rows: int = 16, block_cols: int = 128, cta=(0, 0, 0), stream=None):
+    """tl_gemm with a bf16 C."""
+    _check(lib().tl_gemm_bf16(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C_bf16), M, N, K, G, block_rows, block_cols,
+                              cta[0], cta[1], cta[2], _stream_ptr(stream)), "tl_gemm_bf16")
+
+
+def gemm_grouped_bf16(A: torch.Tensor, B: torch.Tensor, C_bf16: torch.Tensor, offsets: torch.Tensor, E: int,
+                      total_rows: int, N: int, K: int, G: int = 4096, block_rows: int = 16, block_cols: int = 128,
+                      cta=(0, 0, 0), stream=None):
+    _check(lib().tl_gemm_grouped_bf16(_dev_ptr(A), _dev_ptr(B), _dev_ptr(C_bf16), _dev_ptr(offsets), E, total_rows, N, K,
+                                      G, block_rows, block_cols, cta[0], cta[1], cta[2], _stream_ptr(stream)),
+           "tl_gemm_grouped_bf16")
 
 
 def gemm_grouped_swiglu(A: torch.Tensor, B_gate_up: torch.Tensor, H: torch.Tensor, offsets: torch.Tensor, E: int,

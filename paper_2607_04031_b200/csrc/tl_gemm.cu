@@ -65,6 +65,7 @@ struct alignas(64) GemmParams {
     int epi_swiglu;
     __nv_bfloat16* H;
     int64_t ldh;
+    __nv_bfloat16* Cb;          // non-null: C is written as bf16 (one rounding to nearest even) instead of fp32
     // weight-operand geometry
     int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
     int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
@@ -658,6 +659,21 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                                 q[0] = make_uint4(h2[0], h2[1], h2[2], h2[3]);
                                 q[1] = make_uint4(h2[4], h2[5], h2[6], h2[7]);
                             }
+                        } else if (full && p.Cb) {
+                            // 32 columns -> 32 bf16 = four 16-byte stores
+                            if (row < t.rows) {
+                                __nv_bfloat16* cdst = p.Cb + int64_t(t.row0 + row) * p.ldc + t.n0 + c0;
+#pragma unroll
+                                for (int i = 0; i < 32; i += 8)
+                                    if (t.n0 + c0 + i < p.N) {
+                                        uint32_t h[4];
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j)
+                                            h[j] = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[i + 2 * j])))) |
+                                                   (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[i + 2 * j + 1])))) << 16);
+                                        *reinterpret_cast<uint4*>(cdst + i) = make_uint4(h[0], h[1], h[2], h[3]);
+                                    }
+                            }
                         } else if (row < t.rows) {
 #pragma unroll
                             for (int i = 0; i < 32; i += 4)
@@ -679,21 +695,35 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     const bool n_ok = lane_ok && (full ? (t.n0 + n_local < p.N) : true);
                     const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) +
                                            acc * uint32_t(kNumN * acc_cols) + uint32_t(u * acc_cols);
+                    const bool to_bf16 = full && p.Cb != nullptr;
+                    __nv_bfloat16* outb = p.Cb + int64_t(t.row0) * p.ldc + t.n0 + n_local;
                     for (int c0 = 0; c0 < n_mma; c0 += 32) {
                         if (n_mma - c0 >= 32) {
                             uint32_t v[32];
                             tmem_ld_32x32b_x32(taddr + c0, v);
                             tmem_ld_wait();
+                            if (to_bf16) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                                for (int i = 0; i < 32; ++i)
+                                    if (n_ok && c0 + i < t.rows) outb[int64_t(c0 + i) * p.ldc] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                            }
                         } else {
                             uint32_t v[16];
                             tmem_ld_32x32b_x16(taddr + c0, v);
                             tmem_ld_wait();
+                            if (to_bf16) {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                                for (int i = 0; i < 16; ++i)
+                                    if (n_ok && c0 + i < t.rows) outb[int64_t(c0 + i) * p.ldc] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                            }
                         }
                     }
                 }
@@ -805,6 +835,12 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
                         const __nv_bfloat16 lo = swiglu_bf16(sum[q].x, sum[q].y), hi = swiglu_bf16(sum[q].z, sum[q].w);
                         *reinterpret_cast<uint32_t*>(p.H + int64_t(t.row0 + r) * p.ldh + ((t.n0 + c4) >> 1)) =
                             uint32_t(__bfloat16_as_ushort(lo)) | (uint32_t(__bfloat16_as_ushort(hi)) << 16);
+                    } else if (p.Cb) {
+                        const uint32_t lo = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].x))) |
+                                            (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].y))) << 16);
+                        const uint32_t hi = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].z))) |
+                                            (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].w))) << 16);
+                        *reinterpret_cast<uint2*>(p.Cb + int64_t(t.row0 + r) * p.ldc + t.n0 + c4) = make_uint2(lo, hi);
                     } else {
                         *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
                     }
@@ -991,13 +1027,14 @@ struct FixedScratch {
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
                        int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
-                       bool kmajor = false, int elem_bytes = 2, void* d_H_swiglu = nullptr) {
+                       bool kmajor = false, int elem_bytes = 2, void* d_H_swiglu = nullptr, void* d_C_bf16 = nullptr) {
     const int es = elem_bytes;                       // 2: bf16, 1: FP8 (E4M3), K-contiguous weights only
     const int k_shift = es == 1 ? 1 : 0;
     if (es != 2 && !(es == 1 && kmajor)) return TL_ERR_UNSUPPORTED;
     if (rows_total < 0 || N <= 0 || K <= 0 || E < 1) return TL_ERR_INVALID_ARG;
     if (rows_total == 0) return TL_OK;
-    if (!d_A || !d_B || (!d_C && !d_H_swiglu)) return TL_ERR_INVALID_ARG;
+    if (!d_A || !d_B || (!d_C && !d_H_swiglu && !d_C_bf16)) return TL_ERR_INVALID_ARG;
+    if (d_C_bf16 && (N % 8 != 0 || reinterpret_cast<uintptr_t>(d_C_bf16) % 16 != 0)) return TL_ERR_INVALID_ARG;
     if (d_H_swiglu && (N % 64 != 0 || reinterpret_cast<uintptr_t>(d_H_swiglu) % 16 != 0)) return TL_ERR_INVALID_ARG;
     if (rows_total >= (int64_t(1) << 31) || N >= (int64_t(1) << 31) || K * int64_t(E) >= (int64_t(1) << 31))
         return TL_ERR_UNSUPPORTED;
@@ -1258,6 +1295,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     p.w_desc_hi = smem_desc_hi(p.lbo, p.sbo, w_layout);
     p.C = d_C;
+    p.Cb = static_cast<__nv_bfloat16*>(d_C_bf16);
     p.epi_swiglu = d_H_swiglu != nullptr;
     p.H = static_cast<__nv_bfloat16*>(d_H_swiglu);
     p.ldh = N / 2;
@@ -1433,6 +1471,23 @@ int tl_gemm_grouped_fp8_kmajor(const void* d_A_sorted, const void* d_B_experts_n
     if (cta_k != 0 && cta_k != 128 && cta_k != 256) return TL_ERR_UNSUPPORTED;
     return tl::gemm_launch(d_A_sorted, d_B_experts_nk, d_C, d_offsets, E, total_rows, total_rows, N, K, G, tile_n, tile_k,
                            cta_m, cta_n, cta_k / 2, static_cast<cudaStream_t>(cuda_stream), nullptr, true, 1);
+}
+
+int tl_gemm_bf16(const void* d_A, const void* d_B, void* d_C_bf16, int64_t M, int64_t N, int64_t K, int64_t G,
+                 int block_rows, int block_cols, int cta_m, int cta_n, int cta_k, void* cuda_stream) {
+    if (!d_C_bf16) return TL_ERR_INVALID_ARG;
+    return tl::gemm_launch(d_A, d_B, nullptr, nullptr, 1, M, M, N, K, G, block_rows, block_cols, cta_m, cta_n, cta_k,
+                           static_cast<cudaStream_t>(cuda_stream), nullptr, false, 2, nullptr, d_C_bf16);
+}
+
+int tl_gemm_grouped_bf16(const void* d_A_sorted, const void* d_B_experts, void* d_C_bf16, const int32_t* d_offsets, int E,
+                         int64_t total_rows, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols, int cta_m,
+                         int cta_n, int cta_k, void* cuda_stream) {
+    if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
+    if (!d_C_bf16) return TL_ERR_INVALID_ARG;
+    return tl::gemm_launch(d_A_sorted, d_B_experts, nullptr, d_offsets, E, total_rows, total_rows, N, K, G, block_rows,
+                           block_cols, cta_m, cta_n, cta_k, static_cast<cudaStream_t>(cuda_stream), nullptr, false, 2,
+                           nullptr, d_C_bf16);
 }
 
 int tl_gemm_grouped_swiglu(const void* d_A_sorted, const void* d_B_experts_gate_up, void* d_H_bf16, const int32_t* d_offsets,

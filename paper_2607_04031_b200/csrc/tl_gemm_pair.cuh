@@ -336,14 +336,27 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     const int rows = p.M - row0 < 256 ? p.M - row0 : 256;
                     float* out = p.C + int64_t(row0) * p.ldc + n0;
                     const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256u + uint32_t(h) * 256u;
-                    for (int c0 = 0; c0 < 256; c0 += 32) {
-                        if (c0 >= rows) break;
-                        uint32_t v[32];
-                        tmem_ld_32x32b_x32(taddr + c0, v);
-                        tmem_ld_wait();
+                    if (p.Cb == nullptr) {
+                        for (int c0 = 0; c0 < 256; c0 += 32) {
+                            if (c0 >= rows) break;
+                            uint32_t v[32];
+                            tmem_ld_32x32b_x32(taddr + c0, v);
+                            tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (n_ok && c0 + i < rows) __stcs(out + int64_t(c0 + i) * p.ldc + n_local, __uint_as_float(v[i]));
+                            for (int i = 0; i < 32; ++i)
+                                if (n_ok && c0 + i < rows) __stcs(out + int64_t(c0 + i) * p.ldc + n_local, __uint_as_float(v[i]));
+                        }
+                    } else {                                        // bf16 C
+                        __nv_bfloat16* outb = p.Cb + int64_t(row0) * p.ldc + n0 + n_local;
+                        for (int c0 = 0; c0 < 256; c0 += 32) {
+                            if (c0 >= rows) break;
+                            uint32_t v[32];
+                            tmem_ld_32x32b_x32(taddr + c0, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (n_ok && c0 + i < rows) outb[int64_t(c0 + i) * p.ldc] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                        }
                     }
                 }
             }
