@@ -5,4 +5,4 @@ loaded by ``paper_2607_04031_b200.binding`` on first use and every call fails
 loudly when it is missing.  ``paper_2607_04031_b200.inputs`` (seeded synthetic
 inputs) is self-contained.
 """
-__all__ = ["binding", "inputs"]
+__all__ = ["binding", "inputs", "shard"]
