@@ -660,6 +660,9 @@ PROFILE_CASES = {
     "prefill_qkv": ("gemm", 4096, 8192, 10240),
     "relayout_o": ("relayout", 0, 8192, 8192),
     "moe_gate_up": ("moe", 0, 2048, 1536),
+    "kmajor_decode_qkv_m8": ("kmajor", 8, 8192, 10240),     # weights [N][K], (64, 32) memory tiles of Eq. 2
+    "fp8_decode_qkv_m8": ("fp8", 8, 8192, 10240),           # E4M3, 64 x 64 memory tiles
+    "hw_box_load_o": ("hw", 0, 8192, 8192),                 # every 64 x 256 box of the weight through a 2-D view
 }
 
 
@@ -681,6 +684,29 @@ def run_case(args):
         d_off = torch.from_numpy(offsets).to(dev)
         for _ in range(args.steps):
             tl.gemm_grouped(Am, Bt, Cm, d_off, q["experts"], rows, N, K, G, BR, BC)
+    elif kind in ("kmajor", "hw"):
+        w = inputs.bf16_normal((N, K), 0.02, seed=100, device=dev)
+        wt = torch.empty_like(w)
+        tl.relayout(w, wt, N, K, 2, G, 32, 64, tl.TO_TILE_MAJOR)
+        if kind == "kmajor":
+            A = inputs.bf16_normal((M, K), 1.0, seed=200, device=dev)
+            C = torch.empty((M, N), dtype=torch.float32, device=dev)
+            for _ in range(args.steps):
+                tl.gemm_kmajor(A, wt, C, M, N, K, G, 32, 64)
+        else:
+            dst = torch.empty(K * N, dtype=torch.bfloat16, device=dev)
+            coords = torch.tensor([[i, j] for j in range(0, N, 256) for i in range(0, K, 64)], dtype=torch.int32, device=dev)
+            desc = tl.hw_desc([K, N], [1, K], [64, 256], 2, 64, 32, K)
+            for _ in range(args.steps):
+                tl.hw_box_load(desc, wt, coords, dst)
+    elif kind == "fp8":
+        w = inputs.fp8_normal((N, K), 0.05, seed=100, device=dev).view(torch.uint8)
+        wt = torch.empty_like(w)
+        tl.relayout(w, wt, N, K, 1, G, 64, 64, tl.TO_TILE_MAJOR)
+        A = inputs.fp8_normal((M, K), 1.0, seed=200, device=dev).view(torch.uint8)
+        C = torch.empty((M, N), dtype=torch.float32, device=dev)
+        for _ in range(args.steps):
+            tl.gemm_fp8_kmajor(A, wt, C, M, N, K, G, 64, 64)
     else:
         W = inputs.bf16_normal((K, N), 0.02, seed=100, device=dev)
         Wt = torch.empty_like(W)
