@@ -16,6 +16,8 @@ CASES = [  # rows, cols, s, br, bc
     (256, 1024, 1, 64, 64),        # FP8 64 x 64 (Figure 1c)
     (256, 1024, 4, 8, 128),
     (96, 640, 2, 16, 16),          # 32-byte runs
+    (512, 256, 2, 256, 8),         # 16-byte runs of a 4 KB tile: shared-memory kernel, not the copy engine
+    (1056, 2176, 1, 32, 16),       # 16-byte runs, tiles overhang both edges
     (64, 256, 2, 8, 2),            # 4-byte runs: vectors gathered from 4 block rows
     (64, 256, 2, 16, 1),           # 2-byte runs
     (64, 256, 1, 32, 1),           # 1-byte runs
