@@ -473,6 +473,26 @@ def run_ours(args):
     del W_nk, W_nk_tile
     tl.device_status()
 
+    # ---- tile-major aware box loads (Section 4.3, emulated): every 64 x 256 weight-tile load of the gate_up weight
+    # kept [N][K] in (64, 32) memory tiles, through a 2-D and through a 4-D view of the same matrix
+    name, K, N = inputs.LLAMA70B_PROJ[2]
+    w_nk = W_row[name].t().contiguous()
+    w_nk_tile = torch.empty_like(w_nk)
+    tl.relayout(w_nk, w_nk_tile, N, K, 2, G, 32, 64, tl.TO_TILE_MAJOR)
+    del w_nk
+    hw = []
+    boxes_dst = torch.empty((K // 64) * (N // 256) * 64 * 256, dtype=torch.bfloat16, device=dev)
+    c2 = torch.tensor([[i, j] for j in range(0, N, 256) for i in range(0, K, 64)], dtype=torch.int32, device=dev)
+    c4 = torch.tensor([[0, 0, i // 64, j // 256] for j in range(0, N, 256) for i in range(0, K, 64)], dtype=torch.int32,
+                      device=dev)
+    for label, desc, cd in (("2d", tl.hw_desc([K, N], [1, K], [64, 256], 2, 64, 32, K), c2),
+                            ("4d", tl.hw_desc([64, 256, K // 64, N // 256], [1, K, 64, 256 * K], [64, 256, 1, 1], 2, 64, 32, K), c4)):
+        ms = time_calls([lambda: tl.hw_box_load(desc, w_nk_tile, cd, boxes_dst)], 5)
+        hw.append({"view": label, "boxes": int(cd.shape[0]), "ms": ms, "GBps": 2 * 2.0 * K * N / (ms * 1e-3) / 1e9})
+    extra["hw_box_load_gate_up"] = hw
+    del w_nk_tile, boxes_dst
+    tl.device_status()
+
     # ---- prefill leg (M = 4096): tensor-core bound
     Mp = inputs.LLAMA_PREFILL_M
     prefill = []
@@ -498,25 +518,6 @@ def run_ours(args):
                         sum(x["ms"] for x in prefill if x["layout"] == "row")}
     tl.device_status()
 
-    # ---- tile-major aware box loads (Section 4.3, emulated): every 64 x 256 weight-tile load of the gate_up weight
-    # kept [N][K] in (64, 32) memory tiles, through a 2-D and through a 4-D view of the same matrix
-    name, K, N = inputs.LLAMA70B_PROJ[2]
-    w_nk = W_row[name].t().contiguous()
-    w_nk_tile = torch.empty_like(w_nk)
-    tl.relayout(w_nk, w_nk_tile, N, K, 2, G, 32, 64, tl.TO_TILE_MAJOR)
-    del w_nk
-    hw = []
-    boxes_dst = torch.empty((K // 64) * (N // 256) * 64 * 256, dtype=torch.bfloat16, device=dev)
-    c2 = torch.tensor([[i, j] for j in range(0, N, 256) for i in range(0, K, 64)], dtype=torch.int32, device=dev)
-    c4 = torch.tensor([[0, 0, i // 64, j // 256] for j in range(0, N, 256) for i in range(0, K, 64)], dtype=torch.int32,
-                      device=dev)
-    for label, desc, cd in (("2d", tl.hw_desc([K, N], [1, K], [64, 256], 2, 64, 32, K), c2),
-                            ("4d", tl.hw_desc([64, 256, K // 64, N // 256], [1, K, 64, 256 * K], [64, 256, 1, 1], 2, 64, 32, K), c4)):
-        ms = time_calls([lambda: tl.hw_box_load(desc, w_nk_tile, cd, boxes_dst)], 5)
-        hw.append({"view": label, "boxes": int(cd.shape[0]), "ms": ms, "GBps": 2 * 2.0 * K * N / (ms * 1e-3) / 1e9})
-    extra["hw_box_load_gate_up"] = hw
-    del w_nk_tile, boxes_dst
-    tl.device_status()
 
     # ---- Qwen-3-30B-A3B MoE grouped leg
     q = inputs.QWEN_MOE
