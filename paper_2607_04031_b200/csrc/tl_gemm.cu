@@ -8,8 +8,9 @@
 // lands in shared memory in exactly the canonical swizzled operand form that tcgen05.mma reads -- MN-major for
 // weights stored with N contiguous, K-major for weights stored [N][K] (Eq. 2 as printed).  The weights can sit on
 // either side of the instruction:
-//   weights on N (tiles of up to 128 token rows: decode, MoE)  tokens are the M-side operand, one MMA covers all
-//                cta_n weight columns; TMEM lane = token row;
+//   weights on N (tiles of up to 128 token rows: decode, MoE)  tokens are the M-side operand (64-row MMAs for
+//                tiles of up to 64 tokens, else 128 rows; spare rows are zeroed once), one MMA covers all cta_n
+//                weight columns; TMEM lane = token row;
 //   weights on M (256-token tiles)  TMEM lane = weight column, the accumulator holds C transposed.
 // Memory tiles whose rows are shorter than 32 bytes cannot be boxed: four more warps load them with Eq. 1-2
 // address arithmetic and build the operand image by hand (Section 4.4).
@@ -54,6 +55,9 @@ struct alignas(64) GemmParams {
     int M;                      // dense rows (grouped: total rows)
     int N, K, E;
     int BM;                     // token rows per CTA tile: 16, 32, 64, 128 or 256
+    int umma_m;                 // weights-on-N kernels: rows of the MMA's token side, 64 when BM <= 64, else 128
+    int a_rows;                 // token rows a stage holds per 64-wide K slice: max(BM, umma_m) there, else BM; rows
+                                // beyond BM are zeroed once and never written again
     int BN;                     // weight columns per CTA tile: 128 or 256
     int n_tiles, k_iters;
     int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
@@ -341,7 +345,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     const int lane = threadIdx.x & 31;
     TL_TIMELINE_INIT();
     if (threadIdx.x == 0) { TL_STAMP(0); TL_COUNT(10, TL_CLOCK()); TL_COUNT(12, global_timer_ns()); }
-    const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.BM * kAtomBytes;
+    const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.a_rows * kAtomBytes;
     uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
     const int acc_cols = kWN ? kBN : p.BM;                   // TMEM columns of one MMA's accumulator
@@ -385,6 +389,19 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     }
             }
         }
+    }
+    // Token rows between BM and the rows the MMA reads are zeroed once; no copy ever writes them.  (The MMA's token
+    // side has at least 64 rows.  Whatever lies there is multiplied with the weights at full rate, and with stale
+    // data instead of zeros the tensor pipe draws enough power to pull the SM clock down under the board's cap.)
+    if (p.a_rows > p.BM && warp >= 2) {
+        const int per = (p.a_rows - p.BM) * (kAtomBytes / 16);          // 16-byte pieces per 64-wide K slice
+        const int total = p.num_stages * kSubK * per;
+        for (int i = int(threadIdx.x) - 64; i < total; i += int(blockDim.x) - 64) {
+            const int s = i / (kSubK * per), r = i % (kSubK * per);
+            uint8_t* slice = stages + size_t(s) * stage_bytes + kWBytes + size_t(r / per) * p.a_rows * kAtomBytes;
+            *reinterpret_cast<uint4*>(slice + size_t(p.BM) * kAtomBytes + size_t(r % per) * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
     }
     // Launched with programmatic stream serialisation: everything above (barriers, tensor memory, descriptor
     // prefetch) may run while the kernel before this one in the stream is still finishing.  Nothing that kernel
@@ -461,7 +478,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     const int k0 = (kit * kBK) << p.k_shift;        // first K element of the stage
 #pragma unroll
                     for (int sub = 0; sub < kSubK; ++sub)
-                        tma_load_2d(sa + size_t(sub) * p.BM * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
+                        tma_load_2d(sa + size_t(sub) * p.a_rows * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
                                     k0 + ((sub * 64) << p.k_shift), t.row0);
                     if (one_box) {
                         // the usual case, one box per stage: the column part of the coordinates was worked out once
@@ -512,8 +529,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 // operand K-major; M = kUmmaM, N = n_mma
                 const uint32_t w_major = p.w_kmajor ? 0u : (kWN ? (1u << 16) : (1u << 15));
                 // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
+                const uint32_t m_mma = kWN ? uint32_t(p.umma_m) : uint32_t(kUmmaM);
                 const uint32_t idesc = (1u << 4) | (kFp8 ? 0u : (1u << 7) | (1u << 10)) | w_major |
-                                       ((n_mma >> 3) << 17) | ((uint32_t(kUmmaM) >> 4) << 24);
+                                       ((n_mma >> 3) << 17) | ((m_mma >> 4) << 24);
                 const long long ca0 = TL_CLOCK();
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) {
                     ok = false;
@@ -538,7 +556,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 #pragma unroll
                     for (int j = 0; j < kKSteps; ++j) {
                         const uint64_t tok_desc = make_smem_desc(
-                            sa + uint32_t(j >> 2) * uint32_t(p.BM) * kAtomBytes + uint32_t(j & 3) * 32u, 16u, 1024u);
+                            sa + uint32_t(j >> 2) * uint32_t(p.a_rows) * kAtomBytes + uint32_t(j & 3) * 32u, 16u, 1024u);
 #pragma unroll
                         for (int u = 0; u < kNumN; ++u) {
                             const uint64_t w_desc =
@@ -634,9 +652,12 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             }
             if (ok && kWN) {
                 // TMEM lane = token row, columns = the tile's kBN weight columns: each thread owns one row of C.
-                const int row = quarter * 32 + lane;
+                // (MMA of 64 rows: rows 16q..16q+15 sit in the lower half of lane quarter q, the upper 16 lanes of
+                // each quarter hold nothing.)
+                const bool m64 = p.umma_m == 64;
+                const int row = m64 ? (lane < 16 ? quarter * 16 + lane : p.BM) : quarter * 32 + lane;
                 const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * uint32_t(acc_cols);
-                if (quarter * 32 < t.rows) {                     // this lane quarter holds at least one real row
+                if ((m64 ? quarter * 16 : quarter * 32) < t.rows) {      // this lane quarter holds at least one real row
                     float* dst = out + int64_t(row) * ld;
                     const bool gated = full && p.epi_swiglu;
                     __nv_bfloat16* hdst = p.H + int64_t(t.row0 + row) * p.ldh + (t.n0 >> 1);
@@ -943,6 +964,7 @@ static int ilog2(int64_t x) {
 
 struct GemmPlan {
     int BM, BN, BK;
+    int umma_m, a_rows;          // see GemmParams
     int weights_on_n;     // kWN variant of the kernel
     int stream_k;
     int grid;
@@ -987,13 +1009,16 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     if (BN == 256 && BM > 128) return TL_ERR_UNSUPPORTED;   // 2 accumulators x 2 groups x BM columns <= 512
     plan->BM = BM; plan->BN = BN; plan->BK = BK;
     plan->weights_on_n = BM <= 128;                         // tokens fit the 128 rows of the MMA's M side
-    const size_t stage = size_t(BK) * BN * 2 + size_t(BK / 64) * BM * kAtomBytes;
-    // 1 KB of slack to align the stages to 1024 bytes.  With the tokens on the M side the MMA always reads 128
-    // token rows, the tail of which (rows beyond the box) is whatever follows in shared memory: 16 KB more
-    // keep that read inside the allocation.  Those rows only feed accumulator rows that are never stored.
-    const size_t tail = plan->weights_on_n && BM < 128 ? 16 * 1024 : 0;
+    // With the tokens on the M side the MMA reads 64 rows (tiles of up to 64 tokens) or 128: a stage holds that
+    // many token rows per 64-wide K slice, the ones beyond BM zeroed once by the kernel.  They only feed
+    // accumulator rows that are never stored.
+    static const bool m128_only = getenv("TL_UMMA_M128") && atoi(getenv("TL_UMMA_M128")) != 0;    // measurement switch
+    plan->umma_m = BM <= 64 && !m128_only ? 64 : 128;
+    plan->a_rows = plan->weights_on_n && BM < plan->umma_m ? plan->umma_m : BM;
+    const size_t stage = size_t(BK) * BN * 2 + size_t(BK / 64) * plan->a_rows * kAtomBytes;
+    // 1 KB of slack to align the stages to 1024 bytes.
     // 12 KB stay free so that a CTA of the stream-K reduction kernel can be resident next to this one.
-    const size_t budget = kMaxDynamicSmem - 1024 - tail - 12 * 1024;
+    const size_t budget = kMaxDynamicSmem - 1024 - 12 * 1024;
     int stages = int(budget / stage);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return TL_ERR_UNSUPPORTED;
@@ -1002,7 +1027,7 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
         if (cap >= 2 && cap < stages) stages = cap;
     }
     plan->num_stages = stages;
-    plan->smem_bytes = size_t(stages) * stage + 1024 + tail;
+    plan->smem_bytes = size_t(stages) * stage + 1024;
     if (plan->smem_bytes < 120 * 1024) plan->smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
     const int64_t k_iters = ceil_div(K, BK);
     const int64_t total_iters = tile_bound * k_iters;
@@ -1308,6 +1333,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.K = int(K);
     p.E = E;
     p.BM = plan.BM;
+    p.umma_m = plan.umma_m;
+    p.a_rows = plan.a_rows;
     p.BN = plan.BN;
     p.n_tiles = int(ceil_div(N, plan.BN));
     p.k_iters = int(ceil_div(K, int64_t(plan.BK) << k_shift));
