@@ -76,10 +76,13 @@ int tl_device_status(uint32_t* detail);
  *   d_src, d_dst  device, rows*cols*elem_bytes bytes each, must not overlap.
  *   elem_bytes    1, 2 or 4.          G == block_rows*block_cols*elem_bytes.
  *   direction     tl_direction.
- * Enqueues one kernel on the tl_set_stream() stream.  A 16-byte-vectorised
- * kernel staged through shared memory is used when cols*elem_bytes is a
- * multiple of 16 and both pointers are 16-byte aligned; otherwise an
- * element-wise kernel (same result, slower).  rows == 0 or cols == 0 is a no-op.
+ * Enqueues one kernel on the tl_set_stream() stream.  When cols*elem_bytes is
+ * a multiple of 16 and both pointers are 16-byte aligned, block rows of 32
+ * bytes to 1 KB in memory tiles of at most 32 KB are moved by the copy engine
+ * (tensor copy on the row-major side, bulk copy on the tile-major side) and
+ * every other shape by a 16-byte-vectorised kernel staged through shared
+ * memory; otherwise an element-wise kernel runs (same result, slower).
+ * rows == 0 or cols == 0 is a no-op.
  */
 int tl_relayout(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes,
                 int64_t G, int block_rows, int block_cols, int direction);
