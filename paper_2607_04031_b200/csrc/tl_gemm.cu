@@ -407,7 +407,10 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     // prefetch) may run while the kernel before this one in the stream is still finishing.  Nothing that kernel
     // may have written (tokens, expert offsets, the partial-tile workspace, C) is touched before this wait, which
     // returns once it has completed and its writes are visible.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Grouped problems read the expert offsets, which that kernel may have produced, for the tables below; dense
+    // problems build their tables from the launch parameters alone and wait afterwards.
+    const bool tables_first = p.offsets == nullptr;
+    if (!tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
     // tiles before each expert (dense: one "expert" holding all M rows)
     load_row_starts(p, row_start);
     __syncthreads();
@@ -426,11 +429,6 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             range_tab[c] = static_cast<int>(Sched::split(total_iters, grid_eff0, c));
         __syncthreads();
     }
-    // Stream-K: let the reduction kernel that follows in the stream be scheduled already; it does its own
-    // set-up and then blocks until this whole grid has finished.
-    if (p.stream_k && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (threadIdx.x == 0) TL_STAMP(1);
-
     Sched sched;
 #ifdef TL_TIMELINE
     // measurement builds: optionally hand the ranges out in reverse CTA order; record the SM id
@@ -440,6 +438,11 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 #else
     sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
 #endif
+    if (tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Stream-K: let the reduction kernel that follows in the stream be scheduled already; it does its own
+    // set-up and then blocks until this whole grid has finished.
+    if (p.stream_k && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 0) TL_STAMP(1);
     volatile uint32_t* abort_ptr = &abort_flag;
 
     if (warp == 0) {
