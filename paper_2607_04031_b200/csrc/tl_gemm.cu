@@ -313,14 +313,15 @@ __device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, in
 }
 
 // kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256).
-// kWN selects which side of the MMA the weights are on.  A tcgen05.mma of one CTA takes about 180 clocks
-// whatever its shape, so what matters is how many weight bytes one instruction consumes:
+// kWN selects which side of the MMA the weights are on.  The tensor pipe takes N/2 clocks per MMA whatever M is,
+// and the thread that issues the MMAs runs alone in its warp (every scalar instruction between two MMAs costs it
+// several clocks), so for small token tiles what matters is how many weight bytes one instruction consumes:
 //   kWN = false  weights on the M side: kBN/128 MMAs per K step, each 128 (or 64) weight columns x up to 256
 //                tokens.  For prefill (256-token tiles): the accumulator is C transposed, TMEM lane = weight
 //                column, and the epilogue writes 128-byte row segments.
 //   kWN = true   weights on the N side: one MMA per K step covers all kBN (up to 256) weight columns, tokens
 //                (at most 128 per tile) on the M side.  For decode and MoE: 8 KB of weights per instruction
-//                instead of 4 KB, which lifts the instruction-rate ceiling above the HBM rate.  TMEM lane =
+//                instead of 4 KB, half as many instructions per byte streamed.  TMEM lane =
 //                token, and every thread writes its token's row of C in 16-byte pieces.
 template <int kBK, int kBN, bool kWN, bool kFp8>
 __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
@@ -525,6 +526,18 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             Work w;
             bool ok = true;
+            // Descriptor words that do not change: the upper halves, the constant bits of the lower halves, and
+            // the (address >> 4) offsets of every K step (kept in registers: the loop below adds one per MMA).
+            const uint64_t tok_hi64 = smem_desc_hi(16u, 1024u, 2u);
+            const uint32_t tok_hi = uint32_t(tok_hi64 >> 32), tok_lo_const = uint32_t(tok_hi64);
+            const uint32_t w_hi = uint32_t(p.w_desc_hi >> 32), w_lo_const = uint32_t(p.w_desc_hi);
+            uint32_t w_off[kKSteps], tok_off[kKSteps];
+#pragma unroll
+            for (int j = 0; j < kKSteps; ++j) {
+                w_off[j] = p.kstep_off[j] >> 4;
+                tok_off[j] = (uint32_t(j >> 2) * uint32_t(p.a_rows) * kAtomBytes + uint32_t(j & 3) * 32u) >> 4;
+            }
+            const uint32_t ugroup16 = p.ugroup_off >> 4;
             while (ok && sched.next(w)) {
                 const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
                 const uint32_t n_mma = kWN ? uint32_t(kBN) : uint32_t((t.rows + 15) & ~15);
@@ -555,23 +568,17 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     tc_fence_after_sync();
                     TL_STAMP_ONCE(2);
                     const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
-                    const uint32_t sa = sw + kWBytes;
+                    const uint32_t w_lo0 = w_lo_const | ((sw & 0x3FFFFu) >> 4);
+                    const uint32_t tok_lo0 = tok_lo_const | (((sw + kWBytes) & 0x3FFFFu) >> 4);
+                    const uint32_t first = kit > w.kbeg ? 1u : 0u;
 #pragma unroll
                     for (int j = 0; j < kKSteps; ++j) {
-                        const uint64_t tok_desc = make_smem_desc(
-                            sa + uint32_t(j >> 2) * uint32_t(p.a_rows) * kAtomBytes + uint32_t(j & 3) * 32u, 16u, 1024u);
 #pragma unroll
                         for (int u = 0; u < kNumN; ++u) {
-                            const uint64_t w_desc =
-                                make_smem_desc(sw + p.kstep_off[j] + uint32_t(u) * p.ugroup_off, p.w_desc_hi);
-                            const uint32_t accum = (kit > w.kbeg || j > 0) ? 1u : 0u;
-                            if (kFp8) {
-                                if (kWN) umma_f8(d_tmem, tok_desc, w_desc, idesc, accum);
-                                else umma_f8(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc, accum);
-                            } else {
-                                if (kWN) umma_bf16(d_tmem, tok_desc, w_desc, idesc, accum);
-                                else umma_bf16(d_tmem + uint32_t(u * acc_cols), w_desc, tok_desc, idesc, accum);
-                            }
+                            const uint32_t accum = j > 0 ? 1u : first;
+                            const uint32_t w_lo = w_lo0 + w_off[j] + uint32_t(u) * ugroup16;
+                            if (kWN) umma_split<kFp8>(d_tmem, tok_lo0 + tok_off[j], tok_hi, w_lo, w_hi, idesc, accum);
+                            else umma_split<kFp8>(d_tmem + uint32_t(u * acc_cols), w_lo, w_hi, tok_lo0 + tok_off[j], tok_hi, idesc, accum);
                         }
                     }
                     umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
