@@ -92,6 +92,27 @@ __device__ __forceinline__ void umma_pair_f8(uint32_t d_tmem, uint64_t a_desc, u
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the descriptors given as 32-bit halves (constant upper words, offsets added to the lower word).
+template <bool kFp8>
+__device__ __forceinline__ void umma_pair_split(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                uint32_t idesc, uint32_t accumulate) {
+    if (kFp8)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\t"
+            "mov.b64 a, {%1, %2};\n\tmov.b64 b, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], a, b, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\t"
+            "mov.b64 a, {%1, %2};\n\tmov.b64 b, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], a, b, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+}
 // Arrives on the barrier at the same shared-memory offset in both CTAs once the MMAs issued so far are done.
 __device__ __forceinline__ void umma_pair_commit_both(uint64_t* bar) {
     asm volatile(
@@ -269,6 +290,13 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             bool ok = true;
             const long long t_begin = TL_CLK();
             (void)t_begin;
+            // constant descriptor words and per-K-step offsets, in registers for the issue loop
+            const uint64_t tok_hi64 = smem_desc_hi(16u, 1024u, 2u);
+            const uint32_t tok_hi = uint32_t(tok_hi64 >> 32), tok_lo_const = uint32_t(tok_hi64);
+            const uint32_t w_hi = uint32_t(p.w_desc_hi >> 32), w_lo_const = uint32_t(p.w_desc_hi);
+            uint32_t w_off[kKSteps];
+#pragma unroll
+            for (int j = 0; j < kKSteps; ++j) w_off[j] = p.kstep_off[j] >> 4;
             for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
                 const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
                 if (pt.halves == 0) continue;
@@ -292,18 +320,17 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     (void)c0;
                     tc_fence_after_sync();
                     const uint32_t sw = smem_u32(stages + size_t(stage) * kStageBytes);
-                    const uint32_t sa = sw + kWBytes;
+                    const uint32_t w_lo0 = w_lo_const | ((sw & 0x3FFFFu) >> 4);
+                    const uint32_t tok_lo0 = tok_lo_const | (((sw + kWBytes) & 0x3FFFFu) >> 4);
+                    const uint32_t first = kit > 0 ? 1u : 0u;
+                    const bool two = kHalves == 2 && pt.halves == 2;
 #pragma unroll
                     for (int j = 0; j < kKSteps; ++j) {
-                        const uint64_t w_desc = make_smem_desc(sw + p.kstep_off[j], p.w_desc_hi);
-                        const uint64_t tok_desc = make_smem_desc(sa + uint32_t(j) * 32u, 16u, 1024u);
-                        if (kFp8) umma_pair_f8(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
-                        else umma_pair_bf16(d_tmem, w_desc, tok_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
-                        if (kHalves == 2 && pt.halves == 2) {       // the same weights on the second token block
-                            const uint64_t tok2_desc = make_smem_desc(sa + kTokBytes + uint32_t(j) * 32u, 16u, 1024u);
-                            if (kFp8) umma_pair_f8(d_tmem + 256u, w_desc, tok2_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
-                            else umma_pair_bf16(d_tmem + 256u, w_desc, tok2_desc, idesc, (kit > 0 || j > 0) ? 1u : 0u);
-                        }
+                        const uint32_t accum = j > 0 ? 1u : first;
+                        umma_pair_split<kFp8>(d_tmem, w_lo0 + w_off[j], w_hi, tok_lo0 + uint32_t(j) * 2u, tok_hi, idesc, accum);
+                        if (two)                                    // the same weights on the second token block
+                            umma_pair_split<kFp8>(d_tmem + 256u, w_lo0 + w_off[j], w_hi,
+                                                  tok_lo0 + (kTokBytes >> 4) + uint32_t(j) * 2u, tok_hi, idesc, accum);
                     }
                     umma_pair_commit_both(&empty_bar[stage]);       // frees the stage in both CTAs
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
