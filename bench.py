@@ -40,8 +40,8 @@ WORKLOAD = "llama3.1-70b decode linear layers (qkv, o, gate_up, down; M in {1,8,
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode GEMM kernel, from the ncu
 # capture summarised in profiles/ (None until a capture exists for this kernel version).
-NCU_TRAFFIC_RATIO = 172.83 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
-NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 167.99 MB read + 4.84 MB written for 168.23 MB algorithmic; "
+NCU_TRAFFIC_RATIO = 172.81 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
+NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 167.99 MB read + 4.82 MB written for 168.23 MB algorithmic; "
                     "scaled to the step's average launch by bytes processed (traffic is proportional to the weight bytes)")
 
 
