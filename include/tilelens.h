@@ -90,6 +90,17 @@ int tl_relayout(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int 
 int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes,
                    int64_t G, int block_rows, int block_cols, int direction, void* cuda_stream);
 
+/*
+ * The same rewrite for n matrices that share element size, memory tile and direction (the weights of a layer at
+ * load time, Section 5.1), in stream order.  d_srcs, d_dsts, rows, cols: HOST arrays of n entries (device
+ * pointers, extents); each pair as in tl_relayout, no destination overlapping any other buffer of the call.
+ * Matrices that can take the copy-engine path are moved by ONE launch per run of up to 8 of them, without a kernel
+ * boundary in between; the others go through tl_relayout_on one by one.  The first matrix that fails
+ * tl_relayout's argument checks ends the call with that error, the ones before it already enqueued.
+ */
+int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, const int64_t* rows, const int64_t* cols,
+                      int elem_bytes, int64_t G, int block_rows, int block_cols, int direction, void* cuda_stream);
+
 /* ------------------------------------------------------------------ GEMM */
 
 /*

@@ -28,6 +28,7 @@ _SIGNATURES = {
     "tl_device_status": (_int, [ctypes.POINTER(ctypes.c_uint32)]),
     "tl_relayout": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int]),
     "tl_relayout_on": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int, _vp]),
+    "tl_relayout_batch": (_int, [_int, _vp, _vp, _vp, _vp, _int, _i64, _int, _int, _int, _vp]),
     "tl_gemm": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_grouped": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
     "tl_gemm_bf16": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _vp]),
@@ -129,6 +130,17 @@ def relayout(src: torch.Tensor, dst: torch.Tensor, rows: int, cols: int, elem_by
              block_rows: int, block_cols: int, direction: int, stream=None):
     _check(lib().tl_relayout_on(_dev_ptr(src), _dev_ptr(dst), rows, cols, elem_bytes, G, block_rows, block_cols,
                                 direction, _stream_ptr(stream)), "tl_relayout")
+
+
+def relayout_batch(srcs, dsts, shapes, elem_bytes: int, G: int, block_rows: int, block_cols: int,
+                   direction: int = TO_TILE_MAJOR, stream=None):
+    """srcs, dsts: lists of CUDA tensors; shapes: list of (rows, cols).  One launch for the whole list where possible."""
+    n = len(srcs)
+    ptr_arr, i64_arr = ctypes.c_void_p * n, ctypes.c_int64 * n
+    _check(lib().tl_relayout_batch(n, ptr_arr(*[_dev_ptr(t) for t in srcs]), ptr_arr(*[_dev_ptr(t) for t in dsts]),
+                                   i64_arr(*[int(r) for r, _ in shapes]), i64_arr(*[int(c) for _, c in shapes]),
+                                   elem_bytes, G, block_rows, block_cols, direction, _stream_ptr(stream)),
+           "tl_relayout_batch")
 
 
 def gemm(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, M: int, N: int, K: int, G: int = 4096,

@@ -10,6 +10,7 @@
 //                         row is shorter than 16 bytes the vectors of the tile-major side are assembled from
 //                         several shared-memory rows, one piece-wide access per row;
 //   element-wise          for unaligned pointers or pitches.
+// relayout_tma_batch_kernel is relayout_tma_kernel over the step lists of several matrices in one launch.
 #include "tl_common.cuh"
 
 #include <cstdlib>
@@ -352,6 +353,152 @@ static int relayout_tma_launch(const void* d_src, void* d_dst, int64_t rows, int
     return check_cuda(cudaLaunchKernelEx(&cfg, relayout_tma_kernel, p));
 }
 
+// ------------------------------------------------------------------ several matrices in one launch
+// The same ring of copies over the concatenated step lists of up to kBatchMax matrices that share element size,
+// memory tile and direction (the weights of one layer at load time): no kernel boundary, hence no ramp and tail,
+// between them.
+constexpr int kBatchMax = 8;
+
+struct RelayoutTmaBatch {
+    CUtensorMap row_map[kBatchMax];
+    uint8_t* tile_base[kBatchMax];
+    int64_t steps_begin[kBatchMax + 1];    // first global step of each matrix
+    int steps_x[kBatchMax];                // steps along a block row
+    int blocks_per_row[kBatchMax];
+    int nb[kBatchMax];                     // memory tiles per step (min(tile budget, blocks per row))
+    uint32_t* status;
+    int64_t G;
+    int br, n;
+    int to_tile_major;
+};
+
+__global__ void __launch_bounds__(32, kTmaCtasPerSm) relayout_tma_batch_kernel(const __grid_constant__ RelayoutTmaBatch p) {
+    extern __shared__ __align__(1024) uint8_t smem_tma[];
+    __shared__ __align__(8) uint64_t full_bar[kTmaStages];
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x != 0) return;
+    uint8_t* bufs = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_tma) + 127) & ~uintptr_t(127));
+    for (int s = 0; s < kTmaStages; ++s) mbar_init(&full_bar[s], 1);
+    abort_flag = 0;
+    fence_mbar_init();
+    for (int i = 0; i < p.n; ++i) tma_prefetch_desc(&p.row_map[i]);
+    volatile uint32_t* abort_ptr = &abort_flag;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    const int64_t first = blockIdx.x, stride = gridDim.x, total = p.steps_begin[p.n];
+    const int64_t mine = first < total ? (total - first + stride - 1) / stride : 0;
+    struct Step { int m; int brow; int b0; int nbt; };
+    auto locate = [&](int64_t i) {
+        const int64_t g = first + i * stride;
+        int m = 0;
+        while (m + 1 < p.n && g >= p.steps_begin[m + 1]) ++m;
+        const int64_t local = g - p.steps_begin[m];
+        Step st;
+        st.m = m;
+        st.brow = int(local / p.steps_x[m]);
+        st.b0 = int(local % p.steps_x[m]) * p.nb[m];
+        st.nbt = p.blocks_per_row[m] - st.b0 < p.nb[m] ? p.blocks_per_row[m] - st.b0 : p.nb[m];
+        return st;
+    };
+    auto tile_ptr = [&](const Step& st) {
+        return p.tile_base[st.m] + (int64_t(st.brow) * p.blocks_per_row[st.m] + st.b0) * p.G;
+    };
+    auto issue_load = [&](int64_t i) {
+        const Step st = locate(i);
+        const int s = int(i % kTmaStages);
+        uint8_t* buf = bufs + size_t(s) * kTmaTileBytes;
+        if (p.to_tile_major) {
+            mbar_arrive_expect_tx(&full_bar[s], uint32_t(p.nb[st.m]) * uint32_t(p.G));     // a box always counts in full
+            tma_load_3d(buf, &p.row_map[st.m], &full_bar[s], 0, st.brow * p.br, st.b0);
+        } else {
+            mbar_arrive_expect_tx(&full_bar[s], uint32_t(st.nbt) * uint32_t(p.G));
+            bulk_load_1d(buf, tile_ptr(st), uint32_t(st.nbt) * uint32_t(p.G), &full_bar[s]);
+        }
+    };
+    const int64_t ahead = mine < kTmaStages - 1 ? mine : kTmaStages - 1;
+    for (int64_t i = 0; i < ahead; ++i) issue_load(i);
+    for (int64_t i = 0; i < mine; ++i) {
+        const int s = int(i % kTmaStages);
+        if (!mbar_wait_bounded(&full_bar[s], uint32_t(i / kTmaStages) & 1u, abort_ptr, p.status, kWaitRelayoutFull)) break;
+        const Step st = locate(i);
+        const uint8_t* buf = bufs + size_t(s) * kTmaTileBytes;
+        if (p.to_tile_major) bulk_store_1d(tile_ptr(st), buf, uint32_t(st.nbt) * uint32_t(p.G));
+        else tma_store_3d(&p.row_map[st.m], buf, 0, st.brow * p.br, st.b0);
+        bulk_commit_group();
+        if (i + kTmaStages - 1 < mine) {
+            bulk_wait_group_read<1>();
+            issue_load(i + kTmaStages - 1);
+        }
+    }
+    bulk_wait_group_read<0>();
+}
+
+// Whether one matrix can take the copy-engine path (the conditions of relayout_tma_launch).
+static bool relayout_tma_eligible(const void* d_src, const void* d_dst, int64_t rows, int64_t cols, int s, int64_t G, int br,
+                                  int bc) {
+    const int64_t run = int64_t(bc) * s, pitch = cols * s;
+    if (run < 32 || run > 1024 || G > kTmaTileBytes || br > 256) return false;
+    if (pitch % 16 != 0 || pitch >= (int64_t(1) << 40) || rows >= (int64_t(1) << 31)) return false;
+    return reinterpret_cast<uintptr_t>(d_src) % 16 == 0 && reinterpret_cast<uintptr_t>(d_dst) % 16 == 0;
+}
+
+static int relayout_tma_batch_launch(int n, const void* const* srcs, void* const* dsts, const int64_t* rows,
+                                     const int64_t* cols, int s, int64_t G, int br, int bc, int direction,
+                                     cudaStream_t stream) {
+    if (int rc = ensure_control()) return rc;
+    if (int rc = ensure_device_info()) return rc;
+    RelayoutTmaBatch p;
+    memset(&p, 0, sizeof p);
+    const bool to_tile = direction == TL_TO_TILE_MAJOR;
+    const int64_t run = int64_t(bc) * s;
+    int nb_max = int(kTmaTileBytes / G);
+    if (nb_max > 256) nb_max = 256;
+    p.steps_begin[0] = 0;
+    for (int i = 0; i < n; ++i) {
+        const void* row_side = to_tile ? srcs[i] : dsts[i];
+        void* tile_side = to_tile ? dsts[i] : const_cast<void*>(srcs[i]);
+        const int64_t blocks_per_row = cols[i] / bc, pitch = cols[i] * s;
+        const int nb = nb_max > blocks_per_row ? int(blocks_per_row) : nb_max;
+        const uint64_t dims[3] = {uint64_t(run / 4), uint64_t(rows[i]), uint64_t(blocks_per_row)};
+        const uint64_t strides[3] = {4, uint64_t(pitch), uint64_t(run)};
+        const uint32_t box[3] = {uint32_t(run / 4), uint32_t(br), uint32_t(nb)};
+        if (int rc = encode_tensor_map(&p.row_map[i], row_side, int(CU_TENSOR_MAP_DATA_TYPE_UINT32), int(CU_TENSOR_MAP_SWIZZLE_NONE),
+                                       3, dims, strides, box))
+            return rc;
+        p.tile_base[i] = static_cast<uint8_t*>(tile_side);
+        p.blocks_per_row[i] = int(blocks_per_row);
+        p.nb[i] = nb;
+        p.steps_x[i] = int(ceil_div(blocks_per_row, nb));
+        p.steps_begin[i + 1] = p.steps_begin[i] + int64_t(p.steps_x[i]) * (rows[i] / br);
+    }
+    p.status = state().ctl.d_status;
+    p.G = G;
+    p.br = br;
+    p.n = n;
+    p.to_tile_major = to_tile;
+    const size_t smem = size_t(kTmaStages) * kTmaTileBytes + 128;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (int rc = check_cuda(cudaFuncSetAttribute(relayout_tma_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))))
+            return rc;
+        attr_set = true;
+    }
+    const int64_t max_grid = int64_t(state().sm_count) * kTmaCtasPerSm, total = p.steps_begin[n];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(total < max_grid ? total : max_grid));
+    cfg.blockDim = dim3(32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    static const bool no_pdl = getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0;     // measurement switch
+    cfg.numAttrs = no_pdl ? 0 : 1;
+    return check_cuda(cudaLaunchKernelEx(&cfg, relayout_tma_batch_kernel, p));
+}
+
 static int ilog2(int64_t x) {
     int l = 0;
     while ((int64_t(1) << l) < x) ++l;
@@ -442,6 +589,44 @@ int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, i
                    int block_rows, int block_cols, int direction, void* cuda_stream) {
     return tl::relayout_launch(d_src, d_dst, rows, cols, elem_bytes, G, block_rows, block_cols, direction,
                                static_cast<cudaStream_t>(cuda_stream));
+}
+
+int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, const int64_t* rows, const int64_t* cols,
+                      int elem_bytes, int64_t G, int block_rows, int block_cols, int direction, void* cuda_stream) {
+    if (n < 0 || (n > 0 && (!d_srcs || !d_dsts || !rows || !cols))) return TL_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    static const bool no_tma = getenv("TL_RELAYOUT_NO_TMA") && atoi(getenv("TL_RELAYOUT_NO_TMA")) != 0;
+    // One launch when every matrix passes the argument checks of tl_relayout, is non-empty and can take the
+    // copy-engine path; otherwise (and beyond kBatchMax matrices) one tl_relayout_on per matrix, in order.
+    int i = 0;
+    while (i < n) {
+        int m = 0;
+        while (!no_tma && i + m < n && m < tl::kBatchMax) {
+            const int j = i + m;
+            const int64_t bytes = rows[j] * cols[j] * elem_bytes;
+            const uintptr_t a = reinterpret_cast<uintptr_t>(d_srcs[j]), b = reinterpret_cast<uintptr_t>(d_dsts[j]);
+            const bool ok = (elem_bytes == 1 || elem_bytes == 2 || elem_bytes == 4) && block_rows > 0 && block_cols > 0 &&
+                            int64_t(block_rows) * block_cols * elem_bytes == G && tl::is_pow2(block_rows) && tl::is_pow2(block_cols) &&
+                            (direction == TL_TO_TILE_MAJOR || direction == TL_TO_ROW_MAJOR) && rows[j] > 0 && cols[j] > 0 &&
+                            rows[j] % block_rows == 0 && cols[j] % block_cols == 0 && d_srcs[j] && d_dsts[j] &&
+                            !(a < b + bytes && b < a + bytes) &&
+                            tl::relayout_tma_eligible(d_srcs[j], d_dsts[j], rows[j], cols[j], elem_bytes, G, block_rows, block_cols);
+            if (!ok) break;
+            ++m;
+        }
+        if (m >= 2) {
+            if (int rc = tl::relayout_tma_batch_launch(m, d_srcs + i, d_dsts + i, rows + i, cols + i, elem_bytes, G, block_rows,
+                                                       block_cols, direction, stream))
+                return rc;
+            i += m;
+        } else {
+            if (int rc = tl::relayout_launch(d_srcs[i], d_dsts[i], rows[i], cols[i], elem_bytes, G, block_rows, block_cols,
+                                             direction, stream))
+                return rc;
+            ++i;
+        }
+    }
+    return TL_OK;
 }
 
 int tl_relayout(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes, int64_t G,

@@ -88,3 +88,40 @@ def test_errors():
     with pytest.raises(tl.TileLensError) as e:
         tl.relayout(a, a, 64, 64, 2, 2048, 16, 64, tl.TO_TILE_MAJOR)     # in place
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("direction", [0, 1])
+def test_batch_of_matrices_in_one_launch_matches_oracle(direction):
+    # eleven matrices of unequal shapes: a run of eight in one launch, then three; the tile is 16 x 128 bf16
+    from gpu_util import DEV, tl
+    br, bc, s = 16, 128, 2
+    shapes = [(512, 512), (1056, 2176), (16, 128), (48, 1280), (2048, 256), (32, 8192), (640, 384), (16, 256),
+              (4096, 128), (64, 1024), (528, 640)]
+    srcs, dsts, wants = [], [], []
+    for i, (rows, cols) in enumerate(shapes):
+        host = inputs.random_bytes(rows * cols * s, seed=100 + i)
+        srcs.append(torch.from_numpy(host).to(DEV))
+        dsts.append(torch.full_like(srcs[-1], 0xEE))
+        wants.append(tlo.relayout(host, rows, cols, s, br, bc, direction))
+    tl.relayout_batch(srcs, dsts, shapes, s, br * bc * s, br, bc, direction)
+    tl.device_status()
+    for i, (d, w) in enumerate(zip(dsts, wants)):
+        assert np.array_equal(d.cpu().numpy(), w), shapes[i]
+
+
+def test_batch_falls_back_per_matrix_and_reports_argument_errors():
+    from gpu_util import DEV, tl
+    # 8-byte block rows cannot take the copy engine: every matrix goes through the single call
+    br, bc, s = 64, 8, 1
+    shapes = [(128, 64), (64, 256)]
+    hosts = [inputs.random_bytes(r * c * s, seed=7 + i) for i, (r, c) in enumerate(shapes)]
+    srcs = [torch.from_numpy(h).to(DEV) for h in hosts]
+    dsts = [torch.empty_like(t) for t in srcs]
+    tl.relayout_batch(srcs, dsts, shapes, s, br * bc * s, br, bc, tl.TO_TILE_MAJOR)
+    tl.device_status()
+    for h, d, (r, c) in zip(hosts, dsts, shapes):
+        assert np.array_equal(d.cpu().numpy(), tlo.relayout(h, r, c, s, br, bc, tlo.TO_TILE_MAJOR))
+    # a matrix whose rows are not whole blocks ends the call with the single call's error
+    with pytest.raises(tl.TileLensError):
+        tl.relayout_batch(srcs, dsts, [(128, 64), (60, 256)], s, br * bc * s, br, bc, tl.TO_TILE_MAJOR)
+    tl.relayout_batch([], [], [], 2, 4096, 16, 128, tl.TO_TILE_MAJOR)          # empty list: no-op
