@@ -61,6 +61,22 @@ def test_relayout_argument_checks_need_no_device(tl):
     assert L.tl_relayout(bogus_a, ctypes.c_void_p(0x10100), 64, 64, 2, 2048, 16, 64, 0) == 1
 
 
+def test_relayout_batch_argument_checks_need_no_device(tl):
+    L = tl.lib()
+    P2, I2 = ctypes.c_void_p * 2, ctypes.c_int64 * 2
+    srcs, dsts = P2(0x10000, 0x200000), P2(0x90000, 0x300000)
+    # nothing to do; negative count; missing arrays
+    assert L.tl_relayout_batch(0, None, None, None, None, 2, 4096, 16, 128, 0, None) == 0
+    assert L.tl_relayout_batch(-1, srcs, dsts, I2(64, 64), I2(128, 128), 2, 4096, 16, 128, 0, None) == 1
+    assert L.tl_relayout_batch(2, None, dsts, I2(64, 64), I2(128, 128), 2, 4096, 16, 128, 0, None) == 1
+    # the first bad matrix ends the call with tl_relayout's own error: G mismatch, indivisible rows, odd tile
+    assert L.tl_relayout_batch(2, srcs, dsts, I2(64, 64), I2(128, 128), 2, 2048, 16, 128, 0, None) == 1
+    assert L.tl_relayout_batch(2, srcs, dsts, I2(60, 64), I2(128, 128), 2, 4096, 16, 128, 0, None) == 1
+    assert L.tl_relayout_batch(2, srcs, dsts, I2(48, 48), I2(48, 48), 2, 12 * 12 * 2, 12, 12, 0, None) == 2
+    # empty matrices are skipped one by one
+    assert L.tl_relayout_batch(2, srcs, dsts, I2(0, 0), I2(128, 128), 2, 4096, 16, 128, 0, None) == 0
+
+
 def test_read_amp_argument_checks_need_no_device(tl):
     L = tl.lib()
     f, u = ctypes.c_uint64(), ctypes.c_uint64()
