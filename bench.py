@@ -688,6 +688,7 @@ PROFILE_CASES = {
     "kmajor_decode_qkv_m8": ("kmajor", 8, 8192, 10240),     # weights [N][K], (64, 32) memory tiles of Eq. 2
     "fp8_decode_qkv_m8": ("fp8", 8, 8192, 10240),           # E4M3, 64 x 64 memory tiles
     "hw_box_load_o": ("hw", 0, 8192, 8192),                 # every 64 x 256 box of the weight through a 2-D view
+    "relayout_layer": ("relayout_batch", 0, 0, 0),          # the four Llama weights in one launch (3.4 GB resident)
 }
 
 
@@ -709,6 +710,11 @@ def run_case(args):
         d_off = torch.from_numpy(offsets).to(dev)
         for _ in range(args.steps):
             tl.gemm_grouped(Am, Bt, Cm, d_off, q["experts"], rows, N, K, G, BR, BC)
+    elif kind == "relayout_batch":
+        srcs = [inputs.bf16_normal((k, n), 0.02, seed=100 + i, device=dev) for i, (_, k, n) in enumerate(inputs.LLAMA70B_PROJ)]
+        dsts = [torch.empty_like(t) for t in srcs]
+        for _ in range(args.steps):
+            tl.relayout_batch(srcs, dsts, [(k, n) for _, k, n in inputs.LLAMA70B_PROJ], 2, G, BR, BC, tl.TO_TILE_MAJOR)
     elif kind in ("kmajor", "hw"):
         w = inputs.bf16_normal((N, K), 0.02, seed=100, device=dev)
         wt = torch.empty_like(w)
