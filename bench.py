@@ -373,6 +373,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "gemm_kernel, stream-K decode variants <BK=64,BN=256,weights-on-N> (M<=16) and <128,128,weights-on-N> (M=32)", "achieved": gemm_gbs,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
                 "peak_source": f"of {peaks['source']}", "frac_of_nominal_8TBs": gemm_gbs / 8000.0,
+                "frac_of_nominal_7p7TBs_hgx": gemm_gbs / 7700.0,
                 "traffic": NCU_TRAFFIC_RATIO * gemm_step_bytes / 12, "traffic_note": NCU_TRAFFIC_NOTE,
                 "algorithmic_bytes_per_launch_avg": gemm_step_bytes / 12,
                 "avg_launch_us": g_ms / g_n * 1e3,
