@@ -422,6 +422,37 @@ def run_ours(args):
     row_t = sum(x["us"] for x in per_shape if x["layout"] == "row")
     extra["tile_vs_row_time_ratio_decode"] = tile_t / row_t
 
+    # ---- the same twelve products as three independent decode batches on three streams (one per batch size, own
+    # split-K workspace each): CTAs of one product fill the SMs that the tail of another leaves free.  Reported
+    # beside the step, not as the step: inside one decode loop the products depend on each other.
+    try:
+        ws3 = {M: torch.empty(max(tl.gemm_workspace_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ) + 256,
+                              dtype=torch.uint8, device=dev) for M in inputs.LLAMA_DECODE_M}
+        side = {M: torch.cuda.Stream(device=dev) for M in inputs.LLAMA_DECODE_M}
+        main_stream = torch.cuda.current_stream()
+
+        def three_streams():
+            fork = torch.cuda.Event()
+            fork.record(main_stream)
+            for M in inputs.LLAMA_DECODE_M:
+                side[M].wait_event(fork)
+                tl.set_workspace(ws3[M])             # the pointer travels with each launch
+                for name, K, N in inputs.LLAMA70B_PROJ:
+                    tl.gemm(A_dec[name, M], W_tile[name], C_dec[name, M], M, N, K, G, BR, BC, stream=side[M])
+                join = torch.cuda.Event()
+                join.record(side[M])
+                main_stream.wait_event(join)
+
+        ms3 = time_calls([three_streams], 20)
+        tl.set_workspace(None)
+        extra["decode_three_streams"] = {"us": ms3 * 1e3, "GBps": gemm_step_bytes / (ms3 * 1e-3) / 1e9,
+                                         "note": "12 decode products, one stream per batch size (M = 1, 8, 32)"}
+        del ws3
+    except Exception as exc:  # report, never hide
+        tl.set_workspace(None)
+        extra["decode_three_streams"] = {"error": f"{type(exc).__name__}: {exc}"}
+    tl.device_status()
+
     # ---- K-contiguous flavour (weights kept [N][K]; Eq. 2 as printed with the (64, 32) memory tile), M = 8
     W_nk, W_nk_tile = {}, {}
     for name, K, N in inputs.LLAMA70B_PROJ:
