@@ -363,3 +363,34 @@ def test_caller_workspace_and_errors():
     assert e.value.status == 2
     C = torch.zeros((0, N), dtype=torch.float32, device=DEV)
     tl.gemm(A.to(DEV)[:0], Bt, C, 0, N, K, 4096, 16, 128)          # no rows: no-op
+
+
+def test_products_on_two_streams_with_their_own_workspaces_match_serial_runs():
+    # The header's rule for concurrent calls: each needs its own split-K workspace (the pointer travels with the
+    # launch).  Two decode-shaped products on two streams, repeated, must give the bits of the serial runs.
+    from gpu_util import DEV, tile_major_on_device, tl
+    shapes = [(8, 1280, 4096), (32, 2048, 2304)]                        # (M, N, K): both cut stream-K fashion
+    A, Bt, want, ws = [], [], [], []
+    for i, (M, N, K) in enumerate(shapes):
+        A.append(inputs.bf16_normal((M, K), 1.0, seed=40 + i).to(DEV))
+        Bt.append(tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=50 + i), K, N, 16, 128))
+        C = torch.empty((M, N), dtype=torch.float32, device=DEV)
+        tl.gemm(A[i], Bt[i], C, M, N, K, 4096, 16, 128)
+        want.append(C)
+        ws.append(torch.empty(tl.gemm_workspace_bytes(M, N, K) + 256, dtype=torch.uint8, device=DEV))
+    tl.device_status()
+    streams = [torch.cuda.Stream(device=DEV) for _ in shapes]
+    torch.cuda.synchronize()
+    try:
+        for rep in range(10):
+            got = [torch.full_like(w, float("nan")) for w in want]
+            for i, (M, N, K) in enumerate(shapes):
+                tl.set_workspace(ws[i])
+                for _ in range(3):                                       # keep both streams busy at the same time
+                    tl.gemm(A[i], Bt[i], got[i], M, N, K, 4096, 16, 128, stream=streams[i])
+            torch.cuda.synchronize()
+            for g, w in zip(got, want):
+                assert torch.equal(g, w)
+    finally:
+        tl.set_workspace(None)
+    tl.device_status()
