@@ -102,6 +102,7 @@ struct TileInfo {
     int row0;        // first row of A / C
     int rows;        // valid rows (<= BM)
     int expert;
+    int flip;        // odd m-tile of its (expert, n-tile): walks K backwards (see decode_tile)
 };
 
 // ------------------------------------------------------------------ scheduler
@@ -187,6 +188,10 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* 
     t.expert = e;
     t.n0 = (local / mt) * p.BN;
     t.row0 = row_begin + (local % mt) * p.BM;
+    // The m-tiles of one (expert, n-tile) follow each other in the tile order and read the same weight slab.  Odd
+    // ones walk K from the far end, so that what the even one before them read last is read again first, while it
+    // is still in L2.
+    t.flip = (local % mt) & 1;
     t.rows = row_end - t.row0 < p.BM ? row_end - t.row0 : p.BM;
     return t;
 }
@@ -479,7 +484,8 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     uint8_t* sw = stages + size_t(stage) * stage_bytes;
                     uint8_t* sa = sw + kWBytes;
                     mbar_arrive_expect_tx(&full_bar[stage], tx);
-                    const int k0 = (kit * kBK) << p.k_shift;        // first K element of the stage
+                    const int kq = t.flip ? p.k_iters - 1 - kit : kit;
+                    const int k0 = (kq * kBK) << p.k_shift;         // first K element of the stage
 #pragma unroll
                     for (int sub = 0; sub < kSubK; ++sub)
                         tma_load_2d(sa + size_t(sub) * p.a_rows * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
@@ -620,9 +626,10 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                     break;
                 }
                 uint8_t* sw = stages + size_t(stage) * stage_bytes;
-                const int kblk0 = (kit * kBK) >> p.br_log2;
+                const int kq = t.flip ? p.k_iters - 1 - kit : kit;
+                const int kblk0 = (kq * kBK) >> p.br_log2;
                 const uint8_t* src0 = Bexp + (int64_t(kblk0) * p.blocks_per_row + nblk0) * G;
-                const int k_rows_left = p.K - kit * kBK, n_cols_left = p.N - t.n0;
+                const int k_rows_left = p.K - kq * kBK, n_cols_left = p.N - t.n0;
                 const int64_t krow_stride = int64_t(p.blocks_per_row) * G;      // bytes between runs of tiles
                 switch (pieces) {
                     case 1: generic_fill_stage<kBK, kBN, 1>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
