@@ -24,6 +24,10 @@
  *     found on the host before anything is enqueued.  A device-side wait that
  *     ran out (every wait in the kernels is bounded) raises a flag that
  *     tl_device_status() reports after synchronising.
+ *   - Threads.  Host threads may call concurrently (the library serialises its own host-side work).  The stream
+ *     and the workspace set by tl_set_stream() / tl_set_workspace() belong to the calling thread, like CUDA's
+ *     current device; the internal split-K workspace belongs to the device, so calls that can run at the same
+ *     time on one GPU (two streams, two threads) must each bring their own workspace.
  *   - Divisibility (Section 3.3): rows % block_rows == 0 and
  *     cols % block_cols == 0, otherwise TL_ERR_INVALID_ARG; the caller pads.
  *     block_rows and block_cols must be powers of two (Section 3.2), otherwise
@@ -60,12 +64,43 @@ typedef enum { TL_LAYOUT_ROW_MAJOR = 0, TL_LAYOUT_COL_MAJOR = 1, TL_LAYOUT_TILE_
 const char* tl_status_string(int status);
 /* Last cudaError_t / CUresult seen by a call that returned TL_ERR_CUDA (0 if none). */
 int tl_last_cuda_error(void);
-/* Stream used by the calls that take none (tl_relayout, tl_read_amp*).  Default: NULL stream. */
+/* Stream used by the calling thread's calls that take none (tl_relayout, tl_read_amp*).  Default: NULL stream. */
 int tl_set_stream(void* cuda_stream);
 /* Synchronises the device, then returns TL_ERR_TIMEOUT if any kernel since the
  * last call gave up on a bounded wait (and clears the flag), else TL_OK.
  * *detail (may be NULL) receives a code saying which wait expired. */
 int tl_device_status(uint32_t* detail);
+
+/*
+ * Switches of the library, process-wide.  None changes a result; they select between code paths that compute the
+ * same thing (for measurement, and so that tests can reach every path), bound the device-side waits, or arm the
+ * test hook below.  The paper has no counterpart.  Initial values may be preset through environment variables of the
+ * names given in brackets (read once).
+ */
+typedef enum {
+    TL_OPT_PDL = 0,          /* 1 (default): launches use programmatic stream serialisation, 0: plain stream order [TL_NO_PDL=1] */
+    TL_OPT_PREFETCH_STAGES,  /* weight stages a GEMM CTA asks into L2 before it waits for its predecessor; -1 (default): up to 4 [TL_PREFETCH_STAGES] */
+    TL_OPT_PAIR_KERNEL,      /* 1 (default): large dense products run on CTA pairs, 0: single-CTA kernel [TL_NO_PAIR=1] */
+    TL_OPT_PAIR_512,         /* 1 (default): the pair kernel uses 512-token tiles where they fill whole waves, 0: 256-token tiles [TL_PAIR_HALVES=1] */
+    TL_OPT_BOX_PER_BLOCK,    /* 0 (default): one TMA box per pipeline stage, 1: one box per memory tile [TL_BOX_PER_BLOCK] */
+    TL_OPT_MAX_STAGES,       /* 0 (default): as many pipeline stages as fit, n >= 2: at most n [TL_MAX_STAGES] */
+    TL_OPT_UMMA_M128,        /* 0 (default): 64-row MMAs for tiles of up to 64 tokens, 1: always 128 rows [TL_UMMA_M128] */
+    TL_OPT_RELAYOUT_TMA,     /* 1 (default): copy-engine relayout where the shape allows, 0: shared-memory kernel [TL_RELAYOUT_NO_TMA=1] */
+    TL_OPT_LOG,              /* 1: every GEMM launch prints the plan it chose to stderr [TL_LOG] */
+    TL_OPT_WAIT_LIMIT_US,    /* bound of every device-side barrier wait, microseconds; default 2 000 000, accepted 100 .. 60 000 000 */
+    TL_OPT_STALL_ONCE,       /* test hook: 1 = the next tl_gemm* launch, 2 = the next copy-engine relayout launch arms the
+                                first pipeline stage of every CTA for 16 bytes more than its copies deliver, so that
+                                the wait on that stage runs out after TL_OPT_WAIT_LIMIT_US, the kernel gives up (drains
+                                its copies, frees tensor memory, returns) and tl_device_status() reports TL_ERR_TIMEOUT.
+                                That launch's output is undefined.  The option resets itself to 0 when it is consumed. */
+    TL_OPT_MOE_ROW_CAP,      /* grouped products: most token rows per tile; 0 (default): the library's choice, else 16/32/64/128 */
+    TL_OPT_REDUCE_SPLIT,     /* 1 (default): a split tile's partial sums are added by all reduction CTAs inside it, 0: by one */
+    TL_OPT_COUNT_
+} tl_option;
+/* TL_ERR_INVALID_ARG for an unknown option or a value outside the option's range. */
+int tl_set_option(int option, int64_t value);
+/* Current value; -1 for an unknown option. */
+int64_t tl_get_option(int option);
 
 /* -------------------------------------------------------------- relayout */
 
@@ -118,7 +153,9 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
  *                cta_m in {16, 32, 64, 128, 256} (cta_n == 256: at most 128).
  *                Tiles may overhang M, N and K.
  *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,
- *   N % block_cols == 0; row-major: N % 64 == 0.
+ *   N % block_cols == 0; row-major: N % 64 == 0.  N % 4 == 0 (C is written in
+ *   16-byte vectors; only the hand-addressed memory tiles of one or two
+ *   columns could ask for less), else TL_ERR_UNSUPPORTED.
  *   Memory tiles whose rows are at least 32 bytes (16 columns) are read by
  *   TMA, whatever their height.  Narrower ones (block rows down to 2 bytes)
  *   are read by the generic-address path of Section 4.4 (plain loads with
@@ -216,11 +253,41 @@ int tl_gemm_grouped_fp8_kmajor(const void* d_A_sorted_fp8, const void* d_B_exper
                                int64_t N, int64_t K, int64_t G, int tile_n, int tile_k,
                                int cta_m, int cta_n, int cta_k, void* cuda_stream);
 
-/* Bytes of workspace tl_gemm / tl_gemm_grouped may need for these sizes on the current device. */
+/* Bytes of workspace tl_gemm, or tl_gemm_grouped with any number of experts and M rows in total, may need for
+ * these sizes on the current device (an upper bound: the grouped schedule of many experts cuts K over every SM). */
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k);
-/* Hands the library a caller-owned device workspace (256-byte aligned); (NULL, 0) returns to the
- * internal one.  The buffer must stay valid until the last call using it has finished. */
+/* Hands the library a caller-owned device workspace (256-byte aligned) for the CALLING THREAD's GEMM calls;
+ * (NULL, 0) returns to the device's internal one.  The buffer must stay valid until the last call using it has
+ * finished. */
 int tl_set_workspace(void* d_ptr, size_t bytes);
+
+/*
+ * The schedule a GEMM call with these sizes runs on the current device: the CTA grid of Section 2.3 as this
+ * library cuts it.  Host-only; no pointer is needed and nothing is enqueued.  The same code chooses the plan of a
+ * real launch, so feeding tl_read_amp* with (cta_m, cta_n, cta_k) from here counts exactly the tile loads the
+ * kernel issues (Sections 2.5, 6.5).  E == 0: dense (tl_gemm*); E >= 1: grouped with E experts and M rows in
+ * total.  flavour 0: N-contiguous bf16 weights (tl_gemm), 1: K-contiguous bf16 (tl_gemm_kmajor: block_rows =
+ * tile_n, block_cols = tile_k), 2: K-contiguous FP8 (tl_gemm_fp8_kmajor).  Errors as the GEMM call itself
+ * would return them for these sizes.
+ */
+typedef struct tl_gemm_plan_info {
+    int32_t cta_m, cta_n, cta_k;   /* token rows x weight columns of one CTA's tile, weight rows (K elements) per stage.
+                                      CTA-pair kernel: each CTA of a pair owns 128 of the pair's 256 columns and loads them
+                                      once per tile of cta_m = 512 (or 256) token rows */
+    int32_t pair_kernel;           /* 1: CTA pairs (cta_group::2), 0: single-CTA kernel */
+    int32_t stream_k;              /* 1: K ranges cut over the CTAs + reduction kernel; 0: whole tiles */
+    int32_t grid;                  /* CTAs launched */
+    int32_t stages;                /* pipeline depth */
+    int32_t weights_on_n;          /* 1: weights on the N side of the MMA (token tiles of up to 128 rows) */
+    int32_t generic_path;          /* 1: weights loaded by the generic-address path of Section 4.4 */
+    int32_t reserved;
+    int64_t pair_tiles_512, pair_tiles_256;   /* pair kernel: tiles of 512 and of 256 token rows (x 256 columns) */
+    uint64_t workspace_bytes;      /* split-K scratch the launch uses */
+} tl_gemm_plan_info;
+int tl_gemm_plan(int64_t M, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,
+                 int cta_m, int cta_n, int cta_k, int E, int flavour, tl_gemm_plan_info* out);
+/* What the calling thread's most recent GEMM launch ran (zeros before the first). */
+int tl_gemm_last_plan(tl_gemm_plan_info* out);
 
 /*
  * End-to-end form with host buffers: copies A and the ROW-MAJOR weight to the
@@ -258,11 +325,12 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
  *                 the kernel expires; NULL keeps the flag in the array, unread.
  *   limit         problems whose split-K scratch exceeds the array return
  *                 TL_ERR_WORKSPACE and enqueue nothing.  The scratch is
- *                 2 * (number of SMs) * cta_m * cta_n * 4 bytes when
- *                 M <= 64 or the tiles do not fill the SMs evenly, else 0; the
- *                 default tile here is 128 columns wide: on a 148-SM B200
- *                 that admits every M <= 32; M in (32, 64] needs 9.3 MB and
- *                 is refused.
+ *                 2 * (number of SMs) * cta_m * cta_n * 4 bytes when the
+ *                 output tiles do not fill the SMs evenly (fewer tiles than
+ *                 SMs, or a last wave less than 92 % full), else 0; products
+ *                 that run on CTA pairs need none.  The default tile here is
+ *                 128 columns wide: on a 148-SM B200 that admits every
+ *                 M <= 32; M in (32, 64] needs 9.3 MB and is refused.
  *   first call    the first call on each device looks up the array's device
  *                 address (with that device current).  Make that call before
  *                 starting any stream capture.

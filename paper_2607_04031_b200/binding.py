@@ -26,6 +26,10 @@ _SIGNATURES = {
     "tl_last_cuda_error": (_int, []),
     "tl_set_stream": (_int, [_vp]),
     "tl_device_status": (_int, [ctypes.POINTER(ctypes.c_uint32)]),
+    "tl_set_option": (_int, [_int, _i64]),
+    "tl_get_option": (_i64, [_int]),
+    "tl_gemm_plan": (_int, [_i64, _i64, _i64, _i64, _int, _int, _int, _int, _int, _int, _int, _vp]),
+    "tl_gemm_last_plan": (_int, [_vp]),
     "tl_relayout": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int]),
     "tl_relayout_on": (_int, [_vp, _vp, _i64, _i64, _int, _i64, _int, _int, _int, _vp]),
     "tl_relayout_batch": (_int, [_int, _vp, _vp, _vp, _vp, _int, _i64, _int, _int, _int, _vp]),
@@ -58,6 +62,11 @@ _SIGNATURES = {
                                    _u64p, _u64p, _u64p]),
     "tl_read_amp_per_cta": (_int, [_i64, _i64, _i64, _int, _int, _int, _int, _i64, _int, _int, _int, _vp, _vp, _vp]),
 }
+
+# tl_option
+(OPT_PDL, OPT_PREFETCH_STAGES, OPT_PAIR_KERNEL, OPT_PAIR_512, OPT_BOX_PER_BLOCK, OPT_MAX_STAGES, OPT_UMMA_M128,
+ OPT_RELAYOUT_TMA, OPT_LOG, OPT_WAIT_LIMIT_US, OPT_STALL_ONCE, OPT_MOE_ROW_CAP, OPT_REDUCE_SPLIT) = range(13)
+FLAVOUR_N_BF16, FLAVOUR_K_BF16, FLAVOUR_K_FP8 = 0, 1, 2
 
 _lib = None
 
@@ -124,6 +133,62 @@ def device_status():
     st = lib().tl_device_status(ctypes.byref(detail))
     if st != TL_OK:
         raise TileLensError(st, f"tl_device_status detail=0x{detail.value:x}")
+
+
+def set_option(option: int, value: int):
+    _check(lib().tl_set_option(option, value), "tl_set_option")
+
+
+def get_option(option: int) -> int:
+    return int(lib().tl_get_option(option))
+
+
+class option:
+    """with option(OPT_x, v): ... sets a library switch for the block and restores the previous value afterwards."""
+
+    def __init__(self, opt: int, value: int):
+        self.opt, self.value = opt, value
+
+    def __enter__(self):
+        self.old = get_option(self.opt)
+        set_option(self.opt, self.value)
+        return self
+
+    def __exit__(self, *exc):
+        set_option(self.opt, self.old)
+        return False
+
+
+class GemmPlan(ctypes.Structure):
+    """tl_gemm_plan_info"""
+    _fields_ = [("cta_m", ctypes.c_int32), ("cta_n", ctypes.c_int32), ("cta_k", ctypes.c_int32),
+                ("pair_kernel", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("grid", ctypes.c_int32),
+                ("stages", ctypes.c_int32), ("weights_on_n", ctypes.c_int32), ("generic_path", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("pair_tiles_512", ctypes.c_int64), ("pair_tiles_256", ctypes.c_int64),
+                ("workspace_bytes", ctypes.c_uint64)]
+
+    def as_dict(self):
+        return {name: int(getattr(self, name)) for name, _ in self._fields_ if name != "reserved"}
+
+    @property
+    def cta(self):
+        return (int(self.cta_m), int(self.cta_n), int(self.cta_k))
+
+
+def gemm_plan(M: int, N: int, K: int, G: int = 4096, block_rows: int = 16, block_cols: int = 128, cta=(0, 0, 0),
+              E: int = 0, flavour: int = FLAVOUR_N_BF16) -> GemmPlan:
+    """The schedule a GEMM call with these sizes runs (host only, nothing is enqueued)."""
+    out = GemmPlan()
+    _check(lib().tl_gemm_plan(M, N, K, G, block_rows, block_cols, cta[0], cta[1], cta[2], E, flavour,
+                              ctypes.addressof(out)), "tl_gemm_plan")
+    return out
+
+
+def gemm_last_plan() -> GemmPlan:
+    """What this thread's most recent GEMM launch ran."""
+    out = GemmPlan()
+    _check(lib().tl_gemm_last_plan(ctypes.addressof(out)), "tl_gemm_last_plan")
+    return out
 
 
 def relayout(src: torch.Tensor, dst: torch.Tensor, rows: int, cols: int, elem_bytes: int, G: int,

@@ -23,20 +23,29 @@ def needs_build() -> bool:
     return os.path.getmtime(LIB) < max(os.path.getmtime(d) for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB
+def build(force: bool = False, verbose: bool = False, defines=(), lib: str = LIB) -> str:
+    """Compiles every source to an object file (in parallel, one nvcc per file) and links the shared library."""
+    if not force and lib == LIB and not needs_build():
+        return lib
+    from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = f"{LIB}.{os.getpid()}.tmp"
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", tmp] + sources()
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
+             "-I", os.path.join(ROOT, "include"), "-I", CSRC] + [f"-D{d}" for d in defines]
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+        flags += ["-Xptxas", "-v"]
+    objdir = os.path.join(HERE, "build", os.path.basename(lib) + f".{os.getpid()}")
+    os.makedirs(objdir, exist_ok=True)
+    srcs = sources()
+    objs = [os.path.join(objdir, os.path.basename(s)[:-3] + ".o") for s in srcs]
+    with ThreadPoolExecutor(max_workers=len(srcs)) as pool:
+        list(pool.map(lambda so: subprocess.check_call([nvcc] + flags + ["-c", so[0], "-o", so[1]]), zip(srcs, objs)))
+    tmp = f"{lib}.{os.getpid()}.tmp"
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs)
+    os.replace(tmp, lib)
+    for o in objs:
+        os.remove(o)
+    os.rmdir(objdir)
+    return lib
 
 
 if __name__ == "__main__":

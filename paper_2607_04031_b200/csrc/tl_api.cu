@@ -1,35 +1,103 @@
-// Host-side state of the tilelens library: stream, workspace, control block, error reporting.
+// Host-side state of the tilelens library: per-device control block and workspace, per-thread stream and caller
+// workspace, the process-wide option table, error reporting.
 #include "tl_common.cuh"
 
+#include <cstdlib>
+#include <mutex>
 
 namespace tl {
 
-State& state() {
-    static State s;
-    return s;
+namespace {
+
+std::recursive_mutex& api_mutex() {
+    static std::recursive_mutex m;
+    return m;
+}
+
+struct Options {
+    int64_t v[TL_OPT_COUNT_];
+    Options() {
+        set_defaults();
+        // Initial values may come from the environment (read once, when the library is first used), so that a
+        // measurement script can flip a switch without touching the program it runs.
+        static const struct { const char* name; int id; int invert; } env[] = {
+            {"TL_NO_PDL", TL_OPT_PDL, 1},           {"TL_PREFETCH_STAGES", TL_OPT_PREFETCH_STAGES, 0},
+            {"TL_NO_PAIR", TL_OPT_PAIR_KERNEL, 1},  {"TL_BOX_PER_BLOCK", TL_OPT_BOX_PER_BLOCK, 0},
+            {"TL_MAX_STAGES", TL_OPT_MAX_STAGES, 0}, {"TL_UMMA_M128", TL_OPT_UMMA_M128, 0},
+            {"TL_RELAYOUT_NO_TMA", TL_OPT_RELAYOUT_TMA, 1}, {"TL_LOG", TL_OPT_LOG, 0},
+        };
+        for (const auto& e : env)
+            if (const char* s = getenv(e.name)) v[e.id] = e.invert ? (atoi(s) != 0 ? 0 : 1) : atoi(s);
+        if (const char* s = getenv("TL_PAIR_HALVES")) v[TL_OPT_PAIR_512] = atoi(s) == 1 ? 0 : 1;
+    }
+    void set_defaults() {
+        for (auto& x : v) x = 0;
+        v[TL_OPT_PDL] = 1;
+        v[TL_OPT_PREFETCH_STAGES] = -1;
+        v[TL_OPT_PAIR_KERNEL] = 1;
+        v[TL_OPT_PAIR_512] = 1;
+        v[TL_OPT_RELAYOUT_TMA] = 1;
+        v[TL_OPT_WAIT_LIMIT_US] = 2000000;
+        v[TL_OPT_MOE_ROW_CAP] = 0;
+        v[TL_OPT_REDUCE_SPLIT] = 1;
+    }
+};
+
+Options& options() {
+    static Options o;
+    return o;
+}
+
+DeviceState g_devices[kMaxDevices];
+
+}  // namespace
+
+ApiLock::ApiLock() { api_mutex().lock(); }
+ApiLock::~ApiLock() { api_mutex().unlock(); }
+
+ThreadState& tls() {
+    static thread_local ThreadState t;
+    return t;
+}
+
+DeviceState& dev() {
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) {
+        (void)cudaGetLastError();
+        d = 0;
+    }
+    return g_devices[d];
+}
+
+int64_t opt(int option) { return option >= 0 && option < TL_OPT_COUNT_ ? options().v[option] : 0; }
+
+uint64_t wait_limit_ns() {
+    const int64_t us = opt(TL_OPT_WAIT_LIMIT_US);
+    return uint64_t(us > 0 ? us : 1) * 1000ull;
 }
 
 int check_cuda(cudaError_t err) {
     if (err == cudaSuccess) return TL_OK;
-    state().last_cuda_error = static_cast<int>(err);
+    tls().last_cuda_error = static_cast<int>(err);
     (void)cudaGetLastError();   // clear the sticky-less error so later calls start clean
     return TL_ERR_CUDA;
 }
 
 int ensure_device_info() {
-    State& s = state();
-    int dev = -1;
-    if (int rc = check_cuda(cudaGetDevice(&dev))) return rc;
-    if (dev == s.device && s.sm_count > 0) return TL_OK;
+    int d = -1;
+    if (int rc = check_cuda(cudaGetDevice(&d))) return rc;
+    if (d < 0 || d >= kMaxDevices) return TL_ERR_UNSUPPORTED;
+    DeviceState& s = g_devices[d];
+    if (s.sm_count > 0) return TL_OK;
     int sms = 0;
-    if (int rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return rc;
-    s.device = dev;
+    if (int rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, d))) return rc;
     s.sm_count = sms;
     return TL_OK;
 }
 
 int ensure_control() {
-    State& s = state();
+    if (int rc = ensure_device_info()) return rc;
+    DeviceState& s = dev();
     if (s.ctl.d_status) return TL_OK;
     void* p = nullptr;
     if (int rc = check_cuda(cudaMalloc(&p, 1024))) return rc;
@@ -45,17 +113,27 @@ int ensure_control() {
     return TL_OK;
 }
 
+int ensure_smem_attr(const void* kernel, int bytes) {
+    DeviceState& s = dev();
+    for (int i = 0; i < s.smem_attr_n; ++i)
+        if (s.smem_attr_done[i] == kernel) return TL_OK;
+    if (int rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes))) return rc;
+    if (s.smem_attr_n < int(sizeof(s.smem_attr_done) / sizeof(s.smem_attr_done[0]))) s.smem_attr_done[s.smem_attr_n++] = kernel;
+    return TL_OK;
+}
+
 int get_workspace(size_t bytes, void** out) {
-    State& s = state();
     if (bytes == 0) {
         *out = nullptr;
         return TL_OK;
     }
-    if (s.user_ws) {
-        if (s.user_ws_bytes < bytes) return TL_ERR_WORKSPACE;
-        *out = s.user_ws;
+    ThreadState& t = tls();
+    if (t.user_ws) {
+        if (t.user_ws_bytes < bytes) return TL_ERR_WORKSPACE;
+        *out = t.user_ws;
         return TL_OK;
     }
+    DeviceState& s = dev();
     if (s.own_ws_bytes < bytes) {
         // Work already enqueued may still use the old buffer: wait before replacing it.
         if (s.own_ws) {
@@ -91,34 +169,56 @@ const char* tl_status_string(int status) {
     }
 }
 
-int tl_last_cuda_error(void) { return tl::state().last_cuda_error; }
+int tl_last_cuda_error(void) { return tl::tls().last_cuda_error; }
 
 int tl_set_stream(void* cuda_stream) {
-    tl::state().stream = static_cast<cudaStream_t>(cuda_stream);
+    tl::tls().stream = static_cast<cudaStream_t>(cuda_stream);
     return TL_OK;
 }
 
 int tl_set_workspace(void* d_ptr, size_t bytes) {
-    tl::State& s = tl::state();
+    tl::ThreadState& t = tl::tls();
     if (d_ptr == nullptr) {
-        s.user_ws = nullptr;
-        s.user_ws_bytes = 0;
+        t.user_ws = nullptr;
+        t.user_ws_bytes = 0;
         return TL_OK;
     }
     if (reinterpret_cast<uintptr_t>(d_ptr) % 256 != 0) return TL_ERR_ALIGNMENT;
-    s.user_ws = d_ptr;
-    s.user_ws_bytes = bytes;
+    t.user_ws = d_ptr;
+    t.user_ws_bytes = bytes;
     return TL_OK;
 }
 
+int tl_set_option(int option, int64_t value) {
+    tl::ApiLock lock;
+    if (option < 0 || option >= TL_OPT_COUNT_) return TL_ERR_INVALID_ARG;
+    switch (option) {
+        case TL_OPT_PREFETCH_STAGES: if (value < -1 || value > 16) return TL_ERR_INVALID_ARG; break;
+        case TL_OPT_MAX_STAGES: if (value != 0 && (value < 2 || value > 16)) return TL_ERR_INVALID_ARG; break;
+        case TL_OPT_WAIT_LIMIT_US: if (value < 100 || value > 60000000) return TL_ERR_INVALID_ARG; break;
+        case TL_OPT_STALL_ONCE: if (value < 0 || value > 2) return TL_ERR_INVALID_ARG; break;
+        case TL_OPT_MOE_ROW_CAP: if (value != 0 && value != 16 && value != 32 && value != 64 && value != 128) return TL_ERR_INVALID_ARG; break;
+        default: if (value != 0 && value != 1) return TL_ERR_INVALID_ARG; break;
+    }
+    tl::options().v[option] = value;
+    return TL_OK;
+}
+
+int64_t tl_get_option(int option) {
+    tl::ApiLock lock;
+    if (option < 0 || option >= TL_OPT_COUNT_) return -1;
+    return tl::options().v[option];
+}
+
 int tl_device_status(uint32_t* detail) {
+    tl::ApiLock lock;
     if (int rc = tl::ensure_control()) return rc;
     if (int rc = tl::check_cuda(cudaDeviceSynchronize())) return rc;
     uint32_t word = 0;
-    if (int rc = tl::check_cuda(cudaMemcpy(&word, tl::state().ctl.d_status, 4, cudaMemcpyDeviceToHost))) return rc;
+    if (int rc = tl::check_cuda(cudaMemcpy(&word, tl::dev().ctl.d_status, 4, cudaMemcpyDeviceToHost))) return rc;
     if (detail) *detail = word;
     if (word == 0) return TL_OK;
-    if (int rc = tl::check_cuda(cudaMemset(tl::state().ctl.d_status, 0, 4))) return rc;
+    if (int rc = tl::check_cuda(cudaMemset(tl::dev().ctl.d_status, 0, 4))) return rc;
     return TL_ERR_TIMEOUT;
 }
 

@@ -15,8 +15,18 @@
 namespace tl {
 
 // ---------------------------------------------------------------- host state
+//
+// Three kinds of state, all private to the library:
+//   per device   control block, internal split-K workspace, SM count and what was already configured there;
+//   per thread   the stream and the caller's workspace set by tl_set_stream / tl_set_workspace, the last CUDA error;
+//   per process  the option table (tl_set_option) and the tensor-map cache.
+// Every entry point takes one process-wide lock (ApiLock) for its host-side work, so host threads may call
+// concurrently; what they enqueue runs concurrently on the GPU only if the caller gave each its own stream and
+// workspace.
 
-// Device control block (lazily allocated, one per process):
+constexpr int kMaxDevices = 64;
+
+// Device control block (lazily allocated, one per device):
 //   word 0      : timeout flag / detail code written by kernels whose bounded wait expired
 //   bytes 64..  : 17 sets of three uint64 accumulators and a ticket counter of the read-amplification kernel
 struct Control {
@@ -27,25 +37,46 @@ struct Control {
     unsigned long long* h_acc_dev = nullptr;   // device-side address of h_acc
 };
 
-struct State {
+struct DeviceState {
+    Control ctl;
+    void* own_ws = nullptr;              // split-K workspace grown on demand (shared by every thread using the device)
+    size_t own_ws_bytes = 0;
+    int sm_count = 0;
+    int pair_max_clusters = -1;          // co-resident clusters of the CTA-pair kernel (queried once)
+    const void* smem_attr_done[64] = {}; // kernels whose dynamic shared-memory limit was raised on this device
+    int smem_attr_n = 0;
+};
+
+struct ThreadState {
     cudaStream_t stream = nullptr;       // tl_set_stream
     int last_cuda_error = 0;
     void* user_ws = nullptr;             // tl_set_workspace
     size_t user_ws_bytes = 0;
-    void* own_ws = nullptr;              // grown on demand
-    size_t own_ws_bytes = 0;
-    Control ctl;
-    int sm_count = 0;
-    int device = -1;
 };
 
-State& state();
+ThreadState& tls();
+// State of the calling thread's current CUDA device (slot 0 when the device cannot be queried).
+DeviceState& dev();
+// Value of a tl_option (see tilelens.h).
+int64_t opt(int option);
+
+struct ApiLock {
+    ApiLock();
+    ~ApiLock();
+    ApiLock(const ApiLock&) = delete;
+    ApiLock& operator=(const ApiLock&) = delete;
+};
+
 // Records err and returns TL_ERR_CUDA when err != cudaSuccess, else TL_OK.
 int check_cuda(cudaError_t err);
-int ensure_control();                    // allocates the control block once
+int ensure_control();                    // allocates the current device's control block once
 int ensure_device_info();
-// Workspace of at least `bytes` (user's if set, else internal, grown with cudaMalloc).
+// Raises the dynamic shared-memory limit of `kernel` on the current device, once per (device, kernel).
+int ensure_smem_attr(const void* kernel, int bytes);
+// Workspace of at least `bytes` (the calling thread's if set, else the device's internal one, grown with cudaMalloc).
 int get_workspace(size_t bytes, void** out);
+// Wait limit of the kernels' bounded waits, nanoseconds (TL_OPT_WAIT_LIMIT_US).
+uint64_t wait_limit_ns();
 
 // Encodes (and caches) a tiled tensor map; dtype / swizzle are CUtensorMapDataType / CUtensorMapSwizzle values,
 // strides_bytes[0] is the element size and is not passed to the driver.
@@ -104,10 +135,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait: polls the barrier; every 2048 failed polls it looks at the
 // wall clock and at the CTA's abort word.  Returns false when the wait was
-// abandoned (2 s without progress, or another role already gave up); the
+// abandoned (limit_ns without progress, or another role already gave up); the
 // caller must then leave its loop.  `abort_flag` is a shared-memory word.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                                  uint32_t* g_status, uint32_t code) {
+                                                  uint32_t* g_status, uint32_t code, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     uint32_t polls = 0;
@@ -117,7 +148,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
             if (*abort_flag) return false;
             uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > 2000000000ull) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(g_status, 0u, code);
                 return false;

@@ -1,0 +1,731 @@
+// Device side of the tiled GEMM (included by the translation units that instantiate or launch it): parameters,
+// scheduler, helpers and the single-CTA kernel.  See tl_gemm.cu for the overview.
+#pragma once
+
+#include "tl_common.cuh"
+
+#include <cuda_bf16.h>
+
+namespace tl {
+
+constexpr int kGemmThreads = 192;          // TMA path: producer, MMA issuer, four epilogue warps
+constexpr int kGenericThreads = 320;       // generic-address path: four more warps that load the weights by hand
+constexpr int kMaxStages = 16;
+constexpr int kMaxExperts = 1024;
+constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 256 rows
+constexpr int kAtomBytes = 128;            // one swizzle row: 64 bf16
+constexpr int kMaxDynamicSmem = 227 * 1024 - 10 * 1024;   // 227 KB per CTA minus the kernel's static shared memory
+
+struct alignas(64) GemmParams {
+    CUtensorMap tmap_a[kNumBoxChoices];
+    CUtensorMap tmap_b;
+    float* C;
+    float* partials;            // stream-K partial tiles: slot = BM x BN floats
+    const int32_t* offsets;     // grouped: device E+1 row offsets; dense: nullptr
+    uint32_t* status;
+    uint64_t wait_limit_ns;     // bound of every barrier wait in the kernel
+    uint32_t stall_extra_tx;    // test hook: bytes added to what the first stage's barrier expects (0 in normal use)
+    int reduce_split;           // stream-K reduction: 1 = every boundary inside a split tile sums a share of it
+    int64_t ldc;                // N
+    int M;                      // dense rows (grouped: total rows)
+    int N, K, E;
+    int BM;                     // token rows per CTA tile: 16, 32, 64, 128 or 256
+    int umma_m;                 // weights-on-N kernels: rows of the MMA's token side, 64 when BM <= 64, else 128
+    int a_rows;                 // token rows a stage holds per 64-wide K slice: max(BM, umma_m) there, else BM; rows
+                                // beyond BM are zeroed once and never written again
+    int BN;                     // weight columns per CTA tile: 128 or 256
+    int n_tiles, k_iters;
+    int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
+    int num_stages;
+    int prefetch_stages;        // stages of weights each CTA asks into L2 before it waits for its predecessor
+    int pair_big_tiles;         // pair kernel with 512-token tiles: how many tiles are of that size (the rest 256)
+    // Gated epilogue (expert FFN): weight columns 2j / 2j+1 hold gate_j / up_j; H[row][j] = bf16(silu(g) * u)
+    // replaces C.  Weights-on-N kernels only.
+    int epi_swiglu;
+    __nv_bfloat16* H;
+    int64_t ldh;
+    __nv_bfloat16* Cb;          // non-null: C is written as bf16 (one rounding to nearest even) instead of fp32
+    // weight-operand geometry
+    int row_major;              // 1: the weight is not tiled ([K][N] row-major, or [N][K] when w_kmajor)
+    int w_kmajor;               // 1: weights stored [N][K], K contiguous (Eq. 2 as printed): K-major MMA operand
+    int k_inner;                // 1: tensor-map dimensions ordered (64, row in tile, tile along K, atom, tile along N)
+    // Tensor-map coordinates 1..4 of a weight box as shifts and masks of its first K element k and weight column n:
+    // c[i] = ((k >> ck_shift[i]) & ck_mask[i]) + ((n >> cn_shift[i]) & cn_mask[i]) + c_expert[i] * (expert offset).
+    // (Set by the host for the layout at hand: the producer's loop has no layout branches.)
+    int ck_shift[4], ck_mask[4], cn_shift[4], cn_mask[4], c_expert[4];
+    int fp8;                    // 1: both operands are 8-bit floating point (E4M3); needs w_kmajor
+    int k_shift;                // log2(K elements per 2 bytes): a stage holds (BK << k_shift) K-elements
+    int w_atom_log2;            // K-major weights: log2(elements in one swizzle row of 128, 64 or 32 bytes)
+    uint64_t w_desc_hi;         // weight operand's shared-memory descriptor without its start address
+    int br_log2, bc_log2;       // memory tile: rows x contiguous columns of the stored matrix (tiled layouts only)
+    int k_coord_per_expert;     // added per expert to the coordinate of the stacked dimension (blocks or rows)
+    int box_rows, box_atoms;    // rows and 128-byte atoms of one box
+    int kbx, nbx;               // boxes per stage along K and along N
+    uint32_t box_bytes;
+    uint32_t lbo, sbo;          // descriptor strides of the weight operand, bytes
+    uint32_t ugroup_off;        // bytes between the 128-column groups of a 256-column tile
+    uint32_t kstep_off[8];      // byte offset of each 16-row K step inside a stage
+    // generic-address path (Section 4.4: memory tiles that TMA cannot box)
+    int generic_b;              // 1: warps 6..9 load the weights with Eq. 1-2 address arithmetic
+    const uint8_t* B;           // raw weight pointer (generic path only)
+    int64_t expert_bytes;       // K*N*2
+    int blocks_per_row;         // N / bc
+};
+
+struct TileInfo {
+    int n0;          // first weight column
+    int row0;        // first row of A / C
+    int rows;        // valid rows (<= BM)
+    int expert;
+    int flip;        // odd m-tile of its (expert, n-tile): walks K backwards (see decode_tile)
+};
+
+// ------------------------------------------------------------------ scheduler
+struct Work {
+    int tile, kbeg, kend;
+};
+
+constexpr int kRangeTabMax = 256;      // CTAs whose range starts are tabulated in shared memory
+
+struct Sched {
+    int stream_k, k_iters, tiles_total, grid_eff, cta;
+    int next_tile;
+    long long it, it_end, it_begin;
+    const int* tab;     // tab[c] = first flattened iteration of CTA c (grid_eff + 1 entries), or nullptr
+
+    // Even split of the flattened (tile, K iteration) space; a fixed function of the CTA index.
+    __device__ static long long split(long long total, int grid_eff, int c) { return (total * c) / grid_eff; }
+    __device__ long long range_begin(int c) const {
+        return tab ? tab[c] : split(static_cast<long long>(tiles_total) * k_iters, grid_eff, c);
+    }
+    __device__ static int effective_grid(long long total, int grid) { return total < grid ? static_cast<int>(total) : grid; }
+    __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid, int cta_, const int* tab_) {
+        stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_; tab = tab_;
+        grid_eff = effective_grid(static_cast<long long>(tiles_total) * k_iters, grid);
+        next_tile = cta;
+        if (grid_eff == 0 || cta >= grid_eff) { it = it_end = it_begin = 0; next_tile = tiles_total; return; }
+        it_begin = it = range_begin(cta);
+        it_end = range_begin(cta + 1);
+    }
+    __device__ bool next(Work& w) {
+        if (!stream_k) {
+            if (next_tile >= tiles_total) return false;
+            w.tile = next_tile; w.kbeg = 0; w.kend = k_iters;
+            next_tile += gridDim.x;
+            return true;
+        }
+        if (it >= it_end) return false;
+        int t = static_cast<int>(it / k_iters);
+        int kb = static_cast<int>(it - static_cast<long long>(t) * k_iters);
+        long long left = it_end - it;
+        int ke = (k_iters - kb) < left ? k_iters : kb + static_cast<int>(left);
+        w.tile = t; w.kbeg = kb; w.kend = ke;
+        it += ke - kb;
+        return true;
+    }
+    // CTA whose range holds flattened iteration x.
+    __device__ int owner(long long x) const {
+        if (tab) {                                   // largest c with tab[c] <= x
+            int lo = 0, hi = grid_eff;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (tab[mid] <= x) lo = mid; else hi = mid;
+            }
+            return lo;
+        }
+        long long total = static_cast<long long>(tiles_total) * k_iters;
+        int c = static_cast<int>(((x + 1) * grid_eff + total - 1) / total) - 1;
+        if (c < 0) c = 0;
+        if (c >= grid_eff) c = grid_eff - 1;
+        while (c > 0 && range_begin(c) > x) --c;
+        while (c + 1 < grid_eff && range_begin(c + 1) <= x) ++c;
+        return c;
+    }
+    // Partial-tile slot of CTA c for tile t: 2c when the tile is the first thing c works on, else 2c+1.
+    __device__ int slot(int c, int t) const {
+        return 2 * c + (range_begin(c) < static_cast<long long>(t) * k_iters ? 1 : 0);
+    }
+};
+
+__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* prefix, const int* row_start, int tile) {
+    // prefix[e] = tiles of experts before e; tiles of one expert: n-tile major, m-tile minor.
+    int lo = 0, hi = p.E;                  // find e with prefix[e] <= tile < prefix[e+1]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (prefix[mid] <= tile) lo = mid; else hi = mid;
+    }
+    const int e = lo;
+    const int local = tile - prefix[e];
+    const int mt = (prefix[e + 1] - prefix[e]) / p.n_tiles;
+    const int row_begin = row_start[e];
+    const int row_end = row_start[e + 1];
+    TileInfo t;
+    t.expert = e;
+    t.n0 = (local / mt) * p.BN;
+    t.row0 = row_begin + (local % mt) * p.BM;
+    // The m-tiles of one (expert, n-tile) follow each other in the tile order and read the same weight slab.  Odd
+    // ones walk K from the far end, so that what the even one before them read last is read again first, while it
+    // is still in L2.
+    t.flip = (local % mt) & 1;
+    t.rows = row_end - t.row0 < p.BM ? row_end - t.row0 : p.BM;
+    return t;
+}
+
+// Expert row offsets into shared memory (dense problems: one "expert" holding rows 0..M).
+__device__ __forceinline__ void load_row_starts(const GemmParams& p, int* row_start) {
+    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) row_start[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.M);
+}
+
+// prefix[e] = output tiles of the experts before e (n_tiles x m-tiles each); one warp, shuffle scan.
+__device__ __forceinline__ void tile_prefix(const GemmParams& p, const int* row_start, int* prefix) {
+    const int lane = threadIdx.x & 31;
+    int carry = 0;
+    for (int base = 0; base < p.E; base += 32) {
+        const int e = base + lane;
+        int v = 0;
+        if (e < p.E) v = ((row_start[e + 1] - row_start[e] + p.BM - 1) / p.BM) * p.n_tiles;
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (e < p.E) prefix[e] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) prefix[p.E] = carry;
+}
+
+// Shared-memory matrix descriptor: start address, leading and stride byte offsets in 16-byte units; descriptor
+// version 1 (bit 46); swizzle mode in bits 61..63: 2 = 128-byte, 4 = 64-byte, 6 = 32-byte.
+__host__ __device__ __forceinline__ uint64_t smem_desc_hi(uint32_t lbo, uint32_t sbo, uint32_t layout) {
+    return (uint64_t(lbo >> 4) << 16) | (uint64_t(sbo >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(layout) << 61);
+}
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return uint64_t((addr & 0x3FFFFu) >> 4) | smem_desc_hi(lbo, sbo, 2u);
+}
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint64_t hi) {
+    return uint64_t((addr & 0x3FFFFu) >> 4) | hi;
+}
+
+__device__ __forceinline__ void epilogue_bar_sync() {
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+// One warp fills one stage of weights on the generic-address path.  The stage is kBK/br runs of
+// kBN/bc whole memory tiles; run r starts at src0 + r*krow_stride and is kBN*br*2 contiguous bytes.
+// Chunks of 16 bytes are read in memory order, 16 loads in flight per lane; kPieces = rows held by one
+// chunk (1 when a block row is at least 16 bytes).  Rows >= k_rows_left and columns >= n_cols_left
+// (tile overhang) are filled with zeros.
+template <int kBK, int kBN, int kPieces>
+__device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* src0, int64_t krow_stride, int br_log2,
+                                                   int bc_log2, int k_rows_left, int n_cols_left, int lane) {
+    constexpr int kChunks = kBK * kBN * 2 / 16;
+    const int run_log2 = bc_log2 + 1;                       // log2(bytes of one block row)
+    const int g_log2 = br_log2 + run_log2;                  // log2(G)
+    const int seg_log2 = br_log2 + 1 + (kBN == 64 ? 6 : kBN == 128 ? 7 : 8);   // log2(kBN * br * 2): bytes of one run of tiles
+#pragma unroll 1
+    for (int base = 0; base < kChunks; base += 32 * 16) {
+        uint4 v[16];
+        int kl[16], nl[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int byte = (base + i * 32 + lane) << 4;   // byte offset inside the stage's memory image
+            const int seg = byte >> seg_log2, o = byte & ((1 << seg_log2) - 1);
+            const int ib = o & ((1 << g_log2) - 1);         // byte inside the memory tile
+            kl[i] = (seg << br_log2) + (ib >> run_log2);    // Eq. 1 inverted: row and column inside the stage
+            nl[i] = ((o >> g_log2) << bc_log2) + ((ib & ((1 << run_log2) - 1)) >> 1);
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (kl[i] < k_rows_left && nl[i] < n_cols_left)
+                v[i] = __ldg(reinterpret_cast<const uint4*>(src0 + int64_t(seg) * krow_stride + o));
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t word[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+            for (int pc = 0; pc < kPieces; ++pc) {
+                const int k = kl[i] + pc, n = nl[i];
+                uint8_t* dst = sw + (n >> 6) * (kBK * kAtomBytes) + k * kAtomBytes + ((((n & 63) >> 3) ^ (k & 7)) << 4) +
+                               (n & 7) * 2;
+                if (kPieces == 1) *reinterpret_cast<uint4*>(dst) = v[i];
+                else if (kPieces == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(word[2 * pc], word[2 * pc + 1]);
+                else if (kPieces == 4) *reinterpret_cast<uint32_t*>(dst) = word[pc];
+                else *reinterpret_cast<uint16_t*>(dst) = uint16_t(word[pc >> 1] >> ((pc & 1) * 16));
+            }
+        }
+    }
+}
+
+// silu(g) * u in fp32, rounded once to bf16 (nearest even).
+__device__ __forceinline__ __nv_bfloat16 swiglu_bf16(float g, float u) {
+    return __float2bfloat16_rn(g / (1.0f + expf(-g)) * u);
+}
+
+// Tensor-map coordinates of the weight box that starts at K element k and weight column n (kc_expert: the
+// expert's offset along the stacked dimension).
+__device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, int n, int kc_expert, int (&c)[5]) {
+    c[0] = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        c[i + 1] = ((k >> p.ck_shift[i]) & p.ck_mask[i]) + ((n >> p.cn_shift[i]) & p.cn_mask[i]) + p.c_expert[i] * kc_expert;
+}
+
+// kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256).
+// kWN selects which side of the MMA the weights are on.  The tensor pipe takes N/2 clocks per MMA whatever M is,
+// and the thread that issues the MMAs runs alone in its warp (every scalar instruction between two MMAs costs it
+// several clocks), so for small token tiles what matters is how many weight bytes one instruction consumes:
+//   kWN = false  weights on the M side: kBN/128 MMAs per K step, each 128 (or 64) weight columns x up to 256
+//                tokens.  For prefill (256-token tiles): the accumulator is C transposed, TMEM lane = weight
+//                column, and the epilogue writes 128-byte row segments.
+//   kWN = true   weights on the N side: one MMA per K step covers all kBN (up to 256) weight columns, tokens
+//                (at most 128 per tile) on the M side.  For decode and MoE: 8 KB of weights per instruction
+//                instead of 4 KB, half as many instructions per byte streamed.  TMEM lane =
+//                token, and every thread writes its token's row of C in 16-byte pieces.
+template <int kBK, int kBN, bool kWN, bool kFp8>
+__global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+    constexpr int kNumN = kWN ? 1 : (kBN >= 128 ? kBN / 128 : 1);     // MMAs per K step
+    constexpr int kUmmaM = kWN ? 128 : (kBN >= 128 ? 128 : 64);       // rows of the MMA's M side
+    constexpr int kKSteps = kBK / 16;
+    constexpr int kSubK = kBK / 64;                        // token boxes per stage
+    constexpr uint32_t kWBytes = kBK * kBN * 2;            // weight bytes per stage
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t acc_full_bar[2];
+    __shared__ __align__(8) uint64_t acc_empty_bar[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t abort_flag;
+    __shared__ int prefix[kMaxExperts + 1];
+    __shared__ int row_start[kMaxExperts + 1];      // copy of the expert row offsets (dense: 0, M)
+    __shared__ int range_tab[kRangeTabMax + 1];     // stream-K: first flattened iteration of every CTA
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t stage_bytes = kWBytes + uint32_t(kSubK) * p.a_rows * kAtomBytes;
+    uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    const int acc_cols = kWN ? kBN : p.BM;                   // TMEM columns of one MMA's accumulator
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < uint32_t(2 * kNumN * acc_cols)) tmem_cols <<= 1;
+
+    // ---------------------------------------------------------------- set-up
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], p.generic_b ? 2 : 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 4); }
+        abort_flag = 0;
+        fence_mbar_init();
+        if (!p.generic_b) tma_prefetch_desc(&p.tmap_b);
+        for (int i = 0; i < kNumBoxChoices; ++i) tma_prefetch_desc(&p.tmap_a[i]);
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_slot, tmem_cols);
+        tmem_relinquish();
+    }
+    // Dense stream-K problems: while the kernel before this one in the stream is still finishing, ask for the
+    // first stages of this CTA's weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is
+    // the point of coherence, so this is safe whatever that kernel is still writing; it takes the cold start
+    // (page walks, first DRAM accesses) off this kernel's critical path.
+    // (issued by an epilogue thread, which has nothing else to do yet, so that the producer is not held up)
+    if (threadIdx.x == 64 && p.stream_k && !p.generic_b && p.offsets == nullptr && p.prefetch_stages > 0) {
+        const int mt = (p.M + p.BM - 1) / p.BM;
+        const long long total = static_cast<long long>(mt) * p.n_tiles * p.k_iters;
+        const int geff = Sched::effective_grid(total, gridDim.x);
+        if (int(blockIdx.x) < geff) {
+            long long it = Sched::split(total, geff, blockIdx.x);
+            const long long it_end = Sched::split(total, geff, blockIdx.x + 1);
+            for (int s = 0; s < p.prefetch_stages && it < it_end; ++s, ++it) {
+                const int tile = int(it / p.k_iters), kit = int(it - static_cast<long long>(tile) * p.k_iters);
+                const int n0 = (tile / mt) * p.BN;
+                const int kq = ((tile % mt) & 1) ? p.k_iters - 1 - kit : kit;      // odd m-tiles walk K backwards
+                const int k0 = (kq * kBK) << p.k_shift;
+                for (int kb = 0; kb < p.kbx; ++kb)
+                    for (int nb = 0; nb < p.nbx; ++nb) {
+                        int c[5];
+                        weight_box_coords(p, k0 + kb * p.box_rows, n0 + nb * p.box_atoms * 64, 0, c);
+                        tma_prefetch_5d(&p.tmap_b, c[0], c[1], c[2], c[3], c[4]);
+                    }
+            }
+        }
+    }
+    // Token rows between BM and the rows the MMA reads are zeroed once; no copy ever writes them.  (The MMA's token
+    // side has at least 64 rows.  Whatever lies there is multiplied with the weights at full rate, and with stale
+    // data instead of zeros the tensor pipe draws enough power to pull the SM clock down under the board's cap.)
+    if (p.a_rows > p.BM && warp >= 2) {
+        const int per = (p.a_rows - p.BM) * (kAtomBytes / 16);          // 16-byte pieces per 64-wide K slice
+        const int total = p.num_stages * kSubK * per;
+        for (int i = int(threadIdx.x) - 64; i < total; i += int(blockDim.x) - 64) {
+            const int s = i / (kSubK * per), r = i % (kSubK * per);
+            uint8_t* slice = stages + size_t(s) * stage_bytes + kWBytes + size_t(r / per) * p.a_rows * kAtomBytes;
+            *reinterpret_cast<uint4*>(slice + size_t(p.BM) * kAtomBytes + size_t(r % per) * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
+    }
+    // Launched with programmatic stream serialisation: everything above (barriers, tensor memory, descriptor
+    // prefetch) may run while the kernel before this one in the stream is still finishing.  Nothing that kernel
+    // may have written (tokens, expert offsets, the partial-tile workspace, C) is touched before this wait, which
+    // returns once it has completed and its writes are visible.
+    // Grouped problems read the expert offsets, which that kernel may have produced, for the tables below; dense
+    // problems build their tables from the launch parameters alone and wait afterwards.
+    const bool tables_first = p.offsets == nullptr;
+    if (!tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // tiles before each expert (dense: one "expert" holding all M rows)
+    load_row_starts(p, row_start);
+    __syncthreads();
+    if (warp == 2) tile_prefix(p, row_start, prefix);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    const int tiles_total = prefix[p.E];
+    // Range starts of all CTAs, once, so that nothing on the critical path divides 64-bit numbers.
+    const long long total_iters = static_cast<long long>(tiles_total) * p.k_iters;
+    const int grid_eff0 = Sched::effective_grid(total_iters, gridDim.x);
+    const bool use_tab = p.stream_k && grid_eff0 > 0 && grid_eff0 <= kRangeTabMax && total_iters < (1ll << 31);
+    if (use_tab) {
+        for (int c = threadIdx.x; c <= grid_eff0; c += blockDim.x)
+            range_tab[c] = static_cast<int>(Sched::split(total_iters, grid_eff0, c));
+        __syncthreads();
+    }
+    Sched sched;
+    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
+    if (tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Stream-K: let the reduction kernel that follows in the stream be scheduled already; it does its own
+    // set-up and then blocks until this whole grid has finished.
+    if (p.stream_k && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    volatile uint32_t* abort_ptr = &abort_flag;
+
+    if (warp == 0) {
+        // ============================================================ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            Work w;
+            bool ok = true;
+            // the K part of the coordinate maps, in registers for the whole loop
+            const bool one_box = p.kbx == 1 && p.nbx == 1;
+            int ks[4], km[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { ks[i] = p.ck_shift[i]; km[i] = p.ck_mask[i]; }
+            while (ok && sched.next(w)) {
+                const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+                int bi = 0;
+                while ((16 << bi) < t.rows) ++bi;
+                const uint32_t a_bytes = uint32_t(16 << bi) * kAtomBytes;
+                const uint32_t tx = uint32_t(kSubK) * a_bytes + uint32_t(p.kbx * p.nbx) * p.box_bytes;
+                const int kc_expert = t.expert * p.k_coord_per_expert;
+                int cn[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) cn[i] = ((t.n0 >> p.cn_shift[i]) & p.cn_mask[i]) + p.c_expert[i] * kc_expert;
+                for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                    if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* sw = stages + size_t(stage) * stage_bytes;
+                    uint8_t* sa = sw + kWBytes;
+                    // (test hook: the first stage of every CTA may be armed for more bytes than its copies deliver, so
+                    // that the wait on it runs out and the give-up path below is exercised)
+                    mbar_arrive_expect_tx(&full_bar[stage], issued == 0 ? tx + p.stall_extra_tx : tx);
+                    const int kq = t.flip ? p.k_iters - 1 - kit : kit;
+                    const int k0 = (kq * kBK) << p.k_shift;         // first K element of the stage
+#pragma unroll
+                    for (int sub = 0; sub < kSubK; ++sub)
+                        tma_load_2d(sa + size_t(sub) * p.a_rows * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
+                                    k0 + ((sub * 64) << p.k_shift), t.row0);
+                    if (one_box) {
+                        // the usual case, one box per stage: the column part of the coordinates was worked out once
+                        // for the tile, only the K part changes from stage to stage
+                        tma_load_5d(sw, &p.tmap_b, &full_bar[stage], 0, ((k0 >> ks[0]) & km[0]) + cn[0],
+                                    ((k0 >> ks[1]) & km[1]) + cn[1], ((k0 >> ks[2]) & km[2]) + cn[2],
+                                    ((k0 >> ks[3]) & km[3]) + cn[3]);
+                    } else {
+                        for (int kb = 0; kb < p.kbx; ++kb) {
+                            const int k = k0 + kb * p.box_rows;
+                            for (int nb = 0; nb < p.nbx; ++nb) {
+                                const int n = t.n0 + nb * p.box_atoms * 64;
+                                uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
+                                int c[5];
+                                weight_box_coords(p, k, n, kc_expert, c);
+                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], c[0], c[1], c[2], c[3], c[4]);
+                            }
+                        }
+                    }
+                    ++issued;
+                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (!ok || *abort_ptr) {
+                // Giving up: let the copies already issued land before the CTA's shared memory goes away.
+                uint32_t s = stage, ph = phase;
+                const uint32_t back = issued < uint32_t(p.num_stages) ? issued : uint32_t(p.num_stages);
+                for (uint32_t i = 0; i < back; ++i) {
+                    if (s == 0) { s = p.num_stages; ph ^= 1; }
+                    --s;
+                    const uint64_t t0 = global_timer_ns();
+                    const uint64_t drain_ns = p.wait_limit_ns < 20000000ull ? p.wait_limit_ns : 20000000ull;
+                    while (!mbar_try_wait(&full_bar[s], ph) && global_timer_ns() - t0 < drain_ns) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ============================================================= MMA issuer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            Work w;
+            bool ok = true;
+            // Descriptor words that do not change: the upper halves, the constant bits of the lower halves, and
+            // the (address >> 4) offsets of every K step (kept in registers: the loop below adds one per MMA).
+            const uint64_t tok_hi64 = smem_desc_hi(16u, 1024u, 2u);
+            const uint32_t tok_hi = uint32_t(tok_hi64 >> 32), tok_lo_const = uint32_t(tok_hi64);
+            const uint32_t w_hi = uint32_t(p.w_desc_hi >> 32), w_lo_const = uint32_t(p.w_desc_hi);
+            uint32_t w_off[kKSteps], tok_off[kKSteps];
+#pragma unroll
+            for (int j = 0; j < kKSteps; ++j) {
+                w_off[j] = p.kstep_off[j] >> 4;
+                tok_off[j] = (uint32_t(j >> 2) * uint32_t(p.a_rows) * kAtomBytes + uint32_t(j & 3) * 32u) >> 4;
+            }
+            const uint32_t ugroup16 = p.ugroup_off >> 4;
+            while (ok && sched.next(w)) {
+                const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+                const uint32_t n_mma = kWN ? uint32_t(kBN) : uint32_t((t.rows + 15) & ~15);
+                // fp32 accumulate, bf16 x bf16; the weights operand is MN-major (bit 15: A, bit 16: B), the token
+                // operand K-major; M = kUmmaM, N = n_mma
+                const uint32_t w_major = p.w_kmajor ? 0u : (kWN ? (1u << 16) : (1u << 15));
+                // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
+                const uint32_t m_mma = kWN ? uint32_t(p.umma_m) : uint32_t(kUmmaM);
+                const uint32_t idesc = (1u << 4) | (kFp8 ? 0u : (1u << 7) | (1u << 10)) | w_major |
+                                       ((n_mma >> 3) << 17) | ((m_mma >> 4) << 24);
+                if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty, p.wait_limit_ns)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * uint32_t(kNumN * acc_cols);
+                for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                    if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull, p.wait_limit_ns)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
+                    const uint32_t w_lo0 = w_lo_const | ((sw & 0x3FFFFu) >> 4);
+                    const uint32_t tok_lo0 = tok_lo_const | (((sw + kWBytes) & 0x3FFFFu) >> 4);
+                    const uint32_t first = kit > w.kbeg ? 1u : 0u;
+#pragma unroll
+                    for (int j = 0; j < kKSteps; ++j) {
+#pragma unroll
+                        for (int u = 0; u < kNumN; ++u) {
+                            const uint32_t accum = j > 0 ? 1u : first;
+                            const uint32_t w_lo = w_lo0 + w_off[j] + uint32_t(u) * ugroup16;
+                            if (kWN) umma_split<kFp8>(d_tmem, tok_lo0 + tok_off[j], tok_hi, w_lo, w_hi, idesc, accum);
+                            else umma_split<kFp8>(d_tmem + uint32_t(u * acc_cols), w_lo, w_hi, tok_lo0 + tok_off[j], tok_hi, idesc, accum);
+                        }
+                    }
+                    umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
+                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full_bar[acc]);         // accumulator complete
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1;
+            }
+        }
+    } else if (warp >= 6) {
+        // ================================ generic-address weight loader (Section 4.4 of the paper)
+        // Memory tiles whose rows are shorter than a TMA box allows are fetched with plain loads.  A stage's
+        // weights are kBK/br runs of whole memory tiles, each run contiguous in the tile-major buffer, so
+        // the 16-byte chunks are read in memory order (fully coalesced for any tile shape); Eq. 1 inverted
+        // gives every chunk's (row, column), and the chunk (or its 16/(2 bc) row pieces) is stored where the
+        // 128-byte-swizzled MN-major operand layout wants it.  Warp w fills every fourth stage.
+        const int pw = warp - 6;
+        const int br = 1 << p.br_log2, bc = 1 << p.bc_log2;
+        const int run_bytes = bc * 2;                              // one block row
+        const int G = br * run_bytes;
+        const int pieces = run_bytes >= 16 ? 1 : 16 / run_bytes;  // rows held by one 16-byte chunk
+        uint32_t it_global = 0;
+        Work w;
+        bool ok = true;
+        while (ok && sched.next(w)) {
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+            const uint8_t* Bexp = p.B + int64_t(t.expert) * p.expert_bytes;
+            const int nblk0 = t.n0 >> p.bc_log2;
+            for (int kit = w.kbeg; kit < w.kend; ++kit, ++it_global) {
+                if ((it_global & 3u) != uint32_t(pw)) continue;
+                const uint32_t stage = it_global % uint32_t(p.num_stages);
+                const uint32_t phase = (it_global / uint32_t(p.num_stages)) & 1u;
+                if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns)) {
+                    ok = false;
+                    break;
+                }
+                uint8_t* sw = stages + size_t(stage) * stage_bytes;
+                const int kq = t.flip ? p.k_iters - 1 - kit : kit;
+                const int kblk0 = (kq * kBK) >> p.br_log2;
+                const uint8_t* src0 = Bexp + (int64_t(kblk0) * p.blocks_per_row + nblk0) * G;
+                const int k_rows_left = p.K - kq * kBK, n_cols_left = p.N - t.n0;
+                const int64_t krow_stride = int64_t(p.blocks_per_row) * G;      // bytes between runs of tiles
+                switch (pieces) {
+                    case 1: generic_fill_stage<kBK, kBN, 1>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                    case 2: generic_fill_stage<kBK, kBN, 2>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                    case 4: generic_fill_stage<kBK, kBN, 4>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                    default: generic_fill_stage<kBK, kBN, 8>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                }
+                fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor-core (async) proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[stage]);
+            }
+        }
+    } else {
+        // =============================================================== epilogue
+        const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31
+        uint32_t acc = 0, acc_phase = 0;
+        Work w;
+        while (sched.next(w)) {
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+            const bool full = (w.kbeg == 0 && w.kend == p.k_iters);
+            const int n_mma = (t.rows + 15) & ~15;
+            bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull, p.wait_limit_ns);
+            tc_fence_after_sync();
+            float* out;
+            int64_t ld;
+            if (full) {
+                out = p.C + int64_t(t.row0) * p.ldc + t.n0;
+                ld = p.ldc;
+            } else {
+                out = p.partials + size_t(sched.slot(sched.cta, w.tile)) * p.BM * kBN;
+                ld = kBN;
+            }
+            if (ok && kWN) {
+                // TMEM lane = token row, columns = the tile's kBN weight columns: each thread owns one row of C.
+                // (MMA of 64 rows: rows 16q..16q+15 sit in the lower half of lane quarter q, the upper 16 lanes of
+                // each quarter hold nothing.)
+                const bool m64 = p.umma_m == 64;
+                const int row = m64 ? (lane < 16 ? quarter * 16 + lane : p.BM) : quarter * 32 + lane;
+                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * uint32_t(acc_cols);
+                if ((m64 ? quarter * 16 : quarter * 32) < t.rows) {      // this lane quarter holds at least one real row
+                    float* dst = out + int64_t(row) * ld;
+                    const bool gated = full && p.epi_swiglu;
+                    __nv_bfloat16* hdst = p.H + int64_t(t.row0 + row) * p.ldh + (t.n0 >> 1);
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kBN; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(taddr + c0, v);
+                        tmem_ld_wait();
+                        if (gated) {
+                            // 32 columns = 16 (gate, up) pairs -> 16 bf16 = two 16-byte stores
+                            if (row < t.rows && t.n0 + c0 < p.N) {
+                                uint32_t h2[8];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const __nv_bfloat16 lo = swiglu_bf16(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]));
+                                    const __nv_bfloat16 hi = swiglu_bf16(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                                    h2[i] = uint32_t(__bfloat16_as_ushort(lo)) | (uint32_t(__bfloat16_as_ushort(hi)) << 16);
+                                }
+                                uint4* q = reinterpret_cast<uint4*>(hdst + (c0 >> 1));
+                                q[0] = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+                                q[1] = make_uint4(h2[4], h2[5], h2[6], h2[7]);
+                            }
+                        } else if (full && p.Cb) {
+                            // 32 columns -> 32 bf16 = four 16-byte stores
+                            if (row < t.rows) {
+                                __nv_bfloat16* cdst = p.Cb + int64_t(t.row0 + row) * p.ldc + t.n0 + c0;
+#pragma unroll
+                                for (int i = 0; i < 32; i += 8)
+                                    if (t.n0 + c0 + i < p.N) {
+                                        uint32_t h[4];
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j)
+                                            h[j] = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[i + 2 * j])))) |
+                                                   (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[i + 2 * j + 1])))) << 16);
+                                        *reinterpret_cast<uint4*>(cdst + i) = make_uint4(h[0], h[1], h[2], h[3]);
+                                    }
+                            }
+                        } else if (row < t.rows) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4)
+                                if (!full || t.n0 + c0 + i < p.N)
+                                    *reinterpret_cast<float4*>(dst + c0 + i) =
+                                        make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                    __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                        }
+                    }
+                }
+            }
+            if (ok && !kWN) {
+#pragma unroll
+                for (int u = 0; u < kNumN; ++u) {
+                    // M = 128: accumulator row r sits in TMEM lane r.  M = 64: rows 16q..16q+15 sit in the
+                    // lower half of lane quarter q, the upper 16 lanes of each quarter hold nothing.
+                    const int n_local = kUmmaM == 128 ? u * 128 + quarter * 32 + lane : quarter * 16 + lane;
+                    const bool lane_ok = kUmmaM == 128 || lane < 16;
+                    const bool n_ok = lane_ok && (full ? (t.n0 + n_local < p.N) : true);
+                    const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) +
+                                           acc * uint32_t(kNumN * acc_cols) + uint32_t(u * acc_cols);
+                    const bool to_bf16 = full && p.Cb != nullptr;
+                    __nv_bfloat16* outb = p.Cb + int64_t(t.row0) * p.ldc + t.n0 + n_local;
+                    for (int c0 = 0; c0 < n_mma; c0 += 32) {
+                        if (n_mma - c0 >= 32) {
+                            uint32_t v[32];
+                            tmem_ld_32x32b_x32(taddr + c0, v);
+                            tmem_ld_wait();
+                            if (to_bf16) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (n_ok && c0 + i < t.rows) outb[int64_t(c0 + i) * p.ldc] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                            }
+                        } else {
+                            uint32_t v[16];
+                            tmem_ld_32x32b_x16(taddr + c0, v);
+                            tmem_ld_wait();
+                            if (to_bf16) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    if (n_ok && c0 + i < t.rows) outb[int64_t(c0 + i) * p.ldc] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    if (n_ok && c0 + i < t.rows) out[int64_t(c0 + i) * ld + n_local] = __uint_as_float(v[i]);
+                            }
+                        }
+                    }
+                }
+            }
+            // accumulator drained: hand it back to the MMA warp
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty_bar[acc]);
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1;
+
+            if (*abort_ptr) break;
+        }
+    }
+
+    // --------------------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// The kernel's instantiations are compiled in translation units of their own, one per (orientation, element type):
+// weights on the N or on the M side of the MMA, bf16 or FP8.  Each raises the kernel's shared-memory limit on first
+// use per device and launches with the given configuration; TL_ERR_UNSUPPORTED for a (cta_k, cta_n) outside
+// {64, 128} x {64, 128, 256}.
+int launch_gemm_wn_bf16(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
+int launch_gemm_wn_fp8(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
+int launch_gemm_wm_bf16(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
+int launch_gemm_wm_fp8(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
+// CTA-pair kernel (tl_gemm_pair.cu): halves = 2 for 512-token tiles.
+int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream_t stream, const GemmParams& p);
+// Clusters of the pair kernel that can be resident together on the current device.
+int pair_max_active_clusters(int* out);
+constexpr int kPairStagesMax = 8;
+
+}  // namespace tl

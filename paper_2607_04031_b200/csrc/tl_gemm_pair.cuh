@@ -1,8 +1,10 @@
 // Prefill GEMM on CTA pairs (included by tl_gemm.cu after GemmParams and the helpers).
 //
-// A tcgen05.mma issued for one CTA (cta_group::1) takes about 180 clocks whatever its shape, which caps a
-// 128 x 256 x 16 instruction at ~70 % of the tensor peak.  The cta_group::2 form, one instruction spanning
-// the tensor cores of two SMs of a cluster (M = 256), measured 128 clocks for 256 x 256 x 16: the full rate.
+// A tcgen05.mma occupies the tensor pipe for N/2 clocks per 16-deep K step whether it is issued for one CTA
+// (cta_group::1, M = 64 or 128) or for a pair (cta_group::2, M = 256: measured 128 clocks for 256 x 256 x 16).  The
+// pair form therefore does twice the work per instruction and per operand byte staged in shared memory: each CTA
+// holds only its own half of the tile's weights and tokens, and the one thread that issues MMAs has half as many
+// instructions to get out per flop.
 // So for large M two CTAs share one 256-token x 256-column output tile:
 //   - each CTA loads ITS 128 weight columns (the same one-box-per-stage tile-major view as the single-CTA
 //     kernel) and HALF of the 256 token rows; 32 KB per CTA per 64-row K step instead of 48 KB, six stages;
@@ -121,7 +123,6 @@ __device__ __forceinline__ void umma_pair_commit_both(uint64_t* bar) {
         : "memory");
 }
 
-constexpr int kPairStagesMax = 8;
 constexpr int kPairBand = 8;      // m-tiles per band of the tile order
 
 // Tile order: bands of kPairBand m-tiles, inside a band the n-tile index moves slowest.  The clusters that run
@@ -219,20 +220,11 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                                          : p.pair_big_tiles + 2 * (m_tiles * n_pair_tiles - p.pair_big_tiles);
     const int first_tile = int(cluster_id_x()), tile_step = int(num_clusters_x());
 
-#ifdef TL_TIMELINE
-    uint64_t* const dbg = g_timeline ? g_timeline + blockIdx.x * 8 : nullptr;
-    long long w_wait = 0, w_issue = 0;
-#define TL_CLK() clock64()
-#else
-#define TL_CLK() 0ll
-#endif
     if (warp == 0) {
         // ============================================================ TMA producer (one per CTA)
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, issued = 0;
             bool ok = true;
-            const long long t_begin = TL_CLK();
-            (void)t_begin;
             int ks[4], km[4];                                       // K part of the coordinate maps, in registers
 #pragma unroll
             for (int i = 0; i < 4; ++i) { ks[i] = p.ck_shift[i]; km[i] = p.ck_mask[i]; }
@@ -245,13 +237,10 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) cn[i] = (n0 >> p.cn_shift[i]) & p.cn_mask[i];
                 for (int kit = 0; kit < p.k_iters; ++kit) {
-                    const long long c0 = TL_CLK();
-                    if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty)) {
+                    if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns)) {
                         ok = false;
                         break;
                     }
-                    const long long c1 = TL_CLK();
-                    (void)c0; (void)c1;
                     uint8_t* sw = stages + size_t(stage) * kStageBytes;
                     // The leader's producer alone arms the barrier, for the bytes of BOTH CTAs; the peer only
                     // issues its copies.  Their completions may be counted before the leader has armed the
@@ -267,16 +256,10 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     tma_pair_load_5d(sw, &p.tmap_b, full_leader, 0, ((k >> ks[0]) & km[0]) + cn[0], ((k >> ks[1]) & km[1]) + cn[1],
                                      ((k >> ks[2]) & km[2]) + cn[2], ((k >> ks[3]) & km[3]) + cn[3]);
                     ++issued;
-#ifdef TL_TIMELINE
-                    w_wait += c1 - c0; w_issue += TL_CLK() - c1;
-#endif
                     if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
                 }
             }
             (void)issued;
-#ifdef TL_TIMELINE
-            if (dbg) { dbg[0] = TL_CLK() - t_begin; dbg[1] = w_wait; dbg[2] = w_issue; dbg[7] = rank; }
-#endif
         }
     } else if (warp == 1) {
         // ============================================================= MMA issuer (leader CTA only)
@@ -288,8 +271,6 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             const uint32_t idesc = (1u << 4) | (kFp8 ? 0u : (1u << 7) | (1u << 10)) | (p.w_kmajor ? 0u : (1u << 15)) |
                                    ((256u >> 3) << 17) | ((256u >> 4) << 24);
             bool ok = true;
-            const long long t_begin = TL_CLK();
-            (void)t_begin;
             // constant descriptor words and per-K-step offsets, in registers for the issue loop
             const uint64_t tok_hi64 = smem_desc_hi(16u, 1024u, 2u);
             const uint32_t tok_hi = uint32_t(tok_hi64 >> 32), tok_lo_const = uint32_t(tok_hi64);
@@ -300,24 +281,14 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             for (int tile = first_tile; ok && tile < tiles_total; tile += tile_step) {
                 const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
                 if (pt.halves == 0) continue;
-                const long long a0 = TL_CLK();
-                if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty)) break;
-#ifdef TL_TIMELINE
-                w_issue += TL_CLK() - a0;      // (MMA thread: w_issue = cycles waiting for a free accumulator)
-#endif
-                (void)a0;
+                if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty, p.wait_limit_ns)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * 256u;
                 for (int kit = 0; kit < p.k_iters; ++kit) {
-                    const long long c0 = TL_CLK();
-                    if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull)) {
+                    if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull, p.wait_limit_ns)) {
                         ok = false;
                         break;
                     }
-#ifdef TL_TIMELINE
-                    w_wait += TL_CLK() - c0;
-#endif
-                    (void)c0;
                     tc_fence_after_sync();
                     const uint32_t sw = smem_u32(stages + size_t(stage) * kStageBytes);
                     const uint32_t w_lo0 = w_lo_const | ((sw & 0x3FFFFu) >> 4);
@@ -340,9 +311,6 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                 if (kHalves == 1) acc ^= 1;                         // (512-token tiles own both accumulators)
                 if (acc == 0) acc_phase ^= 1;
             }
-#ifdef TL_TIMELINE
-            if (dbg) { dbg[3] = TL_CLK() - t_begin; dbg[4] = w_wait; dbg[5] = w_issue; }
-#endif
         }
     } else {
         // =============================================================== epilogue (both CTAs)
@@ -353,7 +321,7 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
             if (pt.halves == 0) continue;
             const int n0 = pt.n_tile * 256 + int(rank) * 128;
-            const bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull);
+            const bool ok = mbar_wait_bounded(&acc_full_bar[acc], acc_phase, abort_ptr, p.status, kWaitEpilogueAccFull, p.wait_limit_ns);
             tc_fence_after_sync();
             if (ok) {
                 const int n_local = quarter * 32 + lane;

@@ -202,7 +202,7 @@ static int hw_prepare(const tl_hw_desc* d, HwParams* p) {
 // One warp per box (or per run of pieces of a box), eight warps per CTA, at most 8 CTAs per SM.
 static unsigned hw_grid(long long n_boxes) {
     const long long ctas = ceil_div(n_boxes, 8);
-    const long long cap = 8ll * (state().sm_count > 0 ? state().sm_count : 148);
+    const long long cap = 8ll * (dev().sm_count > 0 ? dev().sm_count : 148);
     return unsigned(ctas < 1 ? 1 : (ctas < cap ? ctas : cap));
 }
 
@@ -212,6 +212,7 @@ extern "C" {
 
 int tl_hw_box_offsets(const tl_hw_desc* desc, const int32_t* d_coords, int64_t n_boxes, uint64_t* d_offsets,
                       void* cuda_stream) {
+    tl::ApiLock lock;
     tl::HwParams p;
     if (int rc = tl::hw_prepare(desc, &p)) return rc;
     if (n_boxes < 0) return TL_ERR_INVALID_ARG;
@@ -222,13 +223,14 @@ int tl_hw_box_offsets(const tl_hw_desc* desc, const int32_t* d_coords, int64_t n
     p.n_boxes = n_boxes;
     p.coords = d_coords;
     p.offsets = reinterpret_cast<unsigned long long*>(d_offsets);
-    p.status = tl::state().ctl.d_status;
+    p.status = tl::dev().ctl.d_status;
     tl::hw_offsets_kernel<<<tl::hw_grid(n_boxes), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
     return tl::check_cuda(cudaGetLastError());
 }
 
 int tl_hw_box_load(const tl_hw_desc* desc, const void* d_src_tilemajor, uint64_t src_bytes, const int32_t* d_coords,
                    int64_t n_boxes, void* d_dst, void* cuda_stream) {
+    tl::ApiLock lock;
     tl::HwParams p;
     if (int rc = tl::hw_prepare(desc, &p)) return rc;
     if (n_boxes < 0) return TL_ERR_INVALID_ARG;
@@ -241,7 +243,7 @@ int tl_hw_box_load(const tl_hw_desc* desc, const void* d_src_tilemajor, uint64_t
     p.src = static_cast<const uint8_t*>(d_src_tilemajor);
     p.src_bytes = src_bytes;
     p.dst = static_cast<uint8_t*>(d_dst);
-    p.status = tl::state().ctl.d_status;
+    p.status = tl::dev().ctl.d_status;
     const long long row_bytes = p.u << p.s_log2;
     const bool vec16 = row_bytes >= 16 && reinterpret_cast<uintptr_t>(d_src_tilemajor) % 16 == 0 &&
                        reinterpret_cast<uintptr_t>(d_dst) % 16 == 0;

@@ -200,7 +200,7 @@ static int read_amp_fill(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int c
         if (d_fetched || d_used) return TL_ERR_UNSUPPORTED;
     }
     p.d_acc = d_acc; p.d_fetched = d_fetched; p.d_used = d_used;
-    p.h_out = d_acc ? (totals_out ? totals_out : state().ctl.h_acc_dev) : nullptr;
+    p.h_out = d_acc ? (totals_out ? totals_out : dev().ctl.h_acc_dev) : nullptr;
     p.iters_per_warp = p.layout == TL_LAYOUT_TILE_MAJOR ? p.k_iters : kItersPerWarp;
     *grid_out = 0;
     if (m_tiles == 0) return TL_OK;
@@ -235,8 +235,7 @@ static int read_amp_launch(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static const bool no_pdl = getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0;     // measurement switch
-    cfg.numAttrs = no_pdl ? 0 : 1;
+    cfg.numAttrs = opt(TL_OPT_PDL) != 0 ? 1 : 0;           // measurement switch
     return check_cuda(cudaLaunchKernelEx(&cfg, read_amp_kernel, p));
 }
 
@@ -245,18 +244,19 @@ static int read_amp_totals(int64_t m_tiles, int64_t N, int64_t K, int cta_n, int
                            int64_t wave_tiles = 0) {
     if (!fetched || !used) return TL_ERR_INVALID_ARG;
     if (int rc = ensure_control()) return rc;
-    State& st = state();
+    Control& ctl = dev().ctl;
+    const cudaStream_t stream = tls().stream;
     if (m_tiles == 0) {
         *fetched = *used = 0;
         if (requests) *requests = 0;
         return TL_OK;
     }
-    if (int rc = read_amp_launch(m_tiles, N, K, cta_n, cta_k, layout, G, br, bc, s, st.ctl.d_acc, nullptr, nullptr,
-                                 st.stream, wave_tiles))
+    if (int rc = read_amp_launch(m_tiles, N, K, cta_n, cta_k, layout, G, br, bc, s, ctl.d_acc, nullptr, nullptr,
+                                 stream, wave_tiles))
         return rc;
     // the kernel's last warp wrote the totals into mapped pinned memory; the only wait is this one
-    volatile unsigned long long* h = st.ctl.h_acc;
-    if (int rc = check_cuda(cudaStreamSynchronize(st.stream))) return rc;
+    volatile unsigned long long* h = ctl.h_acc;
+    if (int rc = check_cuda(cudaStreamSynchronize(stream))) return rc;
     *fetched = h[0];
     *used = h[1];
     if (requests) *requests = h[2];
@@ -270,6 +270,7 @@ extern "C" {
 int tl_read_amp(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int layout, int64_t G,
                 int block_rows, int block_cols, int elem_bytes, uint64_t* bytes_fetched, uint64_t* bytes_used,
                 uint64_t* requests) {
+    tl::ApiLock lock;
     if (M < 0) return TL_ERR_INVALID_ARG;
     if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
         return rc;
@@ -280,6 +281,7 @@ int tl_read_amp(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k
 int tl_read_amp_shared(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int64_t wave_ctas, int layout,
                        int64_t G, int block_rows, int block_cols, int elem_bytes, uint64_t* bytes_fetched,
                        uint64_t* bytes_needed, uint64_t* requests) {
+    tl::ApiLock lock;
     if (M < 0 || wave_ctas <= 0) return TL_ERR_INVALID_ARG;
     if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
         return rc;
@@ -302,6 +304,7 @@ int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64
 
 int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int layout, int64_t G,
                       int block_rows, int block_cols, int elem_bytes, uint64_t* d_totals, void* cuda_stream) {
+    tl::ApiLock lock;
     if (M < 0 || !d_totals) return TL_ERR_INVALID_ARG;
     if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
         return rc;
@@ -311,11 +314,12 @@ int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int
     // The accumulators are shared by all launches on the device: launches must be ordered by one stream (they
     // are between tl_read_amp* calls, which all use the stream they are given or the tl_set_stream() stream).
     return tl::read_amp_launch(tl::ceil_div(M, cta_m), N, K, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes,
-                               tl::state().ctl.d_acc, nullptr, nullptr, st, 0,
+                               tl::dev().ctl.d_acc, nullptr, nullptr, st, 0,
                                reinterpret_cast<unsigned long long*>(d_totals));
 }
 
 int tl_read_amp_batch(const tl_read_amp_cfg* h_cfgs, int n, uint64_t* d_totals, void* cuda_stream) {
+    tl::ApiLock lock;
     if (n < 0 || n > tl::kBatchMax || (n > 0 && (!h_cfgs || !d_totals))) return TL_ERR_INVALID_ARG;
     if (n == 0) return TL_OK;
     if (int rc = tl::ensure_control()) return rc;
@@ -332,7 +336,7 @@ int tl_read_amp_batch(const tl_read_amp_cfg* h_cfgs, int n, uint64_t* d_totals, 
         int64_t grid = 0;
         // configuration i accumulates in its own four words of the control block and publishes to its own slot
         if (int rc = tl::read_amp_fill(tl::ceil_div(c.M, c.cta_m), c.N, c.K, c.cta_n, c.cta_k, c.layout, c.G, c.block_rows,
-                                       c.block_cols, c.elem_bytes, tl::state().ctl.d_acc + 4 * (i + 1), nullptr, nullptr, 0,
+                                       c.block_cols, c.elem_bytes, tl::dev().ctl.d_acc + 4 * (i + 1), nullptr, nullptr, 0,
                                        reinterpret_cast<unsigned long long*>(d_totals) + 3 * i, &b.p[b.n], &grid))
             return rc;
         if (grid == 0) {                                    // M == 0: nothing is launched for it, its totals are zero
@@ -361,6 +365,7 @@ int tl_read_amp_batch(const tl_read_amp_cfg* h_cfgs, int n, uint64_t* d_totals, 
 int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
                         int layout, int64_t G, int block_rows, int block_cols, int elem_bytes,
                         uint64_t* bytes_fetched, uint64_t* bytes_used, uint64_t* requests) {
+    tl::ApiLock lock;
     if (!h_offsets || E < 0) return TL_ERR_INVALID_ARG;
     if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
         return rc;
@@ -379,6 +384,7 @@ int tl_read_amp_grouped(const int32_t* h_offsets, int E, int64_t N, int64_t K, i
 int tl_read_amp_per_cta(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int layout, int64_t G,
                         int block_rows, int block_cols, int elem_bytes, uint64_t* d_fetched, uint64_t* d_used,
                         void* cuda_stream) {
+    tl::ApiLock lock;
     if (M < 0) return TL_ERR_INVALID_ARG;
     if (int rc = tl::read_amp_validate(N, K, cta_m, cta_n, cta_k, layout, G, block_rows, block_cols, elem_bytes))
         return rc;

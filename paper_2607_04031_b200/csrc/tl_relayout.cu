@@ -228,6 +228,8 @@ struct RelayoutTmaParams {
     CUtensorMap row_map;     // row-major side
     uint8_t* tile_base;      // tile-major side
     uint32_t* status;
+    uint64_t wait_limit_ns;  // bound of the wait for a buffer's load
+    uint32_t stall_extra_tx; // test hook: bytes added to what the first load's barrier expects (0 in normal use)
     int64_t G;
     int br, nb;              // rows of a memory tile, memory tiles per step
     int blocks_per_row, block_rows;
@@ -261,11 +263,12 @@ __global__ void __launch_bounds__(32, kTmaCtasPerSm) relayout_tma_kernel(const _
         const int b0 = int(step % p.steps_x) * p.nb;
         const int nbt = p.blocks_per_row - b0 < p.nb ? p.blocks_per_row - b0 : p.nb;
         uint8_t* buf = bufs + size_t(s) * kTmaTileBytes;
+        const uint32_t extra = i == 0 ? p.stall_extra_tx : 0u;      // (test hook, see RelayoutTmaParams)
         if (p.to_tile_major) {
-            mbar_arrive_expect_tx(&full_bar[s], uint32_t(p.nb) * uint32_t(p.G));      // a box always counts in full
+            mbar_arrive_expect_tx(&full_bar[s], uint32_t(p.nb) * uint32_t(p.G) + extra);      // a box always counts in full
             tma_load_3d(buf, &p.row_map, &full_bar[s], 0, int(brow) * p.br, b0);
         } else {
-            mbar_arrive_expect_tx(&full_bar[s], uint32_t(nbt) * uint32_t(p.G));
+            mbar_arrive_expect_tx(&full_bar[s], uint32_t(nbt) * uint32_t(p.G) + extra);
             bulk_load_1d(buf, p.tile_base + (brow * p.blocks_per_row + b0) * p.G, uint32_t(nbt) * uint32_t(p.G), &full_bar[s]);
         }
     };
@@ -273,7 +276,7 @@ __global__ void __launch_bounds__(32, kTmaCtasPerSm) relayout_tma_kernel(const _
     for (int64_t i = 0; i < ahead; ++i) issue_load(i);
     for (int64_t i = 0; i < mine; ++i) {
         const int s = int(i % kTmaStages);
-        if (!mbar_wait_bounded(&full_bar[s], uint32_t(i / kTmaStages) & 1u, abort_ptr, p.status, kWaitRelayoutFull)) break;
+        if (!mbar_wait_bounded(&full_bar[s], uint32_t(i / kTmaStages) & 1u, abort_ptr, p.status, kWaitRelayoutFull, p.wait_limit_ns)) break;
         const int64_t step = first + i * stride;
         const int64_t brow = step / p.steps_x;
         const int b0 = int(step % p.steps_x) * p.nb;
@@ -320,7 +323,12 @@ static int relayout_tma_launch(const void* d_src, void* d_dst, int64_t rows, int
                                    strides, box))
         return rc;
     p.tile_base = static_cast<uint8_t*>(tile_side);
-    p.status = state().ctl.d_status;
+    p.status = dev().ctl.d_status;
+    p.wait_limit_ns = wait_limit_ns();
+    if (opt(TL_OPT_STALL_ONCE) == 2) {           // test hook: this launch's first load per CTA never completes its barrier
+        p.stall_extra_tx = 16;
+        tl_set_option(TL_OPT_STALL_ONCE, 0);
+    }
     p.G = G;
     p.br = br;
     p.nb = nb;
@@ -330,13 +338,8 @@ static int relayout_tma_launch(const void* d_src, void* d_dst, int64_t rows, int
     p.steps_total = p.steps_x * (rows / br);
     p.to_tile_major = to_tile;
     const size_t smem = size_t(kTmaStages) * kTmaTileBytes + 128;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (int rc = check_cuda(cudaFuncSetAttribute(relayout_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))))
-            return rc;
-        attr_set = true;
-    }
-    const int64_t max_grid = int64_t(state().sm_count) * kTmaCtasPerSm;
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(relayout_tma_kernel), int(smem))) return rc;
+    const int64_t max_grid = int64_t(dev().sm_count) * kTmaCtasPerSm;
     const int grid = int(p.steps_total < max_grid ? p.steps_total : max_grid);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -347,8 +350,7 @@ static int relayout_tma_launch(const void* d_src, void* d_dst, int64_t rows, int
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static const bool no_pdl = getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0;     // measurement switch
-    cfg.numAttrs = no_pdl ? 0 : 1;
+    cfg.numAttrs = opt(TL_OPT_PDL) != 0 ? 1 : 0;           // measurement switch
     *taken = true;
     return check_cuda(cudaLaunchKernelEx(&cfg, relayout_tma_kernel, p));
 }
@@ -367,6 +369,7 @@ struct RelayoutTmaBatch {
     int blocks_per_row[kBatchMax];
     int nb[kBatchMax];                     // memory tiles per step (min(tile budget, blocks per row))
     uint32_t* status;
+    uint64_t wait_limit_ns;
     int64_t G;
     int br, n;
     int to_tile_major;
@@ -420,7 +423,7 @@ __global__ void __launch_bounds__(32, kTmaCtasPerSm) relayout_tma_batch_kernel(c
     for (int64_t i = 0; i < ahead; ++i) issue_load(i);
     for (int64_t i = 0; i < mine; ++i) {
         const int s = int(i % kTmaStages);
-        if (!mbar_wait_bounded(&full_bar[s], uint32_t(i / kTmaStages) & 1u, abort_ptr, p.status, kWaitRelayoutFull)) break;
+        if (!mbar_wait_bounded(&full_bar[s], uint32_t(i / kTmaStages) & 1u, abort_ptr, p.status, kWaitRelayoutFull, p.wait_limit_ns)) break;
         const Step st = locate(i);
         const uint8_t* buf = bufs + size_t(s) * kTmaTileBytes;
         if (p.to_tile_major) bulk_store_1d(tile_ptr(st), buf, uint32_t(st.nbt) * uint32_t(p.G));
@@ -472,19 +475,15 @@ static int relayout_tma_batch_launch(int n, const void* const* srcs, void* const
         p.steps_x[i] = int(ceil_div(blocks_per_row, nb));
         p.steps_begin[i + 1] = p.steps_begin[i] + int64_t(p.steps_x[i]) * (rows[i] / br);
     }
-    p.status = state().ctl.d_status;
+    p.status = dev().ctl.d_status;
+    p.wait_limit_ns = wait_limit_ns();
     p.G = G;
     p.br = br;
     p.n = n;
     p.to_tile_major = to_tile;
     const size_t smem = size_t(kTmaStages) * kTmaTileBytes + 128;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (int rc = check_cuda(cudaFuncSetAttribute(relayout_tma_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))))
-            return rc;
-        attr_set = true;
-    }
-    const int64_t max_grid = int64_t(state().sm_count) * kTmaCtasPerSm, total = p.steps_begin[n];
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(relayout_tma_batch_kernel), int(smem))) return rc;
+    const int64_t max_grid = int64_t(dev().sm_count) * kTmaCtasPerSm, total = p.steps_begin[n];
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(total < max_grid ? total : max_grid));
     cfg.blockDim = dim3(32);
@@ -494,8 +493,7 @@ static int relayout_tma_batch_launch(int n, const void* const* srcs, void* const
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static const bool no_pdl = getenv("TL_NO_PDL") && atoi(getenv("TL_NO_PDL")) != 0;     // measurement switch
-    cfg.numAttrs = no_pdl ? 0 : 1;
+    cfg.numAttrs = opt(TL_OPT_PDL) != 0 ? 1 : 0;           // measurement switch
     return check_cuda(cudaLaunchKernelEx(&cfg, relayout_tma_batch_kernel, p));
 }
 
@@ -519,11 +517,11 @@ int relayout_launch(const void* d_src, void* d_dst, int64_t rows, int64_t cols, 
     const uintptr_t a = reinterpret_cast<uintptr_t>(d_src), b = reinterpret_cast<uintptr_t>(d_dst);
     if (a < b + bytes && b < a + bytes) return TL_ERR_INVALID_ARG;      // overlap
     if (int rc = ensure_device_info()) return rc;
-    const int sms = state().sm_count;
+    const int sms = dev().sm_count;
 
     {
-        // copy-engine path when the shape allows it (TL_RELAYOUT_NO_TMA=1 keeps the shared-memory kernel)
-        static const bool no_tma = getenv("TL_RELAYOUT_NO_TMA") && atoi(getenv("TL_RELAYOUT_NO_TMA")) != 0;
+        // copy-engine path when the shape allows it (TL_OPT_RELAYOUT_TMA = 0 keeps the shared-memory kernel)
+        const bool no_tma = opt(TL_OPT_RELAYOUT_TMA) == 0;
         bool taken = false;
         if (!no_tma) {
             if (int rc = relayout_tma_launch(d_src, d_dst, rows, cols, s, G, br, bc, direction, stream, &taken)) return rc;
@@ -567,8 +565,8 @@ int relayout_launch(const void* d_src, void* d_dst, int64_t rows, int64_t cols, 
     const int grid = int(p.tiles_total < max_grid ? p.tiles_total : max_grid);
     cudaError_t err = cudaSuccess;
 #define TL_LAUNCH_RELAYOUT(PIECE)                                                                              \
-    err = cudaFuncSetAttribute(relayout_kernel<PIECE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)); \
-    if (err == cudaSuccess) relayout_kernel<PIECE><<<grid, kRelayoutThreads, smem, stream>>>(p);
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(relayout_kernel<PIECE>), 48 * 1024)) return rc; \
+    relayout_kernel<PIECE><<<grid, kRelayoutThreads, smem, stream>>>(p);
     switch (piece) {
         case 16: TL_LAUNCH_RELAYOUT(16) break;
         case 8: TL_LAUNCH_RELAYOUT(8) break;
@@ -587,15 +585,17 @@ extern "C" {
 
 int tl_relayout_on(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes, int64_t G,
                    int block_rows, int block_cols, int direction, void* cuda_stream) {
+    tl::ApiLock lock;
     return tl::relayout_launch(d_src, d_dst, rows, cols, elem_bytes, G, block_rows, block_cols, direction,
                                static_cast<cudaStream_t>(cuda_stream));
 }
 
 int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, const int64_t* rows, const int64_t* cols,
                       int elem_bytes, int64_t G, int block_rows, int block_cols, int direction, void* cuda_stream) {
+    tl::ApiLock lock;
     if (n < 0 || (n > 0 && (!d_srcs || !d_dsts || !rows || !cols))) return TL_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    static const bool no_tma = getenv("TL_RELAYOUT_NO_TMA") && atoi(getenv("TL_RELAYOUT_NO_TMA")) != 0;
+    const bool no_tma = tl::opt(TL_OPT_RELAYOUT_TMA) == 0;
     // One launch when every matrix passes the argument checks of tl_relayout, is non-empty and can take the
     // copy-engine path; otherwise (and beyond kBatchMax matrices) one tl_relayout_on per matrix, in order.
     int i = 0;
@@ -631,8 +631,9 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
 
 int tl_relayout(const void* d_src, void* d_dst, int64_t rows, int64_t cols, int elem_bytes, int64_t G,
                 int block_rows, int block_cols, int direction) {
+    tl::ApiLock lock;
     return tl::relayout_launch(d_src, d_dst, rows, cols, elem_bytes, G, block_rows, block_cols, direction,
-                               tl::state().stream);
+                               tl::tls().stream);
 }
 
 }  // extern "C"

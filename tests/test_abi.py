@@ -106,6 +106,70 @@ def test_gemm_argument_checks_need_no_device(tl):
     assert L.tl_gemm_host_scratch_bytes(16, 512, 512) >= 16 * 512 * 2 + 2 * 512 * 512 * 2 + 16 * 512 * 4
 
 
+def test_output_rows_must_hold_whole_16_byte_vectors(tl):
+    # fp32 C is written in 16-byte vectors; the hand-addressed memory tiles of one or two columns would otherwise
+    # admit an N that is not a multiple of four
+    L = tl.lib()
+    p = ctypes.c_void_p(0x10000)
+    assert L.tl_gemm(p, p, p, 16, 1022, 512, 64, 16, 2, 0, 0, 0, None) == 2
+    assert L.tl_gemm(p, p, p, 16, 1021, 512, 32, 16, 1, 0, 0, 0, None) == 2
+    assert L.tl_gemm_kmajor(p, p, p, 16, 1022, 512, 4096, 2, 1024, 0, 0, 0, None) == 2
+
+
+def test_noalloc_argument_checks_need_no_device(tl):
+    L = tl.lib()
+    p = ctypes.c_void_p(0x10000)
+    call = lambda M=16, N=512, K=512, A=p, B=p, C=p: L.tl_gemm_noalloc(A, B, C, M, N, K, 4096, 16, 128, 0, 0, 0, None, None)
+    assert call(M=0) == 0
+    assert call(M=-1) == 1
+    assert call(N=0) == 1
+
+
+def test_options_and_plan_argument_checks(tl):
+    L = tl.lib()
+    assert L.tl_set_option(99, 0) == 1 and L.tl_get_option(99) == -1
+    assert L.tl_set_option(tl.OPT_PDL, 7) == 1
+    old = tl.get_option(tl.OPT_MAX_STAGES)
+    with tl.option(tl.OPT_MAX_STAGES, 3):
+        assert tl.get_option(tl.OPT_MAX_STAGES) == 3
+    assert tl.get_option(tl.OPT_MAX_STAGES) == old
+    out = tl.GemmPlan()
+    assert L.tl_gemm_plan(16, 512, 512, 4096, 16, 128, 0, 0, 0, 0, 0, None) == 1          # no result buffer
+    assert L.tl_gemm_plan(16, 512, 512, 4096, 16, 128, 0, 0, 0, 0, 5, ctypes.addressof(out)) == 1
+    assert L.tl_gemm_plan(16, 512, 512, 2048, 16, 128, 0, 0, 0, 0, 0, ctypes.addressof(out)) == 1     # G mismatch
+    assert L.tl_gemm_plan(16, 1022, 512, 64, 16, 2, 0, 0, 0, 0, 0, ctypes.addressof(out)) == 2       # N % 4
+    assert L.tl_gemm_last_plan(None) == 1
+
+
+def test_host_threads_may_call_concurrently(tl):
+    # Argument-check paths only (no device here): two threads hammer the entry points, each with its own stream and
+    # workspace settings; every call must return the code the single-threaded call returns.
+    import threading
+    L = tl.lib()
+    p = ctypes.c_void_p(0x10000)
+    bad = []
+
+    def worker(k):
+        L.tl_set_stream(ctypes.c_void_p(0x1000 * (k + 1)))
+        L.tl_set_workspace(ctypes.c_void_p(0x100000 * (k + 1)), 1 << 20)
+        for i in range(3000):
+            if L.tl_gemm(p, p, p, -1, 512, 512, 4096, 16, 128, 0, 0, 0, None) != 1: bad.append(("gemm", k, i))
+            if L.tl_relayout(p, ctypes.c_void_p(0x90000), 60, 64, 2, 2048, 16, 64, 0) != 1: bad.append(("relayout", k, i))
+            if L.tl_set_option(tl.OPT_MAX_STAGES, 2 + (i + k) % 3) != 0: bad.append(("opt", k, i))
+            if not 2 <= L.tl_get_option(tl.OPT_MAX_STAGES) <= 4: bad.append(("get", k, i))
+            if L.tl_set_workspace(ctypes.c_void_p(0x100000 * (k + 1) + 8), 64) != 3: bad.append(("ws", k, i))
+        L.tl_set_workspace(None, 0)
+        L.tl_set_stream(None)
+
+    threads = [threading.Thread(target=worker, args=(k,)) for k in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    L.tl_set_option(tl.OPT_MAX_STAGES, 0)
+    assert not bad, bad[:5]
+
+
 def test_binding_refuses_to_run_without_the_library(tl, monkeypatch):
     monkeypatch.setattr(tl, "_lib", None)
     monkeypatch.setattr(tl, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))

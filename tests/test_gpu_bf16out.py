@@ -17,25 +17,27 @@ SHAPES = [(8, 1024, 2048, (0, 0, 0)),        # decode: stream-K, reduction kerne
 
 @pytest.mark.parametrize("M,N,K,cta", SHAPES)
 def test_one_hot_rows_copy_rows_of_B_exactly(M, N, K, cta):
-    from gpu_util import DEV, tile_major_on_device, tl
+    from gpu_util import DEV, guarded_out, tile_major_on_device, tl
     A, ks = inputs.one_hot_rows(M, K, seed=7)
     B = inputs.bf16_normal((K, N), 0.02, seed=8)
     Bd = tile_major_on_device(B, K, N, 16, 128)
-    C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=DEV)
-    tl.gemm_bf16(A.to(DEV), Bd, C, M, N, K, 4096, 16, 128, cta)
+    g = guarded_out((M, N), torch.bfloat16)
+    tl.gemm_bf16(A.to(DEV), Bd, g.t, M, N, K, 4096, 16, 128, cta)
     tl.device_status()
+    C = g.check()
     assert torch.equal(C.cpu(), B[ks])                   # every value is a bf16 already: the rounding changes nothing
 
 
 @pytest.mark.parametrize("M,N,K,cta", SHAPES)
 def test_random_inputs_are_the_rounded_oracle_product(M, N, K, cta):
-    from gpu_util import DEV, sample_indices, tile_major_on_device, tl
+    from gpu_util import DEV, guarded_out, sample_indices, tile_major_on_device, tl
     A = inputs.bf16_normal((M, K), 1.0, seed=M)
     B = inputs.bf16_normal((K, N), 0.02, seed=N)
     Bd = tile_major_on_device(B, K, N, 16, 128)
-    C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=DEV)
-    tl.gemm_bf16(A.to(DEV), Bd, C, M, N, K, 4096, 16, 128, cta)
+    g = guarded_out((M, N), torch.bfloat16)
+    tl.gemm_bf16(A.to(DEV), Bd, g.t, M, N, K, 4096, 16, 128, cta)
     tl.device_status()
+    C = g.check()
     assert torch.isfinite(C.float()).all()
     ii, jj = sample_indices(M, N, 3000, seed=K)
     ref, S = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), tlo.TILE_MAJOR, 16, 128, M, N, K, ii, jj)
@@ -48,16 +50,17 @@ def test_random_inputs_are_the_rounded_oracle_product(M, N, K, cta):
 
 
 def test_grouped_bf16_output():
-    from gpu_util import DEV, tile_major_on_device, tl
+    from gpu_util import DEV, guarded_out, tile_major_on_device, tl
     E, K, N = 8, 256, 384
     offsets, counts, _ = inputs.zipf_topk_routing(40, E, 3, 1.1, seed=3)
     rows = int(offsets[-1])
     A, ks = inputs.one_hot_rows(rows, K, seed=4)
     B = inputs.bf16_normal((E, K, N), 0.5, seed=5)
     Bt = tile_major_on_device(B.reshape(E * K, N), E * K, N, 16, 128)
-    C = torch.full((rows, N), float("nan"), dtype=torch.bfloat16, device=DEV)
-    tl.gemm_grouped_bf16(A.to(DEV), Bt, C, torch.from_numpy(offsets).to(DEV), E, rows, N, K, 4096, 16, 128)
+    g = guarded_out((rows, N), torch.bfloat16)
+    tl.gemm_grouped_bf16(A.to(DEV), Bt, g.t, torch.from_numpy(offsets).to(DEV), E, rows, N, K, 4096, 16, 128)
     tl.device_status()
+    C = g.check()
     expert = np.searchsorted(offsets, np.arange(rows), side="right") - 1
     want = torch.stack([B[int(e), int(k)] for e, k in zip(expert, ks)])
     assert torch.equal(C.cpu(), want)

@@ -31,10 +31,11 @@ def _run_case(E, hidden, inter, tokens, topk, br, bc, n_check, seed):
         tl.relayout(Wd, Wd_t, E * inter, hidden, 2, G, br, bc, tl.TO_TILE_MAJOR)
     else:
         Wgu_t, Wd_t = Wgu, Wd
-    H = torch.full((rows, inter), float("nan"), dtype=torch.bfloat16, device=DEV)
-    Y = torch.full((rows, hidden), float("nan"), dtype=torch.float32, device=DEV)
-    tl.moe_ffn(X, Wgu_t, Wd_t, H, Y, torch.from_numpy(offsets).to(DEV), E, rows, hidden, inter, G, br, bc)
+    from gpu_util import guarded_out
+    gH, gY = guarded_out((rows, inter), torch.bfloat16), guarded_out((rows, hidden), torch.float32)
+    tl.moe_ffn(X, Wgu_t, Wd_t, gH.t, gY.t, torch.from_numpy(offsets).to(DEV), E, rows, hidden, inter, G, br, bc)
     tl.device_status()
+    H, Y = gH.check(), gY.check()
     assert torch.isfinite(H.float()).all() and torch.isfinite(Y).all()
     rng = np.random.default_rng(seed)
     check = np.unique(np.concatenate([[0, rows - 1], offsets[:-1][counts > 0], rng.integers(0, rows, n_check)]))

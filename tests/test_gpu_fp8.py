@@ -21,11 +21,12 @@ def _weights_nk(B_kn: torch.Tensor, N, K, tile_n, tile_k):
 
 
 def _run(A, W, M, N, K, tile_n, tile_k, cta=(0, 0, 0)):
-    from gpu_util import DEV, tl
-    C = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    from gpu_util import DEV, guarded_out, tl
+    g = guarded_out((M, N), torch.float32)
+    C = g.t
     tl.gemm_fp8_kmajor(A.view(torch.uint8).to(DEV).contiguous(), W, C, M, N, K, tile_n * tile_k, tile_n, tile_k, cta)
     tl.device_status()
-    return C
+    return g.check()
 
 
 TILES = [(64, 64), (32, 128), (16, 256), (128, 32), (8, 512), (0, 0)]        # (64, 64): Figure 1(c)

@@ -254,11 +254,12 @@ def _grouped_case(E, tokens, topk, K, N, br, bc, seed, cta=(0, 0, 0), integer=Fa
         # experts are separate matrices laid end to end: relayout each (equal to one stacked E*K x N relayout)
         tl.relayout(Bd, Bt, E * K, N, 2, br * bc * 2, br, bc, tl.TO_TILE_MAJOR)
         Bd = Bt
-    C = torch.full((rows, N), float("nan"), dtype=torch.float32, device=DEV)
-    tl.gemm_grouped(A.to(DEV), Bd, C, torch.from_numpy(offsets).to(DEV), E, rows, N, K,
+    from gpu_util import guarded_out
+    g = guarded_out((rows, N), torch.float32)
+    tl.gemm_grouped(A.to(DEV), Bd, g.t, torch.from_numpy(offsets).to(DEV), E, rows, N, K,
                     br * bc * 2, br, bc, cta)
     tl.device_status()
-    return offsets, counts, A, Bd, C
+    return offsets, counts, A, Bd, g.check()
 
 
 def _check_grouped(offsets, A, Bd, C, E, K, N, br, bc, samples_per_expert, exact):

@@ -21,11 +21,12 @@ def _weights_nk(B_kn: torch.Tensor, N, K, tile_n, tile_k):
 
 
 def _run(A, W, M, N, K, tile_n, tile_k, cta=(0, 0, 0)):
-    from gpu_util import DEV, tl
-    C = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+    from gpu_util import DEV, guarded_out, tl
+    g = guarded_out((M, N), torch.float32)
+    C = g.t
     tl.gemm_kmajor(A.to(DEV).contiguous(), W, C, M, N, K, tile_n * tile_k * 2, tile_n, tile_k, cta)
     tl.device_status()
-    return C
+    return g.check()
 
 
 TILES = [(32, 64), (16, 128), (8, 256), (64, 64), (1, 2048 // 2), (4, 512), (0, 0), (64, 32), (128, 16)]     # (tile_n, tile_k); (32, 64) = the paper's (a, b) = (64, 32)

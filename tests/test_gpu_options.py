@@ -1,0 +1,331 @@
+"""Code paths behind the library's switches, the plan query, the give-up path and concurrent host threads (GPU).
+
+Every switch selects between two ways of computing the same thing, so each test flips one switch in-process
+(tl_set_option), runs a product or a relayout whose result is exact (integer-valued or one-hot inputs, bytes), and
+compares it with the oracle and with the default path, bit for bit.
+"""
+import threading
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as tlo
+from paper_2607_04031_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+ROW, TILE = tlo.ROW_MAJOR, tlo.TILE_MAJOR
+
+
+def _int_case(M, N, K, br, bc, seed):
+    from gpu_util import DEV, tile_major_on_device
+    A = inputs.bf16_integers((M, K), -8, 8, seed=seed)
+    B = inputs.bf16_integers((K, N), -8, 8, seed=seed + 1)
+    Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
+    want = (A.to(torch.float64) @ B.to(torch.float64)).to(torch.float32)     # exact: integers below 2^24
+    return A, Bd, want
+
+
+def test_one_box_per_memory_tile_gives_the_same_bits():
+    from gpu_util import run_gemm, tl
+    M, N, K = 40, 1024, 1024
+    for br, bc in ((16, 128), (32, 64), (8, 256)):
+        A, Bd, want = _int_case(M, N, K, br, bc, seed=br)
+        with tl.option(tl.OPT_BOX_PER_BLOCK, 1):
+            got = run_gemm(A, Bd, M, N, K, br, bc, (64, 256, 64))          # 2 x 4 memory tiles of 16 x 128 per stage
+            assert tl.get_option(tl.OPT_BOX_PER_BLOCK) == 1
+        assert torch.equal(got.cpu(), want)
+        assert torch.equal(run_gemm(A, Bd, M, N, K, br, bc, (64, 256, 64)).cpu(), want)
+    # random data: same K order on both paths, so the same bits
+    from gpu_util import tile_major_on_device
+    A = inputs.bf16_normal((M, K), 1.0, seed=1)
+    Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=2), K, N, 16, 128)
+    ref = run_gemm(A, Bt, M, N, K, 16, 128)
+    with tl.option(tl.OPT_BOX_PER_BLOCK, 1):
+        assert torch.equal(run_gemm(A, Bt, M, N, K, 16, 128), ref)
+
+
+def test_256_token_pair_tiles_are_what_small_prefill_runs():
+    # M <= 512 with at least 74 pair tiles: too few 512-token tiles to fill a wave of clusters, so the pair kernel
+    # runs its 256-token instantiation by itself (no switch involved).
+    from gpu_util import run_gemm, tl
+    M, N, K = 512, 9728, 256
+    A, Bd, want = _int_case(M, N, K, 16, 128, seed=5)
+    got = run_gemm(A, Bd, M, N, K, 16, 128)
+    plan = tl.gemm_last_plan()
+    assert plan.pair_kernel == 1 and plan.cta_m == 256 and plan.pair_tiles_512 == 0
+    assert torch.equal(got.cpu(), want)
+    A1, ks = inputs.one_hot_rows(M, K, seed=6)
+    B = inputs.bf16_normal((K, N), 0.02, seed=7)
+    from gpu_util import tile_major_on_device
+    assert torch.equal(run_gemm(A1, tile_major_on_device(B, K, N, 16, 128), M, N, K, 16, 128).cpu(), B.float()[ks])
+
+
+@pytest.mark.parametrize("opt_name,value", [("OPT_PAIR_KERNEL", 0), ("OPT_PAIR_512", 0), ("OPT_PDL", 0),
+                                            ("OPT_MAX_STAGES", 2), ("OPT_PREFETCH_STAGES", 0)])
+def test_prefill_switches_give_the_exact_product(opt_name, value):
+    from gpu_util import run_gemm, tl
+    M, N, K = 1800, 5120, 384                      # 512-token tiles and their 256-token remainder by default
+    A, Bd, want = _int_case(M, N, K, 16, 128, seed=11)
+    with tl.option(getattr(tl, opt_name), value):
+        got = run_gemm(A, Bd, M, N, K, 16, 128)
+        plan = tl.gemm_last_plan()
+    assert torch.equal(got.cpu(), want)
+    if opt_name == "OPT_PAIR_KERNEL":
+        assert plan.pair_kernel == 0 and plan.cta == (256, 128, 64)
+    if opt_name == "OPT_PAIR_512":
+        assert plan.pair_kernel == 1 and plan.cta_m == 256
+    if opt_name == "OPT_MAX_STAGES":
+        assert plan.pair_kernel == 1                # the cap applies to the single-CTA kernel only
+
+
+@pytest.mark.parametrize("opt_name,value", [("OPT_UMMA_M128", 1), ("OPT_MAX_STAGES", 2), ("OPT_PREFETCH_STAGES", 0),
+                                            ("OPT_PREFETCH_STAGES", 8), ("OPT_PDL", 0), ("OPT_REDUCE_SPLIT", 0)])
+def test_decode_switches_give_the_same_bits(opt_name, value):
+    from gpu_util import run_gemm, tile_major_on_device, tl
+    for M, N, K in ((8, 2048, 4096), (32, 1024, 8192), (100, 640, 2048)):
+        A = inputs.bf16_normal((M, K), 1.0, seed=M)
+        Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=N), K, N, 16, 128)
+        ref = run_gemm(A, Bt, M, N, K, 16, 128)
+        with tl.option(getattr(tl, opt_name), value):
+            got = run_gemm(A, Bt, M, N, K, 16, 128)
+            if opt_name == "OPT_MAX_STAGES":
+                assert tl.gemm_last_plan().stages == 2
+        assert torch.equal(got, ref), (M, N, K)
+        Ai, Bi, want = _int_case(M, N, K, 16, 128, seed=K)
+        with tl.option(getattr(tl, opt_name), value):
+            assert torch.equal(run_gemm(Ai, Bi, M, N, K, 16, 128).cpu(), want)
+
+
+def test_relayout_without_the_copy_engine_matches_the_oracle():
+    from gpu_util import Guarded, dev_bytes, tl
+    for rows, cols, s, br, bc in ((512, 512, 2, 16, 128), (1056, 2176, 2, 32, 64), (256, 1024, 1, 64, 64)):
+        src = inputs.random_bytes(rows * cols * s, seed=rows + cols)
+        want = tlo.relayout(src, rows, cols, s, br, bc, tlo.TO_TILE_MAJOR)
+        with tl.option(tl.OPT_RELAYOUT_TMA, 0):
+            g = Guarded((rows * cols * s,), torch.uint8)
+            tl.relayout(dev_bytes(src), g.t, rows, cols, s, br * bc * s, br, bc, tl.TO_TILE_MAJOR)
+            assert np.array_equal(g.check().cpu().numpy(), want)
+            gb = Guarded((rows * cols * s,), torch.uint8)
+            tl.relayout(dev_bytes(want), gb.t, rows, cols, s, br * bc * s, br, bc, tl.TO_ROW_MAJOR)
+            assert np.array_equal(gb.check().cpu().numpy(), src)
+            # a batch falls back to one call per matrix
+            g2 = [Guarded((rows * cols * s,), torch.uint8) for _ in range(2)]
+            tl.relayout_batch([dev_bytes(src)] * 2, [x.t for x in g2], [(rows, cols)] * 2, s, br * bc * s, br, bc)
+            for x in g2:
+                assert np.array_equal(x.check().cpu().numpy(), want)
+    tl.device_status()
+
+
+def test_set_option_rejects_what_it_does_not_know():
+    from gpu_util import tl
+    L = tl.lib()
+    assert L.tl_set_option(99, 1) == 1 and L.tl_set_option(-1, 0) == 1
+    assert L.tl_set_option(tl.OPT_PDL, 2) == 1
+    assert L.tl_set_option(tl.OPT_WAIT_LIMIT_US, 5) == 1
+    assert L.tl_set_option(tl.OPT_MAX_STAGES, 1) == 1
+    assert L.tl_get_option(99) == -1
+    assert tl.get_option(tl.OPT_WAIT_LIMIT_US) == 2_000_000
+
+
+# ------------------------------------------------------------------------------------------------ the plan query
+
+PLAN_CASES = [  # M, N, K, block, cta, E, flavour
+    (1, 8192, 8192, (16, 128), (0, 0, 0), 0, 0), (8, 10240, 8192, (16, 128), (0, 0, 0), 0, 0),
+    (32, 57344, 8192, (16, 128), (0, 0, 0), 0, 0), (32, 8192, 28672, (0, 0), (0, 0, 0), 0, 0),
+    (128, 8192, 8192, (32, 64), (128, 128, 64), 0, 0), (16, 8192, 8192, (8, 2), (64, 64, 64), 0, 0),
+    (4096, 8192, 8192, (16, 128), (0, 0, 0), 0, 0), (256, 4096, 2048, (16, 128), (0, 0, 0), 0, 0),
+    (2048, 1536, 2048, (16, 128), (0, 0, 0), 128, 0), (2048, 2048, 768, (16, 128), (0, 0, 0), 128, 0),
+    (8, 10240, 8192, (32, 64), (0, 0, 0), 0, 1), (8, 10240, 8192, (64, 64), (0, 0, 0), 0, 2),
+]
+
+
+@pytest.mark.parametrize("M,N,K,block,cta,E,flavour", PLAN_CASES)
+def test_plan_query_equals_what_the_launch_ran(M, N, K, block, cta, E, flavour):
+    from gpu_util import DEV, tl
+    br, bc = block
+    es = 1 if flavour == 2 else 2
+    G = br * bc * es
+    plan = tl.gemm_plan(M, N, K, G, br, bc, cta, E, flavour)
+    A = torch.zeros((M, K), dtype=torch.uint8 if es == 1 else torch.bfloat16, device=DEV)
+    W = torch.zeros((max(E, 1) * K * N,), dtype=torch.uint8 if es == 1 else torch.bfloat16, device=DEV)
+    C = torch.empty((M, N), dtype=torch.float32, device=DEV)
+    if E:
+        # equal shares of the rows; the schedule on the host side depends on the totals only
+        off = torch.tensor(np.linspace(0, M, E + 1).astype(np.int32), device=DEV)
+        tl.gemm_grouped(A, W, C, off, E, M, N, K, G, br, bc, cta)
+    elif flavour == 0:
+        tl.gemm(A, W, C, M, N, K, G, br, bc, cta)
+    elif flavour == 1:
+        tl.gemm_kmajor(A, W, C, M, N, K, G, br, bc, cta)
+    else:
+        tl.gemm_fp8_kmajor(A, W, C, M, N, K, G, br, bc, cta)
+    tl.device_status()
+    assert tl.gemm_last_plan().as_dict() == plan.as_dict()
+    assert plan.grid >= 1 and plan.stages >= 2
+    if cta != (0, 0, 0):
+        assert plan.cta == cta
+
+
+def test_default_plans_of_the_benchmark_shapes():
+    from gpu_util import tl
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    p = tl.gemm_plan(8, 10240, 8192)
+    assert p.cta == (16, 256, 64) and p.stream_k == 1 and p.grid == sms and p.pair_kernel == 0
+    assert p.workspace_bytes == 2 * sms * 16 * 256 * 4
+    p = tl.gemm_plan(32, 57344, 8192)
+    assert p.cta == (32, 128, 128) and p.stream_k == 1
+    p = tl.gemm_plan(4096, 57344, 8192)
+    assert p.pair_kernel == 1 and p.cta == (512, 128, 64) and p.workspace_bytes == 0 and p.grid % 2 == 0
+    assert 2 * p.pair_tiles_512 + p.pair_tiles_256 == 16 * 224
+
+
+def test_workspace_bound_covers_many_small_experts():
+    # 32 rows over 128 experts: every expert may add a ragged tile, so the grouped grid is far larger than the row
+    # count suggests; the size the header promises for "any number of experts" must cover it.
+    from gpu_util import tl
+    M, N, K, E = 32, 128, 128, 128
+    need = tl.gemm_plan(M, N, K, 4096, 16, 128, (0, 0, 0), E).workspace_bytes
+    assert tl.gemm_workspace_bytes(M, N, K) >= need > 0
+
+
+# ------------------------------------------------------------------------------------------------ giving up
+
+def test_gemm_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
+    # The launch arms its first pipeline stage for 16 bytes more than its copies deliver (test hook): the wait of
+    # the MMA warp on that stage runs out after the shortened limit, every role leaves its loop, the copies in flight
+    # are waited for, tensor memory is freed and the kernel returns.  Nothing faults and nothing waits unbounded.
+    from gpu_util import DEV, run_gemm, tile_major_on_device, tl
+    M, N, K = 16, 512, 512
+    A = inputs.bf16_integers((M, K), -8, 8, seed=1)
+    B = inputs.bf16_integers((K, N), -8, 8, seed=2)
+    Bt = tile_major_on_device(B, K, N, 16, 128)
+    want, _ = tlo.matmul(inputs.bits(A), inputs.bits(Bt.reshape(-1)), TILE, 16, 128, M, N, K)
+    tl.device_status()
+    C = torch.zeros((M, N), dtype=torch.float32, device=DEV)
+    with tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
+        tl.set_option(tl.OPT_STALL_ONCE, 1)
+        tl.gemm(A.to(DEV), Bt, C, M, N, K, 4096, 16, 128)
+        assert tl.get_option(tl.OPT_STALL_ONCE) == 0                     # consumed by that launch
+        with pytest.raises(tl.TileLensError) as e:
+            tl.device_status()
+        # (the MMA warp's wait for the stage, or the epilogue's wait for the accumulator behind it: whichever looked
+        # at the clock first)
+        assert e.value.status == 5 and ("detail=0x200" in str(e.value) or "detail=0x400" in str(e.value))
+    tl.device_status()                                                    # the flag was cleared by the report
+    got = run_gemm(A, Bt, M, N, K, 16, 128)
+    assert np.array_equal(got.cpu().numpy().astype(np.float64), want)
+    # the generic-address path has a second arrival on the same barrier; it gives up the same way
+    Bg = tile_major_on_device(B, K, N, 16, 8)
+    with tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
+        tl.set_option(tl.OPT_STALL_ONCE, 1)
+        tl.gemm(A.to(DEV), Bg, C, M, N, K, 256, 16, 8)
+        with pytest.raises(tl.TileLensError) as e:
+            tl.device_status()
+        assert e.value.status == 5
+    assert np.array_equal(run_gemm(A, Bg, M, N, K, 16, 8).cpu().numpy().astype(np.float64), want)
+
+
+def test_relayout_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
+    from gpu_util import DEV, Guarded, dev_bytes, tl
+    rows, cols, s, br, bc = 512, 512, 2, 16, 128
+    src = inputs.random_bytes(rows * cols * s, seed=3)
+    want = tlo.relayout(src, rows, cols, s, br, bc, tlo.TO_TILE_MAJOR)
+    d_src = dev_bytes(src)
+    tl.device_status()
+    for direction, a, b in ((tl.TO_TILE_MAJOR, d_src, want), (tl.TO_ROW_MAJOR, dev_bytes(want), src)):
+        scratch = torch.zeros(rows * cols * s, dtype=torch.uint8, device=DEV)
+        with tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
+            tl.set_option(tl.OPT_STALL_ONCE, 2)
+            tl.relayout(a, scratch, rows, cols, s, br * bc * s, br, bc, direction)
+            assert tl.get_option(tl.OPT_STALL_ONCE) == 0
+            with pytest.raises(tl.TileLensError) as e:
+                tl.device_status()
+            assert e.value.status == 5 and "detail=0x600" in str(e.value)
+        g = Guarded((rows * cols * s,), torch.uint8)
+        tl.relayout(a, g.t, rows, cols, s, br * bc * s, br, bc, direction)
+        tl.device_status()
+        assert np.array_equal(g.check().cpu().numpy(), b)
+
+
+# ------------------------------------------------------------------------------------------------ PDL ordering
+
+def test_chained_products_wait_for_the_whole_predecessor():
+    # gate_up with K == cta_k has no tile cut along K: no reduction CTA has anything to add.  The down product that
+    # follows in the stream must still see all of H (every reduction CTA waits for the GEMM grid before it leaves).
+    from gpu_util import DEV, tl
+    E, hidden, inter = 16, 128, 512
+    offsets, counts, _ = inputs.zipf_topk_routing(96, E, 4, 1.1, seed=4)
+    rows = int(offsets[-1])
+    X = inputs.bf16_normal((rows, hidden), 1.0, seed=1, device=DEV)
+    Wgu = inputs.bf16_normal((E, hidden, 2 * inter), 0.05, seed=2, device=DEV)
+    Wd = inputs.bf16_normal((E, inter, hidden), 0.05, seed=3, device=DEV)
+    Wgu_t, Wd_t = torch.empty_like(Wgu), torch.empty_like(Wd)
+    tl.relayout(Wgu, Wgu_t, E * hidden, 2 * inter, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    tl.relayout(Wd, Wd_t, E * inter, hidden, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    d_off = torch.from_numpy(offsets).to(DEV)
+
+    def chain():
+        H = torch.zeros((rows, inter), dtype=torch.bfloat16, device=DEV)
+        Y = torch.full((rows, hidden), float("nan"), dtype=torch.float32, device=DEV)
+        for _ in range(20):                                   # back to back, so that launches overlap their ends
+            H.zero_()
+            tl.moe_ffn(X, Wgu_t, Wd_t, H, Y, d_off, E, rows, hidden, inter, 4096, 16, 128)
+        tl.device_status()
+        return H.clone(), Y.clone()
+
+    H1, Y1 = chain()
+    with tl.option(tl.OPT_PDL, 0):
+        H0, Y0 = chain()
+    assert torch.equal(H1, H0) and torch.equal(Y1, Y0)
+    check = np.arange(rows)
+    Hr, Yr, Sr = tlo.moe_ffn_rows(inputs.bits(X), inputs.bits(Wgu_t.reshape(-1)), inputs.bits(Wd_t.reshape(-1)), offsets,
+                                  hidden, inter, tlo.TILE_MAJOR, 16, 128, check)
+    assert np.all(np.abs(Y1.cpu().numpy().astype(np.float64) - Yr) <= 2e-2 * Sr + 1e-6)      # h itself is bf16-rounded
+
+
+# ------------------------------------------------------------------------------------------------ host threads
+
+def test_two_host_threads_with_their_own_streams_and_workspaces():
+    from gpu_util import DEV, tile_major_on_device, tl
+    shapes = [(8, 1280, 4096), (32, 2048, 2304)]
+    A, Bt, want = [], [], []
+    for i, (M, N, K) in enumerate(shapes):
+        A.append(inputs.bf16_normal((M, K), 1.0, seed=60 + i).to(DEV))
+        Bt.append(tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=70 + i), K, N, 16, 128))
+        C = torch.empty((M, N), dtype=torch.float32, device=DEV)
+        tl.gemm(A[i], Bt[i], C, M, N, K, 4096, 16, 128)
+        want.append(C)
+    tl.device_status()
+    errors, results = [], [None, None]
+
+    def worker(i):
+        try:
+            torch.cuda.set_device(0)
+            M, N, K = shapes[i]
+            stream = torch.cuda.Stream(device=DEV)
+            ws = torch.empty(tl.gemm_workspace_bytes(M, N, K) + 256, dtype=torch.uint8, device=DEV)
+            tl.set_workspace(ws)                               # this thread's workspace and stream only
+            tl.set_stream(stream)
+            outs = []
+            for rep in range(40):
+                C = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+                tl.gemm(A[i], Bt[i], C, M, N, K, 4096, 16, 128, stream=stream)
+                outs.append(C)
+            stream.synchronize()
+            results[i] = outs
+            tl.set_workspace(None)
+        except Exception as exc:                               # noqa: BLE001 -- reported by the main thread
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    for i in range(2):
+        for C in results[i]:
+            assert torch.equal(C, want[i])
+    tl.device_status()

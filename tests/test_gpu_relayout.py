@@ -34,23 +34,24 @@ CASES = [  # rows, cols, s, br, bc
 
 @pytest.mark.parametrize("rows,cols,s,br,bc", CASES)
 def test_both_directions_match_oracle(rows, cols, s, br, bc):
-    from gpu_util import DEV, dev_bytes, tl
+    from gpu_util import DEV, Guarded, dev_bytes, tl
     G = br * bc * s
     src = inputs.random_bytes(rows * cols * s, seed=rows + 7 * cols + s)
     want = tlo.relayout(src, rows, cols, s, br, bc, tlo.TO_TILE_MAJOR)
     d_src = dev_bytes(src)
-    d_dst = torch.zeros_like(d_src)
-    tl.relayout(d_src, d_dst, rows, cols, s, G, br, bc, tl.TO_TILE_MAJOR)
+    g_dst = Guarded((rows * cols * s,), torch.uint8)       # outputs sit between guard blocks, checked after the call
+    tl.relayout(d_src, g_dst.t, rows, cols, s, G, br, bc, tl.TO_TILE_MAJOR)
+    d_dst = g_dst.check()
     got = d_dst.cpu().numpy()
     assert np.array_equal(got, want)
-    d_back = torch.zeros_like(d_src)
-    tl.relayout(d_dst, d_back, rows, cols, s, G, br, bc, tl.TO_ROW_MAJOR)
-    assert np.array_equal(d_back.cpu().numpy(), src)
+    g_back = Guarded((rows * cols * s,), torch.uint8)
+    tl.relayout(d_dst, g_back.t, rows, cols, s, G, br, bc, tl.TO_ROW_MAJOR)
+    assert np.array_equal(g_back.check().cpu().numpy(), src)
     # the inverse direction on its own, from the oracle's tile-major bytes
     d_t = dev_bytes(want)
-    d_r = torch.zeros_like(d_t)
-    tl.relayout(d_t, d_r, rows, cols, s, G, br, bc, tl.TO_ROW_MAJOR)
-    assert np.array_equal(d_r.cpu().numpy(), tlo.relayout(want, rows, cols, s, br, bc, tlo.TO_ROW_MAJOR))
+    g_r = Guarded((rows * cols * s,), torch.uint8)
+    tl.relayout(d_t, g_r.t, rows, cols, s, G, br, bc, tl.TO_ROW_MAJOR)
+    assert np.array_equal(g_r.check().cpu().numpy(), tlo.relayout(want, rows, cols, s, br, bc, tlo.TO_ROW_MAJOR))
 
 
 def test_unaligned_pointers_take_the_elementwise_path():
@@ -93,20 +94,21 @@ def test_errors():
 @pytest.mark.parametrize("direction", [0, 1])
 def test_batch_of_matrices_in_one_launch_matches_oracle(direction):
     # eleven matrices of unequal shapes: a run of eight in one launch, then three; the tile is 16 x 128 bf16
-    from gpu_util import DEV, tl
+    from gpu_util import DEV, Guarded, tl
     br, bc, s = 16, 128, 2
     shapes = [(512, 512), (1056, 2176), (16, 128), (48, 1280), (2048, 256), (32, 8192), (640, 384), (16, 256),
               (4096, 128), (64, 1024), (528, 640)]
-    srcs, dsts, wants = [], [], []
+    srcs, guards, wants = [], [], []
     for i, (rows, cols) in enumerate(shapes):
         host = inputs.random_bytes(rows * cols * s, seed=100 + i)
         srcs.append(torch.from_numpy(host).to(DEV))
-        dsts.append(torch.full_like(srcs[-1], 0xEE))
+        guards.append(Guarded((rows * cols * s,), torch.uint8))
+        guards[-1].t.fill_(0xEE)
         wants.append(tlo.relayout(host, rows, cols, s, br, bc, direction))
-    tl.relayout_batch(srcs, dsts, shapes, s, br * bc * s, br, bc, direction)
+    tl.relayout_batch(srcs, [g.t for g in guards], shapes, s, br * bc * s, br, bc, direction)
     tl.device_status()
-    for i, (d, w) in enumerate(zip(dsts, wants)):
-        assert np.array_equal(d.cpu().numpy(), w), shapes[i]
+    for i, (g, w) in enumerate(zip(guards, wants)):
+        assert np.array_equal(g.check().cpu().numpy(), w), shapes[i]
 
 
 def test_batch_falls_back_per_matrix_and_reports_argument_errors():

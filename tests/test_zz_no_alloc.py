@@ -9,9 +9,11 @@ keeps the first call's contents, so the second call proves the clean-up), and th
 problems whose scratch does not fit.  It is collected last so that a failure here cannot hide
 another test's result; it does not depend on any other test having run.
 """
+import numpy as np
 import pytest
 import torch
 
+import oracle as tlo
 from paper_2607_04031_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -38,11 +40,24 @@ def test_matches_tl_gemm_on_two_calls_in_a_row(M, N, K, integer):
     tl.gemm(A, Bt, want, M, N, K, 4096, 16, 128)          # existing entry point (allocating workspace)
     tl.device_status()
     flag = torch.zeros(1, dtype=torch.int32, device=DEV)
+    # against the oracle directly (exact integers), not only against the other entry point
+    exact = None
+    if integer:
+        exact, _ = tlo.matmul(inputs.bits(A), inputs.bits(Bt.reshape(-1)), tlo.TILE_MAJOR, 16, 128, M, N, K)
+    outs = [torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV) for _ in range(2)]
     for call in range(2):
-        got = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+        got = outs[call]
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         tl.gemm_noalloc(A, Bt, got, M, N, K, 4096, 16, 128, timeout_flag=flag)
         torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        if call == 1:
+            # the second call cannot even have loaded a module: the device's free memory is what it was
+            assert free_after == free_before, "tl_gemm_noalloc changed the amount of free device memory"
         assert int(flag.item()) == 0, "a bounded wait expired inside the kernel"
+        if exact is not None:
+            assert np.array_equal(got.cpu().numpy().astype(np.float64), exact), f"call {call} against the oracle"
         # Same kernel; the fixed scratch may make the library pick a narrower tile, hence another split of
         # the K sums.  Integer inputs are exact in any order; otherwise both results lie within the GEMM
         # tests' tolerance of 1e-3 * sum|a b| of the true product, so within twice that of each other.
@@ -62,6 +77,23 @@ def test_matches_tl_gemm_on_two_calls_in_a_row(M, N, K, integer):
     torch.cuda.synchronize()
     assert torch.equal(got2, want2)
     assert torch.equal(got, want) if integer else bool(((got - want).abs() <= 2e-3 * S).all())
+
+
+def test_large_products_that_need_no_scratch_are_not_refused():
+    # Prefill-sized products run on CTA pairs, which keep nothing in scratch memory: the size limit of the fixed
+    # array does not apply to them, whatever the split-K plan of the single-CTA kernel would have asked for.
+    from gpu_util import DEV, tile_major_on_device, tl
+    M, N, K = 1800, 5120, 384
+    A = inputs.bf16_integers((M, K), -8, 8, seed=3)
+    B = inputs.bf16_integers((K, N), -8, 8, seed=4)
+    Bt = tile_major_on_device(B, K, N, 16, 128)
+    want = (A.to(torch.float64) @ B.to(torch.float64)).to(torch.float32)
+    for call in range(2):
+        got = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+        tl.gemm_noalloc(A.to(DEV), Bt, got, M, N, K, 4096, 16, 128)
+        torch.cuda.synchronize()
+        assert tl.gemm_last_plan().pair_kernel == 1
+        assert torch.equal(got.cpu(), want), f"call {call}"
 
 
 def test_refuses_scratch_beyond_the_fixed_array():
