@@ -48,7 +48,7 @@ NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 167.99 MB read + 4.8
 def default_cta(M):
     """CTA tile (token rows, weight columns, weight rows per stage) of the library's decode schedule.  The CPU arm
     may not call the CUDA library, so it counts with these; run_ours() checks them against tl_gemm_plan."""
-    return (16, 256, 64) if M <= 16 else (32, 128, 128)
+    return (16 if M <= 16 else 32, 256, 64)
 
 
 def config_dict(world=1):

@@ -95,6 +95,10 @@ typedef enum {
                                 That launch's output is undefined.  The option resets itself to 0 when it is consumed. */
     TL_OPT_MOE_ROW_CAP,      /* grouped products: most token rows per tile; 0 (default): the library's choice, else 16/32/64/128 */
     TL_OPT_REDUCE_SPLIT,     /* 1 (default): a split tile's partial sums are added by all reduction CTAs inside it, 0: by one */
+    TL_OPT_SM_LIMIT,         /* 0 (default): GEMM grids use every SM; n > 0: at most n CTAs (leaves SMs to concurrent work) */
+    TL_OPT_NO_SCRATCH_PLANS, /* 1 (default): dense decode-sized products prefer schedules without partial tiles in global
+                                memory (whole tiles on a grid that divides the tile count, or split-K inside clusters);
+                                0: always the stream-K cut */
     TL_OPT_COUNT_
 } tl_option;
 /* TL_ERR_INVALID_ARG for an unknown option or a value outside the option's range. */
@@ -280,7 +284,8 @@ typedef struct tl_gemm_plan_info {
     int32_t stages;                /* pipeline depth */
     int32_t weights_on_n;          /* 1: weights on the N side of the MMA (token tiles of up to 128 rows) */
     int32_t generic_path;          /* 1: weights loaded by the generic-address path of Section 4.4 */
-    int32_t reserved;
+    int32_t cluster_k;             /* S > 1: one tile per cluster of S CTAs that split its K loop (sums through distributed
+                                      shared memory, no workspace); else 1 */
     int64_t pair_tiles_512, pair_tiles_256;   /* pair kernel: tiles of 512 and of 256 token rows (x 256 columns) */
     uint64_t workspace_bytes;      /* split-K scratch the launch uses */
 } tl_gemm_plan_info;

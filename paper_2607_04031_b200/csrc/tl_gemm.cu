@@ -229,6 +229,7 @@ struct GemmPlan {
     int umma_m, a_rows;          // see GemmParams
     int weights_on_n;     // kWN variant of the kernel
     int stream_k;
+    int cluster_k;        // > 1: clusters of that many CTAs split the K loop of one tile each (no scratch)
     int grid;
     int num_stages;
     size_t smem_bytes;
@@ -243,10 +244,11 @@ static int pick_bm(int64_t rows) {
 
 // Chooses / validates the CTA tile and the schedule.  rows_max: most rows any one problem has.
 // Default CTA tile (measured on B200, Llama-70B and Qwen-30B shapes).
-//   up to 16 rows      16 x 256 x 64: tokens on the MMA's M side, 256 weight columns per instruction; the
-//                      partial tiles of stream-K are still small (16 KB)
-//   up to 128 rows     rows x 128 x 128: same orientation, narrower tile so that partial tiles stay small,
-//                      deeper K step so that there are half as many barrier hand-offs
+//   up to 64 rows      rows x 256 x 64: tokens on the MMA's M side, 256 weight columns (8 KB of weights) per
+//                      instruction; few enough tiles that a no-scratch schedule exists for the usual shapes (see
+//                      make_plan)
+//   up to 128 rows     128 x 128 x 128: same orientation, deeper K step so that there are half as many barrier
+//                      hand-offs
 //   more rows          256 x 128 x 64 with the weights on the M side (prefill)
 //   grouped            at most 32 rows per tile: most experts have a handful of rows, and a large cap costs
 //                      pipeline stages and partial-tile bytes for every tile
@@ -254,15 +256,16 @@ static int pick_bm(int64_t rows) {
 static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, int* BM, int* BN, int* BK) {
     *BM = pick_bm(rows_max);
     if (grouped && *BM > 32) *BM = 32;
-    if (*BM <= 16 && !narrow_scratch && !grouped) { *BN = 256; *BK = 64; }
+    if (*BM <= 64 && !narrow_scratch && !grouped) { *BN = 256; *BK = 64; }
     else if (*BM <= 128) { *BN = 128; *BK = 128; }
     else { *BN = 128; *BK = 64; }
 }
 
 static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
-                     bool grouped, GemmPlan* plan, bool narrow_scratch = false) {
+                     bool grouped, GemmPlan* plan, bool narrow_scratch = false, bool generic = false) {
     if (int rc = ensure_device_info()) return rc;
-    const int sms = dev().sm_count;
+    int sms = dev().sm_count;
+    if (opt(TL_OPT_SM_LIMIT) > 0 && opt(TL_OPT_SM_LIMIT) < sms) sms = int(opt(TL_OPT_SM_LIMIT));
     int BM = cta_m, BN = cta_n, BK = cta_k;
     if (BM == 0 && BN == 0 && BK == 0) default_tile(rows_max, grouped, narrow_scratch, &BM, &BN, &BK);
     if (BM != 16 && BM != 32 && BM != 64 && BM != 128 && BM != 256) return TL_ERR_UNSUPPORTED;
@@ -297,7 +300,34 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     const int64_t waves = ceil_div(tile_bound, sms);
     const bool even = tile_bound >= sms && double(tile_bound) / double(waves * sms) >= 0.92;
     plan->stream_k = (grouped || !even) ? 1 : 0;
+    plan->cluster_k = 1;
     int64_t grid = plan->stream_k ? (total_iters < sms ? total_iters : sms) : (tile_bound < sms ? tile_bound : sms);
+    // Dense decode-sized products: a schedule without partial tiles in global memory beats the stream-K cut even
+    // when it leaves some SMs idle, because 110 to 130 CTAs already stream at the rate of the whole device
+    // (measured: Llama gate_up, M = 8, 224 whole tiles on 112 CTAs 135 us, cut over 148 CTAs 142 us).  In order:
+    //   1. whole tiles on the largest grid of at least 3/4 of the SMs that divides the tile count;
+    //   2. one tile per cluster of S <= 8 CTAs which split its K loop S ways and add their partial tiles through
+    //      distributed shared memory, for the S that fills most SMs (at least 3/4 of them);
+    //   3. the stream-K cut with its workspace and reduction kernel.
+    if (plan->stream_k && !grouped && plan->weights_on_n && !generic && opt(TL_OPT_NO_SCRATCH_PLANS) != 0) {
+        const int64_t lo = (3 * int64_t(sms) + 3) / 4;
+        int64_t g1 = 0;
+        for (int64_t g = tile_bound < sms ? tile_bound : sms; g >= lo; --g)
+            if (tile_bound % g == 0) { g1 = g; break; }
+        int best_s = 0;
+        for (int s = 2; s <= 8; ++s)
+            if (tile_bound * s <= sms && tile_bound * s >= lo && k_iters >= s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024 &&
+                tile_bound * s > int64_t(best_s) * tile_bound)
+                best_s = s;
+        if (g1 > 0) {
+            plan->stream_k = 0;
+            grid = g1;
+        } else if (best_s > 0) {
+            plan->stream_k = 0;
+            plan->cluster_k = best_s;
+            grid = tile_bound * best_s;
+        }
+    }
     if (grid < 1) grid = 1;
     plan->grid = int(grid);
     plan->ws_bytes = plan->stream_k ? size_t(2) * size_t(grid) * BM * BN * sizeof(float) : 0;   // two slots per CTA
@@ -376,7 +406,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         const int64_t mt_bound = d_offsets ? rows_total / bm_guess + E : ceil_div(rows_total, bm_guess);
         // (the plan counts K in 2-byte units: an 8-bit stage holds twice as many elements)
         if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                               d_offsets != nullptr, &plan, fixed != nullptr))
+                               d_offsets != nullptr, &plan, fixed != nullptr, generic))
             return rc;
     }
     if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
@@ -622,6 +652,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.n_tiles = int(ceil_div(N, plan.BN));
     p.k_iters = int(ceil_div(K, int64_t(plan.BK) << k_shift));
     p.stream_k = plan.stream_k;
+    p.cluster_k = plan.cluster_k;
     p.num_stages = plan.num_stages;
     const int prefetch_env = int(opt(TL_OPT_PREFETCH_STAGES));   // measurement switch, -1: the default below
     // (at most four instructions: the thread that issues them holds up the CTA's first barrier for their duration)
@@ -632,7 +663,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     memset(&info, 0, sizeof info);
     info.cta_m = plan.BM; info.cta_n = plan.BN; info.cta_k = plan.BK << k_shift;
     info.stream_k = plan.stream_k; info.grid = plan.grid; info.stages = plan.num_stages;
-    info.weights_on_n = plan.weights_on_n; info.generic_path = generic ? 1 : 0;
+    info.weights_on_n = plan.weights_on_n; info.generic_path = generic ? 1 : 0; info.cluster_k = plan.cluster_k;
     info.workspace_bytes = plan.ws_bytes;
     // Large dense problems on TMA-readable weights: CTA pairs (cta_group::2 MMAs), see tl_gemm_pair.cuh.
     const bool no_pair = opt(TL_OPT_PAIR_KERNEL) == 0;     // measurement switch
@@ -674,7 +705,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     if (opt(TL_OPT_LOG))
         fprintf(stderr, "[tilelens] gemm kernel: cta %d x %d x %d, weights on %s, %s, grid %d, %d stages, %zu B workspace%s\n",
-                info.cta_m, info.cta_n, info.cta_k, plan.weights_on_n ? "N" : "M", plan.stream_k ? "stream-K" : "whole tiles",
+                info.cta_m, info.cta_n, info.cta_k, plan.weights_on_n ? "N" : "M",
+                plan.stream_k ? "stream-K" : plan.cluster_k > 1 ? "cluster split-K" : "whole tiles",
                 plan.grid, plan.num_stages, plan.ws_bytes, generic ? ", generic-address weights" : "");
     if (plan_only) { *plan_only = info; return TL_OK; }
     last_plan() = info;
@@ -703,11 +735,22 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         cfg.blockDim = dim3(generic ? kGenericThreads : kGemmThreads);
         cfg.dynamicSmemBytes = plan.smem_bytes;
         cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchAttribute attr[2];
+        int n_attr = 0;
+        if (pdl_ok) {
+            attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+            ++n_attr;
+        }
+        if (plan.cluster_k > 1) {
+            attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+            attr[n_attr].val.clusterDim.x = unsigned(plan.cluster_k);
+            attr[n_attr].val.clusterDim.y = 1;
+            attr[n_attr].val.clusterDim.z = 1;
+            ++n_attr;
+        }
         cfg.attrs = attr;
-        cfg.numAttrs = pdl_ok ? 1 : 0;
+        cfg.numAttrs = n_attr;
         if (plan.weights_on_n) rc = es == 1 ? launch_gemm_wn_fp8(plan.BK, plan.BN, &cfg, p) : launch_gemm_wn_bf16(plan.BK, plan.BN, &cfg, p);
         else rc = es == 1 ? launch_gemm_wm_fp8(plan.BK, plan.BN, &cfg, p) : launch_gemm_wm_bf16(plan.BK, plan.BN, &cfg, p);
         if (rc) return rc;

@@ -36,6 +36,9 @@ struct alignas(64) GemmParams {
     int BN;                     // weight columns per CTA tile: 128 or 256
     int n_tiles, k_iters;
     int stream_k;               // 0: whole tiles round-robin, 1: contiguous K-iteration ranges
+    int cluster_k;              // S > 1: launched in clusters of S CTAs; cluster c owns output tile c, CTA rank r of it the
+                                // r-th of S equal parts of the K loop; the partial tiles are added through distributed
+                                // shared memory (no workspace, no reduction kernel).  Dense, weights-on-N kernels only.
     int num_stages;
     int prefetch_stages;        // stages of weights each CTA asks into L2 before it waits for its predecessor
     int pair_big_tiles;         // pair kernel with 512-token tiles: how many tiles are of that size (the rest 256)
@@ -99,6 +102,14 @@ struct Sched {
         return tab ? tab[c] : split(static_cast<long long>(tiles_total) * k_iters, grid_eff, c);
     }
     __device__ static int effective_grid(long long total, int grid) { return total < grid ? static_cast<int>(total) : grid; }
+    // Cluster split-K: the one work item of this CTA (tile = cluster index, the rank's share of the K loop).
+    __device__ void init_cluster(int k_iters_, int tiles_total_, int cluster, int rank, int size) {
+        stream_k = 2; k_iters = k_iters_; tiles_total = tiles_total_; cta = cluster; tab = nullptr; grid_eff = 0;
+        next_tile = cluster;
+        it_begin = it = static_cast<long long>(k_iters_) * rank / size;
+        it_end = static_cast<long long>(k_iters_) * (rank + 1) / size;
+        if (cluster >= tiles_total_) it_end = it;
+    }
     __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid, int cta_, const int* tab_) {
         stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_; tab = tab_;
         grid_eff = effective_grid(static_cast<long long>(tiles_total) * k_iters, grid);
@@ -115,6 +126,11 @@ struct Sched {
             return true;
         }
         if (it >= it_end) return false;
+        if (stream_k == 2) {
+            w.tile = next_tile; w.kbeg = static_cast<int>(it); w.kend = static_cast<int>(it_end);
+            it = it_end;
+            return true;
+        }
         int t = static_cast<int>(it / k_iters);
         int kb = static_cast<int>(it - static_cast<long long>(t) * k_iters);
         long long left = it_end - it;
@@ -288,6 +304,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     constexpr int kKSteps = kBK / 16;
     constexpr int kSubK = kBK / 64;                        // token boxes per stage
     constexpr uint32_t kWBytes = kBK * kBN * 2;            // weight bytes per stage
+    constexpr int kStagePitch = kBN + 4;                   // floats between rows of a partial tile kept in shared memory
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
@@ -321,32 +338,6 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     if (warp == 1) {
         tmem_alloc(&tmem_slot, tmem_cols);
         tmem_relinquish();
-    }
-    // Dense stream-K problems: while the kernel before this one in the stream is still finishing, ask for the
-    // first stages of this CTA's weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is
-    // the point of coherence, so this is safe whatever that kernel is still writing; it takes the cold start
-    // (page walks, first DRAM accesses) off this kernel's critical path.
-    // (issued by an epilogue thread, which has nothing else to do yet, so that the producer is not held up)
-    if (threadIdx.x == 64 && p.stream_k && !p.generic_b && p.offsets == nullptr && p.prefetch_stages > 0) {
-        const int mt = (p.M + p.BM - 1) / p.BM;
-        const long long total = static_cast<long long>(mt) * p.n_tiles * p.k_iters;
-        const int geff = Sched::effective_grid(total, gridDim.x);
-        if (int(blockIdx.x) < geff) {
-            long long it = Sched::split(total, geff, blockIdx.x);
-            const long long it_end = Sched::split(total, geff, blockIdx.x + 1);
-            for (int s = 0; s < p.prefetch_stages && it < it_end; ++s, ++it) {
-                const int tile = int(it / p.k_iters), kit = int(it - static_cast<long long>(tile) * p.k_iters);
-                const int n0 = (tile / mt) * p.BN;
-                const int kq = ((tile % mt) & 1) ? p.k_iters - 1 - kit : kit;      // odd m-tiles walk K backwards
-                const int k0 = (kq * kBK) << p.k_shift;
-                for (int kb = 0; kb < p.kbx; ++kb)
-                    for (int nb = 0; nb < p.nbx; ++nb) {
-                        int c[5];
-                        weight_box_coords(p, k0 + kb * p.box_rows, n0 + nb * p.box_atoms * 64, 0, c);
-                        tma_prefetch_5d(&p.tmap_b, c[0], c[1], c[2], c[3], c[4]);
-                    }
-            }
-        }
     }
     // Token rows between BM and the rows the MMA reads are zeroed once; no copy ever writes them.  (The MMA's token
     // side has at least 64 rows.  Whatever lies there is multiplied with the weights at full rate, and with stale
@@ -388,11 +379,34 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         __syncthreads();
     }
     Sched sched;
-    sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
+    if (p.cluster_k > 1) sched.init_cluster(p.k_iters, tiles_total, int(cluster_id_x()), int(cluster_cta_rank()), p.cluster_k);
+    else sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
+    // Dense problems: while the kernel before this one in the stream is still finishing, ask for the first stages
+    // of this CTA's weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is the point of
+    // coherence, so this is safe whatever that kernel is still writing; it takes the cold start (page walks, first
+    // DRAM accesses) off this kernel's critical path.
+    // (issued by an epilogue thread, which has nothing else to do yet, so that the producer is not held up)
+    if (threadIdx.x == 64 && tables_first && !p.generic_b && p.prefetch_stages > 0) {
+        Sched first = sched;
+        Work w;
+        if (first.next(w)) {
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+            for (int s = 0, kit = w.kbeg; s < p.prefetch_stages && kit < w.kend; ++s, ++kit) {
+                const int kq = t.flip ? p.k_iters - 1 - kit : kit;
+                const int k0 = (kq * kBK) << p.k_shift;
+                for (int kb = 0; kb < p.kbx; ++kb)
+                    for (int nb = 0; nb < p.nbx; ++nb) {
+                        int c[5];
+                        weight_box_coords(p, k0 + kb * p.box_rows, t.n0 + nb * p.box_atoms * 64, 0, c);
+                        tma_prefetch_5d(&p.tmap_b, c[0], c[1], c[2], c[3], c[4]);
+                    }
+            }
+        }
+    }
     if (tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
-    // Stream-K: let the reduction kernel that follows in the stream be scheduled already; it does its own
-    // set-up and then blocks until this whole grid has finished.
-    if (p.stream_k && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Let the kernel that follows in the stream (the stream-K reduction, or the next product) be scheduled already:
+    // it does its own set-up and then blocks until this whole grid has finished.
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     volatile uint32_t* abort_ptr = &abort_flag;
 
     if (warp == 0) {
@@ -591,6 +605,11 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
             if (full) {
                 out = p.C + int64_t(t.row0) * p.ldc + t.n0;
                 ld = p.ldc;
+            } else if (p.cluster_k > 1) {
+                // cluster split-K: the partial tile stays in this CTA's shared memory (the pipeline's stages are
+                // free: this CTA has one work item and its last MMA has completed), rows kStagePitch floats apart
+                out = reinterpret_cast<float*>(stages);
+                ld = kStagePitch;
             } else {
                 out = p.partials + size_t(sched.slot(sched.cta, w.tile)) * p.BM * kBN;
                 ld = kBN;
@@ -708,6 +727,50 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     // --------------------------------------------------------------- teardown
     tc_fence_before_sync();
     __syncthreads();
+    if (kWN && p.cluster_k > 1) {
+        // Cluster split-K: every CTA of the cluster holds its share of the K sum of the same tile in its shared
+        // memory.  CTA rank r adds the r-th share of the tile's 16-byte vectors over all ranks, in rank (= K) order,
+        // reading the peers' copies through distributed shared memory, and writes C.  The first barrier makes the
+        // partial tiles visible cluster-wide; after the second nobody reads a peer's memory any more.  All threads
+        // of all CTAs reach both (every wait before this point is bounded).
+        cluster_sync();
+        if (warp >= 2 && warp < 6 && !*abort_ptr) {
+            const int S = p.cluster_k, rank = int(cluster_cta_rank());
+            const int tile = int(cluster_id_x());
+            if (tile < tiles_total) {
+                const TileInfo t = decode_tile(p, prefix, row_start, tile);
+                constexpr int kVecPerRow = kBN / 4;
+                const int total_vec = t.rows * kVecPerRow;
+                const int v_begin = int(static_cast<long long>(total_vec) * rank / S);
+                const int v_end = int(static_cast<long long>(total_vec) * (rank + 1) / S);
+                const uint32_t base = smem_u32(stages);
+                for (int v = v_begin + (int(threadIdx.x) - 64); v < v_end; v += 128) {
+                    const int r = v / kVecPerRow, c4 = (v % kVecPerRow) * 4;
+                    const uint32_t local = base + uint32_t(r * kStagePitch + c4) * 4u;
+                    float4 x[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < S) x[j] = ld_cluster_f4(map_to_cta(local, uint32_t(j)));
+                    float4 sum = x[0];
+#pragma unroll
+                    for (int j = 1; j < 8; ++j)
+                        if (j < S) { sum.x += x[j].x; sum.y += x[j].y; sum.z += x[j].z; sum.w += x[j].w; }
+                    if (t.n0 + c4 < p.N) {
+                        if (p.Cb) {
+                            const uint32_t lo = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum.x))) |
+                                                (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum.y))) << 16);
+                            const uint32_t hi = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum.z))) |
+                                                (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum.w))) << 16);
+                            *reinterpret_cast<uint2*>(p.Cb + int64_t(t.row0 + r) * p.ldc + t.n0 + c4) = make_uint2(lo, hi);
+                        } else {
+                            *reinterpret_cast<float4*>(p.C + int64_t(t.row0 + r) * p.ldc + t.n0 + c4) = sum;
+                        }
+                    }
+                }
+            }
+        }
+        cluster_sync();
+    }
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, tmem_cols);

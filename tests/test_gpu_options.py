@@ -79,22 +79,61 @@ def test_prefill_switches_give_the_exact_product(opt_name, value):
         assert plan.pair_kernel == 1                # the cap applies to the single-CTA kernel only
 
 
+@pytest.mark.parametrize("no_scratch", [1, 0])
 @pytest.mark.parametrize("opt_name,value", [("OPT_UMMA_M128", 1), ("OPT_MAX_STAGES", 2), ("OPT_PREFETCH_STAGES", 0),
                                             ("OPT_PREFETCH_STAGES", 8), ("OPT_PDL", 0), ("OPT_REDUCE_SPLIT", 0)])
-def test_decode_switches_give_the_same_bits(opt_name, value):
+def test_decode_switches_give_the_same_bits(opt_name, value, no_scratch):
+    # no_scratch = 1: the library's own choice (cluster split-K or whole tiles where such a plan exists);
+    # no_scratch = 0: the stream-K cut with its reduction kernel.  A switch never changes the bits of either.
     from gpu_util import run_gemm, tile_major_on_device, tl
-    for M, N, K in ((8, 2048, 4096), (32, 1024, 8192), (100, 640, 2048)):
-        A = inputs.bf16_normal((M, K), 1.0, seed=M)
-        Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=N), K, N, 16, 128)
-        ref = run_gemm(A, Bt, M, N, K, 16, 128)
-        with tl.option(getattr(tl, opt_name), value):
-            got = run_gemm(A, Bt, M, N, K, 16, 128)
-            if opt_name == "OPT_MAX_STAGES":
-                assert tl.gemm_last_plan().stages == 2
-        assert torch.equal(got, ref), (M, N, K)
-        Ai, Bi, want = _int_case(M, N, K, 16, 128, seed=K)
-        with tl.option(getattr(tl, opt_name), value):
-            assert torch.equal(run_gemm(Ai, Bi, M, N, K, 16, 128).cpu(), want)
+    with tl.option(tl.OPT_NO_SCRATCH_PLANS, no_scratch):
+        for M, N, K in ((8, 2048, 4096), (32, 1024, 8192), (100, 640, 2048), (16, 8192, 2048)):
+            A = inputs.bf16_normal((M, K), 1.0, seed=M)
+            Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=N), K, N, 16, 128)
+            ref = run_gemm(A, Bt, M, N, K, 16, 128)
+            with tl.option(getattr(tl, opt_name), value):
+                got = run_gemm(A, Bt, M, N, K, 16, 128)
+                if opt_name == "OPT_MAX_STAGES":
+                    assert tl.gemm_last_plan().stages == 2
+            assert torch.equal(got, ref), (M, N, K)
+            Ai, Bi, want = _int_case(M, N, K, 16, 128, seed=K)
+            with tl.option(getattr(tl, opt_name), value):
+                assert torch.equal(run_gemm(Ai, Bi, M, N, K, 16, 128).cpu(), want)
+
+
+CLUSTER_CASES = [  # M, N, K, expected cluster size on a 148-SM part (0: some other schedule)
+    (1, 8192, 8192, 4), (8, 10240, 8192, 3), (32, 8192, 28672, 4), (16, 4096, 1024, 8), (64, 6144, 512, 6),
+    (8, 5120, 64, 0), (40, 9472, 2048, 4), (8, 8192, 192, 0), (24, 57344, 1024, 0), (3, 18944, 3584, 2),
+    (8, 10112, 4096, 3),
+]
+
+
+@pytest.mark.parametrize("M,N,K,want_s", CLUSTER_CASES)
+@pytest.mark.parametrize("br,bc", [(16, 128), (0, 0), (32, 64)])
+def test_cluster_split_k_against_the_oracle_and_the_stream_k_cut(M, N, K, want_s, br, bc):
+    # One tile per cluster, the K loop split over its CTAs, partial tiles added through distributed shared memory in
+    # rank (= K) order: exact on integers, inside the tolerance on random data, bit-reproducible, ragged K shares
+    # (K / 64 not a multiple of the cluster size), clipped last tiles (N not a multiple of 256), bf16 output.
+    from gpu_util import DEV, check_against_oracle, guarded_out, run_gemm, sample_indices, tile_major_on_device, tl
+    layout = TILE if br else ROW
+    A, Bd, want = _int_case(M, N, K, br, bc, seed=M + K)
+    got = run_gemm(A, Bd, M, N, K, br, bc)
+    plan = tl.gemm_last_plan()
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert plan.cluster_k == (want_s if want_s else 1), plan.as_dict()
+        assert plan.workspace_bytes == 0 or want_s == 0
+    assert torch.equal(got.cpu(), want)
+    Ar = inputs.bf16_normal((M, K), 1.0, seed=1)
+    Br = inputs.bf16_normal((K, N), 0.02, seed=2)
+    Brd = tile_major_on_device(Br, K, N, br, bc) if br else Br.to(DEV)
+    C = run_gemm(Ar, Brd, M, N, K, br, bc)
+    check_against_oracle(C, Ar, Brd, layout, br, bc, M, N, K, idx=sample_indices(M, N, 3000, seed=3))
+    for _ in range(3):
+        assert torch.equal(run_gemm(Ar, Brd, M, N, K, br, bc), C)
+    g = guarded_out((M, N), torch.bfloat16)
+    tl.gemm_bf16(Ar.to(DEV), Brd, g.t, M, N, K, br * bc * 2, br, bc)
+    tl.device_status()
+    assert torch.equal(g.check(), C.to(torch.bfloat16))                 # the same fp32 sums, rounded once
 
 
 def test_relayout_without_the_copy_engine_matches_the_oracle():
@@ -170,11 +209,18 @@ def test_plan_query_equals_what_the_launch_ran(M, N, K, block, cta, E, flavour):
 def test_default_plans_of_the_benchmark_shapes():
     from gpu_util import tl
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    p = tl.gemm_plan(8, 10240, 8192)
-    assert p.cta == (16, 256, 64) and p.stream_k == 1 and p.grid == sms and p.pair_kernel == 0
-    assert p.workspace_bytes == 2 * sms * 16 * 256 * 4
-    p = tl.gemm_plan(32, 57344, 8192)
-    assert p.cta == (32, 128, 128) and p.stream_k == 1
+    if sms != 148:
+        pytest.skip("the expected grids below are those of a 148-SM B200")
+    # decode: schedules without partial tiles in global memory
+    p = tl.gemm_plan(8, 10240, 8192)                  # 40 tiles, clusters of 3 CTAs split K
+    assert p.cta == (16, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 3, 120, 0)
+    p = tl.gemm_plan(32, 8192, 28672)                 # 32 tiles, clusters of 4
+    assert p.cta == (32, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 4, 128, 0)
+    p = tl.gemm_plan(32, 57344, 8192)                 # 224 whole tiles on 112 CTAs
+    assert p.cta == (32, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 1, 112, 0)
+    with tl.option(tl.OPT_NO_SCRATCH_PLANS, 0):       # the stream-K cut over every SM
+        p = tl.gemm_plan(8, 10240, 8192)
+        assert (p.stream_k, p.cluster_k, p.grid) == (1, 1, sms) and p.workspace_bytes == 2 * sms * 16 * 256 * 4
     p = tl.gemm_plan(4096, 57344, 8192)
     assert p.pair_kernel == 1 and p.cta == (512, 128, 64) and p.workspace_bytes == 0 and p.grid % 2 == 0
     assert 2 * p.pair_tiles_512 + p.pair_tiles_256 == 16 * 224
