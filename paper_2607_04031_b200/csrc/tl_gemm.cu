@@ -62,9 +62,11 @@ __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_consta
     bool active = c < sched.grid_eff;
     int tile = 0, c_lo = 0, c_hi = 0, share = 0, shares = 1;
     if (active) {
+        // (iterations count from the first tile of the part of the schedule that is cut along K)
         const long long b = sched.range_begin(c);
-        tile = int(b / p.k_iters);
-        const long long tile_begin = static_cast<long long>(tile) * p.k_iters;
+        const int cut_tile = int(b / p.k_iters);
+        tile = sched.dp_tiles + cut_tile;
+        const long long tile_begin = static_cast<long long>(cut_tile) * p.k_iters;
         active = b != tile_begin;                          // else the boundary coincides with a tile boundary
         if (active) {
             c_lo = sched.owner(tile_begin);
@@ -250,13 +252,15 @@ static int pick_bm(int64_t rows) {
 //   up to 128 rows     128 x 128 x 128: same orientation, deeper K step so that there are half as many barrier
 //                      hand-offs
 //   more rows          256 x 128 x 64 with the weights on the M side (prefill)
-//   grouped            at most 32 rows per tile: most experts have a handful of rows, and a large cap costs
-//                      pipeline stages and partial-tile bytes for every tile
+//   grouped            at most 32 rows per tile (x 256 x 64): most experts have a handful of rows; caps of 64 and 128
+//                      rows measured the same within 2 % on the Qwen-3 expert products (fewer passes over an
+//                      expert's weights against fewer, larger pipeline stages)
 //   narrow_scratch     (fixed-size scratch) never the 256-column tile
 static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, int* BM, int* BN, int* BK) {
     *BM = pick_bm(rows_max);
-    if (grouped && *BM > 32) *BM = 32;
-    if (*BM <= 64 && !narrow_scratch && !grouped) { *BN = 256; *BK = 64; }
+    const int group_cap = opt(TL_OPT_MOE_ROW_CAP) > 0 ? int(opt(TL_OPT_MOE_ROW_CAP)) : 32;
+    if (grouped && *BM > group_cap) *BM = group_cap;
+    if (*BM <= 64 && !narrow_scratch) { *BN = 256; *BK = 64; }
     else if (*BM <= 128) { *BN = 128; *BK = 128; }
     else { *BN = 128; *BK = 64; }
 }
@@ -278,8 +282,11 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     // many token rows per 64-wide K slice, the ones beyond BM zeroed once by the kernel.  They only feed
     // accumulator rows that are never stored.
     const bool m128_only = opt(TL_OPT_UMMA_M128) != 0;          // measurement switch
-    plan->umma_m = BM <= 64 && !m128_only ? 64 : 128;
-    plan->a_rows = plan->weights_on_n && BM < plan->umma_m ? plan->umma_m : BM;
+    // (umma_m == 64: per tile, 64-row instructions for tiles of up to 64 tokens and 128-row ones above)
+    plan->umma_m = BM <= 128 && !m128_only ? 64 : 128;
+    // (the stage must hold every token row the widest instruction of the launch reads)
+    const int mma_rows_min = m128_only ? 128 : 64;
+    plan->a_rows = plan->weights_on_n && BM < mma_rows_min ? mma_rows_min : BM;
     const size_t stage = size_t(BK) * BN * 2 + size_t(BK / 64) * plan->a_rows * kAtomBytes;
     // 1 KB of slack to align the stages to 1024 bytes.
     // 12 KB stay free so that a CTA of the stream-K reduction kernel can be resident next to this one.

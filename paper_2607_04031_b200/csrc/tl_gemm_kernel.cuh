@@ -90,42 +90,54 @@ struct Work {
 
 constexpr int kRangeTabMax = 256;      // CTAs whose range starts are tabulated in shared memory
 
+// Work of one CTA.  Three schedules:
+//   stream_k == 0   whole tiles, round-robin over the grid;
+//   stream_k == 1   whole rounds of tiles round-robin (dp_tiles = the largest multiple of the grid below the tile
+//                   count: tiles next to each other in the order run at the same time on different SMs and share
+//                   what they read through L2), then the flattened (tile, K iteration) space of the tiles that
+//                   are left cut into one contiguous range per CTA ("stream-K": all SMs stay busy to the end; a
+//                   CTA that owns only part of a tile's K loop leaves a partial tile for the reduction kernel);
+//   stream_k == 2   cluster split-K: tile = cluster index, K loop cut over the cluster's CTAs.
+// All arithmetic of the cut part works on the tiles after dp_tiles ("cut space": iteration x = (tile - dp_tiles) *
+// k_iters + k iteration).
 struct Sched {
-    int stream_k, k_iters, tiles_total, grid_eff, cta;
+    int stream_k, k_iters, tiles_total, grid_eff, cta, grid;
+    int dp_tiles;       // tiles handed out whole before the cut part starts (0 unless stream_k == 1)
     int next_tile;
     long long it, it_end, it_begin;
-    const int* tab;     // tab[c] = first flattened iteration of CTA c (grid_eff + 1 entries), or nullptr
+    const int* tab;     // tab[c] = first iteration (cut space) of CTA c (grid_eff + 1 entries), or nullptr
 
-    // Even split of the flattened (tile, K iteration) space; a fixed function of the CTA index.
+    // Even split of the cut space; a fixed function of the CTA index.
     __device__ static long long split(long long total, int grid_eff, int c) { return (total * c) / grid_eff; }
-    __device__ long long range_begin(int c) const {
-        return tab ? tab[c] : split(static_cast<long long>(tiles_total) * k_iters, grid_eff, c);
-    }
+    __device__ static int whole_rounds_tiles(int tiles_total, int grid) { return grid > 0 ? (tiles_total / grid) * grid : 0; }
+    __device__ long long cut_total() const { return static_cast<long long>(tiles_total - dp_tiles) * k_iters; }
+    __device__ long long range_begin(int c) const { return tab ? tab[c] : split(cut_total(), grid_eff, c); }
     __device__ static int effective_grid(long long total, int grid) { return total < grid ? static_cast<int>(total) : grid; }
     // Cluster split-K: the one work item of this CTA (tile = cluster index, the rank's share of the K loop).
     __device__ void init_cluster(int k_iters_, int tiles_total_, int cluster, int rank, int size) {
         stream_k = 2; k_iters = k_iters_; tiles_total = tiles_total_; cta = cluster; tab = nullptr; grid_eff = 0;
+        grid = 0; dp_tiles = 0;
         next_tile = cluster;
         it_begin = it = static_cast<long long>(k_iters_) * rank / size;
         it_end = static_cast<long long>(k_iters_) * (rank + 1) / size;
         if (cluster >= tiles_total_) it_end = it;
     }
-    __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid, int cta_, const int* tab_) {
-        stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_; tab = tab_;
-        grid_eff = effective_grid(static_cast<long long>(tiles_total) * k_iters, grid);
+    __device__ void init(int stream_k_, int k_iters_, int tiles_total_, int grid_, int cta_, const int* tab_) {
+        stream_k = stream_k_; k_iters = k_iters_; tiles_total = tiles_total_; cta = cta_; tab = tab_; grid = grid_;
+        dp_tiles = stream_k ? whole_rounds_tiles(tiles_total, grid) : 0;
+        grid_eff = effective_grid(cut_total(), grid);
         next_tile = cta;
-        if (grid_eff == 0 || cta >= grid_eff) { it = it_end = it_begin = 0; next_tile = tiles_total; return; }
+        if (grid_eff == 0 || cta >= grid_eff) { it = it_end = it_begin = 0; return; }
         it_begin = it = range_begin(cta);
         it_end = range_begin(cta + 1);
     }
     __device__ bool next(Work& w) {
-        if (!stream_k) {
-            if (next_tile >= tiles_total) return false;
+        if (stream_k != 2 && next_tile < (stream_k ? dp_tiles : tiles_total)) {
             w.tile = next_tile; w.kbeg = 0; w.kend = k_iters;
-            next_tile += gridDim.x;
+            next_tile += grid;
             return true;
         }
-        if (it >= it_end) return false;
+        if (!stream_k || it >= it_end) return false;
         if (stream_k == 2) {
             w.tile = next_tile; w.kbeg = static_cast<int>(it); w.kend = static_cast<int>(it_end);
             it = it_end;
@@ -135,11 +147,11 @@ struct Sched {
         int kb = static_cast<int>(it - static_cast<long long>(t) * k_iters);
         long long left = it_end - it;
         int ke = (k_iters - kb) < left ? k_iters : kb + static_cast<int>(left);
-        w.tile = t; w.kbeg = kb; w.kend = ke;
+        w.tile = dp_tiles + t; w.kbeg = kb; w.kend = ke;
         it += ke - kb;
         return true;
     }
-    // CTA whose range holds flattened iteration x.
+    // CTA whose range holds iteration x of the cut space.
     __device__ int owner(long long x) const {
         if (tab) {                                   // largest c with tab[c] <= x
             int lo = 0, hi = grid_eff;
@@ -149,7 +161,7 @@ struct Sched {
             }
             return lo;
         }
-        long long total = static_cast<long long>(tiles_total) * k_iters;
+        long long total = cut_total();
         int c = static_cast<int>(((x + 1) * grid_eff + total - 1) / total) - 1;
         if (c < 0) c = 0;
         if (c >= grid_eff) c = grid_eff - 1;
@@ -157,13 +169,14 @@ struct Sched {
         while (c + 1 < grid_eff && range_begin(c + 1) <= x) ++c;
         return c;
     }
-    // Partial-tile slot of CTA c for tile t: 2c when the tile is the first thing c works on, else 2c+1.
+    // Partial-tile slot of CTA c for tile t (of the cut part): 2c when the tile is the first thing c works on there, else 2c+1.
     __device__ int slot(int c, int t) const {
-        return 2 * c + (range_begin(c) < static_cast<long long>(t) * k_iters ? 1 : 0);
+        return 2 * c + (range_begin(c) < static_cast<long long>(t - dp_tiles) * k_iters ? 1 : 0);
     }
 };
 
-__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* prefix, const int* row_start, int tile) {
+__device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* prefix, const int* row_start, int tile,
+                                                bool flip_odd = false) {
     // prefix[e] = tiles of experts before e; tiles of one expert: n-tile major, m-tile minor.
     int lo = 0, hi = p.E;                  // find e with prefix[e] <= tile < prefix[e+1]
     while (hi - lo > 1) {
@@ -182,7 +195,9 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* 
     // The m-tiles of one (expert, n-tile) follow each other in the tile order and read the same weight slab.  Odd
     // ones walk K from the far end, so that what the even one before them read last is read again first, while it
     // is still in L2.
-    t.flip = (local % mt) & 1;
+    // (flip_odd: only where one CTA meets these tiles one after another, i.e. in the cut part of the schedule.  Tiles
+    // handed out round-robin run at the same time on different SMs and share the slab while both walk it forwards.)
+    t.flip = flip_odd ? (local % mt) & 1 : 0;
     t.rows = row_end - t.row0 < p.BM ? row_end - t.row0 : p.BM;
     return t;
 }
@@ -370,7 +385,9 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     const uint32_t tmem_base = tmem_slot;
     const int tiles_total = prefix[p.E];
     // Range starts of all CTAs, once, so that nothing on the critical path divides 64-bit numbers.
-    const long long total_iters = static_cast<long long>(tiles_total) * p.k_iters;
+    // (of the part of the schedule that is cut along K: the tiles left after the whole rounds)
+    const long long total_iters =
+        static_cast<long long>(tiles_total - Sched::whole_rounds_tiles(tiles_total, gridDim.x)) * p.k_iters;
     const int grid_eff0 = Sched::effective_grid(total_iters, gridDim.x);
     const bool use_tab = p.stream_k && grid_eff0 > 0 && grid_eff0 <= kRangeTabMax && total_iters < (1ll << 31);
     if (use_tab) {
@@ -390,7 +407,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         Sched first = sched;
         Work w;
         if (first.next(w)) {
-            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile, first.stream_k == 1 && w.tile >= first.dp_tiles);
             for (int s = 0, kit = w.kbeg; s < p.prefetch_stages && kit < w.kend; ++s, ++kit) {
                 const int kq = t.flip ? p.k_iters - 1 - kit : kit;
                 const int k0 = (kq * kBK) << p.k_shift;
@@ -422,7 +439,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 #pragma unroll
             for (int i = 0; i < 4; ++i) { ks[i] = p.ck_shift[i]; km[i] = p.ck_mask[i]; }
             while (ok && sched.next(w)) {
-                const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+                const TileInfo t = decode_tile(p, prefix, row_start, w.tile, sched.stream_k == 1 && w.tile >= sched.dp_tiles);
                 int bi = 0;
                 while ((16 << bi) < t.rows) ++bi;
                 const uint32_t a_bytes = uint32_t(16 << bi) * kAtomBytes;
@@ -507,7 +524,8 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 // operand K-major; M = kUmmaM, N = n_mma
                 const uint32_t w_major = p.w_kmajor ? 0u : (kWN ? (1u << 16) : (1u << 15));
                 // (8-bit operands: format codes 0 = E4M3 in place of 1 = bf16)
-                const uint32_t m_mma = kWN ? uint32_t(p.umma_m) : uint32_t(kUmmaM);
+                // (weights on N: 64-row instructions for tiles of up to 64 tokens unless the launch asks for 128 rows always)
+                const uint32_t m_mma = kWN ? (p.umma_m == 64 && t.rows <= 64 ? 64u : 128u) : uint32_t(kUmmaM);
                 const uint32_t idesc = (1u << 4) | (kFp8 ? 0u : (1u << 7) | (1u << 10)) | w_major |
                                        ((n_mma >> 3) << 17) | ((m_mma >> 4) << 24);
                 if (!mbar_wait_bounded(&acc_empty_bar[acc], acc_phase ^ 1, abort_ptr, p.status, kWaitMmaAccEmpty, p.wait_limit_ns)) {
@@ -561,7 +579,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         Work w;
         bool ok = true;
         while (ok && sched.next(w)) {
-            const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile, sched.stream_k == 1 && w.tile >= sched.dp_tiles);
             const uint8_t* Bexp = p.B + int64_t(t.expert) * p.expert_bytes;
             const int nblk0 = t.n0 >> p.bc_log2;
             for (int kit = w.kbeg; kit < w.kend; ++kit, ++it_global) {
@@ -618,7 +636,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 // TMEM lane = token row, columns = the tile's kBN weight columns: each thread owns one row of C.
                 // (MMA of 64 rows: rows 16q..16q+15 sit in the lower half of lane quarter q, the upper 16 lanes of
                 // each quarter hold nothing.)
-                const bool m64 = p.umma_m == 64;
+                const bool m64 = p.umma_m == 64 && t.rows <= 64;
                 const int row = m64 ? (lane < 16 ? quarter * 16 + lane : p.BM) : quarter * 32 + lane;
                 const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * uint32_t(acc_cols);
                 if ((m64 ? quarter * 16 : quarter * 32) < t.rows) {      // this lane quarter holds at least one real row
