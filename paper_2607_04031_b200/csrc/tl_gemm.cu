@@ -251,13 +251,18 @@ static int pick_bm(int64_t rows) {
 //                      make_plan)
 //   up to 128 rows     128 x 128 x 128: same orientation, deeper K step so that there are half as many barrier
 //                      hand-offs
-//   more rows          256 x 128 x 64 with the weights on the M side (prefill)
+//   more rows          256 x 128 x 64 with the weights on the M side (prefill) when there are enough tiles for the
+//                      CTA-pair kernel, else 128 x 128 x 128
 //   grouped            at most 32 rows per tile (x 256 x 64): most experts have a handful of rows; caps of 64 and 128
 //                      rows measured the same within 2 % on the Qwen-3 expert products (fewer passes over an
 //                      expert's weights against fewer, larger pipeline stages)
 //   narrow_scratch     (fixed-size scratch) never the 256-column tile
-static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, int* BM, int* BN, int* BK) {
+static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, int* BM, int* BN, int* BK,
+                         bool pair_sized = true) {
     *BM = pick_bm(rows_max);
+    // More than 128 rows but too few tiles for the CTA-pair kernel (pair_sized == false): 128-row tiles with the
+    // weights on the N side (Qwen-3 attention projections at M = 256: 14-16 us against 23-25 us with 256-row tiles).
+    if (!grouped && *BM > 128 && !pair_sized) *BM = 128;
     const int group_cap = opt(TL_OPT_MOE_ROW_CAP) > 0 ? int(opt(TL_OPT_MOE_ROW_CAP)) : 32;
     if (grouped && *BM > group_cap) *BM = group_cap;
     if (*BM <= 64 && !narrow_scratch) { *BN = 256; *BK = 64; }
@@ -266,12 +271,12 @@ static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, in
 }
 
 static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
-                     bool grouped, GemmPlan* plan, bool narrow_scratch = false, bool generic = false) {
+                     bool grouped, GemmPlan* plan, bool narrow_scratch = false, bool generic = false, bool pair_sized = true) {
     if (int rc = ensure_device_info()) return rc;
     int sms = dev().sm_count;
     if (opt(TL_OPT_SM_LIMIT) > 0 && opt(TL_OPT_SM_LIMIT) < sms) sms = int(opt(TL_OPT_SM_LIMIT));
     int BM = cta_m, BN = cta_n, BK = cta_k;
-    if (BM == 0 && BN == 0 && BK == 0) default_tile(rows_max, grouped, narrow_scratch, &BM, &BN, &BK);
+    if (BM == 0 && BN == 0 && BK == 0) default_tile(rows_max, grouped, narrow_scratch, &BM, &BN, &BK, pair_sized);
     if (BM != 16 && BM != 32 && BM != 64 && BM != 128 && BM != 256) return TL_ERR_UNSUPPORTED;
     if (BN != 64 && BN != 128 && BN != 256) return TL_ERR_UNSUPPORTED;
     if (BK != 64 && BK != 128) return TL_ERR_UNSUPPORTED;
@@ -321,8 +326,11 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
         int64_t g1 = 0;
         for (int64_t g = tile_bound < sms ? tile_bound : sms; g >= lo; --g)
             if (tile_bound % g == 0) { g1 = g; break; }
+        // (large partial tiles: at most 4 CTAs per cluster, the exchange through distributed shared memory measured
+        // slower than the stream-K cut beyond that)
+        const int s_max = size_t(BM) * (BN + 4) * 4 > 40 * 1024 ? 4 : 8;
         int best_s = 0;
-        for (int s = 2; s <= 8; ++s)
+        for (int s = 2; s <= s_max; ++s)
             if (tile_bound * s <= sms && tile_bound * s >= lo && k_iters >= s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024 &&
                 tile_bound * s > int64_t(best_s) * tile_bound)
                 best_s = s;
@@ -403,17 +411,20 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (reinterpret_cast<uintptr_t>(d_C) % 16 != 0) return TL_ERR_ALIGNMENT;
     }
 
+    if (int rc = ensure_device_info()) return rc;
+    // enough 256 x 256 tiles for every cluster of the CTA-pair kernel to get one
+    const bool pair_sized = ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= dev().sm_count;
     GemmPlan plan;
     {
         // upper bound of tiles: every expert may add one ragged m-tile
         int bm_guess = cta_m, bn_guess = cta_n, bk_guess = cta_k;
         if (cta_m == 0 && cta_n == 0 && cta_k == 0)
-            default_tile(rows_max, d_offsets != nullptr, fixed != nullptr, &bm_guess, &bn_guess, &bk_guess);
+            default_tile(rows_max, d_offsets != nullptr, fixed != nullptr, &bm_guess, &bn_guess, &bk_guess, pair_sized);
         if (bm_guess <= 0 || bn_guess <= 0) return TL_ERR_UNSUPPORTED;
         const int64_t mt_bound = d_offsets ? rows_total / bm_guess + E : ceil_div(rows_total, bm_guess);
         // (the plan counts K in 2-byte units: an 8-bit stage holds twice as many elements)
         if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                               d_offsets != nullptr, &plan, fixed != nullptr, generic))
+                               d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized))
             return rc;
     }
     if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
@@ -677,7 +688,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     // Worth it once every cluster of the machine has at least one 256 x 256 tile; smaller problems keep the
     // single-CTA kernel and its stream-K split.
     if (!no_pair && !d_offsets && !generic && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
-        p.kbx == 1 && p.nbx == 1 && ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= dev().sm_count) {
+        p.kbx == 1 && p.nbx == 1 && pair_sized) {
         int& max_clusters = dev().pair_max_clusters;
         if (max_clusters < 0) {
             int n = 0;
@@ -879,16 +890,19 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {
     tl::ApiLock lock;
     if (M <= 0 || N <= 0 || K <= 0) return 0;
+    if (tl::ensure_device_info()) return 0;
     size_t need = 0;
     for (int grouped = 0; grouped < 2; ++grouped) {         // the larger of the dense and the grouped schedule
         int bm = cta_m, bn = cta_n, bk = cta_k;
-        if (cta_m == 0 && cta_n == 0 && cta_k == 0) tl::default_tile(M, grouped != 0, false, &bm, &bn, &bk);
+        const bool pair_sized = tl::ceil_div(M, 256) * tl::ceil_div(N, 256) * 2 >= tl::dev().sm_count;
+        if (cta_m == 0 && cta_n == 0 && cta_k == 0) tl::default_tile(M, grouped != 0, false, &bm, &bn, &bk, pair_sized);
         if (bm <= 0 || bn <= 0) return 0;
         tl::GemmPlan plan;
         // grouped: every expert may add a ragged m-tile and the number of experts is not known here; with the most
         // the library accepts the K ranges are cut over every SM, which is the largest scratch a launch can ask for
         const int64_t mt = grouped ? M / bm + tl::kMaxExperts : tl::ceil_div(M, bm);
-        if (tl::make_plan(M, mt * tl::ceil_div(N, bn), N, K, cta_m, cta_n, cta_k, grouped != 0, &plan)) return 0;
+        if (tl::make_plan(M, mt * tl::ceil_div(N, bn), N, K, cta_m, cta_n, cta_k, grouped != 0, &plan, false, false, pair_sized))
+            return 0;
         if (plan.ws_bytes > need) need = plan.ws_bytes;
     }
     return need;
