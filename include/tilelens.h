@@ -164,7 +164,9 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
  *   TMA, whatever their height.  Narrower ones (block rows down to 2 bytes)
  *   are read by the generic-address path of Section 4.4 (plain loads with
  *   Eq. 1-2 arithmetic); there the memory tile must fit inside the CTA tile
- *   (block_rows | cta_k, block_cols | cta_n) and G >= 16, else
+ *   (block_rows | cta_k, block_cols | cta_n), G >= 16, and the CTA tile must
+ *   leave room in shared memory for two raw images of a stage's weights
+ *   beside two operand stages (cta_n * cta_k < 256 * 128), else
  *   TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
  * When the output tiles do not fill the SMs (decode, small or grouped
  * problems) the K loops are cut stream-K fashion over all SMs; partial tiles

@@ -89,7 +89,8 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 // Detail codes stored in the status word by kernels that give up.
 enum : uint32_t {
     kWaitProducerEmpty = 0x100, kWaitMmaFull = 0x200, kWaitMmaAccEmpty = 0x300,
-    kWaitEpilogueAccFull = 0x400, kWaitTeardown = 0x500, kWaitRelayoutFull = 0x600
+    kWaitEpilogueAccFull = 0x400, kWaitTeardown = 0x500, kWaitRelayoutFull = 0x600,
+    kBadCopy = 0x700            // a bulk copy's source or destination failed the kernel's own range / alignment check
 };
 
 // ------------------------------------------------------------- device helpers

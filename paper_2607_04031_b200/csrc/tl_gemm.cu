@@ -234,6 +234,7 @@ struct GemmPlan {
     int cluster_k;        // > 1: clusters of that many CTAs split the K loop of one tile each (no scratch)
     int grid;
     int num_stages;
+    int raw_slots;        // generic-address path: raw stage images kept in flight behind the pipeline stages
     size_t smem_bytes;
     size_t ws_bytes;
 };
@@ -299,12 +300,25 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     int stages = int(budget / stage);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return TL_ERR_UNSUPPORTED;
+    plan->raw_slots = 0;
+    const size_t raw_bytes = size_t(BK) * BN * 2;
+    size_t table_bytes = 0;
+    if (generic) {
+        // Two or three operand stages; the rest of shared memory holds raw stage images (the bytes in flight).
+        // (a table of one 16-bit entry per 16-byte chunk of a stage follows the ring)
+        stages = stage >= 40 * 1024 ? 2 : 3;
+        table_bytes = raw_bytes / 8;
+        if (size_t(stages) * stage + 2 * raw_bytes + table_bytes > budget) return TL_ERR_UNSUPPORTED;
+        int raw = int((budget - size_t(stages) * stage - table_bytes) / raw_bytes);
+        plan->raw_slots = raw > kMaxStages ? kMaxStages : raw;
+    }
     {
         const int cap = int(opt(TL_OPT_MAX_STAGES));            // measurement switch
         if (cap >= 2 && cap < stages) stages = cap;
+        if (cap >= 2 && cap < plan->raw_slots) plan->raw_slots = cap;
     }
     plan->num_stages = stages;
-    plan->smem_bytes = size_t(stages) * stage + 1024;
+    plan->smem_bytes = size_t(stages) * stage + size_t(plan->raw_slots) * raw_bytes + table_bytes + 1024;
     if (plan->smem_bytes < 120 * 1024) plan->smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
     const int64_t k_iters = ceil_div(K, BK);
     const int64_t total_iters = tile_bound * k_iters;
@@ -671,6 +685,9 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.k_iters = int(ceil_div(K, int64_t(plan.BK) << k_shift));
     p.stream_k = plan.stream_k;
     p.cluster_k = plan.cluster_k;
+    p.raw_slots = plan.raw_slots;
+    p.smem_limit = uint32_t(plan.smem_bytes);
+    p.b_bytes = int64_t(E) * K * N * es;
     p.num_stages = plan.num_stages;
     const int prefetch_env = int(opt(TL_OPT_PREFETCH_STAGES));   // measurement switch, -1: the default below
     // (at most four instructions: the thread that issues them holds up the CTA's first barrier for their duration)

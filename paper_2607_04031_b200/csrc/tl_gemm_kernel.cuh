@@ -9,7 +9,8 @@
 namespace tl {
 
 constexpr int kGemmThreads = 192;          // TMA path: producer, MMA issuer, four epilogue warps
-constexpr int kGenericThreads = 320;       // generic-address path: four more warps that load the weights by hand
+constexpr int kGenericThreads = 352;       // generic-address path: four more warps that build the weight operand by hand
+                                           // and one that streams the raw memory tiles into shared memory
 constexpr int kMaxStages = 16;
 constexpr int kMaxExperts = 1024;
 constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 256 rows
@@ -69,7 +70,10 @@ struct alignas(64) GemmParams {
     uint32_t ugroup_off;        // bytes between the 128-column groups of a 256-column tile
     uint32_t kstep_off[8];      // byte offset of each 16-row K step inside a stage
     // generic-address path (Section 4.4: memory tiles that TMA cannot box)
-    int generic_b;              // 1: warps 6..9 load the weights with Eq. 1-2 address arithmetic
+    int generic_b;              // 1: warps 6..9 build the weight operand with Eq. 1-2 address arithmetic
+    int raw_slots;              // generic path: ring of raw stage images (memory order) behind the pipeline stages
+    uint32_t smem_limit;        // dynamic shared memory of the launch, bytes (the bulk copies check their destination against it)
+    int64_t b_bytes;            // size of the weight buffer, bytes (... and their source against this)
     const uint8_t* B;           // raw weight pointer (generic path only)
     int64_t expert_bytes;       // K*N*2
     int blocks_per_row;         // N / bc
@@ -243,35 +247,35 @@ __device__ __forceinline__ void epilogue_bar_sync() {
     asm volatile("bar.sync 1, 128;" ::: "memory");
 }
 
-// One warp fills one stage of weights on the generic-address path.  The stage is kBK/br runs of
-// kBN/bc whole memory tiles; run r starts at src0 + r*krow_stride and is kBN*br*2 contiguous bytes.
-// Chunks of 16 bytes are read in memory order, 16 loads in flight per lane; kPieces = rows held by one
-// chunk (1 when a block row is at least 16 bytes).  Rows >= k_rows_left and columns >= n_cols_left
-// (tile overhang) are filled with zeros.
+// One warp builds one stage of weights on the generic-address path.  The stage is kBK/br runs of kBN/bc whole
+// memory tiles; `raw` holds them in memory order, run r at r * kBN*br*2 (bulk copies put them there).  Chunks of 16
+// bytes are read in that order; kPieces = rows held by one chunk (1 when a block row is at least 16 bytes).  Rows >=
+// k_rows_left and columns >= n_cols_left (tile overhang: nothing was copied there) are filled with zeros.
 template <int kBK, int kBN, int kPieces>
-__device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* src0, int64_t krow_stride, int br_log2,
+__device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* raw, int br_log2,
                                                    int bc_log2, int k_rows_left, int n_cols_left, int lane) {
+    // (lane: 0..127 over the four warps that share the stage)
     constexpr int kChunks = kBK * kBN * 2 / 16;
     const int run_log2 = bc_log2 + 1;                       // log2(bytes of one block row)
     const int g_log2 = br_log2 + run_log2;                  // log2(G)
     const int seg_log2 = br_log2 + 1 + (kBN == 64 ? 6 : kBN == 128 ? 7 : 8);   // log2(kBN * br * 2): bytes of one run of tiles
 #pragma unroll 1
-    for (int base = 0; base < kChunks; base += 32 * 16) {
-        uint4 v[16];
-        int kl[16], nl[16];
+    for (int base = 0; base < kChunks; base += 128 * 4) {
+        uint4 v[4];
+        int kl[4], nl[4];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int byte = (base + i * 32 + lane) << 4;   // byte offset inside the stage's memory image
+        for (int i = 0; i < 4; ++i) {
+            const int byte = (base + i * 128 + lane) << 4;  // byte offset inside the stage's memory image
             const int seg = byte >> seg_log2, o = byte & ((1 << seg_log2) - 1);
             const int ib = o & ((1 << g_log2) - 1);         // byte inside the memory tile
             kl[i] = (seg << br_log2) + (ib >> run_log2);    // Eq. 1 inverted: row and column inside the stage
             nl[i] = ((o >> g_log2) << bc_log2) + ((ib & ((1 << run_log2) - 1)) >> 1);
             v[i] = make_uint4(0, 0, 0, 0);
             if (kl[i] < k_rows_left && nl[i] < n_cols_left)
-                v[i] = __ldg(reinterpret_cast<const uint4*>(src0 + int64_t(seg) * krow_stride + o));
+                v[i] = *reinterpret_cast<const uint4*>(raw + byte);
         }
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 4; ++i) {
             const uint32_t word[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
 #pragma unroll
             for (int pc = 0; pc < kPieces; ++pc) {
@@ -280,6 +284,47 @@ __device__ __forceinline__ void generic_fill_stage(uint8_t* sw, const uint8_t* s
                                (n & 7) * 2;
                 if (kPieces == 1) *reinterpret_cast<uint4*>(dst) = v[i];
                 else if (kPieces == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(word[2 * pc], word[2 * pc + 1]);
+                else if (kPieces == 4) *reinterpret_cast<uint32_t*>(dst) = word[pc];
+                else *reinterpret_cast<uint16_t*>(dst) = uint16_t(word[pc >> 1] >> ((pc & 1) * 16));
+            }
+        }
+    }
+}
+
+// Where chunk c of a raw stage image (its c-th 16 bytes in memory order) goes in the swizzled operand image: byte
+// offset of the chunk, or of its first row piece.  The same for every stage of a launch, so it is tabulated once.
+template <int kBK, int kBN>
+__device__ __forceinline__ uint32_t generic_chunk_dst(int c, int br_log2, int bc_log2) {
+    const int run_log2 = bc_log2 + 1, g_log2 = br_log2 + run_log2;
+    const int seg_log2 = br_log2 + 1 + (kBN == 64 ? 6 : kBN == 128 ? 7 : 8);
+    const int byte = c << 4;
+    const int seg = byte >> seg_log2, o = byte & ((1 << seg_log2) - 1);
+    const int ib = o & ((1 << g_log2) - 1);
+    const int k = (seg << br_log2) + (ib >> run_log2);      // Eq. 1 inverted
+    const int n = ((o >> g_log2) << bc_log2) + ((ib & ((1 << run_log2) - 1)) >> 1);
+    return uint32_t((n >> 6) * (kBK * kAtomBytes) + k * kAtomBytes + ((((n & 63) >> 3) ^ (k & 7)) << 4) + (n & 7) * 2);
+}
+
+// The same stage build for a stage that lies wholly inside the matrix (no overhang, so no zero fill): per chunk one
+// table entry, one 16-byte read and kPieces stores.  A chunk's row pieces sit in consecutive rows kl .. kl + kPieces - 1
+// (kl a multiple of kPieces), i.e. 128 bytes apart with the 16-byte column group XOR-ed by the row's low three bits.
+template <int kBK, int kBN, int kPieces>
+__device__ __forceinline__ void generic_fill_stage_interior(uint8_t* sw, const uint8_t* raw, const uint16_t* tab, int lane) {
+    constexpr int kPerLane = kBK * kBN * 2 / 16 / 128;       // lane: 0..127 over the four warps that share the stage
+#pragma unroll 4
+    for (int i = 0; i < kPerLane; ++i) {
+        const int c = i * 128 + lane;
+        const uint32_t d0 = tab[c];
+        const uint4 v = *reinterpret_cast<const uint4*>(raw + (c << 4));
+        if (kPieces == 1) {
+            *reinterpret_cast<uint4*>(sw + d0) = v;
+        } else {
+            const uint32_t word[4] = {v.x, v.y, v.z, v.w};
+            const uint32_t k7 = (d0 >> 7) & 7u, nchunk = ((d0 >> 4) & 7u) ^ k7;
+#pragma unroll
+            for (int pc = 0; pc < kPieces; ++pc) {
+                uint8_t* dst = sw + (((d0 + uint32_t(pc) * kAtomBytes) & ~0x70u) | ((nchunk ^ (k7 + uint32_t(pc))) << 4));
+                if (kPieces == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(word[2 * pc], word[2 * pc + 1]);
                 else if (kPieces == 4) *reinterpret_cast<uint32_t*>(dst) = word[pc];
                 else *reinterpret_cast<uint16_t*>(dst) = uint16_t(word[pc >> 1] >> ((pc & 1) * 16));
             }
@@ -324,6 +369,8 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t raw_full_bar[kMaxStages];      // generic path: raw image landed / raw image consumed
+    __shared__ __align__(8) uint64_t raw_empty_bar[kMaxStages];
     __shared__ __align__(8) uint64_t acc_full_bar[2];
     __shared__ __align__(8) uint64_t acc_empty_bar[2];
     __shared__ uint32_t tmem_slot;
@@ -343,8 +390,10 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
 
     // ---------------------------------------------------------------- set-up
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], p.generic_b ? 2 : 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], p.generic_b ? 5 : 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 4); }
+        if (p.generic_b)
+            for (int r = 0; r < p.raw_slots; ++r) { mbar_init(&raw_full_bar[r], 1); mbar_init(&raw_empty_bar[r], 4); }
         abort_flag = 0;
         fence_mbar_init();
         if (!p.generic_b) tma_prefetch_desc(&p.tmap_b);
@@ -375,6 +424,12 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
     // problems build their tables from the launch parameters alone and wait afterwards.
     const bool tables_first = p.offsets == nullptr;
     if (!tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // generic-address path: the chunk table (see generic_chunk_dst), after the raw ring
+    if (p.generic_b && warp >= 6 && warp < 10) {
+        uint16_t* tab = reinterpret_cast<uint16_t*>(stages + size_t(p.num_stages) * stage_bytes + size_t(p.raw_slots) * kWBytes);
+        for (int c = int(threadIdx.x) - 192; c < int(kWBytes / 16); c += 128)
+            tab[c] = uint16_t(generic_chunk_dst<kBK, kBN>(c, p.br_log2, p.bc_log2));
+    }
     // tiles before each expert (dense: one "expert" holding all M rows)
     load_row_starts(p, row_start);
     __syncthreads();
@@ -563,48 +618,121 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
                 if (acc == 0) acc_phase ^= 1;
             }
         }
-    } else if (warp >= 6) {
-        // ================================ generic-address weight loader (Section 4.4 of the paper)
-        // Memory tiles whose rows are shorter than a TMA box allows are fetched with plain loads.  A stage's
-        // weights are kBK/br runs of whole memory tiles, each run contiguous in the tile-major buffer, so
-        // the 16-byte chunks are read in memory order (fully coalesced for any tile shape); Eq. 1 inverted
-        // gives every chunk's (row, column), and the chunk (or its 16/(2 bc) row pieces) is stored where the
-        // 128-byte-swizzled MN-major operand layout wants it.  Warp w fills every fourth stage.
-        const int pw = warp - 6;
-        const int br = 1 << p.br_log2, bc = 1 << p.bc_log2;
-        const int run_bytes = bc * 2;                              // one block row
-        const int G = br * run_bytes;
-        const int pieces = run_bytes >= 16 ? 1 : 16 / run_bytes;  // rows held by one 16-byte chunk
-        uint32_t it_global = 0;
+    } else if (warp == 10) {
+        // ================================ generic-address path: raw memory tiles -> shared memory
+        // A stage's weights are kBK/br runs of whole memory tiles, each run contiguous in the tile-major buffer
+        // (Eq. 1-2: tiles follow each other along a row of the tile grid).  One untiled bulk copy per run brings them
+        // into a ring of raw stage images, several stages ahead of the warps that permute them: the copy engine
+        // keeps the bytes in flight, no thread holds them in registers.  Lane l issues runs l, l + 32, ...
+        const int br = 1 << p.br_log2;
+        const int G = br << (p.bc_log2 + 1);
+        const uint32_t run_full = uint32_t(kBN) * br * 2;                 // one run of tiles that spans the CTA tile
+        uint8_t* raw_ring = stages + size_t(p.num_stages) * stage_bytes;
+        uint32_t slot = 0, phase = 0, issued = 0;
         Work w;
         bool ok = true;
         while (ok && sched.next(w)) {
             const TileInfo t = decode_tile(p, prefix, row_start, w.tile, sched.stream_k == 1 && w.tile >= sched.dp_tiles);
             const uint8_t* Bexp = p.B + int64_t(t.expert) * p.expert_bytes;
             const int nblk0 = t.n0 >> p.bc_log2;
+            const int n_cols = p.N - t.n0 < kBN ? p.N - t.n0 : kBN;
+            const uint32_t run_bytes = uint32_t(n_cols >> p.bc_log2) * uint32_t(G);      // whole memory tiles inside the matrix
+            for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                int got = 1;
+                if (lane == 0)
+                    got = mbar_wait_bounded(&raw_empty_bar[slot], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns);
+                if (!__shfl_sync(0xffffffffu, got, 0)) { ok = false; break; }
+                const int kq = t.flip ? p.k_iters - 1 - kit : kit;
+                const int k_rows = p.K - kq * kBK < kBK ? p.K - kq * kBK : kBK;
+                const int runs = k_rows >> p.br_log2;
+                if (lane == 0) mbar_arrive_expect_tx(&raw_full_bar[slot], uint32_t(runs) * run_bytes);
+                __syncwarp();
+                const uint8_t* src0 = Bexp + (int64_t((kq * kBK) >> p.br_log2) * p.blocks_per_row + nblk0) * G;
+                uint8_t* dst0 = raw_ring + size_t(slot) * kWBytes;
+                for (int r = lane; r < runs; r += 32) {
+                    uint8_t* dst = dst0 + size_t(r) * run_full;
+                    const uint8_t* src = src0 + int64_t(r) * p.blocks_per_row * G;
+                    // A copy that would leave the weight buffer or this CTA's shared memory, or is not 16-byte
+                    // granular, is not issued: the status word says so and the kernel gives up in the bounded way.
+                    const bool fine = src >= p.B && src + run_bytes <= p.B + p.b_bytes && dst >= smem_raw &&
+                                      dst + run_bytes <= smem_raw + p.smem_limit && run_bytes > 0 && (run_bytes & 15u) == 0 &&
+                                      (reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (smem_u32(dst) & 15u) == 0;
+                    if (fine) {
+                        bulk_load_1d(dst, src, run_bytes, &raw_full_bar[slot]);
+                    } else {
+                        atomicCAS(p.status, 0u, kBadCopy);
+                        *abort_ptr = 1;
+                    }
+                }
+                ++issued;
+                if (++slot == uint32_t(p.raw_slots)) { slot = 0; phase ^= 1; }
+            }
+        }
+        if (lane == 0 && (!ok || *abort_ptr)) {
+            // Giving up: let the copies already issued land before the CTA's shared memory goes away.
+            uint32_t s = slot, ph = phase;
+            const uint32_t back = issued < uint32_t(p.raw_slots) ? issued : uint32_t(p.raw_slots);
+            for (uint32_t i = 0; i < back; ++i) {
+                if (s == 0) { s = p.raw_slots; ph ^= 1; }
+                --s;
+                const uint64_t t0 = global_timer_ns();
+                const uint64_t drain_ns = p.wait_limit_ns < 20000000ull ? p.wait_limit_ns : 20000000ull;
+                while (!mbar_try_wait(&raw_full_bar[s], ph) && global_timer_ns() - t0 < drain_ns) {}
+            }
+        }
+    } else if (warp >= 6) {
+        // ================================ generic-address weight operand (Section 4.4 of the paper)
+        // Memory tiles whose rows are shorter than a TMA box allows.  The raw image of a stage (its memory tiles in
+        // memory order) is read in 16-byte chunks; Eq. 1 inverted gives every chunk's (row, column), and the chunk
+        // (or its 16/(2 bc) row pieces) is stored where the 128-byte-swizzled MN-major operand layout wants it.
+        // The four warps share every stage (a quarter of its chunks each) and each arrives on the stage's barriers.
+        // Every warp takes part in every iteration, in order, so the barrier it polls is never more than one phase
+        // behind the one it asks for (a parity wait cannot tell two phases apart).
+        const int lane4 = (warp - 6) * 32 + lane;
+        const int run_bytes = 2 << p.bc_log2;                      // one block row
+        const int pieces = run_bytes >= 16 ? 1 : 16 / run_bytes;  // rows held by one 16-byte chunk
+        const uint8_t* raw_ring = stages + size_t(p.num_stages) * stage_bytes;
+        const uint16_t* tab = reinterpret_cast<const uint16_t*>(raw_ring + size_t(p.raw_slots) * kWBytes);
+        uint32_t it_global = 0;
+        Work w;
+        bool ok = true;
+        while (ok && sched.next(w)) {
+            const TileInfo t = decode_tile(p, prefix, row_start, w.tile, sched.stream_k == 1 && w.tile >= sched.dp_tiles);
             for (int kit = w.kbeg; kit < w.kend; ++kit, ++it_global) {
-                if ((it_global & 3u) != uint32_t(pw)) continue;
                 const uint32_t stage = it_global % uint32_t(p.num_stages);
                 const uint32_t phase = (it_global / uint32_t(p.num_stages)) & 1u;
-                if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns)) {
+                const uint32_t slot = it_global % uint32_t(p.raw_slots);
+                const uint32_t raw_phase = (it_global / uint32_t(p.raw_slots)) & 1u;
+                if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns) ||
+                    !mbar_wait_bounded(&raw_full_bar[slot], raw_phase, abort_ptr, p.status, kWaitMmaFull, p.wait_limit_ns)) {
                     ok = false;
                     break;
                 }
                 uint8_t* sw = stages + size_t(stage) * stage_bytes;
+                const uint8_t* raw = raw_ring + size_t(slot) * kWBytes;
                 const int kq = t.flip ? p.k_iters - 1 - kit : kit;
-                const int kblk0 = (kq * kBK) >> p.br_log2;
-                const uint8_t* src0 = Bexp + (int64_t(kblk0) * p.blocks_per_row + nblk0) * G;
                 const int k_rows_left = p.K - kq * kBK, n_cols_left = p.N - t.n0;
-                const int64_t krow_stride = int64_t(p.blocks_per_row) * G;      // bytes between runs of tiles
-                switch (pieces) {
-                    case 1: generic_fill_stage<kBK, kBN, 1>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
-                    case 2: generic_fill_stage<kBK, kBN, 2>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
-                    case 4: generic_fill_stage<kBK, kBN, 4>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
-                    default: generic_fill_stage<kBK, kBN, 8>(sw, src0, krow_stride, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane); break;
+                if (k_rows_left >= kBK && n_cols_left >= kBN) {
+                    switch (pieces) {
+                        case 1: generic_fill_stage_interior<kBK, kBN, 1>(sw, raw, tab, lane4); break;
+                        case 2: generic_fill_stage_interior<kBK, kBN, 2>(sw, raw, tab, lane4); break;
+                        case 4: generic_fill_stage_interior<kBK, kBN, 4>(sw, raw, tab, lane4); break;
+                        default: generic_fill_stage_interior<kBK, kBN, 8>(sw, raw, tab, lane4); break;
+                    }
+                } else {
+                    switch (pieces) {
+                        case 1: generic_fill_stage<kBK, kBN, 1>(sw, raw, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane4); break;
+                        case 2: generic_fill_stage<kBK, kBN, 2>(sw, raw, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane4); break;
+                        case 4: generic_fill_stage<kBK, kBN, 4>(sw, raw, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane4); break;
+                        default: generic_fill_stage<kBK, kBN, 8>(sw, raw, p.br_log2, p.bc_log2, k_rows_left, n_cols_left, lane4); break;
+                    }
                 }
                 fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor-core (async) proxy
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&full_bar[stage]);
+                if (lane == 0) {
+                    mbar_arrive(&full_bar[stage]);
+                    mbar_arrive(&raw_empty_bar[slot]);   // the raw image has been read: its slot may be overwritten
+                }
             }
         }
     } else {
@@ -808,5 +936,6 @@ int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream
 // Clusters of the pair kernel that can be resident together on the current device.
 int pair_max_active_clusters(int* out);
 constexpr int kPairStagesMax = 8;
+constexpr int kPairBigThreads = 320;       // pair kernel with 512-token tiles: producer, MMA issuer, eight epilogue warps
 
 }  // namespace tl

@@ -22,8 +22,8 @@ int pair_max_active_clusters(int* out) {
 
 int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream_t stream, const GemmParams& p) {
     if (halves == 2) {
-        if (fp8) gemm_pair_kernel<true, 2><<<2 * clusters, kGenericThreads, smem, stream>>>(p);
-        else gemm_pair_kernel<false, 2><<<2 * clusters, kGenericThreads, smem, stream>>>(p);
+        if (fp8) gemm_pair_kernel<true, 2><<<2 * clusters, kPairBigThreads, smem, stream>>>(p);
+        else gemm_pair_kernel<false, 2><<<2 * clusters, kPairBigThreads, smem, stream>>>(p);
     } else {
         if (fp8) gemm_pair_kernel<true, 1><<<2 * clusters, kGemmThreads, smem, stream>>>(p);
         else gemm_pair_kernel<false, 1><<<2 * clusters, kGemmThreads, smem, stream>>>(p);

@@ -150,7 +150,7 @@ __device__ __forceinline__ PairTile pair_decode(const GemmParams& p, int tile, i
 // Dense problems only (no experts, no stream-K, TMA-readable weights); p.BM == 256, per-CTA tile 128 columns.
 // kHalves = 2 runs with four more epilogue warps (one set per token block): its epilogue is exposed.
 template <bool kFp8, int kHalves>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kHalves == 2 ? kGenericThreads : kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kHalves == 2 ? kPairBigThreads : kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ GemmParams p) {
     constexpr int kBK = 64, kKSteps = 4;
     constexpr uint32_t kWBytes = kBK * 128 * 2;           // this CTA's weight slab per stage
