@@ -40,8 +40,8 @@ WORKLOAD = "llama3.1-70b decode linear layers (qkv, o, gate_up, down; M in {1,8,
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode GEMM kernel, from the ncu
 # capture summarised in profiles/ (None until a capture exists for this kernel version).
-NCU_TRAFFIC_RATIO = 172.81 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
-NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 167.99 MB read + 4.82 MB written for 168.23 MB algorithmic; "
+NCU_TRAFFIC_RATIO = 171.80 / 168.23          # (dram read + write) / algorithmic bytes, decode qkv M=8 capture
+NCU_TRAFFIC_NOTE = ("profiles/gemm_kernel_decode_qkv_m8.md: 168.02 MB read + 3.78 MB written for 168.23 MB algorithmic; "
                     "scaled to the step's average launch by bytes processed (traffic is proportional to the weight bytes)")
 
 
@@ -369,7 +369,9 @@ def run_ours(args):
     step_bytes = sum(relayout_bytes(N, K) for _, K, N in inputs.LLAMA70B_PROJ) + \
         sum(gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
     gemm_step_bytes = sum(gemm_bytes(M, N, K) for _, K, N in inputs.LLAMA70B_PROJ for M in inputs.LLAMA_DECODE_M)
-    launches_per_step = 1 + 12 * 2 + 1       # batched relayout, GEMM + stream-K reduction per product, one batched counter launch
+    # batched relayout, one GEMM launch per product (plus its reduction kernel where the plan is the stream-K cut),
+    # one batched counter launch
+    launches_per_step = 1 + sum(2 if pl.stream_k and pl.grid > 1 else 1 for pl in plans.values()) + 1
 
     tl.set_stream(stream)
     for _ in range(max(3, args.warmup)):
@@ -417,8 +419,12 @@ def run_ours(args):
     g_n *= 12
     r_n *= 4
     gemm_gbs = args.steps * gemm_step_bytes / (g_ms * 1e-3) / 1e9
+    def schedule_name(p_):
+        if p_.stream_k:
+            return "stream-K + streamk_reduce_kernel"
+        return f"split-K in clusters of {p_.cluster_k}" if p_.cluster_k > 1 else f"whole tiles on {p_.grid} CTAs"
     kernels = sorted({f"gemm_kernel<cta {p_.cta_m}x{p_.cta_n}x{p_.cta_k}, weights on {'N' if p_.weights_on_n else 'M'}, "
-                      f"{'stream-K + streamk_reduce_kernel' if p_.stream_k else 'whole tiles'}>" for p_ in plans.values()})
+                      f"{schedule_name(p_)}>" for p_ in plans.values()})
     roofline = {"bound": "hbm", "kernel": "; ".join(kernels), "achieved": gemm_gbs,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
                 "peak_source": f"of {peaks['source']}", "frac_of_nominal_8TBs": gemm_gbs / 8000.0,
@@ -833,6 +839,7 @@ PROFILE_CASES = {
     "kmajor_decode_qkv_m8": ("kmajor", 8, 8192, 10240),     # weights [N][K], (64, 32) memory tiles of Eq. 2
     "fp8_decode_qkv_m8": ("fp8", 8, 8192, 10240),           # E4M3, 64 x 64 memory tiles
     "hw_box_load_o": ("hw", 0, 8192, 8192),                 # every 64 x 256 box of the weight through a 2-D view
+    "generic_16x8_m16": ("generic", 16, 8192, 8192),        # 16 x 8 memory tiles (16-byte rows): generic-address path
     "relayout_layer": ("relayout_batch", 0, 0, 0),          # the four Llama weights in one launch (3.4 GB resident)
 }
 
@@ -860,6 +867,14 @@ def run_case(args):
         dsts = [torch.empty_like(t) for t in srcs]
         for _ in range(args.steps):
             tl.relayout_batch(srcs, dsts, [(k, n) for _, k, n in inputs.LLAMA70B_PROJ], 2, G, BR, BC, tl.TO_TILE_MAJOR)
+    elif kind == "generic":
+        W = inputs.bf16_normal((K, N), 0.02, seed=100, device=dev)
+        Wt = torch.empty_like(W)
+        tl.relayout(W, Wt, K, N, 2, 256, 16, 8, tl.TO_TILE_MAJOR)
+        A = inputs.bf16_normal((M, K), 1.0, seed=200, device=dev)
+        C = torch.empty((M, N), dtype=torch.float32, device=dev)
+        for _ in range(args.steps):
+            tl.gemm(A, Wt, C, M, N, K, 256, 16, 8)
     elif kind in ("kmajor", "hw"):
         w = inputs.bf16_normal((N, K), 0.02, seed=100, device=dev)
         wt = torch.empty_like(w)
