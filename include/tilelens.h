@@ -99,6 +99,8 @@ typedef enum {
     TL_OPT_NO_SCRATCH_PLANS, /* 1 (default): dense decode-sized products prefer schedules without partial tiles in global
                                 memory (whole tiles on a grid that divides the tile count, or split-K inside clusters);
                                 0: always the stream-K cut */
+    TL_OPT_FFN_ONE_LAUNCH,   /* 0 (default): tl_moe_ffn runs its two grouped products as two launches; 1: as two phases of one
+                                cooperative launch where it can (measured slower: 236 against 211 us on the Qwen-3 expert FFN) */
     TL_OPT_COUNT_
 } tl_option;
 /* TL_ERR_INVALID_ARG for an unknown option or a value outside the option's range. */
@@ -204,9 +206,13 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
  * 2j+1; instead of C it writes H[row][j] = bf16(silu(g) * u) (fp32 arithmetic, one rounding to nearest even),
  * d_H_bf16: total_rows x I bf16, 16-byte aligned.  N % 64 == 0; tiles of at most 128 rows (cta_m <= 128), else
  * TL_ERR_UNSUPPORTED.
- * tl_moe_ffn: that call followed by tl_gemm_grouped on H and the experts' I x hidden down weights:
- * Y (fp32, total_rows x hidden) = H x W_down.  Two kernels (plus their stream-K reductions) in stream order, no
- * host synchronisation; d_H_bf16 is caller-owned scratch that holds H afterwards.
+ * tl_moe_ffn: that product followed by the grouped product of H and the experts' I x hidden down weights:
+ * Y (fp32, total_rows x hidden) = H x W_down, no host synchronisation; d_H_bf16 is caller-owned scratch that holds H
+ * afterwards.  Two launches in stream order (the second overlaps the first one's end through programmatic stream
+ * serialisation).  With TL_OPT_FFN_ONE_LAUNCH = 1 and TMA-readable weights both products run as two phases of ONE
+ * cooperative launch instead (a grid-wide barrier with a bounded wait between them; the split tiles of the first
+ * product are summed inside the kernel, those of the second by the small reduction kernel that follows): same bits,
+ * measured slower, and every CTA of its grid has to be resident at the same time.
  */
 /* tl_gemm / tl_gemm_grouped with C written as bf16 (fp32 accumulation, one rounding to nearest even): d_C_bf16
  * M x N (total_rows x N) bf16, 16-byte aligned, N % 8 == 0.  The paper leaves the output type open. */
@@ -289,6 +295,8 @@ typedef struct tl_gemm_plan_info {
     int32_t cluster_k;             /* S > 1: one tile per cluster of S CTAs that split its K loop (sums through distributed
                                       shared memory, no workspace); else 1 */
     int64_t pair_tiles_512, pair_tiles_256;   /* pair kernel: tiles of 512 and of 256 token rows (x 256 columns) */
+    int32_t chained;               /* tl_gemm_last_plan after tl_moe_ffn: 1 when both products ran in one launch */
+    int32_t reserved;
     uint64_t workspace_bytes;      /* split-K scratch the launch uses */
 } tl_gemm_plan_info;
 int tl_gemm_plan(int64_t M, int64_t N, int64_t K, int64_t G, int block_rows, int block_cols,

@@ -66,7 +66,7 @@ _SIGNATURES = {
 # tl_option
 (OPT_PDL, OPT_PREFETCH_STAGES, OPT_PAIR_KERNEL, OPT_PAIR_512, OPT_BOX_PER_BLOCK, OPT_MAX_STAGES, OPT_UMMA_M128,
  OPT_RELAYOUT_TMA, OPT_LOG, OPT_WAIT_LIMIT_US, OPT_STALL_ONCE, OPT_MOE_ROW_CAP, OPT_REDUCE_SPLIT, OPT_SM_LIMIT,
- OPT_NO_SCRATCH_PLANS) = range(15)
+ OPT_NO_SCRATCH_PLANS, OPT_FFN_ONE_LAUNCH) = range(16)
 FLAVOUR_N_BF16, FLAVOUR_K_BF16, FLAVOUR_K_FP8 = 0, 1, 2
 
 _lib = None
@@ -166,6 +166,7 @@ class GemmPlan(ctypes.Structure):
                 ("pair_kernel", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("grid", ctypes.c_int32),
                 ("stages", ctypes.c_int32), ("weights_on_n", ctypes.c_int32), ("generic_path", ctypes.c_int32),
                 ("cluster_k", ctypes.c_int32), ("pair_tiles_512", ctypes.c_int64), ("pair_tiles_256", ctypes.c_int64),
+                ("chained", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_uint64)]
 
     def as_dict(self):

@@ -109,6 +109,8 @@ int ensure_control() {
     if (int rc = check_cuda(cudaHostGetDevicePointer(&h_dev, h, 0))) return rc;
     s.ctl.d_status = static_cast<uint32_t*>(p);
     s.ctl.d_acc = reinterpret_cast<unsigned long long*>(static_cast<char*>(p) + 64);
+    s.d_grid_counter = reinterpret_cast<unsigned long long*>(static_cast<char*>(p) + 960);   // after the 17 x 32 bytes of accumulators
+    s.grid_arrivals = 0;
     s.ctl.h_acc = static_cast<unsigned long long*>(h);
     s.ctl.h_acc_dev = static_cast<unsigned long long*>(h_dev);
     return TL_OK;
@@ -221,6 +223,9 @@ int tl_device_status(uint32_t* detail) {
     if (detail) *detail = word;
     if (word == 0) return TL_OK;
     if (int rc = tl::check_cuda(cudaMemset(tl::dev().ctl.d_status, 0, 4))) return rc;
+    // a kernel that gave up may have left the grid barrier's counter short of what later launches would wait for
+    if (int rc = tl::check_cuda(cudaMemset(tl::dev().d_grid_counter, 0, 8))) return rc;
+    tl::dev().grid_arrivals = 0;
     return TL_ERR_TIMEOUT;
 }
 

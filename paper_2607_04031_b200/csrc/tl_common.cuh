@@ -43,6 +43,8 @@ struct DeviceState {
     size_t own_ws_bytes = 0;
     int sm_count = 0;
     int pair_max_clusters = -1;          // co-resident clusters of the CTA-pair kernel (queried once)
+    unsigned long long* d_grid_counter = nullptr;   // arrival counter of the expert FFN kernel's grid barrier (control block)
+    unsigned long long grid_arrivals = 0;           // arrivals all launches so far will have made
     const void* smem_attr_done[64] = {}; // kernels whose dynamic shared-memory limit was raised on this device
     int smem_attr_n = 0;
 };
@@ -90,7 +92,8 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 enum : uint32_t {
     kWaitProducerEmpty = 0x100, kWaitMmaFull = 0x200, kWaitMmaAccEmpty = 0x300,
     kWaitEpilogueAccFull = 0x400, kWaitTeardown = 0x500, kWaitRelayoutFull = 0x600,
-    kBadCopy = 0x700            // a bulk copy's source or destination failed the kernel's own range / alignment check
+    kBadCopy = 0x700,           // a bulk copy's source or destination failed the kernel's own range / alignment check
+    kWaitGridBarrier = 0x800    // the grid-wide barrier between the two products of the expert FFN kernel
 };
 
 // ------------------------------------------------------------- device helpers
@@ -108,6 +111,9 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_inval(uint64_t* bar) {
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void fence_mbar_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

@@ -34,120 +34,12 @@
 
 namespace tl {
 
-// Stream-K reduction.  The GEMM kernel leaves the partial sum of every (CTA, split tile) in its workspace slot
-// and does no synchronisation of its own; this kernel, ordered after it by the stream, adds the partials of
-// each split tile in K order (lowest CTA first) and writes C.  One CTA per boundary between two ranges of
-// the GEMM grid.  A tile cut by several boundaries is shared between their CTAs: each sums a contiguous share of
-// the tile's 16-byte vectors over ALL contributors, so every element is still one sum in K order and the bits do
-// not depend on how the tile was shared (p.reduce_split == 0: the first boundary inside the tile sums all of it).
 __global__ void __launch_bounds__(128) streamk_reduce_kernel(const __grid_constant__ GemmParams p, int gemm_grid) {
     __shared__ int prefix[kMaxExperts + 1];
     __shared__ int row_start[kMaxExperts + 1];
     __shared__ int slot_of[kRangeTabMax];
-    // Launched with programmatic stream serialisation, and the GEMM kernel lets its dependents launch as soon
-    // as it has started: this grid is resident and has done all of its index arithmetic (which reads only
-    // the call's inputs) while the GEMM grid is still running.  Nothing the GEMM kernel wrote is read before
-    // griddepcontrol.wait, which returns once that grid has completed and its writes are visible.
-    // The kernel after this one in the stream may start its own set-up now; it waits for this grid to complete
-    // before it reads or writes anything.
-    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    load_row_starts(p, row_start);
-    __syncthreads();
-    if (threadIdx.x < 32) tile_prefix(p, row_start, prefix);
-    __syncthreads();
-    Sched sched;
-    sched.init(1, p.k_iters, prefix[p.E], gemm_grid, 0, nullptr);
-    const int c = int(blockIdx.x) + 1;                     // boundary between CTA c-1 and CTA c
-    // Does this boundary cut a tile, and which share of the tile is this CTA's?
-    bool active = c < sched.grid_eff;
-    int tile = 0, c_lo = 0, c_hi = 0, share = 0, shares = 1;
-    if (active) {
-        // (iterations count from the first tile of the part of the schedule that is cut along K)
-        const long long b = sched.range_begin(c);
-        const int cut_tile = int(b / p.k_iters);
-        tile = sched.dp_tiles + cut_tile;
-        const long long tile_begin = static_cast<long long>(cut_tile) * p.k_iters;
-        active = b != tile_begin;                          // else the boundary coincides with a tile boundary
-        if (active) {
-            c_lo = sched.owner(tile_begin);
-            c_hi = sched.owner(tile_begin + p.k_iters - 1);
-            if (p.reduce_split) {
-                share = c - c_lo - 1;                      // boundaries c_lo+1 .. c_hi lie inside the tile
-                shares = c_hi - c_lo;
-            } else {
-                active = c == c_lo + 1;                    // the first boundary inside the tile sums all of it
-            }
-        }
-    }
-    TileInfo t = {0, 0, 0, 0, 0};
-    if (active) {
-        t = decode_tile(p, prefix, row_start, tile);
-        // slots of the contributors, computed before the wait (the load loop below must not divide)
-        for (int j = threadIdx.x; j <= c_hi - c_lo && j < kRangeTabMax; j += blockDim.x) slot_of[j] = sched.slot(c_lo + j, tile);
-    }
-    __syncthreads();
-    // EVERY CTA waits, also those with nothing to add: a grid whose CTAs all left before the GEMM grid finished
-    // would count as complete, and the kernel after it in the stream would stop waiting for the GEMM.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (!active) return;
-    float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
-    const int vec_per_row = p.BN / 4;
-    const int total_vec = t.rows * vec_per_row;
-    const int v_begin = int(static_cast<long long>(total_vec) * share / shares);
-    const int v_end = int(static_cast<long long>(total_vec) * (share + 1) / shares);
-    const size_t slot_floats = size_t(p.BM) * p.BN;
-    for (int v0 = v_begin; v0 < v_end; v0 += 4 * 128) {
-        float4 sum[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) sum[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {         // four contributors' loads in flight together
-            float4 x[4][4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const bool c_ok = c0 + j <= c_hi;
-                const int jj = c_ok ? c0 + j - c_lo : 0;
-                const int slot = jj < kRangeTabMax ? slot_of[jj] : sched.slot(c_lo + jj, tile);
-                const float4* src = reinterpret_cast<const float4*>(p.partials + size_t(slot) * slot_floats);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int v = v0 + q * 128 + int(threadIdx.x);
-                    x[j][q] = (c_ok && v < v_end) ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (c0 + j > c_hi) break;                  // absent contributors add nothing (not even +0)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    sum[q].x += x[j][q].x; sum[q].y += x[j][q].y; sum[q].z += x[j][q].z; sum[q].w += x[j][q].w;
-                }
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int v = v0 + q * 128 + int(threadIdx.x);
-            if (v < v_end) {
-                const int r = v / vec_per_row, c4 = (v % vec_per_row) * 4;
-                if (t.n0 + c4 < p.N) {
-                    if (p.epi_swiglu) {
-                        const __nv_bfloat16 lo = swiglu_bf16(sum[q].x, sum[q].y), hi = swiglu_bf16(sum[q].z, sum[q].w);
-                        *reinterpret_cast<uint32_t*>(p.H + int64_t(t.row0 + r) * p.ldh + ((t.n0 + c4) >> 1)) =
-                            uint32_t(__bfloat16_as_ushort(lo)) | (uint32_t(__bfloat16_as_ushort(hi)) << 16);
-                    } else if (p.Cb) {
-                        const uint32_t lo = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].x))) |
-                                            (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].y))) << 16);
-                        const uint32_t hi = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].z))) |
-                                            (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].w))) << 16);
-                        *reinterpret_cast<uint2*>(p.Cb + int64_t(t.row0 + r) * p.ldc + t.n0 + c4) = make_uint2(lo, hi);
-                    } else {
-                        *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
-                    }
-                }
-            }
-        }
-    }
+    streamk_reduce_body<true>(p, gemm_grid, int(blockIdx.x), prefix, row_start, slot_of);
 }
-
 
 // ======================================================================== host
 
@@ -363,6 +255,19 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     return TL_OK;
 }
 
+static int launch_reduce(const GemmParams& p, int gemm_grid, cudaStream_t stream, bool pdl) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(gemm_grid - 1);
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // overlap its launch with the GEMM grid
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return check_cuda(cudaLaunchKernelEx(&cfg, streamk_reduce_kernel, p, gemm_grid));
+}
+
 // What the calling thread's last GEMM launch ran (tl_gemm_last_plan).
 static tl_gemm_plan_info& last_plan() {
     static thread_local tl_gemm_plan_info info = {};
@@ -380,7 +285,10 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
                        int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
                        bool kmajor = false, int elem_bytes = 2, void* d_H_swiglu = nullptr, void* d_C_bf16 = nullptr,
-                       tl_gemm_plan_info* plan_only = nullptr) {
+                       tl_gemm_plan_info* plan_only = nullptr, GemmParams* params_only = nullptr,
+                       GemmPlan* params_plan = nullptr) {
+    // params_only: everything up to the launch (checks, plan, tensor maps, workspace) and then the kernel's
+    // parameters are handed back instead of being launched (the expert FFN runs two products in one kernel).
     // plan_only: no pointer is looked at, nothing is encoded or enqueued; *plan_only receives what a launch with
     // these sizes would run (the same code decides both, so the two cannot drift apart).
     const int es = elem_bytes;                       // 2: bf16, 1: FP8 (E4M3), K-contiguous weights only
@@ -761,6 +669,11 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.stall_extra_tx = 16;
         tl_set_option(TL_OPT_STALL_ONCE, 0);
     }
+    if (params_only) {
+        *params_only = p;
+        *params_plan = plan;
+        return TL_OK;
+    }
     // The GEMM kernel may be scheduled while its predecessor in the stream is finishing (it waits before touching
     // memory).  TL_OPT_PDL = 0 restores plain stream order for measurement.
     int rc = TL_OK;
@@ -791,18 +704,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (rc) return rc;
     }
     // stream-K: add up the partial tiles, one CTA per boundary between two CTA ranges
-    if (plan.stream_k && plan.grid > 1) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(plan.grid - 1);
-        cfg.blockDim = dim3(128);
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // overlap its launch with the GEMM grid
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = pdl_ok ? 1 : 0;
-        err = cudaLaunchKernelEx(&cfg, streamk_reduce_kernel, p, plan.grid);
-    }
+    if (plan.stream_k && plan.grid > 1) return launch_reduce(p, plan.grid, stream, pdl_ok);
     if (err != cudaSuccess) return check_cuda(err);
     return check_cuda(cudaGetLastError());
 }
@@ -897,6 +799,50 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
                int block_rows, int block_cols, void* cuda_stream) {
     tl::ApiLock lock;
     if (hidden <= 0 || inter <= 0) return TL_ERR_INVALID_ARG;
+    if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
+    if (!d_H_bf16) return TL_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (total_rows > 0 && tl::opt(TL_OPT_FFN_ONE_LAUNCH) != 0) {
+        // Both products in one cooperative launch (tl_gemm_chain.cu) when they share the kernel instantiation and the
+        // grid: TMA-readable weights, the default grouped tile, the stream-K schedule.  Otherwise two launches.
+        tl::GemmParams p1, p2;
+        tl::GemmPlan plan1, plan2;
+        int rc = tl::gemm_launch(d_X_sorted, d_W_gate_up, nullptr, d_offsets, E, total_rows, total_rows, 2 * inter, hidden, G,
+                                 block_rows, block_cols, 0, 0, 0, stream, nullptr, false, 2, d_H_bf16, nullptr, nullptr, &p1,
+                                 &plan1);
+        if (rc) return rc;
+        rc = tl::gemm_launch(d_H_bf16, d_W_down, d_Y, d_offsets, E, total_rows, total_rows, hidden, inter, G, block_rows,
+                             block_cols, 0, 0, 0, stream, nullptr, false, 2, nullptr, nullptr, nullptr, &p2, &plan2);
+        if (rc) return rc;
+        // (the grid is the larger of the two plans': a schedule copes with more CTAs than it has work for)
+        const int grid = plan1.grid > plan2.grid ? plan1.grid : plan2.grid;
+        const bool same = plan1.BM == plan2.BM && plan1.BN == plan2.BN && plan1.BK == plan2.BK &&
+                          plan1.BK == 64 && plan1.BN == 256 && plan1.weights_on_n && plan2.weights_on_n &&
+                          plan1.stream_k && plan2.stream_k && !p1.generic_b && !p2.generic_b && grid > 1 &&
+                          plan1.smem_bytes <= size_t(tl::kMaxDynamicSmem - 10 * 1024) &&
+                          plan2.smem_bytes <= size_t(tl::kMaxDynamicSmem - 10 * 1024);
+        if (same) {
+            tl::DeviceState& d = tl::dev();
+            // one workspace for both phases, sized for the common grid (the first product's partial tiles are summed
+            // before the second one writes its own)
+            const size_t ws_bytes = size_t(2) * size_t(grid) * plan1.BM * plan1.BN * sizeof(float);
+            void* ws = nullptr;
+            if ((rc = tl::get_workspace(ws_bytes, &ws))) return rc;
+            p1.partials = p2.partials = static_cast<float*>(ws);
+            const unsigned long long base = d.grid_arrivals;
+            const size_t smem = plan1.smem_bytes > plan2.smem_bytes ? plan1.smem_bytes : plan2.smem_bytes;
+            rc = tl::launch_gemm_chain(plan1.BK, plan1.BN, grid, smem, stream, p1, p2, d.d_grid_counter,
+                                       base + grid, base + 2ull * grid);
+            if (rc) return rc;
+            d.grid_arrivals = base + 2ull * grid;
+            tl_gemm_plan_info& info = tl::last_plan();
+            memset(&info, 0, sizeof info);
+            info.cta_m = plan2.BM; info.cta_n = plan2.BN; info.cta_k = plan2.BK; info.stream_k = 1; info.grid = grid;
+            info.stages = plan2.num_stages; info.weights_on_n = 1; info.cluster_k = 1; info.workspace_bytes = ws_bytes;
+            info.chained = 1;
+            return tl::launch_reduce(p2, grid, stream, false);
+        }
+    }
     if (int rc = tl_gemm_grouped_swiglu(d_X_sorted, d_W_gate_up, d_H_bf16, d_offsets, E, total_rows, 2 * inter, hidden, G,
                                         block_rows, block_cols, 0, 0, 0, cuda_stream))
         return rc;

@@ -357,8 +357,10 @@ __device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, in
 //                (at most 128 per tile) on the M side.  For decode and MoE: 8 KB of weights per instruction
 //                instead of 4 KB, half as many instructions per byte streamed.  TMEM lane =
 //                token, and every thread writes its token's row of C in 16-byte pieces.
+// (The body is a device function so that one kernel can run two products one after the other, see gemm_chain_kernel:
+// alloc_tmem / free_tmem say whether this call allocates tensor memory at its start and frees it at its end.)
 template <int kBK, int kBN, bool kWN, bool kFp8>
-__global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+__device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, bool free_tmem) {
     constexpr int kNumN = kWN ? 1 : (kBN >= 128 ? kBN / 128 : 1);     // MMAs per K step
     constexpr int kUmmaM = kWN ? 128 : (kBN >= 128 ? 128 : 64);       // rows of the MMA's M side
     constexpr int kKSteps = kBK / 16;
@@ -399,7 +401,7 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         if (!p.generic_b) tma_prefetch_desc(&p.tmap_b);
         for (int i = 0; i < kNumBoxChoices; ++i) tma_prefetch_desc(&p.tmap_a[i]);
     }
-    if (warp == 1) {
+    if (warp == 1 && alloc_tmem) {
         tmem_alloc(&tmem_slot, tmem_cols);
         tmem_relinquish();
     }
@@ -917,9 +919,141 @@ __global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_c
         }
         cluster_sync();
     }
-    if (warp == 1) {
+    if (warp == 1 && free_tmem) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, tmem_cols);
+    }
+    // The barriers are dead from here on; a later call of this body in the same kernel initialises them afresh.
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.num_stages; ++s) { mbar_inval(&full_bar[s]); mbar_inval(&empty_bar[s]); }
+        for (int b = 0; b < 2; ++b) { mbar_inval(&acc_full_bar[b]); mbar_inval(&acc_empty_bar[b]); }
+        if (p.generic_b)
+            for (int r = 0; r < p.raw_slots; ++r) { mbar_inval(&raw_full_bar[r]); mbar_inval(&raw_empty_bar[r]); }
+    }
+    __syncthreads();
+}
+
+template <int kBK, int kBN, bool kWN, bool kFp8>
+__global__ void __launch_bounds__(kGenericThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+    gemm_body<kBK, kBN, kWN, kFp8>(p, true, true);
+}
+
+
+// Stream-K reduction.  The GEMM kernel leaves the partial sum of every (CTA, split tile) in its workspace slot
+// and does no synchronisation of its own; this kernel, ordered after it by the stream, adds the partials of
+// each split tile in K order (lowest CTA first) and writes C.  One CTA per boundary between two ranges of
+// the GEMM grid.  A tile cut by several boundaries is shared between their CTAs: each sums a contiguous share of
+// the tile's 16-byte vectors over ALL contributors, so every element is still one sum in K order and the bits do
+// not depend on how the tile was shared (p.reduce_split == 0: the first boundary inside the tile sums all of it).
+// (A device function, so that a kernel that runs two products can sum the first one's split tiles itself: `boundary`
+// is the index of the boundary this CTA owns, `first` / `nthreads` the threads of the CTA that take part -- they
+// must be whole warps starting at a multiple of 32 -- and `pdl` says whether this is the stand-alone kernel, which
+// waits for the GEMM grid through griddepcontrol.)
+template <bool kStandalone>
+__device__ __forceinline__ void streamk_reduce_body(const GemmParams& p, int gemm_grid, int boundary, int* prefix,
+                                                    int* row_start, int* slot_of) {
+    // Launched with programmatic stream serialisation, and the GEMM kernel lets its dependents launch as soon
+    // as it has started: this grid is resident and has done all of its index arithmetic (which reads only
+    // the call's inputs) while the GEMM grid is still running.  Nothing the GEMM kernel wrote is read before
+    // griddepcontrol.wait, which returns once that grid has completed and its writes are visible.
+    // The kernel after this one in the stream may start its own set-up now; it waits for this grid to complete
+    // before it reads or writes anything.
+    if (kStandalone && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    load_row_starts(p, row_start);
+    __syncthreads();
+    if (threadIdx.x < 32) tile_prefix(p, row_start, prefix);
+    __syncthreads();
+    Sched sched;
+    sched.init(1, p.k_iters, prefix[p.E], gemm_grid, 0, nullptr);
+    const int c = boundary + 1;                            // boundary between CTA c-1 and CTA c
+    // Does this boundary cut a tile, and which share of the tile is this CTA's?
+    bool active = c < sched.grid_eff;
+    int tile = 0, c_lo = 0, c_hi = 0, share = 0, shares = 1;
+    if (active) {
+        // (iterations count from the first tile of the part of the schedule that is cut along K)
+        const long long b = sched.range_begin(c);
+        const int cut_tile = int(b / p.k_iters);
+        tile = sched.dp_tiles + cut_tile;
+        const long long tile_begin = static_cast<long long>(cut_tile) * p.k_iters;
+        active = b != tile_begin;                          // else the boundary coincides with a tile boundary
+        if (active) {
+            c_lo = sched.owner(tile_begin);
+            c_hi = sched.owner(tile_begin + p.k_iters - 1);
+            if (p.reduce_split) {
+                share = c - c_lo - 1;                      // boundaries c_lo+1 .. c_hi lie inside the tile
+                shares = c_hi - c_lo;
+            } else {
+                active = c == c_lo + 1;                    // the first boundary inside the tile sums all of it
+            }
+        }
+    }
+    TileInfo t = {0, 0, 0, 0, 0};
+    if (active) {
+        t = decode_tile(p, prefix, row_start, tile);
+        // slots of the contributors, computed before the wait (the load loop below must not divide)
+        for (int j = threadIdx.x; j <= c_hi - c_lo && j < kRangeTabMax; j += blockDim.x) slot_of[j] = sched.slot(c_lo + j, tile);
+    }
+    __syncthreads();
+    // EVERY CTA waits, also those with nothing to add: a grid whose CTAs all left before the GEMM grid finished
+    // would count as complete, and the kernel after it in the stream would stop waiting for the GEMM.
+    if (kStandalone) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!active) return;
+    float* dst = p.C + int64_t(t.row0) * p.ldc + t.n0;
+    const int vec_per_row = p.BN / 4;
+    const int total_vec = t.rows * vec_per_row;
+    const int v_begin = int(static_cast<long long>(total_vec) * share / shares);
+    const int v_end = int(static_cast<long long>(total_vec) * (share + 1) / shares);
+    const size_t slot_floats = size_t(p.BM) * p.BN;
+    const int nthr = int(blockDim.x);
+    for (int v0 = v_begin; v0 < v_end; v0 += 4 * nthr) {
+        float4 sum[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sum[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {         // four contributors' loads in flight together
+            float4 x[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool c_ok = c0 + j <= c_hi;
+                const int jj = c_ok ? c0 + j - c_lo : 0;
+                const int slot = jj < kRangeTabMax ? slot_of[jj] : sched.slot(c_lo + jj, tile);
+                const float4* src = reinterpret_cast<const float4*>(p.partials + size_t(slot) * slot_floats);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int v = v0 + q * nthr + int(threadIdx.x);
+                    x[j][q] = (c_ok && v < v_end) ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (c0 + j > c_hi) break;                  // absent contributors add nothing (not even +0)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    sum[q].x += x[j][q].x; sum[q].y += x[j][q].y; sum[q].z += x[j][q].z; sum[q].w += x[j][q].w;
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int v = v0 + q * nthr + int(threadIdx.x);
+            if (v < v_end) {
+                const int r = v / vec_per_row, c4 = (v % vec_per_row) * 4;
+                if (t.n0 + c4 < p.N) {
+                    if (p.epi_swiglu) {
+                        const __nv_bfloat16 lo = swiglu_bf16(sum[q].x, sum[q].y), hi = swiglu_bf16(sum[q].z, sum[q].w);
+                        *reinterpret_cast<uint32_t*>(p.H + int64_t(t.row0 + r) * p.ldh + ((t.n0 + c4) >> 1)) =
+                            uint32_t(__bfloat16_as_ushort(lo)) | (uint32_t(__bfloat16_as_ushort(hi)) << 16);
+                    } else if (p.Cb) {
+                        const uint32_t lo = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].x))) |
+                                            (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].y))) << 16);
+                        const uint32_t hi = uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].z))) |
+                                            (uint32_t(__bfloat16_as_ushort(__float2bfloat16_rn(sum[q].w))) << 16);
+                        *reinterpret_cast<uint2*>(p.Cb + int64_t(t.row0 + r) * p.ldc + t.n0 + c4) = make_uint2(lo, hi);
+                    } else {
+                        *reinterpret_cast<float4*>(dst + int64_t(r) * p.ldc + c4) = sum[q];
+                    }
+                }
+            }
+        }
     }
 }
 
@@ -931,6 +1065,10 @@ int launch_gemm_wn_bf16(int bk, int bn, const cudaLaunchConfig_t* cfg, const Gem
 int launch_gemm_wn_fp8(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
 int launch_gemm_wm_bf16(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
 int launch_gemm_wm_fp8(int bk, int bn, const cudaLaunchConfig_t* cfg, const GemmParams& p);
+// Two grouped products in one cooperative launch (tl_gemm_chain.cu); weights-on-N, bf16, tile 64 x 256 only.
+int launch_gemm_chain(int bk, int bn, int grid, size_t smem, cudaStream_t stream, const GemmParams& p1,
+                      const GemmParams& p2, unsigned long long* counter, unsigned long long target1,
+                      unsigned long long target2);
 // CTA-pair kernel (tl_gemm_pair.cu): halves = 2 for 512-token tiles.
 int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream_t stream, const GemmParams& p);
 // Clusters of the pair kernel that can be resident together on the current device.

@@ -116,3 +116,37 @@ def test_unsupported_and_invalid():
     with pytest.raises(tl.TileLensError) as e:
         tl.gemm_grouped_swiglu(X, W, H, off, 1, 300, 96, 128, 0, 0, 0)                      # N not a multiple of 64
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("E,hidden,inter,tokens,topk", [(8, 256, 128, 64, 2), (128, 2048, 768, 256, 8), (16, 128, 512, 96, 4),
+                                                       (3, 4096, 64, 700, 1)])
+def test_one_launch_and_two_launches_give_the_same_bits(E, hidden, inter, tokens, topk):
+    # With TL_OPT_FFN_ONE_LAUNCH = 1 tl_moe_ffn runs both products as two phases of one cooperative launch (a
+    # grid-wide barrier between them, the first product's split tiles summed inside the kernel) instead of two
+    # launches.  Same tiles, same K ranges, same order of every sum: H and Y must agree bit for bit, repeatedly.
+    from gpu_util import DEV, guarded_out, tl
+    offsets, counts, _ = inputs.zipf_topk_routing(tokens, E, topk, 1.1, seed=3)
+    rows = int(offsets[-1])
+    X = inputs.bf16_normal((rows, hidden), 1.0, seed=1, device=DEV)
+    Wgu = inputs.bf16_normal((E, hidden, 2 * inter), 0.05, seed=2, device=DEV)
+    Wd = inputs.bf16_normal((E, inter, hidden), 0.05, seed=3, device=DEV)
+    Wgu_t, Wd_t = torch.empty_like(Wgu), torch.empty_like(Wd)
+    tl.relayout(Wgu, Wgu_t, E * hidden, 2 * inter, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    tl.relayout(Wd, Wd_t, E * inter, hidden, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    d_off = torch.from_numpy(offsets).to(DEV)
+
+    def run():
+        gH, gY = guarded_out((rows, inter), torch.bfloat16), guarded_out((rows, hidden), torch.float32)
+        tl.moe_ffn(X, Wgu_t, Wd_t, gH.t, gY.t, d_off, E, rows, hidden, inter, 4096, 16, 128)
+        chained = tl.gemm_last_plan().chained
+        tl.device_status()
+        return gH.check().clone(), gY.check().clone(), chained
+
+    H0, Y0, chained0 = run()
+    assert chained0 == 0
+    for rep in range(3):
+        with tl.option(tl.OPT_FFN_ONE_LAUNCH, 1):
+            H1, Y1, chained1 = run()
+        assert chained1 == 1, "the one-launch form was not taken"
+        assert torch.equal(H1.view(torch.int16), H0.view(torch.int16)) and torch.equal(Y1, Y0), rep
+    assert torch.isfinite(Y1).all()
