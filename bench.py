@@ -942,7 +942,10 @@ def run_sweep(args):
         torch.cuda.synchronize()
         return statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3      # us
 
-    ctas = ((64, 64, 64), (128, 128, 64), (256, 128, 64))
+    # "CTA tile X x Y" of the workload list is token rows x weight columns; the K step is the kernel's own: 128 weight
+    # rows per stage for the 64- and 128-column tiles (half as many barrier hand-offs per byte: 64 x 64 runs at 3.1
+    # instead of 2.4 TB/s), 64 for the 256-token tile, whose token side already fills the stage
+    ctas = ((64, 64, 128), (128, 128, 128), (256, 128, 64))
     base = {}
     for cta in ctas:
         for M in (1, 16, 128):

@@ -701,6 +701,16 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         cfg.numAttrs = n_attr;
         if (plan.weights_on_n) rc = es == 1 ? launch_gemm_wn_fp8(plan.BK, plan.BN, &cfg, p) : launch_gemm_wn_bf16(plan.BK, plan.BN, &cfg, p);
         else rc = es == 1 ? launch_gemm_wm_fp8(plan.BK, plan.BN, &cfg, p) : launch_gemm_wm_bf16(plan.BK, plan.BN, &cfg, p);
+        if (rc == TL_ERR_CUDA && plan.cluster_k > 1) {
+            // A device (or a partition of one) that cannot place clusters of this size refuses the launch; nothing was
+            // enqueued.  The stream-K cut computes the same product.
+            const int64_t saved = opt(TL_OPT_NO_SCRATCH_PLANS);
+            tl_set_option(TL_OPT_NO_SCRATCH_PLANS, 0);
+            rc = gemm_launch(d_A, d_B, d_C, d_offsets, E, rows_total, rows_max, N, K, G, br, bc, cta_m, cta_n, cta_k, stream,
+                             fixed, kmajor, elem_bytes, d_H_swiglu, d_C_bf16, nullptr, nullptr, nullptr);
+            tl_set_option(TL_OPT_NO_SCRATCH_PLANS, saved);
+            return rc;
+        }
         if (rc) return rc;
     }
     // stream-K: add up the partial tiles, one CTA per boundary between two CTA ranges

@@ -140,7 +140,7 @@ def test_granularity_sweep_layouts_every_cta_tile(G, br, bc):
         ii, jj = rng.integers(0, M, 150), rng.integers(0, N, 150)
         ii[:2], jj[:2] = [0, M - 1], [0, N - 1]
         ref, _ = tlo.matmul_at(inputs.bits(A), inputs.bits(Bd.reshape(-1)), TILE, br, bc, M, N, K, ii, jj)
-        for cta in ((64, 64, 64), (128, 128, 64), (256, 128, 64)):
+        for cta in ((64, 64, 128), (128, 128, 128), (256, 128, 64), (64, 64, 64)):
             C = run_gemm(A, Bd, M, N, K, br, bc, cta)
             assert np.array_equal(C.cpu().numpy()[ii, jj].astype(np.float64), ref), (M, cta)
             assert torch.isfinite(C).all()

@@ -136,6 +136,42 @@ def test_cluster_split_k_against_the_oracle_and_the_stream_k_cut(M, N, K, want_s
     assert torch.equal(g.check(), C.to(torch.bfloat16))                 # the same fp32 sums, rounded once
 
 
+@pytest.mark.parametrize("limit", [100, 37, 1])
+def test_sm_limit_caps_the_grid_and_keeps_the_product_exact(limit):
+    from gpu_util import run_gemm, tl
+    for M, N, K in ((8, 2048, 4096), (200, 1024, 512), (1800, 5120, 384)):
+        A, Bd, want = _int_case(M, N, K, 16, 128, seed=M)
+        with tl.option(tl.OPT_SM_LIMIT, limit):
+            got = run_gemm(A, Bd, M, N, K, 16, 128)
+            plan = tl.gemm_last_plan()
+        assert torch.equal(got.cpu(), want)
+        assert plan.pair_kernel == 1 or plan.grid <= limit, plan.as_dict()      # (the CTA-pair kernel keeps its own grid)
+
+
+@pytest.mark.parametrize("cap", [16, 64, 128])
+def test_grouped_row_cap_keeps_the_products_exact(cap):
+    # tiles of up to 128 token rows per expert: 128-row MMAs for the large experts, 64-row ones for the rest
+    from gpu_util import DEV, guarded_out, tl
+    E, K, N = 12, 512, 768
+    offsets, counts, expert_of_row = inputs.zipf_topk_routing(160, E, 3, 1.1, seed=7)
+    rows = int(offsets[-1])
+    assert counts.max() > 64                                                      # at least one expert needs the 128-row path
+    A = inputs.bf16_integers((rows, K), -8, 8, seed=1)
+    B = inputs.bf16_integers((E, K, N), -8, 8, seed=2)
+    Bt = torch.empty((E, K, N), dtype=torch.bfloat16, device=DEV)
+    tl.relayout(B.to(DEV), Bt, E * K, N, 2, 4096, 16, 128, tl.TO_TILE_MAJOR)
+    want = torch.empty((rows, N), dtype=torch.float32)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        want[r0:r1] = (A[r0:r1].double() @ B[e].double()).float()
+    with tl.option(tl.OPT_MOE_ROW_CAP, cap):
+        g = guarded_out((rows, N), torch.float32)
+        tl.gemm_grouped(A.to(DEV), Bt, g.t, torch.from_numpy(offsets).to(DEV), E, rows, N, K, 4096, 16, 128)
+        assert tl.gemm_last_plan().cta_m == cap
+        tl.device_status()
+    assert torch.equal(g.check().cpu(), want)
+
+
 def test_relayout_without_the_copy_engine_matches_the_oracle():
     from gpu_util import Guarded, dev_bytes, tl
     for rows, cols, s, br, bc in ((512, 512, 2, 16, 128), (1056, 2176, 2, 32, 64), (256, 1024, 1, 64, 64)):
