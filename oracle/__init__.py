@@ -82,6 +82,9 @@ def lib() -> ctypes.CDLL:
         L.tlo_read_amp_shared.argtypes = [i64] * 7 + [ctypes.c_int] + [i64] * 4 + [u64p, u64p, u64p]
         L.tlo_prefetch_degree.restype = i64
         L.tlo_prefetch_degree.argtypes = [ctypes.c_double, ctypes.c_double, i64, i64, i64, i64, i64, i64, ctypes.c_double]
+        L.tlo_tile_arrival.restype = ctypes.c_int
+        L.tlo_tile_arrival.argtypes = [vp, i64, i64, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
+                                       ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
         L.tlo_double_to_bf16.restype = ctypes.c_uint16
         L.tlo_double_to_bf16.argtypes = [ctypes.c_double]
         L.tlo_silu.restype = ctypes.c_double
@@ -227,6 +230,16 @@ def read_amp_shared(M, N, K, BM, BN, BK, P, layout, G, br, bc, s):
     if rc != 0:
         raise ValueError(f"tlo_read_amp_shared rejected its arguments (rc={rc})")
     return int(f.value), int(u.value), int(q.value)
+
+
+def tile_arrival(samples, requests: int, threshold: float = 0.0):
+    """(E[first arrival], E[last arrival], P(last arrival > threshold)) of `requests` independent draws from the sample."""
+    x = np.ascontiguousarray(samples, dtype=np.float64)
+    first, last, late = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    if lib().tlo_tile_arrival(_ptr(x), x.size, requests, threshold, ctypes.byref(first), ctypes.byref(last),
+                              ctypes.byref(late)) != 0:
+        raise ValueError("tlo_tile_arrival rejected its arguments")
+    return first.value, last.value, late.value
 
 
 def prefetch_degree(bandwidth, latency, G, n_sm, ctas_per_sm, p_tile, K, tile_k, collision_factor=1.0) -> int:

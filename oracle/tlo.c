@@ -481,6 +481,48 @@ int64_t tlo_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int6
     return d < cap ? d : cap;
 }
 
+/* Section 6.5 ("Straggler-Induced CTA Stalls"): a CTA issues the n requests of a compute tile together and can
+ * start only when the last one has arrived; the section measures the time to the first arrival ("queueing") and the
+ * time between the first and the last ("straggler wait"), and explains the gap between layouts by the chance that
+ * the slowest of n requests falls in the tail of the per-request latency distribution.
+ * The paper gives that distribution only as figures, so none is assumed here: the caller passes a sample of
+ * per-request latencies (a measurement, a trace), read as the distribution that puts probability 1/N on each
+ * sample value, and the n requests of a tile are read as independent draws from it.  Then, with the sample sorted,
+ *   P(last arrival <= x_(i)) = (i/N)^n,    P(first arrival > x_(i)) = ((N - i)/N)^n,
+ * which give the two expectations below as plain sums over the sorted sample, and
+ *   P(last arrival > t) = 1 - (#{x <= t} / N)^n.
+ * Returns 0, or -1 for bad arguments. */
+static int tlo_cmp_double(const void* a, const void* b) {
+    const double x = *(const double*)a, y = *(const double*)b;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+int tlo_tile_arrival(const double* samples, int64_t N, int64_t n, double threshold, double* first, double* last,
+                     double* p_late) {
+    if (!samples || N <= 0 || n <= 0 || !first || !last) return -1;
+    double* x = (double*)malloc((size_t)N * sizeof(double));
+    if (!x) return -1;
+    for (int64_t i = 0; i < N; ++i) x[i] = samples[i];
+    qsort(x, (size_t)N, sizeof(double), tlo_cmp_double);
+    long double e_max = 0.0L, e_min = 0.0L;
+    int64_t below = 0;
+    for (int64_t i = 1; i <= N; ++i) {
+        /* probability that the largest of n draws is exactly the i-th smallest sample value, and the same for the
+         * smallest of n draws */
+        const long double p_max = powl((long double)i / (long double)N, (long double)n) -
+                                  powl((long double)(i - 1) / (long double)N, (long double)n);
+        const long double p_min = powl((long double)(N - i + 1) / (long double)N, (long double)n) -
+                                  powl((long double)(N - i) / (long double)N, (long double)n);
+        e_max += p_max * (long double)x[i - 1];
+        e_min += p_min * (long double)x[i - 1];
+        if (x[i - 1] <= threshold) ++below;
+    }
+    *first = (double)e_min;
+    *last = (double)e_max;
+    if (p_late) *p_late = (double)(1.0L - powl((long double)below / (long double)N, (long double)n));
+    free(x);
+    return 0;
+}
+
 /* ------------------------------------------- MoE expert FFN (Section 2.3 names the workload; epilogues are ours)
  *
  * The paper's MoE kernel is the two grouped products of an expert FFN; it does not describe what happens between

@@ -118,6 +118,11 @@ int tlo_read_amp_shared(int64_t M, int64_t N, int64_t K, int64_t BM, int64_t BN,
 /* Eq. 6 (Section 5.2): stride-prefetch degree d = min(floor(c*B*L/p_wave), K/TILE_K), B*L in requests of G bytes,
  * p_wave = n_sm * ctas_per_sm * p_tile; c = 1 as printed, 2 "in practice".  Pinned by the inequality the paper
  * derives it from (p_wave*(d+1) >= B*L > p_wave*d when not capped) and its monotonicity, not by a printed value. */
+/* Section 6.5: expected time to the first and to the last arrival of the n requests of a compute tile, and the
+ * probability that the last one arrives after `threshold`, for per-request latencies drawn independently from the
+ * caller's sample (probability 1/N per value). */
+int tlo_tile_arrival(const double* samples, int64_t N, int64_t n, double threshold, double* first, double* last,
+                     double* p_late);
 int64_t tlo_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64_t G, int64_t n_sm, int64_t ctas_per_sm,
                             int64_t p_tile, int64_t K, int64_t tile_k, double collision_factor);
 
