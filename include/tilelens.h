@@ -445,6 +445,20 @@ int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64
                            double collision_factor);
 
 /*
+ * What the request count of a tile costs in time (Section 6.5, "Straggler-Induced CTA Stalls"): a CTA issues the
+ * requests of a compute tile together and starts when the LAST one has arrived; the more requests, the likelier that
+ * the slowest falls in the tail of the per-request latency distribution.  The paper shows its distribution only in
+ * figures, so the caller supplies one: h_latencies, `count` measured per-request latencies (any unit), read as the
+ * distribution that gives each sample value probability 1/count, the `requests` requests of a tile as independent
+ * draws from it (requests = tl_read_amp's request count divided by tile loads).  Returns the expected time to the
+ * first arrival (the section's "queueing" phase), to the last arrival (first + "straggler wait"), and, if p_late
+ * is not NULL, the probability that the last arrival comes after `threshold`.  Host arithmetic only.
+ * TL_ERR_INVALID_ARG for an empty sample, a NaN, or requests <= 0.
+ */
+int tl_tile_arrival_latency(const double* h_latencies, int64_t count, int64_t requests, double threshold,
+                            double* first_arrival, double* last_arrival, double* p_late);
+
+/*
  * tl_read_amp without the wait: the three totals (bytes_fetched, bytes_used, requests) are written to d_totals,
  * 3 uint64 in DEVICE memory (or mapped pinned host memory), by the kernel's last CTA.  Asynchronous on
  * cuda_stream; successive counter calls must be ordered by one stream (they share their accumulators).

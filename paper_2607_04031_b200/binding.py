@@ -50,6 +50,8 @@ _SIGNATURES = {
     "tl_read_amp_batch": (_int, [_vp, _int, _vp, _vp]),
     "tl_read_amp_shared": (_int, [_i64, _i64, _i64, _int, _int, _int, _i64, _int, _i64, _int, _int, _int, _vp, _vp, _vp]),
     "tl_prefetch_degree": (_i64, [ctypes.c_double, ctypes.c_double, _i64, _i64, _i64, _i64, _i64, _i64, ctypes.c_double]),
+    "tl_tile_arrival_latency": (_int, [_vp, _i64, _i64, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
+                                       ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "tl_hw_box_offsets": (_int, [_vp, _vp, _i64, _vp, _vp]),
     "tl_hw_box_load": (_int, [_vp, _vp, ctypes.c_uint64, _vp, _i64, _vp, _vp]),
     "tl_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _int, _int, _int]),
@@ -408,6 +410,17 @@ def prefetch_degree(bandwidth_bytes_per_s: float, latency_s: float, G: int, n_sm
     if d < 0:
         raise ValueError("tl_prefetch_degree: bad arguments")
     return d
+
+
+def tile_arrival_latency(latencies, requests: int, threshold: float = 0.0):
+    """(E[first arrival], E[last arrival], P(last arrival > threshold)) for `requests` requests per tile whose
+    latencies are independent draws from the sample `latencies` (host arithmetic, Section 6.5)."""
+    import numpy as np
+    x = np.ascontiguousarray(latencies, dtype=np.float64)
+    first, last, late = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    _check(lib().tl_tile_arrival_latency(x.ctypes.data, x.size, requests, threshold, ctypes.byref(first),
+                                         ctypes.byref(last), ctypes.byref(late)), "tl_tile_arrival_latency")
+    return first.value, last.value, late.value
 
 
 def read_amp_grouped(offsets_host, N: int, K: int, cta, layout: int, G: int, block_rows: int = 0,

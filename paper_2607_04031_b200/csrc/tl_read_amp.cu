@@ -12,6 +12,10 @@
 //   col-major   the same with the roles of rows and columns exchanged.
 #include "tl_common.cuh"
 
+#include <algorithm>
+#include <cmath>
+#include <vector>
+
 #include <cstdlib>
 #include <cstring>
 
@@ -300,6 +304,40 @@ int64_t tl_prefetch_degree(double bandwidth_bytes_per_s, double latency_s, int64
     const int64_t cap = K / cta_k;
     if (q >= (long double)cap) return cap;
     return (int64_t)q;
+}
+
+int tl_tile_arrival_latency(const double* h_latencies, int64_t count, int64_t requests, double threshold,
+                            double* first_arrival, double* last_arrival, double* p_late) {
+    if (!h_latencies || count <= 0 || requests <= 0 || !first_arrival || !last_arrival) return TL_ERR_INVALID_ARG;
+    std::vector<double> x(h_latencies, h_latencies + count);
+    for (double v : x)
+        if (!(v == v)) return TL_ERR_INVALID_ARG;          // NaN
+    std::sort(x.begin(), x.end());
+    // Summation by parts over the sorted sample: the largest of n draws exceeds x_(i) with probability
+    // 1 - (i/N)^n, the smallest with probability ((N - i)/N)^n, so
+    //   E[max] = x_(N) - sum_i (x_(i+1) - x_(i)) (i/N)^n,    E[min] = x_(1) + sum_i (x_(i+1) - x_(i)) ((N - i)/N)^n.
+    const double N = double(count), n = double(requests);
+    double gap_max = 0.0, gap_min = 0.0, c_max = 0.0, c_min = 0.0;      // Kahan sums
+    int64_t below = 0;
+    for (int64_t i = 1; i < count; ++i) {
+        const double step = x[size_t(i)] - x[size_t(i) - 1];
+        if (step != 0.0) {
+            const double a = step * std::pow(double(i) / N, n) - c_max;
+            const double t = gap_max + a;
+            c_max = (t - gap_max) - a;
+            gap_max = t;
+            const double b = step * std::pow(double(count - i) / N, n) - c_min;
+            const double u = gap_min + b;
+            c_min = (u - gap_min) - b;
+            gap_min = u;
+        }
+    }
+    for (int64_t i = 0; i < count; ++i)
+        if (x[size_t(i)] <= threshold) ++below;
+    *last_arrival = x.back() - gap_max;
+    *first_arrival = x.front() + gap_min;
+    if (p_late) *p_late = 1.0 - std::pow(double(below) / N, n);
+    return TL_OK;
 }
 
 int tl_read_amp_async(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k, int layout, int64_t G,
