@@ -92,6 +92,8 @@ typedef enum {
                                 first pipeline stage of every CTA for 16 bytes more than its copies deliver, so that
                                 the wait on that stage runs out after TL_OPT_WAIT_LIMIT_US, the kernel gives up (drains
                                 its copies, frees tensor memory, returns) and tl_device_status() reports TL_ERR_TIMEOUT.
+                                3 = in the next one-launch tl_moe_ffn CTA 0 does not arrive at the grid barrier, so every
+                                CTA's bounded wait there runs out (detail 0x800).
                                 That launch's output is undefined.  The option resets itself to 0 when it is consumed. */
     TL_OPT_MOE_ROW_CAP,      /* grouped products: most token rows per tile; 0 (default): the library's choice, else 16/32/64/128 */
     TL_OPT_REDUCE_SPLIT,     /* 1 (default): a split tile's partial sums are added by all reduction CTAs inside it, 0: by one */

@@ -841,8 +841,12 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
             p1.partials = p2.partials = static_cast<float*>(ws);
             const unsigned long long base = d.grid_arrivals;
             const size_t smem = plan1.smem_bytes > plan2.smem_bytes ? plan1.smem_bytes : plan2.smem_bytes;
+            // Test hook (TL_OPT_STALL_ONCE = 3): CTA 0 does not arrive at the first grid barrier, so every CTA's bounded
+            // wait there (and at the second barrier, which then cannot fill either) runs out and is reported.
+            const bool skip = tl::opt(TL_OPT_STALL_ONCE) == 3;
+            if (skip) tl_set_option(TL_OPT_STALL_ONCE, 0);
             rc = tl::launch_gemm_chain(plan1.BK, plan1.BN, grid, smem, stream, p1, p2, d.d_grid_counter,
-                                       base + grid, base + 2ull * grid);
+                                       base + grid, base + 2ull * grid, skip);
             if (rc) return rc;
             d.grid_arrivals = base + 2ull * grid;
             tl_gemm_plan_info& info = tl::last_plan();

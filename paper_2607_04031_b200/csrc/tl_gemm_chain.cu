@@ -23,13 +23,14 @@
 namespace tl {
 
 // Returns false when the wait ran out.
+// (skip_arrival: test hook -- this CTA polls without having arrived, so that every CTA's wait runs out.)
 __device__ __forceinline__ bool grid_barrier(unsigned long long* counter, unsigned long long target, uint64_t limit_ns,
-                                             uint32_t* status) {
+                                             uint32_t* status, bool skip_arrival = false) {
     __shared__ int ok_flag;
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();                                   // this CTA's writes before its arrival
-        atomicAdd(counter, 1ull);
+        if (!skip_arrival) atomicAdd(counter, 1ull);
         bool ok = true;
         uint64_t t0 = 0;
         uint32_t polls = 0;
@@ -60,12 +61,12 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* counter, unsign
 template <int kBK, int kBN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_chain_kernel(const __grid_constant__ GemmParams p1, const __grid_constant__ GemmParams p2,
-                  unsigned long long* counter, unsigned long long target1, unsigned long long target2) {
+                  unsigned long long* counter, unsigned long long target1, unsigned long long target2, int skip_cta0) {
     __shared__ int prefix[kMaxExperts + 1];
     __shared__ int row_start[kMaxExperts + 1];
     __shared__ int slot_of[kRangeTabMax];
     gemm_body<kBK, kBN, true, false>(p1, true, false);
-    const bool ok1 = grid_barrier(counter, target1, p1.wait_limit_ns, p1.status);
+    const bool ok1 = grid_barrier(counter, target1, p1.wait_limit_ns, p1.status, skip_cta0 != 0 && blockIdx.x == 0);
     if (ok1 && int(blockIdx.x) + 1 < int(gridDim.x))
         streamk_reduce_body<false>(p1, int(gridDim.x), int(blockIdx.x), prefix, row_start, slot_of);
     grid_barrier(counter, target2, p1.wait_limit_ns, p1.status);
@@ -74,7 +75,7 @@ gemm_chain_kernel(const __grid_constant__ GemmParams p1, const __grid_constant__
 
 int launch_gemm_chain(int bk, int bn, int grid, size_t smem, cudaStream_t stream, const GemmParams& p1,
                       const GemmParams& p2, unsigned long long* counter, unsigned long long target1,
-                      unsigned long long target2) {
+                      unsigned long long target2, bool skip_cta0) {
     if (bk != 64 || bn != 256) return TL_ERR_UNSUPPORTED;
     auto* kernel = gemm_chain_kernel<64, 256>;
     // (this kernel's static shared memory is about 10 KB above the plain GEMM kernel's)
@@ -89,7 +90,7 @@ int launch_gemm_chain(int bk, int bn, int grid, size_t smem, cudaStream_t stream
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return check_cuda(cudaLaunchKernelEx(&cfg, kernel, p1, p2, counter, target1, target2));
+    return check_cuda(cudaLaunchKernelEx(&cfg, kernel, p1, p2, counter, target1, target2, int(skip_cta0)));
 }
 
 }  // namespace tl

@@ -1068,7 +1068,7 @@ int launch_gemm_wm_fp8(int bk, int bn, const cudaLaunchConfig_t* cfg, const Gemm
 // Two grouped products in one cooperative launch (tl_gemm_chain.cu); weights-on-N, bf16, tile 64 x 256 only.
 int launch_gemm_chain(int bk, int bn, int grid, size_t smem, cudaStream_t stream, const GemmParams& p1,
                       const GemmParams& p2, unsigned long long* counter, unsigned long long target1,
-                      unsigned long long target2);
+                      unsigned long long target2, bool skip_cta0);
 // CTA-pair kernel (tl_gemm_pair.cu): halves = 2 for 512-token tiles.
 int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream_t stream, const GemmParams& p);
 // Clusters of the pair kernel that can be resident together on the current device.

@@ -150,3 +150,36 @@ def test_one_launch_and_two_launches_give_the_same_bits(E, hidden, inter, tokens
         assert chained1 == 1, "the one-launch form was not taken"
         assert torch.equal(H1.view(torch.int16), H0.view(torch.int16)) and torch.equal(Y1, Y0), rep
     assert torch.isfinite(Y1).all()
+
+
+def test_grid_barrier_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
+    # One-launch form: CTA 0 stays away from the first grid barrier (test hook), every CTA's bounded wait runs out
+    # after the shortened limit, the kernel still terminates, the status reads TL_ERR_TIMEOUT (detail 0x800), the
+    # arrival counter is reset by the report, and the next call gives the bits of the two-launch form.
+    from gpu_util import DEV, tl
+    E, hidden, inter = 16, 128, 512
+    offsets, counts, _ = inputs.zipf_topk_routing(96, E, 4, 1.1, seed=4)
+    rows = int(offsets[-1])
+    X = inputs.bf16_normal((rows, hidden), 1.0, seed=1, device=DEV)
+    Wgu = inputs.bf16_normal((E, hidden, 2 * inter), 0.05, seed=2, device=DEV)
+    Wd = inputs.bf16_normal((E, inter, hidden), 0.05, seed=3, device=DEV)
+    d_off = torch.from_numpy(offsets).to(DEV)
+    H = torch.zeros((rows, inter), dtype=torch.bfloat16, device=DEV)
+    Y = torch.zeros((rows, hidden), dtype=torch.float32, device=DEV)
+    tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)          # two launches: the reference bits
+    tl.device_status()
+    H0, Y0 = H.clone(), Y.clone()
+    with tl.option(tl.OPT_FFN_ONE_LAUNCH, 1), tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
+        tl.set_option(tl.OPT_STALL_ONCE, 3)
+        tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)
+        assert tl.get_option(tl.OPT_STALL_ONCE) == 0 and tl.gemm_last_plan().chained == 1
+        with pytest.raises(tl.TileLensError) as e:
+            tl.device_status()
+        assert e.value.status == 5 and "detail=0x800" in str(e.value)
+        tl.device_status()
+        for _ in range(2):
+            H.zero_(); Y.zero_()
+            tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)
+            assert tl.gemm_last_plan().chained == 1
+            tl.device_status()
+            assert torch.equal(H.view(torch.int16), H0.view(torch.int16)) and torch.equal(Y, Y0)
