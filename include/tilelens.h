@@ -173,11 +173,15 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
  *   beside two operand stages (cta_n * cta_k < 256 * 128), else
  *   TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
  * When the output tiles do not fill the SMs (decode, small or grouped
- * problems) the K loops are cut stream-K fashion over all SMs; partial tiles
- * go through a workspace and a second small kernel adds them in a fixed
- * order, so results are reproducible run to run.  The workspace is the
- * caller's (tl_set_workspace) or one the library grows on demand; calls that
- * may run concurrently on one GPU must not share a workspace.
+ * problems) the K loops are cut: inside thread-block clusters whose CTAs
+ * add their partial tiles through distributed shared memory where such a
+ * schedule exists (no workspace), else stream-K fashion over all SMs, with
+ * partial tiles going through a workspace and a second small kernel adding
+ * them.  Either way the order of every sum is fixed: results are
+ * reproducible run to run.  tl_gemm_plan() tells which schedule a call runs.
+ * The workspace is the caller's (tl_set_workspace) or one the library grows
+ * on demand; calls that may run concurrently on one GPU must not share a
+ * workspace.
  * M == 0 is a no-op.
  */
 int tl_gemm(const void* d_A_rowmajor, const void* d_B_tilemajor, float* d_C,

@@ -12,20 +12,26 @@
 //                tiles of up to 64 tokens, else 128 rows; spare rows are zeroed once), one MMA covers all cta_n
 //                weight columns; TMEM lane = token row;
 //   weights on M (256-token tiles)  TMEM lane = weight column, the accumulator holds C transposed.
-// Memory tiles whose rows are shorter than 32 bytes cannot be boxed: four more warps load them with Eq. 1-2
-// address arithmetic and build the operand image by hand (Section 4.4).
+// Memory tiles whose rows are shorter than 32 bytes cannot be boxed: one more warp streams them into shared memory
+// with untiled bulk copies and four more permute them into the operand image with Eq. 1-2 arithmetic (Section 4.4).
 //
 // One persistent CTA per SM:
 //   warp 0      TMA producer   (one lane)   ring of shared-memory stages, mbarrier expect-tx
 //   warp 1      MMA issuer     (one lane)   tcgen05.mma into one of two TMEM accumulators
 //   warps 2..5  epilogue                    tcgen05.ld -> fp32 -> C, or silu(gate) * up -> bf16 (expert FFN)
-//   warps 6..9  hand-addressed weight loads (only when the memory tile cannot be boxed)
-// Work is a list of (output tile, K range).  Data-parallel mode hands whole tiles round-robin; stream-K mode cuts
-// the flattened (tile, K iteration) space into one contiguous range per CTA (decode: all SMs stream weights even
-// when there are fewer tiles than SMs).  Partial tiles go to a workspace and a second small kernel
-// (streamk_reduce_kernel, launched with programmatic stream serialisation so that it is resident before this one
-// ends) adds them in K order and writes C.  Nothing ever spins on another CTA; every mbarrier wait is bounded
-// (see mbar_wait_bounded).  Large dense problems run on CTA pairs instead (tl_gemm_pair.cuh).
+//   warps 6..10 generic-address weights     (only when the memory tile cannot be boxed)
+// Work is a list of (output tile, K range); make_plan chooses among
+//   whole tiles round-robin (the tiles fill the SMs, or divide evenly over at least 3/4 of them);
+//   split-K inside clusters: one tile per cluster of up to 8 CTAs, each a share of the K loop, partial tiles added
+//       through distributed shared memory (decode-sized dense products; no workspace);
+//   whole rounds of tiles round-robin, then the flattened (tile, K iteration) space of the rest cut into one
+//       contiguous range per CTA ("stream-K"); partial tiles go to a workspace and a second small kernel
+//       (streamk_reduce_kernel, launched with programmatic stream serialisation so that it is resident before this
+//       one ends) adds them in K order and writes C.
+// Nothing ever spins on another CTA of another cluster; every mbarrier wait is bounded (see mbar_wait_bounded).
+// Large dense problems run on CTA pairs instead (tl_gemm_pair.cuh); the expert FFN can run its two products in one
+// cooperative launch (tl_gemm_chain.cu).  This file: the stream-K reduction kernel, the plan, the tensor maps, the
+// launches and the C entry points; the device code of the GEMM is in tl_gemm_kernel.cuh.
 #include "tl_gemm_kernel.cuh"
 
 #include <cstdio>
