@@ -838,6 +838,7 @@ PROFILE_CASES = {
     "moe_gate_up": ("moe", 0, 2048, 1536),
     "kmajor_decode_qkv_m8": ("kmajor", 8, 8192, 10240),     # weights [N][K], (64, 32) memory tiles of Eq. 2
     "fp8_decode_qkv_m8": ("fp8", 8, 8192, 10240),           # E4M3, 64 x 64 memory tiles
+    "fp8_prefill_o": ("fp8", 4096, 8192, 8192),             # E4M3, 64 x 64 memory tiles, CTA-pair kernel
     "hw_box_load_o": ("hw", 0, 8192, 8192),                 # every 64 x 256 box of the weight through a 2-D view
     "generic_16x8_m16": ("generic", 16, 8192, 8192),        # 16 x 8 memory tiles (16-byte rows): generic-address path
     "relayout_layer": ("relayout_batch", 0, 0, 0),          # the four Llama weights in one launch (3.4 GB resident)

@@ -103,6 +103,8 @@ typedef enum {
                                 0: always the stream-K cut */
     TL_OPT_FFN_ONE_LAUNCH,   /* 0 (default): tl_moe_ffn runs its two grouped products as two launches; 1: as two phases of one
                                 cooperative launch where it can (measured slower: 236 against 211 us on the Qwen-3 expert FFN) */
+    TL_OPT_PAIR_TMA_STORE,   /* 1 (default): the CTA-pair kernel writes C through shared memory with tiled bulk stores, 0: with
+                                plain stores straight from the accumulator registers (same values either way) */
     TL_OPT_COUNT_
 } tl_option;
 /* TL_ERR_INVALID_ARG for an unknown option or a value outside the option's range. */

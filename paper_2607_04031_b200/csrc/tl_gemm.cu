@@ -633,10 +633,17 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         const int64_t big_tiles = halves_off ? 0 : (big_total / max_clusters) * max_clusters;
         const int halves = big_tiles > 0 ? 2 : 1;
         const size_t stage_bytes = 64 * 128 * 2 + size_t(halves) * 128 * kAtomBytes;
-        const int stages = int((kMaxDynamicSmem - 1024) / stage_bytes);
-        p.num_stages = stages < kPairStagesMax ? stages : kPairStagesMax;
+        int stages = int((kMaxDynamicSmem - 1024) / stage_bytes);
+        if (stages > kPairStagesMax) stages = kPairStagesMax;
+        const int stage_cap = int(opt(TL_OPT_MAX_STAGES));
+        if (stage_cap >= 2 && stages > stage_cap) stages = stage_cap;
+        p.num_stages = stages;
         p.pair_big_tiles = int(big_tiles);
-        const size_t smem = size_t(p.num_stages) * stage_bytes + 1024;
+        // behind the stages: 32 x 32 blocks of C on their way to a bulk store, one or two per epilogue warp
+        const size_t out_warp_bytes = size_t(halves == 2 ? 8 : 4) * kPairStageOutBytes;
+        p.out_bufs = size_t(stages) * stage_bytes + 1024 + 2 * out_warp_bytes <= size_t(kPairDynamicSmem) ? 2 : 1;
+        const size_t smem = size_t(stages) * stage_bytes + 1024 + size_t(p.out_bufs) * out_warp_bytes;
+        if (smem > size_t(kPairDynamicSmem)) return TL_ERR_UNSUPPORTED;
         const int64_t pair_tiles = halves == 2 ? big_tiles + 2 * (big_total - big_tiles)
                                                : ceil_div(rows_total, 256) * ceil_div(N, 256);
         const int clusters = int(pair_tiles < max_clusters ? pair_tiles : max_clusters);
@@ -649,6 +656,20 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
             fprintf(stderr, "[tilelens] pair kernel: %lld tiles (%lld of 512 tokens), %d clusters (max active %d), %d stages, %zu B smem\n",
                     (long long)pair_tiles, (long long)big_tiles, clusters, max_clusters, p.num_stages, smem);
         if (plan_only) { *plan_only = info; return TL_OK; }
+        // C as a tensor map (bulk stores need 16-byte aligned rows); otherwise the epilogue stores from registers
+        p.c_tma = 0;
+        {
+            const void* c_base = d_C_bf16 ? d_C_bf16 : static_cast<const void*>(d_C);
+            const int c_es = d_C_bf16 ? 2 : 4;
+            if (opt(TL_OPT_PAIR_TMA_STORE) != 0 && reinterpret_cast<uintptr_t>(c_base) % 16 == 0 && (N * c_es) % 16 == 0) {
+                const uint64_t dims[2] = {uint64_t(N), uint64_t(rows_total)}, str[2] = {uint64_t(c_es), uint64_t(N) * c_es};
+                const uint32_t box[2] = {32, 32};
+                if (int rc = encode_tensor_map(&p.tmap_c, c_base, d_C_bf16 ? int(CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) : int(CU_TENSOR_MAP_DATA_TYPE_FLOAT32),
+                                               int(CU_TENSOR_MAP_SWIZZLE_NONE), 2, dims, str, box))
+                    return rc;
+                p.c_tma = 1;
+            }
+        }
         last_plan() = info;
         return launch_gemm_pair(es == 1, halves, clusters, smem, stream, p);
     }

@@ -20,6 +20,9 @@ constexpr int kMaxDynamicSmem = 227 * 1024 - 10 * 1024;   // 227 KB per CTA minu
 struct alignas(64) GemmParams {
     CUtensorMap tmap_a[kNumBoxChoices];
     CUtensorMap tmap_b;
+    CUtensorMap tmap_c;         // pair kernel, c_tma: C (fp32 or bf16) as [M][N] with boxes of 32 rows x 32 columns
+    int out_bufs;               // pair kernel: 32 x 32 blocks of C each epilogue warp may have on their way (1 or 2)
+    int c_tma;                  // 1: the pair kernel's epilogue stages C in shared memory and writes it with tiled bulk stores
     float* C;
     float* partials;            // stream-K partial tiles: slot = BM x BN floats
     const int32_t* offsets;     // grouped: device E+1 row offsets; dense: nullptr
@@ -1074,6 +1077,8 @@ int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream
 // Clusters of the pair kernel that can be resident together on the current device.
 int pair_max_active_clusters(int* out);
 constexpr int kPairStagesMax = 8;
+constexpr int kPairStageOutBytes = 4096;   // per epilogue warp: 32 tokens x 32 columns of fp32 C on their way to a bulk store
+constexpr int kPairDynamicSmem = 226 * 1024;   // the pair kernels' static shared memory is a few barriers only
 constexpr int kPairBigThreads = 320;       // pair kernel with 512-token tiles: producer, MMA issuer, eight epilogue warps
 
 }  // namespace tl

@@ -5,17 +5,17 @@
 namespace tl {
 
 int pair_max_active_clusters(int* out) {
-    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<false, 1>), kMaxDynamicSmem)) return rc;
-    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<true, 1>), kMaxDynamicSmem)) return rc;
-    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<false, 2>), kMaxDynamicSmem)) return rc;
-    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<true, 2>), kMaxDynamicSmem)) return rc;
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<false, 1>), kPairDynamicSmem)) return rc;
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<true, 1>), kPairDynamicSmem)) return rc;
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<false, 2>), kPairDynamicSmem)) return rc;
+    if (int rc = ensure_smem_attr(reinterpret_cast<const void*>(gemm_pair_kernel<true, 2>), kPairDynamicSmem)) return rc;
     if (int rc = ensure_device_info()) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * dev().sm_count);
-    cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = kMaxDynamicSmem;
+    cfg.blockDim = dim3(kPairBigThreads);
+    cfg.dynamicSmemBytes = kPairDynamicSmem;
     int n = 0;
-    if (int rc = check_cuda(cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<false, 1>, &cfg))) return rc;
+    if (int rc = check_cuda(cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<false, 2>, &cfg))) return rc;
     *out = n > 0 ? n : 1;
     return TL_OK;
 }

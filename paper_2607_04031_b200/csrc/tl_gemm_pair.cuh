@@ -16,7 +16,9 @@
 //     tcgen05.commit is multicast so the
 //     "stage free" and "accumulator ready" barriers of both CTAs fire together; "accumulator drained"
 //     arrivals of both CTAs' epilogue warps go to the leader;
-//   - each CTA's epilogue stores its own 128 columns of C, exactly as in the single-CTA kernel.
+//   - each CTA's epilogue writes its own 128 columns of C: every warp moves 32 tokens x 32 columns at a time from
+//     tensor memory through a 4 KB block of shared memory (behind the pipeline stages) to C with a tiled bulk
+//     store, which clips the ragged edges (plain stores from the registers when the switch is off).
 // With 256 x 256 tiles the kernel is held back by operand traffic out of L2 (32 KB per CTA per 64-row K step).  A
 // tile may therefore cover two 256-token blocks (kHalves = 2): one weight slab per stage serves both (48 KB per CTA
 // for twice the work, four stages), two MMAs per K step into the two halves of tensor memory, and eight epilogue
@@ -292,6 +294,8 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
         // =============================================================== epilogue (both CTAs)
         const int quarter = warp & 3;
         const int my_half = kHalves == 2 ? (warp - 2) >> 2 : 0;     // warps 2..5 drain token block 0, 6..9 block 1
+        uint8_t* out_stage = stages + size_t(p.num_stages) * kStageBytes + size_t(warp - 2) * p.out_bufs * kPairStageOutBytes;
+        uint32_t out_buf = 0;
         uint32_t acc = 0, acc_phase = 0;
         for (int tile = first_tile; tile < tiles_total; tile += tile_step) {
             const PairTile pt = pair_decode<kHalves>(p, tile, m_tiles, n_pair_tiles);
@@ -307,7 +311,47 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                     const int rows = p.M - row0 < 256 ? p.M - row0 : 256;
                     float* out = p.C + int64_t(row0) * p.ldc + n0;
                     const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * 256u + uint32_t(h) * 256u;
-                    if (p.Cb == nullptr) {
+                    if (p.c_tma) {
+                        // The 32 tokens x 32 columns this warp holds after one tcgen05.ld go to shared memory as a
+                        // row-major block (lane = column: conflict-free) and from there to C as one tiled bulk store,
+                        // which clips rows beyond M and columns beyond N.  The next block's tcgen05.ld is in flight
+                        // meanwhile.  The block is reused once the previous store has read it.
+                        const int cx = n0 + quarter * 32, chunks = (rows + 31) >> 5;
+                        uint32_t va[32], vb[32];
+                        auto emit = [&](const uint32_t (&v)[32], int c) {
+                            uint8_t* blk = out_stage + out_buf * kPairStageOutBytes;
+                            if (lane == 0) {
+                                if (p.out_bufs == 2) bulk_wait_group_read<1>(); else bulk_wait_group_read<0>();
+                            }
+                            __syncwarp();
+                            if (p.Cb == nullptr) {
+                                float* st = reinterpret_cast<float*>(blk);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) st[i * 32 + lane] = __uint_as_float(v[i]);
+                            } else {
+                                __nv_bfloat16* st = reinterpret_cast<__nv_bfloat16*>(blk);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) st[i * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                            }
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(&p.tmap_c, blk, cx, row0 + c * 32);
+                                bulk_commit_group();
+                            }
+                            if (p.out_bufs == 2) out_buf ^= 1;
+                        };
+                        tmem_ld_32x32b_x32(taddr, va);
+                        for (int c = 0; c < chunks; c += 2) {
+                            tmem_ld_wait();
+                            if (c + 1 < chunks) tmem_ld_32x32b_x32(taddr + (c + 1) * 32, vb);
+                            emit(va, c);
+                            if (c + 1 >= chunks) break;
+                            tmem_ld_wait();
+                            if (c + 2 < chunks) tmem_ld_32x32b_x32(taddr + (c + 2) * 32, va);
+                            emit(vb, c + 1);
+                        }
+                    } else if (p.Cb == nullptr) {
                         for (int c0 = 0; c0 < 256; c0 += 32) {
                             if (c0 >= rows) break;
                             uint32_t v[32];
@@ -315,7 +359,7 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
                             tmem_ld_wait();
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
-                                if (n_ok && c0 + i < rows) __stcs(out + int64_t(c0 + i) * p.ldc + n_local, __uint_as_float(v[i]));
+                                if (n_ok && c0 + i < rows) out[int64_t(c0 + i) * p.ldc + n_local] = __uint_as_float(v[i]);
                         }
                     } else {                                        // bf16 C
                         __nv_bfloat16* outb = p.Cb + int64_t(row0) * p.ldc + n0 + n_local;
@@ -338,6 +382,7 @@ gemm_pair_kernel(const __grid_constant__ GemmParams p) {
             if (acc == 0) acc_phase ^= 1;
             if (*abort_ptr) break;
         }
+        if (p.c_tma && lane == 0) bulk_wait_group<0>();             // this warp's stores are done before the CTA leaves
     }
 
     // Neither CTA may leave while its peer can still signal its barriers or read its shared memory.

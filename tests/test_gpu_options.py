@@ -62,7 +62,8 @@ def test_256_token_pair_tiles_are_what_small_prefill_runs():
 
 
 @pytest.mark.parametrize("opt_name,value", [("OPT_PAIR_KERNEL", 0), ("OPT_PAIR_512", 0), ("OPT_PDL", 0),
-                                            ("OPT_MAX_STAGES", 2), ("OPT_PREFETCH_STAGES", 0)])
+                                            ("OPT_MAX_STAGES", 2), ("OPT_PREFETCH_STAGES", 0),
+                                            ("OPT_PAIR_TMA_STORE", 0)])
 def test_prefill_switches_give_the_exact_product(opt_name, value):
     from gpu_util import run_gemm, tl
     M, N, K = 1800, 5120, 384                      # 512-token tiles and their 256-token remainder by default
@@ -76,7 +77,29 @@ def test_prefill_switches_give_the_exact_product(opt_name, value):
     if opt_name == "OPT_PAIR_512":
         assert plan.pair_kernel == 1 and plan.cta_m == 256
     if opt_name == "OPT_MAX_STAGES":
-        assert plan.pair_kernel == 1                # the cap applies to the single-CTA kernel only
+        assert plan.pair_kernel == 1 and plan.stages == 2
+    if opt_name == "OPT_PAIR_TMA_STORE":
+        assert plan.pair_kernel == 1 and plan.pair_tiles_512 > 0 and plan.pair_tiles_256 > 0
+
+
+@pytest.mark.parametrize("M,N,K", [(700, 9600, 320), (1800, 5120, 384), (257, 256 * 74, 64)])
+def test_pair_kernel_store_paths_write_the_same_bits(M, N, K):
+    # C through shared memory and tiled bulk stores (default) against plain stores from the accumulator registers:
+    # fp32 and bf16 C, ragged rows and columns, nothing outside C touched (guard blocks on both sides).
+    from gpu_util import DEV, guarded_out, run_gemm, tile_major_on_device, tl
+    A = inputs.bf16_normal((M, K), 1.0, seed=M)
+    Bt = tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=N), K, N, 16, 128)
+    got = {}
+    for mode in (1, 0):
+        with tl.option(tl.OPT_PAIR_TMA_STORE, mode):
+            got[mode] = run_gemm(A, Bt, M, N, K, 16, 128).clone()
+            assert tl.gemm_last_plan().pair_kernel == 1
+            g = guarded_out((M, N), torch.bfloat16)
+            tl.gemm_bf16(A.to(DEV), Bt, g.t, M, N, K, 4096, 16, 128)
+            tl.device_status()
+            got[mode, "bf16"] = g.check().clone()
+    assert torch.equal(got[1], got[0]) and torch.equal(got[1, "bf16"], got[0, "bf16"])
+    assert torch.equal(got[1].to(torch.bfloat16), got[1, "bf16"])
 
 
 @pytest.mark.parametrize("no_scratch", [1, 0])
