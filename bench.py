@@ -836,6 +836,7 @@ PROFILE_CASES = {
     "prefill_qkv": ("gemm", 4096, 8192, 10240),
     "relayout_o": ("relayout", 0, 8192, 8192),
     "moe_gate_up": ("moe", 0, 2048, 1536),
+    "moe_down": ("moe", 0, 768, 2048),
     "kmajor_decode_qkv_m8": ("kmajor", 8, 8192, 10240),     # weights [N][K], (64, 32) memory tiles of Eq. 2
     "fp8_decode_qkv_m8": ("fp8", 8, 8192, 10240),           # E4M3, 64 x 64 memory tiles
     "fp8_prefill_o": ("fp8", 4096, 8192, 8192),             # E4M3, 64 x 64 memory tiles, CTA-pair kernel

@@ -94,7 +94,11 @@ typedef enum {
                                 its copies, frees tensor memory, returns) and tl_device_status() reports TL_ERR_TIMEOUT.
                                 3 = in the next one-launch tl_moe_ffn CTA 0 does not arrive at the grid barrier, so every
                                 CTA's bounded wait there runs out (detail 0x800).
-                                That launch's output is undefined.  The option resets itself to 0 when it is consumed. */
+                                That launch's output is undefined.
+                                4 = the next grouped launch builds the tile tables it prepares ahead of its stream
+                                predecessor's completion from wrong expert offsets, so that its check after the wait
+                                must find them wrong and build them again; the output is the ordinary one.
+                                The option resets itself to 0 when it is consumed. */
     TL_OPT_MOE_ROW_CAP,      /* grouped products: most token rows per tile; 0 (default): the library's choice, else 16/32/64/128 */
     TL_OPT_REDUCE_SPLIT,     /* 1 (default): a split tile's partial sums are added by all reduction CTAs inside it, 0: by one */
     TL_OPT_SM_LIMIT,         /* 0 (default): GEMM grids use every SM; n > 0: at most n CTAs (leaves SMs to concurrent work) */

@@ -696,6 +696,12 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.stall_extra_tx = 16;
         tl_set_option(TL_OPT_STALL_ONCE, 0);
     }
+    // Test hook (TL_OPT_STALL_ONCE = 4): this grouped launch builds its provisional tables from offsets that are
+    // 7 rows off, so that the check after the wait finds them wrong and the tables are built again.
+    if (opt(TL_OPT_STALL_ONCE) == 4 && d_offsets) {
+        p.provisional_skew = 7;
+        tl_set_option(TL_OPT_STALL_ONCE, 0);
+    }
     if (params_only) {
         *params_only = p;
         *params_plan = plan;

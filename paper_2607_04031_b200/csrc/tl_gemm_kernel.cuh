@@ -29,6 +29,7 @@ struct alignas(64) GemmParams {
     uint32_t* status;
     uint64_t wait_limit_ns;     // bound of every barrier wait in the kernel
     uint32_t stall_extra_tx;    // test hook: bytes added to what the first stage's barrier expects (0 in normal use)
+    int provisional_skew;       // test hook: rows added to the expert offsets read before the wait (0 in normal use)
     int reduce_split;           // stream-K reduction: 1 = every boundary inside a split tile sums a share of it
     int64_t ldc;                // N
     int M;                      // dense rows (grouped: total rows)
@@ -210,8 +211,12 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* 
 }
 
 // Expert row offsets into shared memory (dense problems: one "expert" holding rows 0..M).
-__device__ __forceinline__ void load_row_starts(const GemmParams& p, int* row_start) {
-    for (int e = threadIdx.x; e <= p.E; e += blockDim.x) row_start[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.M);
+// (Offsets are clamped to 0..M and read past L1: the GEMM kernel reads them once before and once after it has
+// waited for its predecessor in the stream, see there.)
+__device__ __forceinline__ int clamp_row(int r, int M) { return r < 0 ? 0 : (r > M ? M : r); }
+__device__ __forceinline__ void load_row_starts(const GemmParams& p, int* row_start, int skew = 0) {
+    for (int e = threadIdx.x; e <= p.E; e += blockDim.x)
+        row_start[e] = p.offsets ? clamp_row(__ldcg(p.offsets + e) + skew, p.M) : (e == 0 ? 0 : p.M);
 }
 
 // prefix[e] = output tiles of the experts before e (n_tiles x m-tiles each); one warp, shuffle scan.
@@ -221,7 +226,10 @@ __device__ __forceinline__ void tile_prefix(const GemmParams& p, const int* row_
     for (int base = 0; base < p.E; base += 32) {
         const int e = base + lane;
         int v = 0;
-        if (e < p.E) v = ((row_start[e + 1] - row_start[e] + p.BM - 1) / p.BM) * p.n_tiles;
+        if (e < p.E) {
+            const int rows = row_start[e + 1] - row_start[e];
+            v = rows > 0 ? ((rows + p.BM - 1) / p.BM) * p.n_tiles : 0;
+        }
         int incl = v;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -421,66 +429,78 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
         }
         fence_proxy_async_smem();
     }
-    // Launched with programmatic stream serialisation: everything above (barriers, tensor memory, descriptor
-    // prefetch) may run while the kernel before this one in the stream is still finishing.  Nothing that kernel
-    // may have written (tokens, expert offsets, the partial-tile workspace, C) is touched before this wait, which
-    // returns once it has completed and its writes are visible.
-    // Grouped problems read the expert offsets, which that kernel may have produced, for the tables below; dense
-    // problems build their tables from the launch parameters alone and wait afterwards.
-    const bool tables_first = p.offsets == nullptr;
-    if (!tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Launched with programmatic stream serialisation: everything up to the wait below (barriers, tensor memory,
+    // descriptor prefetch, the schedule's tables, a prefetch of the first weights into L2) may run while the kernel
+    // before this one in the stream is still finishing.  Nothing that kernel may have written (tokens, the
+    // partial-tile workspace, C) is used before the wait, which returns once it has completed and its writes are
+    // visible.  Dense problems build their tables from the launch parameters alone.  Grouped problems read the
+    // expert offsets, which that kernel may still be writing: the tables built before the wait are provisional
+    // (offsets clamped to 0..M, so that whatever was read gives bounded arithmetic), the offsets are read again
+    // after the wait, and the tables are rebuilt if a single one differs.
     // generic-address path: the chunk table (see generic_chunk_dst), after the raw ring
     if (p.generic_b && warp >= 6 && warp < 10) {
         uint16_t* tab = reinterpret_cast<uint16_t*>(stages + size_t(p.num_stages) * stage_bytes + size_t(p.raw_slots) * kWBytes);
         for (int c = int(threadIdx.x) - 192; c < int(kWBytes / 16); c += 128)
             tab[c] = uint16_t(generic_chunk_dst<kBK, kBN>(c, p.br_log2, p.bc_log2));
     }
-    // tiles before each expert (dense: one "expert" holding all M rows)
-    load_row_starts(p, row_start);
-    __syncthreads();
-    if (warp == 2) tile_prefix(p, row_start, prefix);
+    int tiles_total = 0;
+    Sched sched;
+    auto build_tables = [&](int skew) {
+        // tiles before each expert (dense: one "expert" holding all M rows)
+        load_row_starts(p, row_start, skew);
+        __syncthreads();
+        if (warp == 2) tile_prefix(p, row_start, prefix);
+        __syncthreads();
+        tiles_total = prefix[p.E];
+        // Range starts of all CTAs, once, so that nothing on the critical path divides 64-bit numbers.
+        // (of the part of the schedule that is cut along K: the tiles left after the whole rounds)
+        const long long total_iters =
+            static_cast<long long>(tiles_total - Sched::whole_rounds_tiles(tiles_total, gridDim.x)) * p.k_iters;
+        const int grid_eff0 = Sched::effective_grid(total_iters, gridDim.x);
+        const bool use_tab = p.stream_k && grid_eff0 > 0 && grid_eff0 <= kRangeTabMax && total_iters < (1ll << 31);
+        if (use_tab) {
+            for (int c = threadIdx.x; c <= grid_eff0; c += blockDim.x)
+                range_tab[c] = static_cast<int>(Sched::split(total_iters, grid_eff0, c));
+        }
+        __syncthreads();
+        if (p.cluster_k > 1) sched.init_cluster(p.k_iters, tiles_total, int(cluster_id_x()), int(cluster_cta_rank()), p.cluster_k);
+        else sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
+    };
+    build_tables(p.provisional_skew);          // (test hook: wrong on purpose, so that the check below fails)
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
-    const int tiles_total = prefix[p.E];
-    // Range starts of all CTAs, once, so that nothing on the critical path divides 64-bit numbers.
-    // (of the part of the schedule that is cut along K: the tiles left after the whole rounds)
-    const long long total_iters =
-        static_cast<long long>(tiles_total - Sched::whole_rounds_tiles(tiles_total, gridDim.x)) * p.k_iters;
-    const int grid_eff0 = Sched::effective_grid(total_iters, gridDim.x);
-    const bool use_tab = p.stream_k && grid_eff0 > 0 && grid_eff0 <= kRangeTabMax && total_iters < (1ll << 31);
-    if (use_tab) {
-        for (int c = threadIdx.x; c <= grid_eff0; c += blockDim.x)
-            range_tab[c] = static_cast<int>(Sched::split(total_iters, grid_eff0, c));
-        __syncthreads();
-    }
-    Sched sched;
-    if (p.cluster_k > 1) sched.init_cluster(p.k_iters, tiles_total, int(cluster_id_x()), int(cluster_cta_rank()), p.cluster_k);
-    else sched.init(p.stream_k, p.k_iters, tiles_total, gridDim.x, blockIdx.x, use_tab ? range_tab : nullptr);
-    // Dense problems: while the kernel before this one in the stream is still finishing, ask for the first stages
-    // of this CTA's weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is the point of
-    // coherence, so this is safe whatever that kernel is still writing; it takes the cold start (page walks, first
-    // DRAM accesses) off this kernel's critical path.
+    // While the kernel before this one in the stream is still finishing, ask for the first stages of this CTA's
+    // weights to be brought into L2.  A prefetch delivers nothing to the SM and L2 is the point of coherence, so
+    // this is safe whatever that kernel is still writing (and whatever the provisional tables of a grouped problem
+    // point at: coordinates outside the tensor are skipped by the copy engine); it takes the cold start (page walks,
+    // first DRAM accesses) off this kernel's critical path.
     // (issued by an epilogue thread, which has nothing else to do yet, so that the producer is not held up)
-    if (threadIdx.x == 64 && tables_first && !p.generic_b && p.prefetch_stages > 0) {
+    if (threadIdx.x == 64 && !p.generic_b && p.prefetch_stages > 0) {
         Sched first = sched;
         Work w;
         if (first.next(w)) {
             const TileInfo t = decode_tile(p, prefix, row_start, w.tile, first.stream_k == 1 && w.tile >= first.dp_tiles);
+            const int kc_expert = t.expert * p.k_coord_per_expert;
             for (int s = 0, kit = w.kbeg; s < p.prefetch_stages && kit < w.kend; ++s, ++kit) {
                 const int kq = t.flip ? p.k_iters - 1 - kit : kit;
                 const int k0 = (kq * kBK) << p.k_shift;
                 for (int kb = 0; kb < p.kbx; ++kb)
                     for (int nb = 0; nb < p.nbx; ++nb) {
                         int c[5];
-                        weight_box_coords(p, k0 + kb * p.box_rows, t.n0 + nb * p.box_atoms * 64, 0, c);
+                        weight_box_coords(p, k0 + kb * p.box_rows, t.n0 + nb * p.box_atoms * 64, kc_expert, c);
                         tma_prefetch_5d(&p.tmap_b, c[0], c[1], c[2], c[3], c[4]);
                     }
             }
         }
     }
-    if (tables_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.offsets != nullptr) {
+        int differs = 0;
+        for (int e = threadIdx.x; e <= p.E; e += blockDim.x) differs |= row_start[e] != clamp_row(__ldcg(p.offsets + e), p.M);
+        if (__syncthreads_or(differs)) build_tables(0);
+    }
     // Let the kernel that follows in the stream (the stream-K reduction, or the next product) be scheduled already:
     // it does its own set-up and then blocks until this whole grid has finished.
     if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

@@ -195,6 +195,42 @@ def test_grouped_row_cap_keeps_the_products_exact(cap):
     assert torch.equal(g.check().cpu(), want)
 
 
+def test_grouped_tables_built_ahead_of_the_wait_are_checked_and_rebuilt():
+    # A grouped kernel reads the expert offsets and builds its tile tables while its predecessor in the stream may still
+    # be running, then reads the offsets again after waiting for it and rebuilds the tables if one differs.
+    # (a) test hook: the provisional tables come from offsets 7 rows off; (b) the offsets really are written by the
+    # kernel just before the product in the stream, over a stale routing.  Both must give the exact product.
+    from gpu_util import DEV, guarded_out, tile_major_on_device, tl
+    E, N, K = 24, 1024, 512
+    offsets, counts, _ = inputs.zipf_topk_routing(96, E, 4, 1.1, seed=3)
+    stale, _, _ = inputs.zipf_topk_routing(96, E, 4, 0.3, seed=9)
+    rows = int(offsets[-1])
+    assert int(stale[-1]) == rows and not np.array_equal(stale, offsets)
+    A = inputs.bf16_integers((rows, K), -8, 8, seed=21)
+    B = inputs.bf16_integers((E * K, N), -8, 8, seed=22)
+    Bt = tile_major_on_device(B, E * K, N, 16, 128)
+    want = torch.empty((rows, N), dtype=torch.float32)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        want[r0:r1] = (A[r0:r1].double() @ B[e * K:(e + 1) * K].double()).float()
+    Ad, d_new = A.to(DEV), torch.from_numpy(offsets).to(DEV)
+    d_off = d_new.clone()
+    tl.set_option(tl.OPT_STALL_ONCE, 4)
+    g = guarded_out((rows, N), torch.float32)
+    tl.gemm_grouped(Ad, Bt, g.t, d_off, E, rows, N, K, 4096, 16, 128)
+    assert tl.get_option(tl.OPT_STALL_ONCE) == 0
+    tl.device_status()
+    assert torch.equal(g.check().cpu(), want)
+    for _ in range(5):
+        d_off.copy_(torch.from_numpy(stale).to(DEV))
+        torch.cuda.synchronize()
+        g = guarded_out((rows, N), torch.float32)
+        d_off.copy_(d_new)                                   # the product's stream predecessor writes the offsets
+        tl.gemm_grouped(Ad, Bt, g.t, d_off, E, rows, N, K, 4096, 16, 128)
+        tl.device_status()
+        assert torch.equal(g.check().cpu(), want)
+
+
 def test_relayout_without_the_copy_engine_matches_the_oracle():
     from gpu_util import Guarded, dev_bytes, tl
     for rows, cols, s, br, bc in ((512, 512, 2, 16, 128), (1056, 2176, 2, 32, 64), (256, 1024, 1, 64, 64)):
