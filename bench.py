@@ -841,7 +841,8 @@ PROFILE_CASES = {
     "fp8_decode_qkv_m8": ("fp8", 8, 8192, 10240),           # E4M3, 64 x 64 memory tiles
     "fp8_prefill_o": ("fp8", 4096, 8192, 8192),             # E4M3, 64 x 64 memory tiles, CTA-pair kernel
     "hw_box_load_o": ("hw", 0, 8192, 8192),                 # every 64 x 256 box of the weight through a 2-D view
-    "generic_16x8_m16": ("generic", 16, 8192, 8192),        # 16 x 8 memory tiles (16-byte rows): generic-address path
+    "generic_16x8_m16": ("generic", 16, 8192, 8192),        # 16 x 8 memory tiles, permuting generic-address path (switch)
+    "as_stored_16x8_m16": ("as_stored", 16, 8192, 8192),    # 16 x 8 memory tiles (16-byte rows) read as they are
     "relayout_layer": ("relayout_batch", 0, 0, 0),          # the four Llama weights in one launch (3.4 GB resident)
 }
 
@@ -869,7 +870,9 @@ def run_case(args):
         dsts = [torch.empty_like(t) for t in srcs]
         for _ in range(args.steps):
             tl.relayout_batch(srcs, dsts, [(k, n) for _, k, n in inputs.LLAMA70B_PROJ], 2, G, BR, BC, tl.TO_TILE_MAJOR)
-    elif kind == "generic":
+    elif kind in ("generic", "as_stored"):
+        if kind == "generic":
+            tl.set_option(tl.OPT_GENERIC_RAW, 0)            # the permuting path, which these tiles no longer take by default
         W = inputs.bf16_normal((K, N), 0.02, seed=100, device=dev)
         Wt = torch.empty_like(W)
         tl.relayout(W, Wt, K, N, 2, 256, 16, 8, tl.TO_TILE_MAJOR)
@@ -962,8 +965,11 @@ def run_sweep(args):
                 tl.relayout(W[c], Wt[c], K, N, 2, g, br, bc, tl.TO_TILE_MAJOR)
             # the library's rule: 1-row tiles are row-major; tile rows of at least 32 bytes are TMA boxes (128-byte
             # swizzle from 64 columns, 64-/32-byte swizzle for 32/16 columns); shorter rows are hand-addressed
+            # (of those, tiles with 16-byte rows and single-column tiles of at least 8 rows are fetched as stored)
             path = ("row-major view" if br == 1 else "tma" if bc >= 64 else
-                    "tma, %d-byte swizzle" % (bc * 2) if bc in (16, 32) else "generic-address")
+                    "tma, %d-byte swizzle" % (bc * 2) if bc in (16, 32) else
+                    "tma, tiles as stored" if bc == 8 and br >= 8 else
+                    "tma, K-major panels" if bc == 1 and br >= 8 else "generic-address")
             for cta in ctas:
                 ra_t = tl.read_amp(128, N, K, cta, tl.LAYOUT_TILE_MAJOR, g, br, bc, 2)
                 ra_r = tl.read_amp(128, N, K, cta, tl.LAYOUT_ROW_MAJOR, g, 0, 0, 2)
@@ -977,6 +983,7 @@ def run_sweep(args):
                         row[f"M{M}_us"] = round(us, 1)
                         row[f"M{M}_GBps"] = round(gemm_bytes(M, N, K) / us / 1e3)
                         row[f"M{M}_vs_row_major_time"] = round(us / base[cta, M], 3)
+                    row["generic_path"] = tl.gemm_last_plan().generic_path
                 except tl.TileLensError as exc:
                     row["gemm"] = f"unsupported: {exc}"
                 print(json.dumps(row), flush=True)

@@ -107,6 +107,8 @@ typedef enum {
                                 0: always the stream-K cut */
     TL_OPT_FFN_ONE_LAUNCH,   /* 0 (default): tl_moe_ffn runs its two grouped products as two launches; 1: as two phases of one
                                 cooperative launch where it can (measured slower: 236 against 211 us on the Qwen-3 expert FFN) */
+    TL_OPT_GENERIC_RAW,      /* 1 (default): memory tiles with 16-byte rows are copied into shared memory as they are and read by
+                                the MMA through a no-swizzle descriptor, 0: they take the permuting generic-address path */
     TL_OPT_PAIR_TMA_STORE,   /* 1 (default): the CTA-pair kernel writes C through shared memory with tiled bulk stores, 0: with
                                 plain stores straight from the accumulator registers (same values either way) */
     TL_OPT_COUNT_
@@ -303,7 +305,8 @@ typedef struct tl_gemm_plan_info {
     int32_t grid;                  /* CTAs launched */
     int32_t stages;                /* pipeline depth */
     int32_t weights_on_n;          /* 1: weights on the N side of the MMA (token tiles of up to 128 rows) */
-    int32_t generic_path;          /* 1: weights loaded by the generic-address path of Section 4.4 */
+    int32_t generic_path;          /* 1: weights loaded by the generic-address path of Section 4.4 (permuted in shared
+                                      memory); 2: its special case for 16-byte tile rows (raw tiles are the operand) */
     int32_t cluster_k;             /* S > 1: one tile per cluster of S CTAs that split its K loop (sums through distributed
                                       shared memory, no workspace); else 1 */
     int64_t pair_tiles_512, pair_tiles_256;   /* pair kernel: tiles of 512 and of 256 token rows (x 256 columns) */

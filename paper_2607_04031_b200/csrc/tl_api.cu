@@ -42,6 +42,7 @@ struct Options {
         v[TL_OPT_REDUCE_SPLIT] = 1;
         v[TL_OPT_NO_SCRATCH_PLANS] = 1;
         v[TL_OPT_PAIR_TMA_STORE] = 1;
+        v[TL_OPT_GENERIC_RAW] = 1;
     }
 };
 

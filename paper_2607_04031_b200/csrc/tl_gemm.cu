@@ -339,6 +339,13 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (reinterpret_cast<uintptr_t>(d_C) % 16 != 0) return TL_ERR_ALIGNMENT;
     }
 
+    // Two kinds of memory tiles that TMA cannot box as 64-column atoms can still be fetched as they are:
+    //   bc == 8 (16-byte rows): the tiles are core matrices of the no-swizzle MN-major operand layout;
+    //   bc == 1 (a tile = br consecutive K values of one column): the buffer is [K/br][N][br], a K-major operand
+    //           in panels of br K values, swizzle rows of min(128, 2 br) bytes (no swizzle for 16-byte rows).
+    const bool raw_shape = generic && bc == 8 && br >= 8 && opt(TL_OPT_GENERIC_RAW) != 0;
+    const bool kcol_shape = generic && bc == 1 && br >= 8 && opt(TL_OPT_GENERIC_RAW) != 0;
+    bool raw_operand = false, kcol_operand = false;
     if (int rc = ensure_device_info()) return rc;
     // enough 256 x 256 tiles for every cluster of the CTA-pair kernel to get one
     const bool pair_sized = ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= dev().sm_count;
@@ -351,9 +358,24 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         if (bm_guess <= 0 || bn_guess <= 0) return TL_ERR_UNSUPPORTED;
         const int64_t mt_bound = d_offsets ? rows_total / bm_guess + E : ceil_div(rows_total, bm_guess);
         // (the plan counts K in 2-byte units: an 8-bit stage holds twice as many elements)
-        if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                               d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized))
-            return rc;
+        // Memory tiles with 16-byte rows (8 bf16 columns, at least 8 rows) need no permutation: the raw tiles are
+        // core matrices of the MMA's no-swizzle operand layout and the copy engine can fetch them as they are.
+        // Planned like any TMA-readable weight; if the CTA tile then does not hold whole memory tiles, the permuting
+        // path takes over.
+        if (raw_shape) {
+            const int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
+                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
+            raw_operand = rc == TL_OK && plan.BK % br == 0 && plan.BN % bc == 0;
+        }
+        if (kcol_shape) {
+            const int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
+                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
+            kcol_operand = rc == TL_OK;
+        }
+        if (!raw_operand && !kcol_operand)
+            if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
+                                   d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized))
+                return rc;
     }
     if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
     if (d_H_swiglu && !plan.weights_on_n) return TL_ERR_UNSUPPORTED;        // the gated epilogue pairs columns of one token row   // a K tail would read the next expert's rows
@@ -386,6 +408,19 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     p.fp8 = es == 1;
     p.k_shift = k_shift;
     uint32_t w_layout = 2;
+    uint64_t raw_chunk = 2048;                   // raw memory tiles as the operand: bytes per tensor-map row (see below)
+    const bool kcol16 = kcol_operand && br == 8;      // 16-byte tiles: one run of them is a row of K-major core matrices already
+    if (raw_operand || kcol16)
+        while ((uint64_t(plan.BN) * br * 2) % raw_chunk != 0 || (uint64_t(N) * br * 2) % raw_chunk != 0) raw_chunk >>= 1;
+    // The tile-major buffer as plain bytes: (chunk of 8-byte words, chunks along a row of the tile grid, rows of the tile
+    // grid); the box is the stage's cta_k/br runs of whole memory tiles, landed in memory order without swizzle.
+    auto encode_byte_runs = [&]() -> int {
+        const uint64_t run_full = uint64_t(plan.BN) * br * 2, grid_row = uint64_t(N) * br * 2, chunk = raw_chunk;
+        const uint64_t dims[5] = {chunk / 8, grid_row / chunk, uint64_t(K / br) * E, 1, 1};
+        const uint64_t str[5] = {8, chunk, grid_row, grid_row * uint64_t(K / br) * E, grid_row * uint64_t(K / br) * E};
+        const uint32_t box[5] = {uint32_t(chunk / 8), uint32_t(run_full / chunk), uint32_t(plan.BK / br), 1, 1};
+        return encode_tensor_map(&p.tmap_b, d_B, int(CU_TENSOR_MAP_DATA_TYPE_INT64), int(CU_TENSOR_MAP_SWIZZLE_NONE), 5, dims, str, box);
+    };
     // ---- weight operand B
     const int NA = plan.BN / 64;                                  // 128-byte atoms across the CTA tile
     int RB, AB, nb_box = 1, kb_box = 1;         // box: rows, atoms, memory tiles along N and K
@@ -426,6 +461,46 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.w_kmajor = 1;
         p.w_atom_log2 = ilog2(e);
         w_layout = w_row_bytes == 128 ? 2u : w_row_bytes == 64 ? 4u : 6u;
+    } else if (kcol_operand) {
+        // Memory tiles of br rows x 1 column: [K/br][N][br] seen as (e, N, br/e, E*K/br) with swizzle rows of
+        // r = min(128, 2 br) bytes = e elements; the box takes all swizzle rows of the stage's K range for the CTA
+        // tile's columns, so the bytes land as [K row][cta_n rows][r], the canonical K-major operand.
+        RB = plan.BK;
+        AB = NA;
+        w_row_bytes = br * 2 < kAtomBytes ? br * 2 : kAtomBytes;
+        const int e = w_row_bytes / 2;
+        const int swz = w_row_bytes == 128 ? int(CU_TENSOR_MAP_SWIZZLE_128B) : w_row_bytes == 64 ? int(CU_TENSOR_MAP_SWIZZLE_64B)
+                        : w_row_bytes == 32 ? int(CU_TENSOR_MAP_SWIZZLE_32B) : int(CU_TENSOR_MAP_SWIZZLE_NONE);
+        const int k_box = br < plan.BK ? br : plan.BK;
+        const uint64_t big = uint64_t(N) * br * 2 * uint64_t(K / br) * E;
+        if (kcol16) {
+            // (16-byte tiles: consecutive columns' tiles already form the 128-byte core matrices, so the stage's
+            // runs are fetched as plain bytes, see the next case)
+            if (int rc = encode_byte_runs()) return rc;
+        } else {
+            const uint64_t dims[5] = {uint64_t(e), uint64_t(N), uint64_t(br / e), uint64_t(K / br) * E, 1};
+            const uint64_t str[5] = {2, uint64_t(br) * 2, uint64_t(w_row_bytes), uint64_t(N) * br * 2, big};
+            const uint32_t box[5] = {uint32_t(e), uint32_t(plan.BN), uint32_t(k_box / e), uint32_t(plan.BK / k_box), 1};
+            if (int rc = encode_tensor_map(&p.tmap_b, d_B, dtype, swz, 5, dims, str, box)) return rc;
+        }
+        p.k_coord_per_expert = int(K / br);
+        p.br_log2 = ilog2(br);
+        p.bc_log2 = 0;
+        p.w_kmajor = 1;
+        p.w_atom_log2 = ilog2(e);
+        w_layout = w_row_bytes == 128 ? 2u : w_row_bytes == 64 ? 4u : w_row_bytes == 32 ? 6u : 0u;
+    } else if (raw_operand) {
+        // Memory tiles of br rows x 16 bytes.  A stage is cta_k/br runs of cta_n/8 whole tiles, each run contiguous in
+        // the tile-major buffer, so the buffer is seen as plain bytes: (chunk of 8-byte words, chunks along a row of
+        // the tile grid, rows of the tile grid) with chunk = the largest power of two up to 2 KB that divides both
+        // one run and a whole row of the tile grid; the box takes the stage's runs and
+        // lands them in memory order, no swizzle.  Columns beyond N and rows beyond K arrive as zeros.
+        RB = plan.BK;
+        AB = NA;
+        if (int rc = encode_byte_runs()) return rc;
+        p.k_coord_per_expert = int(K / br);
+        p.br_log2 = ilog2(br);
+        p.bc_log2 = ilog2(bc);
     } else if (generic) {
         // No tensor map: warps 6..9 of the kernel compute Eq. 1-2 addresses themselves and build the
         // canonical [atom][cta_k rows][64] image in shared memory.
@@ -508,7 +583,17 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         };
         const int all = -1;
         for (int i = 0; i < 4; ++i) set(i, 0, 0, 0, 0, 0);
-        if (generic) {
+        if (kcol16) {                               // (.., chunk along the tile-grid row, tile-grid row, -, -)
+            set(0, 0, 0, ilog2(int64_t(raw_chunk / 16)), all, 0);
+            set(1, 3, all, 0, 0, 1);
+        } else if (kcol_operand) {                  // (.., weight column, swizzle row in tile, tile along K, -)
+            set(0, 0, 0, 0, all, 0);
+            set(1, p.w_atom_log2, (br >> p.w_atom_log2) - 1, 0, 0, 0);
+            set(2, ilog2(br), all, 0, 0, 1);
+        } else if (raw_operand) {                   // (.., chunk along the tile-grid row, tile-grid row, -, -)
+            set(0, 0, 0, ilog2(int64_t(raw_chunk / (uint64_t(br) * 2))), all, 0);
+            set(1, ilog2(br), all, 0, 0, 1);
+        } else if (generic) {
         } else if (kmajor && row_major) {           // (row of K-elements, N row, -, swizzle row along K, -)
             set(0, 0, 0, 0, all, 1);
             set(2, p.w_atom_log2, all, 0, 0, 0);
@@ -533,8 +618,9 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         }
     }
     p.row_major = row_major;
-    p.kbx = generic ? 0 : plan.BK / (RB * kb_box);
-    p.nbx = generic ? 0 : NA / (AB * nb_box);
+    const bool permuted = generic && !raw_operand && !kcol_operand;     // the generic-address path proper
+    p.kbx = permuted ? 0 : plan.BK / (RB * kb_box);
+    p.nbx = permuted ? 0 : NA / (AB * nb_box);
     p.box_rows = RB * kb_box;                                     // K rows and atoms one instruction covers
     p.box_atoms = AB * nb_box;
     p.box_bytes = uint32_t(RB) * AB * kAtomBytes * nb_box * kb_box;
@@ -562,19 +648,33 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
         w_layout = bc == 32 ? 4u : 6u;
     }
-    if (kmajor) {
+    if (kmajor || kcol_operand) {
         // K-major image: [swizzle row along K][cta_n rows][r bytes]; 8-row groups 8r bytes apart, a K step of one
         // instruction (32 bytes) is 32 bytes further inside the swizzle row, the next swizzle row cta_n rows further.
+        // (16-byte rows, no swizzle: an instruction's K step is two rows, the second cta_n rows further.)
         const uint32_t r = uint32_t(w_row_bytes), steps_per_row = r / 32u;
-        p.lbo = 16;
+        p.lbo = r == 16 ? uint32_t(plan.BN) * 16u : 16u;
         p.sbo = 8u * r;
         p.ugroup_off = 128u * r;
         for (int j = 0; j < plan.BK / 16; ++j)
-            p.kstep_off[j] = (uint32_t(j) / steps_per_row) * uint32_t(plan.BN) * r + (uint32_t(j) % steps_per_row) * 32u;
+            p.kstep_off[j] = r == 16 ? uint32_t(j) * 2u * uint32_t(plan.BN) * 16u
+                                     : (uint32_t(j) / steps_per_row) * uint32_t(plan.BN) * r + (uint32_t(j) % steps_per_row) * 32u;
         p.box_rows = plan.BK << k_shift;
         p.box_atoms = NA;
         p.kbx = p.nbx = 1;
         p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
+    }
+    if (raw_operand) {
+        // The stage holds cta_k/br runs of cta_n/8 memory tiles in memory order.  A memory tile is br/8 core matrices
+        // (8 K rows x 16 bytes) one after the other: the next one along K is 128 bytes further (in the next run when
+        // a tile has only 8 rows), the next one along N one memory tile further; no swizzle.
+        const uint32_t run_full = uint32_t(plan.BN) * br * 2;
+        p.lbo = br >= 16 ? 128u : run_full;
+        p.sbo = uint32_t(G);
+        p.ugroup_off = 16u * uint32_t(G);
+        for (int j = 0; j < plan.BK / 16; ++j)
+            p.kstep_off[j] = uint32_t((j * 16) / br) * run_full + uint32_t((j * 16) % br) * 16u;
+        w_layout = 0u;
     }
     p.w_desc_hi = smem_desc_hi(p.lbo, p.sbo, w_layout);
     p.C = d_C;
@@ -612,13 +712,13 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     memset(&info, 0, sizeof info);
     info.cta_m = plan.BM; info.cta_n = plan.BN; info.cta_k = plan.BK << k_shift;
     info.stream_k = plan.stream_k; info.grid = plan.grid; info.stages = plan.num_stages;
-    info.weights_on_n = plan.weights_on_n; info.generic_path = generic ? 1 : 0; info.cluster_k = plan.cluster_k;
+    info.weights_on_n = plan.weights_on_n; info.generic_path = generic ? (permuted ? 1 : 2) : 0; info.cluster_k = plan.cluster_k;
     info.workspace_bytes = plan.ws_bytes;
     // Large dense problems on TMA-readable weights: CTA pairs (cta_group::2 MMAs), see tl_gemm_pair.cuh.
     const bool no_pair = opt(TL_OPT_PAIR_KERNEL) == 0;     // measurement switch
     // Worth it once every cluster of the machine has at least one 256 x 256 tile; smaller problems keep the
     // single-CTA kernel and its stream-K split.
-    if (!no_pair && !d_offsets && !generic && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
+    if (!no_pair && !d_offsets && !permuted && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
         p.kbx == 1 && p.nbx == 1 && pair_sized) {
         int& max_clusters = dev().pair_max_clusters;
         if (max_clusters < 0) {
@@ -677,7 +777,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         fprintf(stderr, "[tilelens] gemm kernel: cta %d x %d x %d, weights on %s, %s, grid %d, %d stages, %zu B workspace%s\n",
                 info.cta_m, info.cta_n, info.cta_k, plan.weights_on_n ? "N" : "M",
                 plan.stream_k ? "stream-K" : plan.cluster_k > 1 ? "cluster split-K" : "whole tiles",
-                plan.grid, plan.num_stages, plan.ws_bytes, generic ? ", generic-address weights" : "");
+                plan.grid, plan.num_stages, plan.ws_bytes,
+                raw_operand || kcol_operand ? ", raw memory tiles as the operand" : generic ? ", generic-address weights" : "");
     if (plan_only) { *plan_only = info; return TL_OK; }
     last_plan() = info;
     // Split-K scratch (none for whole-tile schedules).  A fixed scratch keeps the previous launch's contents; nothing
@@ -713,7 +814,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(plan.grid);
-        cfg.blockDim = dim3(generic ? kGenericThreads : kGemmThreads);
+        cfg.blockDim = dim3(permuted ? kGenericThreads : kGemmThreads);
         cfg.dynamicSmemBytes = plan.smem_bytes;
         cfg.stream = stream;
         cudaLaunchAttribute attr[2];

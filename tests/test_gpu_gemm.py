@@ -36,6 +36,7 @@ def test_config1_tiny_tile_major_and_row_major():
 # TMA-boxable tiles, row-major, one-row tiles (= row-major), and tiles only the generic-address path can read
 BLOCKS = [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0), (1, 1024), (1, 128),
           (8, 2), (16, 1), (8, 16), (16, 8), (32, 4), (16, 32), (32, 16), (2, 64), (4, 128), (64, 8),
+          (8, 8), (8, 1), (64, 1), (128, 1), (4, 8),
           (2, 1024), (4, 512), (2, 256), (64, 32), (128, 16), (4, 32), (256, 16)]
 
 
@@ -51,7 +52,10 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     Bd = tile_major_on_device(B, K, N, br, bc) if br else B.to(DEV)
     hand_addressed = br > 1 and bc < 16          # rows shorter than 32 bytes; everything else is TMA-boxable
     cta_n, cta_k = (cta[1] or 128), (cta[2] or 64)
-    if hand_addressed and (bc > cta_n or br > cta_k or cta_n * cta_k >= 256 * 128):
+    # of those, single-column tiles of at least 8 rows are read as a K-major operand and tiles with 16-byte rows as
+    # they are (if the CTA tile holds whole memory tiles); the rest is permuted in shared memory
+    as_stored = hand_addressed and br >= 8 and (bc == 1 or (bc == 8 and br <= cta_k))
+    if hand_addressed and not as_stored and (bc > cta_n or br > cta_k or cta_n * cta_k >= 256 * 128):
         # documented limits of the generic-address path: the memory tile must fit inside the CTA tile, and two
         # operand stages plus two raw stage images must fit in shared memory (not with 64 KB of weights per stage)
         from gpu_util import tl
@@ -61,6 +65,13 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
         return
     C = run_gemm(A, Bd, M, N, K, br, bc, cta)
     assert torch.equal(C.cpu(), B.float()[ks])
+    if hand_addressed:
+        from gpu_util import tl
+        assert tl.gemm_last_plan().generic_path == (2 if as_stored else 1)
+        if as_stored and cta_n * cta_k < 256 * 128 and br <= cta_k:
+            with tl.option(tl.OPT_GENERIC_RAW, 0):            # the same tiles through the permuting path
+                assert torch.equal(run_gemm(A, Bd, M, N, K, br, bc, cta).cpu(), B.float()[ks])
+                assert tl.gemm_last_plan().generic_path == 1
 
 
 def test_short_tiles_wider_than_the_cta_tile_and_hand_addressed_tiles_taller_than_it():
@@ -76,6 +87,59 @@ def test_short_tiles_wider_than_the_cta_tile_and_hand_addressed_tiles_taller_tha
     with pytest.raises(tl.TileLensError) as e:
         run_gemm(A, Bd, M, N, K, 128, 8, (32, 128, 64))        # 128 rows do not fit 64
     assert e.value.status == 2
+
+
+AS_STORED = [(16, 8), (8, 8), (64, 8), (16, 1), (8, 1), (32, 1), (64, 1), (128, 1)]
+
+
+@pytest.mark.parametrize("br,bc", AS_STORED)
+def test_tiles_read_as_stored_ragged_edges_grouped_and_prefill(br, bc):
+    # Memory tiles with 16-byte rows (raw tiles = core matrices of the no-swizzle operand) and single-column tiles (a
+    # K-major operand in panels): ragged N and K against the oracle, a grouped product, a prefill-sized product on the
+    # CTA-pair kernel; integer data, so everything is exact; the permuting path must give the same bits.
+    from gpu_util import DEV, guarded_out, run_gemm, tile_major_on_device, tl
+    G = br * bc * 2
+    for M, N, K, cta in ((40, 1160, 1152, (0, 0, 0)), (130, 1096, 640, (128, 128, 128)), (300, 648, 384, (0, 0, 0)),
+                         (9, 2056, 2176, (64, 256, 64))):
+        if K % br:
+            K += br - K % br
+        A = inputs.bf16_integers((M, K), -8, 8, seed=M + br)
+        B = inputs.bf16_integers((K, N), -8, 8, seed=N + bc)
+        Bd = tile_major_on_device(B, K, N, br, bc)
+        want = (A.double() @ B.double()).float()
+        if cta[2] and br > cta[2] and bc == 8:
+            continue                                        # the memory tile must fit the CTA tile
+        C = run_gemm(A, Bd, M, N, K, br, bc, cta)
+        assert tl.gemm_last_plan().generic_path == (2 if (bc == 1 or br <= tl.gemm_last_plan().cta_k) else 1)
+        assert torch.equal(C.cpu(), want), (M, N, K, cta)
+        ref, _ = _oracle_full(A, Bd, TILE, br, bc, M, N, K)
+        assert np.array_equal(C.cpu().numpy().astype(np.float64), ref)
+    # grouped: 12 experts, ragged row counts
+    E, N, K = 12, 768, 512
+    offsets, _, _ = inputs.zipf_topk_routing(64, E, 4, 1.0, seed=br + bc)
+    rows = int(offsets[-1])
+    A = inputs.bf16_integers((rows, K), -8, 8, seed=31)
+    B = inputs.bf16_integers((E * K, N), -8, 8, seed=32)
+    Bd = tile_major_on_device(B, E * K, N, br, bc)
+    want = torch.empty((rows, N), dtype=torch.float32)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        want[r0:r1] = (A[r0:r1].double() @ B[e * K:(e + 1) * K].double()).float()
+    g = guarded_out((rows, N), torch.float32)
+    tl.gemm_grouped(A.to(DEV), Bd, g.t, torch.from_numpy(offsets).to(DEV), E, rows, N, K, G, br, bc)
+    tl.device_status()
+    assert tl.gemm_last_plan().generic_path == 2
+    assert torch.equal(g.check().cpu(), want)
+    # prefill-sized: the CTA-pair kernel reads the same operand image
+    M, N, K = 700, 9600, 256
+    A = inputs.bf16_integers((M, K), -8, 8, seed=41)
+    B = inputs.bf16_integers((K, N), -8, 8, seed=42)
+    Bd = tile_major_on_device(B, K, N, br, bc)
+    C = run_gemm(A, Bd, M, N, K, br, bc)
+    plan = tl.gemm_last_plan()
+    if bc == 1 or br <= 64:
+        assert plan.pair_kernel == 1 and plan.generic_path == 2
+    assert torch.equal(C.cpu(), (A.double() @ B.double()).float())
 
 
 SHAPES = [  # M, N, K
