@@ -843,6 +843,8 @@ PROFILE_CASES = {
     "hw_box_load_o": ("hw", 0, 8192, 8192),                 # every 64 x 256 box of the weight through a 2-D view
     "generic_16x8_m16": ("generic", 16, 8192, 8192),        # 16 x 8 memory tiles, permuting generic-address path (switch)
     "as_stored_16x8_m16": ("as_stored", 16, 8192, 8192),    # 16 x 8 memory tiles (16-byte rows) read as they are
+    "in_place_32x4_m16": ("in_place_32x4", 16, 8192, 8192), # 32 x 4 memory tiles (8-byte rows): fetched as stored, fixed up in place
+    "in_place_8x2_m16": ("in_place_8x2", 16, 8192, 8192),   # 8 x 2 memory tiles (4-byte rows)
     "relayout_layer": ("relayout_batch", 0, 0, 0),          # the four Llama weights in one launch (3.4 GB resident)
 }
 
@@ -870,16 +872,17 @@ def run_case(args):
         dsts = [torch.empty_like(t) for t in srcs]
         for _ in range(args.steps):
             tl.relayout_batch(srcs, dsts, [(k, n) for _, k, n in inputs.LLAMA70B_PROJ], 2, G, BR, BC, tl.TO_TILE_MAJOR)
-    elif kind in ("generic", "as_stored"):
+    elif kind in ("generic", "as_stored") or kind.startswith("in_place"):
         if kind == "generic":
             tl.set_option(tl.OPT_GENERIC_RAW, 0)            # the permuting path, which these tiles no longer take by default
+        br, bc = (16, 8) if not kind.startswith("in_place") else tuple(int(x) for x in kind.split("_")[2].split("x"))
         W = inputs.bf16_normal((K, N), 0.02, seed=100, device=dev)
         Wt = torch.empty_like(W)
-        tl.relayout(W, Wt, K, N, 2, 256, 16, 8, tl.TO_TILE_MAJOR)
+        tl.relayout(W, Wt, K, N, 2, br * bc * 2, br, bc, tl.TO_TILE_MAJOR)
         A = inputs.bf16_normal((M, K), 1.0, seed=200, device=dev)
         C = torch.empty((M, N), dtype=torch.float32, device=dev)
         for _ in range(args.steps):
-            tl.gemm(A, Wt, C, M, N, K, 256, 16, 8)
+            tl.gemm(A, Wt, C, M, N, K, br * bc * 2, br, bc)
     elif kind in ("kmajor", "hw"):
         w = inputs.bf16_normal((N, K), 0.02, seed=100, device=dev)
         wt = torch.empty_like(w)
@@ -951,10 +954,9 @@ def run_sweep(args):
     # rows per stage for the 64- and 128-column tiles (half as many barrier hand-offs per byte: 64 x 64 runs at 3.1
     # instead of 2.4 TB/s), 64 for the 256-token tile, whose token side already fills the stage
     ctas = ((64, 64, 128), (128, 128, 128), (256, 128, 64))
-    base = {}
-    for cta in ctas:
-        for M in (1, 16, 128):
-            base[cta, M] = timed(M, W, 0, 0, 0, cta)
+    for _ in range(200):                                     # clocks up before anything is timed
+        tl.gemm(A[128], W[0], C[128], 128, N, K, 0, 0, 0, ctas[1])
+    torch.cuda.synchronize()
     for g in (32, 256, 1024, 4096, 16384):
         for br in (1, 8, 16, 32):
             bc = g // (2 * br)
@@ -969,7 +971,10 @@ def run_sweep(args):
             path = ("row-major view" if br == 1 else "tma" if bc >= 64 else
                     "tma, %d-byte swizzle" % (bc * 2) if bc in (16, 32) else
                     "tma, tiles as stored" if bc == 8 and br >= 8 else
-                    "tma, K-major panels" if bc == 1 and br >= 8 else "generic-address")
+                    "tma, K-major panels" if bc == 1 and br >= 8 else
+                    "tma as stored + in-place transpose" if bc in (2, 4) and br >= 8 else "generic-address")
+            # the row-major times every row is compared with are taken next to it (same minute, same clocks)
+            base = {(cta, M): timed(M, W, 0, 0, 0, cta) for cta in ctas for M in (1, 16, 128)}
             for cta in ctas:
                 ra_t = tl.read_amp(128, N, K, cta, tl.LAYOUT_TILE_MAJOR, g, br, bc, 2)
                 ra_r = tl.read_amp(128, N, K, cta, tl.LAYOUT_ROW_MAJOR, g, 0, 0, 2)

@@ -107,8 +107,9 @@ typedef enum {
                                 0: always the stream-K cut */
     TL_OPT_FFN_ONE_LAUNCH,   /* 0 (default): tl_moe_ffn runs its two grouped products as two launches; 1: as two phases of one
                                 cooperative launch where it can (measured slower: 236 against 211 us on the Qwen-3 expert FFN) */
-    TL_OPT_GENERIC_RAW,      /* 1 (default): memory tiles with 16-byte rows are copied into shared memory as they are and read by
-                                the MMA through a no-swizzle descriptor, 0: they take the permuting generic-address path */
+    TL_OPT_GENERIC_RAW,      /* 1 (default): memory tiles of at least 8 rows whose rows are 16, 8, 4 or 2 bytes long are copied into
+                                shared memory as stored (and, for 8- and 4-byte rows, transposed there in place) and read by the
+                                MMA through a no-swizzle or K-major descriptor; 0: they take the permuting generic-address path */
     TL_OPT_PAIR_TMA_STORE,   /* 1 (default): the CTA-pair kernel writes C through shared memory with tiled bulk stores, 0: with
                                 plain stores straight from the accumulator registers (same values either way) */
     TL_OPT_COUNT_
@@ -174,12 +175,17 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
  *   columns could ask for less), else TL_ERR_UNSUPPORTED.
  *   Memory tiles whose rows are at least 32 bytes (16 columns) are read by
  *   TMA, whatever their height.  Narrower ones (block rows down to 2 bytes)
- *   are read by the generic-address path of Section 4.4 (plain loads with
- *   Eq. 1-2 arithmetic); there the memory tile must fit inside the CTA tile
- *   (block_rows | cta_k, block_cols | cta_n), G >= 16, and the CTA tile must
- *   leave room in shared memory for two raw images of a stage's weights
- *   beside two operand stages (cta_n * cta_k < 256 * 128), else
- *   TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
+ *   are the generic-address case of Section 4.4.  With at least 8 rows they
+ *   are still fetched by the copy engine as stored: 16-byte rows are read by
+ *   the MMA as they are, single-column tiles as panels of a K-major operand,
+ *   8- and 4-byte rows (up to 64 and 128 rows) after an in-place transpose in
+ *   shared memory; block_rows | cta_k except for single-column tiles.  Tiles
+ *   of fewer rows (and all of them when TL_OPT_GENERIC_RAW is 0) are permuted
+ *   in shared memory with Eq. 1-2 arithmetic; there the memory tile must fit
+ *   inside the CTA tile (block_rows | cta_k, block_cols | cta_n), G >= 16, and
+ *   the CTA tile must leave room in shared memory for two raw images of a
+ *   stage's weights beside two operand stages (cta_n * cta_k < 256 * 128),
+ *   else TL_ERR_UNSUPPORTED.  One-row tiles are row-major.
  * When the output tiles do not fill the SMs (decode, small or grouped
  * problems) the K loops are cut: inside thread-block clusters whose CTAs
  * add their partial tiles through distributed shared memory where such a
@@ -306,7 +312,8 @@ typedef struct tl_gemm_plan_info {
     int32_t stages;                /* pipeline depth */
     int32_t weights_on_n;          /* 1: weights on the N side of the MMA (token tiles of up to 128 rows) */
     int32_t generic_path;          /* 1: weights loaded by the generic-address path of Section 4.4 (permuted in shared
-                                      memory); 2: its special case for 16-byte tile rows (raw tiles are the operand) */
+                                      memory); 2: memory tiles fetched as stored and read by the MMA as they are (16-byte
+                                      rows, single-column tiles); 3: fetched as stored, 8- or 4-byte rows transposed in place */
     int32_t cluster_k;             /* S > 1: one tile per cluster of S CTAs that split its K loop (sums through distributed
                                       shared memory, no workspace); else 1 */
     int64_t pair_tiles_512, pair_tiles_256;   /* pair kernel: tiles of 512 and of 256 token rows (x 256 columns) */

@@ -345,7 +345,11 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     //           in panels of br K values, swizzle rows of min(128, 2 br) bytes (no swizzle for 16-byte rows).
     const bool raw_shape = generic && bc == 8 && br >= 8 && opt(TL_OPT_GENERIC_RAW) != 0;
     const bool kcol_shape = generic && bc == 1 && br >= 8 && opt(TL_OPT_GENERIC_RAW) != 0;
-    bool raw_operand = false, kcol_operand = false;
+    //   bc == 4 or 2 (8- or 4-byte rows), 8 <= br <= 64 or 128: fetched as stored as well, then 2 or 4 neighbouring tiles
+    //           are transposed in place into one br x 8 tile with 16-byte rows (four more warps, see the kernel).
+    const bool fix_shape = generic && ((bc == 4 && br >= 8 && br <= 64) || (bc == 2 && br >= 8 && br <= 128)) &&
+                           opt(TL_OPT_GENERIC_RAW) != 0;
+    bool raw_operand = false, kcol_operand = false, fix_operand = false;
     if (int rc = ensure_device_info()) return rc;
     // enough 256 x 256 tiles for every cluster of the CTA-pair kernel to get one
     const bool pair_sized = ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= dev().sm_count;
@@ -372,7 +376,12 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                                      d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
             kcol_operand = rc == TL_OK;
         }
-        if (!raw_operand && !kcol_operand)
+        if (fix_shape) {
+            const int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
+                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
+            fix_operand = rc == TL_OK && plan.BK % br == 0;
+        }
+        if (!raw_operand && !kcol_operand && !fix_operand)
             if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
                                    d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized))
                 return rc;
@@ -410,7 +419,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     uint32_t w_layout = 2;
     uint64_t raw_chunk = 2048;                   // raw memory tiles as the operand: bytes per tensor-map row (see below)
     const bool kcol16 = kcol_operand && br == 8;      // 16-byte tiles: one run of them is a row of K-major core matrices already
-    if (raw_operand || kcol16)
+    if (raw_operand || kcol16 || fix_operand)
         while ((uint64_t(plan.BN) * br * 2) % raw_chunk != 0 || (uint64_t(N) * br * 2) % raw_chunk != 0) raw_chunk >>= 1;
     // The tile-major buffer as plain bytes: (chunk of 8-byte words, chunks along a row of the tile grid, rows of the tile
     // grid); the box is the stage's cta_k/br runs of whole memory tiles, landed in memory order without swizzle.
@@ -489,7 +498,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.w_kmajor = 1;
         p.w_atom_log2 = ilog2(e);
         w_layout = w_row_bytes == 128 ? 2u : w_row_bytes == 64 ? 4u : w_row_bytes == 32 ? 6u : 0u;
-    } else if (raw_operand) {
+    } else if (raw_operand || fix_operand) {
+        // (8- and 4-byte rows: the same view; the stage is fixed up in shared memory into the image described here)
         // Memory tiles of br rows x 16 bytes.  A stage is cta_k/br runs of cta_n/8 whole tiles, each run contiguous in
         // the tile-major buffer, so the buffer is seen as plain bytes: (chunk of 8-byte words, chunks along a row of
         // the tile grid, rows of the tile grid) with chunk = the largest power of two up to 2 KB that divides both
@@ -501,6 +511,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.k_coord_per_expert = int(K / br);
         p.br_log2 = ilog2(br);
         p.bc_log2 = ilog2(bc);
+        p.generic_b = fix_operand ? 2 : 0;
     } else if (generic) {
         // No tensor map: warps 6..9 of the kernel compute Eq. 1-2 addresses themselves and build the
         // canonical [atom][cta_k rows][64] image in shared memory.
@@ -590,7 +601,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
             set(0, 0, 0, 0, all, 0);
             set(1, p.w_atom_log2, (br >> p.w_atom_log2) - 1, 0, 0, 0);
             set(2, ilog2(br), all, 0, 0, 1);
-        } else if (raw_operand) {                   // (.., chunk along the tile-grid row, tile-grid row, -, -)
+        } else if (raw_operand || fix_operand) {    // (.., chunk along the tile-grid row, tile-grid row, -, -)
             set(0, 0, 0, ilog2(int64_t(raw_chunk / (uint64_t(br) * 2))), all, 0);
             set(1, ilog2(br), all, 0, 0, 1);
         } else if (generic) {
@@ -618,7 +629,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         }
     }
     p.row_major = row_major;
-    const bool permuted = generic && !raw_operand && !kcol_operand;     // the generic-address path proper
+    const bool permuted = generic && !raw_operand && !kcol_operand && !fix_operand;     // the generic-address path proper
     p.kbx = permuted ? 0 : plan.BK / (RB * kb_box);
     p.nbx = permuted ? 0 : NA / (AB * nb_box);
     p.box_rows = RB * kb_box;                                     // K rows and atoms one instruction covers
@@ -664,14 +675,14 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         p.kbx = p.nbx = 1;
         p.box_bytes = uint32_t(plan.BK) * plan.BN * 2;
     }
-    if (raw_operand) {
+    if (raw_operand || fix_operand) {
         // The stage holds cta_k/br runs of cta_n/8 memory tiles in memory order.  A memory tile is br/8 core matrices
         // (8 K rows x 16 bytes) one after the other: the next one along K is 128 bytes further (in the next run when
         // a tile has only 8 rows), the next one along N one memory tile further; no swizzle.
         const uint32_t run_full = uint32_t(plan.BN) * br * 2;
         p.lbo = br >= 16 ? 128u : run_full;
-        p.sbo = uint32_t(G);
-        p.ugroup_off = 16u * uint32_t(G);
+        p.sbo = 16u * uint32_t(br);                 // one br x 8 tile
+        p.ugroup_off = 16u * p.sbo;
         for (int j = 0; j < plan.BK / 16; ++j)
             p.kstep_off[j] = uint32_t((j * 16) / br) * run_full + uint32_t((j * 16) % br) * 16u;
         w_layout = 0u;
@@ -712,13 +723,13 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     memset(&info, 0, sizeof info);
     info.cta_m = plan.BM; info.cta_n = plan.BN; info.cta_k = plan.BK << k_shift;
     info.stream_k = plan.stream_k; info.grid = plan.grid; info.stages = plan.num_stages;
-    info.weights_on_n = plan.weights_on_n; info.generic_path = generic ? (permuted ? 1 : 2) : 0; info.cluster_k = plan.cluster_k;
+    info.weights_on_n = plan.weights_on_n; info.generic_path = generic ? (permuted ? 1 : fix_operand ? 3 : 2) : 0; info.cluster_k = plan.cluster_k;
     info.workspace_bytes = plan.ws_bytes;
     // Large dense problems on TMA-readable weights: CTA pairs (cta_group::2 MMAs), see tl_gemm_pair.cuh.
     const bool no_pair = opt(TL_OPT_PAIR_KERNEL) == 0;     // measurement switch
     // Worth it once every cluster of the machine has at least one 256 x 256 tile; smaller problems keep the
     // single-CTA kernel and its stream-K split.
-    if (!no_pair && !d_offsets && !permuted && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
+    if (!no_pair && !d_offsets && !permuted && !fix_operand && !d_H_swiglu && plan.BM == 256 && plan.BN == 128 && plan.BK == 64 &&
         p.kbx == 1 && p.nbx == 1 && pair_sized) {
         int& max_clusters = dev().pair_max_clusters;
         if (max_clusters < 0) {
@@ -778,7 +789,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                 info.cta_m, info.cta_n, info.cta_k, plan.weights_on_n ? "N" : "M",
                 plan.stream_k ? "stream-K" : plan.cluster_k > 1 ? "cluster split-K" : "whole tiles",
                 plan.grid, plan.num_stages, plan.ws_bytes,
-                raw_operand || kcol_operand ? ", raw memory tiles as the operand" : generic ? ", generic-address weights" : "");
+                raw_operand || kcol_operand ? ", raw memory tiles as the operand" : fix_operand ? ", memory tiles fixed up in place"
+                                                                                    : generic ? ", generic-address weights" : "");
     if (plan_only) { *plan_only = info; return TL_OK; }
     last_plan() = info;
     // Split-K scratch (none for whole-tile schedules).  A fixed scratch keeps the previous launch's contents; nothing
@@ -814,7 +826,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(plan.grid);
-        cfg.blockDim = dim3(permuted ? kGenericThreads : kGemmThreads);
+        cfg.blockDim = dim3(permuted || fix_operand ? kGenericThreads : kGemmThreads);
         cfg.dynamicSmemBytes = plan.smem_bytes;
         cfg.stream = stream;
         cudaLaunchAttribute attr[2];

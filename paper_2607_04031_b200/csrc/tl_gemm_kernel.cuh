@@ -75,6 +75,8 @@ struct alignas(64) GemmParams {
     uint32_t kstep_off[8];      // byte offset of each 16-row K step inside a stage
     // generic-address path (Section 4.4: memory tiles that TMA cannot box)
     int generic_b;              // 1: warps 6..9 build the weight operand with Eq. 1-2 address arithmetic
+                                // 2: memory tiles with 8- or 4-byte rows: the copy engine lands the stage's tiles as stored,
+                                //    warps 6..9 transpose 8- or 4-byte pieces in place (see fixup_stage_in_place)
     int raw_slots;              // generic path: ring of raw stage images (memory order) behind the pipeline stages
     uint32_t smem_limit;        // dynamic shared memory of the launch, bytes (the bulk copies check their destination against it)
     int64_t b_bytes;            // size of the weight buffer, bytes (... and their source against this)
@@ -357,6 +359,116 @@ __device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, in
         c[i + 1] = ((k >> p.ck_shift[i]) & p.ck_mask[i]) + ((n >> p.cn_shift[i]) & p.cn_mask[i]) + p.c_expert[i] * kc_expert;
 }
 
+// Memory tiles of br rows x 4 columns (8-byte rows) or br x 2 columns (4-byte rows), as the copy engine landed them:
+// the stage is an array of groups of 2 (or 4) tiles next to each other along N, 16 br bytes each, and a group covers br
+// rows x 8 columns.  A 16-byte chunk of a tile holds 2 (or 4) rows of its 4 (or 2) columns; the chunks at the same
+// place in the group's tiles hold the same rows.  One thread takes those 2 (or 4) chunks, and writes the 2 (or 4)
+// rows they contain, now 8 columns = 16 bytes wide, at row * 16 inside the same group: afterwards the group is a
+// br x 8 memory tile with 16-byte rows, i.e. br/8 core matrices of the no-swizzle MN-major operand, which the MMA
+// reads as it is.  In place: the threads of a group sit in one warp and all read before any of them writes.
+// 128 threads (tid 0..127) share the stage: kBK * kBN / 16 work items of 32 bytes (8-byte rows) or kBK * kBN / 32 of 64
+// bytes (4-byte rows), both multiples of 128; every item lies inside the stage's kBK * kBN * 2 bytes of weights.
+template <int kBK, int kBN>
+__device__ __forceinline__ void fixup_stage_in_place(uint8_t* sw, int br_log2, int bc_log2, int tid) {
+    const uint32_t group_bytes = 16u << br_log2;
+    // (kBatch work items have their loads in flight together: all reads, then all writes)
+    if (bc_log2 == 2) {
+        constexpr int kItems = kBK * kBN / 16;
+        constexpr int kBatch = kItems >= 512 ? 4 : kItems / 128;
+        static_assert(kItems % (128 * kBatch) == 0, "whole batches");
+        const int tpg_log2 = br_log2 - 1;                          // threads per group: one per pair of rows
+        const uint32_t tile_bytes = 8u << br_log2;
+        for (int item0 = tid; item0 < kItems; item0 += 128 * kBatch) {
+            uint4 a[kBatch], b[kBatch];
+            uint8_t* dst[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int item = item0 + j * 128;
+                const int g = item >> tpg_log2, q = item & ((1 << tpg_log2) - 1);
+                uint8_t* base = sw + size_t(g) * group_bytes;
+                a[j] = *reinterpret_cast<const uint4*>(base + q * 16);                // rows 2q, 2q+1 x columns 0..3
+                b[j] = *reinterpret_cast<const uint4*>(base + tile_bytes + q * 16);   //                x columns 4..7
+                dst[j] = base + q * 32;
+            }
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                *reinterpret_cast<uint4*>(dst[j]) = make_uint4(a[j].x, a[j].y, b[j].x, b[j].y);
+                *reinterpret_cast<uint4*>(dst[j] + 16) = make_uint4(a[j].z, a[j].w, b[j].z, b[j].w);
+            }
+        }
+    } else if (br_log2 <= 4) {
+        // 4-byte rows, tiles of 8 or 16 rows: a group is at most 256 bytes, so a warp's 32 lanes read whole groups as
+        // consecutive 16-byte chunks (lane = chunk: no bank conflicts, which the form below would have here), then the
+        // four lanes that hold the same four rows of the group's four tiles transpose their 4 x 4 words with two
+        // exchanges, and every lane writes one finished row.
+        constexpr int kChunks = kBK * kBN / 8;
+        constexpr int kBatch = 4;
+        static_assert(kChunks % (128 * kBatch) == 0, "whole batches");
+        const int d = 1 << (br_log2 - 2);                          // lanes between neighbouring tiles of a group
+        const int lane = tid & 31;
+        const int pt = (lane >> (br_log2 - 2)) & 3, q = lane & (d - 1);
+        const uint32_t m_hi = (pt & 2) ? 0xffffffffu : 0u, m_odd = (pt & 1) ? 0xffffffffu : 0u;
+        auto pick = [](uint32_t m, uint32_t a, uint32_t b) { return b ^ ((a ^ b) & m); };
+        for (int c0 = tid; c0 < kChunks; c0 += 128 * kBatch) {
+            uint4 v[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j)                        // rows 4q..4q+3 x columns 2 pt, 2 pt + 1
+                v[j] = *reinterpret_cast<const uint4*>(sw + size_t(c0 + j * 128) * 16);
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                uint8_t* group = sw + ((size_t(c0 + j * 128) * 16) & ~size_t(group_bytes - 1));
+                // (pick(m, a, b) = m ? a : b with m all ones or zero: no branches in this loop)
+                const uint32_t r0 = __shfl_xor_sync(0xffffffffu, pick(m_hi, v[j].x, v[j].z), 2 * d);
+                const uint32_t r1 = __shfl_xor_sync(0xffffffffu, pick(m_hi, v[j].y, v[j].w), 2 * d);
+                const uint32_t k0 = pick(m_hi, v[j].z, v[j].x), k1 = pick(m_hi, v[j].w, v[j].y);
+                // rows (2 (pt >> 1), + 1) of tile pt in (k0, k1), of tile pt ^ 2 in (r0, r1); keep row pt, pass on row pt ^ 1
+                const uint32_t g_own = __shfl_xor_sync(0xffffffffu, pick(m_odd, k0, k1), d);
+                const uint32_t g_oth = __shfl_xor_sync(0xffffffffu, pick(m_odd, r0, r1), d);
+                const uint32_t keep_own = pick(m_odd, k1, k0), keep_oth = pick(m_odd, r1, r0);
+                // row 4q + pt of tiles pt, pt ^ 1, pt ^ 2, pt ^ 3 in w0..w3; column pair t of the row comes from tile t
+                const uint32_t w0 = keep_own, w1 = g_own, w2 = keep_oth, w3 = g_oth;
+                const uint32_t x0 = pick(m_odd, w1, w0), x1 = pick(m_odd, w0, w1), x2 = pick(m_odd, w3, w2), x3 = pick(m_odd, w2, w3);
+                uint4 o;
+                o.x = pick(m_hi, x2, x0);
+                o.y = pick(m_hi, x3, x1);
+                o.z = pick(m_hi, x0, x2);
+                o.w = pick(m_hi, x1, x3);
+                *reinterpret_cast<uint4*>(group + (4 * q + pt) * 16) = o;
+            }
+        }
+    } else {
+        constexpr int kItems = kBK * kBN / 32;
+        const int tpg_log2 = br_log2 - 2;                          // one thread per four rows
+        const uint32_t tile_bytes = 4u << br_log2;
+        constexpr int kB2 = kItems >= 256 ? 2 : 1;
+        static_assert(kItems % (128 * kB2) == 0, "whole batches");
+        for (int item0 = tid; item0 < kItems; item0 += 128 * kB2) {
+            uint4 c[kB2][4];
+            uint8_t* dst[kB2];
+#pragma unroll
+            for (int j = 0; j < kB2; ++j) {
+                const int item = item0 + j * 128;
+                const int g = item >> tpg_log2, q = item & ((1 << tpg_log2) - 1);
+                uint8_t* base = sw + size_t(g) * group_bytes;
+#pragma unroll
+                for (int t4 = 0; t4 < 4; ++t4)                       // rows 4q..4q+3 x columns 2 t4, 2 t4 + 1
+                    c[j][t4] = *reinterpret_cast<const uint4*>(base + t4 * tile_bytes + q * 16);
+                dst[j] = base + q * 64;
+            }
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < kB2; ++j) {
+                *reinterpret_cast<uint4*>(dst[j]) = make_uint4(c[j][0].x, c[j][1].x, c[j][2].x, c[j][3].x);
+                *reinterpret_cast<uint4*>(dst[j] + 16) = make_uint4(c[j][0].y, c[j][1].y, c[j][2].y, c[j][3].y);
+                *reinterpret_cast<uint4*>(dst[j] + 32) = make_uint4(c[j][0].z, c[j][1].z, c[j][2].z, c[j][3].z);
+                *reinterpret_cast<uint4*>(dst[j] + 48) = make_uint4(c[j][0].w, c[j][1].w, c[j][2].w, c[j][3].w);
+            }
+        }
+    }
+}
+
 // kBK: weight rows per stage (64 or 128).  kBN: weight columns per CTA tile (64, 128 or 256).
 // kWN selects which side of the MMA the weights are on.  The tensor pipe takes N/2 clocks per MMA whatever M is,
 // and the thread that issues the MMAs runs alone in its warp (every scalar instruction between two MMAs costs it
@@ -403,13 +515,19 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
 
     // ---------------------------------------------------------------- set-up
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], p.generic_b ? 5 : 1); mbar_init(&empty_bar[s], 1); }
+        // (generic_b == 1: the producer and the four permuting warps arrive on a stage's "full" barrier; generic_b == 2:
+        // the copies land on raw_full_bar[stage] and the four warps that fix the stage up arrive on "full")
+        for (int s = 0; s < p.num_stages; ++s) {
+            mbar_init(&full_bar[s], p.generic_b == 1 ? 5 : p.generic_b == 2 ? 4 : 1);
+            mbar_init(&empty_bar[s], 1);
+            if (p.generic_b == 2) mbar_init(&raw_full_bar[s], 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full_bar[b], 1); mbar_init(&acc_empty_bar[b], 4); }
-        if (p.generic_b)
+        if (p.generic_b == 1)
             for (int r = 0; r < p.raw_slots; ++r) { mbar_init(&raw_full_bar[r], 1); mbar_init(&raw_empty_bar[r], 4); }
         abort_flag = 0;
         fence_mbar_init();
-        if (!p.generic_b) tma_prefetch_desc(&p.tmap_b);
+        if (p.generic_b != 1) tma_prefetch_desc(&p.tmap_b);
         for (int i = 0; i < kNumBoxChoices; ++i) tma_prefetch_desc(&p.tmap_a[i]);
     }
     if (warp == 1 && alloc_tmem) {
@@ -438,7 +556,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
     // (offsets clamped to 0..M, so that whatever was read gives bounded arithmetic), the offsets are read again
     // after the wait, and the tables are rebuilt if a single one differs.
     // generic-address path: the chunk table (see generic_chunk_dst), after the raw ring
-    if (p.generic_b && warp >= 6 && warp < 10) {
+    if (p.generic_b == 1 && warp >= 6 && warp < 10) {
         uint16_t* tab = reinterpret_cast<uint16_t*>(stages + size_t(p.num_stages) * stage_bytes + size_t(p.raw_slots) * kWBytes);
         for (int c = int(threadIdx.x) - 192; c < int(kWBytes / 16); c += 128)
             tab[c] = uint16_t(generic_chunk_dst<kBK, kBN>(c, p.br_log2, p.bc_log2));
@@ -477,7 +595,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
     // point at: coordinates outside the tensor are skipped by the copy engine); it takes the cold start (page walks,
     // first DRAM accesses) off this kernel's critical path.
     // (issued by an epilogue thread, which has nothing else to do yet, so that the producer is not held up)
-    if (threadIdx.x == 64 && !p.generic_b && p.prefetch_stages > 0) {
+    if (threadIdx.x == 64 && p.generic_b != 1 && p.prefetch_stages > 0) {
         Sched first = sched;
         Work w;
         if (first.next(w)) {
@@ -515,6 +633,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
             bool ok = true;
             // the K part of the coordinate maps, in registers for the whole loop
             const bool one_box = p.kbx == 1 && p.nbx == 1;
+            uint64_t* land_bar = p.generic_b == 2 ? raw_full_bar : full_bar;      // where a stage's copies are counted
             int ks[4], km[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) { ks[i] = p.ck_shift[i]; km[i] = p.ck_mask[i]; }
@@ -537,17 +656,17 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                     uint8_t* sa = sw + kWBytes;
                     // (test hook: the first stage of every CTA may be armed for more bytes than its copies deliver, so
                     // that the wait on it runs out and the give-up path below is exercised)
-                    mbar_arrive_expect_tx(&full_bar[stage], issued == 0 ? tx + p.stall_extra_tx : tx);
+                    mbar_arrive_expect_tx(&land_bar[stage], issued == 0 ? tx + p.stall_extra_tx : tx);
                     const int kq = t.flip ? p.k_iters - 1 - kit : kit;
                     const int k0 = (kq * kBK) << p.k_shift;         // first K element of the stage
 #pragma unroll
                     for (int sub = 0; sub < kSubK; ++sub)
-                        tma_load_2d(sa + size_t(sub) * p.a_rows * kAtomBytes, &p.tmap_a[bi], &full_bar[stage],
+                        tma_load_2d(sa + size_t(sub) * p.a_rows * kAtomBytes, &p.tmap_a[bi], &land_bar[stage],
                                     k0 + ((sub * 64) << p.k_shift), t.row0);
                     if (one_box) {
                         // the usual case, one box per stage: the column part of the coordinates was worked out once
                         // for the tile, only the K part changes from stage to stage
-                        tma_load_5d(sw, &p.tmap_b, &full_bar[stage], 0, ((k0 >> ks[0]) & km[0]) + cn[0],
+                        tma_load_5d(sw, &p.tmap_b, &land_bar[stage], 0, ((k0 >> ks[0]) & km[0]) + cn[0],
                                     ((k0 >> ks[1]) & km[1]) + cn[1], ((k0 >> ks[2]) & km[2]) + cn[2],
                                     ((k0 >> ks[3]) & km[3]) + cn[3]);
                     } else {
@@ -558,7 +677,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                                 uint8_t* dst = sw + size_t(kb * p.nbx + nb) * p.box_bytes;
                                 int c[5];
                                 weight_box_coords(p, k, n, kc_expert, c);
-                                tma_load_5d(dst, &p.tmap_b, &full_bar[stage], c[0], c[1], c[2], c[3], c[4]);
+                                tma_load_5d(dst, &p.tmap_b, &land_bar[stage], c[0], c[1], c[2], c[3], c[4]);
                             }
                         }
                     }
@@ -575,7 +694,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                     --s;
                     const uint64_t t0 = global_timer_ns();
                     const uint64_t drain_ns = p.wait_limit_ns < 20000000ull ? p.wait_limit_ns : 20000000ull;
-                    while (!mbar_try_wait(&full_bar[s], ph) && global_timer_ns() - t0 < drain_ns) {}
+                    while (!mbar_try_wait(&land_bar[s], ph) && global_timer_ns() - t0 < drain_ns) {}
                 }
             }
         }
@@ -643,7 +762,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 if (acc == 0) acc_phase ^= 1;
             }
         }
-    } else if (warp == 10) {
+    } else if (warp == 10 && p.generic_b == 1) {
         // ================================ generic-address path: raw memory tiles -> shared memory
         // A stage's weights are kBK/br runs of whole memory tiles, each run contiguous in the tile-major buffer
         // (Eq. 1-2: tiles follow each other along a row of the tile grid).  One untiled bulk copy per run brings them
@@ -703,6 +822,30 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 const uint64_t t0 = global_timer_ns();
                 const uint64_t drain_ns = p.wait_limit_ns < 20000000ull ? p.wait_limit_ns : 20000000ull;
                 while (!mbar_try_wait(&raw_full_bar[s], ph) && global_timer_ns() - t0 < drain_ns) {}
+            }
+        }
+    } else if (warp >= 6 && p.generic_b == 2) {
+        // ================================ memory tiles with 8- or 4-byte rows: fixed up where the copy engine put them
+        // Every warp takes part in every stage, in order (a parity wait cannot tell two phases apart).
+        if (warp < 10) {
+            const int tid = (warp - 6) * 32 + lane;
+            uint32_t it_global = 0;
+            Work w;
+            bool ok = true;
+            while (ok && sched.next(w)) {
+                for (int kit = w.kbeg; kit < w.kend; ++kit, ++it_global) {
+                    const uint32_t stage = it_global % uint32_t(p.num_stages);
+                    const uint32_t phase = (it_global / uint32_t(p.num_stages)) & 1u;
+                    if (!mbar_wait_bounded(&raw_full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull, p.wait_limit_ns)) {
+                        ok = false;
+                        break;
+                    }
+                    fixup_stage_in_place<kBK, kBN>(stages + size_t(stage) * stage_bytes, p.br_log2, p.bc_log2, tid);
+                    fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor-core (async) proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&full_bar[stage]);
+                }
+                if (*abort_ptr) break;
             }
         }
     } else if (warp >= 6) {
@@ -950,8 +1093,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) { mbar_inval(&full_bar[s]); mbar_inval(&empty_bar[s]); }
         for (int b = 0; b < 2; ++b) { mbar_inval(&acc_full_bar[b]); mbar_inval(&acc_empty_bar[b]); }
-        if (p.generic_b)
+        if (p.generic_b == 1)
             for (int r = 0; r < p.raw_slots; ++r) { mbar_inval(&raw_full_bar[r]); mbar_inval(&raw_empty_bar[r]); }
+        if (p.generic_b == 2)
+            for (int s = 0; s < p.num_stages; ++s) mbar_inval(&raw_full_bar[s]);
     }
     __syncthreads();
 }

@@ -36,7 +36,7 @@ def test_config1_tiny_tile_major_and_row_major():
 # TMA-boxable tiles, row-major, one-row tiles (= row-major), and tiles only the generic-address path can read
 BLOCKS = [(16, 128), (32, 64), (8, 256), (64, 64), (16, 512), (0, 0), (1, 1024), (1, 128),
           (8, 2), (16, 1), (8, 16), (16, 8), (32, 4), (16, 32), (32, 16), (2, 64), (4, 128), (64, 8),
-          (8, 8), (8, 1), (64, 1), (128, 1), (4, 8),
+          (8, 8), (8, 1), (64, 1), (128, 1), (4, 8), (8, 4), (16, 2), (64, 4), (64, 2), (128, 2), (128, 4), (4, 4),
           (2, 1024), (4, 512), (2, 256), (64, 32), (128, 16), (4, 32), (256, 16)]
 
 
@@ -55,7 +55,9 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     # of those, single-column tiles of at least 8 rows are read as a K-major operand and tiles with 16-byte rows as
     # they are (if the CTA tile holds whole memory tiles); the rest is permuted in shared memory
     as_stored = hand_addressed and br >= 8 and (bc == 1 or (bc == 8 and br <= cta_k))
-    if hand_addressed and not as_stored and (bc > cta_n or br > cta_k or cta_n * cta_k >= 256 * 128):
+    # tiles with 8- or 4-byte rows are fetched as stored too and then transposed in place, 2 or 4 tiles at a time
+    in_place = hand_addressed and br >= 8 and br <= cta_k and ((bc == 4 and br <= 64) or bc == 2)
+    if hand_addressed and not as_stored and not in_place and (bc > cta_n or br > cta_k or cta_n * cta_k >= 256 * 128):
         # documented limits of the generic-address path: the memory tile must fit inside the CTA tile, and two
         # operand stages plus two raw stage images must fit in shared memory (not with 64 KB of weights per stage)
         from gpu_util import tl
@@ -67,8 +69,8 @@ def test_one_hot_rows_copy_rows_of_B_exactly(br, bc, cta):
     assert torch.equal(C.cpu(), B.float()[ks])
     if hand_addressed:
         from gpu_util import tl
-        assert tl.gemm_last_plan().generic_path == (2 if as_stored else 1)
-        if as_stored and cta_n * cta_k < 256 * 128 and br <= cta_k:
+        assert tl.gemm_last_plan().generic_path == (2 if as_stored else 3 if in_place else 1)
+        if (as_stored or in_place) and cta_n * cta_k < 256 * 128 and br <= cta_k:
             with tl.option(tl.OPT_GENERIC_RAW, 0):            # the same tiles through the permuting path
                 assert torch.equal(run_gemm(A, Bd, M, N, K, br, bc, cta).cpu(), B.float()[ks])
                 assert tl.gemm_last_plan().generic_path == 1
@@ -89,13 +91,15 @@ def test_short_tiles_wider_than_the_cta_tile_and_hand_addressed_tiles_taller_tha
     assert e.value.status == 2
 
 
-AS_STORED = [(16, 8), (8, 8), (64, 8), (16, 1), (8, 1), (32, 1), (64, 1), (128, 1)]
+AS_STORED = [(16, 8), (8, 8), (64, 8), (16, 1), (8, 1), (32, 1), (64, 1), (128, 1),
+             (32, 4), (8, 4), (64, 4), (8, 2), (16, 2), (32, 2), (64, 2)]
 
 
 @pytest.mark.parametrize("br,bc", AS_STORED)
 def test_tiles_read_as_stored_ragged_edges_grouped_and_prefill(br, bc):
-    # Memory tiles with 16-byte rows (raw tiles = core matrices of the no-swizzle operand) and single-column tiles (a
-    # K-major operand in panels): ragged N and K against the oracle, a grouped product, a prefill-sized product on the
+    # Memory tiles with 16-byte rows (raw tiles = core matrices of the no-swizzle operand), single-column tiles (a
+    # K-major operand in panels) and tiles with 8- or 4-byte rows (fetched as stored, 2 or 4 neighbours transposed in
+    # place into a tile with 16-byte rows): ragged N and K against the oracle, a grouped product, a prefill-sized product on the
     # CTA-pair kernel; integer data, so everything is exact; the permuting path must give the same bits.
     from gpu_util import DEV, guarded_out, run_gemm, tile_major_on_device, tl
     G = br * bc * 2
@@ -107,10 +111,10 @@ def test_tiles_read_as_stored_ragged_edges_grouped_and_prefill(br, bc):
         B = inputs.bf16_integers((K, N), -8, 8, seed=N + bc)
         Bd = tile_major_on_device(B, K, N, br, bc)
         want = (A.double() @ B.double()).float()
-        if cta[2] and br > cta[2] and bc == 8:
+        if cta[2] and br > cta[2] and bc != 1:
             continue                                        # the memory tile must fit the CTA tile
         C = run_gemm(A, Bd, M, N, K, br, bc, cta)
-        assert tl.gemm_last_plan().generic_path == (2 if (bc == 1 or br <= tl.gemm_last_plan().cta_k) else 1)
+        assert tl.gemm_last_plan().generic_path == ((3 if bc in (2, 4) else 2) if (bc == 1 or br <= tl.gemm_last_plan().cta_k) else 1)
         assert torch.equal(C.cpu(), want), (M, N, K, cta)
         ref, _ = _oracle_full(A, Bd, TILE, br, bc, M, N, K)
         assert np.array_equal(C.cpu().numpy().astype(np.float64), ref)
@@ -128,7 +132,7 @@ def test_tiles_read_as_stored_ragged_edges_grouped_and_prefill(br, bc):
     g = guarded_out((rows, N), torch.float32)
     tl.gemm_grouped(A.to(DEV), Bd, g.t, torch.from_numpy(offsets).to(DEV), E, rows, N, K, G, br, bc)
     tl.device_status()
-    assert tl.gemm_last_plan().generic_path == 2
+    assert tl.gemm_last_plan().generic_path == (3 if bc in (2, 4) else 2)
     assert torch.equal(g.check().cpu(), want)
     # prefill-sized: the CTA-pair kernel reads the same operand image
     M, N, K = 700, 9600, 256
@@ -137,7 +141,9 @@ def test_tiles_read_as_stored_ragged_edges_grouped_and_prefill(br, bc):
     Bd = tile_major_on_device(B, K, N, br, bc)
     C = run_gemm(A, Bd, M, N, K, br, bc)
     plan = tl.gemm_last_plan()
-    if bc == 1 or br <= 64:
+    if bc in (2, 4):
+        assert plan.pair_kernel == 0 and plan.generic_path == 3           # the pair kernel has no warps for the fix-up
+    elif bc == 1 or br <= 64:
         assert plan.pair_kernel == 1 and plan.generic_path == 2
     assert torch.equal(C.cpu(), (A.double() @ B.double()).float())
 

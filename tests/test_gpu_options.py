@@ -356,15 +356,19 @@ def test_gemm_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
     tl.device_status()                                                    # the flag was cleared by the report
     got = run_gemm(A, Bt, M, N, K, 16, 128)
     assert np.array_equal(got.cpu().numpy().astype(np.float64), want)
-    # the generic-address path has a second arrival on the same barrier; it gives up the same way
-    Bg = tile_major_on_device(B, K, N, 16, 8)
-    with tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
-        tl.set_option(tl.OPT_STALL_ONCE, 1)
-        tl.gemm(A.to(DEV), Bg, C, M, N, K, 256, 16, 8)
-        with pytest.raises(tl.TileLensError) as e:
-            tl.device_status()
-        assert e.value.status == 5
-    assert np.array_equal(run_gemm(A, Bg, M, N, K, 16, 8).cpu().numpy().astype(np.float64), want)
+    # The other weight paths give up the same way: the permuting generic-address path (a second arrival on the same
+    # barrier), tiles read as stored, and tiles fixed up in place (the copies land on a barrier of their own, on which
+    # the four fix-up warps wait).
+    for br, bc, raw, path in ((16, 8, 0, 1), (16, 8, 1, 2), (32, 4, 1, 3), (8, 2, 1, 3)):
+        Bg = tile_major_on_device(B, K, N, br, bc)
+        with tl.option(tl.OPT_WAIT_LIMIT_US, 2000), tl.option(tl.OPT_GENERIC_RAW, raw):
+            tl.set_option(tl.OPT_STALL_ONCE, 1)
+            tl.gemm(A.to(DEV), Bg, C, M, N, K, br * bc * 2, br, bc)
+            assert tl.gemm_last_plan().generic_path == path
+            with pytest.raises(tl.TileLensError) as e:
+                tl.device_status()
+            assert e.value.status == 5
+            assert np.array_equal(run_gemm(A, Bg, M, N, K, br, bc).cpu().numpy().astype(np.float64), want)
 
 
 def test_relayout_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
