@@ -12,14 +12,18 @@
 //                tiles of up to 64 tokens, else 128 rows; spare rows are zeroed once), one MMA covers all cta_n
 //                weight columns; TMEM lane = token row;
 //   weights on M (256-token tiles)  TMEM lane = weight column, the accumulator holds C transposed.
-// Memory tiles whose rows are shorter than 32 bytes cannot be boxed: one more warp streams them into shared memory
-// with untiled bulk copies and four more permute them into the operand image with Eq. 1-2 arithmetic (Section 4.4).
+// Memory tiles whose rows are shorter than 32 bytes cannot be boxed as swizzle rows (the generic-address case of
+// Section 4.4).  With at least 8 rows they are still fetched by the copy engine as stored, the buffer seen as plain
+// bytes: tiles with 16-byte rows are core matrices of the no-swizzle MN-major operand and single-column tiles panels of
+// a K-major operand, both read by the MMA as they are; tiles with 8- or 4-byte rows are transposed in place, 2 or 4
+// neighbouring tiles into one with 16-byte rows, by four more warps.  Tiles of fewer rows: one more warp streams them
+// into shared memory with untiled bulk copies and four more permute them into the operand image with Eq. 1-2 arithmetic.
 //
 // One persistent CTA per SM:
 //   warp 0      TMA producer   (one lane)   ring of shared-memory stages, mbarrier expect-tx
 //   warp 1      MMA issuer     (one lane)   tcgen05.mma into one of two TMEM accumulators
 //   warps 2..5  epilogue                    tcgen05.ld -> fp32 -> C, or silu(gate) * up -> bf16 (expert FFN)
-//   warps 6..10 generic-address weights     (only when the memory tile cannot be boxed)
+//   warps 6..10 in-place transpose (6..9) or generic-address weights   (only when a tile row is shorter than 16 bytes)
 // Work is a list of (output tile, K range); make_plan chooses among
 //   whole tiles round-robin (the tiles fill the SMs, or divide evenly over at least 3/4 of them);
 //   split-K inside clusters: one tile per cluster of up to 8 CTAs, each a share of the K loop, partial tiles added

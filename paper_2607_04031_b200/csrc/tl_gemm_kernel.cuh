@@ -9,8 +9,8 @@
 namespace tl {
 
 constexpr int kGemmThreads = 192;          // TMA path: producer, MMA issuer, four epilogue warps
-constexpr int kGenericThreads = 352;       // generic-address path: four more warps that build the weight operand by hand
-                                           // and one that streams the raw memory tiles into shared memory
+constexpr int kGenericThreads = 352;       // tile rows under 16 bytes: four more warps that transpose the stage in place or build
+                                           // the weight operand by hand, and one that streams raw memory tiles into shared memory
 constexpr int kMaxStages = 16;
 constexpr int kMaxExperts = 1024;
 constexpr int kNumBoxChoices = 5;          // token boxes of 16, 32, 64, 128, 256 rows
