@@ -93,7 +93,9 @@ typedef enum {
                                 the wait on that stage runs out after TL_OPT_WAIT_LIMIT_US, the kernel gives up (drains
                                 its copies, frees tensor memory, returns) and tl_device_status() reports TL_ERR_TIMEOUT.
                                 3 = in the next one-launch tl_moe_ffn CTA 0 does not arrive at the grid barrier, so every
-                                CTA's bounded wait there runs out (detail 0x800).
+                                CTA's bounded wait there runs out (detail 0x800); in the counter form
+                                (TL_OPT_FFN_ONE_LAUNCH = 2) CTA 0 does not raise the counters of the m-tiles it stores,
+                                so the waits of the producers that load them run out (detail 0x900).
                                 That launch's output is undefined.
                                 4 = the next grouped launch builds the tile tables it prepares ahead of its stream
                                 predecessor's completion from wrong expert offsets, so that its check after the wait
@@ -105,8 +107,10 @@ typedef enum {
     TL_OPT_NO_SCRATCH_PLANS, /* 1 (default): dense decode-sized products prefer schedules without partial tiles in global
                                 memory (whole tiles on a grid that divides the tile count, or split-K inside clusters);
                                 0: always the stream-K cut */
-    TL_OPT_FFN_ONE_LAUNCH,   /* 0 (default): tl_moe_ffn runs its two grouped products as two launches; 1: as two phases of one
-                                cooperative launch where it can (measured slower: 236 against 211 us on the Qwen-3 expert FFN) */
+    TL_OPT_FFN_ONE_LAUNCH,   /* 0 (default): tl_moe_ffn runs its two grouped products as two launches; where it can, 1: as two
+                                phases of one cooperative launch with grid-wide barriers, 2: as one cooperative launch in which
+                                the second product's loads wait, m-tile by m-tile, for the first product's rows (measured on the
+                                Qwen-3 expert FFN: 203 us with two launches, 241 us and 220 us in one) */
     TL_OPT_GENERIC_RAW,      /* 1 (default): memory tiles of at least 8 rows whose rows are 16, 8, 4 or 2 bytes long are copied into
                                 shared memory as stored (and, for 8- and 4-byte rows, transposed there in place) and read by the
                                 MMA through a no-swizzle or K-major descriptor; 0: they take the permuting generic-address path */
@@ -231,8 +235,11 @@ int tl_gemm_grouped(const void* d_A_sorted, const void* d_B_experts, float* d_C,
  * afterwards.  Two launches in stream order (the second overlaps the first one's end through programmatic stream
  * serialisation).  With TL_OPT_FFN_ONE_LAUNCH = 1 and TMA-readable weights both products run as two phases of ONE
  * cooperative launch instead (a grid-wide barrier with a bounded wait between them; the split tiles of the first
- * product are summed inside the kernel, those of the second by the small reduction kernel that follows): same bits,
- * measured slower, and every CTA of its grid has to be resident at the same time.
+ * product are summed inside the kernel, those of the second by the small reduction kernel that follows): same bits
+ * as two launches.  With TL_OPT_FFN_ONE_LAUNCH = 2 the one launch has no barrier: the first product runs whole tiles
+ * only, its epilogue counts every m-tile of H it has stored, and the second product's loads of an m-tile wait (with
+ * a bound) for that count; a sum of H may then be taken in another order than with two launches (same tolerance).
+ * Both one-launch forms are measured slower than two launches and need every CTA of their grid resident at once.
  */
 /* tl_gemm / tl_gemm_grouped with C written as bf16 (fp32 accumulation, one rounding to nearest even): d_C_bf16
  * M x N (total_rows x N) bf16, 16-byte aligned, N % 8 == 0.  The paper leaves the output type open. */

@@ -204,6 +204,7 @@ int tl_set_option(int option, int64_t value) {
         case TL_OPT_STALL_ONCE: if (value < 0 || value > 4) return TL_ERR_INVALID_ARG; break;
         case TL_OPT_SM_LIMIT: if (value < 0 || value > 4096) return TL_ERR_INVALID_ARG; break;
         case TL_OPT_MOE_ROW_CAP: if (value != 0 && value != 16 && value != 32 && value != 64 && value != 128) return TL_ERR_INVALID_ARG; break;
+        case TL_OPT_FFN_ONE_LAUNCH: if (value < 0 || value > 2) return TL_ERR_INVALID_ARG; break;
         default: if (value != 0 && value != 1) return TL_ERR_INVALID_ARG; break;
     }
     tl::options().v[option] = value;

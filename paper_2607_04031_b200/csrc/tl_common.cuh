@@ -93,7 +93,8 @@ enum : uint32_t {
     kWaitProducerEmpty = 0x100, kWaitMmaFull = 0x200, kWaitMmaAccEmpty = 0x300,
     kWaitEpilogueAccFull = 0x400, kWaitTeardown = 0x500, kWaitRelayoutFull = 0x600,
     kBadCopy = 0x700,           // a bulk copy's source or destination failed the kernel's own range / alignment check
-    kWaitGridBarrier = 0x800    // the grid-wide barrier between the two products of the expert FFN kernel
+    kWaitGridBarrier = 0x800,   // the grid-wide barrier between the two products of the expert FFN kernel
+    kWaitTileFlag = 0x900       // the second product's producer waiting for an m-tile of the first product's output
 };
 
 // ------------------------------------------------------------- device helpers

@@ -981,6 +981,39 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
                           plan1.stream_k && plan2.stream_k && !p1.generic_b && !p2.generic_b && grid > 1 &&
                           plan1.smem_bytes <= size_t(tl::kMaxDynamicSmem - 10 * 1024) &&
                           plan2.smem_bytes <= size_t(tl::kMaxDynamicSmem - 10 * 1024);
+        if (same && tl::opt(TL_OPT_FFN_ONE_LAUNCH) == 2) {
+            // Per-m-tile counters instead of grid barriers (see tl_gemm_chain.cu): the first product as whole tiles
+            // only, the second one as usual with its producer waiting for the rows of H it loads.  The workspace
+            // holds the second product's partial tiles and, behind them, one counter per m-tile, cleared here.
+            const size_t part_bytes = size_t(2) * size_t(grid) * plan2.BM * plan2.BN * sizeof(float);
+            const size_t n_flags = size_t(total_rows / plan1.BM) + size_t(E) + 1;
+            const size_t ws_bytes = part_bytes + n_flags * sizeof(uint32_t);
+            void* ws = nullptr;
+            if ((rc = tl::get_workspace(ws_bytes, &ws))) return rc;
+            uint32_t* flags = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + part_bytes);
+            if ((rc = tl::check_cuda(cudaMemsetAsync(flags, 0, n_flags * sizeof(uint32_t), stream)))) return rc;
+            p1.partials = nullptr;
+            p1.stream_k = 0;
+            p1.tile_flags = p2.tile_flags = flags;
+            p1.tile_flags_mode = 1;
+            p2.tile_flags_mode = 2;
+            p2.tile_flags_target = 4u * uint32_t(p1.n_tiles);          // four epilogue warps per tile of the first product
+            p2.partials = static_cast<float*>(ws);
+            // Test hook (TL_OPT_STALL_ONCE = 3): CTA 0 keeps its arrivals to itself, the waits on its m-tiles run out.
+            if (tl::opt(TL_OPT_STALL_ONCE) == 3) {
+                p1.tile_flags_skip_cta0 = 1;
+                tl_set_option(TL_OPT_STALL_ONCE, 0);
+            }
+            const size_t smem = plan1.smem_bytes > plan2.smem_bytes ? plan1.smem_bytes : plan2.smem_bytes;
+            rc = tl::launch_gemm_chain(plan1.BK, plan1.BN, grid, smem, stream, p1, p2, tl::dev().d_grid_counter, 0, 0, false);
+            if (rc) return rc;
+            tl_gemm_plan_info& info = tl::last_plan();
+            memset(&info, 0, sizeof info);
+            info.cta_m = plan2.BM; info.cta_n = plan2.BN; info.cta_k = plan2.BK; info.stream_k = 1; info.grid = grid;
+            info.stages = plan2.num_stages; info.weights_on_n = 1; info.cluster_k = 1; info.workspace_bytes = ws_bytes;
+            info.chained = 2;
+            return tl::launch_reduce(p2, grid, stream, false);
+        }
         if (same) {
             tl::DeviceState& d = tl::dev();
             // one workspace for both phases, sized for the common grid (the first product's partial tiles are summed

@@ -13,11 +13,26 @@
 // which it raises the status word and goes on, so the kernel always terminates.  All CTAs must be resident at the
 // same time: the kernel is launched cooperatively (the launch fails rather than wait on a CTA that cannot run).
 //
-// Measured on B200 (Qwen-3-30B-A3B expert FFN, 2048 routed rows): 236 us against 211 us for the same two products as
-// two launches.  The boundary between two launches is already hidden by programmatic stream serialisation; with the
-// barriers and the in-kernel sum compiled out the one-launch form only ties (217 us), the two barriers add 12 us
-// (every CTA waits for the slowest, twice) and the in-kernel sum 14 us (its index arithmetic is no longer hidden
-// behind the first product's tail).  tl_moe_ffn therefore uses two launches unless TL_OPT_FFN_ONE_LAUNCH is set.
+// A second form needs no barrier at all: the first product is scheduled as whole tiles only (no partial tiles, nothing
+// to sum), every epilogue warp adds one to a counter of the m-tile whose rows of H it has stored, and the second
+// product's producer waits, tile by tile and with a bound, until the counter of the m-tile it is about to load has
+// reached (warps x column tiles of the first product).  A CTA that runs out of first-product tiles goes straight on
+// to second-product tiles, whose experts were finished long ago: nobody waits for the slowest CTA.  No tile of the
+// first product ever waits, and every CTA finishes its first-product tiles before it starts the second product, so
+// the counters always fill (the cooperative launch keeps all CTAs resident); the counters are cleared by a memset
+// enqueued before the launch.
+//
+// Measured on B200 (Qwen-3-30B-A3B expert FFN, 2048 routed rows, back-to-back calls): 203 us for the two products as
+// two launches, 241 us with the barriers, 220 us with the counters (214 us when launched with programmatic stream
+// serialisation instead of cooperatively, which is not kept: the co-residency the waits rely on would then rest on the
+// grid being no larger than the SM count).  The counter form's first product cannot balance its last, partial round
+// of tiles the way the stream-K cut does (the CTAs that ran one tile more finish 6 % later); giving the other CTAs a
+// larger share of the second product's cut part instead made it slower still (238 us): that part then starts while
+// the last experts' rows of H are still being computed, and waits.
+// The boundary between two launches is already hidden by programmatic stream serialisation: with the barriers and
+// the in-kernel sum compiled out the barrier form only tied with two launches; its two barriers add 12 us (every CTA
+// waits for the slowest, twice) and the in-kernel sum 14 us (its index arithmetic is no longer hidden behind the first
+// product's tail).  tl_moe_ffn therefore uses two launches unless TL_OPT_FFN_ONE_LAUNCH is set.
 #include "tl_gemm_kernel.cuh"
 
 namespace tl {
@@ -66,6 +81,12 @@ gemm_chain_kernel(const __grid_constant__ GemmParams p1, const __grid_constant__
     __shared__ int row_start[kMaxExperts + 1];
     __shared__ int slot_of[kRangeTabMax];
     gemm_body<kBK, kBN, true, false>(p1, true, false);
+    if (p1.tile_flags_mode == 1) {
+        // Per-m-tile counters instead of barriers: the first product runs whole tiles only, every CTA goes straight on to
+        // its tiles of the second product, whose producer waits for the rows it is about to load (see gemm_body).
+        gemm_body<kBK, kBN, true, false>(p2, false, true);
+        return;
+    }
     const bool ok1 = grid_barrier(counter, target1, p1.wait_limit_ns, p1.status, skip_cta0 != 0 && blockIdx.x == 0);
     if (ok1 && int(blockIdx.x) + 1 < int(gridDim.x))
         streamk_reduce_body<false>(p1, int(gridDim.x), int(blockIdx.x), prefix, row_start, slot_of);

@@ -29,6 +29,14 @@ struct alignas(64) GemmParams {
     uint32_t* status;
     uint64_t wait_limit_ns;     // bound of every barrier wait in the kernel
     uint32_t stall_extra_tx;    // test hook: bytes added to what the first stage's barrier expects (0 in normal use)
+    // Two grouped products in one launch, the second one's tokens being the first one's output (expert FFN): one
+    // counter per m-tile.  tile_flags_mode 1: every epilogue warp adds one to tile_flags[m-tile] once its share of a
+    // whole output tile is stored; 2: the producer loads an m-tile's tokens only after tile_flags[m-tile] has reached
+    // tile_flags_target (bounded wait).  0: not used.
+    uint32_t* tile_flags;
+    int tile_flags_mode;
+    uint32_t tile_flags_target;
+    int tile_flags_skip_cta0;   // test hook: CTA 0 does not add to the counters, so that the waits on its m-tiles run out
     int provisional_skew;       // test hook: rows added to the expert offsets read before the wait (0 in normal use)
     int reduce_split;           // stream-K reduction: 1 = every boundary inside a split tile sums a share of it
     int64_t ldc;                // N
@@ -91,6 +99,7 @@ struct TileInfo {
     int rows;        // valid rows (<= BM)
     int expert;
     int flip;        // odd m-tile of its (expert, n-tile): walks K backwards (see decode_tile)
+    int mtile;       // index of the m-tile among all m-tiles of the problem (experts in order)
 };
 
 // ------------------------------------------------------------------ scheduler
@@ -209,6 +218,7 @@ __device__ __forceinline__ TileInfo decode_tile(const GemmParams& p, const int* 
     // handed out round-robin run at the same time on different SMs and share the slab while both walk it forwards.)
     t.flip = flip_odd ? (local % mt) & 1 : 0;
     t.rows = row_end - t.row0 < p.BM ? row_end - t.row0 : p.BM;
+    t.mtile = p.tile_flags_mode ? prefix[e] / p.n_tiles + local % mt : 0;
     return t;
 }
 
@@ -647,6 +657,32 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 int cn[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) cn[i] = ((t.n0 >> p.cn_shift[i]) & p.cn_mask[i]) + p.c_expert[i] * kc_expert;
+                if (p.tile_flags_mode == 2) {
+                    // The tile's token rows are another product's output, written by other CTAs of this launch: wait
+                    // (bounded) until every warp that stores a part of this m-tile has said so (each of them has ordered
+                    // its stores before the copy engine's reads by a proxy fence of its own).
+                    const uint32_t* flag = p.tile_flags + t.mtile;
+                    uint64_t t0 = 0;
+                    uint32_t polls = 0;
+                    while (true) {
+                        uint32_t seen;
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+                        if (seen >= p.tile_flags_target) break;
+                        __nanosleep(64);
+                        if ((++polls & 63u) == 0) {
+                            const uint64_t now = global_timer_ns();
+                            if (t0 == 0) t0 = now;
+                            if (*abort_ptr || now - t0 > p.wait_limit_ns) {
+                                atomicCAS(p.status, 0u, kWaitTileFlag);
+                                *abort_ptr = 1;
+                                ok = false;
+                                break;
+                            }
+                        }
+                    }
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async.global;" ::: "memory");     // (and on the reading side as well)
+                }
                 for (int kit = w.kbeg; kit < w.kend; ++kit) {
                     if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1, abort_ptr, p.status, kWaitProducerEmpty, p.wait_limit_ns)) {
                         ok = false;
@@ -1031,6 +1067,14 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty_bar[acc]);
+            if (p.tile_flags_mode == 1 && ok && full && !(p.tile_flags_skip_cta0 && blockIdx.x == 0)) {
+                // this warp's part of the tile is stored: visible device-wide, also to the copy engines that will read
+                // it as another product's tokens, before the m-tile's counter moves
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(p.tile_flags + t.mtile, 1u);
+            }
             acc ^= 1;
             if (acc == 0) acc_phase ^= 1;
 
@@ -1155,7 +1199,7 @@ __device__ __forceinline__ void streamk_reduce_body(const GemmParams& p, int gem
             }
         }
     }
-    TileInfo t = {0, 0, 0, 0, 0};
+    TileInfo t = {0, 0, 0, 0, 0, 0};
     if (active) {
         t = decode_tile(p, prefix, row_start, tile);
         // slots of the contributors, computed before the wait (the load loop below must not divide)

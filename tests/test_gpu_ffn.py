@@ -17,7 +17,7 @@ def _bf16_steps(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def _run_case(E, hidden, inter, tokens, topk, br, bc, n_check, seed):
+def _run_case(E, hidden, inter, tokens, topk, br, bc, n_check, seed, want_chained=0):
     from gpu_util import DEV, tl
     offsets, counts, _ = inputs.zipf_topk_routing(tokens, E, topk, 1.1, seed=seed)
     rows = int(offsets[-1])
@@ -34,6 +34,7 @@ def _run_case(E, hidden, inter, tokens, topk, br, bc, n_check, seed):
     from gpu_util import guarded_out
     gH, gY = guarded_out((rows, inter), torch.bfloat16), guarded_out((rows, hidden), torch.float32)
     tl.moe_ffn(X, Wgu_t, Wd_t, gH.t, gY.t, torch.from_numpy(offsets).to(DEV), E, rows, hidden, inter, G, br, bc)
+    assert tl.gemm_last_plan().chained == want_chained
     tl.device_status()
     H, Y = gH.check(), gY.check()
     assert torch.isfinite(H.float()).all() and torch.isfinite(Y).all()
@@ -150,6 +151,77 @@ def test_one_launch_and_two_launches_give_the_same_bits(E, hidden, inter, tokens
         assert chained1 == 1, "the one-launch form was not taken"
         assert torch.equal(H1.view(torch.int16), H0.view(torch.int16)) and torch.equal(Y1, Y0), rep
     assert torch.isfinite(Y1).all()
+
+
+@pytest.mark.parametrize("case", [dict(E=8, hidden=256, inter=128, tokens=64, topk=2, n_check=24, seed=5),
+                                  dict(E=16, hidden=128, inter=512, tokens=96, topk=4, n_check=24, seed=6),
+                                  dict(E=3, hidden=4096, inter=64, tokens=700, topk=1, n_check=12, seed=7),
+                                  dict(E=128, hidden=2048, inter=768, tokens=256, topk=8, n_check=12, seed=0)])
+def test_one_launch_with_per_m_tile_counters_against_the_oracle(case):
+    # TL_OPT_FFN_ONE_LAUNCH = 2: one cooperative launch without grid barriers.  The first product runs whole tiles only
+    # (so H may differ from the two-launch form in the order of a sum, never by more than the bound below), every
+    # epilogue warp counts the m-tile it has stored, and the second product's producer waits for the m-tile it loads.
+    # Checked against the oracle with the two-launch form's bounds, and for run-to-run reproducibility.
+    from gpu_util import DEV, tl
+    with tl.option(tl.OPT_FFN_ONE_LAUNCH, 2):
+        _run_case(br=16, bc=128, want_chained=2, **case)
+    E, hidden, inter = case["E"], case["hidden"], case["inter"]
+    offsets, counts, _ = inputs.zipf_topk_routing(case["tokens"], E, case["topk"], 1.1, seed=case["seed"])
+    rows = int(offsets[-1])
+    X = inputs.bf16_normal((rows, hidden), 1.0, seed=11, device=DEV)
+    Wgu = inputs.bf16_normal((E, hidden, 2 * inter), 0.05, seed=12, device=DEV)
+    Wd = inputs.bf16_normal((E, inter, hidden), 0.05, seed=13, device=DEV)
+    d_off = torch.from_numpy(offsets).to(DEV)
+    outs = []
+    for mode in (2, 2, 0):
+        H = torch.zeros((rows, inter), dtype=torch.bfloat16, device=DEV)
+        Y = torch.zeros((rows, hidden), dtype=torch.float32, device=DEV)
+        with tl.option(tl.OPT_FFN_ONE_LAUNCH, mode):
+            tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)
+            tl.device_status()
+        outs.append((H, Y))
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16)) and torch.equal(outs[0][1], outs[1][1])
+    # against the two-launch form: a sum in another order now and then (one bf16 step of h, or a few steps of an h that
+    # is tiny because g or u cancelled, see _run_case)
+    steps = _bf16_steps(inputs.bits(outs[0][0]), inputs.bits(outs[2][0]))
+    assert np.mean(steps == 0) > 0.99
+    h_scale = float(outs[2][0].float().abs().max())
+    assert float((outs[0][0].float() - outs[2][0].float()).abs().max()) <= 2.0 ** -7 * h_scale
+    scale = float(outs[2][1].abs().max())
+    assert float((outs[0][1] - outs[2][1]).abs().max()) <= 2e-3 * scale
+
+
+def test_m_tile_counter_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
+    # Counter form: CTA 0 keeps the arrivals of its tiles to itself (test hook), the producers that need those m-tiles wait
+    # out the shortened limit, the kernel terminates, the status reads TL_ERR_TIMEOUT (detail 0x900), the next call is clean.
+    from gpu_util import DEV, tl
+    E, hidden, inter = 16, 128, 512
+    offsets, counts, _ = inputs.zipf_topk_routing(96, E, 4, 1.1, seed=4)
+    rows = int(offsets[-1])
+    X = inputs.bf16_normal((rows, hidden), 1.0, seed=1, device=DEV)
+    Wgu = inputs.bf16_normal((E, hidden, 2 * inter), 0.05, seed=2, device=DEV)
+    Wd = inputs.bf16_normal((E, inter, hidden), 0.05, seed=3, device=DEV)
+    d_off = torch.from_numpy(offsets).to(DEV)
+    H = torch.zeros((rows, inter), dtype=torch.bfloat16, device=DEV)
+    Y = torch.zeros((rows, hidden), dtype=torch.float32, device=DEV)
+    with tl.option(tl.OPT_FFN_ONE_LAUNCH, 2):
+        tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)
+        tl.device_status()
+        H0, Y0 = H.clone(), Y.clone()
+        with tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
+            tl.set_option(tl.OPT_STALL_ONCE, 3)
+            tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)
+            assert tl.get_option(tl.OPT_STALL_ONCE) == 0 and tl.gemm_last_plan().chained == 2
+            with pytest.raises(tl.TileLensError) as e:
+                tl.device_status()
+            assert e.value.status == 5 and "detail=0x900" in str(e.value)
+        tl.device_status()
+        for _ in range(2):
+            H.zero_(); Y.zero_()
+            tl.moe_ffn(X, Wgu, Wd, H, Y, d_off, E, rows, hidden, inter, 0, 0, 0)
+            assert tl.gemm_last_plan().chained == 2
+            tl.device_status()
+            assert torch.equal(H.view(torch.int16), H0.view(torch.int16)) and torch.equal(Y, Y0)
 
 
 def test_grid_barrier_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
