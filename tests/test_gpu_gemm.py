@@ -104,7 +104,10 @@ def test_tiles_read_as_stored_ragged_edges_grouped_and_prefill(br, bc):
     from gpu_util import DEV, guarded_out, run_gemm, tile_major_on_device, tl
     G = br * bc * 2
     for M, N, K, cta in ((40, 1160, 1152, (0, 0, 0)), (130, 1096, 640, (128, 128, 128)), (300, 648, 384, (0, 0, 0)),
-                         (9, 2056, 2176, (64, 256, 64))):
+                         (9, 2056, 2176, (64, 256, 64)), (24, 1156, 512, (0, 0, 0))):
+        if N % bc:
+            continue                                        # (1156 columns: only for tiles of 1, 2 or 4 columns; the last
+                                                            #  group of 2 or 4 neighbouring tiles is then incomplete)
         if K % br:
             K += br - K % br
         A = inputs.bf16_integers((M, K), -8, 8, seed=M + br)
