@@ -174,7 +174,8 @@ static void default_tile(int64_t rows_max, bool grouped, bool narrow_scratch, in
 }
 
 static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k,
-                     bool grouped, GemmPlan* plan, bool narrow_scratch = false, bool generic = false, bool pair_sized = true) {
+                     bool grouped, GemmPlan* plan, bool narrow_scratch = false, bool generic = false, bool pair_sized = true,
+                     int64_t rows_total = 0) {
     if (int rc = ensure_device_info()) return rc;
     int sms = dev().sm_count;
     if (opt(TL_OPT_SM_LIMIT) > 0 && opt(TL_OPT_SM_LIMIT) < sms) sms = int(opt(TL_OPT_SM_LIMIT));
@@ -228,6 +229,13 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     const int64_t waves = ceil_div(tile_bound, sms);
     const bool even = tile_bound >= sms && double(tile_bound) / double(waves * sms) >= 0.92;
     plan->stream_k = (grouped || !even) ? 1 : 0;
+    // From four whole rounds of short tiles on the kernel cuts nothing (Sched::whole_rounds_tiles); where the host can
+    // tell (dense: the tile count; grouped: at least ceil(rows / BM) m-tiles whatever the routing) it plans whole tiles
+    // outright: no workspace, no reduction kernel.
+    {
+        const int64_t tiles_min = grouped ? ceil_div(rows_total, BM) * ceil_div(N, BN) : tile_bound;
+        if (plan->stream_k && tiles_min >= int64_t(kNoCutRounds) * sms && k_iters <= kNoCutStages) plan->stream_k = 0;
+    }
     plan->cluster_k = 1;
     int64_t grid = plan->stream_k ? (total_iters < sms ? total_iters : sms) : (tile_bound < sms ? tile_bound : sms);
     // Dense decode-sized products: a schedule without partial tiles in global memory beats the stream-K cut even
@@ -372,22 +380,22 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         // path takes over.
         if (raw_shape) {
             const int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
+                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized, rows_total);
             raw_operand = rc == TL_OK && plan.BK % br == 0 && plan.BN % bc == 0;
         }
         if (kcol_shape) {
             const int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
+                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized, rows_total);
             kcol_operand = rc == TL_OK;
         }
         if (fix_shape) {
             const int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized);
+                                     d_offsets != nullptr, &plan, fixed != nullptr, false, pair_sized, rows_total);
             fix_operand = rc == TL_OK && plan.BK % br == 0;
         }
         if (!raw_operand && !kcol_operand && !fix_operand)
             if (int rc = make_plan(rows_max, mt_bound * ceil_div(N, bn_guess), N, K >> k_shift, cta_m, cta_n, cta_k,
-                                   d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized))
+                                   d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized, rows_total))
                 return rc;
     }
     if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
