@@ -229,12 +229,12 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     const int64_t waves = ceil_div(tile_bound, sms);
     const bool even = tile_bound >= sms && double(tile_bound) / double(waves * sms) >= 0.92;
     plan->stream_k = (grouped || !even) ? 1 : 0;
-    // From four whole rounds of short tiles on the kernel cuts nothing (Sched::whole_rounds_tiles); where the host can
-    // tell (dense: the tile count; grouped: at least ceil(rows / BM) m-tiles whatever the routing) it plans whole tiles
-    // outright: no workspace, no reduction kernel.
+    // With short tiles and enough of them the kernel cuts nothing (Sched::no_cut); where the host can tell (dense: the
+    // tile count; grouped: at least ceil(rows / BM) m-tiles whatever the routing) it plans whole tiles outright: no
+    // workspace, no reduction kernel.
     {
         const int64_t tiles_min = grouped ? ceil_div(rows_total, BM) * ceil_div(N, BN) : tile_bound;
-        if (plan->stream_k && tiles_min >= int64_t(kNoCutRounds) * sms && k_iters <= kNoCutStages) plan->stream_k = 0;
+        if (plan->stream_k && tiles_min * 4 >= 3 * int64_t(sms) && k_iters <= kNoCutStages) plan->stream_k = 0;
     }
     plan->cluster_k = 1;
     int64_t grid = plan->stream_k ? (total_iters < sms ? total_iters : sms) : (tile_bound < sms ? tile_bound : sms);
@@ -986,7 +986,7 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
         const int grid = plan1.grid > plan2.grid ? plan1.grid : plan2.grid;
         const bool same = plan1.BM == plan2.BM && plan1.BN == plan2.BN && plan1.BK == plan2.BK &&
                           plan1.BK == 64 && plan1.BN == 256 && plan1.weights_on_n && plan2.weights_on_n &&
-                          plan1.stream_k && plan2.stream_k && !p1.generic_b && !p2.generic_b && grid > 1 &&
+                          plan1.cluster_k == 1 && plan2.cluster_k == 1 && !p1.generic_b && !p2.generic_b && grid > 1 &&
                           plan1.smem_bytes <= size_t(tl::kMaxDynamicSmem - 10 * 1024) &&
                           plan2.smem_bytes <= size_t(tl::kMaxDynamicSmem - 10 * 1024);
         if (same && tl::opt(TL_OPT_FFN_ONE_LAUNCH) == 2) {
@@ -1020,7 +1020,8 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
             info.cta_m = plan2.BM; info.cta_n = plan2.BN; info.cta_k = plan2.BK; info.stream_k = 1; info.grid = grid;
             info.stages = plan2.num_stages; info.weights_on_n = 1; info.cluster_k = 1; info.workspace_bytes = ws_bytes;
             info.chained = 2;
-            return tl::launch_reduce(p2, grid, stream, false);
+            info.stream_k = plan2.stream_k;
+            return plan2.stream_k ? tl::launch_reduce(p2, grid, stream, false) : TL_OK;
         }
         if (same) {
             tl::DeviceState& d = tl::dev();
@@ -1045,7 +1046,8 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
             info.cta_m = plan2.BM; info.cta_n = plan2.BN; info.cta_k = plan2.BK; info.stream_k = 1; info.grid = grid;
             info.stages = plan2.num_stages; info.weights_on_n = 1; info.cluster_k = 1; info.workspace_bytes = ws_bytes;
             info.chained = 1;
-            return tl::launch_reduce(p2, grid, stream, false);
+            info.stream_k = plan2.stream_k;
+            return plan2.stream_k ? tl::launch_reduce(p2, grid, stream, false) : TL_OK;
         }
     }
     if (int rc = tl_gemm_grouped_swiglu(d_X_sorted, d_W_gate_up, d_H_bf16, d_offsets, E, total_rows, 2 * inter, hidden, G,

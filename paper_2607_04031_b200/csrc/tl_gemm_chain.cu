@@ -23,7 +23,8 @@
 // enqueued before the launch.
 //
 // Measured on B200 (Qwen-3-30B-A3B expert FFN, 2048 routed rows, back-to-back calls): 203 us for the two products as
-// two launches, 241 us with the barriers, 220 us with the counters (214 us when launched with programmatic stream
+// two launches, 241 us with the barriers, 220 us with the counters (198, 216-221 and 208-210 us since short tiles are
+// no longer cut along K in either product) (214 us when launched with programmatic stream
 // serialisation instead of cooperatively, which is not kept: the co-residency the waits rely on would then rest on the
 // grid being no larger than the SM count).  The counter form's first product cannot balance its last, partial round
 // of tiles the way the stream-K cut does (the CTAs that ran one tile more finish 6 % later); giving the other CTAs a
@@ -88,7 +89,7 @@ gemm_chain_kernel(const __grid_constant__ GemmParams p1, const __grid_constant__
         return;
     }
     const bool ok1 = grid_barrier(counter, target1, p1.wait_limit_ns, p1.status, skip_cta0 != 0 && blockIdx.x == 0);
-    if (ok1 && int(blockIdx.x) + 1 < int(gridDim.x))
+    if (ok1 && p1.stream_k && int(blockIdx.x) + 1 < int(gridDim.x))
         streamk_reduce_body<false>(p1, int(gridDim.x), int(blockIdx.x), prefix, row_start, slot_of);
     grid_barrier(counter, target2, p1.wait_limit_ns, p1.status);
     gemm_body<kBK, kBN, true, false>(p2, false, true);
