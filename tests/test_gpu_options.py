@@ -231,6 +231,32 @@ def test_grouped_tables_built_ahead_of_the_wait_are_checked_and_rebuilt():
         assert torch.equal(g.check().cpu(), want)
 
 
+@pytest.mark.parametrize("E,rows_per_expert,K,N,host_cut", [(16, 128, 512, 1024, 0),    # the host rules the cut out
+                                                            (96, 1, 512, 1024, 1),      # the kernel does, from 384 tiles
+                                                            (12, 8, 512, 1024, 1),      # 48 tiles: cut over all CTAs
+                                                            (96, 1, 4096, 1024, 1)])    # 64-stage tiles: cut
+def test_grouped_products_with_and_without_the_cut_are_exact(E, rows_per_expert, K, N, host_cut):
+    # Short tiles in sufficient number are handed out whole (no partial tiles, no reduction); otherwise what is left after
+    # the whole rounds is cut along K.  Which of the two runs is decided from the tile count, by the host where the
+    # row count alone settles it, else by the kernel (the reduction kernel then finds nothing to add).  Integer data:
+    # every case must be exact.
+    from gpu_util import DEV, guarded_out, tile_major_on_device, tl
+    offsets = (np.arange(E + 1) * rows_per_expert).astype(np.int32)
+    rows = int(offsets[-1])
+    A = inputs.bf16_integers((rows, K), -8, 8, seed=E)
+    B = inputs.bf16_integers((E * K, N), -8, 8, seed=K)
+    Bt = tile_major_on_device(B, E * K, N, 16, 128)
+    want = torch.empty((rows, N), dtype=torch.float32)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        want[r0:r1] = (A[r0:r1].double() @ B[e * K:(e + 1) * K].double()).float()
+    g = guarded_out((rows, N), torch.float32)
+    tl.gemm_grouped(A.to(DEV), Bt, g.t, torch.from_numpy(offsets).to(DEV), E, rows, N, K, 4096, 16, 128)
+    assert tl.gemm_last_plan().stream_k == host_cut
+    tl.device_status()
+    assert torch.equal(g.check().cpu(), want)
+
+
 def test_relayout_without_the_copy_engine_matches_the_oracle():
     from gpu_util import Guarded, dev_bytes, tl
     for rows, cols, s, br, bc in ((512, 512, 2, 16, 128), (1056, 2176, 2, 32, 64), (256, 1024, 1, 64, 64)):
@@ -319,6 +345,15 @@ def test_default_plans_of_the_benchmark_shapes():
     p = tl.gemm_plan(4096, 57344, 8192)
     assert p.pair_kernel == 1 and p.cta == (512, 128, 64) and p.workspace_bytes == 0 and p.grid % 2 == 0
     assert 2 * p.pair_tiles_512 + p.pair_tiles_256 == 16 * 224
+    # grouped, short tiles (at most 32 stages) and at least 64 m-tiles whatever the routing: whole tiles, nothing is cut
+    for N, K in ((1536, 2048), (2048, 768)):
+        p = tl.gemm_plan(2048, N, K, E=128)
+        assert p.cta == (32, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 1, sms, 0)
+    # too few rows for the host to rule the cut out (the kernel decides from the tile count), and long tiles
+    p = tl.gemm_plan(64, 1536, 2048, E=128)
+    assert p.stream_k == 1 and p.workspace_bytes > 0
+    p = tl.gemm_plan(2048, 2048, 8192, E=128)
+    assert p.stream_k == 1 and p.workspace_bytes > 0
 
 
 def test_workspace_bound_covers_many_small_experts():
