@@ -369,12 +369,15 @@ size_t tl_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K);
  *                 the kernel expires; NULL keeps the flag in the array, unread.
  *   limit         problems whose split-K scratch exceeds the array return
  *                 TL_ERR_WORKSPACE and enqueue nothing.  The scratch is
- *                 2 * (number of SMs) * cta_m * cta_n * 4 bytes when the
- *                 output tiles do not fill the SMs evenly (fewer tiles than
- *                 SMs, or a last wave less than 92 % full), else 0; products
- *                 that run on CTA pairs need none.  The default tile here is
- *                 128 columns wide: on a 148-SM B200 that admits every
- *                 M <= 32; M in (32, 64] needs 9.3 MB and is refused.
+ *                 2 * (number of SMs) * cta_m * cta_n * 4 bytes when the K
+ *                 loops are cut over all SMs, which happens when the output
+ *                 tiles do not fill the SMs evenly (fewer tiles than SMs, or
+ *                 a last wave less than 92 % full) and no schedule without
+ *                 partial tiles in global memory exists (tl_gemm_plan tells);
+ *                 else 0; products that run on CTA pairs need none.  The
+ *                 default tile here is 128 columns wide: on a 148-SM B200 that
+ *                 admits every M <= 32; M in (32, 64] needs 9.3 MB when it is
+ *                 cut and is then refused.
  *   first call    the first call on each device looks up the array's device
  *                 address (with that device current).  Make that call before
  *                 starting any stream capture.

@@ -243,7 +243,7 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     // (measured: Llama gate_up, M = 8, 224 whole tiles on 112 CTAs 135 us, cut over 148 CTAs 142 us).  In order:
     //   1. whole tiles on the largest grid of at least 3/4 of the SMs that divides the tile count;
     //   2. one tile per cluster of S <= 8 CTAs which split its K loop S ways and add their partial tiles through
-    //      distributed shared memory, for the S that fills most SMs (at least 3/4 of them);
+    //      distributed shared memory, for the S that fills most SMs (at least 3/4 of them; small problems: any number);
     //   3. the stream-K cut with its workspace and reduction kernel.
     if (plan->stream_k && !grouped && plan->weights_on_n && !generic && opt(TL_OPT_NO_SCRATCH_PLANS) != 0) {
         const int64_t lo = (3 * int64_t(sms) + 3) / 4;
@@ -258,6 +258,16 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
             if (tile_bound * s <= sms && tile_bound * s >= lo && k_iters >= s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024 &&
                 tile_bound * s > int64_t(best_s) * tile_bound)
                 best_s = s;
+        // Small problems (a few MB of weights: latency, not bandwidth) that fill neither: clusters all the same, however
+        // few, as long as every CTA keeps at least two K iterations.  The cut would give each of many CTAs a single
+        // iteration, a partial tile in global memory each, and a second kernel to add them.
+        // (Qwen-3 attention projections, 128 to 512 tokens: k / v 13.7-16.9 -> 11.4-11.6 us, o at 128 tokens 17.9 -> 14.4 us)
+        if (g1 == 0 && best_s == 0 && total_iters * BK * BN * 2 <= (int64_t(16) << 20))
+            for (int s = s_max; s >= 2; --s)
+                if (tile_bound * s <= sms && k_iters >= 2 * s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024) {
+                    best_s = s;
+                    break;
+                }
         if (g1 > 0) {
             plan->stream_k = 0;
             grid = g1;

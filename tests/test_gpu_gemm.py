@@ -416,10 +416,11 @@ def test_host_buffer_entry_point():
 
 def test_caller_workspace_and_errors():
     from gpu_util import DEV, run_gemm, tile_major_on_device, tl
-    M, N, K = 16, 512, 4096
+    M, N, K = 16, 2304, 8192               # 9 tiles of long K, 38 MB of weights: cut stream-K fashion, through a workspace
     A = inputs.bf16_integers((M, K), -8, 8, seed=1)
     Bt = tile_major_on_device(inputs.bf16_integers((K, N), -8, 8, seed=2), K, N, 16, 128)
     want = run_gemm(A, Bt, M, N, K, 16, 128)
+    assert tl.gemm_last_plan().stream_k == 1 and tl.gemm_last_plan().workspace_bytes > 0
     need = tl.gemm_workspace_bytes(M, N, K)
     assert need > 0
     ws = torch.empty(need, dtype=torch.uint8, device=DEV)
@@ -444,13 +445,14 @@ def test_products_on_two_streams_with_their_own_workspaces_match_serial_runs():
     # The header's rule for concurrent calls: each needs its own split-K workspace (the pointer travels with the
     # launch).  Two decode-shaped products on two streams, repeated, must give the bits of the serial runs.
     from gpu_util import DEV, tile_major_on_device, tl
-    shapes = [(8, 1280, 4096), (32, 2048, 2304)]                        # (M, N, K): both cut stream-K fashion
+    shapes = [(8, 1280, 8192), (32, 2304, 4608)]                        # (M, N, K): both cut stream-K fashion
     A, Bt, want, ws = [], [], [], []
     for i, (M, N, K) in enumerate(shapes):
         A.append(inputs.bf16_normal((M, K), 1.0, seed=40 + i).to(DEV))
         Bt.append(tile_major_on_device(inputs.bf16_normal((K, N), 0.02, seed=50 + i), K, N, 16, 128))
         C = torch.empty((M, N), dtype=torch.float32, device=DEV)
         tl.gemm(A[i], Bt[i], C, M, N, K, 4096, 16, 128)
+        assert tl.gemm_last_plan().stream_k == 1 and tl.gemm_last_plan().workspace_bytes > 0
         want.append(C)
         ws.append(torch.empty(tl.gemm_workspace_bytes(M, N, K) + 256, dtype=torch.uint8, device=DEV))
     tl.device_status()

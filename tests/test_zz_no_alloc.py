@@ -98,7 +98,9 @@ def test_large_products_that_need_no_scratch_are_not_refused():
 
 def test_refuses_scratch_beyond_the_fixed_array():
     from gpu_util import DEV, tl
-    M, N, K = 64, 1024, 4096                               # 2 * SMs * 64 * 128 * 4 bytes > 8 MiB on a B200
+    # 10 tiles of long K and 21 MB of weights: neither clusters nor whole tiles fill the SMs, so the K loops are cut over
+    # all of them and the partial tiles need 2 * SMs * 64 * 128 * 4 bytes > 8 MiB on a B200
+    M, N, K = 64, 1280, 8192
     A, Bt, _ = _case(M, N, K, seed=9, integer=True)
     C = torch.zeros((M, N), dtype=torch.float32, device=DEV)
     need = tl.gemm_workspace_bytes(M, N, K)
