@@ -43,6 +43,7 @@ struct DeviceState {
     size_t own_ws_bytes = 0;
     int sm_count = 0;
     int pair_max_clusters = -1;          // co-resident clusters of the CTA-pair kernel (queried once)
+    int cluster_cap[9] = {};             // co-resident clusters of S = 2..8 CTAs of the GEMM kernel (0: not queried yet)
     unsigned long long* d_grid_counter = nullptr;   // arrival counter of the expert FFN kernel's grid barrier (control block)
     unsigned long long grid_arrivals = 0;           // arrivals all launches so far will have made
     const void* smem_attr_done[64] = {}; // kernels whose dynamic shared-memory limit was raised on this device

@@ -253,18 +253,42 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
         // (large partial tiles: at most 4 CTAs per cluster, the exchange through distributed shared memory measured
         // slower than the stream-K cut beyond that)
         const int s_max = size_t(BM) * (BN + 4) * 4 > 40 * 1024 ? 4 : 8;
+        // every cluster of the launch must be resident at once (clusters live inside one GPC: 148 SMs hold 45 clusters of
+        // 3 CTAs but only 15 of 8); a second wave of clusters costs more than any other schedule
+        auto fits = [&](int s) -> bool {
+            int& cap = dev().cluster_cap[s];
+            if (cap == 0) {
+                int n = 0;
+                cap = gemm_max_active_clusters(s, &n) == TL_OK && n > 0 ? n : -1;
+            }
+            const int64_t limit = opt(TL_OPT_SM_LIMIT) > 0 && cap > 0 ? (int64_t(cap) * sms) / dev().sm_count : cap;
+            return cap > 0 && tile_bound <= limit;
+        };
         int best_s = 0;
         for (int s = 2; s <= s_max; ++s)
             if (tile_bound * s <= sms && tile_bound * s >= lo && k_iters >= s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024 &&
-                tile_bound * s > int64_t(best_s) * tile_bound)
+                tile_bound * s > int64_t(best_s) * tile_bound && fits(s))
                 best_s = s;
+        // Clusters that fill fewer SMs still beat the cut while the weights are few enough: c CTAs stream at about
+        // min(c x 65 GB/s, the device's 7.2 TB/s), the cut at the device's rate plus about 6 us for its partial tiles,
+        // its second kernel and the wake-up (29 to 92 MB of weights on 56 to 104 CTAs: 6 to 27 % faster than the cut).
+        if (g1 == 0 && best_s == 0) {
+            const int64_t bytes = total_iters * BK * BN * 2;
+            for (int s = s_max; s >= 2; --s) {
+                const int64_t c = tile_bound * s;
+                if (c > sms || k_iters < 2 * s || size_t(BM) * (BN + 4) * 4 > plan->smem_bytes - 1024 || !fits(s)) continue;
+                const int64_t rate = c * 65 < 7200 ? c * 65 : 7200;                 // GB/s = bytes per ns
+                if (bytes / rate <= bytes / 7200 + 6000) best_s = s;
+                break;                                                              // (the largest cluster that fits, or none)
+            }
+        }
         // Small problems (a few MB of weights: latency, not bandwidth) that fill neither: clusters all the same, however
         // few, as long as every CTA keeps at least two K iterations.  The cut would give each of many CTAs a single
         // iteration, a partial tile in global memory each, and a second kernel to add them.
         // (Qwen-3 attention projections, 128 to 512 tokens: k / v 13.7-16.9 -> 11.4-11.6 us, o at 128 tokens 17.9 -> 14.4 us)
         if (g1 == 0 && best_s == 0 && total_iters * BK * BN * 2 <= (int64_t(16) << 20))
             for (int s = s_max; s >= 2; --s)
-                if (tile_bound * s <= sms && k_iters >= 2 * s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024) {
+                if (tile_bound * s <= sms && k_iters >= 2 * s && size_t(BM) * (BN + 4) * 4 <= plan->smem_bytes - 1024 && fits(s)) {
                     best_s = s;
                     break;
                 }

@@ -1297,6 +1297,9 @@ int launch_gemm_wm_fp8(int bk, int bn, const cudaLaunchConfig_t* cfg, const Gemm
 int launch_gemm_chain(int bk, int bn, int grid, size_t smem, cudaStream_t stream, const GemmParams& p1,
                       const GemmParams& p2, unsigned long long* counter, unsigned long long target1,
                       unsigned long long target2, bool skip_cta0);
+// Clusters of `size` CTAs of the single-CTA GEMM kernel (one CTA per SM) that can be resident at the same time on the
+// current device: clusters live inside one GPC, so 148 SMs hold 45 clusters of 3 but only 15 of 8.
+int gemm_max_active_clusters(int size, int* out);
 // CTA-pair kernel (tl_gemm_pair.cu): halves = 2 for 512-token tiles.
 int launch_gemm_pair(bool fp8, int halves, int clusters, size_t smem, cudaStream_t stream, const GemmParams& p);
 // Clusters of the pair kernel that can be resident together on the current device.

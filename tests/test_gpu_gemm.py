@@ -416,7 +416,7 @@ def test_host_buffer_entry_point():
 
 def test_caller_workspace_and_errors():
     from gpu_util import DEV, run_gemm, tile_major_on_device, tl
-    M, N, K = 16, 2304, 8192               # 9 tiles of long K, 38 MB of weights: cut stream-K fashion, through a workspace
+    M, N, K = 16, 2304, 28672              # 9 tiles of long K, 132 MB of weights: cut stream-K fashion, through a workspace
     A = inputs.bf16_integers((M, K), -8, 8, seed=1)
     Bt = tile_major_on_device(inputs.bf16_integers((K, N), -8, 8, seed=2), K, N, 16, 128)
     want = run_gemm(A, Bt, M, N, K, 16, 128)
@@ -445,7 +445,7 @@ def test_products_on_two_streams_with_their_own_workspaces_match_serial_runs():
     # The header's rule for concurrent calls: each needs its own split-K workspace (the pointer travels with the
     # launch).  Two decode-shaped products on two streams, repeated, must give the bits of the serial runs.
     from gpu_util import DEV, tile_major_on_device, tl
-    shapes = [(8, 1280, 8192), (32, 2304, 4608)]                        # (M, N, K): both cut stream-K fashion
+    shapes = [(8, 1280, 28672), (32, 2304, 28672)]                      # (M, N, K): both cut stream-K fashion
     A, Bt, want, ws = [], [], [], []
     for i, (M, N, K) in enumerate(shapes):
         A.append(inputs.bf16_normal((M, K), 1.0, seed=40 + i).to(DEV))

@@ -125,9 +125,10 @@ def test_decode_switches_give_the_same_bits(opt_name, value, no_scratch):
 
 
 CLUSTER_CASES = [  # M, N, K, expected cluster size on a 148-SM part (0: some other schedule)
-    # (64 x 6144 x 512: too few tiles to fill the SMs with clusters, but only 6 MB of weights: clusters all the same)
-    (1, 8192, 8192, 4), (8, 10240, 8192, 3), (32, 8192, 28672, 4), (16, 4096, 1024, 8), (64, 6144, 512, 4),
-    (8, 5120, 64, 0), (40, 9472, 2048, 4), (8, 8192, 192, 0), (24, 57344, 1024, 0), (3, 18944, 3584, 2),
+    # (64 x 6144 x 512: too few tiles to fill the SMs with clusters, but only 6 MB of weights: clusters all the same;
+    #  16 tiles: 15 clusters of 8 CTAs can be resident, 22 of 6; 37 tiles: 33 clusters of 4, 45 of 3)
+    (1, 8192, 8192, 4), (8, 10240, 8192, 3), (32, 8192, 28672, 4), (16, 4096, 1024, 6), (64, 6144, 512, 4),
+    (8, 5120, 64, 0), (40, 9472, 2048, 3), (8, 8192, 192, 0), (24, 57344, 1024, 0), (3, 18944, 3584, 2),
     (8, 10112, 4096, 3),
 ]
 

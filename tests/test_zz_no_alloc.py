@@ -98,9 +98,9 @@ def test_large_products_that_need_no_scratch_are_not_refused():
 
 def test_refuses_scratch_beyond_the_fixed_array():
     from gpu_util import DEV, tl
-    # 10 tiles of long K and 21 MB of weights: neither clusters nor whole tiles fill the SMs, so the K loops are cut over
-    # all of them and the partial tiles need 2 * SMs * 64 * 128 * 4 bytes > 8 MiB on a B200
-    M, N, K = 64, 1280, 8192
+    # 5 tiles of very long K and 37 MB of weights: neither whole tiles nor clusters (at most 40 CTAs) are worth it, so the
+    # K loops are cut over all SMs and the partial tiles need 2 * SMs * 64 * 128 * 4 bytes > 8 MiB on a B200
+    M, N, K = 64, 640, 28672
     A, Bt, _ = _case(M, N, K, seed=9, integer=True)
     C = torch.zeros((M, N), dtype=torch.float32, device=DEV)
     need = tl.gemm_workspace_bytes(M, N, K)
