@@ -388,12 +388,12 @@ __device__ __forceinline__ void weight_box_coords(const GemmParams& p, int k, in
 // Memory tiles of br rows x 4 columns (8-byte rows) or br x 2 columns (4-byte rows), as the copy engine landed them:
 // the stage is an array of groups of 2 (or 4) tiles next to each other along N, 16 br bytes each, and a group covers br
 // rows x 8 columns.  A 16-byte chunk of a tile holds 2 (or 4) rows of its 4 (or 2) columns; the chunks at the same
-// place in the group's tiles hold the same rows.  One thread takes those 2 (or 4) chunks, and writes the 2 (or 4)
-// rows they contain, now 8 columns = 16 bytes wide, at row * 16 inside the same group: afterwards the group is a
-// br x 8 memory tile with 16-byte rows, i.e. br/8 core matrices of the no-swizzle MN-major operand, which the MMA
-// reads as it is.  In place: the threads of a group sit in one warp and all read before any of them writes.
-// 128 threads (tid 0..127) share the stage: kBK * kBN / 16 work items of 32 bytes (8-byte rows) or kBK * kBN / 32 of 64
-// bytes (4-byte rows), both multiples of 128; every item lies inside the stage's kBK * kBN * 2 bytes of weights.
+// place in the group's tiles hold the same rows.  Writing every row's 2 (or 4) pieces side by side at row * 16 inside
+// the same group turns it into a br x 8 memory tile with 16-byte rows, i.e. br/8 core matrices of the no-swizzle
+// MN-major operand, which the MMA reads as it is.  In place: a group is handled by one warp, which reads all of it
+// before it writes any of it.  8-byte rows: a thread takes the 2 chunks that hold the same row pair and writes 2 rows;
+// 4-byte rows: see below.  128 threads (tid 0..127) share the stage; every access lies inside the stage's
+// kBK * kBN * 2 bytes of weights.
 template <int kBK, int kBN>
 __device__ __forceinline__ void fixup_stage_in_place(uint8_t* sw, int br_log2, int bc_log2, int tid) {
     const uint32_t group_bytes = 16u << br_log2;
