@@ -116,6 +116,10 @@ typedef enum {
                                 MMA through a no-swizzle or K-major descriptor; 0: they take the permuting generic-address path */
     TL_OPT_PAIR_TMA_STORE,   /* 1 (default): the CTA-pair kernel writes C through shared memory with tiled bulk stores, 0: with
                                 plain stores straight from the accumulator registers (same values either way) */
+    TL_OPT_PLAN_AS_IF_SMS,   /* test hook, 0 (default) = off: n > 0 makes tl_gemm_plan answer as if the current device had n SMs,
+                                without asking the CUDA runtime anything (co-resident clusters of S CTAs: those of a B200 when
+                                n is 148, else n / S), so that the planning rules can be tested on a machine without a GPU.
+                                Launches refuse to run while it is set (TL_ERR_INVALID_ARG). */
     TL_OPT_COUNT_
 } tl_option;
 /* TL_ERR_INVALID_ARG for an unknown option or a value outside the option's range. */

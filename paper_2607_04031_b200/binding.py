@@ -68,7 +68,7 @@ _SIGNATURES = {
 # tl_option
 (OPT_PDL, OPT_PREFETCH_STAGES, OPT_PAIR_KERNEL, OPT_PAIR_512, OPT_BOX_PER_BLOCK, OPT_MAX_STAGES, OPT_UMMA_M128,
  OPT_RELAYOUT_TMA, OPT_LOG, OPT_WAIT_LIMIT_US, OPT_STALL_ONCE, OPT_MOE_ROW_CAP, OPT_REDUCE_SPLIT, OPT_SM_LIMIT,
- OPT_NO_SCRATCH_PLANS, OPT_FFN_ONE_LAUNCH, OPT_GENERIC_RAW, OPT_PAIR_TMA_STORE) = range(18)
+ OPT_NO_SCRATCH_PLANS, OPT_FFN_ONE_LAUNCH, OPT_GENERIC_RAW, OPT_PAIR_TMA_STORE, OPT_PLAN_AS_IF_SMS) = range(19)
 FLAVOUR_N_BF16, FLAVOUR_K_BF16, FLAVOUR_K_FP8 = 0, 1, 2
 
 _lib = None

@@ -64,6 +64,7 @@ ThreadState& tls() {
 }
 
 DeviceState& dev() {
+    if (opt(TL_OPT_PLAN_AS_IF_SMS)) return g_devices[0];        // test hook: see ensure_device_info
     int d = 0;
     if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) {
         (void)cudaGetLastError();
@@ -87,6 +88,16 @@ int check_cuda(cudaError_t err) {
 }
 
 int ensure_device_info() {
+    if (const int64_t fake = opt(TL_OPT_PLAN_AS_IF_SMS)) {      // test hook: no CUDA call at all
+        DeviceState& s = g_devices[0];
+        if (s.sm_count != int(fake)) {
+            s.sm_count = int(fake);
+            s.pair_max_clusters = int(fake) / 2;
+            static const int b200[9] = {0, 0, 74, 45, 33, 26, 22, 15, 15};
+            for (int c = 2; c <= 8; ++c) s.cluster_cap[c] = fake == 148 ? b200[c] : (int(fake) / c > 0 ? int(fake) / c : -1);
+        }
+        return TL_OK;
+    }
     int d = -1;
     if (int rc = check_cuda(cudaGetDevice(&d))) return rc;
     if (d < 0 || d >= kMaxDevices) return TL_ERR_UNSUPPORTED;
@@ -203,9 +214,16 @@ int tl_set_option(int option, int64_t value) {
         case TL_OPT_WAIT_LIMIT_US: if (value < 100 || value > 60000000) return TL_ERR_INVALID_ARG; break;
         case TL_OPT_STALL_ONCE: if (value < 0 || value > 4) return TL_ERR_INVALID_ARG; break;
         case TL_OPT_SM_LIMIT: if (value < 0 || value > 4096) return TL_ERR_INVALID_ARG; break;
+        case TL_OPT_PLAN_AS_IF_SMS: if (value < 0 || value > 4096) return TL_ERR_INVALID_ARG; break;
         case TL_OPT_MOE_ROW_CAP: if (value != 0 && value != 16 && value != 32 && value != 64 && value != 128) return TL_ERR_INVALID_ARG; break;
         case TL_OPT_FFN_ONE_LAUNCH: if (value < 0 || value > 2) return TL_ERR_INVALID_ARG; break;
         default: if (value != 0 && value != 1) return TL_ERR_INVALID_ARG; break;
+    }
+    if (option == TL_OPT_PLAN_AS_IF_SMS && tl::options().v[option] != value) {
+        // entering or leaving the hook: slot 0 forgets the SM count and the cluster numbers it held
+        tl::g_devices[0].sm_count = 0;
+        tl::g_devices[0].pair_max_clusters = -1;
+        for (int& c : tl::g_devices[0].cluster_cap) c = 0;
     }
     tl::options().v[option] = value;
     return TL_OK;

@@ -434,6 +434,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     }
     if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
     if (d_H_swiglu && !plan.weights_on_n) return TL_ERR_UNSUPPORTED;        // the gated epilogue pairs columns of one token row   // a K tail would read the next expert's rows
+    if (!plan_only && opt(TL_OPT_PLAN_AS_IF_SMS) != 0) return TL_ERR_INVALID_ARG;      // the planning test hook is on
     if (!fixed && !plan_only)
         if (int rc = ensure_control()) return rc;
 

@@ -1,4 +1,6 @@
 """Host-side arithmetic of the library that needs no GPU (CPU only)."""
+import pytest
+
 import oracle as tlo
 from paper_2607_04031_b200 import binding as tl
 
@@ -61,3 +63,84 @@ def test_tile_arrival_latency_rejects_bad_arguments():
     assert L.tl_tile_arrival_latency(None, 2, 4, 0.0, ctypes.byref(a), ctypes.byref(b), None) == 1
     bad = np.array([1.0, float("nan")])
     assert L.tl_tile_arrival_latency(bad.ctypes.data, 2, 4, 0.0, ctypes.byref(a), ctypes.byref(b), None) == 1
+
+
+# ---- the planning rules, asked as if the device were a 148-SM B200 (test hook: no CUDA call is made)
+
+def _plans_as_if(sms):
+    return tl.option(tl.OPT_PLAN_AS_IF_SMS, sms)
+
+
+def test_plans_of_the_benchmark_shapes_without_a_gpu():
+    with _plans_as_if(148):
+        # decode: schedules without partial tiles in global memory
+        p = tl.gemm_plan(8, 10240, 8192)                  # 40 tiles, clusters of 3 CTAs split K (45 such clusters fit)
+        assert p.cta == (16, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 3, 120, 0)
+        p = tl.gemm_plan(32, 8192, 28672)                 # 32 tiles, clusters of 4 (33 fit)
+        assert p.cta == (32, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 4, 128, 0)
+        p = tl.gemm_plan(1, 57344, 8192)                  # 224 whole tiles on 112 CTAs
+        assert p.cta == (16, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 1, 112, 0)
+        # prefill: CTA pairs, 512-token tiles in whole waves of 74 clusters, the rest as 256-token tiles
+        p = tl.gemm_plan(4096, 8192, 8192)
+        assert p.pair_kernel == 1 and p.cta == (512, 128, 64) and p.grid == 148
+        assert (p.pair_tiles_512, p.pair_tiles_256) == (222, 68) and p.workspace_bytes == 0
+        # Qwen expert products: short tiles, at least 64 m-tiles whatever the routing: whole tiles, nothing is cut
+        for N, K in ((1536, 2048), (2048, 768)):
+            p = tl.gemm_plan(2048, N, K, E=128)
+            assert p.cta == (32, 256, 64) and (p.stream_k, p.cluster_k, p.grid, p.workspace_bytes) == (0, 1, 148, 0)
+    assert tl.get_option(tl.OPT_PLAN_AS_IF_SMS) == 0
+
+
+def test_cluster_plans_respect_how_many_clusters_can_be_resident():
+    with _plans_as_if(148):
+        # 16 tiles: 16 clusters of 8 CTAs would fill 128 SMs, but only 15 can be resident at once: 6 CTAs per cluster
+        assert tl.gemm_plan(16, 4096, 1024).cluster_k == 6
+        # 37 tiles: 33 clusters of 4 fit, 45 of 3
+        p = tl.gemm_plan(40, 9472, 2048)
+        assert (p.cluster_k, p.grid) == (3, 111)
+        # 18 tiles x 8 = 144 CTAs does not fit either
+        p = tl.gemm_plan(8, 4608, 4096)
+        assert (p.stream_k, p.cluster_k, p.grid) == (0, 6, 108)
+    with _plans_as_if(64):                                # a smaller part: 64 / S clusters of S CTAs
+        p = tl.gemm_plan(8, 2048, 8192)                   # 8 tiles x 8 CTAs = 64
+        assert (p.stream_k, p.cluster_k, p.grid) == (0, 8, 64)
+
+
+def test_when_the_k_loops_are_cut_over_all_sms():
+    with _plans_as_if(148):
+        # few tiles of very long K and many bytes: neither whole tiles nor under-filled clusters are worth it
+        p = tl.gemm_plan(16, 2304, 28672)
+        assert (p.stream_k, p.cluster_k, p.grid) == (1, 1, 148) and p.workspace_bytes == 2 * 148 * 16 * 256 * 4
+        # the same tiles with fewer bytes: clusters, although they fill only 72 SMs
+        p = tl.gemm_plan(16, 2304, 8192)
+        assert (p.stream_k, p.cluster_k, p.grid) == (0, 8, 72)
+        # a few MB of weights: clusters, however few
+        p = tl.gemm_plan(256, 512, 2048)
+        assert (p.stream_k, p.cluster_k, p.grid, p.cta) == (0, 4, 32, (128, 128, 128))
+        # grouped: too few rows for the host to rule the cut out (the kernel decides from the tile count); long tiles
+        assert tl.gemm_plan(64, 1536, 2048, E=128).stream_k == 1
+        assert tl.gemm_plan(2048, 2048, 8192, E=128).stream_k == 1
+        # with the no-scratch schedules switched off: always the cut
+        with tl.option(tl.OPT_NO_SCRATCH_PLANS, 0):
+            p = tl.gemm_plan(8, 10240, 8192)
+            assert (p.stream_k, p.cluster_k, p.grid) == (1, 1, 148)
+
+
+def test_weight_paths_by_memory_tile_shape():
+    with _plans_as_if(148):
+        path = lambda br, bc, cta=(0, 0, 0): tl.gemm_plan(16, 8192, 8192, br * bc * 2, br, bc, cta).generic_path
+        assert path(16, 128) == 0 and path(32, 16) == 0 and path(16, 32) == 0           # TMA boxes
+        assert path(16, 8) == 2 and path(8, 8) == 2 and path(64, 8) == 2                 # 16-byte rows: as stored
+        assert path(16, 1) == 2 and path(8, 1) == 2 and path(128, 1) == 2                # single-column tiles: K-major panels
+        assert path(32, 4) == 3 and path(8, 2) == 3 and path(8, 4) == 3                  # 8- and 4-byte rows: in place
+        assert path(64, 4) == 3 and path(64, 2) == 3 and path(128, 2, (32, 128, 128)) == 3
+        with pytest.raises(tl.TileLensError):                                             # a 128-row tile does not fit 64-row stages
+            path(128, 2)
+        assert path(4, 8) == 1 and path(4, 4) == 1                                        # fewer than 8 rows: permuted
+        with tl.option(tl.OPT_GENERIC_RAW, 0):
+            assert path(16, 8) == 1 and path(32, 4) == 1 and path(16, 1) == 1
+
+
+def test_launches_are_refused_while_the_planning_hook_is_on():
+    with _plans_as_if(148):
+        assert tl.lib().tl_gemm(1 << 12, 1 << 13, 1 << 14, 16, 512, 512, 4096, 16, 128, 0, 0, 0, None) == 1
