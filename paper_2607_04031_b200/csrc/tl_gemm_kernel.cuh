@@ -400,27 +400,35 @@ __device__ __forceinline__ void fixup_stage_in_place(uint8_t* sw, int br_log2, i
     // (kBatch work items have their loads in flight together: all reads, then all writes)
     if (bc_log2 == 2) {
         constexpr int kItems = kBK * kBN / 16;
-        constexpr int kBatch = kItems >= 512 ? 4 : kItems / 128;
+        constexpr int kBatch = kItems >= 1024 ? 8 : (kItems >= 512 ? 4 : kItems / 128);
         static_assert(kItems % (128 * kBatch) == 0, "whole batches");
         const int tpg_log2 = br_log2 - 1;                          // threads per group: one per pair of rows
         const uint32_t tile_bytes = 8u << br_log2;
-        for (int item0 = tid; item0 < kItems; item0 += 128 * kBatch) {
-            uint4 a[kBatch], b[kBatch];
-            uint8_t* dst[kBatch];
+        // Item i writes rows 2i and 2i+1 of the finished image, 32 bytes at i * 32.  Of every eight lanes four write their
+        // second row first, so that the eight 16-byte stores of a quarter warp fall into eight different bank groups
+        // (stores 32 bytes apart would pair up).  Those lanes fetch the two 8-byte halves of each chunk in the other
+        // order, so the rows come out of the loads in the order they are stored and no register has to be picked;
+        // which lanes: such that lanes l and l + 8 differ, which keeps the sixteen 8-byte loads of a half warp apart too.
+        const uint32_t hi_first = ((uint32_t(tid) >> 2) ^ (uint32_t(tid) >> 3)) & 1u;
+        const uint32_t src0 = (uint32_t(tid) >> tpg_log2) * group_bytes + (uint32_t(tid) & ((1u << tpg_log2) - 1)) * 16u;
+        const uint32_t h0 = hi_first * 8u, h1 = 8u - h0;
+        // (128 items further = 4096 bytes further: a group of br / 2 items is 16 br bytes)
+        for (int it = 0; it < kItems / (128 * kBatch); ++it) {
+            uint2 a0[kBatch], a1[kBatch], b0[kBatch], b1[kBatch];
 #pragma unroll
             for (int j = 0; j < kBatch; ++j) {
-                const int item = item0 + j * 128;
-                const int g = item >> tpg_log2, q = item & ((1 << tpg_log2) - 1);
-                uint8_t* base = sw + size_t(g) * group_bytes;
-                a[j] = *reinterpret_cast<const uint4*>(base + q * 16);                // rows 2q, 2q+1 x columns 0..3
-                b[j] = *reinterpret_cast<const uint4*>(base + tile_bytes + q * 16);   //                x columns 4..7
-                dst[j] = base + q * 32;
+                const uint8_t* src = sw + src0 + uint32_t(it * kBatch + j) * 4096u;
+                a0[j] = *reinterpret_cast<const uint2*>(src + h0);                // one row x columns 0..3
+                a1[j] = *reinterpret_cast<const uint2*>(src + h1);                // the other row
+                b0[j] = *reinterpret_cast<const uint2*>(src + tile_bytes + h0);   // x columns 4..7
+                b1[j] = *reinterpret_cast<const uint2*>(src + tile_bytes + h1);
             }
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < kBatch; ++j) {
-                *reinterpret_cast<uint4*>(dst[j]) = make_uint4(a[j].x, a[j].y, b[j].x, b[j].y);
-                *reinterpret_cast<uint4*>(dst[j] + 16) = make_uint4(a[j].z, a[j].w, b[j].z, b[j].w);
+                uint8_t* dst = sw + size_t(tid + (it * kBatch + j) * 128) * 32;
+                *reinterpret_cast<uint4*>(dst + 2 * h0) = make_uint4(a0[j].x, a0[j].y, b0[j].x, b0[j].y);
+                *reinterpret_cast<uint4*>(dst + 2 * h1) = make_uint4(a1[j].x, a1[j].y, b1[j].x, b1[j].y);
             }
         }
     } else {
