@@ -126,6 +126,20 @@ def test_when_the_k_loops_are_cut_over_all_sms():
             assert (p.stream_k, p.cluster_k, p.grid) == (1, 1, 148)
 
 
+def test_the_reported_workspace_covers_every_plan():
+    # tl_gemm_workspace_bytes is what a caller sizes its own workspace from: never less than the plan of that call
+    with _plans_as_if(148):
+        seen = 0
+        for M in (1, 8, 16, 32, 48, 64, 100, 128, 256, 700, 4096):
+            for N in (256, 1280, 2304, 8192, 10240, 57344):
+                for K in (64, 512, 2048, 8192, 28672):
+                    plan = tl.gemm_plan(M, N, K)
+                    assert tl.gemm_workspace_bytes(M, N, K) >= plan.workspace_bytes, (M, N, K)
+                    assert (plan.workspace_bytes > 0) == (plan.stream_k == 1), (M, N, K)
+                    seen += plan.stream_k
+        assert seen > 0                                   # the cut is among the schedules looked at
+
+
 def test_weight_paths_by_memory_tile_shape():
     with _plans_as_if(148):
         path = lambda br, bc, cta=(0, 0, 0): tl.gemm_plan(16, 8192, 8192, br * bc * 2, br, bc, cta).generic_path
