@@ -20,10 +20,18 @@ def _pick(rng, xs):
     return xs[int(rng.integers(0, len(xs)))]
 
 
-def _case(rng):
-    flavour = _pick(rng, ["n", "n", "k", "fp8"])
+# memory tiles with rows of 16 bytes and less: read as stored, transposed in place, K-major panels, or permuted
+NARROW = [(8, 8), (16, 8), (32, 8), (64, 8), (128, 8), (8, 4), (16, 4), (32, 4), (64, 4), (8, 2), (16, 2), (32, 2), (64, 2),
+          (128, 2), (8, 1), (16, 1), (32, 1), (64, 1), (128, 1), (4, 8), (4, 4), (2, 8), (4, 16)]
+
+
+def _case(rng, narrow=False):
+    flavour = "n" if narrow else _pick(rng, ["n", "n", "k", "fp8"])
     s = 1 if flavour == "fp8" else 2
-    if flavour == "n":
+    if narrow:
+        br, bc = _pick(rng, NARROW)
+        k_unit, n_unit = max(br, 64), 64
+    elif flavour == "n":
         br, bc = _pick(rng, [(0, 0), (1, 256), (2, 128), (4, 64), (8, 64), (16, 128), (32, 64), (64, 32), (128, 16), (16, 16),
                              (8, 8), (32, 4), (2, 1024), (64, 64), (8, 512)])
         k_unit, n_unit = max(br, 64), max(bc, 64)
@@ -44,9 +52,19 @@ def _case(rng):
 
 @pytest.mark.parametrize("seed", range(160))
 def test_random_configuration_is_exact(seed):
-    from gpu_util import DEV, tl
     rng = np.random.default_rng(1000 + seed)
-    flavour, s, br, bc, M, N, K, cta = _case(rng)
+    _run(seed, rng, _case(rng))
+
+
+@pytest.mark.parametrize("seed", range(120))
+def test_random_narrow_tile_configuration_is_exact(seed):
+    rng = np.random.default_rng(5000 + seed)
+    _run(seed, rng, _case(rng, narrow=True))
+
+
+def _run(seed, rng, case):
+    from gpu_util import DEV, tl
+    flavour, s, br, bc, M, N, K, cta = case
     G = br * bc * s
     if flavour == "fp8":
         A = inputs.fp8_integers((M, K), -6, 6, seed=seed)
