@@ -480,6 +480,40 @@ def run_ours(args):
     row_t = sum(x["us"] for x in per_shape if x["layout"] == "row")
     extra["tile_vs_row_time_ratio_decode"] = tile_t / row_t
 
+    # ---- the twelve products captured once into a CUDA graph and replayed, next to the same calls issued directly
+    # (alternating, so that both see the same clocks).  The kernels and their programmatic dependencies are the same;
+    # what a replay saves is the host's launch work between them.
+    with sampler.window("decode_cuda_graph"):
+        try:
+            def gemms12():
+                for M in inputs.LLAMA_DECODE_M:
+                    for name, K, N in inputs.LLAMA70B_PROJ:
+                        tl.gemm(A_dec[name, M], W_tile[name], C_dec[name, M], M, N, K, G, BR, BC)
+
+            gemms12()
+            torch.cuda.synchronize()
+            graph12 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph12):
+                gemms12()
+            evs = {"direct": [], "graph": []}
+            for rep_ in range(21):
+                for kind, fn in (("direct", gemms12), ("graph", graph12.replay)):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    fn()
+                    b.record()
+                    if rep_ > 0:
+                        evs[kind].append((a, b))
+            torch.cuda.synchronize()
+            tl.device_status()
+            med = {k: statistics.median(a.elapsed_time(b) for a, b in v) for k, v in evs.items()}
+            extra["decode_cuda_graph"] = {"direct_us": med["direct"] * 1e3, "graph_us": med["graph"] * 1e3,
+                                          "graph_GBps": gemm_step_bytes / (med["graph"] * 1e-3) / 1e9,
+                                          "note": "the step's 12 decode products back to back: direct calls and one replayed graph"}
+            del graph12
+        except Exception as exc:  # report, never hide
+            extra["decode_cuda_graph"] = {"error": f"{type(exc).__name__}: {exc}"}
+
     # ---- the same twelve products as three independent decode batches on three streams (one per batch size, own
     # split-K workspace each): CTAs of one product fill the SMs that the tail of another leaves free.  Reported
     # beside the step, not as the step: inside one decode loop the products depend on each other.

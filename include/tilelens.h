@@ -28,6 +28,16 @@
  *     and the workspace set by tl_set_stream() / tl_set_workspace() belong to the calling thread, like CUDA's
  *     current device; the internal split-K workspace belongs to the device, so calls that can run at the same
  *     time on one GPU (two streams, two threads) must each bring their own workspace.
+ *   - Stream capture.  Every call that only enqueues work (the relayouts, the device-buffer products, tl_moe_ffn,
+ *     tl_read_amp_async / tl_read_amp_batch, tl_hw_*) may be issued on a stream that is being captured into a CUDA
+ *     graph, and the graph replays the same launches with the same bits: nothing a launch needs lives in host state
+ *     that a replay would miss.  Two conditions.  The library's first use of a device, a kernel or a problem shape
+ *     allocates and configures (control block, shared-memory attributes, tensor maps), which a capture forbids: make
+ *     the same calls once before capturing.  And a captured launch whose schedule needs split-K scratch takes it only
+ *     from the calling thread's workspace (tl_set_workspace), which must then live as long as the graph; without one
+ *     it returns TL_ERR_WORKSPACE, because the internal workspace is replaced when a later call needs a larger one.
+ *     tl_moe_ffn always runs as two launches while its stream is being captured.  tl_gemm_host, tl_read_amp and
+ *     tl_device_status synchronise and are not for capture.
  *   - Divisibility (Section 3.3): rows % block_rows == 0 and
  *     cols % block_cols == 0, otherwise TL_ERR_INVALID_ARG; the caller pads.
  *     block_rows and block_cols must be powers of two (Section 3.2), otherwise
@@ -50,7 +60,7 @@ typedef enum {
     TL_ERR_ALIGNMENT = 3,     /* pointer or pitch not aligned as the call requires */
     TL_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed: see tl_last_cuda_error() */
     TL_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired, or a kernel refused an input (detail code) */
-    TL_ERR_WORKSPACE = 6      /* caller-supplied workspace too small */
+    TL_ERR_WORKSPACE = 6      /* caller-supplied workspace too small (or none, for a captured launch that needs scratch) */
 } tl_status;
 
 typedef enum { TL_TO_TILE_MAJOR = 0, TL_TO_ROW_MAJOR = 1 } tl_direction;

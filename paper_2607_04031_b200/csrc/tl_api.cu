@@ -138,7 +138,16 @@ int ensure_smem_attr(const void* kernel, int bytes) {
     return TL_OK;
 }
 
-int get_workspace(size_t bytes, void** out) {
+bool stream_is_capturing(cudaStream_t stream) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return true;                                      // a capture gone wrong: treat like one in progress
+    }
+    return st != cudaStreamCaptureStatusNone;
+}
+
+int get_workspace(size_t bytes, void** out, cudaStream_t stream) {
     if (bytes == 0) {
         *out = nullptr;
         return TL_OK;
@@ -149,6 +158,9 @@ int get_workspace(size_t bytes, void** out) {
         *out = t.user_ws;
         return TL_OK;
     }
+    // A captured launch would keep this address in its graph, while the internal buffer is replaced whenever a later
+    // call needs a larger one (and growing it synchronises and allocates, which a capture forbids).
+    if (stream_is_capturing(stream)) return TL_ERR_WORKSPACE;
     DeviceState& s = dev();
     if (s.own_ws_bytes < bytes) {
         // Work already enqueued may still use the old buffer: wait before replacing it.

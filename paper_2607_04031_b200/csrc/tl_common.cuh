@@ -77,7 +77,10 @@ int ensure_device_info();
 // Raises the dynamic shared-memory limit of `kernel` on the current device, once per (device, kernel).
 int ensure_smem_attr(const void* kernel, int bytes);
 // Workspace of at least `bytes` (the calling thread's if set, else the device's internal one, grown with cudaMalloc).
-int get_workspace(size_t bytes, void** out);
+// While `stream` is being captured only the calling thread's workspace is handed out (TL_ERR_WORKSPACE otherwise).
+int get_workspace(size_t bytes, void** out, cudaStream_t stream);
+// True while `stream` is being captured into a CUDA graph.
+bool stream_is_capturing(cudaStream_t stream);
 // Wait limit of the kernels' bounded waits, nanoseconds (TL_OPT_WAIT_LIMIT_US).
 uint64_t wait_limit_ns();
 

@@ -846,7 +846,7 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (fixed) {
         if (plan.ws_bytes > fixed->ws_bytes) return TL_ERR_WORKSPACE;
         ws = plan.ws_bytes ? fixed->ws : nullptr;
-    } else if (int rc = get_workspace(plan.ws_bytes, &ws)) {
+    } else if (int rc = get_workspace(plan.ws_bytes, &ws, stream)) {
         return rc;
     }
     p.partials = static_cast<float*>(ws);
@@ -1005,7 +1005,9 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
     if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
     if (!d_H_bf16) return TL_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (total_rows > 0 && tl::opt(TL_OPT_FFN_ONE_LAUNCH) != 0) {
+    // (Not while the stream is being captured: the barrier form counts arrivals from a base the host keeps, which a
+    // replayed graph would not advance.)
+    if (total_rows > 0 && tl::opt(TL_OPT_FFN_ONE_LAUNCH) != 0 && !tl::stream_is_capturing(stream)) {
         // Both products in one cooperative launch (tl_gemm_chain.cu) when they share the kernel instantiation and the
         // grid: TMA-readable weights, the default grouped tile, the stream-K schedule.  Otherwise two launches.
         tl::GemmParams p1, p2;
@@ -1032,7 +1034,7 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
             const size_t n_flags = size_t(total_rows / plan1.BM) + size_t(E) + 1;
             const size_t ws_bytes = part_bytes + n_flags * sizeof(uint32_t);
             void* ws = nullptr;
-            if ((rc = tl::get_workspace(ws_bytes, &ws))) return rc;
+            if ((rc = tl::get_workspace(ws_bytes, &ws, stream))) return rc;
             uint32_t* flags = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + part_bytes);
             if ((rc = tl::check_cuda(cudaMemsetAsync(flags, 0, n_flags * sizeof(uint32_t), stream)))) return rc;
             p1.partials = nullptr;
@@ -1064,7 +1066,7 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
             // before the second one writes its own)
             const size_t ws_bytes = size_t(2) * size_t(grid) * plan1.BM * plan1.BN * sizeof(float);
             void* ws = nullptr;
-            if ((rc = tl::get_workspace(ws_bytes, &ws))) return rc;
+            if ((rc = tl::get_workspace(ws_bytes, &ws, stream))) return rc;
             p1.partials = p2.partials = static_cast<float*>(ws);
             const unsigned long long base = d.grid_arrivals;
             const size_t smem = plan1.smem_bytes > plan2.smem_bytes ? plan1.smem_bytes : plan2.smem_bytes;
