@@ -480,6 +480,35 @@ def run_ours(args):
     row_t = sum(x["us"] for x in per_shape if x["layout"] == "row")
     extra["tile_vs_row_time_ratio_decode"] = tile_t / row_t
 
+    # ---- between decode and prefill: the same four weights at 128 and 256 token rows (one launch per event pair; the
+    # four weights rotate, 1.7 GB between two uses of the same one)
+    mid = []
+    with sampler.window("mid_batch"):
+        for M in (128, 256):
+            A_mid = {K: inputs.bf16_normal((M, K), 1.0, seed=700 + M + K // 1024, device=str(dev))
+                     for K in sorted({K for _, K, _ in inputs.LLAMA70B_PROJ})}
+            C_mid = {N: torch.empty((M, N), dtype=torch.float32, device=dev) for N in sorted({N for _, _, N in inputs.LLAMA70B_PROJ})}
+            evs = {name: [] for name, _, _ in inputs.LLAMA70B_PROJ}
+            for rep_ in range(6):
+                for name, K, N in inputs.LLAMA70B_PROJ:
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    tl.gemm(A_mid[K], W_tile[name], C_mid[N], M, N, K, G, BR, BC)
+                    b.record()
+                    if rep_ > 0:
+                        evs[name].append((a, b))
+            torch.cuda.synchronize()
+            for name, K, N in inputs.LLAMA70B_PROJ:
+                med = statistics.median(a.elapsed_time(b) for a, b in evs[name])
+                pl = tl.gemm_plan(M, N, K, G, BR, BC)
+                mid.append({"proj": name, "M": M, "us": med * 1e3, "GBps": gemm_bytes(M, N, K) / (med * 1e-3) / 1e9,
+                            "TFLOPs": 2.0 * M * N * K / (med * 1e-3) / 1e12, "cta": list(pl.cta),
+                            "schedule": "stream-K" if pl.stream_k else f"clusters of {pl.cluster_k}" if pl.cluster_k > 1
+                            else f"whole tiles on {pl.grid} CTAs"})
+            del A_mid, C_mid
+    extra["llama_mid_batch"] = mid
+    tl.device_status()
+
     # ---- the twelve products captured once into a CUDA graph and replayed, next to the same calls issued directly
     # (alternating, so that both see the same clocks).  The kernels and their programmatic dependencies are the same;
     # what a replay saves is the host's launch work between them.

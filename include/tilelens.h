@@ -184,7 +184,10 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
  *   d_C          device, 16-byte aligned, M*N floats, fully overwritten.
  *   cta_m/n/k    the CTA tile: cta_m token rows x cta_n weight columns per CTA,
  *                cta_k weight rows per pipeline stage.  0,0,0 lets the library
- *                choose.  Instantiated: cta_n in {64, 128, 256}, cta_k in {64, 128},
+ *                choose (by M: M x 256 x 64 up to 64 rows, 128 x 128 x 128 or
+ *                128 x 256 x 64 up to 512 rows, whichever its planner ranks
+ *                ahead for the shape, CTA pairs on 256- or 512-row tiles for
+ *                prefill; tl_gemm_plan() tells).  Instantiated: cta_n in {64, 128, 256}, cta_k in {64, 128},
  *                cta_m in {16, 32, 64, 128, 256} (cta_n == 256: at most 128).
  *                Tiles may overhang M, N and K.
  *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,

@@ -156,6 +156,7 @@ static int pick_bm(int64_t rows) {
 //                      hand-offs
 //   more rows          256 x 128 x 64 with the weights on the M side (prefill) when there are enough tiles for the
 //                      CTA-pair kernel, else 128 x 128 x 128
+//   65 to 512 rows     dense products on TMA-readable weights may take 128 x 256 x 64 instead (gemm_launch ranks the two)
 //   grouped            at most 32 rows per tile (x 256 x 64): most experts have a handful of rows; caps of 64 and 128
 //                      rows measured the same within 2 % on the Qwen-3 expert products (fewer passes over an
 //                      expert's weights against fewer, larger pipeline stages)
@@ -333,6 +334,27 @@ struct FixedScratch {
     uint32_t* status;    // word the kernel raises when a bounded wait expires
 };
 
+// Rough time of a dense weights-on-N plan, for choosing between the 128- and the 256-column tile at 65 to 512 token
+// rows (K in 2-byte units).  What one CTA pulls into shared memory at about 90 GB/s (measured 75-105: weight slabs and
+// the token rows that come with each, most of them L2 hits), not faster than HBM delivers the weights once; plus the
+// exchange of partial tiles inside a cluster (about 6 us for 128 KB tiles, 3 us for 64 KB), 12 us for the partial
+// tiles and the second kernel of a stream-K cut, and a fixed 8 us.  Fitted to Llama-70B and Qwen-3 shapes at 96-512 rows; it only has to rank two plans.
+static double mid_tile_estimate_us(const GemmPlan& pl, int64_t rows, int64_t N, int64_t K) {
+    const double tiles = double(ceil_div(rows, pl.BM)) * double(ceil_div(N, pl.BN));
+    const double k_iters = double(ceil_div(K, pl.BK));
+    const double stage = double(pl.BK) * pl.BN * 2 + double(pl.BK) * pl.a_rows * 2;
+    double iters;                                           // K iterations of the busiest CTA
+    if (pl.stream_k) iters = tiles * k_iters / pl.grid;
+    else if (pl.cluster_k > 1) iters = double(ceil_div(int64_t(k_iters), pl.cluster_k));
+    else iters = double(ceil_div(int64_t(tiles), pl.grid)) * k_iters;
+    double us = iters * stage / 90e3;                       // 90 GB/s = 90e3 bytes per us
+    const double hbm = double(N) * double(K) * 2 / 5.8e6;   // 5.8 TB/s with token rows in the way
+    if (hbm > us) us = hbm;
+    if (pl.cluster_k > 1) us += double(pl.BM) * pl.BN * 4 / 65536 * 3.0;
+    if (pl.stream_k) us += 12.0;
+    return us + 8.0;
+}
+
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
                        int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
@@ -399,6 +421,33 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (int rc = ensure_device_info()) return rc;
     // enough 256 x 256 tiles for every cluster of the CTA-pair kernel to get one
     const bool pair_sized = ceil_div(rows_total, 256) * ceil_div(N, 256) * 2 >= dev().sm_count;
+    // Dense products of 65 to 512 token rows on TMA-readable weights are bound by what one SM can pull out of L2: a
+    // 128-row token slab comes with every weight slab, and with 128 weight columns per tile it is half of all bytes
+    // (Llama gate_up at 128 tokens: 190 us).  Twice the columns per tile (128 x 256 x 64) make it a third (167 us),
+    // but halve the number of tiles.  The wider tile is taken where it has a schedule without partial tiles in global
+    // memory (they are 128 KB each: down at 384 tokens, K cut over all CTAs, 213 us with the narrow tile against 289)
+    // and mid_tile_estimate_us says it is ahead.  Where the default would be the CTA-pair kernel: up to 384 rows the
+    // wide tile (gate_up at 256 tokens 255 against 308 us), beyond that the pair kernel.
+    if (cta_m == 0 && cta_n == 0 && cta_k == 0 && !d_offsets && !fixed && !generic && rows_max > 64 && rows_max <= 512 &&
+        !(rows_max > 384 && pair_sized)) {
+        GemmPlan wide, other;
+        if (make_plan(rows_max, ceil_div(rows_total, 128) * ceil_div(N, 256), N, K >> k_shift, 128, 256, 64, false, &wide,
+                      false, false, pair_sized, rows_total) == TL_OK &&
+            wide.stream_k == 0) {
+            int bm = 0, bn = 0, bk = 0;
+            default_tile(rows_max, false, false, &bm, &bn, &bk, pair_sized);
+            bool take = bm > 128;                           // against the pair kernel
+            if (!take && make_plan(rows_max, ceil_div(rows_total, bm) * ceil_div(N, bn), N, K >> k_shift, 0, 0, 0, false,
+                                   &other, false, false, pair_sized, rows_total) == TL_OK)
+                take = mid_tile_estimate_us(wide, rows_total, N, K >> k_shift) <
+                       0.97 * mid_tile_estimate_us(other, rows_total, N, K >> k_shift);
+            if (take) {
+                cta_m = 128;
+                cta_n = 256;
+                cta_k = 64;
+            }
+        }
+    }
     GemmPlan plan;
     {
         // upper bound of tiles: every expert may add one ragged m-tile

@@ -26,6 +26,24 @@ def _int_case(M, N, K, br, bc, seed):
     return A, Bd, want
 
 
+@pytest.mark.parametrize("M,N,K,want_plan", [
+    (128, 256 * 112, 512, ((128, 256, 64), 0, 1, 112)),       # whole wide tiles on 112 CTAs
+    (200, 10240, 4608, ((128, 128, 128), 1, 1, 148)),         # 80 wide tiles would have to be cut: the narrow tile (also cut)
+    (100, 10240, 4096, ((128, 256, 64), 0, 3, 120)),          # 40 wide tiles, split-K in clusters of 3
+    (300, 4096, 4096, ((128, 256, 64), 0, 2, 96)),            # 48 wide tiles in clusters of 2 against a cut of the narrow ones
+    (256, 512, 2048, ((128, 128, 128), 0, 4, 32)),            # small weights: the narrow tile
+])
+def test_products_between_decode_and_prefill_are_exact_on_the_tile_the_library_picks(M, N, K, want_plan):
+    from gpu_util import run_gemm, tl
+    A, Bd, want = _int_case(M, N, K, 16, 128, seed=M + N)
+    got = run_gemm(A, Bd, M, N, K, 16, 128)
+    p = tl.gemm_last_plan()
+    assert (p.cta, p.stream_k, p.cluster_k, p.grid) == want_plan, p.as_dict()
+    assert torch.equal(got.cpu(), want)
+    for cta in ((128, 256, 64), (128, 128, 128)):             # and both candidates give the same bits (exact integers)
+        assert torch.equal(run_gemm(A, Bd, M, N, K, 16, 128, cta).cpu(), want)
+
+
 def test_one_box_per_memory_tile_gives_the_same_bits():
     from gpu_util import run_gemm, tl
     M, N, K = 40, 1024, 1024
@@ -82,7 +100,7 @@ def test_prefill_switches_give_the_exact_product(opt_name, value):
         assert plan.pair_kernel == 1 and plan.pair_tiles_512 > 0 and plan.pair_tiles_256 > 0
 
 
-@pytest.mark.parametrize("M,N,K", [(700, 9600, 320), (1800, 5120, 384), (257, 256 * 74, 64)])
+@pytest.mark.parametrize("M,N,K", [(700, 9600, 320), (1800, 5120, 384), (385, 256 * 74, 64)])
 def test_pair_kernel_store_paths_write_the_same_bits(M, N, K):
     # C through shared memory and tiled bulk stores (default) against plain stores from the accumulator registers:
     # fp32 and bf16 C, ragged rows and columns, nothing outside C touched (guard blocks on both sides).

@@ -126,6 +126,31 @@ def test_when_the_k_loops_are_cut_over_all_sms():
             assert (p.stream_k, p.cluster_k, p.grid) == (1, 1, 148)
 
 
+def test_tile_of_dense_products_between_decode_and_prefill():
+    with _plans_as_if(148):
+        plan = lambda M, N, K: tl.gemm_plan(M, N, K)
+        # enough tiles either way: 256 weight columns per tile halve the share of token rows in what an SM loads
+        p = plan(128, 57344, 8192)
+        assert (p.cta, p.stream_k, p.cluster_k, p.grid) == ((128, 256, 64), 0, 1, 112)
+        p = plan(128, 10240, 8192)                        # 40 wide tiles in clusters of 3; the narrow tile would be cut
+        assert (p.cta, p.stream_k, p.cluster_k, p.grid) == ((128, 256, 64), 0, 3, 120)
+        # 256 rows, where the default would be the CTA-pair kernel: the wide tile up to 384 rows
+        p = plan(256, 57344, 8192)
+        assert (p.cta, p.pair_kernel, p.stream_k) == ((128, 256, 64), 0, 0)
+        p = plan(512, 57344, 8192)
+        assert p.pair_kernel == 1
+        # small weights: more, smaller tiles win (latency, not bandwidth)
+        assert plan(128, 512, 2048).cta == (128, 128, 128) and plan(256, 4096, 2048).cta == (128, 128, 128)
+        # the wide tile only where it needs no partial tiles in global memory
+        p = plan(384, 8192, 28672)
+        assert (p.cta, p.stream_k) == ((128, 128, 128), 1)
+        # a cut of the narrow tile against clusters of the wide one
+        p = plan(384, 4096, 4096)
+        assert (p.cta, p.stream_k, p.cluster_k) == ((128, 256, 64), 0, 2)
+        # decode and prefill sizes are not touched
+        assert plan(64, 57344, 8192).cta == (64, 256, 64) and plan(4096, 8192, 8192).pair_kernel == 1
+
+
 def test_the_reported_workspace_covers_every_plan():
     # tl_gemm_workspace_bytes is what a caller sizes its own workspace from: never less than the plan of that call
     with _plans_as_if(148):
