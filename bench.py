@@ -697,7 +697,24 @@ def run_ours(args):
     ffn_bytes = active * 2 * (hid * 2 * inter + inter * hid) + 2 * rows * hid + 2 * 2 * rows * inter + 4 * rows * hid
     moe.append({"proj": "expert_ffn_chain", "layout": "tile", "us": ms * 1e3, "GBps": ffn_bytes / (ms * 1e-3) / 1e9,
                 "active_experts": active, "note": "tl_moe_ffn: grouped gate_up + silu*mul epilogue -> bf16 h -> grouped down"})
-    del Wgu_t, Wdn_t, Xm, Hm, Ym
+    del Xm, Hm, Ym
+    # the same expert FFN with more tokens routed the same way (64 and 256 rows per expert on average): the grouped
+    # tile grows with the rows per expert
+    for tokens_big in (1024, 4096):
+        off_b, cnt_b, _ = inputs.zipf_topk_routing(tokens_big, q["experts"], q["topk"], q["zipf_alpha"], seed=0)
+        rows_b, act_b = int(off_b[-1]), int((cnt_b > 0).sum())
+        d_off_b = torch.from_numpy(off_b).to(dev)
+        Xb = inputs.bf16_normal((rows_b, hid), 1.0, seed=413, device=str(dev))
+        Hb = torch.empty((rows_b, inter), dtype=torch.bfloat16, device=dev)
+        Yb = torch.empty((rows_b, hid), dtype=torch.float32, device=dev)
+        ms = time_calls([lambda: tl.moe_ffn(Xb, Wgu_t, Wdn_t, Hb, Yb, d_off_b, q["experts"], rows_b, hid, inter, G, BR, BC)], 6)
+        fl = 2.0 * rows_b * (hid * 2 * inter + inter * hid)
+        by = act_b * 2 * (hid * 2 * inter + inter * hid) + 2 * rows_b * hid + 2 * 2 * rows_b * inter + 4 * rows_b * hid
+        moe.append({"proj": "expert_ffn_chain", "tokens": tokens_big, "rows": rows_b, "layout": "tile", "us": ms * 1e3,
+                    "GBps": by / (ms * 1e-3) / 1e9, "TFLOPs": fl / (ms * 1e-3) / 1e12, "active_experts": act_b,
+                    "cta": list(tl.gemm_plan(rows_b, 2 * inter, hid, G, BR, BC, (0, 0, 0), q["experts"]).cta)})
+        del Xb, Hb, Yb, d_off_b
+    del Wgu_t, Wdn_t
     moe_window.__exit__(None, None, None)
     extra["qwen_moe"] = moe
     tl.device_status()

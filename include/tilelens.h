@@ -111,7 +111,8 @@ typedef enum {
                                 predecessor's completion from wrong expert offsets, so that its check after the wait
                                 must find them wrong and build them again; the output is the ordinary one.
                                 The option resets itself to 0 when it is consumed. */
-    TL_OPT_MOE_ROW_CAP,      /* grouped products: most token rows per tile; 0 (default): the library's choice, else 16/32/64/128 */
+    TL_OPT_MOE_ROW_CAP,      /* grouped products: most token rows per tile; 0 (default): the library's choice (32, or 64 / 128 when
+                                the experts average more than 24 / 48 rows and there are enough such tiles), else 16/32/64/128 */
     TL_OPT_REDUCE_SPLIT,     /* 1 (default): a split tile's partial sums are added by all reduction CTAs inside it, 0: by one */
     TL_OPT_SM_LIMIT,         /* 0 (default): GEMM grids use every SM; n > 0: at most n CTAs (leaves SMs to concurrent work) */
     TL_OPT_NO_SCRATCH_PLANS, /* 1 (default): dense decode-sized products prefer schedules without partial tiles in global

@@ -355,6 +355,22 @@ static double mid_tile_estimate_us(const GemmPlan& pl, int64_t rows, int64_t N, 
     return us + 8.0;
 }
 
+// Token rows per tile of a grouped product whose caller left the tile to the library (0: the default of 32).  The
+// 32-row tile suits routings that leave most experts a handful of rows (Qwen-3 at 256 tokens: 16 rows per expert on
+// average).  With more rows per expert every further m-tile of an expert pulls the expert's weights out of L2 again,
+// so the tile grows with the average: 64 rows from 25 rows per expert on, 128 from 49 on, both 256 columns wide
+// (Qwen-3 gate_up / down at 1024 tokens: 194 / 129 -> 151 / 90 us; at 4096 tokens 575 / 397 -> 293 / 186 us) -- but
+// only while the larger tiles still number at least one per SM: few large tiles would have to be cut along K.
+// TL_OPT_MOE_ROW_CAP fixes the row count instead.
+static int grouped_tile_rows(int64_t rows_total, int E, int64_t N) {
+    if (opt(TL_OPT_MOE_ROW_CAP) != 0 || E < 1) return 0;
+    if (ensure_device_info()) return 0;
+    const int64_t avg = rows_total / E, n_tiles = ceil_div(N, 256), sms = dev().sm_count;
+    if (avg > 48 && rows_total / 128 * n_tiles >= sms) return 128;
+    if (avg > 24 && rows_total / 64 * n_tiles >= sms) return 64;
+    return 0;
+}
+
 static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32_t* d_offsets, int E,
                        int64_t rows_total, int64_t rows_max, int64_t N, int64_t K, int64_t G, int br, int bc,
                        int cta_m, int cta_n, int cta_k, cudaStream_t stream, const FixedScratch* fixed = nullptr,
@@ -447,6 +463,9 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                 cta_k = 64;
             }
         }
+    }
+    if (cta_m == 0 && cta_n == 0 && cta_k == 0 && d_offsets && !fixed && !generic) {
+        if (const int rows = grouped_tile_rows(rows_total, E, N)) { cta_m = rows; cta_n = 256; cta_k = 64; }
     }
     GemmPlan plan;
     {
@@ -1054,6 +1073,17 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
     if (!d_offsets && total_rows > 0) return TL_ERR_INVALID_ARG;
     if (!d_H_bf16) return TL_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // One tile for both products (the smaller of what each would take by itself), so that every form of the chain runs
+    // the same tiles.
+    int ffn_m = 0, ffn_n = 0, ffn_k = 0;
+    {
+        const int r1 = tl::grouped_tile_rows(total_rows, E, 2 * inter), r2 = tl::grouped_tile_rows(total_rows, E, hidden);
+        const int r = r1 < r2 ? r1 : r2;
+        const bool tma_rows = block_rows == 0 || block_cols >= 16;          // (narrower memory tiles keep their own path)
+        if (r > 0 && tma_rows) { ffn_m = r; ffn_n = 256; ffn_k = 64; }
+        // (a routing that would grow one product's tile alone: both at the default 32 rows)
+        else if ((r1 > 0 || r2 > 0) && tma_rows) { ffn_m = 32; ffn_n = 256; ffn_k = 64; }
+    }
     // (Not while the stream is being captured: the barrier form counts arrivals from a base the host keeps, which a
     // replayed graph would not advance.)
     if (total_rows > 0 && tl::opt(TL_OPT_FFN_ONE_LAUNCH) != 0 && !tl::stream_is_capturing(stream)) {
@@ -1062,11 +1092,11 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
         tl::GemmParams p1, p2;
         tl::GemmPlan plan1, plan2;
         int rc = tl::gemm_launch(d_X_sorted, d_W_gate_up, nullptr, d_offsets, E, total_rows, total_rows, 2 * inter, hidden, G,
-                                 block_rows, block_cols, 0, 0, 0, stream, nullptr, false, 2, d_H_bf16, nullptr, nullptr, &p1,
-                                 &plan1);
+                                 block_rows, block_cols, ffn_m, ffn_n, ffn_k, stream, nullptr, false, 2, d_H_bf16, nullptr,
+                                 nullptr, &p1, &plan1);
         if (rc) return rc;
         rc = tl::gemm_launch(d_H_bf16, d_W_down, d_Y, d_offsets, E, total_rows, total_rows, hidden, inter, G, block_rows,
-                             block_cols, 0, 0, 0, stream, nullptr, false, 2, nullptr, nullptr, nullptr, &p2, &plan2);
+                             block_cols, ffn_m, ffn_n, ffn_k, stream, nullptr, false, 2, nullptr, nullptr, nullptr, &p2, &plan2);
         if (rc) return rc;
         // (the grid is the larger of the two plans': a schedule copes with more CTAs than it has work for)
         const int grid = plan1.grid > plan2.grid ? plan1.grid : plan2.grid;
@@ -1137,10 +1167,10 @@ int tl_moe_ffn(const void* d_X_sorted, const void* d_W_gate_up, const void* d_W_
         }
     }
     if (int rc = tl_gemm_grouped_swiglu(d_X_sorted, d_W_gate_up, d_H_bf16, d_offsets, E, total_rows, 2 * inter, hidden, G,
-                                        block_rows, block_cols, 0, 0, 0, cuda_stream))
+                                        block_rows, block_cols, ffn_m, ffn_n, ffn_k, cuda_stream))
         return rc;
-    return tl_gemm_grouped(d_H_bf16, d_W_down, d_Y, d_offsets, E, total_rows, hidden, inter, G, block_rows, block_cols, 0,
-                           0, 0, cuda_stream);
+    return tl_gemm_grouped(d_H_bf16, d_W_down, d_Y, d_offsets, E, total_rows, hidden, inter, G, block_rows, block_cols, ffn_m,
+                           ffn_n, ffn_k, cuda_stream);
 }
 
 size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int cta_n, int cta_k) {
@@ -1148,17 +1178,27 @@ size_t tl_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int cta_m, int c
     if (M <= 0 || N <= 0 || K <= 0) return 0;
     if (tl::ensure_device_info()) return 0;
     size_t need = 0;
-    for (int grouped = 0; grouped < 2; ++grouped) {         // the larger of the dense and the grouped schedule
+    // the largest of the dense schedule and the grouped ones (the grouped tile grows with the rows per expert, and the
+    // number of experts is not known here: 32, 64 and 128 rows are all looked at)
+    for (int variant = 0; variant < 4; ++variant) {
+        const bool grouped = variant != 0;
         int bm = cta_m, bn = cta_n, bk = cta_k;
         const bool pair_sized = tl::ceil_div(M, 256) * tl::ceil_div(N, 256) * 2 >= tl::dev().sm_count;
-        if (cta_m == 0 && cta_n == 0 && cta_k == 0) tl::default_tile(M, grouped != 0, false, &bm, &bn, &bk, pair_sized);
+        const bool free_tile = cta_m == 0 && cta_n == 0 && cta_k == 0;
+        if (!free_tile && variant > 1) break;
+        if (free_tile) tl::default_tile(M, grouped, false, &bm, &bn, &bk, pair_sized);
+        if (free_tile && variant == 2) { bm = 64; bn = 256; bk = 64; }
+        if (free_tile && variant == 3) { bm = 128; bn = 256; bk = 64; }
         if (bm <= 0 || bn <= 0) return 0;
         tl::GemmPlan plan;
         // grouped: every expert may add a ragged m-tile and the number of experts is not known here; with the most
         // the library accepts the K ranges are cut over every SM, which is the largest scratch a launch can ask for
         const int64_t mt = grouped ? M / bm + tl::kMaxExperts : tl::ceil_div(M, bm);
-        if (tl::make_plan(M, mt * tl::ceil_div(N, bn), N, K, cta_m, cta_n, cta_k, grouped != 0, &plan, false, false, pair_sized))
+        if (tl::make_plan(M, mt * tl::ceil_div(N, bn), N, K, variant > 1 ? bm : cta_m, variant > 1 ? bn : cta_n,
+                          variant > 1 ? bk : cta_k, grouped, &plan, false, false, pair_sized)) {
+            if (variant > 1) continue;
             return 0;
+        }
         if (plan.ws_bytes > need) need = plan.ws_bytes;
     }
     return need;

@@ -392,6 +392,29 @@ def test_qwen_moe_full_size_sampled(name, K, N):
     _check_grouped(offsets, A, Bd, C, q["experts"], K, N, 16, 128, samples_per_expert=48, exact=False)
 
 
+@pytest.mark.parametrize("tokens,want_cta", [(512, (64, 256, 64)), (1024, (128, 256, 64))])
+@pytest.mark.parametrize("name,K,N", inputs.QWEN_MOE_PROJ)
+def test_qwen_moe_with_more_tokens_runs_larger_tiles(name, K, N, tokens, want_cta):
+    # more rows per expert than the benchmark's routing leaves: the library's grouped tile grows with the average
+    from gpu_util import tl
+    q = inputs.QWEN_MOE
+    offsets, counts, A, Bd, C = _grouped_case(q["experts"], tokens, q["topk"], K, N, 16, 128, seed=1, integer=True)
+    p = tl.gemm_last_plan()
+    assert p.cta == want_cta and p.stream_k == 0
+    _check_grouped(offsets, A, Bd, C, q["experts"], K, N, 16, 128, samples_per_expert=64, exact=True)
+    # every element of the busiest and of the smallest expert against the exact integer product
+    order = np.argsort(counts)
+    for e in (int(order[-1]), int(order[np.nonzero(counts[order])[0][0]])):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        want = A[r0:r1].double() @ inputs_from_tile_major(Bd[e], K, N).double()
+        assert torch.equal(C[r0:r1].cpu().double(), want)
+
+
+def inputs_from_tile_major(Bt_e, K, N):
+    """One expert's K x N weights back in row-major order (host side, for exact checks)."""
+    return Bt_e.cpu().reshape(K // 16, N // 128, 16, 128).permute(0, 2, 1, 3).reshape(K, N)
+
+
 @pytest.mark.parametrize("name,K,N", inputs.QWEN_ATTN_PROJ)
 def test_qwen_attention_projections(name, K, N):
     from gpu_util import check_against_oracle, run_gemm, sample_indices, tile_major_on_device

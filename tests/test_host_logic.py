@@ -151,6 +151,27 @@ def test_tile_of_dense_products_between_decode_and_prefill():
         assert plan(64, 57344, 8192).cta == (64, 256, 64) and plan(4096, 8192, 8192).pair_kernel == 1
 
 
+def test_grouped_tile_grows_with_the_rows_per_expert():
+    with _plans_as_if(148):
+        grouped = lambda rows, E, N, K: tl.gemm_plan(rows, N, K, 4096, 16, 128, (0, 0, 0), E)
+        # the Qwen-3 routing of the benchmark: 16 rows per expert on average
+        p = grouped(2048, 128, 1536, 2048)
+        assert (p.cta, p.stream_k, p.grid, p.workspace_bytes) == ((32, 256, 64), 0, 148, 0)
+        assert grouped(3072, 128, 1536, 2048).cta == (32, 256, 64)           # 24 rows
+        assert grouped(4096, 128, 1536, 2048).cta == (64, 256, 64)           # 32 rows
+        assert grouped(8192, 128, 1536, 2048).cta == (128, 256, 64)          # 64 rows
+        assert grouped(32768, 128, 2048, 768).cta == (128, 256, 64)
+        # many rows per expert but few tiles: the small tile, which needs no cut
+        p = grouped(2048, 16, 1024, 512)
+        assert (p.cta, p.stream_k) == ((32, 256, 64), 0)
+        # a fixed row cap switches the rule off
+        with tl.option(tl.OPT_MOE_ROW_CAP, 32):
+            assert grouped(32768, 128, 1536, 2048).cta == (32, 256, 64)
+        # what tl_gemm_workspace_bytes reports covers the larger tiles too
+        for rows, E, N, K in ((8192, 128, 1536, 2048), (700, 4, 512, 8192), (40000, 100, 2048, 768)):
+            assert tl.gemm_workspace_bytes(rows, N, K) >= grouped(rows, E, N, K).workspace_bytes
+
+
 def test_the_reported_workspace_covers_every_plan():
     # tl_gemm_workspace_bytes is what a caller sizes its own workspace from: never less than the plan of that call
     with _plans_as_if(148):
