@@ -185,11 +185,13 @@ int tl_relayout_batch(int n, const void* const* d_srcs, void* const* d_dsts, con
  *   d_C          device, 16-byte aligned, M*N floats, fully overwritten.
  *   cta_m/n/k    the CTA tile: cta_m token rows x cta_n weight columns per CTA,
  *                cta_k weight rows per pipeline stage.  0,0,0 lets the library
- *                choose (by M: M x 256 x 64 up to 64 rows, 128 x 128 x 128 or
- *                128 x 256 x 64 up to 512 rows, whichever its planner ranks
- *                ahead for the shape, CTA pairs on 256- or 512-row tiles for
+ *                choose (by M: M x 256 x 64 up to 64 rows, 128 x 128 x 128,
+ *                128 x 256 x 64 or 256 x 256 x 64 up to 512 rows, whichever its
+ *                planner ranks ahead for the shape, CTA pairs on 256- or 512-row tiles for
  *                prefill; tl_gemm_plan() tells).  Instantiated: cta_n in {64, 128, 256}, cta_k in {64, 128},
- *                cta_m in {16, 32, 64, 128, 256} (cta_n == 256: at most 128).
+ *                cta_m in {16, 32, 64, 128, 256} (cta_n == 256: at most 128, or
+ *                256 x 256 x 64 for dense problems whose tiles need no split
+ *                of K: two 128-row token blocks share each weight slab).
  *                Tiles may overhang M, N and K.
  *   K % 8 == 0 (16-byte row pitch of A); tile-major: K % block_rows == 0,
  *   N % block_cols == 0; row-major: N % 64 == 0.  N % 4 == 0 (C is written in

@@ -185,9 +185,12 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     if (BM != 16 && BM != 32 && BM != 64 && BM != 128 && BM != 256) return TL_ERR_UNSUPPORTED;
     if (BN != 64 && BN != 128 && BN != 256) return TL_ERR_UNSUPPORTED;
     if (BK != 64 && BK != 128) return TL_ERR_UNSUPPORTED;
-    if (BN == 256 && BM > 128) return TL_ERR_UNSUPPORTED;   // 2 accumulators x 2 groups x BM columns <= 512
+    // 256 x 256 x 64: the weights-on-N kernel with two 128-row token blocks per tile, one weight slab per stage serving
+    // both through the two accumulators (dense problems, whole-tile schedules only: see the end of this function)
+    const bool two_blocks = BM == 256 && BN == 256 && BK == 64 && !grouped && !generic && !narrow_scratch;
+    if (BN == 256 && BM > 128 && !two_blocks) return TL_ERR_UNSUPPORTED;   // 2 accumulators x 2 groups x BM columns <= 512
     plan->BM = BM; plan->BN = BN; plan->BK = BK;
-    plan->weights_on_n = BM <= 128;                         // tokens fit the 128 rows of the MMA's M side
+    plan->weights_on_n = BM <= 128 || two_blocks;           // tokens fit the 128 rows of the MMA's M side
     // With the tokens on the M side the MMA reads 64 rows (tiles of up to 64 tokens) or 128: a stage holds that
     // many token rows per 64-wide K slice, the ones beyond BM zeroed once by the kernel.  They only feed
     // accumulator rows that are never stored.
@@ -304,6 +307,8 @@ static int make_plan(int64_t rows_max, int64_t tile_bound, int64_t N, int64_t K,
     }
     if (grid < 1) grid = 1;
     plan->grid = int(grid);
+    // (a tile of two token blocks owns both accumulators and is never cut: its partial tile would be 256 KB)
+    if (two_blocks && (plan->stream_k || plan->cluster_k > 1)) return TL_ERR_UNSUPPORTED;
     plan->ws_bytes = plan->stream_k ? size_t(2) * size_t(grid) * BM * BN * sizeof(float) : 0;   // two slots per CTA
     return TL_OK;
 }
@@ -447,7 +452,15 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     if (cta_m == 0 && cta_n == 0 && cta_k == 0 && !d_offsets && !fixed && !generic && rows_max > 64 && rows_max <= 512 &&
         !(rows_max > 384 && pair_sized)) {
         GemmPlan wide, other;
-        if (make_plan(rows_max, ceil_div(rows_total, 128) * ceil_div(N, 256), N, K >> k_shift, 128, 256, 64, false, &wide,
+        // 129 to 256 rows: both 128-row blocks on one weight slab per stage (256 x 256 x 64, whole tiles only), where
+        // there are enough tiles: a third less out of L2 again (Llama gate_up at 256 rows 257 -> 235 us)
+        if (rows_max > 128 && rows_max <= 256 &&
+            make_plan(rows_max, ceil_div(N, 256), N, K >> k_shift, 256, 256, 64, false, &wide, false, false, pair_sized,
+                      rows_total) == TL_OK) {
+            cta_m = 256;
+            cta_n = 256;
+            cta_k = 64;
+        } else if (make_plan(rows_max, ceil_div(rows_total, 128) * ceil_div(N, 256), N, K >> k_shift, 128, 256, 64, false, &wide,
                       false, false, pair_sized, rows_total) == TL_OK &&
             wide.stream_k == 0) {
             int bm = 0, bn = 0, bk = 0;

@@ -93,6 +93,9 @@ struct alignas(64) GemmParams {
     int blocks_per_row;         // N / bc
 };
 
+struct tl_true { static constexpr bool value = true; };
+struct tl_false { static constexpr bool value = false; };
+
 struct TileInfo {
     int n0;          // first weight column
     int row0;        // first row of A / C
@@ -751,6 +754,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 tok_off[j] = (uint32_t(j >> 2) * uint32_t(p.a_rows) * kAtomBytes + uint32_t(j & 3) * 32u) >> 4;
             }
             const uint32_t ugroup16 = p.ugroup_off >> 4;
+            // Tiles of two 128-row token blocks (weights on N, BM = 256): every K step is issued twice, on the same
+            // weight slab, into the two accumulators, which then both belong to the tile.
+            const bool two_blocks = kWN && p.BM > 128;
             while (ok && sched.next(w)) {
                 const TileInfo t = decode_tile(p, prefix, row_start, w.tile);
                 const uint32_t n_mma = kWN ? uint32_t(kBN) : uint32_t((t.rows + 15) & ~15);
@@ -768,32 +774,45 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * uint32_t(kNumN * acc_cols);
-                for (int kit = w.kbeg; kit < w.kend; ++kit) {
-                    if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull, p.wait_limit_ns)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after_sync();
-                    const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
-                    const uint32_t w_lo0 = w_lo_const | ((sw & 0x3FFFFu) >> 4);
-                    const uint32_t tok_lo0 = tok_lo_const | (((sw + kWBytes) & 0x3FFFFu) >> 4);
-                    const uint32_t first = kit > w.kbeg ? 1u : 0u;
-#pragma unroll
-                    for (int j = 0; j < kKSteps; ++j) {
-#pragma unroll
-                        for (int u = 0; u < kNumN; ++u) {
-                            const uint32_t accum = j > 0 ? 1u : first;
-                            const uint32_t w_lo = w_lo0 + w_off[j] + uint32_t(u) * ugroup16;
-                            if (kWN) umma_split<kFp8>(d_tmem, tok_lo0 + tok_off[j], tok_hi, w_lo, w_hi, idesc, accum);
-                            else umma_split<kFp8>(d_tmem + uint32_t(u * acc_cols), w_lo, w_hi, tok_lo0 + tok_off[j], tok_hi, idesc, accum);
+                // (the loop exists twice so that the usual one carries nothing for the second token block: the issuing
+                // thread has no slack)
+                auto k_loop = [&](auto second_block) {
+                    for (int kit = w.kbeg; kit < w.kend; ++kit) {
+                        if (!mbar_wait_bounded(&full_bar[stage], phase, abort_ptr, p.status, kWaitMmaFull, p.wait_limit_ns)) {
+                            ok = false;
+                            break;
                         }
+                        tc_fence_after_sync();
+                        const uint32_t sw = smem_u32(stages + size_t(stage) * stage_bytes);
+                        const uint32_t w_lo0 = w_lo_const | ((sw & 0x3FFFFu) >> 4);
+                        const uint32_t tok_lo0 = tok_lo_const | (((sw + kWBytes) & 0x3FFFFu) >> 4);
+                        const uint32_t first = kit > w.kbeg ? 1u : 0u;
+#pragma unroll
+                        for (int j = 0; j < kKSteps; ++j) {
+#pragma unroll
+                            for (int u = 0; u < kNumN; ++u) {
+                                const uint32_t accum = j > 0 ? 1u : first;
+                                const uint32_t w_lo = w_lo0 + w_off[j] + uint32_t(u) * ugroup16;
+                                if (kWN) {
+                                    umma_split<kFp8>(d_tmem, tok_lo0 + tok_off[j], tok_hi, w_lo, w_hi, idesc, accum);
+                                    if (decltype(second_block)::value)   // rows 128.. of the token slab: 128 swizzle rows further
+                                        umma_split<kFp8>(d_tmem + uint32_t(kBN), tok_lo0 + tok_off[j] + ((128u * kAtomBytes) >> 4),
+                                                         tok_hi, w_lo, w_hi, idesc, accum);
+                                } else {
+                                    umma_split<kFp8>(d_tmem + uint32_t(u * acc_cols), w_lo, w_hi, tok_lo0 + tok_off[j], tok_hi, idesc,
+                                                     accum);
+                                }
+                            }
+                        }
+                        umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
+                        if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
                     }
-                    umma_commit(&empty_bar[stage]);      // frees the stage once these MMAs have read it
-                    if (++stage == uint32_t(p.num_stages)) { stage = 0; phase ^= 1; }
-                }
+                };
+                if (kWN && two_blocks && t.rows > 128) k_loop(tl_true{});
+                else k_loop(tl_false{});
                 if (!ok) break;
                 umma_commit(&acc_full_bar[acc]);         // accumulator complete
-                acc ^= 1;
+                if (!two_blocks) acc ^= 1;               // (two blocks: the tile owned both accumulators)
                 if (acc == 0) acc_phase ^= 1;
             }
         }
@@ -968,9 +987,12 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 // (MMA of 64 rows: rows 16q..16q+15 sit in the lower half of lane quarter q, the upper 16 lanes of
                 // each quarter hold nothing.)
                 const bool m64 = p.umma_m == 64 && t.rows <= 64;
-                const int row = m64 ? (lane < 16 ? quarter * 16 + lane : p.BM) : quarter * 32 + lane;
-                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * uint32_t(acc_cols);
-                if ((m64 ? quarter * 16 : quarter * 32) < t.rows) {      // this lane quarter holds at least one real row
+                // (tiles of two 128-row token blocks, BM = 256: the second block's rows sit in the second accumulator)
+                const int blocks = p.BM > 128 && t.rows > 128 ? 2 : 1;
+                for (int blk = 0; blk < blocks; ++blk) {
+                const int row = m64 ? (lane < 16 ? quarter * 16 + lane : p.BM) : blk * 128 + quarter * 32 + lane;
+                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + (acc + uint32_t(blk)) * uint32_t(acc_cols);
+                if ((m64 ? quarter * 16 : blk * 128 + quarter * 32) < t.rows) {      // this lane quarter holds at least one real row
                     float* dst = out + int64_t(row) * ld;
                     const bool gated = full && p.epi_swiglu;
                     __nv_bfloat16* hdst = p.H + int64_t(t.row0 + row) * p.ldh + (t.n0 >> 1);
@@ -1017,6 +1039,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                                                     __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
                         }
                     }
+                }
                 }
             }
             if (ok && !kWN) {
@@ -1074,7 +1097,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, bool alloc_tmem, 
                 __syncwarp();
                 if (lane == 0) atomicAdd(p.tile_flags + t.mtile, 1u);
             }
-            acc ^= 1;
+            if (!(kWN && p.BM > 128)) acc ^= 1;          // (two token blocks: the tile owned both accumulators)
             if (acc == 0) acc_phase ^= 1;
 
             if (*abort_ptr) break;

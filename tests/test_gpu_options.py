@@ -44,6 +44,49 @@ def test_products_between_decode_and_prefill_are_exact_on_the_tile_the_library_p
         assert torch.equal(run_gemm(A, Bd, M, N, K, 16, 128, cta).cpu(), want)
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 256 * 112, 512), (200, 256 * 112, 320), (130, 256 * 148, 64), (300, 256 * 148, 256),
+                                   (512, 256 * 74, 192), (257, 256 * 148 + 128, 128)])
+def test_tiles_of_two_token_blocks_are_exact(M, N, K):
+    # 256 x 256 x 64 in the weights-on-N kernel: one weight slab per stage, two 128-row token blocks, both accumulators
+    # owned by the tile.  Whole, ragged and single-block last tiles; fp32 and bf16 C; the [N][K] flavour and FP8.
+    from gpu_util import DEV, guarded_out, run_gemm, tl
+    A, Bd, want = _int_case(M, N, K, 16, 128, seed=M + K)
+    got = run_gemm(A, Bd, M, N, K, 16, 128, (256, 256, 64))
+    p = tl.gemm_last_plan()
+    assert p.cta == (256, 256, 64) and p.stream_k == 0 and p.cluster_k == 1 and p.pair_kernel == 0 and p.weights_on_n == 1
+    assert torch.equal(got.cpu(), want)
+    g = guarded_out((M, N), torch.bfloat16)
+    tl.gemm_bf16(A.to(DEV), Bd, g.t, M, N, K, 4096, 16, 128, (256, 256, 64))
+    tl.device_status()
+    assert torch.equal(g.check().cpu(), want.to(torch.bfloat16))
+    if M <= 256:                                              # the library's own choice for 129 to 256 rows
+        got = run_gemm(A, Bd, M, N, K, 16, 128)
+        assert tl.gemm_last_plan().cta == ((256, 256, 64) if M > 128 else (128, 256, 64))
+        assert torch.equal(got.cpu(), want)
+    # K-contiguous weights, bf16 and FP8
+    Bh = inputs.bf16_integers((K, N), -8, 8, seed=M + K + 1)
+    Wnk = Bh.t().contiguous().to(DEV)
+    C = guarded_out((M, N), torch.float32)
+    tl.gemm_kmajor(A.to(DEV), Wnk, C.t, M, N, K, 0, 0, 0, (256, 256, 64))
+    tl.device_status()
+    assert tl.gemm_last_plan().cta == (256, 256, 64) and torch.equal(C.check().cpu(), want)
+    if K % 128 != 0:                                          # (the plain FP8 array wants whole 128-byte rows)
+        return
+    A8, B8 = inputs.fp8_integers((M, K), -6, 6, seed=M), inputs.fp8_integers((K, N), -6, 6, seed=N)
+    C = guarded_out((M, N), torch.float32)
+    tl.gemm_fp8_kmajor(A8.to(DEV), B8.t().contiguous().to(DEV), C.t, M, N, K, 0, 0, 0, (256, 256, 128))
+    tl.device_status()
+    assert torch.equal(C.check().cpu().double(), A8.double() @ B8.double())
+
+
+def test_a_tile_of_two_token_blocks_is_refused_where_it_would_be_cut():
+    from gpu_util import run_gemm, tl
+    A, Bd, _ = _int_case(200, 1024, 512, 16, 128, seed=9)
+    with pytest.raises(tl.TileLensError) as e:
+        run_gemm(A, Bd, 200, 1024, 512, 16, 128, (256, 256, 64))          # 4 tiles: clusters or a cut, neither of which it has
+    assert e.value.status == 2
+
+
 def test_one_box_per_memory_tile_gives_the_same_bits():
     from gpu_util import run_gemm, tl
     M, N, K = 40, 1024, 1024

@@ -134,9 +134,17 @@ def test_tile_of_dense_products_between_decode_and_prefill():
         assert (p.cta, p.stream_k, p.cluster_k, p.grid) == ((128, 256, 64), 0, 1, 112)
         p = plan(128, 10240, 8192)                        # 40 wide tiles in clusters of 3; the narrow tile would be cut
         assert (p.cta, p.stream_k, p.cluster_k, p.grid) == ((128, 256, 64), 0, 3, 120)
-        # 256 rows, where the default would be the CTA-pair kernel: the wide tile up to 384 rows
+        # 129 to 256 rows with enough tiles for whole-tile schedules: both 128-row blocks on one weight slab per stage
         p = plan(256, 57344, 8192)
+        assert (p.cta, p.pair_kernel, p.stream_k, p.cluster_k, p.grid, p.stages) == ((256, 256, 64), 0, 0, 1, 112, 3)
+        p = plan(256, 8192, 28672)                        # 32 such tiles would have to be cut: the wide tile in clusters
+        assert (p.cta, p.stream_k, p.cluster_k) == ((128, 256, 64), 0, 2)
+        # where the default would be the CTA-pair kernel: the wide tile up to 384 rows
+        p = plan(384, 57344, 8192)
         assert (p.cta, p.pair_kernel, p.stream_k) == ((128, 256, 64), 0, 0)
+        # the two-block tile is refused outright where its schedule would leave partial tiles
+        with pytest.raises(tl.TileLensError):
+            tl.gemm_plan(256, 8192, 28672, 4096, 16, 128, (256, 256, 64))
         p = plan(512, 57344, 8192)
         assert p.pair_kernel == 1
         # small weights: more, smaller tiles win (latency, not bandwidth)
