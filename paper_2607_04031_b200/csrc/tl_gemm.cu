@@ -339,6 +339,45 @@ struct FixedScratch {
     uint32_t* status;    // word the kernel raises when a bounded wait expires
 };
 
+// The CTA-pair kernel's schedule on `clusters` co-resident clusters, in units of one 256-token tile run by the
+// 256-token instantiation.  It mixes whole waves of 512-token tiles with 256-token tiles for the rest (*big_tiles on
+// entry: how many 512-token tiles that mix has); with few waves the mix can lose to 256-token tiles alone: a 512-token
+// tile that M leaves half empty, and every 256-token tile run by the 512-token instantiation (shorter pipeline,
+// accumulators not alternating), costs about 1.5 units, a full 512-token tile 1.8.  The busiest cluster of both
+// schedules is worked out from the kernel's own tile order; *big_tiles is set to 0 where 256-token tiles alone are
+// ahead by a tenth (Llama qkv at 640 rows: 74 + 12 tiles 172 us, 120 small ones 119 us; gate_up at 1024 rows keeps
+// 444 + 8).  Returns the units of the schedule chosen.
+static double pair_schedule_units(int64_t rows_total, int64_t N, int clusters, int64_t* big_tiles) {
+    const int64_t n_t = ceil_div(N, 256), m_big = ceil_div(rows_total, 512), big_total = m_big * n_t;
+    const int C = clusters < 1 ? 1 : (clusters < 256 ? clusters : 256);
+    const double small_only = double(ceil_div(ceil_div(rows_total, 256) * n_t, int64_t(C)));
+    if (*big_tiles <= 0) return small_only;
+    const int64_t all = *big_tiles + 2 * (big_total - *big_tiles);
+    double load[256] = {0.0};
+    auto m_tile_of = [&](int64_t tile) {                            // pair_tile_coords of the kernel, m part
+        const int64_t band_tiles = 8 * n_t, band = tile / band_tiles, r = tile - band * band_tiles;
+        const int64_t band_rows = m_big - band * 8 < 8 ? m_big - band * 8 : 8;
+        return band * 8 + r % band_rows;
+    };
+    for (int64_t t = 0; t < all; ++t) {
+        double cost;
+        if (t < *big_tiles) {
+            cost = rows_total - m_tile_of(t) * 512 > 256 ? 1.8 : 1.5;
+        } else {
+            const int64_t sidx = t - *big_tiles, row0 = m_tile_of(*big_tiles + (sidx >> 1)) * 512 + (sidx & 1) * 256;
+            cost = row0 < rows_total ? 1.5 : 0.0;
+        }
+        load[t % C] += cost;
+    }
+    double mixed = 0.0;
+    for (int c = 0; c < C; ++c) mixed = load[c] > mixed ? load[c] : mixed;
+    if (small_only < 0.9 * mixed) {
+        *big_tiles = 0;
+        return small_only;
+    }
+    return mixed;
+}
+
 // Rough time of a dense weights-on-N plan, for choosing between the 128- and the 256-column tile at 65 to 512 token
 // rows (K in 2-byte units).  What one CTA pulls into shared memory at about 90 GB/s (measured 75-105: weight slabs and
 // the token rows that come with each, most of them L2 hits), not faster than HBM delivers the weights once; plus the
@@ -472,6 +511,26 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                        0.97 * mid_tile_estimate_us(other, rows_total, N, K >> k_shift);
             if (take) {
                 cta_m = 128;
+                cta_n = 256;
+                cta_k = 64;
+            }
+        }
+    }
+    // More rows, where the CTA-pair kernel is the default: its 74 clusters take 256 x 256 tiles in whole waves, and a
+    // tile count just above a multiple of 74 costs a whole wave more (Llama down at 1024 rows: 128 tiles, two waves,
+    // 410 us).  The two-block tile does the same tile on one SM in about 1.7 units of a pair's 256-token tile; where its
+    // whole-tile schedule fits the tile count better by a tenth it is taken (128 tiles on 128 CTAs: 351 us).
+    if (cta_m == 0 && cta_n == 0 && cta_k == 0 && !d_offsets && !fixed && !generic && rows_max > 512 && pair_sized &&
+        opt(TL_OPT_PAIR_KERNEL) != 0) {
+        GemmPlan two;
+        const int64_t tiles = ceil_div(rows_total, 256) * ceil_div(N, 256);
+        if (make_plan(rows_max, tiles, N, K >> k_shift, 256, 256, 64, false, &two, false, false, pair_sized, rows_total) == TL_OK) {
+            int clusters = dev().pair_max_clusters;
+            if (clusters <= 0) clusters = dev().sm_count / 2;             // (not asked yet: at most one pair per two SMs)
+            int64_t big = opt(TL_OPT_PAIR_512) == 0 ? 0 : (ceil_div(rows_total, 512) * ceil_div(N, 256) / clusters) * clusters;
+            const double pair_units = pair_schedule_units(rows_total, N, clusters, &big);
+            if (1.7 * double(ceil_div(tiles, int64_t(two.grid))) < 0.9 * pair_units) {
+                cta_m = 256;
                 cta_n = 256;
                 cta_k = 64;
             }
@@ -869,7 +928,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
         // clusters; what is left of the tile grid runs as 256-token tiles.  TL_OPT_PAIR_512 = 0: 256-token tiles only.
         const bool halves_off = opt(TL_OPT_PAIR_512) == 0;
         const int64_t big_total = ceil_div(rows_total, 512) * ceil_div(N, 256);
-        const int64_t big_tiles = halves_off ? 0 : (big_total / max_clusters) * max_clusters;
+        int64_t big_tiles = halves_off ? 0 : (big_total / max_clusters) * max_clusters;
+        if (big_tiles > 0) (void)pair_schedule_units(rows_total, N, max_clusters, &big_tiles);
         const int halves = big_tiles > 0 ? 2 : 1;
         const size_t stage_bytes = 64 * 128 * 2 + size_t(halves) * 128 * kAtomBytes;
         int stages = int((kMaxDynamicSmem - 1024) / stage_bytes);

@@ -79,6 +79,22 @@ def test_tiles_of_two_token_blocks_are_exact(M, N, K):
     assert torch.equal(C.check().cpu().double(), A8.double() @ B8.double())
 
 
+@pytest.mark.parametrize("M,N,K,want", [(1024, 8192, 256, ("two", 128)),     # 128 tiles: one wave of two-block tiles
+                                        (640, 10240, 192, ("two", 120)),
+                                        (768, 256 * 74, 2176, ("pair", 0)),    # two waves of half-empty 512-token tiles: small only
+                                        (1024, 256 * 224, 64, ("pair", 444))])
+def test_a_few_waves_above_512_rows_are_exact_on_the_schedule_the_library_picks(M, N, K, want):
+    from gpu_util import run_gemm, tl
+    A, Bd, exact = _int_case(M, N, K, 16, 128, seed=M + N)
+    got = run_gemm(A, Bd, M, N, K, 16, 128)
+    p = tl.gemm_last_plan()
+    if want[0] == "two":
+        assert (p.pair_kernel, p.cta, p.grid) == (0, (256, 256, 64), want[1])
+    else:
+        assert p.pair_kernel == 1 and p.pair_tiles_512 == want[1]
+    assert torch.equal(got.cpu(), exact)
+
+
 def test_a_tile_of_two_token_blocks_is_refused_where_it_would_be_cut():
     from gpu_util import run_gemm, tl
     A, Bd, _ = _int_case(200, 1024, 512, 16, 128, seed=9)
@@ -153,10 +169,10 @@ def test_pair_kernel_store_paths_write_the_same_bits(M, N, K):
     got = {}
     for mode in (1, 0):
         with tl.option(tl.OPT_PAIR_TMA_STORE, mode):
-            got[mode] = run_gemm(A, Bt, M, N, K, 16, 128).clone()
+            got[mode] = run_gemm(A, Bt, M, N, K, 16, 128, (256, 128, 64)).clone()      # (the pair kernel's tile, by name)
             assert tl.gemm_last_plan().pair_kernel == 1
             g = guarded_out((M, N), torch.bfloat16)
-            tl.gemm_bf16(A.to(DEV), Bt, g.t, M, N, K, 4096, 16, 128)
+            tl.gemm_bf16(A.to(DEV), Bt, g.t, M, N, K, 4096, 16, 128, (256, 128, 64))
             tl.device_status()
             got[mode, "bf16"] = g.check().clone()
     assert torch.equal(got[1], got[0]) and torch.equal(got[1, "bf16"], got[0, "bf16"])

@@ -159,6 +159,27 @@ def test_tile_of_dense_products_between_decode_and_prefill():
         assert plan(64, 57344, 8192).cta == (64, 256, 64) and plan(4096, 8192, 8192).pair_kernel == 1
 
 
+def test_schedules_of_a_few_waves_above_512_rows():
+    with _plans_as_if(148):
+        plan = lambda M, N, K: tl.gemm_plan(M, N, K)
+        # prefill proper: whole waves of 512-token pair tiles, 256-token tiles for the rest
+        p = plan(4096, 10240, 8192)
+        assert (p.pair_kernel, p.pair_tiles_512, p.pair_tiles_256) == (1, 296, 48)
+        p = plan(1024, 57344, 8192)
+        assert (p.pair_kernel, p.pair_tiles_512, p.pair_tiles_256) == (1, 444, 8)
+        # M leaves every other 512-token tile half empty and there are ten waves: 256-token tiles alone
+        p = plan(768, 57344, 8192)
+        assert (p.pair_kernel, p.cta, p.pair_tiles_512, p.pair_tiles_256) == (1, (256, 128, 64), 0, 672)
+        # 128 tiles: two waves of pairs, or one wave of two-block tiles on 128 CTAs
+        p = plan(1024, 8192, 28672)
+        assert (p.pair_kernel, p.cta, p.stream_k, p.cluster_k, p.grid) == (0, (256, 256, 64), 0, 1, 128)
+        p = plan(640, 10240, 8192)                        # 120 tiles on 120 CTAs
+        assert (p.pair_kernel, p.cta, p.grid) == (0, (256, 256, 64), 120)
+        # the pair kernel switched off: none of this applies
+        with tl.option(tl.OPT_PAIR_KERNEL, 0):
+            assert plan(1024, 8192, 28672).cta == (256, 128, 64)
+
+
 def test_grouped_tile_grows_with_the_rows_per_expert():
     with _plans_as_if(148):
         grouped = lambda rows, E, N, K: tl.gemm_plan(rows, N, K, 4096, 16, 128, (0, 0, 0), E)
