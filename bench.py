@@ -912,6 +912,8 @@ PROFILE_CASES = {
     "decode_qkv_m8": ("gemm", 8, 8192, 10240),
     "decode_o_m32": ("gemm", 32, 8192, 8192),
     "decode_down_m1": ("gemm", 1, 28672, 8192),
+    "mid_gate_up_m128": ("gemm", 128, 8192, 57344),         # 128 x 256 x 64 tiles, whole tiles on 112 CTAs
+    "mid_gate_up_m256": ("gemm", 256, 8192, 57344),         # 256 x 256 x 64: two token blocks per weight slab
     "prefill_o": ("gemm", 4096, 8192, 8192),
     "prefill_qkv": ("gemm", 4096, 8192, 10240),
     "relayout_o": ("relayout", 0, 8192, 8192),
