@@ -488,8 +488,16 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
     // memory (they are 128 KB each: down at 384 tokens, K cut over all CTAs, 213 us with the narrow tile against 289)
     // and mid_tile_estimate_us says it is ahead.  Where the default would be the CTA-pair kernel: up to 384 rows the
     // wide tile (gate_up at 256 tokens 255 against 308 us), beyond that the pair kernel.
+    // (129 to 256 rows with less than 8192 weight rows and tiles for at least three quarters of the pair kernel's waves
+    // stay with CTA pairs: with a short K loop their deeper pipeline and hidden epilogue count for more than the token
+    // rows they load -- gate_up-shaped, 256 rows: K = 4096 132 us against 145-148, K = 1024 57 against 70-75; K = 8192 a tie)
+    bool pairs_ahead = false;
+    if (rows_max > 128 && rows_max <= 256 && pair_sized && (K >> k_shift) < 8192 && opt(TL_OPT_PAIR_KERNEL) != 0) {
+        const int64_t tiles = ceil_div(N, 256), clusters = dev().sm_count / 2;
+        pairs_ahead = 4 * tiles >= 3 * ceil_div(tiles, clusters) * clusters;
+    }
     if (cta_m == 0 && cta_n == 0 && cta_k == 0 && !d_offsets && !fixed && !generic && rows_max > 64 && rows_max <= 512 &&
-        !(rows_max > 384 && pair_sized)) {
+        !(rows_max > 384 && pair_sized) && !pairs_ahead) {
         GemmPlan wide, other;
         // 129 to 256 rows: both 128-row blocks on one weight slab per stage (256 x 256 x 64, whole tiles only), where
         // there are enough tiles: a third less out of L2 again (Llama gate_up at 256 rows 257 -> 235 us)

@@ -137,6 +137,8 @@ def test_tile_of_dense_products_between_decode_and_prefill():
         # 129 to 256 rows with enough tiles for whole-tile schedules: both 128-row blocks on one weight slab per stage
         p = plan(256, 57344, 8192)
         assert (p.cta, p.pair_kernel, p.stream_k, p.cluster_k, p.grid, p.stages) == ((256, 256, 64), 0, 0, 1, 112, 3)
+        p = plan(256, 57344, 4096)                        # a shorter K loop: CTA pairs on 256-token tiles
+        assert (p.pair_kernel, p.pair_tiles_512, p.pair_tiles_256) == (1, 0, 224)
         p = plan(256, 8192, 28672)                        # 32 such tiles would have to be cut: the wide tile in clusters
         assert (p.cta, p.stream_k, p.cluster_k) == ((128, 256, 64), 0, 2)
         # where the default would be the CTA-pair kernel: the wide tile up to 384 rows
