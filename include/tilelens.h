@@ -337,7 +337,8 @@ typedef struct tl_gemm_plan_info {
     int32_t stream_k;              /* 1: K ranges cut over the CTAs + reduction kernel; 0: whole tiles */
     int32_t grid;                  /* CTAs launched */
     int32_t stages;                /* pipeline depth */
-    int32_t weights_on_n;          /* 1: weights on the N side of the MMA (token tiles of up to 128 rows) */
+    int32_t weights_on_n;          /* 1: weights on the N side of the MMA (token tiles of up to 128 rows, or 256 x 256 x 64:
+                                      two 128-row token blocks per tile) */
     int32_t generic_path;          /* 1: weights loaded by the generic-address path of Section 4.4 (permuted in shared
                                       memory); 2: memory tiles fetched as stored and read by the MMA as they are (16-byte
                                       rows, single-column tiles); 3: fetched as stored, 8- or 4-byte rows transposed in place */
