@@ -69,6 +69,49 @@ def test_llama_prefill_every_tile_sampled(name, K, N):
     assert float(np.max(err / np.maximum(S, 1e-300))) <= 1e-4
 
 
+# Between decode and prefill the library picks the tile and the schedule from the shape: each kind once at full size.
+MID_CASES = [
+    ("gate_up", 128, "wide"),          # 128 x 256 x 64, whole tiles on 112 CTAs
+    ("qkv", 128, "wide_clusters"),     # the same tile, split-K inside clusters of 3
+    ("gate_up", 256, "two_blocks"),    # 256 x 256 x 64: two token blocks per weight slab
+    ("down", 384, "cut"),              # 128 x 128 x 128 with the stream-K cut and its reduction kernel
+    ("qkv", 640, "two_blocks"),        # 120 tiles on 120 CTAs instead of two waves of pairs
+    ("gate_up", 768, "pairs_256"),     # CTA pairs on 256-token tiles only (512-token tiles would be half empty)
+    ("down", 1024, "two_blocks"),      # 128 tiles on 128 CTAs
+]
+
+
+@pytest.mark.parametrize("proj,M,kind", MID_CASES)
+def test_llama_between_decode_and_prefill_every_tile_sampled(proj, M, kind):
+    from gpu_util import DEV, run_gemm, tl
+    K, N = next((k, n) for name, k, n in inputs.LLAMA70B_PROJ if name == proj)
+    A = inputs.bf16_normal((M, K), 1.0, seed=43, device=DEV)
+    B = inputs.bf16_normal((K, N), 0.02, seed=44, device=DEV)
+    Bt = torch.empty_like(B)
+    tl.relayout(B, Bt, K, N, 2, G, BR, BC, tl.TO_TILE_MAJOR)
+    del B
+    C = run_gemm(A, Bt, M, N, K, BR, BC)
+    p = tl.gemm_last_plan()
+    if kind == "wide":
+        assert (p.cta, p.stream_k, p.cluster_k) == ((128, 256, 64), 0, 1)
+    elif kind == "wide_clusters":
+        assert (p.cta, p.stream_k, p.cluster_k) == ((128, 256, 64), 0, 3)
+    elif kind == "two_blocks":
+        assert (p.cta, p.pair_kernel, p.stream_k, p.cluster_k) == ((256, 256, 64), 0, 0, 1)
+    elif kind == "cut":
+        assert (p.cta, p.stream_k) == ((128, 128, 128), 1)
+    else:
+        assert (p.pair_kernel, p.pair_tiles_512) == (1, 0)
+    assert torch.isfinite(C).all()
+    ii, jj = per_tile_sample(M, N, seed=K + N + M, per_tile=8, lines=4)
+    got = C[torch.from_numpy(ii).to(DEV), torch.from_numpy(jj).to(DEV)].cpu().numpy().astype(np.float64)
+    del C
+    ref, S = tlo.matmul_at(inputs.bits(A), inputs.bits(Bt.reshape(-1)), TILE, BR, BC, M, N, K, ii, jj)
+    err = np.abs(got - ref)
+    assert np.all(err <= 1e-3 * S), f"max err/S = {np.max(err / np.maximum(S, 1e-300)):.3e}"
+    assert float(np.max(err / np.maximum(S, 1e-300))) <= 1e-4
+
+
 @pytest.mark.parametrize("name,K,N", inputs.QWEN_MOE_PROJ)
 def test_qwen_moe_every_tile_sampled(name, K, N):
     from gpu_util import DEV, guarded_out, tl
