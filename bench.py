@@ -745,9 +745,24 @@ def run_ours(args):
                         if rep_ > 0:
                             evs[layout].append((a, b))
             torch.cuda.synchronize()
+            # the same launches back to back without an event between them, direct and as one replayed CUDA graph
+            def chain_():
+                for c in range(copies):
+                    tl.gemm(Aq, Wt[c], Cq, 256, N, K, G, BR, BC)
+            chain_us = {}
+            try:
+                graph_q = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph_q):
+                    chain_()
+                for kind, fn in (("direct", chain_), ("graph", graph_q.replay)):
+                    chain_us[kind] = time_calls([fn], 8) * 1e3 / copies
+                del graph_q
+            except Exception as exc:  # report, never hide
+                chain_us = {"error": f"{type(exc).__name__}: {exc}"}
             for layout in ("tile", "row"):
                 med = statistics.median(a.elapsed_time(b) for a, b in evs[layout])
                 qattn.append({"proj": name, "M": 256, "layout": layout, "us": med * 1e3,
+                              **({"back_to_back_us": chain_us} if layout == "tile" else {}),
                               "GBps": gemm_bytes(256, N, K) / (med * 1e-3) / 1e9,
                               "TFLOPs": 2.0 * 256 * N * K / (med * 1e-3) / 1e12,
                               "cta": list(tl.gemm_plan(256, N, K, G, BR, BC).cta)})
