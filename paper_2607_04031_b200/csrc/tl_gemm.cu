@@ -382,7 +382,8 @@ static double pair_schedule_units(int64_t rows_total, int64_t N, int clusters, i
 // rows (K in 2-byte units).  What one CTA pulls into shared memory at about 90 GB/s (measured 75-105: weight slabs and
 // the token rows that come with each, most of them L2 hits), not faster than HBM delivers the weights once; plus the
 // exchange of partial tiles inside a cluster (about 6 us for 128 KB tiles, 3 us for 64 KB), 12 us for the partial
-// tiles and the second kernel of a stream-K cut, and a fixed 8 us.  Fitted to Llama-70B and Qwen-3 shapes at 96-512 rows; it only has to rank two plans.
+// tiles and the second kernel of a stream-K cut, and a fixed 8 us.  Fitted to Llama-70B and Qwen-3 shapes at 96-512
+// rows; it only has to rank two plans.
 static double mid_tile_estimate_us(const GemmPlan& pl, int64_t rows, int64_t N, int64_t K) {
     const double tiles = double(ceil_div(rows, pl.BM)) * double(ceil_div(N, pl.BN));
     const double k_iters = double(ceil_div(K, pl.BK));
@@ -580,8 +581,8 @@ static int gemm_launch(const void* d_A, const void* d_B, float* d_C, const int32
                                    d_offsets != nullptr, &plan, fixed != nullptr, generic, pair_sized, rows_total))
                 return rc;
     }
-    if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;
-    if (d_H_swiglu && !plan.weights_on_n) return TL_ERR_UNSUPPORTED;        // the gated epilogue pairs columns of one token row   // a K tail would read the next expert's rows
+    if (d_offsets && K % (int64_t(plan.BK) << k_shift) != 0) return TL_ERR_UNSUPPORTED;   // a K tail would read the next expert's rows
+    if (d_H_swiglu && !plan.weights_on_n) return TL_ERR_UNSUPPORTED;        // the gated epilogue pairs columns of one token row
     if (!plan_only && opt(TL_OPT_PLAN_AS_IF_SMS) != 0) return TL_ERR_INVALID_ARG;      // the planning test hook is on
     if (!fixed && !plan_only)
         if (int rc = ensure_control()) return rc;
