@@ -485,6 +485,25 @@ def test_gemm_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
             assert np.array_equal(run_gemm(A, Bg, M, N, K, br, bc).cpu().numpy().astype(np.float64), want)
 
 
+def test_two_block_tiles_give_up_the_same_way():
+    # The tile of two token blocks owns both accumulators and hands them back on one barrier: a stage that never fills
+    # must end its MMA and epilogue roles like any other launch, and the next launch on the same tile must be exact.
+    from gpu_util import DEV, run_gemm, tl
+    M, N, K = 256, 256 * 112, 128
+    A, Bd, want = _int_case(M, N, K, 16, 128, seed=77)
+    C = torch.zeros((M, N), dtype=torch.float32, device=DEV)
+    tl.device_status()
+    with tl.option(tl.OPT_WAIT_LIMIT_US, 2000):
+        tl.set_option(tl.OPT_STALL_ONCE, 1)
+        tl.gemm(A.to(DEV), Bd, C, M, N, K, 4096, 16, 128, (256, 256, 64))
+        assert tl.gemm_last_plan().cta == (256, 256, 64) and tl.get_option(tl.OPT_STALL_ONCE) == 0
+        with pytest.raises(tl.TileLensError) as e:
+            tl.device_status()
+        assert e.value.status == 5
+    tl.device_status()
+    assert torch.equal(run_gemm(A, Bd, M, N, K, 16, 128, (256, 256, 64)).cpu(), want)
+
+
 def test_relayout_wait_that_runs_out_is_reported_and_the_next_call_is_clean():
     from gpu_util import DEV, Guarded, dev_bytes, tl
     rows, cols, s, br, bc = 512, 512, 2, 16, 128
