@@ -18,7 +18,9 @@ G, BR, BC = 4096, 16, 128
 
 def _products():
     # (M, N, K, forced cut): split-K inside clusters, whole tiles, and the stream-K cut (which needs scratch)
-    return [(8, 1024, 4096, False), (16, 148 * 256, 256, False), (24, 1280, 2048, True)]
+    # ... then a tile of two token blocks (128 tiles on 128 CTAs) and a product on CTA pairs
+    return [(8, 1024, 4096, False), (16, 148 * 256, 256, False), (24, 1280, 2048, True), (1024, 8192, 256, False),
+            (512, 19200, 128, False)]
 
 
 class _Step:
@@ -114,8 +116,9 @@ def test_a_captured_step_replays_the_bits_of_direct_calls():
         step.issue()
         tl.device_status()
         want[seed] = [t.clone() for t in step.outputs()]
-    kinds = [(p.stream_k, p.cluster_k > 1) for p in step.plans]
+    kinds = [(p.stream_k, p.cluster_k > 1) for p in step.plans[:3]]
     assert kinds == [(0, True), (0, False), (1, False)], kinds     # clusters, whole tiles, the cut
+    assert step.plans[3].cta == (256, 256, 64) and step.plans[4].pair_kernel == 1
     # the dense and grouped products are exact integers
     for i, (M, N, K, _) in enumerate(_products()):
         exact = step.A[i].double() @ step.W_row[i].double()
